@@ -1,0 +1,367 @@
+#!/usr/bin/env python
+"""Benchmark of shared-KV decode attention (KVSharer's generation path) on B200.
+
+One *step* = one decode step of the whole model's attention path: for every layer in
+order, append the new token's K/V (own-cache layers only) and run the layer's attention
+over the slot the strategy points it to.  Inputs are seeded and synthetic; the cache is
+resident in HBM before timing starts.
+
+    python bench.py --gpus 1 --steps 100 --warmup 10          # this library
+    python bench.py --impl reference --steps 3 --warmup 1      # the fp64 CPU oracle
+
+Prints ONE JSON line (rank 0).
+"""
+from __future__ import annotations
+
+import argparse
+import hashlib
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "shared-KV decode attention throughput (attention-path tokens/s; KV-read GB/s in roofline)"
+UNIT = "tokens/s"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+# DRAM traffic of one launch of the dominant kernel from an ncu capture, valid only for the
+# kernel source it was taken with (sha256 of csrc/kvs_kernels.cu); see profiles/.
+NCU_TRAFFIC = {
+    # "workload": {"kernel_sha256": "...", "dram_bytes_per_launch": int}
+}
+
+
+def _kernel_hash() -> str:
+    p = os.path.join(ROOT, "paper_2410_18517_b200", "csrc", "kvs_kernels.cu")
+    return hashlib.sha256(open(p, "rb").read()).hexdigest()
+
+
+def _peak_hbm():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(p) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi polling in a child process while the timed regions run (read-only)."""
+
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index = gpu_index
+        self.proc = None
+        self.path = f"/tmp/kvs_bench_clocks_{os.getpid()}.csv"
+
+    def start(self):
+        try:
+            self.f = open(self.path, "w")
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.gpu_index), f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                 "-lms", "20"], stdout=self.f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self) -> dict:
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.f.close()
+        sm, mx, reasons, power = [], [], set(), []
+        try:
+            for line in open(self.path):
+                parts = [p.strip() for p in line.split(",")]
+                if len(parts) < 9:
+                    continue
+                try:
+                    sm.append(float(parts[1])); mx.append(float(parts[2])); power.append(float(parts[3]))
+                except ValueError:
+                    continue
+                for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"),
+                                     parts[5:9]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+            os.remove(self.path)
+        except Exception:
+            pass
+        if sm:
+            # "under load": the upper half of samples by power draw
+            thr = statistics.median(power)
+            loaded = [s for s, p in zip(sm, power) if p >= thr] or sm
+            out.update(sm_mhz=statistics.median(loaded), sm_max_mhz=max(mx), reasons=sorted(reasons),
+                       samples=len(sm), power_w_max=max(power))
+        return out
+
+
+def cpu_baseline(w, seconds_target: float = 15.0) -> dict:
+    """Time the oracle, as it stands, on a bounded sample of this workload's units."""
+    import numpy as np
+    import torch
+
+    import oracle
+    import synth_inputs as si
+
+    n = w.context + 1
+    distinct = 64
+    g = torch.Generator().manual_seed(0)
+    K = torch.randn(distinct, n, w.D, generator=g).to(w.torch_dtype).double().numpy()
+    V = torch.randn(distinct, n, w.D, generator=g).to(w.torch_dtype).double().numpy()
+    q = torch.randn(distinct, w.D, generator=g).to(w.torch_dtype).double().numpy()
+    oracle.attend_units(q[:8], K[:8], V[:8])            # load the library, warm the threads
+    t0 = time.perf_counter()
+    oracle.attend_units(q, K, V)
+    t1 = time.perf_counter() - t0
+    reps = max(1, min(64, int(seconds_target / max(t1, 1e-3))))
+    t0 = time.perf_counter()
+    for _ in range(reps):
+        oracle.attend_units(q, K, V)
+    dt = time.perf_counter() - t0
+    units = distinct * reps
+    units_per_step = w.L * w.B * w.Hq
+    step_s = dt / units * units_per_step
+    return {"value": w.B / step_s, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": f"{units} (sequence, q-head) units of n={n} rows ({distinct} distinct x {reps}) in {dt:.2f} s, "
+                      f"extrapolated to the {units_per_step} units of one step",
+            "units_per_s": units / dt}
+
+
+def run_reference(args, w):
+    """The oracle as the reference arm: each step is a bounded sample of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+
+    per = []
+    for i in range(args.warmup + args.steps):
+        r = cpu_baseline(w, seconds_target=4.0)
+        if i >= args.warmup:
+            per.append(r)
+    val = statistics.mean(x["value"] for x in per)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": 1e3 * w.B / val, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": workload_config(w, 1),
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+                         "sample": per[-1]["sample"]},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+
+
+def workload_config(w, n_gpus):
+    return {"workload": w.name, "layers": w.L, "q_heads": w.Hq, "kv_heads": w.Hkv, "head_dim": w.D,
+            "batch_per_gpu": w.B, "global_batch": w.B * n_gpus, "context": w.context, "storage": w.dtype,
+            "shared_layers": w.n_shared, "share_map": [int(x) for x in w.share_map()],
+            "parallelism": f"batch-sharded x{n_gpus}, no collective on the data path",
+            "l2": "inputs larger than L2: every layer launch streams its whole slot "
+                  f"({w.kv_read_bytes_per_layer(w.context) / 2**20:.0f} MiB) and "
+                  f"{w.L - w.n_shared} distinct slots are cycled"}
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="kvs", choices=["kvs", "reference"])
+    ap.add_argument("--workload", default="7b_mha")
+    ap.add_argument("--e2e-steps", type=int, default=20)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "kvs":
+        args.warmup = 3
+
+    import synth_inputs as si
+
+    w = si.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, w)
+        return
+
+    import torch
+
+    from paper_2410_18517_b200 import SharedKVCache
+    from paper_2410_18517_b200 import build as kbuild
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+
+        if rank == 0:
+            kbuild.build()
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    else:
+        kbuild.build()
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if dist is not None:
+        dist.barrier()
+
+    K, W, E = args.steps, args.warmup, args.e2e_steps
+    total_steps = W + K + K + (3 + E)          # value pass, per-launch-timed pass, e2e pass
+    sm = w.share_map()
+    cache = SharedKVCache(w.L, w.Hq, w.Hkv, w.D, w.B, w.context + total_steps, w.dtype, share_map=sm,
+                          device=local_rank)
+    # Every rank decodes its own batch of sequences (batch sharding): own seed, no exchange.
+    seed = 1000 + rank
+    for l in range(w.L):
+        if sm[l] != l:
+            continue
+        k, v = si.context_kv(w, l, device=dev, base_seed=seed)
+        cache.append(l, k, v)
+        del k, v
+    n_in = 8                                    # distinct input sets cycled over steps
+    qs = [[si.step_qkv(w, t, l, device=dev, base_seed=seed) for l in range(w.L)] for t in range(n_in)]
+    outs = [torch.empty(w.B, w.Hq, w.D, dtype=torch.float32, device=dev) for _ in range(w.L)]
+    torch.cuda.synchronize(dev)
+
+    def one_step(t, events=None):
+        ins = qs[t % n_in]
+        for l in range(w.L):
+            q, k, v = ins[l]
+            if sm[l] == l:
+                cache.append(l, k, v)
+            else:
+                cache.append(l, None, None, w.B, 1)
+            if events is not None:
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                cache.decode_attention(l, q, outs[l])
+                e1.record()
+                events.append((e0, e1))
+            else:
+                cache.decode_attention(l, q, outs[l])
+
+    def sync_all():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize(dev)
+
+    sampler = ClockSampler(local_rank)
+    for t in range(W):
+        one_step(t)
+    sync_all()
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.1)
+    st0 = cache.stats()
+    n_start = cache.seq_len(0)
+    sync_all()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    for t in range(K):
+        one_step(W + t)
+    ev1.record()
+    sync_all()
+    ms = ev0.elapsed_time(ev1)
+    st1 = cache.stats()
+    if dist is not None:
+        tmax = torch.tensor([ms], device=dev)
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+        ms = float(tmax.item())
+    launches = sum(st1[k] - st0[k] for k in ("append_launches", "attention_launches", "combine_launches"))
+    kv_read = st1["kv_bytes_read"] - st0["kv_bytes_read"]
+    kv_app = st1["kv_bytes_appended"] - st0["kv_bytes_appended"]
+
+    # Same K steps again with a CUDA event pair around every attention call: gives the
+    # duration of the dominant kernel's launches (split-K kernel + its small combine).
+    events = []
+    rb0 = cache.stats()["kv_bytes_read"]
+    for t in range(K):
+        one_step(W + K + t, events)
+    sync_all()
+    att_ms = [a.elapsed_time(b) for a, b in events]
+    att_bytes = cache.stats()["kv_bytes_read"] - rb0
+    att_launch_ms = sum(att_ms) / len(att_ms)
+    bytes_per_launch = att_bytes / len(att_ms)
+
+    # End to end through the host-buffer entry point: pinned host inputs copied in, outputs copied out.
+    host = []
+    for t in range(4):
+        ql = torch.stack([qs[t][l][0] for l in range(w.L)]).cpu().pin_memory()
+        kl = torch.stack([qs[t][l][1] for l in range(w.L)]).cpu().pin_memory()
+        vl = torch.stack([qs[t][l][2] for l in range(w.L)]).cpu().pin_memory()
+        host.append((ql, kl, vl))
+    out_host = torch.empty(w.L, w.B, w.Hq, w.D, dtype=torch.float32).pin_memory()
+    for t in range(3):
+        h2d, d2h = cache.step_host(*host[t % 4], out_host)
+    sync_all()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for t in range(E):
+        h2d, d2h = cache.step_host(*host[t % 4], out_host)
+    e1.record()
+    sync_all()
+    e2e_ms = e0.elapsed_time(e1)
+    if dist is not None:
+        tmax = torch.tensor([e2e_ms], device=dev)
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+        e2e_ms = float(tmax.item())
+    clocks = sampler.stop() if rank == 0 else None
+    status = cache.device_status()
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    peak, peak_kind = _peak_hbm()
+    achieved = bytes_per_launch / (att_launch_ms * 1e-3) / 1e9
+    traffic = None
+    rec = NCU_TRAFFIC.get(w.name)
+    if rec and rec["kernel_sha256"] == _kernel_hash():
+        traffic = rec["dram_bytes_per_launch"]
+    step_ms = ms / K
+    n_mid = n_start + K // 2
+    pool_unshared = cache.pool_bytes // cache.num_slots() * w.L
+    line = {
+        "metric": METRIC, "value": world * w.B / (step_ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K,
+        "warmup": W, "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f32", "data": "synthetic", "config": workload_config(w, world),
+        "kv_read_gbs_whole_step": kv_read / (ms * 1e-3) / 1e9,
+        "kv_read_frac_of_8tbs_nominal": kv_read / (ms * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
+        "kv_bytes_read_per_step": kv_read // K, "kv_bytes_appended_per_step": kv_app // K,
+        "pool_bytes": cache.pool_bytes, "pool_bytes_unshared": pool_unshared,
+        "kv_memory_saved_frac": 1.0 - cache.pool_bytes / pool_unshared,
+        "context_mid_run": n_mid,
+        "roofline": {"bound": "hbm", "kernel": "decode_splitk_scalar (+ decode_combine_kernel, same event pair)",
+                     "achieved": achieved, "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
+                     "frac": achieved / peak, "frac_of_8tbs_nominal": achieved / NOMINAL_HBM_GBS,
+                     "traffic": traffic, "bytes_per_launch": bytes_per_launch, "ms_per_launch": att_launch_ms,
+                     "launches_timed": len(att_ms)},
+        "e2e": {"value": world * w.B / (e2e_ms / E * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h, "steps": E, "ms_per_step": e2e_ms / E},
+        "gpu_launches": launches,
+        "clocks": clocks,
+        "device_status": status,
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        line["cpu_baseline"] = cpu_baseline(w)
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

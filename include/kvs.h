@@ -1,0 +1,210 @@
+/*
+ * kvs.h -- C ABI of the shared-KV decode-attention library for NVIDIA B200 (sm_100a).
+ *
+ * The library implements the inference side of KVSharer (layer-wise KV cache
+ * sharing): a per-model strategy says which layers' KV caches are replaced by
+ * which earlier layers' caches (Section 3, Section 3.2, Fig. 3 of the paper).
+ * During generation every layer still computes its own queries and runs the
+ * unchanged attention, but a layer whose cache is replaced reads the keys and
+ * values of its source layer and computes (appends) none of its own.
+ *
+ * Instead of copying a cache from layer to layer, the library keeps ONE cache
+ * slot per layer that computes its own K/V and gives every layer an index into
+ * those slots.  Results are those of the literal copy; memory is
+ * (layers - shared layers) / layers of the unshared pool.
+ *
+ * Conventions for every call
+ *   - returns a kvs_status; never throws, never aborts; on an error nothing
+ *     has been written and no kernel has been launched;
+ *   - "host" / "device" on a pointer says which memory it must point to;
+ *   - the caller owns every buffer it passes (pool, workspace, q, k, v, out);
+ *     the library owns only the kvs_ctx and small host tables;
+ *   - work is enqueued on the given CUDA stream (a cudaStream_t passed as
+ *     void*, NULL = the legacy default stream) and returns without waiting,
+ *     except where a call says otherwise;
+ *   - all sequences of a batch have the same length (no ragged batches).
+ *
+ * Memory layout of the pool (device, caller-owned, bound with kvs_bind_memory):
+ *   plane(slot, kv) with kv = 0 for K and 1 for V, each plane being
+ *   [max_batch][n_kv_heads][row_stride][head_dim] elements of the storage
+ *   type, row_stride = max_seq rounded up to a multiple of 128 rows;
+ *   plane(slot, kv) starts (2 * slot + kv) * plane_bytes into the pool.
+ *   One token row of one head is head_dim contiguous elements; the rows of one
+ *   (sequence, head) are contiguous, so a tile of consecutive tokens is one
+ *   contiguous run of bytes.
+ */
+#ifndef KVS_H_
+#define KVS_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct kvs_ctx kvs_ctx;
+
+typedef enum {
+    KVS_OK = 0,
+    KVS_ERR_INVALID_ARG = 1,   /* NULL pointer, index or size out of range, unsupported shape */
+    KVS_ERR_BAD_SHARE_MAP = 2, /* a source later than its target, or a negative entry        */
+    KVS_ERR_STATE = 3,         /* call made in the wrong state (see each call)                */
+    KVS_ERR_CAPACITY = 4,      /* an append would exceed max_seq                              */
+    KVS_ERR_OOM = 5,           /* a bound buffer is smaller than kvs_required_bytes said      */
+    KVS_ERR_CUDA = 6,          /* a CUDA runtime or driver call failed                        */
+    KVS_ERR_TIMEOUT = 7        /* a bounded device-side wait ran out (see kvs_last_device_status) */
+} kvs_status;
+
+typedef enum { KVS_BF16 = 0, KVS_F32 = 1 } kvs_dtype;
+
+typedef struct {
+    int32_t n_layers;     /* L >= 1                                                 */
+    int32_t n_q_heads;    /* Hq; must be a multiple of n_kv_heads; Hq/Hkv in {1,2,4,8} */
+    int32_t n_kv_heads;   /* Hkv >= 1                                               */
+    int32_t head_dim;     /* 64 or 128                                              */
+    int32_t max_batch;    /* largest batch any call will pass                       */
+    int32_t max_seq;      /* capacity in tokens of every slot                       */
+    int32_t dtype;        /* kvs_dtype: storage type of Q, K and V                  */
+    float softmax_scale;  /* 0 means 1/sqrt(head_dim)                               */
+    int32_t device;       /* CUDA device ordinal the context lives on               */
+} kvs_config;
+
+typedef struct {
+    uint64_t append_launches;     /* kernels launched by kvs_append                          */
+    uint64_t append_skipped;      /* kvs_append calls on sharing layers (no launch)          */
+    uint64_t attention_launches;  /* split-K kernels launched                                */
+    uint64_t combine_launches;    /* combine kernels launched                                */
+    uint64_t kv_bytes_read;       /* 2*B*Hkv*n*D*elem summed over attention calls            */
+    uint64_t kv_bytes_appended;   /* 2*B*Hkv*n_new*D*elem summed over launched appends       */
+} kvs_stats_t;
+
+/* Tuning knobs for kvs_set_option.  Defaults are chosen by the library. */
+typedef enum {
+    KVS_OPT_MAX_CTAS = 0,   /* upper bound on thread blocks of the split-K kernel; 0 = auto  */
+    KVS_OPT_KERNEL = 1      /* 0 = auto, 1 = scalar-FMA path, 2 = grouped tensor-core path   */
+} kvs_option;
+
+/* ---- life cycle ------------------------------------------------------------ */
+
+/* Create a context.  cfg: host.  *out receives the context.  The strategy
+ * starts as the identity (no layer shares).  No CUDA call is made here.
+ * Errors: INVALID_ARG for NULLs, non-positive sizes, Hq % Hkv != 0, group size
+ * not in {1,2,4,8}, head_dim not in {64,128}, unknown dtype.                    */
+kvs_status kvs_create(const kvs_config* cfg, kvs_ctx** out);
+
+/* Destroy a context.  Frees host tables only; the caller's buffers are untouched.
+ * The caller must have synchronised any stream that still runs work of this ctx. */
+kvs_status kvs_destroy(kvs_ctx* ctx);
+
+/* Install the sharing strategy (Section 3: a list saying which layers' KV caches
+ * are replaced by which other layers').  share_map: host, n_layers entries;
+ * share_map[l] == l means layer l computes its own cache, share_map[l] == s < l
+ * means layer l uses the cache of layer s.  The paper always replaces the layer
+ * nearer the output by the one nearer the input (Section 3.1), so s > l is
+ * rejected with BAD_SHARE_MAP, as is s < 0.  Chains are legal and are followed
+ * to the layer that computes its own cache.  Slots are numbered densely in
+ * layer order over the layers that compute their own cache.
+ * STATE unless every slot is empty (the strategy is fixed before inference).
+ * Changes the required pool size: call before kvs_required_bytes/kvs_bind_memory;
+ * a context that already has memory bound must be re-bound afterwards.          */
+kvs_status kvs_set_share_map(kvs_ctx* ctx, const int32_t* share_map);
+
+/* Bytes the caller must provide: pool = n_slots * 2 planes, workspace = split-K
+ * partial results, a status word and staging for kvs_step_host.  Both host out. */
+kvs_status kvs_required_bytes(const kvs_ctx* ctx, size_t* pool_bytes, size_t* workspace_bytes);
+
+/* Hand the context its device memory.  pool, workspace: device, 256-byte
+ * aligned, at least the sizes kvs_required_bytes reported (else OOM).  The pool
+ * is zero-filled on the default stream and the call waits for that, so that
+ * rows past a slot's length never hold non-finite bit patterns.  Queries device
+ * properties; CUDA errors give KVS_ERR_CUDA.  Resets all slot lengths to 0.    */
+kvs_status kvs_bind_memory(kvs_ctx* ctx, void* pool, size_t pool_bytes,
+                           void* workspace, size_t workspace_bytes);
+
+/* Forget every cached token (all slot lengths become 0).  Host-side only. */
+kvs_status kvs_reset(kvs_ctx* ctx);
+
+/* ---- the hot path ------------------------------------------------------------ */
+
+/* Store the new tokens' keys and values of one layer (Section 3.2; a layer whose
+ * cache is replaced computes no KV -- caption of Table 1).
+ *   layer computes its own cache: k, v are device pointers to
+ *       [batch][n_new][n_kv_heads][head_dim] of the storage type; their rows are
+ *       copied bit for bit to rows len .. len+n_new-1 of the layer's slot and the
+ *       slot length grows by n_new.  One kernel launch on `stream`.
+ *   layer's cache is replaced: returns KVS_OK at once; no launch, no length
+ *       change, k and v are not read and may be NULL.
+ * Errors: STATE before kvs_bind_memory; INVALID_ARG for a bad layer, batch < 1,
+ * batch > max_batch, n_new < 1, NULL k/v on an own-cache layer, or a batch that
+ * differs from the one the slot already holds rows for; CAPACITY if
+ * len + n_new > max_seq.                                                        */
+kvs_status kvs_append(kvs_ctx* ctx, int32_t layer, const void* k, const void* v,
+                      int32_t batch, int32_t n_new, void* stream);
+
+/* Attention of one layer's queries over the cache the layer uses (its own slot,
+ * or its source layer's slot as it stands now -- Section 3.2: the source ran
+ * earlier in the same forward pass, so its newest token is included):
+ *   out[b][hq][:] = sum_j softmax_j(scale * q[b][hq] . K[b][hq/G][j]) V[b][hq/G][j]
+ * over all n cached rows j, no mask, G = n_q_heads / n_kv_heads.
+ *   q:   device, [batch][n_q_heads][head_dim], storage type
+ *   out: device, [batch][n_q_heads][head_dim], float32
+ * Launches the split-K kernel and the combine kernel on `stream`; partial
+ * results go through the bound workspace, so calls on one context must not
+ * overlap on the GPU (use one stream, or order them).
+ * Errors: STATE before kvs_bind_memory or when the slot is empty; INVALID_ARG
+ * for a bad layer, NULLs, batch < 1 or batch > the batch the slot was filled for. */
+kvs_status kvs_decode_attention(kvs_ctx* ctx, int32_t layer, const void* q, float* out,
+                                int32_t batch, void* stream);
+
+/* One whole decode step from HOST buffers: for every layer in order, append the
+ * layer's new token (own-cache layers only) and run its attention.
+ *   q_host:   host, [n_layers][batch][n_q_heads][head_dim], storage type
+ *   k_host, v_host: host, [n_layers][batch][1][n_kv_heads][head_dim], storage type
+ *             (entries of sharing layers are not copied to the device)
+ *   out_host: host, [n_layers][batch][n_q_heads][head_dim], float32
+ * Copies inputs host->device into the workspace staging area, runs the layers,
+ * copies the result device->host, all on `stream`, and waits for the stream.
+ * Pinned host memory makes the copies asynchronous; pageable memory also works.
+ * h2d_bytes / d2h_bytes (host, may be NULL) receive the bytes copied.
+ * Errors: as kvs_append / kvs_decode_attention; nothing is launched on an error
+ * found before the first copy.                                                  */
+kvs_status kvs_step_host(kvs_ctx* ctx, const void* q_host, const void* k_host, const void* v_host,
+                         float* out_host, int32_t batch, void* stream,
+                         uint64_t* h2d_bytes, uint64_t* d2h_bytes);
+
+/* ---- introspection (index and layout checks are exact) ----------------------- */
+
+kvs_status kvs_num_slots(const kvs_ctx* ctx, int32_t* n_slots);
+kvs_status kvs_slot_of_layer(const kvs_ctx* ctx, int32_t layer, int32_t* slot);
+/* Tokens visible to `layer` now (the length of the slot it reads). */
+kvs_status kvs_seq_len(const kvs_ctx* ctx, int32_t layer, int32_t* len);
+/* Rows between consecutive (sequence, head) units of a plane. */
+kvs_status kvs_row_stride(const kvs_ctx* ctx, int32_t* rows);
+/* Byte offset into the pool of plane (slot, kv), kv = 0 for K, 1 for V. */
+kvs_status kvs_plane_offset(const kvs_ctx* ctx, int32_t slot, int32_t kv, size_t* offset);
+kvs_status kvs_stats(const kvs_ctx* ctx, kvs_stats_t* stats);
+/* Reads the device status word (waits for the default stream's prior work on it):
+ * 0 = no device-side problem; KVS_ERR_TIMEOUT = a bounded wait inside a kernel ran
+ * out and the kernel returned early (its output is then undefined).             */
+kvs_status kvs_last_device_status(kvs_ctx* ctx, int32_t* device_status);
+kvs_status kvs_set_option(kvs_ctx* ctx, int32_t option, int32_t value);
+/* How the last kvs_decode_attention call was decomposed: thread blocks launched,
+ * rows per tile, and 1 or 2 for the scalar / tensor-core kernel.                */
+kvs_status kvs_last_launch(const kvs_ctx* ctx, int32_t* ctas, int32_t* tile_rows, int32_t* kernel);
+const char* kvs_status_string(kvs_status s);
+
+/* ---- measurement support ------------------------------------------------------ */
+
+/* Stream `bytes` (a non-zero multiple of 32768) from device memory `src` through the same
+ * bulk-copy / shared-memory ring the attention kernel uses and fold them into
+ * a checksum written to *checksum (device, 8 bytes).  Gives the read bandwidth
+ * this staging scheme reaches when no arithmetic competes with it.  `device`
+ * is the ordinal `src` lives on.  One launch on `stream`.                       */
+kvs_status kvs_read_roof(const void* src, size_t bytes, uint64_t* checksum, int32_t device,
+                         void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* KVS_H_ */

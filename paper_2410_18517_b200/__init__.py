@@ -1,0 +1,113 @@
+"""Decode attention over a layer-shared KV cache (KVSharer's inference path) for B200.
+
+``binding`` exposes the C ABI one to one.  ``SharedKVCache`` is a small holder
+that lets PyTorch own the device memory (pool and workspace tensors) and the
+stream, and forwards every operation to the compiled library.
+"""
+from __future__ import annotations
+
+from . import binding
+from .binding import (  # noqa: F401
+    KVS_BF16, KVS_F32, KVS_OK, KVS_OPT_KERNEL, KVS_OPT_MAX_CTAS, KvsError,
+)
+
+__all__ = ["binding", "SharedKVCache", "KvsError"]
+
+
+class SharedKVCache:
+    """One context + the torch tensors backing it.
+
+    ``share_map[l] == l``: layer l computes its own K/V; ``share_map[l] == s < l``:
+    layer l reads layer s's cache and appends nothing.
+    """
+
+    def __init__(self, n_layers, n_q_heads, n_kv_heads, head_dim, max_batch, max_seq, dtype="bf16",
+                 share_map=None, softmax_scale=0.0, device=0):
+        import torch
+
+        self._torch = torch
+        self.device = torch.device("cuda", device)
+        self.dtype = {"bf16": torch.bfloat16, "f32": torch.float32}[dtype]
+        self.shape = (n_layers, n_q_heads, n_kv_heads, head_dim)
+        self.ctx = binding.kvs_create(n_layers, n_q_heads, n_kv_heads, head_dim, max_batch, max_seq,
+                                      KVS_BF16 if dtype == "bf16" else KVS_F32, softmax_scale, device)
+        try:
+            if share_map is not None:
+                binding.kvs_set_share_map(self.ctx, share_map)
+            self.pool_bytes, self.workspace_bytes = binding.kvs_required_bytes(self.ctx)
+            self.pool = torch.empty(self.pool_bytes, dtype=torch.uint8, device=self.device)
+            self.workspace = torch.empty(self.workspace_bytes, dtype=torch.uint8, device=self.device)
+            binding.kvs_bind_memory(self.ctx, self.pool, self.pool_bytes, self.workspace, self.workspace_bytes)
+        except Exception:
+            binding.kvs_destroy(self.ctx)
+            self.ctx = None
+            raise
+
+    def close(self):
+        if getattr(self, "ctx", None):
+            self._torch.cuda.synchronize(self.device)
+            binding.kvs_destroy(self.ctx)
+            self.ctx = None
+            self.pool = self.workspace = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _stream(self) -> int:
+        return self._torch.cuda.current_stream(self.device).cuda_stream
+
+    def append(self, layer, k=None, v=None, batch=None, n_new=None):
+        """k, v: ``[batch][n_new][n_kv_heads][head_dim]`` contiguous device tensors (None on a sharing layer)."""
+        if k is not None:
+            assert k.is_contiguous() and v.is_contiguous() and k.dtype == self.dtype and v.dtype == self.dtype
+            assert k.shape == v.shape and k.shape[2:] == (self.shape[2], self.shape[3])
+            batch, n_new = k.shape[0], k.shape[1]
+        binding.kvs_append(self.ctx, layer, k, v, batch, n_new, self._stream())
+
+    def decode_attention(self, layer, q, out=None):
+        """q: ``[batch][n_q_heads][head_dim]``; returns float32 ``[batch][n_q_heads][head_dim]``."""
+        torch = self._torch
+        assert q.is_contiguous() and q.dtype == self.dtype and q.shape[1:] == (self.shape[1], self.shape[3])
+        if out is None:
+            out = torch.empty(q.shape, dtype=torch.float32, device=self.device)
+        binding.kvs_decode_attention(self.ctx, layer, q, out, q.shape[0], self._stream())
+        return out
+
+    def step_host(self, q_host, k_host, v_host, out_host):
+        """One decode step over all layers from host tensors (see ``kvs_step_host``)."""
+        return binding.kvs_step_host(self.ctx, q_host, k_host, v_host, out_host, q_host.shape[1], self._stream())
+
+    def plane(self, slot, kv):
+        """View of plane (slot, kv) as ``[max_batch][n_kv_heads][row_stride][head_dim]``."""
+        off = binding.kvs_plane_offset(self.ctx, slot, kv)
+        nxt = binding.kvs_plane_offset(self.ctx, 0, 1)
+        rs = binding.kvs_row_stride(self.ctx)
+        return self.pool[off:off + nxt].view(self.dtype).view(-1, self.shape[2], rs, self.shape[3])
+
+    # plain forwards
+    def num_slots(self):
+        return binding.kvs_num_slots(self.ctx)
+
+    def slot_of_layer(self, layer):
+        return binding.kvs_slot_of_layer(self.ctx, layer)
+
+    def seq_len(self, layer):
+        return binding.kvs_seq_len(self.ctx, layer)
+
+    def reset(self):
+        binding.kvs_reset(self.ctx)
+
+    def stats(self):
+        return binding.kvs_stats(self.ctx)
+
+    def device_status(self):
+        return binding.kvs_last_device_status(self.ctx)
+
+    def set_option(self, option, value):
+        binding.kvs_set_option(self.ctx, option, value)
+
+    def last_launch(self):
+        return binding.kvs_last_launch(self.ctx)

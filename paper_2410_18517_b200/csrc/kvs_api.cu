@@ -1,0 +1,455 @@
+// Host side of the C ABI declared in include/kvs.h: the layer -> slot indirection
+// table, slot lengths, capacity and state checks, byte accounting, and the launches.
+#include "../../include/kvs.h"
+
+#include "kvs_kernels.h"
+
+#include <cmath>
+#include <cstring>
+#include <mutex>
+#include <new>
+#include <vector>
+
+namespace {
+
+constexpr size_t kAlign = 256;
+constexpr int kRowStrideQuantum = 128;
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+}  // namespace
+
+struct kvs_ctx {
+    kvs_config cfg;
+    int G = 1;
+    int elem = 2;
+    int row_bytes = 0;
+    int row_stride = 0;        // rows between units of a plane
+    size_t plane_bytes = 0;
+    float scale = 0.f;
+
+    std::vector<int32_t> share_map, root, slot_of_layer;
+    int n_slots = 0;
+    std::vector<int32_t> slot_len;
+    int cur_batch = 0;         // batch the cached rows were appended for (0 = none yet)
+
+    bool bound = false;
+    char* pool = nullptr;
+    char* ws = nullptr;
+    int sm_count = 148;
+
+    // workspace carve-up (byte offsets)
+    size_t off_status = 0, off_part_o = 0, off_part_ml = 0, off_stage_q = 0, off_stage_k = 0, off_stage_v = 0,
+           off_stage_out = 0, ws_bytes = 0;
+
+    int opt_max_ctas = 0;
+    int opt_kernel = 0;
+    kvs::DecodePlan last_plan{};
+    kvs_stats_t stats{};
+};
+
+namespace {
+
+void resolve_map(kvs_ctx* c) {
+    const int L = c->cfg.n_layers;
+    c->root.assign(L, 0);
+    c->slot_of_layer.assign(L, -1);
+    int n = 0;
+    for (int l = 0; l < L; ++l) {
+        if (c->share_map[l] == l) {
+            c->root[l] = l;
+            c->slot_of_layer[l] = n++;
+        } else {
+            // sources precede targets, so the source is already resolved
+            c->root[l] = c->root[c->share_map[l]];
+            c->slot_of_layer[l] = c->slot_of_layer[c->root[l]];
+        }
+    }
+    c->n_slots = n;
+    c->slot_len.assign(n, 0);
+    c->cur_batch = 0;
+}
+
+void layout_workspace(kvs_ctx* c) {
+    const kvs_config& f = c->cfg;
+    const size_t units = (size_t)f.max_batch * f.n_kv_heads;
+    const size_t pieces = units + kvs::kMaxCtas;
+    size_t off = 0;
+    c->off_status = off;
+    off += kAlign;
+    c->off_part_o = off;
+    off = align_up(off + pieces * c->G * f.head_dim * sizeof(float), kAlign);
+    c->off_part_ml = off;
+    off = align_up(off + pieces * c->G * 2 * sizeof(float), kAlign);
+    const size_t L = f.n_layers;
+    c->off_stage_q = off;
+    off = align_up(off + L * f.max_batch * f.n_q_heads * f.head_dim * c->elem, kAlign);
+    c->off_stage_k = off;
+    off = align_up(off + L * f.max_batch * f.n_kv_heads * f.head_dim * c->elem, kAlign);
+    c->off_stage_v = off;
+    off = align_up(off + L * f.max_batch * f.n_kv_heads * f.head_dim * c->elem, kAlign);
+    c->off_stage_out = off;
+    off = align_up(off + L * f.max_batch * f.n_q_heads * f.head_dim * sizeof(float), kAlign);
+    c->ws_bytes = off;
+}
+
+std::once_flag g_init_flag[64];
+cudaError_t g_init_err[64];
+
+cudaError_t init_device_once(int device) {
+    if (device < 0 || device >= 64) return cudaErrorInvalidDevice;
+    std::call_once(g_init_flag[device], [device]() { g_init_err[device] = kvs::init_kernels(); });
+    return g_init_err[device];
+}
+
+// RAII: make ctx's device current for the duration of a call.
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = true;
+    explicit DeviceGuard(int dev) {
+        if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+        if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+        target = dev;
+    }
+    ~DeviceGuard() {
+        if (ok && prev != target) cudaSetDevice(prev);
+    }
+    int target = -1;
+};
+
+kvs_status check_append(kvs_ctx* c, int layer, const void* k, const void* v, int batch, int n_new, bool* sharing) {
+    if (!c) return KVS_ERR_INVALID_ARG;
+    if (!c->bound) return KVS_ERR_STATE;
+    if (layer < 0 || layer >= c->cfg.n_layers) return KVS_ERR_INVALID_ARG;
+    if (batch < 1 || batch > c->cfg.max_batch || n_new < 1) return KVS_ERR_INVALID_ARG;
+    *sharing = c->share_map[layer] != layer;
+    if (*sharing) return KVS_OK;
+    if (!k || !v) return KVS_ERR_INVALID_ARG;
+    if (c->cur_batch != 0 && batch != c->cur_batch) return KVS_ERR_INVALID_ARG;
+    const int slot = c->slot_of_layer[layer];
+    if ((long long)c->slot_len[slot] + n_new > c->cfg.max_seq) return KVS_ERR_CAPACITY;
+    return KVS_OK;
+}
+
+kvs_status check_attention(kvs_ctx* c, int layer, const void* q, const void* out, int batch) {
+    if (!c) return KVS_ERR_INVALID_ARG;
+    if (!c->bound) return KVS_ERR_STATE;
+    if (layer < 0 || layer >= c->cfg.n_layers || !q || !out) return KVS_ERR_INVALID_ARG;
+    if (batch < 1 || batch > c->cfg.max_batch) return KVS_ERR_INVALID_ARG;
+    const int slot = c->slot_of_layer[layer];
+    if (c->slot_len[slot] == 0) return KVS_ERR_STATE;
+    if (batch > c->cur_batch) return KVS_ERR_INVALID_ARG;
+    return KVS_OK;
+}
+
+kvs_status do_append(kvs_ctx* c, int layer, const void* k, const void* v, int batch, int n_new, cudaStream_t st) {
+    const int slot = c->slot_of_layer[layer];
+    char* kp = c->pool + (size_t)(2 * slot) * c->plane_bytes;
+    char* vp = kp + c->plane_bytes;
+    if (kvs::launch_append(k, v, kp, vp, batch, n_new, c->cfg.n_kv_heads, c->row_bytes, c->row_stride,
+                           c->slot_len[slot], st) != cudaSuccess)
+        return KVS_ERR_CUDA;
+    c->slot_len[slot] += n_new;
+    c->cur_batch = batch;
+    c->stats.append_launches += 1;
+    c->stats.kv_bytes_appended += 2ull * batch * c->cfg.n_kv_heads * n_new * c->row_bytes;
+    return KVS_OK;
+}
+
+kvs_status do_attention(kvs_ctx* c, int layer, const void* q, float* out, int batch, cudaStream_t st) {
+    const int slot = c->slot_of_layer[layer];
+    kvs::DecodeArgs a;
+    a.q = q;
+    a.kplane = c->pool + (size_t)(2 * slot) * c->plane_bytes;
+    a.vplane = c->pool + (size_t)(2 * slot + 1) * c->plane_bytes;
+    a.part_o = reinterpret_cast<float*>(c->ws + c->off_part_o);
+    a.part_ml = reinterpret_cast<float*>(c->ws + c->off_part_ml);
+    a.out = out;
+    a.status = reinterpret_cast<int*>(c->ws + c->off_status);
+    a.n = c->slot_len[slot];
+    a.row_stride = c->row_stride;
+    a.units = batch * c->cfg.n_kv_heads;
+    a.G = c->G;
+    a.D = c->cfg.head_dim;
+    a.dtype = c->cfg.dtype;
+    a.scale_log2 = c->scale * 1.4426950408889634f;
+    kvs::DecodePlan plan;
+    kvs::plan_decode_scalar(a.units, a.n, a.G, a.D, a.dtype, c->sm_count, c->opt_max_ctas, &plan);
+    if (kvs::launch_decode_scalar(a, plan, st) != cudaSuccess) return KVS_ERR_CUDA;
+    if (kvs::launch_combine(a, plan, st) != cudaSuccess) return KVS_ERR_CUDA;
+    c->last_plan = plan;
+    c->stats.attention_launches += 1;
+    c->stats.combine_launches += 1;
+    c->stats.kv_bytes_read += 2ull * a.units * a.n * c->row_bytes;
+    return KVS_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+kvs_status kvs_create(const kvs_config* cfg, kvs_ctx** out) {
+    if (!cfg || !out) return KVS_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (cfg->n_layers < 1 || cfg->n_q_heads < 1 || cfg->n_kv_heads < 1 || cfg->max_batch < 1 || cfg->max_seq < 1)
+        return KVS_ERR_INVALID_ARG;
+    if (cfg->n_q_heads % cfg->n_kv_heads != 0) return KVS_ERR_INVALID_ARG;
+    const int G = cfg->n_q_heads / cfg->n_kv_heads;
+    if (G != 1 && G != 2 && G != 4 && G != 8) return KVS_ERR_INVALID_ARG;
+    if (cfg->head_dim != 64 && cfg->head_dim != 128) return KVS_ERR_INVALID_ARG;
+    if (cfg->dtype != KVS_BF16 && cfg->dtype != KVS_F32) return KVS_ERR_INVALID_ARG;
+    if (cfg->device < 0 || cfg->device >= 64) return KVS_ERR_INVALID_ARG;
+    if (!(cfg->softmax_scale >= 0.f) || std::isinf(cfg->softmax_scale)) return KVS_ERR_INVALID_ARG;
+    if (cfg->max_seq > (1 << 30) - kRowStrideQuantum) return KVS_ERR_INVALID_ARG;
+    kvs_ctx* c = new (std::nothrow) kvs_ctx();
+    if (!c) return KVS_ERR_OOM;
+    c->cfg = *cfg;
+    c->G = G;
+    c->elem = cfg->dtype == KVS_BF16 ? 2 : 4;
+    c->row_bytes = cfg->head_dim * c->elem;
+    c->row_stride = (cfg->max_seq + kRowStrideQuantum - 1) / kRowStrideQuantum * kRowStrideQuantum;
+    c->plane_bytes = (size_t)cfg->max_batch * cfg->n_kv_heads * c->row_stride * c->row_bytes;
+    c->scale = cfg->softmax_scale > 0.f ? cfg->softmax_scale : 1.0f / std::sqrt((float)cfg->head_dim);
+    c->share_map.resize(cfg->n_layers);
+    for (int l = 0; l < cfg->n_layers; ++l) c->share_map[l] = l;
+    resolve_map(c);
+    layout_workspace(c);
+    *out = c;
+    return KVS_OK;
+}
+
+kvs_status kvs_destroy(kvs_ctx* ctx) {
+    if (!ctx) return KVS_ERR_INVALID_ARG;
+    delete ctx;
+    return KVS_OK;
+}
+
+kvs_status kvs_set_share_map(kvs_ctx* ctx, const int32_t* share_map) {
+    if (!ctx || !share_map) return KVS_ERR_INVALID_ARG;
+    for (int s = 0; s < ctx->n_slots; ++s)
+        if (ctx->slot_len[s] != 0) return KVS_ERR_STATE;
+    const int L = ctx->cfg.n_layers;
+    for (int l = 0; l < L; ++l)
+        if (share_map[l] < 0 || share_map[l] > l) return KVS_ERR_BAD_SHARE_MAP;
+    const int old_slots = ctx->n_slots;
+    for (int l = 0; l < L; ++l) ctx->share_map[l] = share_map[l];
+    resolve_map(ctx);
+    // A pool bound for fewer slots than the new strategy needs can no longer be used.
+    if (ctx->bound && ctx->n_slots > old_slots) {
+        ctx->bound = false;
+        ctx->pool = nullptr;
+        ctx->ws = nullptr;
+    }
+    return KVS_OK;
+}
+
+kvs_status kvs_required_bytes(const kvs_ctx* ctx, size_t* pool_bytes, size_t* workspace_bytes) {
+    if (!ctx || !pool_bytes || !workspace_bytes) return KVS_ERR_INVALID_ARG;
+    *pool_bytes = (size_t)ctx->n_slots * 2 * ctx->plane_bytes;
+    *workspace_bytes = ctx->ws_bytes;
+    return KVS_OK;
+}
+
+kvs_status kvs_bind_memory(kvs_ctx* ctx, void* pool, size_t pool_bytes, void* workspace, size_t workspace_bytes) {
+    if (!ctx || !pool || !workspace) return KVS_ERR_INVALID_ARG;
+    if (((uintptr_t)pool % kAlign) != 0 || ((uintptr_t)workspace % kAlign) != 0) return KVS_ERR_INVALID_ARG;
+    const size_t need_pool = (size_t)ctx->n_slots * 2 * ctx->plane_bytes;
+    if (pool_bytes < need_pool || workspace_bytes < ctx->ws_bytes) return KVS_ERR_OOM;
+    DeviceGuard guard(ctx->cfg.device);
+    if (!guard.ok) return KVS_ERR_CUDA;
+    if (init_device_once(ctx->cfg.device) != cudaSuccess) return KVS_ERR_CUDA;
+    int sms = 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, ctx->cfg.device) != cudaSuccess) return KVS_ERR_CUDA;
+    if (cudaMemsetAsync(pool, 0, need_pool, 0) != cudaSuccess) return KVS_ERR_CUDA;
+    if (cudaMemsetAsync(workspace, 0, ctx->ws_bytes, 0) != cudaSuccess) return KVS_ERR_CUDA;
+    if (cudaStreamSynchronize(0) != cudaSuccess) return KVS_ERR_CUDA;
+    ctx->sm_count = sms;
+    ctx->pool = static_cast<char*>(pool);
+    ctx->ws = static_cast<char*>(workspace);
+    ctx->bound = true;
+    for (auto& x : ctx->slot_len) x = 0;
+    ctx->cur_batch = 0;
+    return KVS_OK;
+}
+
+kvs_status kvs_reset(kvs_ctx* ctx) {
+    if (!ctx) return KVS_ERR_INVALID_ARG;
+    for (auto& x : ctx->slot_len) x = 0;
+    ctx->cur_batch = 0;
+    return KVS_OK;
+}
+
+kvs_status kvs_append(kvs_ctx* ctx, int32_t layer, const void* k, const void* v, int32_t batch, int32_t n_new,
+                      void* stream) {
+    bool sharing = false;
+    kvs_status s = check_append(ctx, layer, k, v, batch, n_new, &sharing);
+    if (s != KVS_OK) return s;
+    if (sharing) {
+        ctx->stats.append_skipped += 1;
+        return KVS_OK;
+    }
+    DeviceGuard guard(ctx->cfg.device);
+    if (!guard.ok) return KVS_ERR_CUDA;
+    return do_append(ctx, layer, k, v, batch, n_new, static_cast<cudaStream_t>(stream));
+}
+
+kvs_status kvs_decode_attention(kvs_ctx* ctx, int32_t layer, const void* q, float* out, int32_t batch, void* stream) {
+    kvs_status s = check_attention(ctx, layer, q, out, batch);
+    if (s != KVS_OK) return s;
+    DeviceGuard guard(ctx->cfg.device);
+    if (!guard.ok) return KVS_ERR_CUDA;
+    return do_attention(ctx, layer, q, out, batch, static_cast<cudaStream_t>(stream));
+}
+
+kvs_status kvs_step_host(kvs_ctx* ctx, const void* q_host, const void* k_host, const void* v_host, float* out_host,
+                         int32_t batch, void* stream, uint64_t* h2d_bytes, uint64_t* d2h_bytes) {
+    if (!ctx || !q_host || !k_host || !v_host || !out_host) return KVS_ERR_INVALID_ARG;
+    if (!ctx->bound) return KVS_ERR_STATE;
+    const kvs_config& f = ctx->cfg;
+    if (batch < 1 || batch > f.max_batch) return KVS_ERR_INVALID_ARG;
+    if (ctx->cur_batch != 0 && batch != ctx->cur_batch) return KVS_ERR_INVALID_ARG;
+    // every own-cache slot grows by one token; check all capacities before any work
+    for (int sl = 0; sl < ctx->n_slots; ++sl)
+        if (ctx->slot_len[sl] + 1 > f.max_seq) return KVS_ERR_CAPACITY;
+    DeviceGuard guard(f.device);
+    if (!guard.ok) return KVS_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t q_layer = (size_t)batch * f.n_q_heads * f.head_dim * ctx->elem;
+    const size_t kv_layer = (size_t)batch * f.n_kv_heads * f.head_dim * ctx->elem;
+    const size_t out_layer = (size_t)batch * f.n_q_heads * f.head_dim * sizeof(float);
+    char* dq = ctx->ws + ctx->off_stage_q;
+    char* dk = ctx->ws + ctx->off_stage_k;
+    char* dv = ctx->ws + ctx->off_stage_v;
+    char* dout = ctx->ws + ctx->off_stage_out;
+    uint64_t h2d = 0;
+    if (cudaMemcpyAsync(dq, q_host, q_layer * f.n_layers, cudaMemcpyHostToDevice, st) != cudaSuccess) return KVS_ERR_CUDA;
+    h2d += q_layer * f.n_layers;
+    // K/V of own-cache layers only; consecutive own-cache layers go in one copy
+    for (int l = 0; l < f.n_layers;) {
+        if (ctx->share_map[l] != l) { ++l; continue; }
+        int e = l;
+        while (e + 1 < f.n_layers && ctx->share_map[e + 1] == e + 1) ++e;
+        const size_t off = kv_layer * l, len = kv_layer * (e - l + 1);
+        if (cudaMemcpyAsync(dk + off, (const char*)k_host + off, len, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+            cudaMemcpyAsync(dv + off, (const char*)v_host + off, len, cudaMemcpyHostToDevice, st) != cudaSuccess)
+            return KVS_ERR_CUDA;
+        h2d += 2 * len;
+        l = e + 1;
+    }
+    for (int l = 0; l < f.n_layers; ++l) {
+        if (ctx->share_map[l] == l) {
+            kvs_status s = do_append(ctx, l, dk + kv_layer * l, dv + kv_layer * l, batch, 1, st);
+            if (s != KVS_OK) return s;
+        } else {
+            ctx->stats.append_skipped += 1;
+        }
+        kvs_status s = do_attention(ctx, l, dq + q_layer * l, reinterpret_cast<float*>(dout + out_layer * l), batch, st);
+        if (s != KVS_OK) return s;
+    }
+    if (cudaMemcpyAsync(out_host, dout, out_layer * f.n_layers, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return KVS_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return KVS_ERR_CUDA;
+    if (h2d_bytes) *h2d_bytes = h2d;
+    if (d2h_bytes) *d2h_bytes = out_layer * f.n_layers;
+    return KVS_OK;
+}
+
+kvs_status kvs_num_slots(const kvs_ctx* ctx, int32_t* n_slots) {
+    if (!ctx || !n_slots) return KVS_ERR_INVALID_ARG;
+    *n_slots = ctx->n_slots;
+    return KVS_OK;
+}
+
+kvs_status kvs_slot_of_layer(const kvs_ctx* ctx, int32_t layer, int32_t* slot) {
+    if (!ctx || !slot || layer < 0 || layer >= ctx->cfg.n_layers) return KVS_ERR_INVALID_ARG;
+    *slot = ctx->slot_of_layer[layer];
+    return KVS_OK;
+}
+
+kvs_status kvs_seq_len(const kvs_ctx* ctx, int32_t layer, int32_t* len) {
+    if (!ctx || !len || layer < 0 || layer >= ctx->cfg.n_layers) return KVS_ERR_INVALID_ARG;
+    *len = ctx->slot_len[ctx->slot_of_layer[layer]];
+    return KVS_OK;
+}
+
+kvs_status kvs_row_stride(const kvs_ctx* ctx, int32_t* rows) {
+    if (!ctx || !rows) return KVS_ERR_INVALID_ARG;
+    *rows = ctx->row_stride;
+    return KVS_OK;
+}
+
+kvs_status kvs_plane_offset(const kvs_ctx* ctx, int32_t slot, int32_t kv, size_t* offset) {
+    if (!ctx || !offset || slot < 0 || slot >= ctx->n_slots || (kv != 0 && kv != 1)) return KVS_ERR_INVALID_ARG;
+    *offset = (size_t)(2 * slot + kv) * ctx->plane_bytes;
+    return KVS_OK;
+}
+
+kvs_status kvs_stats(const kvs_ctx* ctx, kvs_stats_t* stats) {
+    if (!ctx || !stats) return KVS_ERR_INVALID_ARG;
+    *stats = ctx->stats;
+    return KVS_OK;
+}
+
+kvs_status kvs_last_device_status(kvs_ctx* ctx, int32_t* device_status) {
+    if (!ctx || !device_status) return KVS_ERR_INVALID_ARG;
+    if (!ctx->bound) return KVS_ERR_STATE;
+    DeviceGuard guard(ctx->cfg.device);
+    if (!guard.ok) return KVS_ERR_CUDA;
+    int v = 0;
+    if (cudaMemcpy(&v, ctx->ws + ctx->off_status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess)
+        return KVS_ERR_CUDA;
+    *device_status = v;
+    return KVS_OK;
+}
+
+kvs_status kvs_set_option(kvs_ctx* ctx, int32_t option, int32_t value) {
+    if (!ctx) return KVS_ERR_INVALID_ARG;
+    switch (option) {
+        case KVS_OPT_MAX_CTAS:
+            if (value < 0 || value > kvs::kMaxCtas) return KVS_ERR_INVALID_ARG;
+            ctx->opt_max_ctas = value;
+            return KVS_OK;
+        case KVS_OPT_KERNEL:
+            if (value < 0 || value > 2) return KVS_ERR_INVALID_ARG;
+            ctx->opt_kernel = value;
+            return KVS_OK;
+        default:
+            return KVS_ERR_INVALID_ARG;
+    }
+}
+
+kvs_status kvs_last_launch(const kvs_ctx* ctx, int32_t* ctas, int32_t* tile_rows, int32_t* kernel) {
+    if (!ctx || !ctas || !tile_rows || !kernel) return KVS_ERR_INVALID_ARG;
+    *ctas = ctx->last_plan.NC;
+    *tile_rows = ctx->last_plan.tile_rows;
+    *kernel = ctx->last_plan.kernel;
+    return KVS_OK;
+}
+
+const char* kvs_status_string(kvs_status s) {
+    switch (s) {
+        case KVS_OK: return "ok";
+        case KVS_ERR_INVALID_ARG: return "invalid argument";
+        case KVS_ERR_BAD_SHARE_MAP: return "bad share map";
+        case KVS_ERR_STATE: return "call made in the wrong state";
+        case KVS_ERR_CAPACITY: return "slot capacity exceeded";
+        case KVS_ERR_OOM: return "bound buffer too small";
+        case KVS_ERR_CUDA: return "CUDA call failed";
+        case KVS_ERR_TIMEOUT: return "device-side wait timed out";
+    }
+    return "unknown status";
+}
+
+kvs_status kvs_read_roof(const void* src, size_t bytes, uint64_t* checksum, int32_t device, void* stream) {
+    if (!src || !checksum || bytes == 0 || bytes % 32768 != 0 || device < 0 || device >= 64) return KVS_ERR_INVALID_ARG;
+    DeviceGuard guard(device);
+    if (!guard.ok) return KVS_ERR_CUDA;
+    if (init_device_once(device) != cudaSuccess) return KVS_ERR_CUDA;
+    int sms = 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess) return KVS_ERR_CUDA;
+    if (kvs::launch_read_roof(src, bytes, reinterpret_cast<unsigned long long*>(checksum), sms,
+                              static_cast<cudaStream_t>(stream)) != cudaSuccess)
+        return KVS_ERR_CUDA;
+    return KVS_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,521 @@
+// sm_100a kernels of the shared-KV decode path:
+//   kv_append_kernel      new-token K/V rows -> slot planes (16-byte vectors)
+//   decode_splitk_scalar  persistent split-K attention, bulk-copy ring, fp32 FMA
+//   decode_combine_kernel merges the pieces of every (sequence, kv-head) unit
+//   read_roof_kernel      the same ring with no arithmetic (bandwidth ceiling)
+#include "kvs_device.cuh"
+#include "kvs_kernels.h"
+
+#include <algorithm>
+
+namespace kvs {
+
+// --------------------------------------------------------------------------------------
+// K1: append.  k/v: [B][n_new][Hkv][row] -> plane [B][Hkv][row_stride][row], rows len0...
+// One thread moves 16 bytes.  blockIdx.y = 0 copies K, 1 copies V.
+// --------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) kv_append_kernel(const uint4* __restrict__ k, const uint4* __restrict__ v,
+                                                        uint4* __restrict__ kplane, uint4* __restrict__ vplane,
+                                                        long long total_vecs, int n_new, int Hkv, int row_vecs,
+                                                        int row_stride, int len0) {
+    const uint4* __restrict__ src = blockIdx.y == 0 ? k : v;
+    uint4* __restrict__ dst = blockIdx.y == 0 ? kplane : vplane;
+    for (long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x; idx < total_vecs;
+         idx += (long long)gridDim.x * blockDim.x) {
+        const int c = (int)(idx % row_vecs);
+        long long r = idx / row_vecs;
+        const int h = (int)(r % Hkv);
+        r /= Hkv;
+        const int t = (int)(r % n_new);
+        const long long b = r / n_new;
+        const long long drow = (b * Hkv + h) * (long long)row_stride + len0 + t;
+        dst[drow * row_vecs + c] = src[idx];
+    }
+}
+
+cudaError_t launch_append(const void* k, const void* v, void* kplane, void* vplane, int B, int n_new, int Hkv,
+                          int row_bytes, int row_stride, int len0, cudaStream_t stream) {
+    const int row_vecs = row_bytes / 16;
+    const long long total = (long long)B * n_new * Hkv * row_vecs;
+    const long long blocks = std::min<long long>((total + 255) / 256, 148 * 16);
+    dim3 grid((unsigned)blocks, 2);
+    kv_append_kernel<<<grid, 256, 0, stream>>>((const uint4*)k, (const uint4*)v, (uint4*)kplane, (uint4*)vplane, total,
+                                               n_new, Hkv, row_vecs, row_stride, len0);
+    return cudaGetLastError();
+}
+
+// --------------------------------------------------------------------------------------
+// Work decomposition shared by the split-K kernel and the combine kernel.
+// Thread block c owns tiles [c*T/NC, (c+1)*T/NC) of the line of T tiles.
+// --------------------------------------------------------------------------------------
+__host__ __device__ __forceinline__ long long first_tile_of_cta(long long c, long long T, int NC) {
+    return (c * T) / NC;
+}
+// The thread block that owns tile gt (inverse of the above).
+__host__ __device__ __forceinline__ int cta_of_tile(long long gt, long long T, int NC) {
+    return (int)(((gt + 1) * NC + T - 1) / T - 1);
+}
+
+// --------------------------------------------------------------------------------------
+// K2a: scalar split-K decode attention.
+//
+// Shapes: T = storage type, D = head size, G = q-heads per kv-head.
+// A token row is RB = D*sizeof(T) bytes and is read by LPR = RB/16 lanes, 16 bytes
+// each, so a warp reads 32/LPR consecutive rows (512 contiguous bytes) per shared-memory
+// load: conflict-free without any swizzle.  A tile is 16 KiB of K and 16 KiB of V rows,
+// fetched by two 1-D bulk copies that complete on the stage's mbarrier.  Warp 8 is the
+// producer (one elected lane issues copies); warps 0..7 consume.
+//
+// Every group of LPR lanes keeps its own online-softmax state (running max, sum and
+// un-normalised output chunk) over the rows it is dealt, so no block-wide
+// synchronisation happens per tile; groups are merged once per piece.
+// --------------------------------------------------------------------------------------
+constexpr int kConsumerWarps = 8;
+constexpr int kConsumerThreads = kConsumerWarps * 32;
+constexpr int kScalarThreads = kConsumerThreads + 32;
+constexpr int kTileBytes = 16384;  // per K tile and per V tile
+
+template <typename T, int D, int G>
+struct ScalarShape {
+    static constexpr int RB = D * (int)sizeof(T);
+    static constexpr int LPR = RB / 16;
+    static constexpr int EPL = 16 / (int)sizeof(T);
+    static constexpr int GPW = 32 / LPR;                  // lane groups per warp
+    static constexpr int NG = kConsumerWarps * GPW;       // lane groups per block
+    static constexpr int TN = kTileBytes / RB;            // rows per tile
+    static constexpr int R = TN / NG;                     // rows per group per tile
+    static constexpr int STAGES = (G <= 2) ? 3 : 6;
+    static constexpr int MIN_BLOCKS = (G <= 2) ? 2 : 1;
+    static constexpr int QBYTES = G * RB;
+    static constexpr int STAGE_BYTES = 2 * kTileBytes + QBYTES;
+    static constexpr int SCRATCH_FLOATS = NG * (D + 2);
+    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + SCRATCH_FLOATS * 4 + 2 * STAGES * 8 + 16;
+    static_assert(R >= 1 && R <= LPR && (R & (R - 1)) == 0, "rows per group must be a power of two <= lanes per row");
+    static_assert(TN % NG == 0, "tile rows must divide evenly among lane groups");
+};
+
+template <int N>
+struct Log2 {
+    static constexpr int value = 1 + Log2<N / 2>::value;
+};
+template <>
+struct Log2<1> {
+    static constexpr int value = 0;
+};
+
+// Sum NV per-lane partial sums over a group of lanes by recursive halving: after the
+// call, the lane whose index within the group has top bits i holds the full sum of
+// value i.  OFF is the current xor distance (starts at lanes-per-group / 2).
+template <int NV, int OFF>
+__device__ __forceinline__ float reduce_transpose(float (&v)[NV], int lig) {
+    if constexpr (NV == 1) {
+        float x = v[0];
+#pragma unroll
+        for (int o = OFF; o >= 1; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+        return x;
+    } else {
+        constexpr int H = NV / 2;
+        const bool upper = (lig & OFF) != 0;
+        float w[H];
+#pragma unroll
+        for (int k = 0; k < H; ++k) {
+            const float send = upper ? v[k] : v[k + H];
+            const float keep = upper ? v[k + H] : v[k];
+            w[k] = keep + __shfl_xor_sync(0xffffffffu, send, OFF);
+        }
+        return reduce_transpose<H, OFF / 2>(w, lig);
+    }
+}
+
+struct ScalarKernelArgs {
+    const char* q;
+    const char* kplane;
+    const char* vplane;
+    float* part_o;
+    float* part_ml;
+    int* status;
+    int n;
+    int row_stride;
+    int tpu;
+    long long T;
+    float scale_log2;
+};
+
+template <typename T, int D, int G>
+__global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G>::MIN_BLOCKS)
+    decode_splitk_scalar(const ScalarKernelArgs a) {
+    using S = ScalarShape<T, D, G>;
+    constexpr int RB = S::RB, LPR = S::LPR, EPL = S::EPL, NG = S::NG, TN = S::TN, R = S::R, STAGES = S::STAGES;
+    constexpr int SH = Log2<LPR>::value - Log2<R>::value;  // lane-in-group >> SH = row index held after the reduction
+
+    extern __shared__ __align__(128) unsigned char smem[];
+    unsigned char* stage_base = smem;
+    float* scratch = reinterpret_cast<float*>(smem + STAGES * S::STAGE_BYTES);
+    uint64_t* full_bar = reinterpret_cast<uint64_t*>(scratch + S::SCRATCH_FLOATS);
+    uint64_t* empty_bar = full_bar + STAGES;
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(empty_bar + STAGES);
+
+    const int tid = threadIdx.x;
+    const int warp = tid >> 5;
+    const int lane = tid & 31;
+    const int NC = gridDim.x;
+    const long long t0 = first_tile_of_cta(blockIdx.x, a.T, NC);
+    const long long t1 = first_tile_of_cta(blockIdx.x + 1, a.T, NC);
+
+    if (tid == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(&full_bar[s], 1);
+            mbar_init(&empty_bar[s], kConsumerWarps);
+        }
+        abort_flag[0] = 0;
+        abort_flag[1] = 0;  // second word: bounds the producer's drain after a give-up
+        fence_mbar_init();
+    }
+    __syncthreads();
+
+    if (warp == kConsumerWarps) {
+        // ------------------------------ producer ------------------------------
+        if (lane == 0) {
+            int it = 0;
+            bool ok = true;
+            for (long long gt = t0; gt < t1 && ok; ++gt, ++it) {
+                const int st = it % STAGES;
+                if (it >= STAGES) ok = mbar_wait_bounded(&empty_bar[st], ((it / STAGES) - 1) & 1, abort_flag, a.status);
+                if (!ok) break;
+                const long long u = gt / a.tpu;
+                const int ti = (int)(gt - u * a.tpu);
+                const int row0 = ti * TN;
+                const int rows = min(TN, a.n - row0);
+                const uint32_t bytes = (uint32_t)rows * RB;
+                const bool with_q = (gt == t0) || (ti == 0);
+                unsigned char* sb = stage_base + st * S::STAGE_BYTES;
+                mbar_arrive_expect_tx(&full_bar[st], 2 * bytes + (with_q ? S::QBYTES : 0));
+                const long long off = (u * a.row_stride + row0) * (long long)RB;
+                bulk_g2s(sb, a.kplane + off, bytes, &full_bar[st]);
+                bulk_g2s(sb + kTileBytes, a.vplane + off, bytes, &full_bar[st]);
+                if (with_q) bulk_g2s(sb + 2 * kTileBytes, a.q + u * (long long)S::QBYTES, S::QBYTES, &full_bar[st]);
+            }
+            if (!ok) {
+                // Gave up: still wait (bounded) for copies already issued, so that none
+                // is in flight into this block's shared memory when it exits.
+                for (int j = max(0, it - STAGES); j < it; ++j)
+                    mbar_wait_bounded(&full_bar[j % STAGES], (j / STAGES) & 1, abort_flag + 1, a.status);
+            }
+        }
+        return;
+    }
+
+    // ---------------------------------- consumers ----------------------------------
+    const int lig = lane & (LPR - 1);                 // lane within its row group
+    const int grp = warp * S::GPW + lane / LPR;       // row group within the block
+    const int my_i = lig >> SH;                       // row (of the R) whose score this lane ends up holding
+
+    int it = 0;
+    long long gt = t0;
+    while (gt < t1) {
+        const long long u = gt / a.tpu;
+        const int ti0 = (int)(gt - u * a.tpu);
+        const int piece_tiles = (int)min((long long)(a.tpu - ti0), t1 - gt);
+
+        float qf[G][EPL];
+        float m[G], lsum[G], acc[G][EPL];
+#pragma unroll
+        for (int g = 0; g < G; ++g) {
+            m[g] = -1.0e30f;
+            lsum[g] = 0.f;
+#pragma unroll
+            for (int e = 0; e < EPL; ++e) acc[g][e] = 0.f;
+        }
+
+        for (int k = 0; k < piece_tiles; ++k, ++it) {
+            const int st = it % STAGES;
+            if (!mbar_wait_bounded(&full_bar[st], (it / STAGES) & 1, abort_flag, a.status)) return;
+            const unsigned char* ks = stage_base + st * S::STAGE_BYTES;
+            const unsigned char* vs = ks + kTileBytes;
+            if (k == 0) {
+                const unsigned char* qs = vs + kTileBytes;
+#pragma unroll
+                for (int g = 0; g < G; ++g) {
+                    const uint4 raw = *reinterpret_cast<const uint4*>(qs + g * RB + lig * 16);
+                    Unpack<T>::run(raw, qf[g]);
+#pragma unroll
+                    for (int e = 0; e < EPL; ++e) qf[g][e] *= a.scale_log2;
+                }
+            }
+            const int valid = min(TN, a.n - (ti0 + k) * TN);
+
+            // scores: partial dot products of this lane's 16-byte chunk
+            float s[G][R];
+#pragma unroll
+            for (int i = 0; i < R; ++i) {
+                const int row = grp + NG * i;
+                const uint4 raw = *reinterpret_cast<const uint4*>(ks + row * RB + lig * 16);
+                float kf[EPL];
+                Unpack<T>::run(raw, kf);
+#pragma unroll
+                for (int g = 0; g < G; ++g) {
+                    float d = 0.f;
+#pragma unroll
+                    for (int e = 0; e < EPL; ++e) d = fmaf(qf[g][e], kf[e], d);
+                    s[g][i] = d;
+                }
+            }
+            // online softmax per q-head, local to the lane group
+            float p[G][R];
+            const bool mine_valid = (grp + NG * my_i) < valid;
+#pragma unroll
+            for (int g = 0; g < G; ++g) {
+                float sv = reduce_transpose<R, LPR / 2>(s[g], lig);
+                sv = mine_valid ? sv : -INFINITY;
+                float tmax = sv;
+#pragma unroll
+                for (int o = LPR / 2; o >= LPR / R; o >>= 1) tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, o));
+                const float m_new = fmaxf(m[g], tmax);
+                const float alpha = fast_exp2(m[g] - m_new);
+                const float pv = fast_exp2(sv - m_new);
+                m[g] = m_new;
+                lsum[g] = lsum[g] * alpha + pv;
+#pragma unroll
+                for (int e = 0; e < EPL; ++e) acc[g][e] *= alpha;
+#pragma unroll
+                for (int i = 0; i < R; ++i) p[g][i] = __shfl_sync(0xffffffffu, pv, i << SH, LPR);
+            }
+            // weighted sum of value rows
+#pragma unroll
+            for (int i = 0; i < R; ++i) {
+                const int row = grp + NG * i;
+                if (row < valid) {
+                    const uint4 raw = *reinterpret_cast<const uint4*>(vs + row * RB + lig * 16);
+                    float vf[EPL];
+                    Unpack<T>::run(raw, vf);
+#pragma unroll
+                    for (int g = 0; g < G; ++g)
+#pragma unroll
+                        for (int e = 0; e < EPL; ++e) acc[g][e] = fmaf(p[g][i], vf[e], acc[g][e]);
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&empty_bar[st]);
+        }
+
+        // ---- end of piece: merge the NG lane groups, one q-head at a time ----
+        const long long pid = u + blockIdx.x;
+#pragma unroll
+        for (int g = 0; g < G; ++g) {
+            // lanes with equal top bits hold duplicates of lsum; add across the R distinct ones
+            float l = lsum[g];
+#pragma unroll
+            for (int o = LPR / 2; o >= LPR / R; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
+            named_bar_sync(1, kConsumerThreads);  // scratch free again
+            float* row = scratch + grp * (D + 2);
+#pragma unroll
+            for (int e = 0; e < EPL; ++e) row[lig * EPL + e] = acc[g][e];
+            if (lig == 0) {
+                row[D] = m[g];
+                row[D + 1] = l;
+            }
+            named_bar_sync(1, kConsumerThreads);
+            for (int d = tid; d < D; d += kConsumerThreads) {
+                float M = -1.0e30f;
+#pragma unroll
+                for (int j = 0; j < NG; ++j) M = fmaxf(M, scratch[j * (D + 2) + D]);
+                float o = 0.f, den = 0.f;
+#pragma unroll
+                for (int j = 0; j < NG; ++j) {
+                    const float w = fast_exp2(scratch[j * (D + 2) + D] - M);
+                    o = fmaf(w, scratch[j * (D + 2) + d], o);
+                    den = fmaf(w, scratch[j * (D + 2) + D + 1], den);
+                }
+                a.part_o[(pid * G + g) * D + d] = o;
+                if (d == 0) {
+                    a.part_ml[(pid * G + g) * 2] = M;
+                    a.part_ml[(pid * G + g) * 2 + 1] = den;
+                }
+            }
+        }
+        gt += piece_tiles;
+    }
+}
+
+// --------------------------------------------------------------------------------------
+// K3: combine.  One block per unit, D threads; out = sum_c w_c o_c / sum_c w_c l_c with
+// w_c = 2^(m_c - M), M = max_c m_c over the pieces c of the unit.
+// --------------------------------------------------------------------------------------
+__global__ void decode_combine_kernel(const float* __restrict__ part_o, const float* __restrict__ part_ml,
+                                      float* __restrict__ out, int G, int D, int tpu, long long T, int NC) {
+    const long long u = blockIdx.x;
+    const int c0 = cta_of_tile(u * tpu, T, NC);
+    const int c1 = cta_of_tile((u + 1) * tpu - 1, T, NC);
+    const int d = threadIdx.x;
+    for (int g = 0; g < G; ++g) {
+        float M = -1.0e30f;
+        for (int c = c0; c <= c1; ++c) M = fmaxf(M, part_ml[((u + c) * G + g) * 2]);
+        float o = 0.f, den = 0.f;
+        for (int c = c0; c <= c1; ++c) {
+            const long long pid = u + c;
+            const float w = fast_exp2(part_ml[(pid * G + g) * 2] - M);
+            o = fmaf(w, part_o[(pid * G + g) * D + d], o);
+            den = fmaf(w, part_ml[(pid * G + g) * 2 + 1], den);
+        }
+        out[(u * G + g) * D + d] = o / den;
+    }
+}
+
+cudaError_t launch_combine(const DecodeArgs& a, const DecodePlan& plan, cudaStream_t stream) {
+    decode_combine_kernel<<<a.units, a.D, 0, stream>>>(a.part_o, a.part_ml, a.out, a.G, a.D, plan.tpu, plan.T, plan.NC);
+    return cudaGetLastError();
+}
+
+// --------------------------------------------------------------------------------------
+// Launch plumbing for the scalar kernel.
+// --------------------------------------------------------------------------------------
+template <typename T, int D, int G>
+static cudaError_t set_attr_one() {
+    return cudaFuncSetAttribute(decode_splitk_scalar<T, D, G>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                ScalarShape<T, D, G>::SMEM_BYTES);
+}
+
+template <typename T, int D>
+static cudaError_t set_attr_groups() {
+    cudaError_t e;
+    if ((e = set_attr_one<T, D, 1>()) != cudaSuccess) return e;
+    if ((e = set_attr_one<T, D, 2>()) != cudaSuccess) return e;
+    if ((e = set_attr_one<T, D, 4>()) != cudaSuccess) return e;
+    return set_attr_one<T, D, 8>();
+}
+
+template <typename T, int D, int G>
+static cudaError_t launch_scalar_one(const ScalarKernelArgs& ka, int NC, cudaStream_t stream) {
+    decode_splitk_scalar<T, D, G><<<NC, kScalarThreads, ScalarShape<T, D, G>::SMEM_BYTES, stream>>>(ka);
+    return cudaGetLastError();
+}
+
+template <typename T, int D>
+static cudaError_t launch_scalar_groups(int G, const ScalarKernelArgs& ka, int NC, cudaStream_t stream) {
+    switch (G) {
+        case 1: return launch_scalar_one<T, D, 1>(ka, NC, stream);
+        case 2: return launch_scalar_one<T, D, 2>(ka, NC, stream);
+        case 4: return launch_scalar_one<T, D, 4>(ka, NC, stream);
+        case 8: return launch_scalar_one<T, D, 8>(ka, NC, stream);
+        default: return cudaErrorInvalidValue;
+    }
+}
+
+void plan_decode_scalar(int units, int n, int G, int D, int dtype, int sm_count, int max_ctas, DecodePlan* plan) {
+    const int rb = D * (dtype == 0 ? 2 : 4);
+    plan->tile_rows = kTileBytes / rb;
+    plan->tpu = (n + plan->tile_rows - 1) / plan->tile_rows;
+    plan->T = (long long)units * plan->tpu;
+    const int per_sm = (G <= 2) ? 2 : 1;
+    int cap = sm_count * per_sm;
+    if (max_ctas > 0) cap = std::min(cap, max_ctas);
+    cap = std::min(cap, kMaxCtas);
+    plan->NC = (int)std::min<long long>(plan->T, cap);
+    plan->kernel = 1;
+}
+
+cudaError_t launch_decode_scalar(const DecodeArgs& a, const DecodePlan& plan, cudaStream_t stream) {
+    ScalarKernelArgs ka;
+    ka.q = (const char*)a.q;
+    ka.kplane = (const char*)a.kplane;
+    ka.vplane = (const char*)a.vplane;
+    ka.part_o = a.part_o;
+    ka.part_ml = a.part_ml;
+    ka.status = a.status;
+    ka.n = a.n;
+    ka.row_stride = a.row_stride;
+    ka.tpu = plan.tpu;
+    ka.T = plan.T;
+    ka.scale_log2 = a.scale_log2;
+    if (a.dtype == 0) {
+        if (a.D == 128) return launch_scalar_groups<__nv_bfloat16, 128>(a.G, ka, plan.NC, stream);
+        if (a.D == 64) return launch_scalar_groups<__nv_bfloat16, 64>(a.G, ka, plan.NC, stream);
+    } else {
+        if (a.D == 128) return launch_scalar_groups<float, 128>(a.G, ka, plan.NC, stream);
+        if (a.D == 64) return launch_scalar_groups<float, 64>(a.G, ka, plan.NC, stream);
+    }
+    return cudaErrorInvalidValue;
+}
+
+// --------------------------------------------------------------------------------------
+// K4: read roof.  Same producer, same ring, consumers only fold the bytes together.
+// --------------------------------------------------------------------------------------
+constexpr int kRoofStages = 3;
+constexpr int kRoofStageBytes = 2 * kTileBytes;
+constexpr int kRoofSmem = kRoofStages * kRoofStageBytes + 2 * kRoofStages * 8 + 16;
+
+__global__ void __launch_bounds__(kScalarThreads, 2)
+    read_roof_kernel(const char* __restrict__ src, long long n_tiles, unsigned long long* checksum) {
+    extern __shared__ __align__(128) unsigned char smem[];
+    uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + kRoofStages * kRoofStageBytes);
+    uint64_t* empty_bar = full_bar + kRoofStages;
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(empty_bar + kRoofStages);
+    __shared__ int local_status;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const long long t0 = first_tile_of_cta(blockIdx.x, n_tiles, gridDim.x);
+    const long long t1 = first_tile_of_cta(blockIdx.x + 1, n_tiles, gridDim.x);
+    if (tid == 0) {
+        for (int s = 0; s < kRoofStages; ++s) {
+            mbar_init(&full_bar[s], 1);
+            mbar_init(&empty_bar[s], kConsumerWarps);
+        }
+        *abort_flag = 0;
+        local_status = 0;
+        fence_mbar_init();
+    }
+    __syncthreads();
+    if (warp == kConsumerWarps) {
+        if (lane == 0) {
+            int it = 0;
+            for (long long gt = t0; gt < t1; ++gt, ++it) {
+                const int st = it % kRoofStages;
+                if (it >= kRoofStages &&
+                    !mbar_wait_bounded(&empty_bar[st], ((it / kRoofStages) - 1) & 1, abort_flag, &local_status))
+                    break;
+                unsigned char* sb = smem + st * kRoofStageBytes;
+                mbar_arrive_expect_tx(&full_bar[st], kRoofStageBytes);
+                bulk_g2s(sb, src + gt * kRoofStageBytes, kTileBytes, &full_bar[st]);
+                bulk_g2s(sb + kTileBytes, src + gt * kRoofStageBytes + kTileBytes, kTileBytes, &full_bar[st]);
+            }
+        }
+        return;
+    }
+    unsigned int x = 0;
+    int it = 0;
+    for (long long gt = t0; gt < t1; ++gt, ++it) {
+        const int st = it % kRoofStages;
+        if (!mbar_wait_bounded(&full_bar[st], (it / kRoofStages) & 1, abort_flag, &local_status)) return;
+        const uint4* sb = reinterpret_cast<const uint4*>(smem + st * kRoofStageBytes);
+#pragma unroll
+        for (int j = 0; j < kRoofStageBytes / 16 / kConsumerThreads; ++j) {
+            const uint4 r = sb[j * kConsumerThreads + tid];
+            x ^= r.x ^ r.y ^ r.z ^ r.w;
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&empty_bar[st]);
+    }
+#pragma unroll
+    for (int o = 16; o >= 1; o >>= 1) x ^= __shfl_xor_sync(0xffffffffu, x, o);
+    if (lane == 0) atomicXor(checksum, (unsigned long long)x);
+}
+
+cudaError_t launch_read_roof(const void* src, size_t bytes, unsigned long long* checksum, int sm_count,
+                             cudaStream_t stream) {
+    const long long n_tiles = (long long)(bytes / kRoofStageBytes);
+    const int NC = (int)std::min<long long>(n_tiles, 2LL * sm_count);
+    cudaError_t e = cudaMemsetAsync(checksum, 0, 8, stream);
+    if (e != cudaSuccess) return e;
+    read_roof_kernel<<<NC, kScalarThreads, kRoofSmem, stream>>>((const char*)src, n_tiles, checksum);
+    return cudaGetLastError();
+}
+
+cudaError_t init_kernels() {
+    cudaError_t e;
+    if ((e = set_attr_groups<__nv_bfloat16, 128>()) != cudaSuccess) return e;
+    if ((e = set_attr_groups<__nv_bfloat16, 64>()) != cudaSuccess) return e;
+    if ((e = set_attr_groups<float, 128>()) != cudaSuccess) return e;
+    if ((e = set_attr_groups<float, 64>()) != cudaSuccess) return e;
+    return cudaFuncSetAttribute(read_roof_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kRoofSmem);
+}
+
+}  // namespace kvs

@@ -1,0 +1,57 @@
+// Internal launcher interface between the host API and the sm_100a kernels.
+#pragma once
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+namespace kvs {
+
+// How one decode-attention call is cut into work.  A *unit* is one
+// (sequence, kv-head) pair, i.e. n contiguous K rows and n contiguous V rows.
+// Units are cut into tiles of tile_rows rows; all tiles of all units form one
+// line of T tiles which is divided evenly among NC persistent thread blocks.
+// Each (thread block, unit) overlap is a *piece* and yields one partial result,
+// stored at index unit + block.
+struct DecodePlan {
+    int tile_rows;   // rows per tile
+    int tpu;         // tiles per unit = ceil(n / tile_rows)
+    long long T;     // total tiles = units * tpu
+    int NC;          // thread blocks launched
+    int kernel;      // 1 = scalar, 2 = tensor-core
+};
+
+struct DecodeArgs {
+    const void* q;        // [B][Hq][D] storage type
+    const void* kplane;   // plane of the slot read: [B][Hkv][row_stride][D]
+    const void* vplane;
+    float* part_o;        // [units + NC][G][D]
+    float* part_ml;       // [units + NC][G][2]  (max in log2 domain, sum)
+    float* out;           // [B][Hq][D]
+    int* status;          // device status word
+    int n;                // rows cached per unit
+    int row_stride;       // rows between units of a plane
+    int units;            // B * Hkv
+    int G;                // q-heads per kv-head
+    int D;
+    int dtype;            // 0 bf16, 1 f32
+    float scale_log2;     // softmax scale * log2(e)
+};
+
+// Largest number of thread blocks any plan may use (sizes the partial buffers).
+constexpr int kMaxCtas = 1024;
+
+// Fill `plan` for the scalar kernel on a device with `sm_count` SMs.
+// max_ctas <= 0 means automatic.  Host-only arithmetic (no CUDA call).
+void plan_decode_scalar(int units, int n, int G, int D, int dtype, int sm_count, int max_ctas, DecodePlan* plan);
+
+// One-time per-process kernel attribute set-up for the current device.
+cudaError_t init_kernels();
+
+cudaError_t launch_append(const void* k, const void* v, void* kplane, void* vplane, int B, int n_new, int Hkv,
+                          int row_bytes, int row_stride, int len0, cudaStream_t stream);
+cudaError_t launch_decode_scalar(const DecodeArgs& a, const DecodePlan& plan, cudaStream_t stream);
+cudaError_t launch_combine(const DecodeArgs& a, const DecodePlan& plan, cudaStream_t stream);
+cudaError_t launch_read_roof(const void* src, size_t bytes, unsigned long long* checksum, int sm_count,
+                             cudaStream_t stream);
+
+}  // namespace kvs

@@ -1,0 +1,251 @@
+"""Parity of the CUDA path (through the C ABI) with the fp64 oracle on the same seeded inputs.
+
+Bit-exact for indices, lengths and cached K/V; max-abs 2e-3 and relative-L2 1e-3 for
+attention outputs (bf16 or fp32 inputs, fp32 accumulation).
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import synth_inputs as si
+from paper_2410_18517_b200 import KVS_OPT_MAX_CTAS, KvsError, SharedKVCache
+from paper_2410_18517_b200 import binding as kb
+from paper_2410_18517_b200 import build as kbuild
+
+from helpers import SampledRun, assert_close, make_cache, run_small
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    kbuild.build()
+
+
+@pytest.fixture(autouse=True)
+def _release_device_memory():
+    yield
+    import gc
+
+    gc.collect()
+    torch.cuda.empty_cache()
+
+
+# ------------------------------------------------------------------ the tiny configuration, whole
+def test_tiny_config_every_output_and_every_cached_bit():
+    """L=4, 4 heads, D=64, B=2, 128 context rows, fp32, strategy {0,1,2,1}: one decode step and
+    eight more, compared in full."""
+    w = si.WORKLOADS["tiny"]
+    cache, orc, worst = run_small(w, steps=9)
+    assert cache.num_slots() == 3
+    st = cache.stats()
+    assert st["append_launches"] == 3 + 9 * 3 and st["append_skipped"] == 1 + 9
+    assert st["attention_launches"] == 9 * 4 and st["combine_launches"] == 9 * 4
+    assert [cache.seq_len(l) for l in range(4)] == [137] * 4
+    assert worst[0] < 1e-4       # fp32 storage: far inside the bf16 tolerance
+
+
+# ------------------------------------------------------------------ shapes, tails, strategies
+SHAPES = [
+    # dtype, D, Hq, Hkv
+    ("bf16", 128, 4, 4), ("bf16", 128, 8, 2), ("bf16", 128, 4, 2), ("bf16", 128, 8, 1),
+    ("bf16", 64, 4, 4), ("bf16", 64, 8, 2),
+    ("f32", 64, 2, 2), ("f32", 128, 2, 2), ("f32", 128, 4, 1),
+]
+
+
+@pytest.mark.parametrize("dtype,D,Hq,Hkv", SHAPES)
+@pytest.mark.parametrize("context", [0, 63, 64, 65, 200, 1031])
+def test_shapes_and_ragged_tails(dtype, D, Hq, Hkv, context):
+    """Context lengths around the 32/64/128-row tile edges, 3 decode steps, chain strategy."""
+    w = si.Workload(f"s_{dtype}_{D}_{Hq}_{Hkv}_{context}", L=4, Hq=Hq, Hkv=Hkv, D=D, B=3, context=context,
+                    dtype=dtype, n_shared=0, map_seed=0, steps=3, fixed_map=(0, 0, 1, 2))
+    cache, orc, _ = run_small(w, steps=3)
+    assert cache.num_slots() == 1
+
+
+@pytest.mark.parametrize("max_ctas", [1, 2, 5, 37, 0])
+def test_any_split_of_the_tile_line_gives_the_same_answer(max_ctas):
+    """The tile line of all units is cut at arbitrary places; results must not depend on it."""
+    w = si.Workload(f"split_{max_ctas}", L=2, Hq=4, Hkv=4, D=128, B=2, context=1500, dtype="bf16",
+                    n_shared=1, map_seed=0, steps=2, fixed_map=(0, 0))
+    cache, _, _ = run_small(w, steps=2, options=[(KVS_OPT_MAX_CTAS, max_ctas)])
+    if max_ctas:
+        assert cache.last_launch()["ctas"] == max_ctas
+
+
+def test_many_small_units_per_block():
+    """More units than thread blocks and only a few tiles each: blocks span several whole units."""
+    w = si.Workload("many_units", L=1, Hq=16, Hkv=16, D=128, B=40, context=130, dtype="bf16",
+                    n_shared=0, map_seed=0, steps=1)
+    run_small(w, steps=1)
+
+
+def test_explicit_softmax_scale():
+    w = si.Workload("scaled", L=1, Hq=2, Hkv=2, D=64, B=1, context=300, dtype="bf16", n_shared=0, map_seed=0, steps=1)
+    run_small(w, steps=1, scale=0.2)
+
+
+def test_smaller_batch_than_max_batch():
+    w = si.Workload("subbatch", L=2, Hq=4, Hkv=2, D=128, B=2, context=100, dtype="bf16", n_shared=1, map_seed=0,
+                    steps=1, fixed_map=(0, 0))
+    cache = SharedKVCache(w.L, w.Hq, w.Hkv, w.D, 5, 256, "bf16", share_map=[0, 0])
+    orc = oracle.Oracle(w.L, w.Hq, w.Hkv, w.D, w.B, [0, 0])
+    k, v = si.context_kv(w, 0)
+    cache.append(0, k.cuda(), v.cuda())
+    orc.layer_forward(0, None, k.double().numpy(), v.double().numpy())
+    for l in range(2):
+        q, _, _ = si.step_qkv(w, 0, l)
+        ref = orc.layer_forward(l, q.double().numpy())
+        assert_close(cache.decode_attention(l, q.cuda()).cpu().numpy(), ref)
+    with pytest.raises(KvsError) as e:      # more sequences than were cached
+        cache.decode_attention(0, torch.zeros(3, 4, 128, dtype=torch.bfloat16, device="cuda"))
+    assert e.value.status == kb.KVS_ERR_INVALID_ARG
+
+
+# ------------------------------------------------------------------ sharing semantics on the device
+def test_append_on_sharing_layer_changes_no_byte_and_no_length():
+    w = si.WORKLOADS["tiny"]
+    cache = make_cache(w, 8)
+    for l in range(w.L):
+        k, v = si.context_kv(w, l)
+        cache.append(l, k.cuda(), v.cuda())
+    torch.cuda.synchronize()
+    before = cache.pool.clone()
+    lens = [cache.seq_len(l) for l in range(w.L)]
+    launches = cache.stats()["append_launches"]
+    _, k, v = si.step_qkv(w, 0, 3)
+    cache.append(3, k.cuda(), v.cuda())        # layer 3 shares layer 1's cache
+    cache.append(3, None, None, w.B, 5)        # pointers are not needed at all
+    torch.cuda.synchronize()
+    assert torch.equal(before, cache.pool)
+    assert [cache.seq_len(l) for l in range(w.L)] == lens
+    assert cache.stats()["append_launches"] == launches and cache.stats()["append_skipped"] == 3
+
+
+def test_sharing_layer_sees_the_sources_newest_token():
+    w = si.Workload("newest", L=2, Hq=2, Hkv=2, D=64, B=1, context=4, dtype="f32", n_shared=1, map_seed=0, steps=1,
+                    fixed_map=(0, 0))
+    cache = make_cache(w, 2)
+    k, v = si.context_kv(w, 0)
+    cache.append(0, k.cuda(), v.cuda())
+    q = torch.zeros(1, 2, 64, device="cuda")
+    knew = torch.zeros(1, 1, 2, 64, device="cuda")
+    vnew = torch.full((1, 1, 2, 64), 100.0, device="cuda")
+    cache.append(0, knew, vnew)
+    out = cache.decode_attention(1, q)        # q = 0: uniform weights over 5 rows, the new one included
+    ref = (v[0].double().sum(0) + 100.0) / 5.0
+    np.testing.assert_allclose(out[0].cpu().numpy(), ref.numpy(), atol=1e-4)
+    assert cache.seq_len(1) == 5
+
+
+def test_error_paths_launch_nothing():
+    w = si.WORKLOADS["tiny"]
+    cache = make_cache(w, 0)               # capacity exactly 128
+    q = torch.zeros(2, 4, 64, device="cuda")
+    with pytest.raises(KvsError) as e:     # empty slot
+        cache.decode_attention(0, q)
+    assert e.value.status == kb.KVS_ERR_STATE
+    k, v = si.context_kv(w, 0)
+    cache.append(0, k.cuda(), v.cuda())
+    _, k1, v1 = si.step_qkv(w, 0, 0)
+    torch.cuda.synchronize()
+    before = cache.pool.clone()
+    with pytest.raises(KvsError) as e:     # 129th row
+        cache.append(0, k1.cuda(), v1.cuda())
+    assert e.value.status == kb.KVS_ERR_CAPACITY
+    with pytest.raises(KvsError) as e:     # a different batch than the cached one
+        cache.append(1, k1[:1].contiguous().cuda(), v1[:1].contiguous().cuda())
+    assert e.value.status == kb.KVS_ERR_INVALID_ARG
+    with pytest.raises(KvsError) as e:     # strategy is fixed once rows are cached
+        kb.kvs_set_share_map(cache.ctx, [0, 0, 0, 0])
+    assert e.value.status == kb.KVS_ERR_STATE
+    with pytest.raises(KvsError):
+        kb.kvs_append(cache.ctx, 1, None, None, 2, 1)
+    torch.cuda.synchronize()
+    assert torch.equal(before, cache.pool) and cache.seq_len(0) == 128
+    cache.reset()
+    assert cache.seq_len(0) == 0
+    kb.kvs_set_share_map(cache.ctx, [0, 0, 0, 0])
+    assert cache.num_slots() == 1
+
+
+def test_repeat_runs_are_bit_identical():
+    w = si.Workload("det", L=1, Hq=8, Hkv=2, D=128, B=4, context=3000, dtype="bf16", n_shared=0, map_seed=0, steps=1)
+    cache = make_cache(w, 1)
+    k, v = si.context_kv(w, 0, device="cuda")
+    cache.append(0, k, v)
+    q = si.step_qkv(w, 0, 0, device="cuda")[0]
+    a = cache.decode_attention(0, q).clone()
+    for _ in range(3):
+        assert torch.equal(a, cache.decode_attention(0, q))
+
+
+def test_step_host_equals_per_layer_calls():
+    w = si.WORKLOADS["tiny"]
+    a, b = make_cache(w, 4), make_cache(w, 4)
+    for l in range(w.L):
+        k, v = si.context_kv(w, l)
+        a.append(l, k.cuda(), v.cuda())
+        b.append(l, k.cuda(), v.cuda())
+    for t in range(3):
+        qs, ks, vs = zip(*[si.step_qkv(w, t, l) for l in range(w.L)])
+        qh, kh, vh = torch.stack(qs).pin_memory(), torch.stack(ks).pin_memory(), torch.stack(vs).pin_memory()
+        oh = torch.empty(w.L, w.B, w.Hq, w.D, dtype=torch.float32).pin_memory()
+        h2d, d2h = a.step_host(qh, kh, vh, oh)
+        assert d2h == oh.numel() * 4
+        assert h2d == qh.numel() * 4 + 2 * 3 * kh[0].numel() * 4      # K/V of the 3 own-cache layers only
+        for l in range(w.L):
+            b.append(l, ks[l].cuda(), vs[l].cuda())
+            assert torch.equal(b.decode_attention(l, qs[l].cuda()).cpu(), oh[l])
+    torch.cuda.synchronize()
+    assert torch.equal(a.pool, b.pool)
+
+
+def test_read_roof_checksum():
+    x = torch.randint(0, 2**31 - 1, (3 * 32768 // 4 * 7,), dtype=torch.int32, device="cuda")
+    chk = torch.zeros(1, dtype=torch.int64, device="cuda")
+    kb.kvs_read_roof(x, x.numel() * 4, chk, 0, torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    ref = np.bitwise_xor.reduce(x.cpu().numpy().view(np.uint32))
+    assert int(chk.item()) == int(ref)
+
+
+# ------------------------------------------------------------------ full-size configurations, sampled units
+def test_7b_mha_full_size_sampled_units():
+    """32 layers, 32 heads, D=128, B=8, 4096 context, bf16, 8 of 32 layers sharing: the
+    benchmark's launch configuration; 64 sampled (layer, b, head) units incl. every sharing layer."""
+    run = SampledRun(si.WORKLOADS["7b_mha"], steps=2, n_samples=64)
+    assert run.cache.num_slots() == 24
+    run.load_context()
+    run.step(0, check=True)
+    run.step(1, check=True)
+    run.check_cached_rows()
+    assert run.cache.device_status() == 0
+    st = run.cache.stats()
+    assert st["append_launches"] == 24 * 3 and st["append_skipped"] == 8 * 3
+    assert st["kv_bytes_read"] == sum(2 * 8 * 32 * n * 256 for n in (4097, 4098)) * 32
+
+
+def test_gqa_long_full_size_sampled_units():
+    """32 q-heads over 8 kv-heads, B=4, 32768 context, 10 of 32 layers sharing."""
+    run = SampledRun(si.WORKLOADS["gqa_long"], steps=1, n_samples=48)
+    assert run.cache.num_slots() == 22
+    run.load_context()
+    run.step(0, check=True)
+    run.check_cached_rows()
+    assert run.cache.device_status() == 0
+
+
+def test_13b_mha_64_steps_sampled_units():
+    """40 layers, 40 heads, B=16, 8192 context, 12 of 40 sharing, 64 consecutive steps with appends;
+    sampled units checked at steps 1, 32 and 64, appended rows bit-exact."""
+    run = SampledRun(si.WORKLOADS["13b_mha"], steps=64, n_samples=52)
+    assert run.cache.num_slots() == 28
+    run.load_context()
+    for t in range(64):
+        run.step(t, check=(t in (0, 31, 63)))
+    run.check_cached_rows()
+    assert [run.cache.seq_len(l) for l in range(40)] == [8192 + 64] * 40
+    assert run.cache.device_status() == 0
