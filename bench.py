@@ -127,7 +127,7 @@ def cpu_baseline(w, seconds_target: float = 15.0) -> dict:
     t0 = time.perf_counter()
     oracle.attend_units(q, K, V)
     t1 = time.perf_counter() - t0
-    reps = max(1, min(64, int(seconds_target / max(t1, 1e-3))))
+    reps = max(1, min(4096, int(seconds_target / max(t1, 1e-3))))
     t0 = time.perf_counter()
     for _ in range(reps):
         oracle.attend_units(q, K, V)

@@ -66,6 +66,11 @@ WORKLOADS = {
                      n_shared=1, map_seed=0, steps=9, fixed_map=(0, 1, 2, 1)),
     "7b_mha": Workload("7b_mha", L=32, Hq=32, Hkv=32, D=128, B=8, context=4096, dtype="bf16",
                        n_shared=8, map_seed=2, steps=20),
+    # the 7B shape cut to 4 layers (2 GiB pool): small enough for profiler captures
+    "7b_mha_l4": Workload("7b_mha_l4", L=4, Hq=32, Hkv=32, D=128, B=8, context=4096, dtype="bf16",
+                          n_shared=1, map_seed=0, steps=20, fixed_map=(0, 1, 2, 1)),
+    "gqa_long_l4": Workload("gqa_long_l4", L=4, Hq=32, Hkv=8, D=128, B=4, context=32768, dtype="bf16",
+                            n_shared=1, map_seed=0, steps=20, fixed_map=(0, 1, 2, 1)),
     "13b_mha": Workload("13b_mha", L=40, Hq=40, Hkv=40, D=128, B=16, context=8192, dtype="bf16",
                         n_shared=12, map_seed=3, steps=64),
     "gqa_long": Workload("gqa_long", L=32, Hq=32, Hkv=8, D=128, B=4, context=32768, dtype="bf16",
