@@ -41,6 +41,9 @@ struct kvs_ctx {
     size_t off_status = 0, off_part_o = 0, off_part_ml = 0, off_stage_q = 0, off_stage_k = 0, off_stage_v = 0,
            off_stage_out = 0, ws_bytes = 0;
 
+    alignas(64) unsigned char tensor_map[128];  // TMA view of the pool (bf16 storage only)
+    bool have_tensor_map = false;
+
     int opt_max_ctas = 0;
     int opt_kernel = 0;
     kvs::DecodePlan last_plan{};
@@ -97,7 +100,10 @@ cudaError_t g_init_err[64];
 
 cudaError_t init_device_once(int device) {
     if (device < 0 || device >= 64) return cudaErrorInvalidDevice;
-    std::call_once(g_init_flag[device], [device]() { g_init_err[device] = kvs::init_kernels(); });
+    std::call_once(g_init_flag[device], [device]() {
+        g_init_err[device] = kvs::init_kernels();
+        if (g_init_err[device] == cudaSuccess) g_init_err[device] = kvs::init_mma_kernels();
+    });
     return g_init_err[device];
 }
 
@@ -173,8 +179,18 @@ kvs_status do_attention(kvs_ctx* c, int layer, const void* q, float* out, int ba
     a.dtype = c->cfg.dtype;
     a.scale_log2 = c->scale * 1.4426950408889634f;
     kvs::DecodePlan plan;
-    kvs::plan_decode_scalar(a.units, a.n, a.G, a.D, a.dtype, c->sm_count, c->opt_max_ctas, &plan);
-    if (kvs::launch_decode_scalar(a, plan, st) != cudaSuccess) return KVS_ERR_CUDA;
+    // bf16 groups of 4 or more q-heads per kv-head are a real (if thin) contraction: tensor cores.
+    const bool use_mma = c->have_tensor_map && (c->opt_kernel == 2 || (c->opt_kernel == 0 && c->G >= 4));
+    if (use_mma) {
+        const long long plane_rows = (long long)c->cfg.max_batch * c->cfg.n_kv_heads * c->row_stride;
+        kvs::plan_decode_mma(a.units, a.n, a.D, c->sm_count, c->opt_max_ctas, &plan);
+        if (kvs::launch_decode_mma(a, plan, c->tensor_map, plane_rows * (2 * slot), plane_rows * (2 * slot + 1), st) !=
+            cudaSuccess)
+            return KVS_ERR_CUDA;
+    } else {
+        kvs::plan_decode_scalar(a.units, a.n, a.G, a.D, a.dtype, c->sm_count, c->opt_max_ctas, &plan);
+        if (kvs::launch_decode_scalar(a, plan, st) != cudaSuccess) return KVS_ERR_CUDA;
+    }
     if (kvs::launch_combine(a, plan, st) != cudaSuccess) return KVS_ERR_CUDA;
     c->last_plan = plan;
     c->stats.attention_launches += 1;
@@ -262,6 +278,14 @@ kvs_status kvs_bind_memory(kvs_ctx* ctx, void* pool, size_t pool_bytes, void* wo
     if (cudaMemsetAsync(pool, 0, need_pool, 0) != cudaSuccess) return KVS_ERR_CUDA;
     if (cudaMemsetAsync(workspace, 0, ctx->ws_bytes, 0) != cudaSuccess) return KVS_ERR_CUDA;
     if (cudaStreamSynchronize(0) != cudaSuccess) return KVS_ERR_CUDA;
+    ctx->have_tensor_map = false;
+    if (ctx->cfg.dtype == KVS_BF16) {
+        const long long total_rows = (long long)(need_pool / ctx->row_bytes);
+        if (total_rows >= (1ll << 31)) return KVS_ERR_INVALID_ARG;
+        if (kvs::make_pool_tensor_map(ctx->tensor_map, pool, total_rows, ctx->cfg.head_dim) != cudaSuccess)
+            return KVS_ERR_CUDA;
+        ctx->have_tensor_map = true;
+    }
     ctx->sm_count = sms;
     ctx->pool = static_cast<char*>(pool);
     ctx->ws = static_cast<char*>(workspace);
@@ -410,6 +434,7 @@ kvs_status kvs_set_option(kvs_ctx* ctx, int32_t option, int32_t value) {
             return KVS_OK;
         case KVS_OPT_KERNEL:
             if (value < 0 || value > 2) return KVS_ERR_INVALID_ARG;
+            if (value == 2 && ctx->cfg.dtype != KVS_BF16) return KVS_ERR_INVALID_ARG;  // tensor-core path is bf16 only
             ctx->opt_kernel = value;
             return KVS_OK;
         default:

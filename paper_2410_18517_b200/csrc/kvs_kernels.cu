@@ -338,31 +338,33 @@ __global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G>::MIN_BLOC
 }
 
 // --------------------------------------------------------------------------------------
-// K3: combine.  One block per unit, D threads; out = sum_c w_c o_c / sum_c w_c l_c with
-// w_c = 2^(m_c - M), M = max_c m_c over the pieces c of the unit.
+// K3: combine.  One block per (unit, q-head), D threads; out = sum_c w_c o_c / sum_c w_c l_c
+// with w_c = 2^(m_c - M), M = max_c m_c over the pieces c of the unit, always summed in
+// piece order so that the result does not depend on which block finished first.
 // --------------------------------------------------------------------------------------
 __global__ void decode_combine_kernel(const float* __restrict__ part_o, const float* __restrict__ part_ml,
                                       float* __restrict__ out, int G, int D, int tpu, long long T, int NC) {
-    const long long u = blockIdx.x;
+    const long long u = blockIdx.x / G;
+    const int g = blockIdx.x % G;
     const int c0 = cta_of_tile(u * tpu, T, NC);
     const int c1 = cta_of_tile((u + 1) * tpu - 1, T, NC);
     const int d = threadIdx.x;
-    for (int g = 0; g < G; ++g) {
-        float M = -1.0e30f;
-        for (int c = c0; c <= c1; ++c) M = fmaxf(M, part_ml[((u + c) * G + g) * 2]);
-        float o = 0.f, den = 0.f;
-        for (int c = c0; c <= c1; ++c) {
-            const long long pid = u + c;
-            const float w = fast_exp2(part_ml[(pid * G + g) * 2] - M);
-            o = fmaf(w, part_o[(pid * G + g) * D + d], o);
-            den = fmaf(w, part_ml[(pid * G + g) * 2 + 1], den);
-        }
-        out[(u * G + g) * D + d] = o / den;
+    float M = -1.0e30f;
+    for (int c = c0; c <= c1; ++c) M = fmaxf(M, part_ml[((u + c) * G + g) * 2]);
+    float o = 0.f, den = 0.f;
+#pragma unroll 4
+    for (int c = c0; c <= c1; ++c) {
+        const long long pid = u + c;
+        const float w = fast_exp2(part_ml[(pid * G + g) * 2] - M);
+        o = fmaf(w, part_o[(pid * G + g) * D + d], o);
+        den = fmaf(w, part_ml[(pid * G + g) * 2 + 1], den);
     }
+    out[(u * G + g) * D + d] = o / den;
 }
 
 cudaError_t launch_combine(const DecodeArgs& a, const DecodePlan& plan, cudaStream_t stream) {
-    decode_combine_kernel<<<a.units, a.D, 0, stream>>>(a.part_o, a.part_ml, a.out, a.G, a.D, plan.tpu, plan.T, plan.NC);
+    decode_combine_kernel<<<a.units * a.G, a.D, 0, stream>>>(a.part_o, a.part_ml, a.out, a.G, a.D, plan.tpu, plan.T,
+                                                            plan.NC);
     return cudaGetLastError();
 }
 

@@ -44,8 +44,20 @@ constexpr int kMaxCtas = 1024;
 // max_ctas <= 0 means automatic.  Host-only arithmetic (no CUDA call).
 void plan_decode_scalar(int units, int n, int G, int D, int dtype, int sm_count, int max_ctas, DecodePlan* plan);
 
+// Same for the tensor-core kernel (bf16 storage only).
+void plan_decode_mma(int units, int n, int D, int sm_count, int max_ctas, DecodePlan* plan);
+
 // One-time per-process kernel attribute set-up for the current device.
 cudaError_t init_kernels();
+cudaError_t init_mma_kernels();
+
+// Encode the TMA tensor map of a bf16 pool seen as [total_rows][D]; `storage` is 128 bytes,
+// 64-byte aligned, host memory.
+cudaError_t make_pool_tensor_map(void* storage, void* pool, long long total_rows, int D);
+
+// krow0 / vrow0: first row of the K / V plane in the pool-wide row numbering.
+cudaError_t launch_decode_mma(const DecodeArgs& a, const DecodePlan& plan, const void* tensor_map, long long krow0,
+                              long long vrow0, cudaStream_t stream);
 
 cudaError_t launch_append(const void* k, const void* v, void* kplane, void* vplane, int B, int n_new, int Hkv,
                           int row_bytes, int row_stride, int len0, cudaStream_t stream);

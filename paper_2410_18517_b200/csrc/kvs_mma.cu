@@ -1,0 +1,401 @@
+// K2b: grouped-query split-K decode attention on the tensor cores (bf16 storage only).
+//
+// The G q-heads that share one kv-head form the (zero-padded) 16-row M side of
+// mma.sync.m16n8k16 bf16 -> fp32 tiles: S = Q K^T over 16-token blocks, then O += P V with
+// the softmax weights split as P = P_hi + P_lo (two bf16 terms) so that the second
+// contraction keeps ~16 bits of P.  K/V tiles arrive by TMA tensor-map copies with the
+// 128-byte swizzle, which makes ldmatrix (K) and ldmatrix.trans (V) conflict-free.
+// Work decomposition, partial-result layout and the combine kernel are those of the scalar
+// path.  One producer warp, four consumer warps; each consumer warp owns 16-token blocks.
+#include <cuda.h>
+
+#include <algorithm>
+
+#include "kvs_device.cuh"
+#include "kvs_kernels.h"
+
+namespace kvs {
+
+namespace {
+
+constexpr int kMmaWarps = 4;
+constexpr int kMmaConsumerThreads = kMmaWarps * 32;
+constexpr int kMmaThreads = kMmaConsumerThreads + 32;
+constexpr int kMmaTileBytes = 16384;
+constexpr int kMmaQBytes = 2048;  // room for 8 heads x 128 x bf16
+constexpr int kMmaStages = 3;
+
+template <int D>
+struct MmaShape {
+    static constexpr int RB = D * 2;
+    static constexpr int HALVES = D / 64;                  // 128-byte column blocks per row
+    static constexpr int TN = kMmaTileBytes / RB;          // rows per tile: 64 (D=128) or 128 (D=64)
+    static constexpr int BPW = TN / (kMmaWarps * 16);      // 16-token blocks per warp per tile
+    static constexpr int KSTEPS = D / 16;
+    static constexpr int NB = D / 8;
+    static constexpr int STAGE_BYTES = 2 * kMmaTileBytes + kMmaQBytes;
+    static constexpr int SCRATCH_FLOATS = kMmaWarps * (D + 2);
+    static constexpr int SMEM_BYTES = 1024 + kMmaStages * STAGE_BYTES + SCRATCH_FLOATS * 4 + 2 * kMmaStages * 8 + 16;
+};
+
+__device__ __forceinline__ void tma_load_2d(void* dst_smem, const CUtensorMap* tmap, int x, int y, uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(
+            smem_u32(dst_smem)),
+        "l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y), "r"(smem_u32(bar))
+        : "memory");
+}
+
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t saddr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(saddr));
+}
+
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t saddr) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(saddr));
+}
+
+// D(16x8) += A(16x16) B(16x8), rows 8..15 of A are zero padding: their accumulators are
+// kept in throw-away registers (c2, c3) that stay zero.
+__device__ __forceinline__ void mma_bf16_upper(float& c0, float& c1, uint32_t a_klo, uint32_t a_khi, uint32_t b0,
+                                               uint32_t b1) {
+    float z2 = 0.f, z3 = 0.f;
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(c0), "+f"(c1), "+f"(z2), "+f"(z3)
+        : "r"(a_klo), "r"(0u), "r"(a_khi), "r"(0u), "r"(b0), "r"(b1));
+}
+
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+
+__device__ __forceinline__ float bf16_round(float x) { return __bfloat162float(__float2bfloat16_rn(x)); }
+
+struct MmaKernelArgs {
+    const char* q;
+    float* part_o;
+    float* part_ml;
+    int* status;
+    int n;
+    int row_stride;
+    int tpu;
+    long long T;
+    long long krow0;  // first row of the K plane within the pool-wide row index
+    long long vrow0;
+    float scale_log2;
+};
+
+template <int D, int G>
+__global__ void __launch_bounds__(kMmaThreads, 2)
+    decode_splitk_mma(const __grid_constant__ CUtensorMap tmap, const MmaKernelArgs a) {
+    using S = MmaShape<D>;
+    constexpr int TN = S::TN, KSTEPS = S::KSTEPS, NB = S::NB, BPW = S::BPW;
+    constexpr int QBYTES = G * S::RB;
+
+    extern __shared__ unsigned char smem_raw[];
+    // 128-byte swizzled tiles need 1024-byte aligned bases
+    unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
+    float* scratch = reinterpret_cast<float*>(smem + kMmaStages * S::STAGE_BYTES);
+    uint64_t* full_bar = reinterpret_cast<uint64_t*>(scratch + S::SCRATCH_FLOATS);
+    uint64_t* empty_bar = full_bar + kMmaStages;
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(empty_bar + kMmaStages);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int NC = gridDim.x;
+    const long long t0 = ((long long)blockIdx.x * a.T) / NC;
+    const long long t1 = ((long long)(blockIdx.x + 1) * a.T) / NC;
+
+    if (tid == 0) {
+        for (int s = 0; s < kMmaStages; ++s) {
+            mbar_init(&full_bar[s], 1);
+            mbar_init(&empty_bar[s], kMmaWarps);
+        }
+        abort_flag[0] = 0;
+        abort_flag[1] = 0;
+        fence_mbar_init();
+    }
+    __syncthreads();
+
+    if (warp == kMmaWarps) {
+        // ------------------------------ producer ------------------------------
+        if (lane == 0) {
+            int it = 0;
+            bool ok = true;
+            for (long long gt = t0; gt < t1; ++gt, ++it) {
+                const int st = it % kMmaStages;
+                if (it >= kMmaStages)
+                    ok = mbar_wait_bounded(&empty_bar[st], ((it / kMmaStages) - 1) & 1, abort_flag, a.status);
+                if (!ok) break;
+                const long long u = gt / a.tpu;
+                const int ti = (int)(gt - u * a.tpu);
+                const bool with_q = (gt == t0) || (ti == 0);
+                unsigned char* sb = smem + st * S::STAGE_BYTES;
+                mbar_arrive_expect_tx(&full_bar[st], 2 * kMmaTileBytes + (with_q ? QBYTES : 0));
+                const long long row = u * a.row_stride + (long long)ti * TN;
+#pragma unroll
+                for (int h = 0; h < S::HALVES; ++h) {
+                    tma_load_2d(sb + h * (TN * 128), &tmap, h * 64, (int)(a.krow0 + row), &full_bar[st]);
+                    tma_load_2d(sb + kMmaTileBytes + h * (TN * 128), &tmap, h * 64, (int)(a.vrow0 + row), &full_bar[st]);
+                }
+                if (with_q) bulk_g2s(sb + 2 * kMmaTileBytes, a.q + u * (long long)QBYTES, QBYTES, &full_bar[st]);
+            }
+            if (!ok) {
+                for (int j = max(0, it - kMmaStages); j < it; ++j)
+                    mbar_wait_bounded(&full_bar[j % kMmaStages], (j / kMmaStages) & 1, abort_flag + 1, a.status);
+            }
+        }
+        return;
+    }
+
+    // ---------------------------------- consumers ----------------------------------
+    const int row = lane >> 2;   // q-head row of the accumulator fragment (rows 8..15 are padding)
+    const int quad = lane & 3;
+
+    int it = 0;
+    long long gt = t0;
+    while (gt < t1) {
+        const long long u = gt / a.tpu;
+        const int ti0 = (int)(gt - u * a.tpu);
+        const int piece_tiles = (int)min((long long)(a.tpu - ti0), t1 - gt);
+
+        uint32_t qa[KSTEPS][2];
+        float o[NB][2];
+        float m = -1.0e30f, lsum = 0.f;
+#pragma unroll
+        for (int nb = 0; nb < NB; ++nb) o[nb][0] = o[nb][1] = 0.f;
+
+        for (int k = 0; k < piece_tiles; ++k, ++it) {
+            const int st = it % kMmaStages;
+            if (!mbar_wait_bounded(&full_bar[st], (it / kMmaStages) & 1, abort_flag, a.status)) return;
+            const unsigned char* ks = smem + st * S::STAGE_BYTES;
+            const uint32_t ks_u32 = smem_u32(ks);
+            const uint32_t vs_u32 = ks_u32 + kMmaTileBytes;
+            if (k == 0) {
+                // A fragments of Q: row g < G real, the rest zero
+                const uint32_t* qs = reinterpret_cast<const uint32_t*>(ks + 2 * kMmaTileBytes);
+#pragma unroll
+                for (int s = 0; s < KSTEPS; ++s) {
+                    qa[s][0] = row < G ? qs[row * (D / 2) + s * 8 + quad] : 0u;
+                    qa[s][1] = row < G ? qs[row * (D / 2) + s * 8 + 4 + quad] : 0u;
+                }
+            }
+            const int valid = a.n - (ti0 + k) * TN;  // rows of this tile that exist (may exceed TN)
+
+#pragma unroll
+            for (int blk = 0; blk < BPW; ++blk) {
+                const int tok0 = (warp * BPW + blk) * 16;
+                // ---- S = Q K^T for 16 tokens: two 8-token column blocks ----
+                float s[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
+                {
+                    const int t = tok0 + ((lane >> 4) << 3) + (lane & 7);
+                    const uint32_t rowaddr = ks_u32 + t * 128;
+                    const int sw = t & 7;
+#pragma unroll
+                    for (int st_k = 0; st_k < KSTEPS; ++st_k) {
+                        const int half = st_k >> 2;
+                        const int chunk = ((st_k & 3) << 1) + ((lane >> 3) & 1);
+                        uint32_t b[4];
+                        ldmatrix_x4(b, rowaddr + half * (TN * 128) + ((chunk ^ sw) << 4));
+                        mma_bf16_upper(s[0][0], s[0][1], qa[st_k][0], qa[st_k][1], b[0], b[1]);
+                        mma_bf16_upper(s[1][0], s[1][1], qa[st_k][0], qa[st_k][1], b[2], b[3]);
+                    }
+                }
+                // ---- online softmax for row `row`, tokens tok0 + nb*8 + quad*2 + j ----
+                float tmax = -INFINITY;
+#pragma unroll
+                for (int nb = 0; nb < 2; ++nb)
+#pragma unroll
+                    for (int j = 0; j < 2; ++j) {
+                        const int tok = tok0 + nb * 8 + quad * 2 + j;
+                        s[nb][j] = tok < valid ? s[nb][j] * a.scale_log2 : -INFINITY;
+                        tmax = fmaxf(tmax, s[nb][j]);
+                    }
+                tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 1));
+                tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 2));
+                const float m_new = fmaxf(m, tmax);
+                const float alpha = fast_exp2(m - m_new);
+                m = m_new;
+                float p[2][2];
+                float psum = 0.f;
+#pragma unroll
+                for (int nb = 0; nb < 2; ++nb)
+#pragma unroll
+                    for (int j = 0; j < 2; ++j) {
+                        p[nb][j] = fast_exp2(s[nb][j] - m_new);
+                        psum += p[nb][j];
+                    }
+                lsum = lsum * alpha + psum;
+#pragma unroll
+                for (int nb = 0; nb < NB; ++nb) {
+                    o[nb][0] *= alpha;
+                    o[nb][1] *= alpha;
+                }
+                // P = P_hi + P_lo as A fragments (k = tokens): klo = tokens 0..7, khi = tokens 8..15
+                const float h00 = bf16_round(p[0][0]), h01 = bf16_round(p[0][1]);
+                const float h10 = bf16_round(p[1][0]), h11 = bf16_round(p[1][1]);
+                const uint32_t phi_lo = pack_bf16(h00, h01), phi_hi = pack_bf16(h10, h11);
+                const uint32_t plo_lo = pack_bf16(p[0][0] - h00, p[0][1] - h01);
+                const uint32_t plo_hi = pack_bf16(p[1][0] - h10, p[1][1] - h11);
+                // ---- O += P V: 16 tokens x D, two 8-wide column blocks per ldmatrix ----
+                {
+                    const int t = tok0 + (((lane >> 3) & 1) << 3) + (lane & 7);
+                    const uint32_t rowaddr = vs_u32 + t * 128;
+                    const int sw = t & 7;
+#pragma unroll
+                    for (int nbp = 0; nbp < NB / 2; ++nbp) {
+                        const int chunkg = nbp * 2 + (lane >> 4);
+                        const int half = chunkg >> 3;
+                        const int chunk = chunkg & 7;
+                        uint32_t b[4];
+                        ldmatrix_x4_trans(b, rowaddr + half * (TN * 128) + ((chunk ^ sw) << 4));
+                        mma_bf16_upper(o[2 * nbp][0], o[2 * nbp][1], phi_lo, phi_hi, b[0], b[1]);
+                        mma_bf16_upper(o[2 * nbp][0], o[2 * nbp][1], plo_lo, plo_hi, b[0], b[1]);
+                        mma_bf16_upper(o[2 * nbp + 1][0], o[2 * nbp + 1][1], phi_lo, phi_hi, b[2], b[3]);
+                        mma_bf16_upper(o[2 * nbp + 1][0], o[2 * nbp + 1][1], plo_lo, plo_hi, b[2], b[3]);
+                    }
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&empty_bar[st]);
+        }
+
+        // ---- end of piece: merge the four warps, one q-head at a time ----
+        const long long pid = u + blockIdx.x;
+        float l = lsum;
+        l += __shfl_xor_sync(0xffffffffu, l, 1);
+        l += __shfl_xor_sync(0xffffffffu, l, 2);
+#pragma unroll
+        for (int g = 0; g < G; ++g) {
+            named_bar_sync(1, kMmaConsumerThreads);
+            if (row == g) {
+                float* dst = scratch + warp * (D + 2);
+#pragma unroll
+                for (int nb = 0; nb < NB; ++nb) {
+                    dst[nb * 8 + quad * 2] = o[nb][0];
+                    dst[nb * 8 + quad * 2 + 1] = o[nb][1];
+                }
+                if (quad == 0) {
+                    dst[D] = m;
+                    dst[D + 1] = l;
+                }
+            }
+            named_bar_sync(1, kMmaConsumerThreads);
+            for (int d = tid; d < D; d += kMmaConsumerThreads) {
+                float M = -1.0e30f;
+#pragma unroll
+                for (int j = 0; j < kMmaWarps; ++j) M = fmaxf(M, scratch[j * (D + 2) + D]);
+                float acc = 0.f, den = 0.f;
+#pragma unroll
+                for (int j = 0; j < kMmaWarps; ++j) {
+                    const float w = fast_exp2(scratch[j * (D + 2) + D] - M);
+                    acc = fmaf(w, scratch[j * (D + 2) + d], acc);
+                    den = fmaf(w, scratch[j * (D + 2) + D + 1], den);
+                }
+                a.part_o[(pid * G + g) * D + d] = acc;
+                if (d == 0) {
+                    a.part_ml[(pid * G + g) * 2] = M;
+                    a.part_ml[(pid * G + g) * 2 + 1] = den;
+                }
+            }
+        }
+        gt += piece_tiles;
+    }
+}
+
+template <int D, int G>
+cudaError_t set_attr() {
+    return cudaFuncSetAttribute(decode_splitk_mma<D, G>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                MmaShape<D>::SMEM_BYTES);
+}
+
+template <int D, int G>
+cudaError_t launch_one(const CUtensorMap& tm, const MmaKernelArgs& ka, int NC, cudaStream_t stream) {
+    decode_splitk_mma<D, G><<<NC, kMmaThreads, MmaShape<D>::SMEM_BYTES, stream>>>(tm, ka);
+    return cudaGetLastError();
+}
+
+template <int D>
+cudaError_t launch_groups(int G, const CUtensorMap& tm, const MmaKernelArgs& ka, int NC, cudaStream_t stream) {
+    switch (G) {
+        case 1: return launch_one<D, 1>(tm, ka, NC, stream);
+        case 2: return launch_one<D, 2>(tm, ka, NC, stream);
+        case 4: return launch_one<D, 4>(tm, ka, NC, stream);
+        case 8: return launch_one<D, 8>(tm, ka, NC, stream);
+        default: return cudaErrorInvalidValue;
+    }
+}
+
+}  // namespace
+
+cudaError_t init_mma_kernels() {
+    cudaError_t e;
+    if ((e = set_attr<128, 1>()) != cudaSuccess) return e;
+    if ((e = set_attr<128, 2>()) != cudaSuccess) return e;
+    if ((e = set_attr<128, 4>()) != cudaSuccess) return e;
+    if ((e = set_attr<128, 8>()) != cudaSuccess) return e;
+    if ((e = set_attr<64, 1>()) != cudaSuccess) return e;
+    if ((e = set_attr<64, 2>()) != cudaSuccess) return e;
+    if ((e = set_attr<64, 4>()) != cudaSuccess) return e;
+    return set_attr<64, 8>();
+}
+
+// Tensor map over the whole pool seen as [total_rows][D] bf16, box = 64 columns x tile rows,
+// 128-byte swizzle.  `storage` must be 64-byte aligned and hold sizeof(CUtensorMap) = 128 bytes.
+cudaError_t make_pool_tensor_map(void* storage, void* pool, long long total_rows, int D) {
+    typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                 const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                 CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
+    if (e != cudaSuccess) return e;
+    if (qres != cudaDriverEntryPointSuccess || fn == nullptr) return cudaErrorNotSupported;
+    const int tile_rows = kMmaTileBytes / (D * 2);
+    cuuint64_t dims[2] = {(cuuint64_t)D, (cuuint64_t)total_rows};
+    cuuint64_t strides[1] = {(cuuint64_t)D * 2};
+    cuuint32_t box[2] = {64u, (cuuint32_t)tile_rows};
+    cuuint32_t estr[2] = {1u, 1u};
+    CUresult r = reinterpret_cast<EncodeFn>(fn)(reinterpret_cast<CUtensorMap*>(storage), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16,
+                                                2, pool, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? cudaSuccess : cudaErrorInvalidValue;
+}
+
+void plan_decode_mma(int units, int n, int D, int sm_count, int max_ctas, DecodePlan* plan) {
+    plan->tile_rows = kMmaTileBytes / (D * 2);
+    plan->tpu = (n + plan->tile_rows - 1) / plan->tile_rows;
+    plan->T = (long long)units * plan->tpu;
+    int cap = sm_count * 2;
+    if (max_ctas > 0) cap = std::min(cap, max_ctas);
+    cap = std::min(cap, kMaxCtas);
+    plan->NC = (int)std::min<long long>(plan->T, cap);
+    plan->kernel = 2;
+}
+
+cudaError_t launch_decode_mma(const DecodeArgs& a, const DecodePlan& plan, const void* tensor_map, long long krow0,
+                              long long vrow0, cudaStream_t stream) {
+    MmaKernelArgs ka;
+    ka.q = (const char*)a.q;
+    ka.part_o = a.part_o;
+    ka.part_ml = a.part_ml;
+    ka.status = a.status;
+    ka.n = a.n;
+    ka.row_stride = a.row_stride;
+    ka.tpu = plan.tpu;
+    ka.T = plan.T;
+    ka.krow0 = krow0;
+    ka.vrow0 = vrow0;
+    ka.scale_log2 = a.scale_log2;
+    const CUtensorMap& tm = *reinterpret_cast<const CUtensorMap*>(tensor_map);
+    if (a.D == 128) return launch_groups<128>(a.G, tm, ka, plan.NC, stream);
+    if (a.D == 64) return launch_groups<64>(a.G, tm, ka, plan.NC, stream);
+    return cudaErrorInvalidValue;
+}
+
+}  // namespace kvs

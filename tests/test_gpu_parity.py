@@ -9,7 +9,7 @@ import torch
 
 import oracle
 import synth_inputs as si
-from paper_2410_18517_b200 import KVS_OPT_MAX_CTAS, KvsError, SharedKVCache
+from paper_2410_18517_b200 import KVS_OPT_KERNEL, KVS_OPT_MAX_CTAS, KvsError, SharedKVCache
 from paper_2410_18517_b200 import binding as kb
 from paper_2410_18517_b200 import build as kbuild
 
@@ -63,6 +63,38 @@ def test_shapes_and_ragged_tails(dtype, D, Hq, Hkv, context):
                     dtype=dtype, n_shared=0, map_seed=0, steps=3, fixed_map=(0, 0, 1, 2))
     cache, orc, _ = run_small(w, steps=3)
     assert cache.num_slots() == 1
+
+
+@pytest.mark.parametrize("kernel", [1, 2])
+@pytest.mark.parametrize("D,Hq,Hkv", [(128, 4, 4), (128, 4, 2), (128, 8, 2), (128, 8, 1), (64, 2, 2), (64, 4, 2),
+                                      (64, 8, 2), (64, 8, 1)])
+@pytest.mark.parametrize("context", [0, 15, 127, 128, 129, 700])
+def test_both_kernels_on_every_group_size(kernel, D, Hq, Hkv, context):
+    """bf16: the scalar and the tensor-core kernel, forced, on group sizes 1, 2, 4 and 8."""
+    w = si.Workload(f"k{kernel}_{D}_{Hq}_{Hkv}_{context}", L=3, Hq=Hq, Hkv=Hkv, D=D, B=2, context=context,
+                    dtype="bf16", n_shared=1, map_seed=0, steps=2, fixed_map=(0, 1, 0))
+    cache, _, _ = run_small(w, steps=2, options=[(KVS_OPT_KERNEL, kernel)])
+    assert cache.last_launch()["kernel"] == kernel
+
+
+def test_auto_kernel_choice():
+    """Groups of four or more bf16 q-heads go to the tensor cores; fp32 storage never does."""
+    for Hq, Hkv, dtype, want in [(4, 4, "bf16", 1), (4, 2, "bf16", 1), (8, 2, "bf16", 2), (8, 1, "bf16", 2),
+                                 (8, 2, "f32", 1)]:
+        w = si.Workload(f"auto_{Hq}_{Hkv}_{dtype}", L=1, Hq=Hq, Hkv=Hkv, D=128, B=1, context=100, dtype=dtype,
+                        n_shared=0, map_seed=0, steps=1)
+        cache, _, _ = run_small(w, steps=1)
+        assert cache.last_launch()["kernel"] == want
+    with pytest.raises(KvsError):
+        cache.set_option(KVS_OPT_KERNEL, 2)          # the last cache is fp32
+
+
+@pytest.mark.parametrize("max_ctas", [1, 2, 5, 37, 0])
+def test_tensor_core_kernel_any_split(max_ctas):
+    w = si.Workload(f"mma_split_{max_ctas}", L=2, Hq=8, Hkv=2, D=128, B=2, context=1500, dtype="bf16",
+                    n_shared=1, map_seed=0, steps=2, fixed_map=(0, 0))
+    cache, _, _ = run_small(w, steps=2, options=[(KVS_OPT_MAX_CTAS, max_ctas), (KVS_OPT_KERNEL, 2)])
+    assert cache.last_launch()["kernel"] == 2
 
 
 @pytest.mark.parametrize("max_ctas", [1, 2, 5, 37, 0])
