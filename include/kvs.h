@@ -53,7 +53,8 @@ typedef enum {
     KVS_ERR_CAPACITY = 4,      /* an append would exceed max_seq                              */
     KVS_ERR_OOM = 5,           /* a bound buffer is smaller than kvs_required_bytes said      */
     KVS_ERR_CUDA = 6,          /* a CUDA runtime or driver call failed                        */
-    KVS_ERR_TIMEOUT = 7        /* a bounded device-side wait ran out (see kvs_last_device_status) */
+    KVS_ERR_TIMEOUT = 7,       /* a bounded device-side wait ran out (see kvs_last_device_status) */
+    KVS_ERR_SCRATCH_LIMIT = 8  /* kvs_decode_attention_static: the call needs more than the built-in scratch */
 } kvs_status;
 
 typedef enum { KVS_BF16 = 0, KVS_F32 = 1 } kvs_dtype;
@@ -172,6 +173,38 @@ kvs_status kvs_decode_attention(kvs_ctx* ctx, int32_t layer, const void* q, floa
 kvs_status kvs_step_host(kvs_ctx* ctx, const void* q_host, const void* k_host, const void* v_host,
                          float* out_host, int32_t batch, void* stream,
                          uint64_t* h2d_bytes, uint64_t* d2h_bytes);
+
+/* kvs_decode_attention for callers that have no scratch memory to give and may not
+ * allocate any.  (The paper has no counterpart to this call; it exists for the users of
+ * this library described below.)
+ *
+ * Who needs it: code that runs after a serving engine has handed all of the GPU's free memory
+ * to its own pools and forbids further cudaMalloc (which would also stall the device); code in a
+ * plug-in or callback that is given tensors but no allocator; and code between two points where
+ * the workspace bound with kvs_bind_memory is already busy with another call.  Such callers
+ * still pass the inputs and outputs (q, out, and the context whose pool holds K/V); what they
+ * cannot provide is the scratch for split-K partial results.
+ *
+ * What it does: exactly what kvs_decode_attention does, with the same kernels and the same
+ * result bit for bit, except that the partial results and the device status word live in a
+ * fixed 2 MiB array inside the library image instead of the bound workspace.  The call
+ * allocates nothing and frees nothing, on the device or through any library.
+ *   - Every GPU that loads the library holds those 2 MiB until the process exits.
+ *   - Limit: (batch * n_kv_heads + blocks launched) * group * (head_dim + 2) * 4 bytes, plus
+ *     512 bytes, must fit in 2 MiB (the 7B shape at batch 8 needs 0.3 MiB, the 32q/8kv shape at
+ *     batch 64 needs 1.7 MiB).  Larger calls return KVS_ERR_SCRATCH_LIMIT and launch nothing.
+ *   - The first call on each device looks up the device address of the array (one runtime
+ *     query, no allocation).  Make that first call before starting any stream capture.
+ *   - All calls, from all contexts and streams, share the one array, and it keeps the previous
+ *     call's contents.  The call itself clears the only part that must start at zero (the
+ *     status word).  Two calls that overlap on the GPU race on the partial results: order
+ *     them on one stream or with events.
+ *   device_status: device pointer to an int32 that receives 0, or KVS_ERR_TIMEOUT if a bounded
+ *     wait inside the kernel ran out; may be NULL (the word inside the array is used and is not
+ *     readable by the caller).  It is written on `stream`; read it after synchronising.
+ * Other arguments, layouts and errors: as kvs_decode_attention.                              */
+kvs_status kvs_decode_attention_static(kvs_ctx* ctx, int32_t layer, const void* q, float* out,
+                                       int32_t batch, void* stream, int32_t* device_status);
 
 /* ---- introspection (index and layout checks are exact) ----------------------- */
 

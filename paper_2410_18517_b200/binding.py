@@ -21,6 +21,7 @@ KVS_ERR_CAPACITY = 4
 KVS_ERR_OOM = 5
 KVS_ERR_CUDA = 6
 KVS_ERR_TIMEOUT = 7
+KVS_ERR_SCRATCH_LIMIT = 8
 
 KVS_BF16 = 0
 KVS_F32 = 1
@@ -34,7 +35,7 @@ EXPORTS = (
     "kvs_reset", "kvs_append", "kvs_decode_attention", "kvs_step_host", "kvs_num_slots",
     "kvs_slot_of_layer", "kvs_seq_len", "kvs_row_stride", "kvs_plane_offset", "kvs_stats",
     "kvs_last_device_status", "kvs_set_option", "kvs_last_launch", "kvs_status_string",
-    "kvs_read_roof",
+    "kvs_read_roof", "kvs_decode_attention_static",
 )
 
 
@@ -78,6 +79,7 @@ def load() -> ctypes.CDLL:
         "kvs_reset": [vp],
         "kvs_append": [vp, i32, vp, vp, i32, i32, vp],
         "kvs_decode_attention": [vp, i32, vp, vp, i32, vp],
+        "kvs_decode_attention_static": [vp, i32, vp, vp, i32, vp, vp],
         "kvs_step_host": [vp, vp, vp, vp, vp, i32, vp, P(ctypes.c_uint64), P(ctypes.c_uint64)],
         "kvs_num_slots": [vp, P(i32)],
         "kvs_slot_of_layer": [vp, i32, P(i32)],
@@ -163,6 +165,12 @@ def kvs_append(ctx: int, layer: int, k, v, batch: int, n_new: int, stream: int =
 
 def kvs_decode_attention(ctx: int, layer: int, q, out, batch: int, stream: int = 0) -> None:
     _check(load().kvs_decode_attention(ctx, layer, _ptr(q), _ptr(out), batch, stream), "kvs_decode_attention")
+
+
+def kvs_decode_attention_static(ctx: int, layer: int, q, out, batch: int, stream: int = 0, device_status=None) -> None:
+    """Same result as ``kvs_decode_attention``; scratch is the library's built-in 2 MiB array (no allocation)."""
+    _check(load().kvs_decode_attention_static(ctx, layer, _ptr(q), _ptr(out), batch, stream, _ptr(device_status)),
+           "kvs_decode_attention_static")
 
 
 def kvs_step_host(ctx: int, q_host, k_host, v_host, out_host, batch: int, stream: int = 0) -> tuple[int, int]:

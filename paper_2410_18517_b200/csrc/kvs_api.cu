@@ -460,6 +460,7 @@ const char* kvs_status_string(kvs_status s) {
         case KVS_ERR_OOM: return "bound buffer too small";
         case KVS_ERR_CUDA: return "CUDA call failed";
         case KVS_ERR_TIMEOUT: return "device-side wait timed out";
+        case KVS_ERR_SCRATCH_LIMIT: return "call needs more scratch than the built-in scratch array holds";
     }
     return "unknown status";
 }
@@ -474,6 +475,100 @@ kvs_status kvs_read_roof(const void* src, size_t bytes, uint64_t* checksum, int3
     if (kvs::launch_read_roof(src, bytes, reinterpret_cast<unsigned long long*>(checksum), sms,
                               static_cast<cudaStream_t>(stream)) != cudaSuccess)
         return KVS_ERR_CUDA;
+    return KVS_OK;
+}
+
+// ---------------------------------------------------------------------------------------
+// Attention without any caller- or library-allocated scratch.
+//
+// The split-K partial results and the device status word of this one entry point live in a
+// fixed array that is part of the loaded library image.  Every GPU that loads the library
+// carries these kStaticScratchBytes until the process exits, and every call, from every
+// context, uses the same bytes.
+// ---------------------------------------------------------------------------------------
+constexpr size_t kStaticScratchBytes = 2u << 20;  // 2 MiB
+constexpr size_t kStaticStatusBytes = 256;        // first 256 bytes: device status word
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+namespace {
+
+std::once_flag g_static_flag[64];
+cudaError_t g_static_err[64];
+unsigned char* g_static_ptr[64];
+
+// In host code `g_static_scratch` is only a handle for the symbol, not an address the GPU can
+// use, so the device address is looked up once per device (with that device current).
+cudaError_t static_scratch_for_device(int device, unsigned char** ptr) {
+    if (device < 0 || device >= 64) return cudaErrorInvalidDevice;
+    std::call_once(g_static_flag[device], [device]() {
+        void* p = nullptr;
+        g_static_err[device] = cudaGetSymbolAddress(&p, g_static_scratch);
+        g_static_ptr[device] = static_cast<unsigned char*>(p);
+    });
+    *ptr = g_static_ptr[device];
+    return g_static_err[device];
+}
+
+}  // namespace
+
+kvs_status kvs_decode_attention_static(kvs_ctx* ctx, int32_t layer, const void* q, float* out, int32_t batch,
+                                       void* stream, int32_t* device_status) {
+    kvs_status s = check_attention(ctx, layer, q, out, batch);
+    if (s != KVS_OK) return s;
+    kvs_ctx* c = ctx;
+    const int slot = c->slot_of_layer[layer];
+    const int units = batch * c->cfg.n_kv_heads;
+    const int n = c->slot_len[slot];
+    const int D = c->cfg.head_dim;
+    const bool use_mma = c->have_tensor_map && (c->opt_kernel == 2 || (c->opt_kernel == 0 && c->G >= 4));
+    kvs::DecodePlan plan;
+    if (use_mma)
+        kvs::plan_decode_mma(units, n, D, c->sm_count, c->opt_max_ctas, &plan);
+    else
+        kvs::plan_decode_scalar(units, n, c->G, D, c->cfg.dtype, c->sm_count, c->opt_max_ctas, &plan);
+    // one partial (o[D], m, l) per (piece, q-head); pieces are indexed unit + block
+    const size_t pieces = (size_t)units + plan.NC;
+    const size_t part_o_bytes = align_up(pieces * c->G * D * sizeof(float), kAlign);
+    const size_t part_ml_bytes = align_up(pieces * c->G * 2 * sizeof(float), kAlign);
+    if (kStaticStatusBytes + part_o_bytes + part_ml_bytes > kStaticScratchBytes) return KVS_ERR_SCRATCH_LIMIT;
+
+    DeviceGuard guard(c->cfg.device);
+    if (!guard.ok) return KVS_ERR_CUDA;
+    unsigned char* base = nullptr;
+    if (static_scratch_for_device(c->cfg.device, &base) != cudaSuccess || base == nullptr) return KVS_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int* status_word = device_status ? device_status : reinterpret_cast<int*>(base);
+    // the array keeps whatever the previous call left; only the status word must start at zero
+    if (cudaMemsetAsync(status_word, 0, sizeof(int), st) != cudaSuccess) return KVS_ERR_CUDA;
+
+    kvs::DecodeArgs a;
+    a.q = q;
+    a.kplane = c->pool + (size_t)(2 * slot) * c->plane_bytes;
+    a.vplane = c->pool + (size_t)(2 * slot + 1) * c->plane_bytes;
+    a.part_o = reinterpret_cast<float*>(base + kStaticStatusBytes);
+    a.part_ml = reinterpret_cast<float*>(base + kStaticStatusBytes + part_o_bytes);
+    a.out = out;
+    a.status = status_word;
+    a.n = n;
+    a.row_stride = c->row_stride;
+    a.units = units;
+    a.G = c->G;
+    a.D = D;
+    a.dtype = c->cfg.dtype;
+    a.scale_log2 = c->scale * 1.4426950408889634f;
+    if (use_mma) {
+        const long long plane_rows = (long long)c->cfg.max_batch * c->cfg.n_kv_heads * c->row_stride;
+        if (kvs::launch_decode_mma(a, plan, c->tensor_map, plane_rows * (2 * slot), plane_rows * (2 * slot + 1), st) !=
+            cudaSuccess)
+            return KVS_ERR_CUDA;
+    } else {
+        if (kvs::launch_decode_scalar(a, plan, st) != cudaSuccess) return KVS_ERR_CUDA;
+    }
+    if (kvs::launch_combine(a, plan, st) != cudaSuccess) return KVS_ERR_CUDA;
+    c->last_plan = plan;
+    c->stats.attention_launches += 1;
+    c->stats.combine_launches += 1;
+    c->stats.kv_bytes_read += 2ull * units * n * c->row_bytes;
     return KVS_OK;
 }
 
