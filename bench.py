@@ -206,7 +206,7 @@ def main():
 
     import torch
 
-    from paper_2410_18517_b200 import SharedKVCache
+    from paper_2410_18517_b200 import SharedKVCache, dist_util
     from paper_2410_18517_b200 import build as kbuild
 
     rank = int(os.environ.get("RANK", "0"))
@@ -284,10 +284,7 @@ def main():
     sync_all()
     ms = ev0.elapsed_time(ev1)
     st1 = cache.stats()
-    if dist is not None:
-        tmax = torch.tensor([ms], device=dev)
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        ms = float(tmax.item())
+    ms = dist_util.max_over_ranks(ms, dev)
     launches = sum(st1[k] - st0[k] for k in ("append_launches", "attention_launches", "combine_launches"))
     kv_read = st1["kv_bytes_read"] - st0["kv_bytes_read"]
     kv_app = st1["kv_bytes_appended"] - st0["kv_bytes_appended"]
@@ -322,10 +319,7 @@ def main():
     e1.record()
     sync_all()
     e2e_ms = e0.elapsed_time(e1)
-    if dist is not None:
-        tmax = torch.tensor([e2e_ms], device=dev)
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        e2e_ms = float(tmax.item())
+    e2e_ms = dist_util.max_over_ranks(e2e_ms, dev)
     clocks = sampler.stop() if rank == 0 else None
     status = cache.device_status()
 
@@ -345,7 +339,7 @@ def main():
     n_mid = n_start + K // 2
     pool_unshared = cache.pool_bytes // cache.num_slots() * w.L
     line = {
-        "metric": METRIC, "value": world * w.B / (step_ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K,
+        "metric": METRIC, "value": dist_util.whole_job_rate(w.B, world, step_ms), "unit": UNIT, "n_gpus": world, "steps": K,
         "warmup": W, "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f32", "data": "synthetic", "config": workload_config(w, world),
         "kv_read_gbs_whole_step": kv_read / (ms * 1e-3) / 1e9,
@@ -360,7 +354,7 @@ def main():
                      "frac": achieved / peak, "frac_of_8tbs_nominal": achieved / NOMINAL_HBM_GBS,
                      "traffic": traffic, "bytes_per_launch": bytes_per_launch, "ms_per_launch": att_launch_ms,
                      "launches_timed": len(att_ms)},
-        "e2e": {"value": world * w.B / (e2e_ms / E * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+        "e2e": {"value": dist_util.whole_job_rate(w.B, world, e2e_ms / E), "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "steps": E, "ms_per_step": e2e_ms / E},
         "gpu_launches": launches,
         "clocks": clocks,

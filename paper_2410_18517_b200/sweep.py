@@ -1,0 +1,122 @@
+"""Sweep of the grouped-query shape (32 layers, 32 q-heads / 8 kv-heads, D=128, bf16) over batch,
+context and shared-layer fraction.  One JSON line per point: time per decode step, attention-path
+tokens/s, KV-read GB/s and pool size.
+
+    python -m paper_2410_18517_b200.sweep [--out FILE] [--steps K] [--only B,N,P]
+
+A *step* is one pass over all layers (append on computing layers + attention on every layer).
+Each point is timed twice: launched call by call from Python, and as a replay of a CUDA graph of
+one step (which takes the host's launch cost out; the graph re-runs the same step, so the cache
+length stays fixed while it is timed).  All computing layers are loaded with the same seeded K/V
+block: values do not affect bandwidth and parity is checked elsewhere.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import sys
+
+import torch
+
+import synth_inputs as si
+from paper_2410_18517_b200 import SharedKVCache
+
+HBM_BYTES_USABLE = 170 * 2**30      # leave head-room below the 180 GB of a B200
+
+
+def pool_bytes(w: si.Workload, extra_rows: int) -> int:
+    rs = (w.context + extra_rows + 127) // 128 * 128
+    return (w.L - w.n_shared) * 2 * w.B * w.Hkv * rs * w.D * w.elem_bytes
+
+
+def time_point(w: si.Workload, steps: int, device=0) -> dict:
+    extra = 2 * steps + 16
+    rec = {"workload": w.name, "batch": w.B, "context": w.context, "shared_layers": w.n_shared,
+           "pool_bytes": pool_bytes(w, extra), "pool_bytes_unshared": pool_bytes(w.scaled(n_shared=0), extra)}
+    if rec["pool_bytes"] > HBM_BYTES_USABLE:
+        rec["fits"] = False
+        return rec
+    rec["fits"] = True
+    sm = w.share_map()
+    rec["share_map"] = [int(x) for x in sm]
+    dev = torch.device("cuda", device)
+    cache = SharedKVCache(w.L, w.Hq, w.Hkv, w.D, w.B, w.context + extra, w.dtype, share_map=sm, device=device)
+    k, v = si.context_kv(w, 0, device=dev)
+    for l in range(w.L):
+        if sm[l] == l:
+            cache.append(l, k, v)
+    del k, v
+    ins = [si.step_qkv(w, 0, l, device=dev) for l in range(w.L)]
+    outs = [torch.empty(w.B, w.Hq, w.D, dtype=torch.float32, device=dev) for _ in range(w.L)]
+
+    def one_step():
+        for l in range(w.L):
+            q, kk, vv = ins[l]
+            if sm[l] == l:
+                cache.append(l, kk, vv)
+            cache.decode_attention(l, q, outs[l])
+
+    def timed(fn, n):
+        torch.cuda.synchronize(dev)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(n):
+            fn()
+        e1.record()
+        torch.cuda.synchronize(dev)
+        return e0.elapsed_time(e1) / n
+
+    for _ in range(3):
+        one_step()
+    b0 = cache.stats()["kv_bytes_read"]
+    ms = timed(one_step, steps)
+    read_per_step = (cache.stats()["kv_bytes_read"] - b0) / steps
+    rec.update(ms_per_step=ms, tokens_per_s=w.B / (ms * 1e-3), kv_read_gbs=read_per_step / (ms * 1e-3) / 1e9,
+               kv_bytes_read_per_step=read_per_step, kernel=cache.last_launch()["kernel"],
+               ctas=cache.last_launch()["ctas"])
+
+    # graph replay of one step
+    side = torch.cuda.Stream(device=dev)
+    side.wait_stream(torch.cuda.current_stream(dev))
+    with torch.cuda.stream(side):
+        one_step()
+        graph = torch.cuda.CUDAGraph()
+        b0 = cache.stats()["kv_bytes_read"]
+        with torch.cuda.graph(graph, stream=side):
+            one_step()
+        read_graph = cache.stats()["kv_bytes_read"] - b0
+    torch.cuda.current_stream(dev).wait_stream(side)
+    graph.replay()
+    ms_g = timed(graph.replay, steps)
+    rec.update(graph_ms_per_step=ms_g, graph_tokens_per_s=w.B / (ms_g * 1e-3),
+               graph_kv_read_gbs=read_graph / (ms_g * 1e-3) / 1e9, device_status=cache.device_status())
+    cache.close()
+    del cache, ins, outs, graph
+    torch.cuda.empty_cache()
+    return rec
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--out", default=None)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--only", default=None, help="B,N,P of a single point")
+    args = ap.parse_args()
+    pts = si.sweep_points()
+    if args.only:
+        B, N, P = (int(x) for x in args.only.split(","))
+        pts = [p for p in pts if (p.B, p.context, p.n_shared) == (B, N, P)]
+    f = open(args.out, "w") if args.out else None
+    for w in pts:
+        rec = time_point(w, args.steps)
+        line = json.dumps(rec)
+        print(line, flush=True)
+        if f:
+            f.write(line + "\n")
+            f.flush()
+    if f:
+        f.close()
+
+
+if __name__ == "__main__":
+    sys.exit(main())
