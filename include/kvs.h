@@ -83,7 +83,12 @@ typedef struct {
 /* Tuning knobs for kvs_set_option.  Defaults are chosen by the library. */
 typedef enum {
     KVS_OPT_MAX_CTAS = 0,   /* upper bound on thread blocks of the split-K kernel; 0 = auto  */
-    KVS_OPT_KERNEL = 1      /* 0 = auto, 1 = scalar-FMA path, 2 = grouped tensor-core path   */
+    KVS_OPT_KERNEL = 1,     /* 0 = auto, 1 = scalar-FMA path, 2 = grouped tensor-core path   */
+    KVS_OPT_EARLY_START = 2 /* 1 (default): kernels are launched so that they may start while
+                               the previous kernel on the stream drains, and prefetch K/V rows
+                               that nothing in flight writes; they wait for the previous kernel
+                               before reading q, newly appended rows, or writing anything.
+                               0: plain stream-ordered launches.  Results are identical.      */
 } kvs_option;
 
 /* ---- life cycle ------------------------------------------------------------ */

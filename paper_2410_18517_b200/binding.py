@@ -28,6 +28,7 @@ KVS_F32 = 1
 
 KVS_OPT_MAX_CTAS = 0
 KVS_OPT_KERNEL = 1
+KVS_OPT_EARLY_START = 2
 
 # every symbol include/kvs.h declares
 EXPORTS = (

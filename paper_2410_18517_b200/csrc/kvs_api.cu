@@ -44,8 +44,18 @@ struct kvs_ctx {
     alignas(64) unsigned char tensor_map[128];  // TMA view of the pool (bf16 storage only)
     bool have_tensor_map = false;
 
+    // Launch bookkeeping for early-start (programmatic) launches.  Every kernel of this context
+    // gets a sequence number.  A split-K kernel lets its successor start only after its own
+    // wait, so when any later kernel runs, everything before the latest split-K kernel is
+    // complete; appends newer than that may still be in flight.
+    uint64_t seq = 0;
+    uint64_t last_splitk_seq = 0;
+    std::vector<uint64_t> app_seq_latest, app_seq_prev;   // per slot, 0 = none
+    std::vector<int32_t> app_start_latest;                // first row the latest append wrote
+
     int opt_max_ctas = 0;
     int opt_kernel = 0;
+    int opt_pdl = 1;
     kvs::DecodePlan last_plan{};
     kvs_stats_t stats{};
 };
@@ -70,6 +80,17 @@ void resolve_map(kvs_ctx* c) {
     c->n_slots = n;
     c->slot_len.assign(n, 0);
     c->cur_batch = 0;
+    c->app_seq_latest.assign(n, 0);
+    c->app_seq_prev.assign(n, 0);
+    c->app_start_latest.assign(n, 0);
+}
+
+// Rows of `slot` that no kernel possibly still in flight writes (see kvs_ctx::seq).
+int safe_rows_of(const kvs_ctx* c, int slot) {
+    const uint64_t complete_upto = c->last_splitk_seq ? c->last_splitk_seq - 1 : 0;
+    if (c->app_seq_latest[slot] <= complete_upto) return c->slot_len[slot];
+    if (c->app_seq_prev[slot] <= complete_upto) return c->app_start_latest[slot];
+    return 0;
 }
 
 void layout_workspace(kvs_ctx* c) {
@@ -152,8 +173,12 @@ kvs_status do_append(kvs_ctx* c, int layer, const void* k, const void* v, int ba
     char* kp = c->pool + (size_t)(2 * slot) * c->plane_bytes;
     char* vp = kp + c->plane_bytes;
     if (kvs::launch_append(k, v, kp, vp, batch, n_new, c->cfg.n_kv_heads, c->row_bytes, c->row_stride,
-                           c->slot_len[slot], st) != cudaSuccess)
+                           c->slot_len[slot], c->opt_pdl != 0, st) != cudaSuccess)
         return KVS_ERR_CUDA;
+    c->seq += 1;
+    c->app_seq_prev[slot] = c->app_seq_latest[slot];
+    c->app_seq_latest[slot] = c->seq;
+    c->app_start_latest[slot] = c->slot_len[slot];
     c->slot_len[slot] += n_new;
     c->cur_batch = batch;
     c->stats.append_launches += 1;
@@ -178,6 +203,10 @@ kvs_status do_attention(kvs_ctx* c, int layer, const void* q, float* out, int ba
     a.D = c->cfg.head_dim;
     a.dtype = c->cfg.dtype;
     a.scale_log2 = c->scale * 1.4426950408889634f;
+    a.programmatic = c->opt_pdl != 0;
+    a.safe_rows = safe_rows_of(c, slot);
+    c->seq += 2;                       // split-K kernel, then combine
+    c->last_splitk_seq = c->seq - 1;
     kvs::DecodePlan plan;
     // bf16 groups of 4 or more q-heads per kv-head are a real (if thin) contraction: tensor cores.
     const bool use_mma = c->have_tensor_map && (c->opt_kernel == 2 || (c->opt_kernel == 0 && c->G >= 4));
@@ -292,6 +321,10 @@ kvs_status kvs_bind_memory(kvs_ctx* ctx, void* pool, size_t pool_bytes, void* wo
     ctx->bound = true;
     for (auto& x : ctx->slot_len) x = 0;
     ctx->cur_batch = 0;
+    // the device was idle a moment ago: nothing of this context is in flight
+    for (auto& x : ctx->app_seq_latest) x = 0;
+    for (auto& x : ctx->app_seq_prev) x = 0;
+    ctx->last_splitk_seq = 0;
     return KVS_OK;
 }
 
@@ -432,6 +465,10 @@ kvs_status kvs_set_option(kvs_ctx* ctx, int32_t option, int32_t value) {
             if (value < 0 || value > kvs::kMaxCtas) return KVS_ERR_INVALID_ARG;
             ctx->opt_max_ctas = value;
             return KVS_OK;
+        case KVS_OPT_EARLY_START:
+            if (value != 0 && value != 1) return KVS_ERR_INVALID_ARG;
+            ctx->opt_pdl = value;
+            return KVS_OK;
         case KVS_OPT_KERNEL:
             if (value < 0 || value > 2) return KVS_ERR_INVALID_ARG;
             if (value == 2 && ctx->cfg.dtype != KVS_BF16) return KVS_ERR_INVALID_ARG;  // tensor-core path is bf16 only
@@ -556,6 +593,10 @@ kvs_status kvs_decode_attention_static(kvs_ctx* ctx, int32_t layer, const void* 
     a.D = D;
     a.dtype = c->cfg.dtype;
     a.scale_log2 = c->scale * 1.4426950408889634f;
+    a.programmatic = false;            // plain launches: starts after everything before it on the stream
+    a.safe_rows = 0;
+    c->seq += 2;
+    c->last_splitk_seq = c->seq - 1;
     if (use_mma) {
         const long long plane_rows = (long long)c->cfg.max_batch * c->cfg.n_kv_heads * c->row_stride;
         if (kvs::launch_decode_mma(a, plan, c->tensor_map, plane_rows * (2 * slot), plane_rows * (2 * slot + 1), st) !=

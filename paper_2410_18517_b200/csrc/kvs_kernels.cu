@@ -18,6 +18,8 @@ __global__ void __launch_bounds__(256) kv_append_kernel(const uint4* __restrict_
                                                         uint4* __restrict__ kplane, uint4* __restrict__ vplane,
                                                         long long total_vecs, int n_new, int Hkv, int row_vecs,
                                                         int row_stride, int len0) {
+    pdl_launch_dependents();
+    pdl_wait();
     const uint4* __restrict__ src = blockIdx.y == 0 ? k : v;
     uint4* __restrict__ dst = blockIdx.y == 0 ? kplane : vplane;
     for (long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x; idx < total_vecs;
@@ -34,14 +36,13 @@ __global__ void __launch_bounds__(256) kv_append_kernel(const uint4* __restrict_
 }
 
 cudaError_t launch_append(const void* k, const void* v, void* kplane, void* vplane, int B, int n_new, int Hkv,
-                          int row_bytes, int row_stride, int len0, cudaStream_t stream) {
+                          int row_bytes, int row_stride, int len0, bool programmatic, cudaStream_t stream) {
     const int row_vecs = row_bytes / 16;
     const long long total = (long long)B * n_new * Hkv * row_vecs;
     const long long blocks = std::min<long long>((total + 255) / 256, 148 * 16);
     dim3 grid((unsigned)blocks, 2);
-    kv_append_kernel<<<grid, 256, 0, stream>>>((const uint4*)k, (const uint4*)v, (uint4*)kplane, (uint4*)vplane, total,
-                                               n_new, Hkv, row_vecs, row_stride, len0);
-    return cudaGetLastError();
+    return launch_kernel(kv_append_kernel, grid, dim3(256), 0, stream, programmatic, (const uint4*)k, (const uint4*)v,
+                         (uint4*)kplane, (uint4*)vplane, total, n_new, Hkv, row_vecs, row_stride, len0);
 }
 
 // --------------------------------------------------------------------------------------
@@ -139,6 +140,7 @@ struct ScalarKernelArgs {
     int tpu;
     long long T;
     float scale_log2;
+    int safe_rows;  // rows of every unit that no kernel possibly still running writes
 };
 
 template <typename T, int D, int G>
@@ -176,12 +178,10 @@ __global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G>::MIN_BLOC
     if (warp == kConsumerWarps) {
         // ------------------------------ producer ------------------------------
         if (lane == 0) {
-            int it = 0;
-            bool ok = true;
-            for (long long gt = t0; gt < t1 && ok; ++gt, ++it) {
-                const int st = it % STAGES;
-                if (it >= STAGES) ok = mbar_wait_bounded(&empty_bar[st], ((it / STAGES) - 1) & 1, abort_flag, a.status);
-                if (!ok) break;
+            // Issue the copies of tile `gt` into stage `st`.  kv / qpart select which of the
+            // stage's copies are issued now; the barrier is armed with the stage's full byte
+            // count by whichever call comes first (arm = true).
+            auto issue = [&](long long gt, int st, bool arm, bool kv, bool qpart) {
                 const long long u = gt / a.tpu;
                 const int ti = (int)(gt - u * a.tpu);
                 const int row0 = ti * TN;
@@ -189,11 +189,35 @@ __global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G>::MIN_BLOC
                 const uint32_t bytes = (uint32_t)rows * RB;
                 const bool with_q = (gt == t0) || (ti == 0);
                 unsigned char* sb = stage_base + st * S::STAGE_BYTES;
-                mbar_arrive_expect_tx(&full_bar[st], 2 * bytes + (with_q ? S::QBYTES : 0));
-                const long long off = (u * a.row_stride + row0) * (long long)RB;
-                bulk_g2s(sb, a.kplane + off, bytes, &full_bar[st]);
-                bulk_g2s(sb + kTileBytes, a.vplane + off, bytes, &full_bar[st]);
-                if (with_q) bulk_g2s(sb + 2 * kTileBytes, a.q + u * (long long)S::QBYTES, S::QBYTES, &full_bar[st]);
+                if (arm) mbar_arrive_expect_tx(&full_bar[st], 2 * bytes + (with_q ? S::QBYTES : 0));
+                if (kv) {
+                    const long long off = (u * a.row_stride + row0) * (long long)RB;
+                    bulk_g2s(sb, a.kplane + off, bytes, &full_bar[st]);
+                    bulk_g2s(sb + kTileBytes, a.vplane + off, bytes, &full_bar[st]);
+                }
+                if (qpart && with_q)
+                    bulk_g2s(sb + 2 * kTileBytes, a.q + u * (long long)S::QBYTES, S::QBYTES, &full_bar[st]);
+            };
+            // Before the preceding kernel in the stream is known to have finished, only K/V
+            // tiles made entirely of rows that no kernel still in flight can be writing are
+            // fetched (rows below safe_rows); q and everything else come after the wait.
+            int npre = 0;
+            for (; npre < STAGES && t0 + npre < t1; ++npre) {
+                const long long gt = t0 + npre;
+                const int ti = (int)(gt % a.tpu);
+                if ((long long)(ti + 1) * TN > a.safe_rows) break;
+                issue(gt, npre, true, true, false);
+            }
+            pdl_wait();
+            pdl_launch_dependents();
+            for (int j = 0; j < npre; ++j) issue(t0 + j, j, false, false, true);
+            int it = npre;
+            bool ok = true;
+            for (long long gt = t0 + npre; gt < t1 && ok; ++gt, ++it) {
+                const int st = it % STAGES;
+                if (it >= STAGES) ok = mbar_wait_bounded(&empty_bar[st], ((it / STAGES) - 1) & 1, abort_flag, a.status);
+                if (!ok) break;
+                issue(gt, st, true, true, true);
             }
             if (!ok) {
                 // Gave up: still wait (bounded) for copies already issued, so that none
@@ -206,6 +230,8 @@ __global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G>::MIN_BLOC
     }
 
     // ---------------------------------- consumers ----------------------------------
+    pdl_wait();               // partial results of the previous call may still be read until here
+    pdl_launch_dependents();
     const int lig = lane & (LPR - 1);                 // lane within its row group
     const int grp = warp * S::GPW + lane / LPR;       // row group within the block
     const int my_i = lig >> SH;                       // row (of the R) whose score this lane ends up holding
@@ -344,6 +370,8 @@ __global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G>::MIN_BLOC
 // --------------------------------------------------------------------------------------
 __global__ void decode_combine_kernel(const float* __restrict__ part_o, const float* __restrict__ part_ml,
                                       float* __restrict__ out, int G, int D, int tpu, long long T, int NC) {
+    pdl_launch_dependents();
+    pdl_wait();
     const long long u = blockIdx.x / G;
     const int g = blockIdx.x % G;
     const int c0 = cta_of_tile(u * tpu, T, NC);
@@ -363,9 +391,8 @@ __global__ void decode_combine_kernel(const float* __restrict__ part_o, const fl
 }
 
 cudaError_t launch_combine(const DecodeArgs& a, const DecodePlan& plan, cudaStream_t stream) {
-    decode_combine_kernel<<<a.units * a.G, a.D, 0, stream>>>(a.part_o, a.part_ml, a.out, a.G, a.D, plan.tpu, plan.T,
-                                                            plan.NC);
-    return cudaGetLastError();
+    return launch_kernel(decode_combine_kernel, dim3(a.units * a.G), dim3(a.D), 0, stream, a.programmatic,
+                         (const float*)a.part_o, (const float*)a.part_ml, a.out, a.G, a.D, plan.tpu, plan.T, plan.NC);
 }
 
 // --------------------------------------------------------------------------------------
@@ -387,18 +414,18 @@ static cudaError_t set_attr_groups() {
 }
 
 template <typename T, int D, int G>
-static cudaError_t launch_scalar_one(const ScalarKernelArgs& ka, int NC, cudaStream_t stream) {
-    decode_splitk_scalar<T, D, G><<<NC, kScalarThreads, ScalarShape<T, D, G>::SMEM_BYTES, stream>>>(ka);
-    return cudaGetLastError();
+static cudaError_t launch_scalar_one(const ScalarKernelArgs& ka, int NC, bool programmatic, cudaStream_t stream) {
+    return launch_kernel(decode_splitk_scalar<T, D, G>, dim3(NC), dim3(kScalarThreads),
+                         ScalarShape<T, D, G>::SMEM_BYTES, stream, programmatic, ka);
 }
 
 template <typename T, int D>
-static cudaError_t launch_scalar_groups(int G, const ScalarKernelArgs& ka, int NC, cudaStream_t stream) {
+static cudaError_t launch_scalar_groups(int G, const ScalarKernelArgs& ka, int NC, bool pdl, cudaStream_t stream) {
     switch (G) {
-        case 1: return launch_scalar_one<T, D, 1>(ka, NC, stream);
-        case 2: return launch_scalar_one<T, D, 2>(ka, NC, stream);
-        case 4: return launch_scalar_one<T, D, 4>(ka, NC, stream);
-        case 8: return launch_scalar_one<T, D, 8>(ka, NC, stream);
+        case 1: return launch_scalar_one<T, D, 1>(ka, NC, pdl, stream);
+        case 2: return launch_scalar_one<T, D, 2>(ka, NC, pdl, stream);
+        case 4: return launch_scalar_one<T, D, 4>(ka, NC, pdl, stream);
+        case 8: return launch_scalar_one<T, D, 8>(ka, NC, pdl, stream);
         default: return cudaErrorInvalidValue;
     }
 }
@@ -429,12 +456,14 @@ cudaError_t launch_decode_scalar(const DecodeArgs& a, const DecodePlan& plan, cu
     ka.tpu = plan.tpu;
     ka.T = plan.T;
     ka.scale_log2 = a.scale_log2;
+    ka.safe_rows = a.programmatic ? a.safe_rows : 0;
+    const bool pdl = a.programmatic;
     if (a.dtype == 0) {
-        if (a.D == 128) return launch_scalar_groups<__nv_bfloat16, 128>(a.G, ka, plan.NC, stream);
-        if (a.D == 64) return launch_scalar_groups<__nv_bfloat16, 64>(a.G, ka, plan.NC, stream);
+        if (a.D == 128) return launch_scalar_groups<__nv_bfloat16, 128>(a.G, ka, plan.NC, pdl, stream);
+        if (a.D == 64) return launch_scalar_groups<__nv_bfloat16, 64>(a.G, ka, plan.NC, pdl, stream);
     } else {
-        if (a.D == 128) return launch_scalar_groups<float, 128>(a.G, ka, plan.NC, stream);
-        if (a.D == 64) return launch_scalar_groups<float, 64>(a.G, ka, plan.NC, stream);
+        if (a.D == 128) return launch_scalar_groups<float, 128>(a.G, ka, plan.NC, pdl, stream);
+        if (a.D == 64) return launch_scalar_groups<float, 64>(a.G, ka, plan.NC, pdl, stream);
     }
     return cudaErrorInvalidValue;
 }

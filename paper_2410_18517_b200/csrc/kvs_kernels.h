@@ -35,6 +35,8 @@ struct DecodeArgs {
     int D;
     int dtype;            // 0 bf16, 1 f32
     float scale_log2;     // softmax scale * log2(e)
+    int safe_rows;        // rows per unit that no kernel possibly still in flight is writing
+    bool programmatic;    // launch with programmatic stream serialization (early start, explicit wait)
 };
 
 // Largest number of thread blocks any plan may use (sizes the partial buffers).
@@ -60,7 +62,7 @@ cudaError_t launch_decode_mma(const DecodeArgs& a, const DecodePlan& plan, const
                               long long vrow0, cudaStream_t stream);
 
 cudaError_t launch_append(const void* k, const void* v, void* kplane, void* vplane, int B, int n_new, int Hkv,
-                          int row_bytes, int row_stride, int len0, cudaStream_t stream);
+                          int row_bytes, int row_stride, int len0, bool programmatic, cudaStream_t stream);
 cudaError_t launch_decode_scalar(const DecodeArgs& a, const DecodePlan& plan, cudaStream_t stream);
 cudaError_t launch_combine(const DecodeArgs& a, const DecodePlan& plan, cudaStream_t stream);
 cudaError_t launch_read_roof(const void* src, size_t bytes, unsigned long long* checksum, int sm_count,

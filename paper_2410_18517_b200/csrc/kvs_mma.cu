@@ -88,6 +88,7 @@ struct MmaKernelArgs {
     long long krow0;  // first row of the K plane within the pool-wide row index
     long long vrow0;
     float scale_log2;
+    int safe_rows;  // rows of every unit that no kernel possibly still running writes
 };
 
 template <int D, int G>
@@ -124,25 +125,46 @@ __global__ void __launch_bounds__(kMmaThreads, 2)
     if (warp == kMmaWarps) {
         // ------------------------------ producer ------------------------------
         if (lane == 0) {
-            int it = 0;
-            bool ok = true;
-            for (long long gt = t0; gt < t1; ++gt, ++it) {
-                const int st = it % kMmaStages;
-                if (it >= kMmaStages)
-                    ok = mbar_wait_bounded(&empty_bar[st], ((it / kMmaStages) - 1) & 1, abort_flag, a.status);
-                if (!ok) break;
+            // Issue the copies of tile `gt` into stage `st` (see the scalar kernel: the barrier
+            // is armed once with the stage's full byte count, K/V and q may be issued apart).
+            auto issue = [&](long long gt, int st, bool arm, bool kv, bool qpart) {
                 const long long u = gt / a.tpu;
                 const int ti = (int)(gt - u * a.tpu);
                 const bool with_q = (gt == t0) || (ti == 0);
                 unsigned char* sb = smem + st * S::STAGE_BYTES;
-                mbar_arrive_expect_tx(&full_bar[st], 2 * kMmaTileBytes + (with_q ? QBYTES : 0));
-                const long long row = u * a.row_stride + (long long)ti * TN;
+                if (arm) mbar_arrive_expect_tx(&full_bar[st], 2 * kMmaTileBytes + (with_q ? QBYTES : 0));
+                if (kv) {
+                    const long long row = u * a.row_stride + (long long)ti * TN;
 #pragma unroll
-                for (int h = 0; h < S::HALVES; ++h) {
-                    tma_load_2d(sb + h * (TN * 128), &tmap, h * 64, (int)(a.krow0 + row), &full_bar[st]);
-                    tma_load_2d(sb + kMmaTileBytes + h * (TN * 128), &tmap, h * 64, (int)(a.vrow0 + row), &full_bar[st]);
+                    for (int h = 0; h < S::HALVES; ++h) {
+                        tma_load_2d(sb + h * (TN * 128), &tmap, h * 64, (int)(a.krow0 + row), &full_bar[st]);
+                        tma_load_2d(sb + kMmaTileBytes + h * (TN * 128), &tmap, h * 64, (int)(a.vrow0 + row),
+                                    &full_bar[st]);
+                    }
                 }
-                if (with_q) bulk_g2s(sb + 2 * kMmaTileBytes, a.q + u * (long long)QBYTES, QBYTES, &full_bar[st]);
+                if (qpart && with_q)
+                    bulk_g2s(sb + 2 * kMmaTileBytes, a.q + u * (long long)QBYTES, QBYTES, &full_bar[st]);
+            };
+            // Until the preceding kernel in the stream is known to have finished, fetch only
+            // K/V tiles made entirely of rows that no kernel still in flight can be writing.
+            int npre = 0;
+            for (; npre < kMmaStages && t0 + npre < t1; ++npre) {
+                const long long gt = t0 + npre;
+                const int ti = (int)(gt % a.tpu);
+                if ((long long)(ti + 1) * TN > a.safe_rows) break;
+                issue(gt, npre, true, true, false);
+            }
+            pdl_wait();
+            pdl_launch_dependents();
+            for (int j = 0; j < npre; ++j) issue(t0 + j, j, false, false, true);
+            int it = npre;
+            bool ok = true;
+            for (long long gt = t0 + npre; gt < t1; ++gt, ++it) {
+                const int st = it % kMmaStages;
+                if (it >= kMmaStages)
+                    ok = mbar_wait_bounded(&empty_bar[st], ((it / kMmaStages) - 1) & 1, abort_flag, a.status);
+                if (!ok) break;
+                issue(gt, st, true, true, true);
             }
             if (!ok) {
                 for (int j = max(0, it - kMmaStages); j < it; ++j)
@@ -153,6 +175,8 @@ __global__ void __launch_bounds__(kMmaThreads, 2)
     }
 
     // ---------------------------------- consumers ----------------------------------
+    pdl_wait();               // partial results of the previous call may still be read until here
+    pdl_launch_dependents();
     const int row = lane >> 2;   // q-head row of the accumulator fragment (rows 8..15 are padding)
     const int quad = lane & 3;
 
@@ -314,18 +338,18 @@ cudaError_t set_attr() {
 }
 
 template <int D, int G>
-cudaError_t launch_one(const CUtensorMap& tm, const MmaKernelArgs& ka, int NC, cudaStream_t stream) {
-    decode_splitk_mma<D, G><<<NC, kMmaThreads, MmaShape<D>::SMEM_BYTES, stream>>>(tm, ka);
-    return cudaGetLastError();
+cudaError_t launch_one(const CUtensorMap& tm, const MmaKernelArgs& ka, int NC, bool pdl, cudaStream_t stream) {
+    return launch_kernel(decode_splitk_mma<D, G>, dim3(NC), dim3(kMmaThreads), MmaShape<D>::SMEM_BYTES, stream, pdl, tm,
+                         ka);
 }
 
 template <int D>
-cudaError_t launch_groups(int G, const CUtensorMap& tm, const MmaKernelArgs& ka, int NC, cudaStream_t stream) {
+cudaError_t launch_groups(int G, const CUtensorMap& tm, const MmaKernelArgs& ka, int NC, bool pdl, cudaStream_t stream) {
     switch (G) {
-        case 1: return launch_one<D, 1>(tm, ka, NC, stream);
-        case 2: return launch_one<D, 2>(tm, ka, NC, stream);
-        case 4: return launch_one<D, 4>(tm, ka, NC, stream);
-        case 8: return launch_one<D, 8>(tm, ka, NC, stream);
+        case 1: return launch_one<D, 1>(tm, ka, NC, pdl, stream);
+        case 2: return launch_one<D, 2>(tm, ka, NC, pdl, stream);
+        case 4: return launch_one<D, 4>(tm, ka, NC, pdl, stream);
+        case 8: return launch_one<D, 8>(tm, ka, NC, pdl, stream);
         default: return cudaErrorInvalidValue;
     }
 }
@@ -392,9 +416,10 @@ cudaError_t launch_decode_mma(const DecodeArgs& a, const DecodePlan& plan, const
     ka.krow0 = krow0;
     ka.vrow0 = vrow0;
     ka.scale_log2 = a.scale_log2;
+    ka.safe_rows = a.programmatic ? a.safe_rows : 0;
     const CUtensorMap& tm = *reinterpret_cast<const CUtensorMap*>(tensor_map);
-    if (a.D == 128) return launch_groups<128>(a.G, tm, ka, plan.NC, stream);
-    if (a.D == 64) return launch_groups<64>(a.G, tm, ka, plan.NC, stream);
+    if (a.D == 128) return launch_groups<128>(a.G, tm, ka, plan.NC, a.programmatic, stream);
+    if (a.D == 64) return launch_groups<64>(a.G, tm, ka, plan.NC, a.programmatic, stream);
     return cudaErrorInvalidValue;
 }
 

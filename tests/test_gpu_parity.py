@@ -9,7 +9,7 @@ import torch
 
 import oracle
 import synth_inputs as si
-from paper_2410_18517_b200 import KVS_OPT_KERNEL, KVS_OPT_MAX_CTAS, KvsError, SharedKVCache
+from paper_2410_18517_b200 import KVS_OPT_EARLY_START, KVS_OPT_KERNEL, KVS_OPT_MAX_CTAS, KvsError, SharedKVCache
 from paper_2410_18517_b200 import binding as kb
 from paper_2410_18517_b200 import build as kbuild
 
@@ -105,6 +105,20 @@ def test_any_split_of_the_tile_line_gives_the_same_answer(max_ctas):
     cache, _, _ = run_small(w, steps=2, options=[(KVS_OPT_MAX_CTAS, max_ctas)])
     if max_ctas:
         assert cache.last_launch()["ctas"] == max_ctas
+
+
+@pytest.mark.parametrize("early", [0, 1])
+@pytest.mark.parametrize("Hq,Hkv", [(4, 4), (8, 2)])
+def test_early_start_launches_change_nothing(early, Hq, Hkv):
+    """Kernels that may start while their predecessor drains (and prefetch rows nothing in flight
+    writes) against plain stream-ordered launches: same bits, and both match the oracle.  The
+    context is appended immediately before the first step, 12 steps follow back to back."""
+    w = si.Workload(f"early_{Hq}_{Hkv}", L=4, Hq=Hq, Hkv=Hkv, D=128, B=2, context=900, dtype="bf16", n_shared=2,
+                    map_seed=0, steps=12, fixed_map=(0, 0, 2, 2))
+    cache, _, _ = run_small(w, steps=12, options=[(KVS_OPT_EARLY_START, early)])
+    ref_cache, _, _ = run_small(w, steps=12, options=[(KVS_OPT_EARLY_START, 0)], check_cache=False)
+    q = si.step_qkv(w, 99, 1, device="cuda")[0]
+    assert torch.equal(cache.decode_attention(1, q), ref_cache.decode_attention(1, q))
 
 
 def test_many_small_units_per_block():
