@@ -169,8 +169,11 @@ kvs_status kvs_decode_attention(kvs_ctx* ctx, int32_t layer, const void* q, floa
  *   k_host, v_host: host, [n_layers][batch][1][n_kv_heads][head_dim], storage type
  *             (entries of sharing layers are not copied to the device)
  *   out_host: host, [n_layers][batch][n_q_heads][head_dim], float32
- * Copies inputs host->device into the workspace staging area, runs the layers,
- * copies the result device->host, all on `stream`, and waits for the stream.
+ * Copies inputs host->device into the workspace staging area, runs the layers on
+ * `stream`, copies the result device->host, and waits until all of it is done.  The
+ * copies run on a second stream owned by the context (created at the first call,
+ * together with a few events) in four chunks of layers, so that they overlap the
+ * layers of the neighbouring chunks.
  * Pinned host memory makes the copies asynchronous; pageable memory also works.
  * h2d_bytes / d2h_bytes (host, may be NULL) receive the bytes copied.
  * Errors: as kvs_append / kvs_decode_attention; nothing is launched on an error

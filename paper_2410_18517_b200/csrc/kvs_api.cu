@@ -53,6 +53,12 @@ struct kvs_ctx {
     std::vector<uint64_t> app_seq_latest, app_seq_prev;   // per slot, 0 = none
     std::vector<int32_t> app_start_latest;                // first row the latest append wrote
 
+    // kvs_step_host: second stream and events that overlap the host copies with the layers
+    static constexpr int kChunks = 4;
+    bool copy_ready = false;
+    cudaStream_t copy_stream = nullptr;
+    cudaEvent_t ev_in[kChunks] = {}, ev_done[kChunks] = {}, ev_start = nullptr;
+
     int opt_max_ctas = 0;
     int opt_kernel = 0;
     int opt_pdl = 1;
@@ -264,6 +270,17 @@ kvs_status kvs_create(const kvs_config* cfg, kvs_ctx** out) {
 
 kvs_status kvs_destroy(kvs_ctx* ctx) {
     if (!ctx) return KVS_ERR_INVALID_ARG;
+    if (ctx->copy_ready) {
+        DeviceGuard guard(ctx->cfg.device);
+        if (guard.ok) {
+            for (int i = 0; i < kvs_ctx::kChunks; ++i) {
+                cudaEventDestroy(ctx->ev_in[i]);
+                cudaEventDestroy(ctx->ev_done[i]);
+            }
+            cudaEventDestroy(ctx->ev_start);
+            cudaStreamDestroy(ctx->copy_stream);
+        }
+    }
     delete ctx;
     return KVS_OK;
 }
@@ -378,33 +395,65 @@ kvs_status kvs_step_host(kvs_ctx* ctx, const void* q_host, const void* k_host, c
     char* dv = ctx->ws + ctx->off_stage_v;
     char* dout = ctx->ws + ctx->off_stage_out;
     uint64_t h2d = 0;
-    if (cudaMemcpyAsync(dq, q_host, q_layer * f.n_layers, cudaMemcpyHostToDevice, st) != cudaSuccess) return KVS_ERR_CUDA;
-    h2d += q_layer * f.n_layers;
-    // K/V of own-cache layers only; consecutive own-cache layers go in one copy
-    for (int l = 0; l < f.n_layers;) {
-        if (ctx->share_map[l] != l) { ++l; continue; }
-        int e = l;
-        while (e + 1 < f.n_layers && ctx->share_map[e + 1] == e + 1) ++e;
-        const size_t off = kv_layer * l, len = kv_layer * (e - l + 1);
-        if (cudaMemcpyAsync(dk + off, (const char*)k_host + off, len, cudaMemcpyHostToDevice, st) != cudaSuccess ||
-            cudaMemcpyAsync(dv + off, (const char*)v_host + off, len, cudaMemcpyHostToDevice, st) != cudaSuccess)
-            return KVS_ERR_CUDA;
-        h2d += 2 * len;
-        l = e + 1;
+    // The layers are cut into a few chunks; a second stream copies chunk c+1's inputs in and
+    // chunk c-1's outputs out while chunk c computes, so only the first input copy and the last
+    // output copy are exposed.
+    if (!ctx->copy_ready) {
+        if (cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking) != cudaSuccess) return KVS_ERR_CUDA;
+        for (int i = 0; i < kvs_ctx::kChunks; ++i)
+            if (cudaEventCreateWithFlags(&ctx->ev_in[i], cudaEventDisableTiming) != cudaSuccess ||
+                cudaEventCreateWithFlags(&ctx->ev_done[i], cudaEventDisableTiming) != cudaSuccess)
+                return KVS_ERR_CUDA;
+        if (cudaEventCreateWithFlags(&ctx->ev_start, cudaEventDisableTiming) != cudaSuccess) return KVS_ERR_CUDA;
+        ctx->copy_ready = true;
     }
-    for (int l = 0; l < f.n_layers; ++l) {
-        if (ctx->share_map[l] == l) {
-            kvs_status s = do_append(ctx, l, dk + kv_layer * l, dv + kv_layer * l, batch, 1, st);
-            if (s != KVS_OK) return s;
-        } else {
-            ctx->stats.append_skipped += 1;
-        }
-        kvs_status s = do_attention(ctx, l, dq + q_layer * l, reinterpret_cast<float*>(dout + out_layer * l), batch, st);
-        if (s != KVS_OK) return s;
-    }
-    if (cudaMemcpyAsync(out_host, dout, out_layer * f.n_layers, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+    cudaStream_t cs = ctx->copy_stream;
+    const int L = f.n_layers;
+    const int chunks = L < kvs_ctx::kChunks ? L : kvs_ctx::kChunks;
+    // the copy stream starts after whatever the caller already queued on `st`
+    if (cudaEventRecord(ctx->ev_start, st) != cudaSuccess || cudaStreamWaitEvent(cs, ctx->ev_start, 0) != cudaSuccess)
         return KVS_ERR_CUDA;
-    if (cudaStreamSynchronize(st) != cudaSuccess) return KVS_ERR_CUDA;
+    for (int c = 0; c < chunks; ++c) {
+        const int l0 = (int)((long long)c * L / chunks), l1 = (int)((long long)(c + 1) * L / chunks);
+        if (cudaMemcpyAsync(dq + q_layer * l0, (const char*)q_host + q_layer * l0, q_layer * (l1 - l0),
+                            cudaMemcpyHostToDevice, cs) != cudaSuccess)
+            return KVS_ERR_CUDA;
+        h2d += q_layer * (l1 - l0);
+        // K/V of own-cache layers only; consecutive own-cache layers go in one copy
+        for (int l = l0; l < l1;) {
+            if (ctx->share_map[l] != l) { ++l; continue; }
+            int e = l;
+            while (e + 1 < l1 && ctx->share_map[e + 1] == e + 1) ++e;
+            const size_t off = kv_layer * l, len = kv_layer * (e - l + 1);
+            if (cudaMemcpyAsync(dk + off, (const char*)k_host + off, len, cudaMemcpyHostToDevice, cs) != cudaSuccess ||
+                cudaMemcpyAsync(dv + off, (const char*)v_host + off, len, cudaMemcpyHostToDevice, cs) != cudaSuccess)
+                return KVS_ERR_CUDA;
+            h2d += 2 * len;
+            l = e + 1;
+        }
+        if (cudaEventRecord(ctx->ev_in[c], cs) != cudaSuccess) return KVS_ERR_CUDA;
+    }
+    for (int c = 0; c < chunks; ++c) {
+        const int l0 = (int)((long long)c * L / chunks), l1 = (int)((long long)(c + 1) * L / chunks);
+        if (cudaStreamWaitEvent(st, ctx->ev_in[c], 0) != cudaSuccess) return KVS_ERR_CUDA;
+        for (int l = l0; l < l1; ++l) {
+            if (ctx->share_map[l] == l) {
+                kvs_status s = do_append(ctx, l, dk + kv_layer * l, dv + kv_layer * l, batch, 1, st);
+                if (s != KVS_OK) return s;
+            } else {
+                ctx->stats.append_skipped += 1;
+            }
+            kvs_status s =
+                do_attention(ctx, l, dq + q_layer * l, reinterpret_cast<float*>(dout + out_layer * l), batch, st);
+            if (s != KVS_OK) return s;
+        }
+        if (cudaEventRecord(ctx->ev_done[c], st) != cudaSuccess || cudaStreamWaitEvent(cs, ctx->ev_done[c], 0) != cudaSuccess)
+            return KVS_ERR_CUDA;
+        if (cudaMemcpyAsync((char*)out_host + out_layer * l0, dout + out_layer * l0, out_layer * (l1 - l0),
+                            cudaMemcpyDeviceToHost, cs) != cudaSuccess)
+            return KVS_ERR_CUDA;
+    }
+    if (cudaStreamSynchronize(cs) != cudaSuccess || cudaStreamSynchronize(st) != cudaSuccess) return KVS_ERR_CUDA;
     if (h2d_bytes) *h2d_bytes = h2d;
     if (d2h_bytes) *d2h_bytes = out_layer * f.n_layers;
     return KVS_OK;
