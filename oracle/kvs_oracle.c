@@ -201,20 +201,15 @@ static void ensure_cap(oracle_state *st, int l, int need) {
     st->cap[l] = nc;
 }
 
-/* One layer of one forward pass (Section 3.2).
+/* The cache side of one layer's turn in a forward pass (Section 3.2).
  *   layer computes its own cache : append the n_new new rows of
  *       k_new / v_new, laid out [B][n_new][Hkv][D];
  *   layer's cache is replaced    : k_new / v_new are ignored (may be NULL) and
  *       the cache of layer share_map[l], as it stands after that layer's own
- *       turn in this pass, is copied over this layer's cache;
- * then, if q != NULL ([B][Hq][D]), the unchanged attention of the layer's
- * queries over the layer's cache is written to out ([B][Hq][D]).
- * Returns 0, or -1 on a bad argument / empty cache.                          */
-int oracle_layer_forward(oracle_state *st, int l, const double *q,
-                         const double *k_new, const double *v_new, int n_new,
-                         double *out) {
-    if (!st || l < 0 || l >= st->L || n_new < 0) return -1;
-    const int D = st->D, Hkv = st->Hkv, Hq = st->Hq, B = st->B;
+ *       turn in this pass, is copied over this layer's cache.
+ * Returns 0, or -1 on a bad argument.                                          */
+static int update_cache(oracle_state *st, int l, const double *k_new, const double *v_new, int n_new) {
+    const int D = st->D, Hkv = st->Hkv, B = st->B;
     const int src = st->share_map[l];
     if (src == l) {
         if (n_new > 0) {
@@ -239,6 +234,19 @@ int oracle_layer_forward(oracle_state *st, int l, const double *q,
         }
         st->len[l] = st->len[src];
     }
+    return 0;
+}
+
+/* One layer of one generation step (Section 3.2): the cache update above, then,
+ * if q != NULL ([B][Hq][D]), the unchanged attention of the layer's one query
+ * per head over the layer's whole cache, written to out ([B][Hq][D]).
+ * Returns 0, or -1 on a bad argument / empty cache.                          */
+int oracle_layer_forward(oracle_state *st, int l, const double *q,
+                         const double *k_new, const double *v_new, int n_new,
+                         double *out) {
+    if (!st || l < 0 || l >= st->L || n_new < 0) return -1;
+    const int D = st->D, Hkv = st->Hkv, Hq = st->Hq, B = st->B;
+    if (update_cache(st, l, k_new, v_new, n_new) != 0) return -1;
     if (q) {
         if (!out || st->len[l] <= 0) return -1;
         const int G = Hq / Hkv;
@@ -252,6 +260,34 @@ int oracle_layer_forward(oracle_state *st, int l, const double *q,
                                    n, D, st->scale, out + o);
             }
     }
+    return 0;
+}
+
+/* One layer of the prefill pass (Section 3.2 applies the strategy to prefill as
+ * well as to generation): the same cache update, then n_q queries per head,
+ * q [B][n_q][Hq][D], which are the newest n_q positions of the layer's cache.
+ * The paper does not restate the mask; decoder models process a prompt with
+ * the causal one, so query i (0-based) sees rows 0 .. len - n_q + i and
+ * nothing later.  out is [B][n_q][Hq][D].  With n_q = 1 this is
+ * oracle_layer_forward.  Returns 0, or -1 on a bad argument.                  */
+int oracle_layer_prefill(oracle_state *st, int l, const double *q, int n_q,
+                         const double *k_new, const double *v_new, int n_new,
+                         double *out) {
+    if (!st || l < 0 || l >= st->L || n_new < 0 || n_q < 1 || !q || !out) return -1;
+    const int D = st->D, Hkv = st->Hkv, Hq = st->Hq, B = st->B;
+    if (update_cache(st, l, k_new, v_new, n_new) != 0) return -1;
+    const int n = st->len[l];
+    if (n_q > n) return -1;
+    const int G = Hq / Hkv;
+#pragma omp parallel for collapse(2) schedule(dynamic)
+    for (int b = 0; b < B; ++b)
+        for (int i = 0; i < n_q; ++i)
+            for (int hq = 0; hq < Hq; ++hq) {
+                int hk = hq / G;
+                size_t o = (((size_t)b * n_q + i) * Hq + hq) * D;
+                oracle_attend_unit(q + o, st->K[l][b * Hkv + hk], st->V[l][b * Hkv + hk],
+                                   n - n_q + i + 1, D, st->scale, out + o);
+            }
     return 0;
 }
 

@@ -59,6 +59,8 @@ def _load():
     lib.oracle_destroy.restype = None
     lib.oracle_layer_forward.argtypes = [ctypes.c_void_p, ctypes.c_int, _dp, _dp, _dp, ctypes.c_int, _dp]
     lib.oracle_layer_forward.restype = ctypes.c_int
+    lib.oracle_layer_prefill.argtypes = [ctypes.c_void_p, ctypes.c_int, _dp, ctypes.c_int, _dp, _dp, ctypes.c_int, _dp]
+    lib.oracle_layer_prefill.restype = ctypes.c_int
     lib.oracle_len.argtypes = [ctypes.c_void_p, ctypes.c_int]
     lib.oracle_len.restype = ctypes.c_int
     lib.oracle_get_cache.argtypes = [ctypes.c_void_p, ctypes.c_int, _dp, _dp]
@@ -181,6 +183,26 @@ class Oracle:
         rc = self._lib.oracle_layer_forward(self._h, l, qp, kp, vp, n_new, op)
         if rc != 0:
             raise RuntimeError("oracle_layer_forward rejected its arguments")
+        return out
+
+    def layer_prefill(self, l, q, k_new=None, v_new=None):
+        """One layer of the prefill pass: ``q[B][n_q][Hq][D]`` are the newest n_q positions (causal).
+
+        ``k_new``/``v_new``: ``[B][n_new][Hkv][D]`` (ignored on a sharing layer).  Returns ``out[B][n_q][Hq][D]``.
+        """
+        n_new = 0
+        kp = vp = None
+        if k_new is not None:
+            k_new, v_new = _f64(k_new), _f64(v_new)
+            assert k_new.shape == v_new.shape and k_new.shape[0] == self.B and k_new.shape[2:] == (self.Hkv, self.D)
+            n_new = k_new.shape[1]
+            kp, vp = _p(k_new), _p(v_new)
+        q = _f64(q)
+        assert q.ndim == 4 and q.shape[0] == self.B and q.shape[2:] == (self.Hq, self.D)
+        out = np.empty_like(q)
+        rc = self._lib.oracle_layer_prefill(self._h, l, _p(q), q.shape[1], kp, vp, n_new, _p(out))
+        if rc != 0:
+            raise RuntimeError("oracle_layer_prefill rejected its arguments")
         return out
 
     def step(self, q, k_new, v_new):

@@ -316,3 +316,62 @@ def test_pins_would_catch_a_transposed_group_mapping():
     got = o.layer_forward(0, q[None], K.transpose(1, 0, 2)[None], V.transpose(1, 0, 2)[None])[0]
     np.testing.assert_allclose(got, right, atol=1e-13)
     assert np.abs(got - wrong).max() > 1e-2
+
+
+# ---------------------------------------------------------------- prefill (causal, many queries)
+@pytest.mark.parametrize("Hq,Hkv,D,T", [(4, 4, 16, 33), (8, 2, 32, 17), (4, 1, 8, 64)])
+def test_prefill_identity_map_equals_torch_causal_sdpa_fp64(Hq, Hkv, D, T):
+    L, B = 2, 2
+    rng = np.random.default_rng(31)
+    o = oracle.Oracle(L, Hq, Hkv, D, B, np.arange(L))
+    G = Hq // Hkv
+    for l in range(L):
+        q = rng.standard_normal((B, T, Hq, D))
+        k = rng.standard_normal((B, T, Hkv, D))
+        v = rng.standard_normal((B, T, Hkv, D))
+        out = o.layer_prefill(l, q, k, v)
+        qt = torch.from_numpy(q).permute(0, 2, 1, 3)
+        kt = torch.from_numpy(k).permute(0, 2, 1, 3).repeat_interleave(G, dim=1)
+        vt = torch.from_numpy(v).permute(0, 2, 1, 3).repeat_interleave(G, dim=1)
+        ref = torch.nn.functional.scaled_dot_product_attention(qt, kt, vt, is_causal=True).permute(0, 2, 1, 3).numpy()
+        np.testing.assert_allclose(out, ref, rtol=0, atol=1e-12)
+
+
+@pytest.mark.parametrize("share_map", [[0, 1, 2, 1], [0, 0, 1, 2], [0, 1, 2, 3]])
+def test_prefill_chunks_with_sharing_against_brute_force(share_map):
+    """Two prompt chunks (5 rows, then 7): a query sees everything cached before its chunk plus its
+    chunk up to itself; a sharing layer uses its root layer's rows, current chunk included."""
+    L, Hq, Hkv, D, B = 4, 4, 2, 8, 2
+    rng = np.random.default_rng(hash(tuple(share_map)) % (2**32))
+    o = oracle.Oracle(L, Hq, Hkv, D, B, share_map)
+    G = Hq // Hkv
+    ks = [[rng.standard_normal((B, T, Hkv, D)) for T in (5, 7)] for _ in range(L)]
+    vs = [[rng.standard_normal((B, T, Hkv, D)) for T in (5, 7)] for _ in range(L)]
+    for c, T in enumerate((5, 7)):
+        for l in range(L):
+            q = rng.standard_normal((B, T, Hq, D))
+            out = o.layer_prefill(l, q, ks[l][c], vs[l][c])
+            r = l
+            while share_map[r] != r:
+                r = share_map[r]
+            K = np.concatenate(ks[r][: c + 1], axis=1)
+            V = np.concatenate(vs[r][: c + 1], axis=1)
+            n = K.shape[1]
+            for b in range(B):
+                for i in range(T):
+                    for hq in range(Hq):
+                        lim = n - T + i + 1
+                        ref = brute_attention(q[b, i, hq], K[b, :lim, hq // G], V[b, :lim, hq // G])
+                        np.testing.assert_allclose(out[b, i, hq], ref, atol=1e-13)
+
+
+def test_prefill_first_query_of_an_empty_cache_returns_first_value_row_and_one_query_is_decode():
+    o = oracle.Oracle(1, 2, 2, 4, 1, [0])
+    k, v, q = (RNG.standard_normal((1, 6, 2, 4)) for _ in range(3))
+    out = o.layer_prefill(0, q, k, v)
+    np.testing.assert_array_equal(out[0, 0], v[0, 0])
+    o2 = oracle.Oracle(1, 2, 2, 4, 1, [0])
+    o2.layer_forward(0, None, k[:, :5], v[:, :5])
+    np.testing.assert_array_equal(o2.layer_forward(0, q[:, 5], k[:, 5:], v[:, 5:]), out[:, 5])
+    with pytest.raises(RuntimeError):
+        o.layer_prefill(0, RNG.standard_normal((1, 7, 2, 4)))     # more queries than cached rows
