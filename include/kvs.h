@@ -78,6 +78,7 @@ typedef struct {
     uint64_t combine_launches;    /* combine kernels launched                                */
     uint64_t kv_bytes_read;       /* 2*B*Hkv*n*D*elem summed over attention calls            */
     uint64_t kv_bytes_appended;   /* 2*B*Hkv*n_new*D*elem summed over launched appends       */
+    uint64_t prefill_launches;    /* tensor-core prefill kernels launched                    */
 } kvs_stats_t;
 
 /* Tuning knobs for kvs_set_option.  Defaults are chosen by the library. */
@@ -162,6 +163,20 @@ kvs_status kvs_append(kvs_ctx* ctx, int32_t layer, const void* k, const void* v,
  * for a bad layer, NULLs, batch < 1 or batch > the batch the slot was filled for. */
 kvs_status kvs_decode_attention(kvs_ctx* ctx, int32_t layer, const void* q, float* out,
                                 int32_t batch, void* stream);
+
+/* Prefill attention of one layer (Section 3.2: the strategy is applied to the prefill pass
+ * as it is to generation).  The n_q queries per head are the newest n_q positions of the cache
+ * the layer uses (its own slot, or its source layer's), i.e. call it after kvs_append has
+ * stored those positions' K/V (on a sharing layer: after the source layer's append).  Causal
+ * mask (the paper does not restate it; this is the usual decoder mask): query i sees rows
+ * 0 .. n - n_q + i of the n cached rows.  Works for a whole prompt (n == n_q) and for a later
+ * chunk of it (n > n_q).
+ *   q:   device, [batch][n_q][n_q_heads][head_dim], storage type, 16-byte aligned
+ *   out: device, [batch][n_q][n_q_heads][head_dim], float32
+ * One tcgen05 tensor-core kernel on `stream`; bf16 storage and head_dim 128 only (other
+ * configurations: INVALID_ARG).  Other errors as kvs_decode_attention; n_q > n: INVALID_ARG. */
+kvs_status kvs_prefill_attention(kvs_ctx* ctx, int32_t layer, const void* q, float* out,
+                                 int32_t batch, int32_t n_q, void* stream);
 
 /* One whole decode step from HOST buffers: for every layer in order, append the
  * layer's new token (own-cache layers only) and run its attention.

@@ -76,6 +76,16 @@ class SharedKVCache:
         binding.kvs_decode_attention(self.ctx, layer, q, out, q.shape[0], self._stream())
         return out
 
+    def prefill_attention(self, layer, q, out=None):
+        """q: ``[batch][n_q][n_q_heads][head_dim]`` (the newest n_q positions, causal); returns float32 of that shape."""
+        torch = self._torch
+        assert q.is_contiguous() and q.dtype == self.dtype and q.ndim == 4
+        assert q.shape[2:] == (self.shape[1], self.shape[3])
+        if out is None:
+            out = torch.empty(q.shape, dtype=torch.float32, device=self.device)
+        binding.kvs_prefill_attention(self.ctx, layer, q, out, q.shape[0], q.shape[1], self._stream())
+        return out
+
     def step_host(self, q_host, k_host, v_host, out_host):
         """One decode step over all layers from host tensors (see ``kvs_step_host``)."""
         return binding.kvs_step_host(self.ctx, q_host, k_host, v_host, out_host, q_host.shape[1], self._stream())

@@ -36,7 +36,7 @@ EXPORTS = (
     "kvs_reset", "kvs_append", "kvs_decode_attention", "kvs_step_host", "kvs_num_slots",
     "kvs_slot_of_layer", "kvs_seq_len", "kvs_row_stride", "kvs_plane_offset", "kvs_stats",
     "kvs_last_device_status", "kvs_set_option", "kvs_last_launch", "kvs_status_string",
-    "kvs_read_roof", "kvs_decode_attention_static",
+    "kvs_read_roof", "kvs_decode_attention_static", "kvs_prefill_attention",
 )
 
 
@@ -53,6 +53,7 @@ class kvs_stats_t(ctypes.Structure):
         ("append_launches", ctypes.c_uint64), ("append_skipped", ctypes.c_uint64),
         ("attention_launches", ctypes.c_uint64), ("combine_launches", ctypes.c_uint64),
         ("kv_bytes_read", ctypes.c_uint64), ("kv_bytes_appended", ctypes.c_uint64),
+        ("prefill_launches", ctypes.c_uint64),
     ]
 
 
@@ -81,6 +82,7 @@ def load() -> ctypes.CDLL:
         "kvs_append": [vp, i32, vp, vp, i32, i32, vp],
         "kvs_decode_attention": [vp, i32, vp, vp, i32, vp],
         "kvs_decode_attention_static": [vp, i32, vp, vp, i32, vp, vp],
+        "kvs_prefill_attention": [vp, i32, vp, vp, i32, i32, vp],
         "kvs_step_host": [vp, vp, vp, vp, vp, i32, vp, P(ctypes.c_uint64), P(ctypes.c_uint64)],
         "kvs_num_slots": [vp, P(i32)],
         "kvs_slot_of_layer": [vp, i32, P(i32)],
@@ -166,6 +168,10 @@ def kvs_append(ctx: int, layer: int, k, v, batch: int, n_new: int, stream: int =
 
 def kvs_decode_attention(ctx: int, layer: int, q, out, batch: int, stream: int = 0) -> None:
     _check(load().kvs_decode_attention(ctx, layer, _ptr(q), _ptr(out), batch, stream), "kvs_decode_attention")
+
+
+def kvs_prefill_attention(ctx: int, layer: int, q, out, batch: int, n_q: int, stream: int = 0) -> None:
+    _check(load().kvs_prefill_attention(ctx, layer, _ptr(q), _ptr(out), batch, n_q, stream), "kvs_prefill_attention")
 
 
 def kvs_decode_attention_static(ctx: int, layer: int, q, out, batch: int, stream: int = 0, device_status=None) -> None:

@@ -130,6 +130,7 @@ cudaError_t init_device_once(int device) {
     std::call_once(g_init_flag[device], [device]() {
         g_init_err[device] = kvs::init_kernels();
         if (g_init_err[device] == cudaSuccess) g_init_err[device] = kvs::init_mma_kernels();
+        if (g_init_err[device] == cudaSuccess) g_init_err[device] = kvs::init_prefill_kernels();
     });
     return g_init_err[device];
 }
@@ -372,6 +373,34 @@ kvs_status kvs_decode_attention(kvs_ctx* ctx, int32_t layer, const void* q, floa
     DeviceGuard guard(ctx->cfg.device);
     if (!guard.ok) return KVS_ERR_CUDA;
     return do_attention(ctx, layer, q, out, batch, static_cast<cudaStream_t>(stream));
+}
+
+kvs_status kvs_prefill_attention(kvs_ctx* ctx, int32_t layer, const void* q, float* out, int32_t batch, int32_t n_q,
+                                 void* stream) {
+    if (!ctx) return KVS_ERR_INVALID_ARG;
+    if (!ctx->bound) return KVS_ERR_STATE;
+    if (layer < 0 || layer >= ctx->cfg.n_layers || !q || !out) return KVS_ERR_INVALID_ARG;
+    if (batch < 1 || batch > ctx->cfg.max_batch || n_q < 1) return KVS_ERR_INVALID_ARG;
+    if (ctx->cfg.dtype != KVS_BF16 || ctx->cfg.head_dim != 128 || !ctx->have_tensor_map) return KVS_ERR_INVALID_ARG;
+    if (((uintptr_t)q % 16) != 0 || ((uintptr_t)out % 16) != 0) return KVS_ERR_INVALID_ARG;
+    const int slot = ctx->slot_of_layer[layer];
+    const int n = ctx->slot_len[slot];
+    if (n == 0) return KVS_ERR_STATE;
+    if (batch > ctx->cur_batch || n_q > n) return KVS_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->cfg.device);
+    if (!guard.ok) return KVS_ERR_CUDA;
+    const long long plane_rows = (long long)ctx->cfg.max_batch * ctx->cfg.n_kv_heads * ctx->row_stride;
+    if (kvs::launch_prefill(q, out, reinterpret_cast<int*>(ctx->ws + ctx->off_status), ctx->tensor_map, batch, n_q,
+                            ctx->cfg.n_q_heads, ctx->G, n, ctx->row_stride, plane_rows * (2 * slot),
+                            plane_rows * (2 * slot + 1), ctx->scale * 1.4426950408889634f,
+                            static_cast<cudaStream_t>(stream)) != cudaSuccess)
+        return KVS_ERR_CUDA;
+    // a plain launch: it starts only after everything before it on the stream has finished
+    ctx->seq += 1;
+    ctx->last_splitk_seq = ctx->seq;
+    ctx->stats.prefill_launches += 1;
+    ctx->stats.kv_bytes_read += 0;  // prefill is compute-bound; its K/V reads are not counted as decode traffic
+    return KVS_OK;
 }
 
 kvs_status kvs_step_host(kvs_ctx* ctx, const void* q_host, const void* k_host, const void* v_host, float* out_host,

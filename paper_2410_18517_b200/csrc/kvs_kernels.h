@@ -61,6 +61,12 @@ cudaError_t make_pool_tensor_map(void* storage, void* pool, long long total_rows
 cudaError_t launch_decode_mma(const DecodeArgs& a, const DecodePlan& plan, const void* tensor_map, long long krow0,
                               long long vrow0, cudaStream_t stream);
 
+// Tensor-core prefill attention (bf16, head size 128): q [B][T][Hq][128], out fp32 of the same shape.
+cudaError_t init_prefill_kernels();
+cudaError_t launch_prefill(const void* q, float* out, int* status, const void* pool_tensor_map, int B, int T, int Hq,
+                           int G, int n, int row_stride, long long krow0, long long vrow0, float scale_log2,
+                           cudaStream_t stream);
+
 cudaError_t launch_append(const void* k, const void* v, void* kplane, void* vplane, int B, int n_new, int Hkv,
                           int row_bytes, int row_stride, int len0, bool programmatic, cudaStream_t stream);
 cudaError_t launch_decode_scalar(const DecodeArgs& a, const DecodePlan& plan, cudaStream_t stream);
