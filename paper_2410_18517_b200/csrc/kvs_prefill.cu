@@ -3,14 +3,16 @@
 // n_q queries per head (the newest n_q positions of the slot the layer reads, causal mask)
 // against the slot's K/V rows: a dense contraction, so it runs on tcgen05.mma with the
 // accumulators in tensor memory.  One thread block = 128 queries of one (sequence, q-head):
-//   warp 4 (one lane)  TMA producer: Q tile once, then K/V tiles of 128 keys, 2 stages
+//   warp 4 (one lane)  TMA producer: Q tile once, then K and V tiles of 128 keys
 //   warp 5 (one lane)  MMA issuer:   S = Q K^T  (128x128x128, bf16 -> fp32 in TMEM)
-//                                    O_tile = P V with P = P_hi + P_lo (two bf16 terms)
+//                                    O += P V with P = P_hi + P_lo (two bf16 terms, read from TMEM)
 //   warps 0..3         softmax: thread r owns query row r = TMEM lane r; reads S with
-//                      tcgen05.ld, keeps the running max / sum / output row in registers,
-//                      writes P_hi, P_lo to shared memory in the swizzled K-major layout
-// K/V/Q tiles land in the 128-byte-swizzled layout the MMA shared-memory descriptors expect
-// (K and Q K-major, V MN-major).  bf16 storage, head size 128.
+//                      tcgen05.ld, writes P_hi / P_lo over S with tcgen05.st, and rescales the
+//                      output row in TMEM only when the running maximum grows by more than 2^8
+// Two blocks share an SM (96 KiB of shared memory and 256 TMEM columns each), so one block's
+// softmax overlaps the other's tensor-core work.  K/V/Q tiles land in the 128-byte-swizzled
+// layout the MMA shared-memory descriptors expect (K and Q K-major, V MN-major).
+// bf16 storage, head size 128.
 #include <cuda.h>
 
 #include <algorithm>
@@ -26,8 +28,7 @@ constexpr int kPfThreads = 192;
 constexpr int kPfTile = 128;                 // queries per block and keys per tile
 constexpr int kPfHalfBytes = kPfTile * 128;  // 128 rows x 64 bf16: one swizzled column block
 constexpr int kPfMatBytes = 2 * kPfHalfBytes;  // a 128 x 128 bf16 operand
-constexpr int kPfStages = 2;
-constexpr int kPfSmemBytes = 1024 + kPfMatBytes /*Q*/ + kPfStages * 2 * kPfMatBytes /*K,V*/ + 2 * kPfMatBytes /*P*/ + 256;
+constexpr int kPfSmemBytes = 1024 + 3 * kPfMatBytes /*Q, K, V*/ + 256;
 constexpr uint32_t kTmemCols = 256;          // S: columns [0,128), O tile: [128,256)
 
 __device__ __forceinline__ void tma_load_2d_pf(void* dst, const CUtensorMap* tmap, int x, int y, uint64_t* bar) {
@@ -77,6 +78,19 @@ __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t desc_a, uint
         : "memory");
 }
 
+// Same, with the A operand read from tensor memory (row = lane, two bf16 per 32-bit column).
+__device__ __forceinline__ void umma_bf16_ts(uint32_t tmem_d, uint32_t tmem_a, uint64_t desc_b, uint32_t idesc,
+                                             uint32_t accumulate) {
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, {%5, %6, %7, %8}, p;\n\t"
+        "}\n" ::"r"(tmem_d),
+        "r"(tmem_a), "l"(desc_b), "r"(idesc), "r"(accumulate), "r"(0u), "r"(0u), "r"(0u), "r"(0u)
+        : "memory");
+}
+
 __device__ __forceinline__ void umma_commit(uint64_t* bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
                  : "memory");
@@ -84,7 +98,6 @@ __device__ __forceinline__ void umma_commit(uint64_t* bar) {
 
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
 // 32 consecutive fp32 columns of this thread's TMEM lane.
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
@@ -104,6 +117,28 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
     for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
 
+// 32 fp32 columns of this thread's TMEM lane, written back.
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const float (&v)[32]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,"
+        "%31,%32};" ::"r"(taddr),
+        "f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3]), "f"(v[4]), "f"(v[5]), "f"(v[6]), "f"(v[7]), "f"(v[8]), "f"(v[9]),
+        "f"(v[10]), "f"(v[11]), "f"(v[12]), "f"(v[13]), "f"(v[14]), "f"(v[15]), "f"(v[16]), "f"(v[17]), "f"(v[18]),
+        "f"(v[19]), "f"(v[20]), "f"(v[21]), "f"(v[22]), "f"(v[23]), "f"(v[24]), "f"(v[25]), "f"(v[26]), "f"(v[27]),
+        "f"(v[28]), "f"(v[29]), "f"(v[30]), "f"(v[31])
+        : "memory");
+}
+
+// 16 packed 32-bit columns (32 bf16 values) of this thread's TMEM lane.
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&v)[16]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};" ::"r"(taddr),
+        "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]), "r"(v[9]),
+        "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15])
+        : "memory");
+}
+
 __device__ __forceinline__ uint32_t pack2_bf16(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t*>(&v);
@@ -120,22 +155,45 @@ struct PrefillArgs {
     float scale_log2;
 };
 
-__global__ void __launch_bounds__(kPfThreads, 1)
+// One softmax pass over a 32-column chunk of S: p = 2^(x*scale - m_ref) (0 where masked),
+// split into bf16 hi and lo words (2 keys per word).  Returns the chunk's sum of p.
+template <bool MASK>
+__device__ __forceinline__ float softmax_chunk(const float (&x)[32], float scale_log2, float m_ref, int key_first,
+                                               int limit, uint32_t (&hi)[16], uint32_t (&lo)[16]) {
+    float sum = 0.f;
+#pragma unroll
+    for (int i = 0; i < 32; i += 2) {
+        float p0 = fast_exp2(fmaf(x[i], scale_log2, -m_ref));
+        float p1 = fast_exp2(fmaf(x[i + 1], scale_log2, -m_ref));
+        if (MASK) {
+            p0 = (key_first + i <= limit) ? p0 : 0.f;
+            p1 = (key_first + i + 1 <= limit) ? p1 : 0.f;
+        }
+        sum += p0 + p1;
+        const uint32_t h = pack2_bf16(p0, p1);
+        hi[i >> 1] = h;
+        lo[i >> 1] = pack2_bf16(p0 - __uint_as_float(h << 16), p1 - __uint_as_float(h & 0xffff0000u));
+    }
+    return sum;
+}
+
+__global__ void __launch_bounds__(kPfThreads, 2)
     prefill_attention_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_kv,
                          const PrefillArgs a) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     unsigned char* sQ = smem;
-    unsigned char* sKV = sQ + kPfMatBytes;                       // stage s: K at +s*2*Mat, V right after it
-    unsigned char* sPhi = sKV + kPfStages * 2 * kPfMatBytes;
-    unsigned char* sPlo = sPhi + kPfMatBytes;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(sPlo + kPfMatBytes);
-    uint64_t* q_full = bars;            // 1
-    uint64_t* kv_full = bars + 1;       // 2
-    uint64_t* kv_empty = bars + 3;      // 2
-    uint64_t* s_full = bars + 5;        // 1
-    uint64_t* p_full = bars + 6;        // 1 (128 arrivals)
-    uint64_t* o_full = bars + 7;        // 1
+    unsigned char* sK = sQ + kPfMatBytes;
+    unsigned char* sV = sK + kPfMatBytes;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(sV + kPfMatBytes);
+    uint64_t* q_full = bars;
+    uint64_t* k_full = bars + 1;
+    uint64_t* k_empty = bars + 2;
+    uint64_t* v_full = bars + 3;
+    uint64_t* v_empty = bars + 4;
+    uint64_t* s_full = bars + 5;
+    uint64_t* p_full = bars + 6;        // 128 arrivals
+    uint64_t* o_full = bars + 7;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 8);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 9);
 
@@ -150,14 +208,7 @@ __global__ void __launch_bounds__(kPfThreads, 1)
     const int nt = last_key / kPfTile + 1;
 
     if (tid == 0) {
-        mbar_init(q_full, 1);
-        for (int s = 0; s < kPfStages; ++s) {
-            mbar_init(&kv_full[s], 1);
-            mbar_init(&kv_empty[s], 1);
-        }
-        mbar_init(s_full, 1);
-        mbar_init(p_full, 128);
-        mbar_init(o_full, 1);
+        for (int i = 0; i < 8; ++i) mbar_init(&bars[i], i == 6 ? 128 : 1);
         abort_flag[0] = 0;
         fence_mbar_init();
     }
@@ -171,8 +222,8 @@ __global__ void __launch_bounds__(kPfThreads, 1)
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
-    const uint32_t tmem_s = tmem_base;
-    const uint32_t tmem_o = tmem_base + 128;
+    const uint32_t tmem_s = tmem_base;         // S (fp32, 128 columns); P_hi / P_lo (bf16 pairs) overwrite it
+    const uint32_t tmem_o = tmem_base + 128;   // running output rows
 
     if (warp == 4) {
         // ------------------------------ TMA producer ------------------------------
@@ -182,23 +233,23 @@ __global__ void __launch_bounds__(kPfThreads, 1)
             tma_load_4d(sQ + kPfHalfBytes, &tmap_q, 64, hq, q0, b, q_full);
             const long long unit_row = ((long long)b * Hkv + hk) * a.row_stride;
             for (int j = 0; j < nt; ++j) {
-                const int s = j & 1;
-                if (j >= kPfStages &&
-                    !mbar_wait_bounded(&kv_empty[s], ((j >> 1) - 1) & 1, abort_flag, a.status))
-                    break;
-                unsigned char* sK = sKV + s * 2 * kPfMatBytes;
-                unsigned char* sV = sK + kPfMatBytes;
-                mbar_arrive_expect_tx(&kv_full[s], 2 * kPfMatBytes);
                 const long long row = unit_row + (long long)j * kPfTile;
+                if (j >= 1 && !mbar_wait_bounded(k_empty, (j - 1) & 1, abort_flag, a.status)) break;
+                mbar_arrive_expect_tx(k_full, kPfMatBytes);
 #pragma unroll
                 for (int h = 0; h < 2; ++h)
 #pragma unroll
-                    for (int rb = 0; rb < 2; ++rb) {
+                    for (int rb = 0; rb < 2; ++rb)
                         tma_load_2d_pf(sK + h * kPfHalfBytes + rb * 8192, &tmap_kv, h * 64, (int)(a.krow0 + row + rb * 64),
-                                       &kv_full[s]);
+                                       k_full);
+                if (j >= 1 && !mbar_wait_bounded(v_empty, (j - 1) & 1, abort_flag, a.status)) break;
+                mbar_arrive_expect_tx(v_full, kPfMatBytes);
+#pragma unroll
+                for (int h = 0; h < 2; ++h)
+#pragma unroll
+                    for (int rb = 0; rb < 2; ++rb)
                         tma_load_2d_pf(sV + h * kPfHalfBytes + rb * 8192, &tmap_kv, h * 64, (int)(a.vrow0 + row + rb * 64),
-                                       &kv_full[s]);
-                    }
+                                       v_full);
             }
         }
     } else if (warp == 5) {
@@ -206,9 +257,8 @@ __global__ void __launch_bounds__(kPfThreads, 1)
         if (lane == 0) {
             const uint32_t idesc_s = instr_desc_bf16(0);
             const uint32_t idesc_o = instr_desc_bf16(1);
-            const uint32_t q_addr = smem_u32(sQ), phi_addr = smem_u32(sPhi), plo_addr = smem_u32(sPlo);
-            auto issue_s = [&](int j) {
-                const uint32_t k_addr = smem_u32(sKV + (j & 1) * 2 * kPfMatBytes);
+            const uint32_t q_addr = smem_u32(sQ), k_addr = smem_u32(sK), v_addr = smem_u32(sV);
+            auto issue_s = [&]() {
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {   // 16 head-dim columns per step; 4 steps per 64-column block
                     const uint32_t off = (ks >> 2) * kPfHalfBytes + (ks & 3) * 32;
@@ -216,34 +266,34 @@ __global__ void __launch_bounds__(kPfThreads, 1)
                               idesc_s, ks > 0);
                 }
                 umma_commit(s_full);
+                umma_commit(k_empty);     // the K tile may be overwritten once S is done
             };
             bool ok = mbar_wait_bounded(q_full, 0, abort_flag, a.status) &&
-                      mbar_wait_bounded(&kv_full[0], 0, abort_flag, a.status);
+                      mbar_wait_bounded(k_full, 0, abort_flag, a.status);
             if (ok) {
                 tc_fence_after();
-                issue_s(0);
+                issue_s();
             }
             for (int j = 0; j < nt && ok; ++j) {
-                ok = mbar_wait_bounded(p_full, j & 1, abort_flag, a.status);
+                ok = mbar_wait_bounded(p_full, j & 1, abort_flag, a.status) &&
+                     mbar_wait_bounded(v_full, j & 1, abort_flag, a.status);
                 if (!ok) break;
                 tc_fence_after();
-                const uint32_t v_addr = smem_u32(sKV + (j & 1) * 2 * kPfMatBytes + kPfMatBytes);
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {   // 16 keys per step
-                    const uint32_t a_off = (ks >> 2) * kPfHalfBytes + (ks & 3) * 32;
+                for (int ks = 0; ks < 8; ++ks) {   // 16 keys per step: 8 TMEM columns of bf16 pairs
                     // V is MN-major: 64 head-dim columns contiguous per key row, the other 64 one
                     // column block (LBO) away; 8-key groups 1024 bytes (SBO) apart
                     const uint64_t vdesc = smem_desc_sw128(v_addr + ks * 16 * 128, kPfHalfBytes, 1024);
-                    umma_bf16(tmem_o, smem_desc_sw128(phi_addr + a_off, 16, 1024), vdesc, idesc_o, ks > 0);
-                    umma_bf16(tmem_o, smem_desc_sw128(plo_addr + a_off, 16, 1024), vdesc, idesc_o, 1);
+                    umma_bf16_ts(tmem_o, tmem_s + ks * 8, vdesc, idesc_o, (j > 0) || (ks > 0));        // P_hi
+                    umma_bf16_ts(tmem_o, tmem_s + 64 + ks * 8, vdesc, idesc_o, 1);                   // P_lo
                 }
                 umma_commit(o_full);
-                umma_commit(&kv_empty[j & 1]);
+                umma_commit(v_empty);
                 if (j + 1 < nt) {
-                    ok = mbar_wait_bounded(&kv_full[(j + 1) & 1], ((j + 1) >> 1) & 1, abort_flag, a.status);
+                    ok = mbar_wait_bounded(k_full, (j + 1) & 1, abort_flag, a.status);
                     if (!ok) break;
                     tc_fence_after();
-                    issue_s(j + 1);
+                    issue_s();
                 }
             }
         }
@@ -252,81 +302,100 @@ __global__ void __launch_bounds__(kPfThreads, 1)
         const int r = tid;                                   // query row in the block = TMEM lane
         const int qpos = min(q0 + r, a.T - 1);               // padding rows repeat the last query
         const int limit = a.n - a.T + qpos;                  // last key this query may see
+        const int block_min_limit = a.n - a.T + q0;          // smallest limit of any row of the block
         const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
-        float acc[128];
-#pragma unroll
-        for (int i = 0; i < 128; ++i) acc[i] = 0.f;
-        float m = -1.0e30f, l = 0.f;
+        const uint32_t ts = tmem_s + lane_addr, to = tmem_o + lane_addr;
+        float m_ref = -1.0e30f, l = 0.f;                     // p is taken relative to m_ref (log2 domain)
         bool ok = true;
         for (int j = 0; j < nt; ++j) {
             ok = mbar_wait_bounded(s_full, j & 1, abort_flag, a.status);
             if (!ok) break;
             tc_fence_after();
             const int key0 = j * kPfTile;
-            // pass 1: row maximum of the masked, scaled scores
+            const bool mask = key0 + kPfTile - 1 > block_min_limit;   // block-uniform
+            // pass 1: row maximum of the (masked) scores
             float mx = -INFINITY;
 #pragma unroll 1
             for (int c = 0; c < 4; ++c) {
                 float x[32];
-                tmem_ld32(tmem_s + lane_addr + c * 32, x);
+                tmem_ld32(ts + c * 32, x);
+                if (mask) {
 #pragma unroll
-                for (int i = 0; i < 32; ++i)
-                    mx = fmaxf(mx, (key0 + c * 32 + i <= limit) ? x[i] * a.scale_log2 : -INFINITY);
+                    for (int i = 0; i < 32; ++i) mx = fmaxf(mx, (key0 + c * 32 + i <= limit) ? x[i] : -INFINITY);
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) mx = fmaxf(mx, x[i]);
+                }
             }
-            const float m_new = fmaxf(m, mx);
-            const float alpha = fast_exp2(m - m_new);
-            // pass 2: p = 2^(x - m_new), split into two bf16 terms, into the swizzled A-operand layout
+            mx *= a.scale_log2;
+            // The reference maximum only moves when the new one is more than 8 (a factor 256) above
+            // it; then the output row and the sum accumulated so far are rescaled.  PV of the
+            // previous tile has finished (S of this tile was issued after it), so O is quiet.
+            const bool grow = mx > m_ref + 8.0f;
+            if (__any_sync(0xffffffffu, grow)) {
+                const float m_new = grow ? mx : m_ref;
+                const float alpha = fast_exp2(m_ref - m_new);
+                if (j > 0) {
+#pragma unroll 1
+                    for (int c = 0; c < 4; ++c) {
+                        float o[32];
+                        tmem_ld32(to + c * 32, o);
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) o[i] *= alpha;
+                        tmem_st32(to + c * 32, o);
+                    }
+                }
+                l *= alpha;
+                m_ref = m_new;
+            }
+            // pass 2, upper key half first: P_hi / P_lo overwrite S, so a column may only be written
+            // once the scores in it have been read.  P_hi[keys k] -> columns k/2, P_lo -> 64 + k/2.
+            uint32_t hi3[16], hi2[16], hi1[16], hi0[16], lo[16];
             float lsum = 0.f;
+            {
+                float x[32];
+                tmem_ld32(ts + 96, x);
+                lsum += mask ? softmax_chunk<true>(x, a.scale_log2, m_ref, key0 + 96, limit, hi3, lo)
+                             : softmax_chunk<false>(x, a.scale_log2, m_ref, key0 + 96, limit, hi3, lo);
+                tmem_ld32(ts + 64, x);          // all scores of columns 64..127 are now in registers
+                tmem_st16(ts + 64 + 48, lo);
+                lsum += mask ? softmax_chunk<true>(x, a.scale_log2, m_ref, key0 + 64, limit, hi2, lo)
+                             : softmax_chunk<false>(x, a.scale_log2, m_ref, key0 + 64, limit, hi2, lo);
+                tmem_st16(ts + 64 + 32, lo);
+                tmem_ld32(ts + 32, x);
+                lsum += mask ? softmax_chunk<true>(x, a.scale_log2, m_ref, key0 + 32, limit, hi1, lo)
+                             : softmax_chunk<false>(x, a.scale_log2, m_ref, key0 + 32, limit, hi1, lo);
+                tmem_st16(ts + 64 + 16, lo);
+                tmem_ld32(ts, x);               // columns 0..63 are now in registers too
+                tmem_st16(ts + 32, hi2);
+                tmem_st16(ts + 48, hi3);
+                tmem_st16(ts + 16, hi1);
+                lsum += mask ? softmax_chunk<true>(x, a.scale_log2, m_ref, key0, limit, hi0, lo)
+                             : softmax_chunk<false>(x, a.scale_log2, m_ref, key0, limit, hi0, lo);
+                tmem_st16(ts, hi0);
+                tmem_st16(ts + 64, lo);
+            }
+            l += lsum;
+            asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+            tc_fence_before();
+            mbar_arrive(p_full);
+        }
+        if (ok) ok = mbar_wait_bounded(o_full, (nt - 1) & 1, abort_flag, a.status);
+        if (ok) {
+            tc_fence_after();
+            const float inv = 1.0f / l;
+            const bool store = q0 + r < a.T;
+            float4* dst = reinterpret_cast<float4*>(a.out + (((long long)b * a.T + min(q0 + r, a.T - 1)) * a.Hq + hq) * 128);
 #pragma unroll 1
             for (int c = 0; c < 4; ++c) {
-                float x[32];
-                tmem_ld32(tmem_s + lane_addr + c * 32, x);
-                uint32_t hi[16], lo[16];
-#pragma unroll
-                for (int i = 0; i < 32; i += 2) {
-                    const float p0 = (key0 + c * 32 + i <= limit) ? fast_exp2(x[i] * a.scale_log2 - m_new) : 0.f;
-                    const float p1 = (key0 + c * 32 + i + 1 <= limit) ? fast_exp2(x[i + 1] * a.scale_log2 - m_new) : 0.f;
-                    lsum += p0 + p1;
-                    const float h0 = __bfloat162float(__float2bfloat16_rn(p0));
-                    const float h1 = __bfloat162float(__float2bfloat16_rn(p1));
-                    hi[i >> 1] = pack2_bf16(h0, h1);
-                    lo[i >> 1] = pack2_bf16(p0 - h0, p1 - h1);
-                }
-                // keys c*32 .. c*32+31 = column block c/2, 16-byte chunks (c%2)*4 .. +3 of row r
-                const uint32_t row_off = (c >> 1) * kPfHalfBytes + r * 128;
-#pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    const uint32_t chunk = ((c & 1) * 4 + k) ^ (r & 7);
-                    *reinterpret_cast<uint4*>(sPhi + row_off + chunk * 16) =
-                        make_uint4(hi[4 * k], hi[4 * k + 1], hi[4 * k + 2], hi[4 * k + 3]);
-                    *reinterpret_cast<uint4*>(sPlo + row_off + chunk * 16) =
-                        make_uint4(lo[4 * k], lo[4 * k + 1], lo[4 * k + 2], lo[4 * k + 3]);
-                }
-            }
-            l = l * alpha + lsum;
-            m = m_new;
-            tc_fence_before();
-            fence_async_smem();
-            mbar_arrive(p_full);
-            // O_tile = P V of this tile, folded into the running output row
-            ok = mbar_wait_bounded(o_full, j & 1, abort_flag, a.status);
-            if (!ok) break;
-            tc_fence_after();
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
                 float o[32];
-                tmem_ld32(tmem_o + lane_addr + c * 32, o);
+                tmem_ld32(to + c * 32, o);
+                if (store) {
 #pragma unroll
-                for (int i = 0; i < 32; ++i) acc[c * 32 + i] = fmaf(acc[c * 32 + i], alpha, o[i]);
+                    for (int i = 0; i < 8; ++i)
+                        dst[c * 8 + i] = make_float4(o[4 * i] * inv, o[4 * i + 1] * inv, o[4 * i + 2] * inv, o[4 * i + 3] * inv);
+                }
             }
-            tc_fence_before();
-        }
-        if (ok && q0 + r < a.T) {
-            const float inv = 1.0f / l;
-            float4* dst = reinterpret_cast<float4*>(a.out + (((long long)b * a.T + (q0 + r)) * a.Hq + hq) * 128);
-#pragma unroll
-            for (int i = 0; i < 32; ++i)
-                dst[i] = make_float4(acc[4 * i] * inv, acc[4 * i + 1] * inv, acc[4 * i + 2] * inv, acc[4 * i + 3] * inv);
         }
     }
     // every thread of every role ends here; tensor memory is released by the warp that took it
