@@ -49,7 +49,8 @@ typedef struct {
     int L, Hq, Hkv, D, B;
     double scale;    /* 1/sqrt(D) unless the caller fixed another one        */
     int *share_map;  /* share_map[l] = layer whose cache layer l uses        */
-    int *len;        /* cached tokens of layer l's own (possibly copied) cache */
+    int **ulen;      /* ulen[l][b*Hkv+h]: cached tokens of that (sequence, head) of layer l;
+                        equal across a layer until an intra-layer method evicts rows */
     int *cap;        /* allocated tokens per unit of layer l                 */
     double ***K;     /* K[l][b*Hkv+h] -> [cap][D] row-major                  */
     double ***V;
@@ -168,7 +169,8 @@ oracle_state *oracle_create(int L, int Hq, int Hkv, int D, int B,
     st->scale = (scale > 0.0) ? scale : 1.0 / sqrt((double)D);
     st->share_map = (int *)malloc(sizeof(int) * L);
     memcpy(st->share_map, share_map, sizeof(int) * L);
-    st->len = (int *)calloc(L, sizeof(int));
+    st->ulen = (int **)calloc(L, sizeof(int *));
+    for (int l = 0; l < L; ++l) st->ulen[l] = (int *)calloc((size_t)B * Hkv, sizeof(int));
     st->cap = (int *)calloc(L, sizeof(int));
     st->K = (double ***)calloc(L, sizeof(double **));
     st->V = (double ***)calloc(L, sizeof(double **));
@@ -185,7 +187,8 @@ void oracle_destroy(oracle_state *st) {
         for (int u = 0; u < st->B * st->Hkv; ++u) { free(st->K[l][u]); free(st->V[l][u]); }
         free(st->K[l]); free(st->V[l]);
     }
-    free(st->K); free(st->V); free(st->len); free(st->cap); free(st->share_map);
+    for (int l = 0; l < st->L; ++l) free(st->ulen[l]);
+    free(st->K); free(st->V); free(st->ulen); free(st->cap); free(st->share_map);
     free(st);
 }
 
@@ -208,31 +211,44 @@ static void ensure_cap(oracle_state *st, int l, int need) {
  *       the cache of layer share_map[l], as it stands after that layer's own
  *       turn in this pass, is copied over this layer's cache.
  * Returns 0, or -1 on a bad argument.                                          */
+static int max_unit_len(const oracle_state *st, int l) {
+    int m = 0;
+    for (int u = 0; u < st->B * st->Hkv; ++u) if (st->ulen[l][u] > m) m = st->ulen[l][u];
+    return m;
+}
+
+static int uniform_len(const oracle_state *st, int l) {   /* common length, or -1 if units differ */
+    for (int u = 1; u < st->B * st->Hkv; ++u) if (st->ulen[l][u] != st->ulen[l][0]) return -1;
+    return st->ulen[l][0];
+}
+
 static int update_cache(oracle_state *st, int l, const double *k_new, const double *v_new, int n_new) {
     const int D = st->D, Hkv = st->Hkv, B = st->B;
     const int src = st->share_map[l];
     if (src == l) {
         if (n_new > 0) {
             if (!k_new || !v_new) return -1;
-            ensure_cap(st, l, st->len[l] + n_new);
+            ensure_cap(st, l, max_unit_len(st, l) + n_new);
             for (int b = 0; b < B; ++b)
-                for (int t = 0; t < n_new; ++t)
-                    for (int h = 0; h < Hkv; ++h) {
+                for (int h = 0; h < Hkv; ++h) {
+                    const int u = b * Hkv + h;
+                    for (int t = 0; t < n_new; ++t) {
                         size_t in = (((size_t)b * n_new + t) * Hkv + h) * D;
-                        size_t row = (size_t)(st->len[l] + t) * D;
-                        memcpy(st->K[l][b * Hkv + h] + row, k_new + in, sizeof(double) * D);
-                        memcpy(st->V[l][b * Hkv + h] + row, v_new + in, sizeof(double) * D);
+                        size_t row = (size_t)(st->ulen[l][u] + t) * D;
+                        memcpy(st->K[l][u] + row, k_new + in, sizeof(double) * D);
+                        memcpy(st->V[l][u] + row, v_new + in, sizeof(double) * D);
                     }
-            st->len[l] += n_new;
+                    st->ulen[l][u] += n_new;
+                }
         }
     } else {
-        /* literal copy of the previously computed layer's cache */
-        ensure_cap(st, l, st->len[src]);
+        /* literal copy of the previously computed layer's cache (sparsified or not) */
+        ensure_cap(st, l, max_unit_len(st, src));
         for (int u = 0; u < B * Hkv; ++u) {
-            memcpy(st->K[l][u], st->K[src][u], sizeof(double) * (size_t)st->len[src] * D);
-            memcpy(st->V[l][u], st->V[src][u], sizeof(double) * (size_t)st->len[src] * D);
+            memcpy(st->K[l][u], st->K[src][u], sizeof(double) * (size_t)st->ulen[src][u] * D);
+            memcpy(st->V[l][u], st->V[src][u], sizeof(double) * (size_t)st->ulen[src][u] * D);
+            st->ulen[l][u] = st->ulen[src][u];
         }
-        st->len[l] = st->len[src];
     }
     return 0;
 }
@@ -248,16 +264,16 @@ int oracle_layer_forward(oracle_state *st, int l, const double *q,
     const int D = st->D, Hkv = st->Hkv, Hq = st->Hq, B = st->B;
     if (update_cache(st, l, k_new, v_new, n_new) != 0) return -1;
     if (q) {
-        if (!out || st->len[l] <= 0) return -1;
+        if (!out) return -1;
+        for (int u = 0; u < B * Hkv; ++u) if (st->ulen[l][u] <= 0) return -1;
         const int G = Hq / Hkv;
-        const int n = st->len[l];
 #pragma omp parallel for collapse(2) schedule(static)
         for (int b = 0; b < B; ++b)
             for (int hq = 0; hq < Hq; ++hq) {
                 int hk = hq / G;
                 size_t o = ((size_t)b * Hq + hq) * D;
                 oracle_attend_unit(q + o, st->K[l][b * Hkv + hk], st->V[l][b * Hkv + hk],
-                                   n, D, st->scale, out + o);
+                                   st->ulen[l][b * Hkv + hk], D, st->scale, out + o);
             }
     }
     return 0;
@@ -276,8 +292,8 @@ int oracle_layer_prefill(oracle_state *st, int l, const double *q, int n_q,
     if (!st || l < 0 || l >= st->L || n_new < 0 || n_q < 1 || !q || !out) return -1;
     const int D = st->D, Hkv = st->Hkv, Hq = st->Hq, B = st->B;
     if (update_cache(st, l, k_new, v_new, n_new) != 0) return -1;
-    const int n = st->len[l];
-    if (n_q > n) return -1;
+    const int n = uniform_len(st, l);   /* positions are only defined while no rows were evicted */
+    if (n < 0 || n_q > n) return -1;
     const int G = Hq / Hkv;
 #pragma omp parallel for collapse(2) schedule(dynamic)
     for (int b = 0; b < B; ++b)
@@ -291,18 +307,57 @@ int oracle_layer_prefill(oracle_state *st, int l, const double *q, int n_q,
     return 0;
 }
 
+/* Longest (sequence, head) of layer l's cache (all are equal unless rows were evicted). */
 int oracle_len(const oracle_state *st, int l) {
-    return (st && l >= 0 && l < st->L) ? st->len[l] : -1;
+    return (st && l >= 0 && l < st->L) ? max_unit_len(st, l) : -1;
 }
 
-/* Copy layer l's cache out as [B][Hkv][len][D] (K then V into separate
- * buffers), for bit-exact comparison with what the GPU pool holds.           */
+int oracle_unit_len(const oracle_state *st, int l, int b, int h) {
+    if (!st || l < 0 || l >= st->L || b < 0 || b >= st->B || h < 0 || h >= st->Hkv) return -1;
+    return st->ulen[l][b * st->Hkv + h];
+}
+
+/* Intra-layer compression applied to a layer that computes its own cache (Section 4.4 and the
+ * reproduction appendix: each layer's cache is sparsified in turn by H2O / PyramidInfer, and
+ * a layer that shares receives the sparsified cache of its source, which here happens by the
+ * usual literal copy at the sharing layer's next turn).  Which rows survive is the outside
+ * method's decision: keep[(b*Hkv+h)*keep_stride + j], j < n_keep[b*Hkv+h], strictly ascending
+ * row indices of unit (b,h).  The kept rows move to the front in order; the rest is gone.
+ * Returns 0, or -1 for a sharing layer, an empty or non-ascending or out-of-range list.      */
+int oracle_evict(oracle_state *st, int l, const int *keep, const int *n_keep, int keep_stride) {
+    if (!st || l < 0 || l >= st->L || !keep || !n_keep || st->share_map[l] != l) return -1;
+    const int D = st->D;
+    for (int u = 0; u < st->B * st->Hkv; ++u) {
+        if (n_keep[u] < 1 || n_keep[u] > st->ulen[l][u] || n_keep[u] > keep_stride) return -1;
+        for (int j = 0; j < n_keep[u]; ++j) {
+            int r = keep[(size_t)u * keep_stride + j];
+            if (r < 0 || r >= st->ulen[l][u] || (j > 0 && r <= keep[(size_t)u * keep_stride + j - 1])) return -1;
+        }
+    }
+    for (int u = 0; u < st->B * st->Hkv; ++u) {
+        for (int j = 0; j < n_keep[u]; ++j) {
+            int r = keep[(size_t)u * keep_stride + j];
+            memmove(st->K[l][u] + (size_t)j * D, st->K[l][u] + (size_t)r * D, sizeof(double) * D);
+            memmove(st->V[l][u] + (size_t)j * D, st->V[l][u] + (size_t)r * D, sizeof(double) * D);
+        }
+        st->ulen[l][u] = n_keep[u];
+    }
+    return 0;
+}
+
+/* Copy layer l's cache out as [B][Hkv][len][D] with len = oracle_len (K then V into
+ * separate buffers; rows past a unit's own length are zero), for bit-exact comparison
+ * with what the GPU pool holds.                                               */
 int oracle_get_cache(const oracle_state *st, int l, double *K_out, double *V_out) {
     if (!st || l < 0 || l >= st->L) return -1;
-    size_t rows = (size_t)st->len[l] * st->D;
+    const int n = max_unit_len(st, l);
+    size_t rows = (size_t)n * st->D;
     for (int u = 0; u < st->B * st->Hkv; ++u) {
-        memcpy(K_out + u * rows, st->K[l][u], sizeof(double) * rows);
-        memcpy(V_out + u * rows, st->V[l][u], sizeof(double) * rows);
+        size_t have = (size_t)st->ulen[l][u] * st->D;
+        memcpy(K_out + u * rows, st->K[l][u], sizeof(double) * have);
+        memcpy(V_out + u * rows, st->V[l][u], sizeof(double) * have);
+        memset(K_out + u * rows + have, 0, sizeof(double) * (rows - have));
+        memset(V_out + u * rows + have, 0, sizeof(double) * (rows - have));
     }
     return 0;
 }

@@ -63,6 +63,10 @@ def _load():
     lib.oracle_layer_prefill.restype = ctypes.c_int
     lib.oracle_len.argtypes = [ctypes.c_void_p, ctypes.c_int]
     lib.oracle_len.restype = ctypes.c_int
+    lib.oracle_unit_len.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_int]
+    lib.oracle_unit_len.restype = ctypes.c_int
+    lib.oracle_evict.argtypes = [ctypes.c_void_p, ctypes.c_int, _ip, _ip, ctypes.c_int]
+    lib.oracle_evict.restype = ctypes.c_int
     lib.oracle_get_cache.argtypes = [ctypes.c_void_p, ctypes.c_int, _dp, _dp]
     lib.oracle_get_cache.restype = ctypes.c_int
     _lib = lib
@@ -211,6 +215,18 @@ class Oracle:
 
     def length(self, l) -> int:
         return int(self._lib.oracle_len(self._h, l))
+
+    def unit_len(self, l, b, h) -> int:
+        return int(self._lib.oracle_unit_len(self._h, l, b, h))
+
+    def evict(self, l, keep, n_keep):
+        """Keep only rows ``keep[b][h][:n_keep[b][h]]`` (strictly ascending) of every unit of layer l."""
+        keep = np.ascontiguousarray(np.asarray(keep, dtype=np.int32))
+        n_keep = np.ascontiguousarray(np.asarray(n_keep, dtype=np.int32))
+        assert keep.ndim == 3 and keep.shape[:2] == (self.B, self.Hkv) and n_keep.shape == (self.B, self.Hkv)
+        rc = self._lib.oracle_evict(self._h, l, keep.ctypes.data_as(_ip), n_keep.ctypes.data_as(_ip), keep.shape[2])
+        if rc != 0:
+            raise RuntimeError("oracle_evict rejected its arguments")
 
     def cache(self, l):
         """Layer l's cache as (K, V), each ``[B][Hkv][len][D]`` float64."""

@@ -375,3 +375,81 @@ def test_prefill_first_query_of_an_empty_cache_returns_first_value_row_and_one_q
     np.testing.assert_array_equal(o2.layer_forward(0, q[:, 5], k[:, 5:], v[:, 5:]), out[:, 5])
     with pytest.raises(RuntimeError):
         o.layer_prefill(0, RNG.standard_normal((1, 7, 2, 4)))     # more queries than cached rows
+
+
+# ---------------------------------------------------------------- eviction (intra-layer compression mechanics)
+def _random_keep(rng, B, Hkv, n, lo_frac=0.5):
+    n_keep = rng.integers(max(1, int(n * lo_frac)), n + 1, size=(B, Hkv)).astype(np.int32)
+    keep = np.zeros((B, Hkv, n), dtype=np.int32)
+    for b in range(B):
+        for h in range(Hkv):
+            keep[b, h, : n_keep[b, h]] = np.sort(rng.choice(n, size=n_keep[b, h], replace=False))
+    return keep, n_keep
+
+
+def test_eviction_against_brute_force_with_sharing_and_later_appends():
+    """Layer 1's cache is sparsified; layer 3 shares it and must see exactly the kept rows (and the
+    rows appended afterwards); layers 0 and 2 are untouched."""
+    L, Hq, Hkv, D, B, ctx = 4, 4, 2, 8, 2, 12
+    sm = [0, 1, 2, 1]
+    rng = np.random.default_rng(77)
+    o, kc, vc, qs, ks, vs, outs = run_oracle(L, Hq, Hkv, D, B, sm, ctx, 1, rng)
+    keep, n_keep = _random_keep(rng, B, Hkv, ctx + 1)
+    o.evict(1, keep, n_keep)
+    q2 = rng.standard_normal((L, B, Hq, D))
+    k2 = rng.standard_normal((L, B, 1, Hkv, D))
+    v2 = rng.standard_normal((L, B, 1, Hkv, D))
+    out2 = o.step(q2, k2, v2)
+    G = Hq // Hkv
+    for l in range(L):
+        r = 1 if l == 3 else l
+        Kfull = np.concatenate([kc[r], ks[0, r]], axis=1)         # [B][ctx+1][Hkv][D] before eviction
+        Vfull = np.concatenate([vc[r], vs[0, r]], axis=1)
+        for b in range(B):
+            for hq in range(Hq):
+                h = hq // G
+                rows = keep[b, h, : n_keep[b, h]] if r == 1 else np.arange(ctx + 1)
+                K = np.concatenate([Kfull[b, rows, h], k2[r, b, :, h]], axis=0)
+                V = np.concatenate([Vfull[b, rows, h], v2[r, b, :, h]], axis=0)
+                np.testing.assert_allclose(out2[l, b, hq], brute_attention(q2[l, b, hq], K, V), atol=1e-13)
+                assert o.unit_len(l, b, h) == len(rows) + 1
+    assert o.length(1) == int(n_keep.max()) + 1 and o.length(0) == ctx + 2
+
+
+def test_removing_one_row_follows_the_softmax_removal_identity():
+    """out' = (out * Z - e_j v_j) / (Z - e_j): dropping row j removes its term from both sums."""
+    n, D = 9, 8
+    q, K, V = RNG.standard_normal(D), RNG.standard_normal((n, D)), RNG.standard_normal((n, D))
+    o = oracle.Oracle(1, 1, 1, D, 1, [0])
+    o.layer_forward(0, None, K[None, :, None], V[None, :, None])
+    full = o.layer_forward(0, q[None, None])[0, 0]
+    j = 4
+    rows = np.array([[[r for r in range(n) if r != j] + [0]]], dtype=np.int32)
+    o.evict(0, rows, [[n - 1]])
+    got = o.layer_forward(0, q[None, None])[0, 0]
+    sc = K @ q / np.sqrt(D)
+    e = np.exp(sc - sc.max())
+    ref = (full * e.sum() - e[j] * V[j]) / (e.sum() - e[j])
+    np.testing.assert_allclose(got, ref, atol=1e-13)
+
+
+def test_keeping_everything_changes_nothing_and_bad_lists_are_rejected():
+    L, Hq, Hkv, D, B = 2, 2, 2, 4, 1
+    rng = np.random.default_rng(5)
+    o, *_ = run_oracle(L, Hq, Hkv, D, B, [0, 0], 5, 1, rng)
+    K0, V0 = o.cache(0)
+    o.evict(0, np.tile(np.arange(6, dtype=np.int32), (B, Hkv, 1)), np.full((B, Hkv), 6))
+    K1, V1 = o.cache(0)
+    np.testing.assert_array_equal(K0, K1)
+    np.testing.assert_array_equal(V0, V1)
+    for bad_keep, bad_n in (([[[3, 2, 0, 0, 0, 0]] * 2], [[2, 2]]),      # not ascending
+                            ([[[0, 6, 0, 0, 0, 0]] * 2], [[2, 2]]),      # out of range
+                            ([[[0, 1, 2, 3, 4, 5]] * 2], [[0, 1]])):     # empty unit
+        with pytest.raises(RuntimeError):
+            o.evict(0, bad_keep, bad_n)
+    with pytest.raises(RuntimeError):
+        o.evict(1, np.zeros((B, Hkv, 6), dtype=np.int32), np.ones((B, Hkv)))     # layer 1 shares
+    # prefill positions are undefined once units differ in length
+    o.evict(0, [[[0, 1, 2, 0, 0, 0], [0, 1, 0, 0, 0, 0]]], [[3, 2]])
+    with pytest.raises(RuntimeError):
+        o.layer_prefill(0, rng.standard_normal((B, 1, Hq, D)))
