@@ -79,6 +79,7 @@ typedef struct {
     uint64_t kv_bytes_read;       /* 2*B*Hkv*n*D*elem summed over attention calls            */
     uint64_t kv_bytes_appended;   /* 2*B*Hkv*n_new*D*elem summed over launched appends       */
     uint64_t prefill_launches;    /* tensor-core prefill kernels launched                    */
+    uint64_t evict_launches;      /* kvs_evict calls that launched                           */
 } kvs_stats_t;
 
 /* Tuning knobs for kvs_set_option.  Defaults are chosen by the library. */
@@ -178,6 +179,28 @@ kvs_status kvs_decode_attention(kvs_ctx* ctx, int32_t layer, const void* q, floa
 kvs_status kvs_prefill_attention(kvs_ctx* ctx, int32_t layer, const void* q, float* out,
                                  int32_t batch, int32_t n_q, void* stream);
 
+/* Keep only some rows of a layer's cache (the mechanics of combining layer sharing with an
+ * intra-layer compression method, Section 4.4 and the reproduction appendix: each layer's cache
+ * is sparsified in turn, and a layer that shares uses the sparsified cache of its source as it
+ * is).  Which rows survive is the outside method's decision; this call only applies it.
+ *   layer:  must compute its own cache (INVALID_ARG for a sharing layer); every layer that shares
+ *           it sees the change, because they read the same slot
+ *   keep:   device, int32 [batch][n_kv_heads][keep_stride]; the first n_keep[b*Hkv+h] entries of a
+ *           unit are the row indices to keep, strictly ascending, each below the unit's length
+ *   n_keep: host, int32 [batch * n_kv_heads], each in [1, current length of the unit]
+ * The kept rows move to the front of the unit in order, bit for bit; afterwards the units of the
+ * slot may differ in length ("ragged").  Appends then extend every unit at its own end,
+ * kvs_decode_attention uses each unit's own length, kvs_seq_len reports the longest unit and
+ * kvs_unit_len one unit; kvs_prefill_attention refuses a ragged slot (STATE).  One copy and two
+ * kernels on `stream`.  A list that is not ascending or out of range cannot be seen by the host:
+ * the kernel skips the offending entries and sets the device status word to KVS_ERR_INVALID_ARG.
+ * Errors: STATE before bind or on an empty slot; INVALID_ARG for bad sizes or batch != cached batch. */
+kvs_status kvs_evict(kvs_ctx* ctx, int32_t layer, const int32_t* keep, const int32_t* n_keep,
+                     int32_t keep_stride, int32_t batch, void* stream);
+
+/* Rows cached for sequence b, kv-head h of the slot `layer` reads. */
+kvs_status kvs_unit_len(const kvs_ctx* ctx, int32_t layer, int32_t b, int32_t h, int32_t* len);
+
 /* One whole decode step from HOST buffers: for every layer in order, append the
  * layer's new token (own-cache layers only) and run its attention.
  *   q_host:   host, [n_layers][batch][n_q_heads][head_dim], storage type
@@ -233,7 +256,7 @@ kvs_status kvs_decode_attention_static(kvs_ctx* ctx, int32_t layer, const void* 
 
 kvs_status kvs_num_slots(const kvs_ctx* ctx, int32_t* n_slots);
 kvs_status kvs_slot_of_layer(const kvs_ctx* ctx, int32_t layer, int32_t* slot);
-/* Tokens visible to `layer` now (the length of the slot it reads). */
+/* Tokens visible to `layer` now (the length of the slot it reads; of its longest unit if ragged). */
 kvs_status kvs_seq_len(const kvs_ctx* ctx, int32_t layer, int32_t* len);
 /* Rows between consecutive (sequence, head) units of a plane. */
 kvs_status kvs_row_stride(const kvs_ctx* ctx, int32_t* rows);

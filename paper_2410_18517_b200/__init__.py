@@ -86,6 +86,15 @@ class SharedKVCache:
         binding.kvs_prefill_attention(self.ctx, layer, q, out, q.shape[0], q.shape[1], self._stream())
         return out
 
+    def evict(self, layer, keep, n_keep):
+        """keep: device int32 ``[batch][Hkv][stride]`` ascending row lists; n_keep: ``[batch][Hkv]`` counts (host)."""
+        assert keep.is_contiguous() and keep.dtype == self._torch.int32 and keep.ndim == 3
+        counts = [int(x) for x in self._torch.as_tensor(n_keep).reshape(-1).tolist()]
+        binding.kvs_evict(self.ctx, layer, keep, counts, keep.shape[2], keep.shape[0], self._stream())
+
+    def unit_len(self, layer, b, h):
+        return binding.kvs_unit_len(self.ctx, layer, b, h)
+
     def step_host(self, q_host, k_host, v_host, out_host):
         """One decode step over all layers from host tensors (see ``kvs_step_host``)."""
         return binding.kvs_step_host(self.ctx, q_host, k_host, v_host, out_host, q_host.shape[1], self._stream())

@@ -37,6 +37,7 @@ EXPORTS = (
     "kvs_slot_of_layer", "kvs_seq_len", "kvs_row_stride", "kvs_plane_offset", "kvs_stats",
     "kvs_last_device_status", "kvs_set_option", "kvs_last_launch", "kvs_status_string",
     "kvs_read_roof", "kvs_decode_attention_static", "kvs_prefill_attention",
+    "kvs_evict", "kvs_unit_len",
 )
 
 
@@ -53,7 +54,7 @@ class kvs_stats_t(ctypes.Structure):
         ("append_launches", ctypes.c_uint64), ("append_skipped", ctypes.c_uint64),
         ("attention_launches", ctypes.c_uint64), ("combine_launches", ctypes.c_uint64),
         ("kv_bytes_read", ctypes.c_uint64), ("kv_bytes_appended", ctypes.c_uint64),
-        ("prefill_launches", ctypes.c_uint64),
+        ("prefill_launches", ctypes.c_uint64), ("evict_launches", ctypes.c_uint64),
     ]
 
 
@@ -83,6 +84,8 @@ def load() -> ctypes.CDLL:
         "kvs_decode_attention": [vp, i32, vp, vp, i32, vp],
         "kvs_decode_attention_static": [vp, i32, vp, vp, i32, vp, vp],
         "kvs_prefill_attention": [vp, i32, vp, vp, i32, i32, vp],
+        "kvs_evict": [vp, i32, vp, P(i32), i32, i32, vp],
+        "kvs_unit_len": [vp, i32, i32, i32, P(i32)],
         "kvs_step_host": [vp, vp, vp, vp, vp, i32, vp, P(ctypes.c_uint64), P(ctypes.c_uint64)],
         "kvs_num_slots": [vp, P(i32)],
         "kvs_slot_of_layer": [vp, i32, P(i32)],
@@ -172,6 +175,18 @@ def kvs_decode_attention(ctx: int, layer: int, q, out, batch: int, stream: int =
 
 def kvs_prefill_attention(ctx: int, layer: int, q, out, batch: int, n_q: int, stream: int = 0) -> None:
     _check(load().kvs_prefill_attention(ctx, layer, _ptr(q), _ptr(out), batch, n_q, stream), "kvs_prefill_attention")
+
+
+def kvs_evict(ctx: int, layer: int, keep, n_keep, keep_stride: int, batch: int, stream: int = 0) -> None:
+    """keep: device int32 ``[batch][Hkv][keep_stride]``; n_keep: host sequence of batch*Hkv counts."""
+    counts = (ctypes.c_int32 * len(n_keep))(*[int(x) for x in n_keep])
+    _check(load().kvs_evict(ctx, layer, _ptr(keep), counts, keep_stride, batch, stream), "kvs_evict")
+
+
+def kvs_unit_len(ctx: int, layer: int, b: int, h: int) -> int:
+    v = ctypes.c_int32()
+    _check(load().kvs_unit_len(ctx, layer, b, h, ctypes.byref(v)), "kvs_unit_len")
+    return v.value
 
 
 def kvs_decode_attention_static(ctx: int, layer: int, q, out, batch: int, stream: int = 0, device_status=None) -> None:

@@ -32,6 +32,11 @@ struct kvs_ctx {
     std::vector<int32_t> slot_len;
     int cur_batch = 0;         // batch the cached rows were appended for (0 = none yet)
 
+    // Ragged slots: after kvs_evict the units of a slot differ in length; the lengths then live in
+    // a device array (one per slot, in the workspace) with a host mirror.
+    std::vector<char> ragged;                       // per slot
+    std::vector<std::vector<int32_t>> unit_len_host;  // per slot, [max_batch * Hkv]
+
     bool bound = false;
     char* pool = nullptr;
     char* ws = nullptr;
@@ -39,7 +44,7 @@ struct kvs_ctx {
 
     // workspace carve-up (byte offsets)
     size_t off_status = 0, off_part_o = 0, off_part_ml = 0, off_stage_q = 0, off_stage_k = 0, off_stage_v = 0,
-           off_stage_out = 0, ws_bytes = 0;
+           off_stage_out = 0, off_unit_len = 0, off_counts = 0, ws_bytes = 0;
 
     alignas(64) unsigned char tensor_map[128];  // TMA view of the pool (bf16 storage only)
     bool have_tensor_map = false;
@@ -89,6 +94,12 @@ void resolve_map(kvs_ctx* c) {
     c->app_seq_latest.assign(n, 0);
     c->app_seq_prev.assign(n, 0);
     c->app_start_latest.assign(n, 0);
+    c->ragged.assign(n, 0);
+    c->unit_len_host.assign(n, std::vector<int32_t>());
+}
+
+int* unit_len_dev(const kvs_ctx* c, int slot) {
+    return reinterpret_cast<int*>(c->ws + c->off_unit_len) + (size_t)slot * c->cfg.max_batch * c->cfg.n_kv_heads;
 }
 
 // Rows of `slot` that no kernel possibly still in flight writes (see kvs_ctx::seq).
@@ -119,6 +130,10 @@ void layout_workspace(kvs_ctx* c) {
     off = align_up(off + L * f.max_batch * f.n_kv_heads * f.head_dim * c->elem, kAlign);
     c->off_stage_out = off;
     off = align_up(off + L * f.max_batch * f.n_q_heads * f.head_dim * sizeof(float), kAlign);
+    c->off_unit_len = off;      // per slot (at most one per layer): int32 [max_batch * Hkv]
+    off = align_up(off + L * units * sizeof(int32_t), kAlign);
+    c->off_counts = off;        // staging for the kept-row counts of one kvs_evict call
+    off = align_up(off + units * sizeof(int32_t), kAlign);
     c->ws_bytes = off;
 }
 
@@ -179,9 +194,17 @@ kvs_status do_append(kvs_ctx* c, int layer, const void* k, const void* v, int ba
     const int slot = c->slot_of_layer[layer];
     char* kp = c->pool + (size_t)(2 * slot) * c->plane_bytes;
     char* vp = kp + c->plane_bytes;
+    const bool rag = c->ragged[slot] != 0;
     if (kvs::launch_append(k, v, kp, vp, batch, n_new, c->cfg.n_kv_heads, c->row_bytes, c->row_stride,
-                           c->slot_len[slot], c->opt_pdl != 0, st) != cudaSuccess)
+                           c->slot_len[slot], rag ? unit_len_dev(c, slot) : nullptr, c->opt_pdl != 0, st) != cudaSuccess)
         return KVS_ERR_CUDA;
+    if (rag) {
+        const int units = batch * c->cfg.n_kv_heads;
+        if (kvs::launch_add_len(unit_len_dev(c, slot), n_new, units, c->opt_pdl != 0, st) != cudaSuccess)
+            return KVS_ERR_CUDA;
+        for (int u = 0; u < units; ++u) c->unit_len_host[slot][u] += n_new;
+        c->seq += 1;
+    }
     c->seq += 1;
     c->app_seq_prev[slot] = c->app_seq_latest[slot];
     c->app_seq_latest[slot] = c->seq;
@@ -212,6 +235,7 @@ kvs_status do_attention(kvs_ctx* c, int layer, const void* q, float* out, int ba
     a.scale_log2 = c->scale * 1.4426950408889634f;
     a.programmatic = c->opt_pdl != 0;
     a.safe_rows = safe_rows_of(c, slot);
+    a.unit_len = c->ragged[slot] ? unit_len_dev(c, slot) : nullptr;
     c->seq += 2;                       // split-K kernel, then combine
     c->last_splitk_seq = c->seq - 1;
     kvs::DecodePlan plan;
@@ -231,7 +255,13 @@ kvs_status do_attention(kvs_ctx* c, int layer, const void* q, float* out, int ba
     c->last_plan = plan;
     c->stats.attention_launches += 1;
     c->stats.combine_launches += 1;
-    c->stats.kv_bytes_read += 2ull * a.units * a.n * c->row_bytes;
+    if (c->ragged[slot]) {
+        unsigned long long rows = 0;
+        for (int u = 0; u < a.units; ++u) rows += c->unit_len_host[slot][u];
+        c->stats.kv_bytes_read += 2ull * rows * c->row_bytes;
+    } else {
+        c->stats.kv_bytes_read += 2ull * a.units * a.n * c->row_bytes;
+    }
     return KVS_OK;
 }
 
@@ -338,6 +368,7 @@ kvs_status kvs_bind_memory(kvs_ctx* ctx, void* pool, size_t pool_bytes, void* wo
     ctx->ws = static_cast<char*>(workspace);
     ctx->bound = true;
     for (auto& x : ctx->slot_len) x = 0;
+    for (auto& x : ctx->ragged) x = 0;
     ctx->cur_batch = 0;
     // the device was idle a moment ago: nothing of this context is in flight
     for (auto& x : ctx->app_seq_latest) x = 0;
@@ -348,6 +379,7 @@ kvs_status kvs_bind_memory(kvs_ctx* ctx, void* pool, size_t pool_bytes, void* wo
 
 kvs_status kvs_reset(kvs_ctx* ctx) {
     if (!ctx) return KVS_ERR_INVALID_ARG;
+    for (auto& x : ctx->ragged) x = 0;
     for (auto& x : ctx->slot_len) x = 0;
     ctx->cur_batch = 0;
     return KVS_OK;
@@ -385,7 +417,7 @@ kvs_status kvs_prefill_attention(kvs_ctx* ctx, int32_t layer, const void* q, flo
     if (((uintptr_t)q % 16) != 0 || ((uintptr_t)out % 16) != 0) return KVS_ERR_INVALID_ARG;
     const int slot = ctx->slot_of_layer[layer];
     const int n = ctx->slot_len[slot];
-    if (n == 0) return KVS_ERR_STATE;
+    if (n == 0 || ctx->ragged[slot]) return KVS_ERR_STATE;   // positions are undefined once rows were evicted
     if (batch > ctx->cur_batch || n_q > n) return KVS_ERR_INVALID_ARG;
     DeviceGuard guard(ctx->cfg.device);
     if (!guard.ok) return KVS_ERR_CUDA;
@@ -400,6 +432,58 @@ kvs_status kvs_prefill_attention(kvs_ctx* ctx, int32_t layer, const void* q, flo
     ctx->last_splitk_seq = ctx->seq;
     ctx->stats.prefill_launches += 1;
     ctx->stats.kv_bytes_read += 0;  // prefill is compute-bound; its K/V reads are not counted as decode traffic
+    return KVS_OK;
+}
+
+kvs_status kvs_evict(kvs_ctx* ctx, int32_t layer, const int32_t* keep, const int32_t* n_keep, int32_t keep_stride,
+                     int32_t batch, void* stream) {
+    if (!ctx || !keep || !n_keep) return KVS_ERR_INVALID_ARG;
+    if (!ctx->bound) return KVS_ERR_STATE;
+    if (layer < 0 || layer >= ctx->cfg.n_layers || keep_stride < 1) return KVS_ERR_INVALID_ARG;
+    if (ctx->share_map[layer] != layer) return KVS_ERR_INVALID_ARG;   // a sharing layer has no cache of its own
+    const int slot = ctx->slot_of_layer[layer];
+    if (ctx->slot_len[slot] == 0) return KVS_ERR_STATE;
+    if (batch < 1 || batch != ctx->cur_batch) return KVS_ERR_INVALID_ARG;
+    const int units = batch * ctx->cfg.n_kv_heads;
+    int longest = 0;
+    for (int u = 0; u < units; ++u) {
+        const int have = ctx->ragged[slot] ? ctx->unit_len_host[slot][u] : ctx->slot_len[slot];
+        if (n_keep[u] < 1 || n_keep[u] > have || n_keep[u] > keep_stride) return KVS_ERR_INVALID_ARG;
+        longest = n_keep[u] > longest ? n_keep[u] : longest;
+    }
+    DeviceGuard guard(ctx->cfg.device);
+    if (!guard.ok) return KVS_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int* counts = reinterpret_cast<int*>(ctx->ws + ctx->off_counts);
+    int* lens = unit_len_dev(ctx, slot);
+    if (cudaMemcpyAsync(counts, n_keep, sizeof(int32_t) * units, cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return KVS_ERR_CUDA;
+    char* kp = ctx->pool + (size_t)(2 * slot) * ctx->plane_bytes;
+    const bool pdl = ctx->opt_pdl != 0;
+    if (kvs::launch_evict(kp, kp + ctx->plane_bytes, keep, counts, ctx->ragged[slot] ? lens : nullptr,
+                          ctx->slot_len[slot], units, keep_stride, ctx->row_bytes, ctx->row_stride,
+                          reinterpret_cast<int*>(ctx->ws + ctx->off_status), false, st) != cudaSuccess ||
+        kvs::launch_set_len(lens, counts, units, pdl, st) != cudaSuccess)
+        return KVS_ERR_CUDA;
+    ctx->unit_len_host[slot].assign((size_t)ctx->cfg.max_batch * ctx->cfg.n_kv_heads, 0);
+    for (int u = 0; u < units; ++u) ctx->unit_len_host[slot][u] = n_keep[u];
+    ctx->ragged[slot] = 1;
+    ctx->slot_len[slot] = longest;
+    // every row of the slot may just have moved: nothing of it may be fetched early
+    ctx->seq += 2;
+    ctx->app_seq_prev[slot] = ctx->seq;
+    ctx->app_seq_latest[slot] = ctx->seq;
+    ctx->app_start_latest[slot] = 0;
+    ctx->stats.evict_launches += 1;
+    return KVS_OK;
+}
+
+kvs_status kvs_unit_len(const kvs_ctx* ctx, int32_t layer, int32_t b, int32_t h, int32_t* len) {
+    if (!ctx || !len || layer < 0 || layer >= ctx->cfg.n_layers) return KVS_ERR_INVALID_ARG;
+    if (b < 0 || b >= ctx->cfg.max_batch || h < 0 || h >= ctx->cfg.n_kv_heads) return KVS_ERR_INVALID_ARG;
+    const int slot = ctx->slot_of_layer[layer];
+    *len = ctx->ragged[slot] ? ctx->unit_len_host[slot][(size_t)b * ctx->cfg.n_kv_heads + h]
+                             : (b < ctx->cur_batch ? ctx->slot_len[slot] : 0);
     return KVS_OK;
 }
 
@@ -673,6 +757,7 @@ kvs_status kvs_decode_attention_static(kvs_ctx* ctx, int32_t layer, const void* 
     a.scale_log2 = c->scale * 1.4426950408889634f;
     a.programmatic = false;            // plain launches: starts after everything before it on the stream
     a.safe_rows = 0;
+    a.unit_len = c->ragged[slot] ? unit_len_dev(c, slot) : nullptr;
     c->seq += 2;
     c->last_splitk_seq = c->seq - 1;
     if (use_mma) {

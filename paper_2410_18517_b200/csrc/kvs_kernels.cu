@@ -17,7 +17,7 @@ namespace kvs {
 __global__ void __launch_bounds__(256) kv_append_kernel(const uint4* __restrict__ k, const uint4* __restrict__ v,
                                                         uint4* __restrict__ kplane, uint4* __restrict__ vplane,
                                                         long long total_vecs, int n_new, int Hkv, int row_vecs,
-                                                        int row_stride, int len0) {
+                                                        int row_stride, int len0, const int* __restrict__ unit_len) {
     pdl_launch_dependents();
     pdl_wait();
     const uint4* __restrict__ src = blockIdx.y == 0 ? k : v;
@@ -30,19 +30,91 @@ __global__ void __launch_bounds__(256) kv_append_kernel(const uint4* __restrict_
         r /= Hkv;
         const int t = (int)(r % n_new);
         const long long b = r / n_new;
-        const long long drow = (b * Hkv + h) * (long long)row_stride + len0 + t;
+        const int first = unit_len ? unit_len[b * Hkv + h] : len0;   // ragged slots append per unit
+        const long long drow = (b * Hkv + h) * (long long)row_stride + first + t;
         dst[drow * row_vecs + c] = src[idx];
     }
 }
 
 cudaError_t launch_append(const void* k, const void* v, void* kplane, void* vplane, int B, int n_new, int Hkv,
-                          int row_bytes, int row_stride, int len0, bool programmatic, cudaStream_t stream) {
+                          int row_bytes, int row_stride, int len0, const int* unit_len, bool programmatic, cudaStream_t stream) {
     const int row_vecs = row_bytes / 16;
     const long long total = (long long)B * n_new * Hkv * row_vecs;
     const long long blocks = std::min<long long>((total + 255) / 256, 148 * 16);
     dim3 grid((unsigned)blocks, 2);
     return launch_kernel(kv_append_kernel, grid, dim3(256), 0, stream, programmatic, (const uint4*)k, (const uint4*)v,
-                         (uint4*)kplane, (uint4*)vplane, total, n_new, Hkv, row_vecs, row_stride, len0);
+                         (uint4*)kplane, (uint4*)vplane, total, n_new, Hkv, row_vecs, row_stride, len0, unit_len);
+}
+
+// --------------------------------------------------------------------------------------
+// Eviction: keep only the listed rows of every unit, moved to the front in order.  One block
+// per (unit, K or V plane); rows go through shared memory 64 at a time, and because the list
+// is strictly ascending (keep[j] >= j) a later chunk never reads a row an earlier chunk wrote.
+// A list that is not ascending or points past the unit's length sets the status word to 1
+// (invalid argument) and the offending entry is treated as "keep the row already there".
+// --------------------------------------------------------------------------------------
+constexpr int kEvictChunk = 64;
+
+__global__ void __launch_bounds__(256) kv_evict_kernel(uint4* __restrict__ kplane, uint4* __restrict__ vplane,
+                                                       const int* __restrict__ keep, const int* __restrict__ counts,
+                                                       const int* __restrict__ old_len, int old_uniform, int keep_stride,
+                                                       int row_vecs, int row_stride, int* status) {
+    __shared__ uint4 buf[kEvictChunk * 32];   // 64 rows of up to 512 bytes
+    pdl_launch_dependents();
+    pdl_wait();
+    const int u = blockIdx.x;
+    uint4* base = (blockIdx.y == 0 ? kplane : vplane) + (long long)u * row_stride * row_vecs;
+    const int cnt = counts[u];
+    const int old = old_len ? old_len[u] : old_uniform;
+    const int* list = keep + (long long)u * keep_stride;
+    for (int c0 = 0; c0 < cnt; c0 += kEvictChunk) {
+        const int rows = min(kEvictChunk, cnt - c0);
+        for (int idx = threadIdx.x; idx < rows * row_vecs; idx += blockDim.x) {
+            const int j = idx / row_vecs, v = idx - j * row_vecs;
+            int src = list[c0 + j];
+            const bool bad = src >= old || src < c0 + j || (c0 + j > 0 && list[c0 + j - 1] >= src);
+            if (bad) {
+                if (v == 0) atomicExch(status, 1);
+                src = c0 + j;
+            }
+            buf[idx] = base[(long long)src * row_vecs + v];
+        }
+        __syncthreads();
+        for (int idx = threadIdx.x; idx < rows * row_vecs; idx += blockDim.x) base[(long long)c0 * row_vecs + idx] = buf[idx];
+        __syncthreads();
+    }
+}
+
+__global__ void set_len_kernel(int* __restrict__ unit_len, const int* __restrict__ counts, int units) {
+    pdl_launch_dependents();
+    pdl_wait();
+    const int u = blockIdx.x * blockDim.x + threadIdx.x;
+    if (u < units) unit_len[u] = counts[u];
+}
+
+__global__ void add_len_kernel(int* __restrict__ unit_len, int delta, int units) {
+    pdl_launch_dependents();
+    pdl_wait();
+    const int u = blockIdx.x * blockDim.x + threadIdx.x;
+    if (u < units) unit_len[u] += delta;
+}
+
+cudaError_t launch_evict(void* kplane, void* vplane, const int* keep, const int* counts, const int* old_len,
+                         int old_uniform, int units, int keep_stride, int row_bytes, int row_stride, int* status,
+                         bool programmatic, cudaStream_t stream) {
+    return launch_kernel(kv_evict_kernel, dim3(units, 2), dim3(256), 0, stream, programmatic, (uint4*)kplane,
+                         (uint4*)vplane, keep, counts, old_len, old_uniform, keep_stride, row_bytes / 16, row_stride,
+                         status);
+}
+
+cudaError_t launch_set_len(int* unit_len, const int* counts, int units, bool programmatic, cudaStream_t stream) {
+    return launch_kernel(set_len_kernel, dim3((units + 127) / 128), dim3(128), 0, stream, programmatic, unit_len, counts,
+                         units);
+}
+
+cudaError_t launch_add_len(int* unit_len, int delta, int units, bool programmatic, cudaStream_t stream) {
+    return launch_kernel(add_len_kernel, dim3((units + 127) / 128), dim3(128), 0, stream, programmatic, unit_len, delta,
+                         units);
 }
 
 // --------------------------------------------------------------------------------------
@@ -141,6 +213,7 @@ struct ScalarKernelArgs {
     long long T;
     float scale_log2;
     int safe_rows;  // rows of every unit that no kernel possibly still running writes
+    const int* unit_len;  // per-unit row counts of a ragged slot, or nullptr (then n holds for all)
 };
 
 template <typename T, int D, int G>
@@ -185,12 +258,17 @@ __global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G>::MIN_BLOC
                 const long long u = gt / a.tpu;
                 const int ti = (int)(gt - u * a.tpu);
                 const int row0 = ti * TN;
-                const int rows = min(TN, a.n - row0);
+                const int n_u = a.unit_len ? a.unit_len[u] : a.n;
+                const int rows = max(0, min(TN, n_u - row0));     // a ragged unit may end before this tile
                 const uint32_t bytes = (uint32_t)rows * RB;
                 const bool with_q = (gt == t0) || (ti == 0);
                 unsigned char* sb = stage_base + st * S::STAGE_BYTES;
-                if (arm) mbar_arrive_expect_tx(&full_bar[st], 2 * bytes + (with_q ? S::QBYTES : 0));
-                if (kv) {
+                if (arm) {
+                    const uint32_t total = 2 * bytes + (with_q ? S::QBYTES : 0);
+                    if (total) mbar_arrive_expect_tx(&full_bar[st], total);
+                    else mbar_arrive(&full_bar[st]);
+                }
+                if (kv && bytes) {
                     const long long off = (u * a.row_stride + row0) * (long long)RB;
                     bulk_g2s(sb, a.kplane + off, bytes, &full_bar[st]);
                     bulk_g2s(sb + kTileBytes, a.vplane + off, bytes, &full_bar[st]);
@@ -242,6 +320,7 @@ __global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G>::MIN_BLOC
         const long long u = gt / a.tpu;
         const int ti0 = (int)(gt - u * a.tpu);
         const int piece_tiles = (int)min((long long)(a.tpu - ti0), t1 - gt);
+        const int n_u = a.unit_len ? a.unit_len[u] : a.n;
 
         float qf[G][EPL];
         float m[G], lsum[G], acc[G][EPL];
@@ -268,7 +347,12 @@ __global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G>::MIN_BLOC
                     for (int e = 0; e < EPL; ++e) qf[g][e] *= a.scale_log2;
                 }
             }
-            const int valid = min(TN, a.n - (ti0 + k) * TN);
+            const int valid = min(TN, n_u - (ti0 + k) * TN);   // <= 0 for tiles past a ragged unit's end
+            if (valid <= 0) {
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&empty_bar[st]);
+                continue;
+            }
 
             // scores: partial dot products of this lane's 16-byte chunk
             float s[G][R];
@@ -456,7 +540,8 @@ cudaError_t launch_decode_scalar(const DecodeArgs& a, const DecodePlan& plan, cu
     ka.tpu = plan.tpu;
     ka.T = plan.T;
     ka.scale_log2 = a.scale_log2;
-    ka.safe_rows = a.programmatic ? a.safe_rows : 0;
+    ka.safe_rows = (a.programmatic && !a.unit_len) ? a.safe_rows : 0;
+    ka.unit_len = a.unit_len;
     const bool pdl = a.programmatic;
     if (a.dtype == 0) {
         if (a.D == 128) return launch_scalar_groups<__nv_bfloat16, 128>(a.G, ka, plan.NC, pdl, stream);

@@ -35,6 +35,7 @@ struct DecodeArgs {
     int D;
     int dtype;            // 0 bf16, 1 f32
     float scale_log2;     // softmax scale * log2(e)
+    const int* unit_len;  // device, [units]: rows cached per unit when units differ (else nullptr and n holds)
     int safe_rows;        // rows per unit that no kernel possibly still in flight is writing
     bool programmatic;    // launch with programmatic stream serialization (early start, explicit wait)
 };
@@ -68,7 +69,17 @@ cudaError_t launch_prefill(const void* q, float* out, int* status, const void* p
                            cudaStream_t stream);
 
 cudaError_t launch_append(const void* k, const void* v, void* kplane, void* vplane, int B, int n_new, int Hkv,
-                          int row_bytes, int row_stride, int len0, bool programmatic, cudaStream_t stream);
+                          int row_bytes, int row_stride, int len0, const int* unit_len, bool programmatic, cudaStream_t stream);
+
+// Ragged slots (rows evicted by an outside intra-layer method).
+//   launch_evict:   per unit u, rows keep[u*keep_stride + j], j < counts[u], move to rows 0..counts[u]-1
+//                   (K and V planes); old lengths are old_len[u] or, if old_len is nullptr, old_uniform
+//   launch_set_len: unit_len[u] = counts[u];  launch_add_len: unit_len[u] += delta
+cudaError_t launch_evict(void* kplane, void* vplane, const int* keep, const int* counts, const int* old_len,
+                         int old_uniform, int units, int keep_stride, int row_bytes, int row_stride, int* status,
+                         bool programmatic, cudaStream_t stream);
+cudaError_t launch_set_len(int* unit_len, const int* counts, int units, bool programmatic, cudaStream_t stream);
+cudaError_t launch_add_len(int* unit_len, int delta, int units, bool programmatic, cudaStream_t stream);
 cudaError_t launch_decode_scalar(const DecodeArgs& a, const DecodePlan& plan, cudaStream_t stream);
 cudaError_t launch_combine(const DecodeArgs& a, const DecodePlan& plan, cudaStream_t stream);
 cudaError_t launch_read_roof(const void* src, size_t bytes, unsigned long long* checksum, int sm_count,

@@ -89,6 +89,7 @@ struct MmaKernelArgs {
     long long vrow0;
     float scale_log2;
     int safe_rows;  // rows of every unit that no kernel possibly still running writes
+    const int* unit_len;  // per-unit row counts of a ragged slot, or nullptr (then n holds for all)
 };
 
 template <int D, int G>
@@ -131,9 +132,15 @@ __global__ void __launch_bounds__(kMmaThreads, 2)
                 const long long u = gt / a.tpu;
                 const int ti = (int)(gt - u * a.tpu);
                 const bool with_q = (gt == t0) || (ti == 0);
+                const int n_u = a.unit_len ? a.unit_len[u] : a.n;
+                const bool have = ti * TN < n_u;                  // a ragged unit may end before this tile
                 unsigned char* sb = smem + st * S::STAGE_BYTES;
-                if (arm) mbar_arrive_expect_tx(&full_bar[st], 2 * kMmaTileBytes + (with_q ? QBYTES : 0));
-                if (kv) {
+                if (arm) {
+                    const uint32_t total = (have ? 2 * kMmaTileBytes : 0) + (with_q ? QBYTES : 0);
+                    if (total) mbar_arrive_expect_tx(&full_bar[st], total);
+                    else mbar_arrive(&full_bar[st]);
+                }
+                if (kv && have) {
                     const long long row = u * a.row_stride + (long long)ti * TN;
 #pragma unroll
                     for (int h = 0; h < S::HALVES; ++h) {
@@ -186,6 +193,7 @@ __global__ void __launch_bounds__(kMmaThreads, 2)
         const long long u = gt / a.tpu;
         const int ti0 = (int)(gt - u * a.tpu);
         const int piece_tiles = (int)min((long long)(a.tpu - ti0), t1 - gt);
+        const int n_u = a.unit_len ? a.unit_len[u] : a.n;
 
         uint32_t qa[KSTEPS][2];
         float o[NB][2];
@@ -208,7 +216,12 @@ __global__ void __launch_bounds__(kMmaThreads, 2)
                     qa[s][1] = row < G ? qs[row * (D / 2) + s * 8 + 4 + quad] : 0u;
                 }
             }
-            const int valid = a.n - (ti0 + k) * TN;  // rows of this tile that exist (may exceed TN)
+            const int valid = n_u - (ti0 + k) * TN;  // rows of this tile that exist (may exceed TN or be <= 0)
+            if (valid <= 0) {   // tile past the end of a ragged unit: nothing was loaded, nothing to add
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&empty_bar[st]);
+                continue;
+            }
 
 #pragma unroll
             for (int blk = 0; blk < BPW; ++blk) {
@@ -416,7 +429,8 @@ cudaError_t launch_decode_mma(const DecodeArgs& a, const DecodePlan& plan, const
     ka.krow0 = krow0;
     ka.vrow0 = vrow0;
     ka.scale_log2 = a.scale_log2;
-    ka.safe_rows = a.programmatic ? a.safe_rows : 0;
+    ka.safe_rows = (a.programmatic && !a.unit_len) ? a.safe_rows : 0;
+    ka.unit_len = a.unit_len;
     const CUtensorMap& tm = *reinterpret_cast<const CUtensorMap*>(tensor_map);
     if (a.D == 128) return launch_groups<128>(a.G, tm, ka, plan.NC, a.programmatic, stream);
     if (a.D == 64) return launch_groups<64>(a.G, tm, ka, plan.NC, a.programmatic, stream);
