@@ -11,6 +11,7 @@ from .oracle import (  # noqa: F401
     attend_units,
     build,
     combine_partials,
+    mean_cosine,
     num_threads,
     partial_unit,
     slot_table,

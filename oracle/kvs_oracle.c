@@ -362,6 +362,65 @@ int oracle_get_cache(const oracle_state *st, int l, double *K_out, double *V_out
     return 0;
 }
 
+/* ---- the data-parallel part of strategy searching (Section 3.1) --------------
+ * "KV cache similarity": the cache of every layer is averaged over the calibration
+ * samples (here: over the B sequences held), keys and values are each flattened,
+ * and the Euclidean distance between the representations of any two layers is
+ * taken.  Reading of the ambiguous "average the keys and values separately": the
+ * representation of a layer is the sample-mean of its keys, flattened, followed by
+ * the sample-mean of its values, flattened; the distance is the 2-norm of the
+ * difference of two such vectors.  All layers must hold equally long, un-evicted
+ * caches.  dist is [L][L], symmetric, zero diagonal.  Returns 0 or -1.          */
+int oracle_layer_distances(const oracle_state *st, double *dist) {
+    if (!st || !dist) return -1;
+    const int L = st->L, U = st->B * st->Hkv, B = st->B, Hkv = st->Hkv, D = st->D;
+    const int n = uniform_len(st, 0);
+    if (n <= 0) return -1;
+    for (int l = 1; l < L; ++l) if (uniform_len(st, l) != n) return -1;
+    (void)U;
+    const size_t P = (size_t)Hkv * n * D;            /* elements of one flattened K (or V) */
+    double *rep = (double *)calloc((size_t)L * 2 * P, sizeof(double));
+    for (int l = 0; l < L; ++l)
+        for (int h = 0; h < Hkv; ++h)
+            for (size_t e = 0; e < (size_t)n * D; ++e) {
+                double sk = 0.0, sv = 0.0;
+                for (int b = 0; b < B; ++b) {
+                    sk += st->K[l][b * Hkv + h][e];
+                    sv += st->V[l][b * Hkv + h][e];
+                }
+                rep[((size_t)l * 2 + 0) * P + (size_t)h * n * D + e] = sk / B;
+                rep[((size_t)l * 2 + 1) * P + (size_t)h * n * D + e] = sv / B;
+            }
+    for (int i = 0; i < L; ++i)
+        for (int j = 0; j < L; ++j) {
+            double s = 0.0;
+            for (size_t e = 0; e < 2 * P; ++e) {
+                double d = rep[(size_t)i * 2 * P + e] - rep[(size_t)j * 2 * P + e];
+                s += d * d;
+            }
+            dist[(size_t)i * L + j] = sqrt(s);
+        }
+    free(rep);
+    return 0;
+}
+
+/* "Avg_Cos_Sim" (Algorithm 1, Section 3.1): the last-layer output representations of
+ * two models on the calibration sentences, a and b, each [S][dim], are averaged over the
+ * S sentences and the cosine similarity of the two averaged vectors is returned.        */
+double oracle_mean_cosine(const double *a, const double *b, int S, long long dim) {
+    double dot = 0.0, na = 0.0, nb = 0.0;
+    for (long long e = 0; e < dim; ++e) {
+        double ma = 0.0, mb = 0.0;
+        for (int s = 0; s < S; ++s) {
+            ma += a[(size_t)s * dim + e];
+            mb += b[(size_t)s * dim + e];
+        }
+        ma /= S; mb /= S;
+        dot += ma * mb; na += ma * ma; nb += mb * mb;
+    }
+    return dot / (sqrt(na) * sqrt(nb));
+}
+
 /* Many independent units at once (the benchmark's CPU-baseline leg and the
  * sampled-unit parity checks at sizes the stateful oracle cannot hold):
  * unit u has query q[u][D], keys K[u][n][D], values V[u][n][D].              */

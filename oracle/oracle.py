@@ -67,6 +67,10 @@ def _load():
     lib.oracle_unit_len.restype = ctypes.c_int
     lib.oracle_evict.argtypes = [ctypes.c_void_p, ctypes.c_int, _ip, _ip, ctypes.c_int]
     lib.oracle_evict.restype = ctypes.c_int
+    lib.oracle_layer_distances.argtypes = [ctypes.c_void_p, _dp]
+    lib.oracle_layer_distances.restype = ctypes.c_int
+    lib.oracle_mean_cosine.argtypes = [_dp, _dp, ctypes.c_int, ctypes.c_longlong]
+    lib.oracle_mean_cosine.restype = ctypes.c_double
     lib.oracle_get_cache.argtypes = [ctypes.c_void_p, ctypes.c_int, _dp, _dp]
     lib.oracle_get_cache.restype = ctypes.c_int
     _lib = lib
@@ -128,6 +132,13 @@ def combine_partials(o, m, l) -> np.ndarray:
     out = np.empty(D, dtype=np.float64)
     _load().oracle_combine_partials(S, D, _p(o), _p(m), _p(l), _p(out))
     return out
+
+
+def mean_cosine(a, b) -> float:
+    """Cosine similarity of the sentence-means of ``a[S][dim]`` and ``b[S][dim]``."""
+    a, b = _f64(a), _f64(b)
+    assert a.ndim == 2 and a.shape == b.shape
+    return float(_load().oracle_mean_cosine(_p(a), _p(b), a.shape[0], a.shape[1]))
 
 
 def slot_table(share_map):
@@ -227,6 +238,13 @@ class Oracle:
         rc = self._lib.oracle_evict(self._h, l, keep.ctypes.data_as(_ip), n_keep.ctypes.data_as(_ip), keep.shape[2])
         if rc != 0:
             raise RuntimeError("oracle_evict rejected its arguments")
+
+    def layer_distances(self) -> np.ndarray:
+        """``[L][L]`` Euclidean distances between the sample-mean K/V representations of the layers."""
+        d = np.empty((self.L, self.L), dtype=np.float64)
+        if self._lib.oracle_layer_distances(self._h, _p(d)) != 0:
+            raise RuntimeError("oracle_layer_distances needs equally long, un-evicted caches")
+        return d
 
     def cache(self, l):
         """Layer l's cache as (K, V), each ``[B][Hkv][len][D]`` float64."""

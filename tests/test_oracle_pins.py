@@ -453,3 +453,57 @@ def test_keeping_everything_changes_nothing_and_bad_lists_are_rejected():
     o.evict(0, [[[0, 1, 2, 0, 0, 0], [0, 1, 0, 0, 0, 0]]], [[3, 2]])
     with pytest.raises(RuntimeError):
         o.layer_prefill(0, rng.standard_normal((B, 1, Hq, D)))
+
+
+# ---------------------------------------------------------------- strategy-search reductions
+def test_layer_distances_against_numpy_and_metric_properties():
+    L, Hq, Hkv, D, B, n = 5, 2, 2, 4, 6, 7
+    rng = np.random.default_rng(13)
+    o = oracle.Oracle(L, Hq, Hkv, D, B, np.arange(L))
+    ks = rng.standard_normal((L, B, n, Hkv, D))
+    vs = rng.standard_normal((L, B, n, Hkv, D))
+    ks[3], vs[3] = ks[1], vs[1]                       # two identical layers
+    ks[4], vs[4] = 2.0 * ks[0], 2.0 * vs[0]           # one layer is twice another
+    for l in range(L):
+        o.layer_forward(l, None, ks[l], vs[l])
+    d = o.layer_distances()
+    rep = np.concatenate([ks.mean(axis=1).reshape(L, -1), vs.mean(axis=1).reshape(L, -1)], axis=1)
+    ref = np.linalg.norm(rep[:, None, :] - rep[None, :, :], axis=2)
+    np.testing.assert_allclose(d, ref, atol=1e-12)
+    assert np.all(np.diag(d) == 0) and np.array_equal(d, d.T) and d[1, 3] == 0
+    assert d[0, 4] == pytest.approx(np.linalg.norm(rep[0]), abs=1e-12)            # |2x - x| = |x|
+    for i in range(L):
+        for j in range(L):
+            for k in range(L):
+                assert d[i, j] <= d[i, k] + d[k, j] + 1e-12
+    # the mean is over sequences: permuting them changes nothing
+    o2 = oracle.Oracle(L, Hq, Hkv, D, B, np.arange(L))
+    perm = rng.permutation(B)
+    for l in range(L):
+        o2.layer_forward(l, None, ks[l][perm], vs[l][perm])
+    np.testing.assert_allclose(o2.layer_distances(), d, atol=1e-12)
+
+
+def test_layer_distances_need_equal_unevicted_caches():
+    o = oracle.Oracle(2, 1, 1, 4, 1, [0, 1])
+    o.layer_forward(0, None, RNG.standard_normal((1, 3, 1, 4)), RNG.standard_normal((1, 3, 1, 4)))
+    with pytest.raises(RuntimeError):
+        o.layer_distances()                           # layer 1 is empty
+
+
+def test_mean_cosine_against_numpy_and_closed_forms():
+    rng = np.random.default_rng(17)
+    a, b = rng.standard_normal((5, 33)), rng.standard_normal((5, 33))
+    ma, mb = a.mean(0), b.mean(0)
+    assert oracle.mean_cosine(a, b) == pytest.approx(ma @ mb / np.linalg.norm(ma) / np.linalg.norm(mb), abs=1e-14)
+    assert oracle.mean_cosine(a, a) == pytest.approx(1.0, abs=1e-14)
+    assert oracle.mean_cosine(a, -3.0 * a) == pytest.approx(-1.0, abs=1e-14)
+    assert oracle.mean_cosine(a, 7.5 * b) == pytest.approx(oracle.mean_cosine(a, b), abs=1e-14)
+    e0, e1 = np.zeros((2, 4)), np.zeros((2, 4))
+    e0[:, 0], e1[:, 1] = 1.0, 1.0
+    assert oracle.mean_cosine(e0, e1) == 0.0
+    # only the mean matters: sentences whose deviations cancel do not change the result
+    dev = rng.standard_normal((1, 33))
+    a2 = np.concatenate([a + dev, a - dev])
+    b2 = np.concatenate([b, b])
+    assert oracle.mean_cosine(a2, b2) == pytest.approx(oracle.mean_cosine(a, b), abs=1e-13)
