@@ -80,6 +80,7 @@ typedef struct {
     uint64_t kv_bytes_appended;   /* 2*B*Hkv*n_new*D*elem summed over launched appends       */
     uint64_t prefill_launches;    /* tensor-core prefill kernels launched                    */
     uint64_t evict_launches;      /* kvs_evict calls that launched                           */
+    uint64_t search_launches;     /* kernels launched by kvs_layer_distances / kvs_mean_cosine */
 } kvs_stats_t;
 
 /* Tuning knobs for kvs_set_option.  Defaults are chosen by the library. */
@@ -200,6 +201,26 @@ kvs_status kvs_evict(kvs_ctx* ctx, int32_t layer, const int32_t* keep, const int
 
 /* Rows cached for sequence b, kv-head h of the slot `layer` reads. */
 kvs_status kvs_unit_len(const kvs_ctx* ctx, int32_t layer, int32_t b, int32_t h, int32_t* len);
+
+/* ---- the data-parallel reductions of strategy searching (Section 3.1, Algorithm 1) -------- */
+
+/* Euclidean distances between the KV caches of every pair of layers.  The caches currently in
+ * the pool play the calibration run: the first `batch` cached sequences are the samples.  Per
+ * layer, keys and values are averaged over the samples, each flattened, and laid end to end
+ * (reading of the paper's "average the keys and values separately"); dist[i][j] is the 2-norm of
+ * the difference of layers i and j's vectors (a sharing layer has its source's cache: distance 0).
+ *   dist: device, float32 [n_layers][n_layers], symmetric, zero diagonal.
+ * Two kernels on `stream`; reads every cached element once.  Sorting the pairs (descending, as
+ * the search does) is left to the caller.
+ * Errors: STATE unless every slot holds the same non-zero number of rows and none is ragged;
+ * INVALID_ARG for batch > cached batch or more than 80 layers.                                */
+kvs_status kvs_layer_distances(kvs_ctx* ctx, int32_t batch, float* dist, void* stream);
+
+/* Cosine similarity of two models' averaged output representations: a and b are device tensors
+ * [n_samples][dim] of the context's storage type (8-byte aligned, dim even); each is averaged
+ * over the samples and *out (device, float32) receives cos(mean a, mean b).  Two kernels.       */
+kvs_status kvs_mean_cosine(kvs_ctx* ctx, const void* a, const void* b, int32_t n_samples, int64_t dim,
+                           float* out, void* stream);
 
 /* One whole decode step from HOST buffers: for every layer in order, append the
  * layer's new token (own-cache layers only) and run its attention.

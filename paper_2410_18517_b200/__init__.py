@@ -29,6 +29,7 @@ class SharedKVCache:
         self.device = torch.device("cuda", device)
         self.dtype = {"bf16": torch.bfloat16, "f32": torch.float32}[dtype]
         self.shape = (n_layers, n_q_heads, n_kv_heads, head_dim)
+        self.max_batch = max_batch
         self.ctx = binding.kvs_create(n_layers, n_q_heads, n_kv_heads, head_dim, max_batch, max_seq,
                                       KVS_BF16 if dtype == "bf16" else KVS_F32, softmax_scale, device)
         try:
@@ -94,6 +95,30 @@ class SharedKVCache:
 
     def unit_len(self, layer, b, h):
         return binding.kvs_unit_len(self.ctx, layer, b, h)
+
+    def layer_distances(self, batch=None):
+        """float32 ``[L][L]`` distances between the layers' sample-mean K/V representations."""
+        torch = self._torch
+        L = self.shape[0]
+        dist = torch.empty(L, L, dtype=torch.float32, device=self.device)
+        if batch is None:
+            batch = self._cached_batch()
+        binding.kvs_layer_distances(self.ctx, batch, dist, self._stream())
+        return dist
+
+    def _cached_batch(self):
+        b = 0
+        while b < self.max_batch and self.unit_len(0, b, 0) > 0:
+            b += 1
+        return b
+
+    def mean_cosine(self, a, b):
+        """cos(mean over samples of a, mean over samples of b) for ``[S][dim]`` device tensors (float32 scalar tensor)."""
+        torch = self._torch
+        assert a.shape == b.shape and a.ndim == 2 and a.is_contiguous() and b.is_contiguous() and a.dtype == self.dtype
+        out = torch.empty(1, dtype=torch.float32, device=self.device)
+        binding.kvs_mean_cosine(self.ctx, a, b, a.shape[0], a.shape[1], out, self._stream())
+        return out
 
     def step_host(self, q_host, k_host, v_host, out_host):
         """One decode step over all layers from host tensors (see ``kvs_step_host``)."""

@@ -37,7 +37,7 @@ EXPORTS = (
     "kvs_slot_of_layer", "kvs_seq_len", "kvs_row_stride", "kvs_plane_offset", "kvs_stats",
     "kvs_last_device_status", "kvs_set_option", "kvs_last_launch", "kvs_status_string",
     "kvs_read_roof", "kvs_decode_attention_static", "kvs_prefill_attention",
-    "kvs_evict", "kvs_unit_len",
+    "kvs_evict", "kvs_unit_len", "kvs_layer_distances", "kvs_mean_cosine",
 )
 
 
@@ -55,6 +55,7 @@ class kvs_stats_t(ctypes.Structure):
         ("attention_launches", ctypes.c_uint64), ("combine_launches", ctypes.c_uint64),
         ("kv_bytes_read", ctypes.c_uint64), ("kv_bytes_appended", ctypes.c_uint64),
         ("prefill_launches", ctypes.c_uint64), ("evict_launches", ctypes.c_uint64),
+        ("search_launches", ctypes.c_uint64),
     ]
 
 
@@ -86,6 +87,8 @@ def load() -> ctypes.CDLL:
         "kvs_prefill_attention": [vp, i32, vp, vp, i32, i32, vp],
         "kvs_evict": [vp, i32, vp, P(i32), i32, i32, vp],
         "kvs_unit_len": [vp, i32, i32, i32, P(i32)],
+        "kvs_layer_distances": [vp, i32, vp, vp],
+        "kvs_mean_cosine": [vp, vp, vp, i32, ctypes.c_int64, vp, vp],
         "kvs_step_host": [vp, vp, vp, vp, vp, i32, vp, P(ctypes.c_uint64), P(ctypes.c_uint64)],
         "kvs_num_slots": [vp, P(i32)],
         "kvs_slot_of_layer": [vp, i32, P(i32)],
@@ -187,6 +190,14 @@ def kvs_unit_len(ctx: int, layer: int, b: int, h: int) -> int:
     v = ctypes.c_int32()
     _check(load().kvs_unit_len(ctx, layer, b, h, ctypes.byref(v)), "kvs_unit_len")
     return v.value
+
+
+def kvs_layer_distances(ctx: int, batch: int, dist, stream: int = 0) -> None:
+    _check(load().kvs_layer_distances(ctx, batch, _ptr(dist), stream), "kvs_layer_distances")
+
+
+def kvs_mean_cosine(ctx: int, a, b, n_samples: int, dim: int, out, stream: int = 0) -> None:
+    _check(load().kvs_mean_cosine(ctx, _ptr(a), _ptr(b), n_samples, dim, _ptr(out), stream), "kvs_mean_cosine")
 
 
 def kvs_decode_attention_static(ctx: int, layer: int, q, out, batch: int, stream: int = 0, device_status=None) -> None:

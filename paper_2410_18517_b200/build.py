@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libkvs.so")
-SOURCES = ["kvs_api.cu", "kvs_kernels.cu", "kvs_mma.cu", "kvs_prefill.cu"]
+SOURCES = ["kvs_api.cu", "kvs_kernels.cu", "kvs_mma.cu", "kvs_prefill.cu", "kvs_search.cu"]
 HEADERS = ["kvs_device.cuh", "kvs_kernels.h", os.path.join("..", "..", "include", "kvs.h")]
 
 NVCC_FLAGS = [

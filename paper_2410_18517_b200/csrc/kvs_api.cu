@@ -4,6 +4,7 @@
 
 #include "kvs_kernels.h"
 
+#include <algorithm>
 #include <cmath>
 #include <cstring>
 #include <mutex>
@@ -44,7 +45,7 @@ struct kvs_ctx {
 
     // workspace carve-up (byte offsets)
     size_t off_status = 0, off_part_o = 0, off_part_ml = 0, off_stage_q = 0, off_stage_k = 0, off_stage_v = 0,
-           off_stage_out = 0, off_unit_len = 0, off_counts = 0, ws_bytes = 0;
+           off_stage_out = 0, off_unit_len = 0, off_counts = 0, off_search = 0, ws_bytes = 0;
 
     alignas(64) unsigned char tensor_map[128];  // TMA view of the pool (bf16 storage only)
     bool have_tensor_map = false;
@@ -134,6 +135,12 @@ void layout_workspace(kvs_ctx* c) {
     off = align_up(off + L * units * sizeof(int32_t), kAlign);
     c->off_counts = off;        // staging for the kept-row counts of one kvs_evict call
     off = align_up(off + units * sizeof(int32_t), kAlign);
+    c->off_search = off;        // per-block partial sums of the strategy-search reductions
+    {
+        const size_t need = std::max(kvs::distance_partial_bytes(f.n_layers <= kvs::kMaxLayersSearch ? f.n_layers : 4),
+                                     (size_t)kvs::kSearchMaxBlocks * 3 * sizeof(double));
+        off = align_up(off + need, kAlign);
+    }
     c->ws_bytes = off;
 }
 
@@ -484,6 +491,45 @@ kvs_status kvs_unit_len(const kvs_ctx* ctx, int32_t layer, int32_t b, int32_t h,
     const int slot = ctx->slot_of_layer[layer];
     *len = ctx->ragged[slot] ? ctx->unit_len_host[slot][(size_t)b * ctx->cfg.n_kv_heads + h]
                              : (b < ctx->cur_batch ? ctx->slot_len[slot] : 0);
+    return KVS_OK;
+}
+
+kvs_status kvs_layer_distances(kvs_ctx* ctx, int32_t batch, float* dist, void* stream) {
+    if (!ctx || !dist) return KVS_ERR_INVALID_ARG;
+    if (!ctx->bound) return KVS_ERR_STATE;
+    if (ctx->cfg.n_layers > kvs::kMaxLayersSearch) return KVS_ERR_INVALID_ARG;
+    if (batch < 1 || batch > ctx->cur_batch) return ctx->cur_batch == 0 ? KVS_ERR_STATE : KVS_ERR_INVALID_ARG;
+    const int n = ctx->slot_len[0];
+    if (n == 0) return KVS_ERR_STATE;
+    for (int s = 0; s < ctx->n_slots; ++s)
+        if (ctx->slot_len[s] != n || ctx->ragged[s]) return KVS_ERR_STATE;   // equally long, un-evicted caches only
+    DeviceGuard guard(ctx->cfg.device);
+    if (!guard.ok) return KVS_ERR_CUDA;
+    if (kvs::launch_layer_distances(ctx->pool, (long long)ctx->plane_bytes, ctx->slot_of_layer.data(), ctx->cfg.n_layers,
+                                    batch, ctx->cfg.n_kv_heads, n, ctx->row_stride, ctx->cfg.head_dim, ctx->cfg.dtype,
+                                    reinterpret_cast<float*>(ctx->ws + ctx->off_search), dist, ctx->sm_count,
+                                    static_cast<cudaStream_t>(stream)) != cudaSuccess)
+        return KVS_ERR_CUDA;
+    ctx->seq += 2;
+    ctx->last_splitk_seq = ctx->seq;     // plain launches: everything before them has finished when they run
+    ctx->stats.search_launches += 2;
+    return KVS_OK;
+}
+
+kvs_status kvs_mean_cosine(kvs_ctx* ctx, const void* a, const void* b, int32_t n_samples, int64_t dim, float* out,
+                           void* stream) {
+    if (!ctx || !a || !b || !out) return KVS_ERR_INVALID_ARG;
+    if (!ctx->bound) return KVS_ERR_STATE;
+    if (n_samples < 1 || dim < 2 || (dim & 1) != 0) return KVS_ERR_INVALID_ARG;
+    if (((uintptr_t)a % 8) != 0 || ((uintptr_t)b % 8) != 0) return KVS_ERR_INVALID_ARG;
+    DeviceGuard guard(ctx->cfg.device);
+    if (!guard.ok) return KVS_ERR_CUDA;
+    if (kvs::launch_mean_cosine(a, b, n_samples, dim, ctx->cfg.dtype, reinterpret_cast<double*>(ctx->ws + ctx->off_search),
+                                out, ctx->sm_count, static_cast<cudaStream_t>(stream)) != cudaSuccess)
+        return KVS_ERR_CUDA;
+    ctx->seq += 2;
+    ctx->last_splitk_seq = ctx->seq;
+    ctx->stats.search_launches += 2;
     return KVS_OK;
 }
 

@@ -68,6 +68,16 @@ cudaError_t launch_prefill(const void* q, float* out, int* status, const void* p
                            int G, int n, int row_stride, long long krow0, long long vrow0, float scale_log2,
                            cudaStream_t stream);
 
+// Strategy-search reductions (see kvs_search.cu).
+constexpr int kMaxLayersSearch = 80;     // shared-memory bound of the distance kernel
+constexpr int kSearchMaxBlocks = 512;    // sizes the per-block partial buffers
+size_t distance_partial_bytes(int L);
+cudaError_t launch_layer_distances(const void* pool, long long plane_bytes, const int* slot_of_layer, int L, int B,
+                                   int Hkv, int n, int row_stride, int D, int dtype, float* partial, float* dist,
+                                   int sm_count, cudaStream_t stream);
+cudaError_t launch_mean_cosine(const void* a, const void* b, int S, long long dim, int dtype, double* partial,
+                               float* out, int sm_count, cudaStream_t stream);
+
 cudaError_t launch_append(const void* k, const void* v, void* kplane, void* vplane, int B, int n_new, int Hkv,
                           int row_bytes, int row_stride, int len0, const int* unit_len, bool programmatic, cudaStream_t stream);
 
