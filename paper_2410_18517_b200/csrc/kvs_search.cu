@@ -37,6 +37,24 @@ __device__ __forceinline__ float2 load2<float>(const float* p) {
     return *reinterpret_cast<const float2*>(p);
 }
 
+// Eight consecutive elements as floats (16 bytes of bf16, 32 bytes of fp32), added into s.
+template <typename T>
+__device__ __forceinline__ void add8(const T* p, float (&s)[8]);
+template <>
+__device__ __forceinline__ void add8<__nv_bfloat16>(const __nv_bfloat16* p, float (&s)[8]) {
+    const uint4 r = *reinterpret_cast<const uint4*>(p);
+    float f[8];
+    Unpack<__nv_bfloat16>::run(r, f);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) s[i] += f[i];
+}
+template <>
+__device__ __forceinline__ void add8<float>(const float* p, float (&s)[8]) {
+    const float4 a = *reinterpret_cast<const float4*>(p), b = *reinterpret_cast<const float4*>(p + 4);
+    s[0] += a.x; s[1] += a.y; s[2] += a.z; s[3] += a.w;
+    s[4] += b.x; s[5] += b.y; s[6] += b.z; s[7] += b.w;
+}
+
 struct DistArgs {
     const char* pool;
     float* partial;            // [blocks][Lp*Lp]
@@ -67,27 +85,33 @@ __global__ void __launch_bounds__(kDistThreads) layer_distance_kernel(const Dist
     const float inv_b = 1.0f / a.B;
     for (long long c = blockIdx.x; c < chunks; c += gridDim.x) {
         // ---- means of this chunk's positions, all layers ----
-        const long long p = c * kDistChunk + 2 * tid;
-        if (p < a.P) {
-            const int kv = (int)(p / kv_elems);
-            const long long rem = p - kv * kv_elems;
-            const int h = (int)(rem / unit_elems);
-            const long long e = rem - h * unit_elems;
-            for (int l = 0; l < a.L; ++l) {
-                const T* base = reinterpret_cast<const T*>(a.pool + (long long)(2 * a.slot_of_layer[l] + kv) * a.plane_bytes) +
-                                (long long)h * a.row_stride * a.D + e;
-                float sx = 0.f, sy = 0.f;
-#pragma unroll 6
-                for (int b = 0; b < a.B; ++b) {
-                    const float2 v = load2<T>(base + (long long)b * a.Hkv * a.row_stride * a.D);
-                    sx += v.x;
-                    sy += v.y;
+        // 64 groups of 8 consecutive positions (16-byte loads); the 4 quarters of the block take
+        // every fourth layer.  A unit holds a multiple of 8 elements, so a group never straddles two.
+        // Position 8*pg + i of the chunk is stored at column 64*i + pg: the order of positions inside
+        // a chunk is irrelevant to the sums and this one keeps the stores conflict-free.
+        {
+            const int pg = tid & 63, lq = tid >> 6;
+            const long long p = c * kDistChunk + 8 * pg;
+            if (p < a.P) {
+                const int kv = (int)(p / kv_elems);
+                const long long rem = p - kv * kv_elems;
+                const int h = (int)(rem / unit_elems);
+                const long long e = rem - h * unit_elems;
+                const long long bstride = (long long)a.Hkv * a.row_stride * a.D;
+                for (int l = lq; l < a.L; l += 4) {
+                    const T* base = reinterpret_cast<const T*>(a.pool + (long long)(2 * a.slot_of_layer[l] + kv) * a.plane_bytes) +
+                                    (long long)h * a.row_stride * a.D + e;
+                    float s8[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+#pragma unroll 8
+                    for (int b = 0; b < a.B; ++b) add8<T>(base + b * bstride, s8);
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) M[l * kDistStride + 64 * i + pg] = s8[i] * inv_b;
                 }
-                M[l * kDistStride + 2 * tid] = sx * inv_b;
-                M[l * kDistStride + 2 * tid + 1] = sy * inv_b;
+            } else {
+                for (int l = lq; l < a.L; l += 4)
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) M[l * kDistStride + 64 * i + pg] = 0.f;
             }
-        } else {
-            for (int l = 0; l < a.L; ++l) M[l * kDistStride + 2 * tid] = M[l * kDistStride + 2 * tid + 1] = 0.f;
         }
         __syncthreads();
         // ---- squared differences of every layer pair over the chunk ----
@@ -145,16 +169,35 @@ __global__ void __launch_bounds__(256) mean_cosine_kernel(const T* __restrict__ 
                                                           long long dim, double* __restrict__ partial) {
     float dot = 0.f, na = 0.f, nb = 0.f;
     const float inv = 1.0f / S;
-    for (long long e = 2 * ((long long)blockIdx.x * blockDim.x + threadIdx.x); e < dim; e += 2LL * gridDim.x * blockDim.x) {
-        float ax = 0.f, ay = 0.f, bx = 0.f, by = 0.f;
-        for (int s = 0; s < S; ++s) {
-            const float2 va = load2<T>(a + s * dim + e), vb = load2<T>(b + s * dim + e);
-            ax += va.x; ay += va.y; bx += vb.x; by += vb.y;
+    const bool wide = (dim % 8 == 0) && ((reinterpret_cast<uintptr_t>(a) | reinterpret_cast<uintptr_t>(b)) % 32 == 0);
+    if (wide) {
+        for (long long e = 8 * ((long long)blockIdx.x * blockDim.x + threadIdx.x); e < dim; e += 8LL * gridDim.x * blockDim.x) {
+            float sa[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f}, sb[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+#pragma unroll 4
+            for (int s = 0; s < S; ++s) {
+                add8<T>(a + s * dim + e, sa);
+                add8<T>(b + s * dim + e, sb);
+            }
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const float x = sa[i] * inv, y = sb[i] * inv;
+                dot = fmaf(x, y, dot);
+                na = fmaf(x, x, na);
+                nb = fmaf(y, y, nb);
+            }
         }
-        ax *= inv; ay *= inv; bx *= inv; by *= inv;
-        dot = fmaf(ax, bx, fmaf(ay, by, dot));
-        na = fmaf(ax, ax, fmaf(ay, ay, na));
-        nb = fmaf(bx, bx, fmaf(by, by, nb));
+    } else {
+        for (long long e = 2 * ((long long)blockIdx.x * blockDim.x + threadIdx.x); e < dim; e += 2LL * gridDim.x * blockDim.x) {
+            float ax = 0.f, ay = 0.f, bx = 0.f, by = 0.f;
+            for (int s = 0; s < S; ++s) {
+                const float2 va = load2<T>(a + s * dim + e), vb = load2<T>(b + s * dim + e);
+                ax += va.x; ay += va.y; bx += vb.x; by += vb.y;
+            }
+            ax *= inv; ay *= inv; bx *= inv; by *= inv;
+            dot = fmaf(ax, bx, fmaf(ay, by, dot));
+            na = fmaf(ax, ax, fmaf(ay, ay, na));
+            nb = fmaf(bx, bx, fmaf(by, by, nb));
+        }
     }
     __shared__ float red[3][8];
 #pragma unroll
@@ -230,7 +273,7 @@ cudaError_t launch_layer_distances(const void* pool, long long plane_bytes, cons
 
 cudaError_t launch_mean_cosine(const void* a, const void* b, int S, long long dim, int dtype, double* partial,
                                float* out, int sm_count, cudaStream_t stream) {
-    const long long pairs = (dim + 1) / 2;
+    const long long pairs = (dim + 7) / 8;
     const int blocks = (int)std::max<long long>(1, std::min<long long>((pairs + 255) / 256, std::min(4 * sm_count, kSearchMaxBlocks)));
     if (dtype == 0)
         mean_cosine_kernel<__nv_bfloat16><<<blocks, 256, 0, stream>>>((const __nv_bfloat16*)a, (const __nv_bfloat16*)b, S,
