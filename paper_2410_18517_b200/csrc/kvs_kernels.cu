@@ -143,10 +143,24 @@ __host__ __device__ __forceinline__ int cta_of_tile(long long gt, long long T, i
 // un-normalised output chunk) over the rows it is dealt, so no block-wide
 // synchronisation happens per tile; groups are merged once per piece.
 // --------------------------------------------------------------------------------------
-constexpr int kConsumerWarps = 8;
+#ifndef KVS_CONSUMER_WARPS
+#define KVS_CONSUMER_WARPS 8
+#endif
+constexpr int kConsumerWarps = KVS_CONSUMER_WARPS;
 constexpr int kConsumerThreads = kConsumerWarps * 32;
 constexpr int kScalarThreads = kConsumerThreads + 32;
-constexpr int kTileBytes = 16384;  // per K tile and per V tile
+// Tile size, ring depth and blocks per SM of the scalar kernel for groups of 1 or 2 q-heads
+// (compile-time; the defaults are the measured best on B200).
+#ifndef KVS_TILE_BYTES
+#define KVS_TILE_BYTES 32768
+#endif
+#ifndef KVS_STAGES
+#define KVS_STAGES 3
+#endif
+#ifndef KVS_BLOCKS_PER_SM
+#define KVS_BLOCKS_PER_SM 1
+#endif
+constexpr int kTileBytes = KVS_TILE_BYTES;  // per K tile and per V tile
 
 template <typename T, int D, int G>
 struct ScalarShape {
@@ -157,8 +171,8 @@ struct ScalarShape {
     static constexpr int NG = kConsumerWarps * GPW;       // lane groups per block
     static constexpr int TN = kTileBytes / RB;            // rows per tile
     static constexpr int R = TN / NG;                     // rows per group per tile
-    static constexpr int STAGES = (G <= 2) ? 3 : 6;
-    static constexpr int MIN_BLOCKS = (G <= 2) ? 2 : 1;
+    static constexpr int STAGES = (G <= 2) ? KVS_STAGES : (6 * 16384) / kTileBytes;
+    static constexpr int MIN_BLOCKS = (G <= 2) ? KVS_BLOCKS_PER_SM : 1;
     static constexpr int QBYTES = G * RB;
     static constexpr int STAGE_BYTES = 2 * kTileBytes + QBYTES;
     static constexpr int SCRATCH_FLOATS = NG * (D + 2);
@@ -519,7 +533,7 @@ void plan_decode_scalar(int units, int n, int G, int D, int dtype, int sm_count,
     plan->tile_rows = kTileBytes / rb;
     plan->tpu = (n + plan->tile_rows - 1) / plan->tile_rows;
     plan->T = (long long)units * plan->tpu;
-    const int per_sm = (G <= 2) ? 2 : 1;
+    const int per_sm = (G <= 2) ? KVS_BLOCKS_PER_SM : 1;
     int cap = sm_count * per_sm;
     if (max_ctas > 0) cap = std::min(cap, max_ctas);
     cap = std::min(cap, kMaxCtas);
@@ -557,7 +571,8 @@ cudaError_t launch_decode_scalar(const DecodeArgs& a, const DecodePlan& plan, cu
 // K4: read roof.  Same producer, same ring, consumers only fold the bytes together.
 // --------------------------------------------------------------------------------------
 constexpr int kRoofStages = 3;
-constexpr int kRoofStageBytes = 2 * kTileBytes;
+constexpr int kRoofTileBytes = 16384;
+constexpr int kRoofStageBytes = 2 * kRoofTileBytes;
 constexpr int kRoofSmem = kRoofStages * kRoofStageBytes + 2 * kRoofStages * 8 + 16;
 
 __global__ void __launch_bounds__(kScalarThreads, 2)
@@ -590,8 +605,8 @@ __global__ void __launch_bounds__(kScalarThreads, 2)
                     break;
                 unsigned char* sb = smem + st * kRoofStageBytes;
                 mbar_arrive_expect_tx(&full_bar[st], kRoofStageBytes);
-                bulk_g2s(sb, src + gt * kRoofStageBytes, kTileBytes, &full_bar[st]);
-                bulk_g2s(sb + kTileBytes, src + gt * kRoofStageBytes + kTileBytes, kTileBytes, &full_bar[st]);
+                bulk_g2s(sb, src + gt * kRoofStageBytes, kRoofTileBytes, &full_bar[st]);
+                bulk_g2s(sb + kRoofTileBytes, src + gt * kRoofStageBytes + kRoofTileBytes, kRoofTileBytes, &full_bar[st]);
             }
         }
         return;

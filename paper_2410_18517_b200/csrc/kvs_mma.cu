@@ -18,12 +18,26 @@ namespace kvs {
 
 namespace {
 
-constexpr int kMmaWarps = 4;
+// Consumer warps, tile size, ring depth and blocks per SM (compile-time; defaults = measured best).
+#ifndef KVS_MMA_WARPS
+#define KVS_MMA_WARPS 4
+#endif
+#ifndef KVS_MMA_TILE_BYTES
+#define KVS_MMA_TILE_BYTES 16384
+#endif
+#ifndef KVS_MMA_STAGES
+#define KVS_MMA_STAGES 4
+#endif
+#ifndef KVS_MMA_BLOCKS_PER_SM
+#define KVS_MMA_BLOCKS_PER_SM 1
+#endif
+constexpr int kMmaWarps = KVS_MMA_WARPS;
 constexpr int kMmaConsumerThreads = kMmaWarps * 32;
 constexpr int kMmaThreads = kMmaConsumerThreads + 32;
-constexpr int kMmaTileBytes = 16384;
+constexpr int kMmaTileBytes = KVS_MMA_TILE_BYTES;
 constexpr int kMmaQBytes = 2048;  // room for 8 heads x 128 x bf16
-constexpr int kMmaStages = 3;
+constexpr int kMmaStages = KVS_MMA_STAGES;
+constexpr int kBoxRows = 64;      // the pool's tensor map moves boxes of 64 columns x 64 rows (8 KiB)
 
 template <int D>
 struct MmaShape {
@@ -93,7 +107,7 @@ struct MmaKernelArgs {
 };
 
 template <int D, int G>
-__global__ void __launch_bounds__(kMmaThreads, 2)
+__global__ void __launch_bounds__(kMmaThreads, KVS_MMA_BLOCKS_PER_SM)
     decode_splitk_mma(const __grid_constant__ CUtensorMap tmap, const MmaKernelArgs a) {
     using S = MmaShape<D>;
     constexpr int TN = S::TN, KSTEPS = S::KSTEPS, NB = S::NB, BPW = S::BPW;
@@ -143,11 +157,14 @@ __global__ void __launch_bounds__(kMmaThreads, 2)
                 if (kv && have) {
                     const long long row = u * a.row_stride + (long long)ti * TN;
 #pragma unroll
-                    for (int h = 0; h < S::HALVES; ++h) {
-                        tma_load_2d(sb + h * (TN * 128), &tmap, h * 64, (int)(a.krow0 + row), &full_bar[st]);
-                        tma_load_2d(sb + kMmaTileBytes + h * (TN * 128), &tmap, h * 64, (int)(a.vrow0 + row),
-                                    &full_bar[st]);
-                    }
+                    for (int h = 0; h < S::HALVES; ++h)
+#pragma unroll
+                        for (int rb = 0; rb < TN / kBoxRows; ++rb) {
+                            const int off = h * (TN * 128) + rb * (kBoxRows * 128);
+                            tma_load_2d(sb + off, &tmap, h * 64, (int)(a.krow0 + row) + rb * kBoxRows, &full_bar[st]);
+                            tma_load_2d(sb + kMmaTileBytes + off, &tmap, h * 64, (int)(a.vrow0 + row) + rb * kBoxRows,
+                                        &full_bar[st]);
+                        }
                 }
                 if (qpart && with_q)
                     bulk_g2s(sb + 2 * kMmaTileBytes, a.q + u * (long long)QBYTES, QBYTES, &full_bar[st]);
@@ -381,7 +398,7 @@ cudaError_t init_mma_kernels() {
     return set_attr<64, 8>();
 }
 
-// Tensor map over the whole pool seen as [total_rows][D] bf16, box = 64 columns x tile rows,
+// Tensor map over the whole pool seen as [total_rows][D] bf16, box = 64 columns x 64 rows,
 // 128-byte swizzle.  `storage` must be 64-byte aligned and hold sizeof(CUtensorMap) = 128 bytes.
 cudaError_t make_pool_tensor_map(void* storage, void* pool, long long total_rows, int D) {
     typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -392,10 +409,9 @@ cudaError_t make_pool_tensor_map(void* storage, void* pool, long long total_rows
     cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres);
     if (e != cudaSuccess) return e;
     if (qres != cudaDriverEntryPointSuccess || fn == nullptr) return cudaErrorNotSupported;
-    const int tile_rows = kMmaTileBytes / (D * 2);
     cuuint64_t dims[2] = {(cuuint64_t)D, (cuuint64_t)total_rows};
     cuuint64_t strides[1] = {(cuuint64_t)D * 2};
-    cuuint32_t box[2] = {64u, (cuuint32_t)tile_rows};
+    cuuint32_t box[2] = {64u, (cuuint32_t)kBoxRows};
     cuuint32_t estr[2] = {1u, 1u};
     CUresult r = reinterpret_cast<EncodeFn>(fn)(reinterpret_cast<CUtensorMap*>(storage), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16,
                                                 2, pool, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
@@ -408,7 +424,7 @@ void plan_decode_mma(int units, int n, int D, int sm_count, int max_ctas, Decode
     plan->tile_rows = kMmaTileBytes / (D * 2);
     plan->tpu = (n + plan->tile_rows - 1) / plan->tile_rows;
     plan->T = (long long)units * plan->tpu;
-    int cap = sm_count * 2;
+    int cap = sm_count * KVS_MMA_BLOCKS_PER_SM;
     if (max_ctas > 0) cap = std::min(cap, max_ctas);
     cap = std::min(cap, kMaxCtas);
     plan->NC = (int)std::min<long long>(plan->T, cap);
