@@ -230,8 +230,8 @@ kvs_status kvs_mean_cosine(kvs_ctx* ctx, const void* a, const void* b, int32_t n
  *   out_host: host, [n_layers][batch][n_q_heads][head_dim], float32
  * Copies inputs host->device into the workspace staging area, runs the layers on
  * `stream`, copies the result device->host, and waits until all of it is done.  The
- * copies run on a second stream owned by the context (created at the first call,
- * together with a few events) in four chunks of layers, so that they overlap the
+ * copies run on two extra streams owned by the context (created at the first call,
+ * together with a few events) in eight chunks of layers, so that they overlap the
  * layers of the neighbouring chunks.
  * Pinned host memory makes the copies asynchronous; pageable memory also works.
  * h2d_bytes / d2h_bytes (host, may be NULL) receive the bytes copied.

@@ -60,9 +60,9 @@ struct kvs_ctx {
     std::vector<int32_t> app_start_latest;                // first row the latest append wrote
 
     // kvs_step_host: second stream and events that overlap the host copies with the layers
-    static constexpr int kChunks = 4;
+    static constexpr int kChunks = 8;
     bool copy_ready = false;
-    cudaStream_t copy_stream = nullptr;
+    cudaStream_t copy_stream = nullptr, out_stream = nullptr;
     cudaEvent_t ev_in[kChunks] = {}, ev_done[kChunks] = {}, ev_start = nullptr;
 
     int opt_max_ctas = 0;
@@ -317,6 +317,7 @@ kvs_status kvs_destroy(kvs_ctx* ctx) {
             }
             cudaEventDestroy(ctx->ev_start);
             cudaStreamDestroy(ctx->copy_stream);
+            cudaStreamDestroy(ctx->out_stream);
         }
     }
     delete ctx;
@@ -554,11 +555,14 @@ kvs_status kvs_step_host(kvs_ctx* ctx, const void* q_host, const void* k_host, c
     char* dv = ctx->ws + ctx->off_stage_v;
     char* dout = ctx->ws + ctx->off_stage_out;
     uint64_t h2d = 0;
-    // The layers are cut into a few chunks; a second stream copies chunk c+1's inputs in and
+    // The layers are cut into chunks; one extra stream copies chunk c+1's inputs in and another copies
     // chunk c-1's outputs out while chunk c computes, so only the first input copy and the last
-    // output copy are exposed.
+    // output copy are exposed.  Chunk c+1's copies are queued before chunk c's kernels so that the
+    // host never stands between the device and its next piece of work.
     if (!ctx->copy_ready) {
-        if (cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking) != cudaSuccess) return KVS_ERR_CUDA;
+        if (cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking) != cudaSuccess ||
+            cudaStreamCreateWithFlags(&ctx->out_stream, cudaStreamNonBlocking) != cudaSuccess)
+            return KVS_ERR_CUDA;
         for (int i = 0; i < kvs_ctx::kChunks; ++i)
             if (cudaEventCreateWithFlags(&ctx->ev_in[i], cudaEventDisableTiming) != cudaSuccess ||
                 cudaEventCreateWithFlags(&ctx->ev_done[i], cudaEventDisableTiming) != cudaSuccess)
@@ -566,17 +570,18 @@ kvs_status kvs_step_host(kvs_ctx* ctx, const void* q_host, const void* k_host, c
         if (cudaEventCreateWithFlags(&ctx->ev_start, cudaEventDisableTiming) != cudaSuccess) return KVS_ERR_CUDA;
         ctx->copy_ready = true;
     }
-    cudaStream_t cs = ctx->copy_stream;
+    cudaStream_t cs = ctx->copy_stream, os = ctx->out_stream;
     const int L = f.n_layers;
     const int chunks = L < kvs_ctx::kChunks ? L : kvs_ctx::kChunks;
-    // the copy stream starts after whatever the caller already queued on `st`
-    if (cudaEventRecord(ctx->ev_start, st) != cudaSuccess || cudaStreamWaitEvent(cs, ctx->ev_start, 0) != cudaSuccess)
+    // the copy streams start after whatever the caller already queued on `st`
+    if (cudaEventRecord(ctx->ev_start, st) != cudaSuccess || cudaStreamWaitEvent(cs, ctx->ev_start, 0) != cudaSuccess ||
+        cudaStreamWaitEvent(os, ctx->ev_start, 0) != cudaSuccess)
         return KVS_ERR_CUDA;
-    for (int c = 0; c < chunks; ++c) {
+    auto copy_in = [&](int c) -> bool {
         const int l0 = (int)((long long)c * L / chunks), l1 = (int)((long long)(c + 1) * L / chunks);
         if (cudaMemcpyAsync(dq + q_layer * l0, (const char*)q_host + q_layer * l0, q_layer * (l1 - l0),
                             cudaMemcpyHostToDevice, cs) != cudaSuccess)
-            return KVS_ERR_CUDA;
+            return false;
         h2d += q_layer * (l1 - l0);
         // K/V of own-cache layers only; consecutive own-cache layers go in one copy
         for (int l = l0; l < l1;) {
@@ -586,14 +591,16 @@ kvs_status kvs_step_host(kvs_ctx* ctx, const void* q_host, const void* k_host, c
             const size_t off = kv_layer * l, len = kv_layer * (e - l + 1);
             if (cudaMemcpyAsync(dk + off, (const char*)k_host + off, len, cudaMemcpyHostToDevice, cs) != cudaSuccess ||
                 cudaMemcpyAsync(dv + off, (const char*)v_host + off, len, cudaMemcpyHostToDevice, cs) != cudaSuccess)
-                return KVS_ERR_CUDA;
+                return false;
             h2d += 2 * len;
             l = e + 1;
         }
-        if (cudaEventRecord(ctx->ev_in[c], cs) != cudaSuccess) return KVS_ERR_CUDA;
-    }
+        return cudaEventRecord(ctx->ev_in[c], cs) == cudaSuccess;
+    };
+    if (!copy_in(0)) return KVS_ERR_CUDA;
     for (int c = 0; c < chunks; ++c) {
         const int l0 = (int)((long long)c * L / chunks), l1 = (int)((long long)(c + 1) * L / chunks);
+        if (c + 1 < chunks && !copy_in(c + 1)) return KVS_ERR_CUDA;
         if (cudaStreamWaitEvent(st, ctx->ev_in[c], 0) != cudaSuccess) return KVS_ERR_CUDA;
         for (int l = l0; l < l1; ++l) {
             if (ctx->share_map[l] == l) {
@@ -606,13 +613,15 @@ kvs_status kvs_step_host(kvs_ctx* ctx, const void* q_host, const void* k_host, c
                 do_attention(ctx, l, dq + q_layer * l, reinterpret_cast<float*>(dout + out_layer * l), batch, st);
             if (s != KVS_OK) return s;
         }
-        if (cudaEventRecord(ctx->ev_done[c], st) != cudaSuccess || cudaStreamWaitEvent(cs, ctx->ev_done[c], 0) != cudaSuccess)
+        if (cudaEventRecord(ctx->ev_done[c], st) != cudaSuccess || cudaStreamWaitEvent(os, ctx->ev_done[c], 0) != cudaSuccess)
             return KVS_ERR_CUDA;
         if (cudaMemcpyAsync((char*)out_host + out_layer * l0, dout + out_layer * l0, out_layer * (l1 - l0),
-                            cudaMemcpyDeviceToHost, cs) != cudaSuccess)
+                            cudaMemcpyDeviceToHost, os) != cudaSuccess)
             return KVS_ERR_CUDA;
     }
-    if (cudaStreamSynchronize(cs) != cudaSuccess || cudaStreamSynchronize(st) != cudaSuccess) return KVS_ERR_CUDA;
+    if (cudaStreamSynchronize(os) != cudaSuccess || cudaStreamSynchronize(cs) != cudaSuccess ||
+        cudaStreamSynchronize(st) != cudaSuccess)
+        return KVS_ERR_CUDA;
     if (h2d_bytes) *h2d_bytes = h2d;
     if (d2h_bytes) *d2h_bytes = out_layer * f.n_layers;
     return KVS_OK;

@@ -121,6 +121,27 @@ def test_early_start_launches_change_nothing(early, Hq, Hkv):
     assert torch.equal(cache.decode_attention(1, q), ref_cache.decode_attention(1, q))
 
 
+@pytest.mark.parametrize("case", range(24))
+def test_random_small_configurations(case):
+    """Seeded random layers / heads / group size / head size / type / batch / context / strategy
+    (chains and fan-out included), a few decode steps, everything compared."""
+    rng = np.random.default_rng(1000 + case)
+    L = int(rng.integers(1, 7))
+    Hkv = int(rng.choice([1, 2, 3, 4]))
+    G = int(rng.choice([1, 2, 4, 8]))
+    D = int(rng.choice([64, 128]))
+    dtype = str(rng.choice(["bf16", "bf16", "f32"]))
+    B = int(rng.integers(1, 5))
+    context = int(rng.integers(0, 400))
+    sm = tuple(int(rng.integers(0, l + 1)) if rng.random() < 0.5 else l for l in range(L))
+    w = si.Workload(f"rand_{case}", L=L, Hq=Hkv * G, Hkv=Hkv, D=D, B=B, context=context, dtype=dtype, n_shared=0,
+                    map_seed=0, steps=3, fixed_map=sm)
+    opts = [(KVS_OPT_MAX_CTAS, int(rng.integers(1, 40)))] if rng.random() < 0.5 else []
+    cache, orc, _ = run_small(w, steps=int(rng.integers(1, 4)), options=opts)
+    n_slots, _, _ = oracle.slot_table(sm)
+    assert cache.num_slots() == n_slots
+
+
 def test_many_small_units_per_block():
     """More units than thread blocks and only a few tiles each: blocks span several whole units."""
     w = si.Workload("many_units", L=1, Hq=16, Hkv=16, D=128, B=40, context=130, dtype="bf16",
