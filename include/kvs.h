@@ -61,7 +61,7 @@ typedef enum { KVS_BF16 = 0, KVS_F32 = 1 } kvs_dtype;
 
 typedef struct {
     int32_t n_layers;     /* L >= 1                                                 */
-    int32_t n_q_heads;    /* Hq; must be a multiple of n_kv_heads; Hq/Hkv in {1,2,4,8} */
+    int32_t n_q_heads;    /* Hq; a multiple of n_kv_heads; Hq/Hkv in 1..8 (3,5,6,7: bf16 only) */
     int32_t n_kv_heads;   /* Hkv >= 1                                               */
     int32_t head_dim;     /* 64 or 128                                              */
     int32_t max_batch;    /* largest batch any call will pass                       */
@@ -99,7 +99,7 @@ typedef enum {
 /* Create a context.  cfg: host.  *out receives the context.  The strategy
  * starts as the identity (no layer shares).  No CUDA call is made here.
  * Errors: INVALID_ARG for NULLs, non-positive sizes, Hq % Hkv != 0, group size
- * not in {1,2,4,8}, head_dim not in {64,128}, unknown dtype.                    */
+ * above 8 (or 3, 5, 6, 7 with fp32 storage), head_dim not in {64,128}, unknown dtype. */
 kvs_status kvs_create(const kvs_config* cfg, kvs_ctx** out);
 
 /* Destroy a context.  Frees host tables only; the caller's buffers are untouched.

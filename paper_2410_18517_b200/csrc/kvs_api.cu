@@ -247,7 +247,7 @@ kvs_status do_attention(kvs_ctx* c, int layer, const void* q, float* out, int ba
     c->last_splitk_seq = c->seq - 1;
     kvs::DecodePlan plan;
     // bf16 groups of 4 or more q-heads per kv-head are a real (if thin) contraction: tensor cores.
-    const bool use_mma = c->have_tensor_map && (c->opt_kernel == 2 || (c->opt_kernel == 0 && c->G >= 4));
+    const bool use_mma = c->have_tensor_map && (c->opt_kernel == 2 || (c->opt_kernel == 0 && c->G >= 3));
     if (use_mma) {
         const long long plane_rows = (long long)c->cfg.max_batch * c->cfg.n_kv_heads * c->row_stride;
         kvs::plan_decode_mma(a.units, a.n, a.D, c->sm_count, c->opt_max_ctas, &plan);
@@ -283,7 +283,10 @@ kvs_status kvs_create(const kvs_config* cfg, kvs_ctx** out) {
         return KVS_ERR_INVALID_ARG;
     if (cfg->n_q_heads % cfg->n_kv_heads != 0) return KVS_ERR_INVALID_ARG;
     const int G = cfg->n_q_heads / cfg->n_kv_heads;
-    if (G != 1 && G != 2 && G != 4 && G != 8) return KVS_ERR_INVALID_ARG;
+    const bool pow2_group = (G == 1 || G == 2 || G == 4 || G == 8);
+    if (G > 8) return KVS_ERR_INVALID_ARG;
+    // groups of 3, 5, 6 or 7 q-heads exist only on the tensor-core kernel, which is bf16-only
+    if (!pow2_group && cfg->dtype != KVS_BF16) return KVS_ERR_INVALID_ARG;
     if (cfg->head_dim != 64 && cfg->head_dim != 128) return KVS_ERR_INVALID_ARG;
     if (cfg->dtype != KVS_BF16 && cfg->dtype != KVS_F32) return KVS_ERR_INVALID_ARG;
     if (cfg->device < 0 || cfg->device >= 64) return KVS_ERR_INVALID_ARG;
@@ -689,6 +692,8 @@ kvs_status kvs_set_option(kvs_ctx* ctx, int32_t option, int32_t value) {
         case KVS_OPT_KERNEL:
             if (value < 0 || value > 2) return KVS_ERR_INVALID_ARG;
             if (value == 2 && ctx->cfg.dtype != KVS_BF16) return KVS_ERR_INVALID_ARG;  // tensor-core path is bf16 only
+            if (value == 1 && ctx->G != 1 && ctx->G != 2 && ctx->G != 4 && ctx->G != 8)
+                return KVS_ERR_INVALID_ARG;                                          // scalar path: groups of 1, 2, 4, 8
             ctx->opt_kernel = value;
             return KVS_OK;
         default:
@@ -774,7 +779,7 @@ kvs_status kvs_decode_attention_static(kvs_ctx* ctx, int32_t layer, const void* 
     const int units = batch * c->cfg.n_kv_heads;
     const int n = c->slot_len[slot];
     const int D = c->cfg.head_dim;
-    const bool use_mma = c->have_tensor_map && (c->opt_kernel == 2 || (c->opt_kernel == 0 && c->G >= 4));
+    const bool use_mma = c->have_tensor_map && (c->opt_kernel == 2 || (c->opt_kernel == 0 && c->G >= 3));
     kvs::DecodePlan plan;
     if (use_mma)
         kvs::plan_decode_mma(units, n, D, c->sm_count, c->opt_max_ctas, &plan);

@@ -104,14 +104,18 @@ struct MmaKernelArgs {
     float scale_log2;
     int safe_rows;  // rows of every unit that no kernel possibly still running writes
     const int* unit_len;  // per-unit row counts of a ragged slot, or nullptr (then n holds for all)
+    int G;          // q-heads per kv-head, 1..8
 };
 
-template <int D, int G>
+// G (q-heads per kv-head, 1..8) is a run-time argument: it only selects which rows of the padded
+// 16-row M side are real, so one kernel per head size serves every group size.
+template <int D>
 __global__ void __launch_bounds__(kMmaThreads, KVS_MMA_BLOCKS_PER_SM)
     decode_splitk_mma(const __grid_constant__ CUtensorMap tmap, const MmaKernelArgs a) {
     using S = MmaShape<D>;
     constexpr int TN = S::TN, KSTEPS = S::KSTEPS, NB = S::NB, BPW = S::BPW;
-    constexpr int QBYTES = G * S::RB;
+    const int G = a.G;
+    const int QBYTES = G * S::RB;
 
     extern __shared__ unsigned char smem_raw[];
     // 128-byte swizzled tiles need 1024-byte aligned bases
@@ -323,7 +327,6 @@ __global__ void __launch_bounds__(kMmaThreads, KVS_MMA_BLOCKS_PER_SM)
         float l = lsum;
         l += __shfl_xor_sync(0xffffffffu, l, 1);
         l += __shfl_xor_sync(0xffffffffu, l, 2);
-#pragma unroll
         for (int g = 0; g < G; ++g) {
             named_bar_sync(1, kMmaConsumerThreads);
             if (row == g) {
@@ -361,41 +364,22 @@ __global__ void __launch_bounds__(kMmaThreads, KVS_MMA_BLOCKS_PER_SM)
     }
 }
 
-template <int D, int G>
+template <int D>
 cudaError_t set_attr() {
-    return cudaFuncSetAttribute(decode_splitk_mma<D, G>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    return cudaFuncSetAttribute(decode_splitk_mma<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 MmaShape<D>::SMEM_BYTES);
 }
 
-template <int D, int G>
-cudaError_t launch_one(const CUtensorMap& tm, const MmaKernelArgs& ka, int NC, bool pdl, cudaStream_t stream) {
-    return launch_kernel(decode_splitk_mma<D, G>, dim3(NC), dim3(kMmaThreads), MmaShape<D>::SMEM_BYTES, stream, pdl, tm,
-                         ka);
-}
-
 template <int D>
-cudaError_t launch_groups(int G, const CUtensorMap& tm, const MmaKernelArgs& ka, int NC, bool pdl, cudaStream_t stream) {
-    switch (G) {
-        case 1: return launch_one<D, 1>(tm, ka, NC, pdl, stream);
-        case 2: return launch_one<D, 2>(tm, ka, NC, pdl, stream);
-        case 4: return launch_one<D, 4>(tm, ka, NC, pdl, stream);
-        case 8: return launch_one<D, 8>(tm, ka, NC, pdl, stream);
-        default: return cudaErrorInvalidValue;
-    }
+cudaError_t launch_one(const CUtensorMap& tm, const MmaKernelArgs& ka, int NC, bool pdl, cudaStream_t stream) {
+    return launch_kernel(decode_splitk_mma<D>, dim3(NC), dim3(kMmaThreads), MmaShape<D>::SMEM_BYTES, stream, pdl, tm, ka);
 }
 
 }  // namespace
 
 cudaError_t init_mma_kernels() {
-    cudaError_t e;
-    if ((e = set_attr<128, 1>()) != cudaSuccess) return e;
-    if ((e = set_attr<128, 2>()) != cudaSuccess) return e;
-    if ((e = set_attr<128, 4>()) != cudaSuccess) return e;
-    if ((e = set_attr<128, 8>()) != cudaSuccess) return e;
-    if ((e = set_attr<64, 1>()) != cudaSuccess) return e;
-    if ((e = set_attr<64, 2>()) != cudaSuccess) return e;
-    if ((e = set_attr<64, 4>()) != cudaSuccess) return e;
-    return set_attr<64, 8>();
+    cudaError_t e = set_attr<128>();
+    return e != cudaSuccess ? e : set_attr<64>();
 }
 
 // Tensor map over the whole pool seen as [total_rows][D] bf16, box = 64 columns x 64 rows,
@@ -448,8 +432,10 @@ cudaError_t launch_decode_mma(const DecodeArgs& a, const DecodePlan& plan, const
     ka.safe_rows = (a.programmatic && !a.unit_len) ? a.safe_rows : 0;
     ka.unit_len = a.unit_len;
     const CUtensorMap& tm = *reinterpret_cast<const CUtensorMap*>(tensor_map);
-    if (a.D == 128) return launch_groups<128>(a.G, tm, ka, plan.NC, a.programmatic, stream);
-    if (a.D == 64) return launch_groups<64>(a.G, tm, ka, plan.NC, a.programmatic, stream);
+    ka.G = a.G;
+    if (a.G < 1 || a.G > 8) return cudaErrorInvalidValue;
+    if (a.D == 128) return launch_one<128>(tm, ka, plan.NC, a.programmatic, stream);
+    if (a.D == 64) return launch_one<64>(tm, ka, plan.NC, a.programmatic, stream);
     return cudaErrorInvalidValue;
 }
 

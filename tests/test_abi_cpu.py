@@ -48,6 +48,17 @@ def test_create_rejects_bad_configs(kw):
     assert e.value.status == kb.KVS_ERR_INVALID_ARG
 
 
+def test_group_sizes():
+    for G in range(1, 9):
+        c = _create(Hq=2 * G, Hkv=2, D=128, dt=kb.KVS_BF16)      # every group size up to 8 with bf16
+        kb.kvs_destroy(c)
+    for G in (1, 2, 4, 8):
+        kb.kvs_destroy(_create(Hq=2 * G, Hkv=2, dt=kb.KVS_F32))
+    for G in (3, 5, 6, 7):
+        with pytest.raises(kb.KvsError):
+            _create(Hq=2 * G, Hkv=2, dt=kb.KVS_F32)
+
+
 def test_identity_map_by_default_and_tiny_strategy():
     c = _create()
     assert kb.kvs_num_slots(c) == 4

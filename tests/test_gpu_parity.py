@@ -77,6 +77,18 @@ def test_both_kernels_on_every_group_size(kernel, D, Hq, Hkv, context):
     assert cache.last_launch()["kernel"] == kernel
 
 
+@pytest.mark.parametrize("G", [3, 5, 6, 7])
+@pytest.mark.parametrize("D", [64, 128])
+def test_group_sizes_that_are_not_powers_of_two(G, D):
+    """48 q-heads over 8 kv-heads (InternLM2-20B's shape) is a group of 6: bf16 only, tensor-core kernel."""
+    w = si.Workload(f"g{G}_{D}", L=3, Hq=2 * G, Hkv=2, D=D, B=2, context=333, dtype="bf16", n_shared=1, map_seed=0,
+                    steps=2, fixed_map=(0, 1, 0))
+    cache, _, _ = run_small(w, steps=2)
+    assert cache.last_launch()["kernel"] == 2
+    with pytest.raises(KvsError):
+        cache.set_option(KVS_OPT_KERNEL, 1)           # the scalar kernel has groups of 1, 2, 4, 8 only
+
+
 def test_auto_kernel_choice():
     """Groups of four or more bf16 q-heads go to the tensor cores; fp32 storage never does."""
     for Hq, Hkv, dtype, want in [(4, 4, "bf16", 1), (4, 2, "bf16", 1), (8, 2, "bf16", 2), (8, 1, "bf16", 2),
