@@ -117,13 +117,9 @@ class ClockSampler:
         return out
 
 
-def cpu_baseline(w, seconds_target: float = 15.0) -> dict:
-    """Time the oracle, as it stands, on a bounded sample of this workload's units."""
-    import numpy as np
+def cpu_sample(w):
+    """Seeded inputs of 64 (sequence, q-head) units of this workload, widened to float64."""
     import torch
-
-    import oracle
-    import synth_inputs as si
 
     n = w.context + 1
     distinct = 64
@@ -131,6 +127,15 @@ def cpu_baseline(w, seconds_target: float = 15.0) -> dict:
     K = torch.randn(distinct, n, w.D, generator=g).to(w.torch_dtype).double().numpy()
     V = torch.randn(distinct, n, w.D, generator=g).to(w.torch_dtype).double().numpy()
     q = torch.randn(distinct, w.D, generator=g).to(w.torch_dtype).double().numpy()
+    return q, K, V
+
+
+def cpu_baseline(w, seconds_target: float = 15.0, sample=None) -> dict:
+    """Time the oracle, as it stands, on a bounded sample of this workload's units."""
+    import oracle
+
+    q, K, V = sample if sample is not None else cpu_sample(w)
+    distinct, n = K.shape[0], K.shape[1]
     oracle.attend_units(q[:8], K[:8], V[:8])            # load the library, warm the threads
     t0 = time.perf_counter()
     oracle.attend_units(q, K, V)
@@ -156,9 +161,13 @@ def run_reference(args, w):
         return
     import oracle
 
+    # every step is a bounded sample; its size shrinks with the number of steps asked for so
+    # that the whole run stays within about three minutes
+    per_step_s = max(0.2, min(4.0, 150.0 / max(1, args.warmup + args.steps)))
+    sample = cpu_sample(w)
     per = []
     for i in range(args.warmup + args.steps):
-        r = cpu_baseline(w, seconds_target=4.0)
+        r = cpu_baseline(w, seconds_target=per_step_s, sample=sample)
         if i >= args.warmup:
             per.append(r)
     val = statistics.mean(x["value"] for x in per)
