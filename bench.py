@@ -39,8 +39,8 @@ FALLBACK_HBM_GBS = 6650.0
 NCU_TRAFFIC = {
     1: {"files": ("kvs_kernels.cu", "kvs_device.cuh"), "dram_bytes": 541.28e6, "kv_bytes": 537.13e6,
         "sha256": "5a859312f183a0732ab0dbea121eb0817d775f5df9796696642a9ad32c7822b7"},
-    2: {"files": ("kvs_mma.cu", "kvs_device.cuh"), "dram_bytes": 542.16e6, "kv_bytes": 536.90e6,
-        "sha256": "38be758128205e3d463afa7db4609fe25247acad7752f2db8d711cdccdbad8a7"},
+    2: {"files": ("kvs_mma.cu", "kvs_device.cuh"), "dram_bytes": 541.96e6, "kv_bytes": 536.90e6,
+        "sha256": "71f7e785126570c7b293c6f999372f033a41d2baa01ff905f4dd602c748bac99"},
 }
 
 
