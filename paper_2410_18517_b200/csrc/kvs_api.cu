@@ -223,16 +223,36 @@ kvs_status do_append(kvs_ctx* c, int layer, const void* k, const void* v, int ba
     return KVS_OK;
 }
 
-kvs_status do_attention(kvs_ctx* c, int layer, const void* q, float* out, int batch, cudaStream_t st) {
-    const int slot = c->slot_of_layer[layer];
+// Where one attention call keeps its split-K partial results and reports device-side trouble.
+struct AttentionScratch {
+    float* part_o;
+    float* part_ml;
+    int* status;
+    bool programmatic;   // early-start launches (only when the call follows this context's own kernels)
+};
+
+// Which kernel serves the context's shape and how the call is cut into work.  bf16 groups of three
+// or more q-heads per kv-head are a real (if thin) contraction and go to the tensor cores.
+bool choose_plan(const kvs_ctx* c, int units, int n, kvs::DecodePlan* plan) {
+    const bool use_mma = c->have_tensor_map && (c->opt_kernel == 2 || (c->opt_kernel == 0 && c->G >= 3));
+    if (use_mma)
+        kvs::plan_decode_mma(units, n, c->cfg.head_dim, c->sm_count, c->opt_max_ctas, plan);
+    else
+        kvs::plan_decode_scalar(units, n, c->G, c->cfg.head_dim, c->cfg.dtype, c->sm_count, c->opt_max_ctas, plan);
+    return use_mma;
+}
+
+// Split-K kernel + combine kernel of one layer, with the given plan and scratch.
+kvs_status run_attention(kvs_ctx* c, int slot, const void* q, float* out, int batch, const kvs::DecodePlan& plan,
+                         bool use_mma, const AttentionScratch& scratch, cudaStream_t st) {
     kvs::DecodeArgs a;
     a.q = q;
     a.kplane = c->pool + (size_t)(2 * slot) * c->plane_bytes;
     a.vplane = c->pool + (size_t)(2 * slot + 1) * c->plane_bytes;
-    a.part_o = reinterpret_cast<float*>(c->ws + c->off_part_o);
-    a.part_ml = reinterpret_cast<float*>(c->ws + c->off_part_ml);
+    a.part_o = scratch.part_o;
+    a.part_ml = scratch.part_ml;
     a.out = out;
-    a.status = reinterpret_cast<int*>(c->ws + c->off_status);
+    a.status = scratch.status;
     a.n = c->slot_len[slot];
     a.row_stride = c->row_stride;
     a.units = batch * c->cfg.n_kv_heads;
@@ -240,22 +260,17 @@ kvs_status do_attention(kvs_ctx* c, int layer, const void* q, float* out, int ba
     a.D = c->cfg.head_dim;
     a.dtype = c->cfg.dtype;
     a.scale_log2 = c->scale * 1.4426950408889634f;
-    a.programmatic = c->opt_pdl != 0;
-    a.safe_rows = safe_rows_of(c, slot);
+    a.programmatic = scratch.programmatic;
+    a.safe_rows = scratch.programmatic ? safe_rows_of(c, slot) : 0;
     a.unit_len = c->ragged[slot] ? unit_len_dev(c, slot) : nullptr;
     c->seq += 2;                       // split-K kernel, then combine
     c->last_splitk_seq = c->seq - 1;
-    kvs::DecodePlan plan;
-    // bf16 groups of 4 or more q-heads per kv-head are a real (if thin) contraction: tensor cores.
-    const bool use_mma = c->have_tensor_map && (c->opt_kernel == 2 || (c->opt_kernel == 0 && c->G >= 3));
     if (use_mma) {
         const long long plane_rows = (long long)c->cfg.max_batch * c->cfg.n_kv_heads * c->row_stride;
-        kvs::plan_decode_mma(a.units, a.n, a.D, c->sm_count, c->opt_max_ctas, &plan);
         if (kvs::launch_decode_mma(a, plan, c->tensor_map, plane_rows * (2 * slot), plane_rows * (2 * slot + 1), st) !=
             cudaSuccess)
             return KVS_ERR_CUDA;
     } else {
-        kvs::plan_decode_scalar(a.units, a.n, a.G, a.D, a.dtype, c->sm_count, c->opt_max_ctas, &plan);
         if (kvs::launch_decode_scalar(a, plan, st) != cudaSuccess) return KVS_ERR_CUDA;
     }
     if (kvs::launch_combine(a, plan, st) != cudaSuccess) return KVS_ERR_CUDA;
@@ -270,6 +285,16 @@ kvs_status do_attention(kvs_ctx* c, int layer, const void* q, float* out, int ba
         c->stats.kv_bytes_read += 2ull * a.units * a.n * c->row_bytes;
     }
     return KVS_OK;
+}
+
+kvs_status do_attention(kvs_ctx* c, int layer, const void* q, float* out, int batch, cudaStream_t st) {
+    const int slot = c->slot_of_layer[layer];
+    kvs::DecodePlan plan;
+    const bool use_mma = choose_plan(c, batch * c->cfg.n_kv_heads, c->slot_len[slot], &plan);
+    const AttentionScratch scratch = {reinterpret_cast<float*>(c->ws + c->off_part_o),
+                                      reinterpret_cast<float*>(c->ws + c->off_part_ml),
+                                      reinterpret_cast<int*>(c->ws + c->off_status), c->opt_pdl != 0};
+    return run_attention(c, slot, q, out, batch, plan, use_mma, scratch, st);
 }
 
 }  // namespace
@@ -777,14 +802,9 @@ kvs_status kvs_decode_attention_static(kvs_ctx* ctx, int32_t layer, const void* 
     kvs_ctx* c = ctx;
     const int slot = c->slot_of_layer[layer];
     const int units = batch * c->cfg.n_kv_heads;
-    const int n = c->slot_len[slot];
     const int D = c->cfg.head_dim;
-    const bool use_mma = c->have_tensor_map && (c->opt_kernel == 2 || (c->opt_kernel == 0 && c->G >= 3));
     kvs::DecodePlan plan;
-    if (use_mma)
-        kvs::plan_decode_mma(units, n, D, c->sm_count, c->opt_max_ctas, &plan);
-    else
-        kvs::plan_decode_scalar(units, n, c->G, D, c->cfg.dtype, c->sm_count, c->opt_max_ctas, &plan);
+    const bool use_mma = choose_plan(c, units, c->slot_len[slot], &plan);
     // one partial (o[D], m, l) per (piece, q-head); pieces are indexed unit + block
     const size_t pieces = (size_t)units + plan.NC;
     const size_t part_o_bytes = align_up(pieces * c->G * D * sizeof(float), kAlign);
@@ -799,41 +819,11 @@ kvs_status kvs_decode_attention_static(kvs_ctx* ctx, int32_t layer, const void* 
     int* status_word = device_status ? device_status : reinterpret_cast<int*>(base);
     // the array keeps whatever the previous call left; only the status word must start at zero
     if (cudaMemsetAsync(status_word, 0, sizeof(int), st) != cudaSuccess) return KVS_ERR_CUDA;
-
-    kvs::DecodeArgs a;
-    a.q = q;
-    a.kplane = c->pool + (size_t)(2 * slot) * c->plane_bytes;
-    a.vplane = c->pool + (size_t)(2 * slot + 1) * c->plane_bytes;
-    a.part_o = reinterpret_cast<float*>(base + kStaticStatusBytes);
-    a.part_ml = reinterpret_cast<float*>(base + kStaticStatusBytes + part_o_bytes);
-    a.out = out;
-    a.status = status_word;
-    a.n = n;
-    a.row_stride = c->row_stride;
-    a.units = units;
-    a.G = c->G;
-    a.D = D;
-    a.dtype = c->cfg.dtype;
-    a.scale_log2 = c->scale * 1.4426950408889634f;
-    a.programmatic = false;            // plain launches: starts after everything before it on the stream
-    a.safe_rows = 0;
-    a.unit_len = c->ragged[slot] ? unit_len_dev(c, slot) : nullptr;
-    c->seq += 2;
-    c->last_splitk_seq = c->seq - 1;
-    if (use_mma) {
-        const long long plane_rows = (long long)c->cfg.max_batch * c->cfg.n_kv_heads * c->row_stride;
-        if (kvs::launch_decode_mma(a, plan, c->tensor_map, plane_rows * (2 * slot), plane_rows * (2 * slot + 1), st) !=
-            cudaSuccess)
-            return KVS_ERR_CUDA;
-    } else {
-        if (kvs::launch_decode_scalar(a, plan, st) != cudaSuccess) return KVS_ERR_CUDA;
-    }
-    if (kvs::launch_combine(a, plan, st) != cudaSuccess) return KVS_ERR_CUDA;
-    c->last_plan = plan;
-    c->stats.attention_launches += 1;
-    c->stats.combine_launches += 1;
-    c->stats.kv_bytes_read += 2ull * units * n * c->row_bytes;
-    return KVS_OK;
+    // plain launches: the kernels start after everything before them on the stream
+    const AttentionScratch scratch = {reinterpret_cast<float*>(base + kStaticStatusBytes),
+                                      reinterpret_cast<float*>(base + kStaticStatusBytes + part_o_bytes), status_word,
+                                      false};
+    return run_attention(c, slot, q, out, batch, plan, use_mma, scratch, st);
 }
 
 }  // extern "C"
