@@ -157,24 +157,37 @@ struct PrefillArgs {
 
 // One softmax pass over a 32-column chunk of S: p = 2^(x*scale - m_ref) (0 where masked),
 // split into bf16 hi and lo words (2 keys per word).  Returns the chunk's sum of p.
+// max(a, b, c) in one instruction
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+
+// One softmax pass over a 32-column chunk of S: p = 2^(x*scale - m_ref) (0 where masked),
+// split into bf16 hi and lo words (2 keys per word).  Returns the chunk's sum of p.  The scale,
+// the sum and the hi/lo split use the packed two-float instructions.
 template <bool MASK>
 __device__ __forceinline__ float softmax_chunk(const float (&x)[32], float scale_log2, float m_ref, int key_first,
                                                int limit, uint32_t (&hi)[16], uint32_t (&lo)[16]) {
-    float sum = 0.f;
+    const float2 sc = make_float2(scale_log2, scale_log2), nm = make_float2(-m_ref, -m_ref);
+    const float2 minus1 = make_float2(-1.f, -1.f);
+    float2 sum = make_float2(0.f, 0.f);
 #pragma unroll
     for (int i = 0; i < 32; i += 2) {
-        float p0 = fast_exp2(fmaf(x[i], scale_log2, -m_ref));
-        float p1 = fast_exp2(fmaf(x[i + 1], scale_log2, -m_ref));
+        const float2 t = __ffma2_rn(make_float2(x[i], x[i + 1]), sc, nm);
+        float2 p = make_float2(fast_exp2(t.x), fast_exp2(t.y));
         if (MASK) {
-            p0 = (key_first + i <= limit) ? p0 : 0.f;
-            p1 = (key_first + i + 1 <= limit) ? p1 : 0.f;
+            p.x = (key_first + i <= limit) ? p.x : 0.f;
+            p.y = (key_first + i + 1 <= limit) ? p.y : 0.f;
         }
-        sum += p0 + p1;
-        const uint32_t h = pack2_bf16(p0, p1);
+        sum = __fadd2_rn(sum, p);
+        const uint32_t h = pack2_bf16(p.x, p.y);
         hi[i >> 1] = h;
-        lo[i >> 1] = pack2_bf16(p0 - __uint_as_float(h << 16), p1 - __uint_as_float(h & 0xffff0000u));
+        const float2 r = __ffma2_rn(make_float2(__uint_as_float(h << 16), __uint_as_float(h & 0xffff0000u)), minus1, p);
+        lo[i >> 1] = pack2_bf16(r.x, r.y);
     }
-    return sum;
+    return sum.x + sum.y;
 }
 
 __global__ void __launch_bounds__(kPfThreads, 2)
@@ -324,7 +337,7 @@ __global__ void __launch_bounds__(kPfThreads, 2)
                     for (int i = 0; i < 32; ++i) mx = fmaxf(mx, (key0 + c * 32 + i <= limit) ? x[i] : -INFINITY);
                 } else {
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) mx = fmaxf(mx, x[i]);
+                    for (int i = 0; i < 32; i += 2) mx = fmax3(mx, x[i], x[i + 1]);
                 }
             }
             mx *= a.scale_log2;
