@@ -160,21 +160,27 @@ constexpr int kScalarThreads = kConsumerThreads + 32;
 #ifndef KVS_BLOCKS_PER_SM
 #define KVS_BLOCKS_PER_SM 1
 #endif
-constexpr int kTileBytes = KVS_TILE_BYTES;  // per K tile and per V tile
+constexpr int kTileBytes = KVS_TILE_BYTES;  // per K tile and per V tile (default geometry)
+// Second geometry, used for one q-head per kv-head when a launch streams more than kLongLaunchBytes:
+// 5 stages of 16 KiB tiles sustain ~3 % more on multi-gigabyte launches, the default is better below.
+constexpr int kLongTileBytes = 16384;
+constexpr int kLongStages = 5;
+constexpr long long kLongLaunchBytes = 1500000000LL;
 
-template <typename T, int D, int G>
+template <typename T, int D, int G, int GEOM = 0>
 struct ScalarShape {
+    static constexpr int TILE = GEOM == 1 ? kLongTileBytes : kTileBytes;
     static constexpr int RB = D * (int)sizeof(T);
     static constexpr int LPR = RB / 16;
     static constexpr int EPL = 16 / (int)sizeof(T);
     static constexpr int GPW = 32 / LPR;                  // lane groups per warp
     static constexpr int NG = kConsumerWarps * GPW;       // lane groups per block
-    static constexpr int TN = kTileBytes / RB;            // rows per tile
+    static constexpr int TN = TILE / RB;                  // rows per tile
     static constexpr int R = TN / NG;                     // rows per group per tile
-    static constexpr int STAGES = (G <= 2) ? KVS_STAGES : (6 * 16384) / kTileBytes;
+    static constexpr int STAGES = GEOM == 1 ? kLongStages : ((G <= 2) ? KVS_STAGES : (6 * 16384) / kTileBytes);
     static constexpr int MIN_BLOCKS = (G <= 2) ? KVS_BLOCKS_PER_SM : 1;
     static constexpr int QBYTES = G * RB;
-    static constexpr int STAGE_BYTES = 2 * kTileBytes + QBYTES;
+    static constexpr int STAGE_BYTES = 2 * TILE + QBYTES;
     static constexpr int SCRATCH_FLOATS = NG * (D + 2);
     static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + SCRATCH_FLOATS * 4 + 2 * STAGES * 8 + 16;
     static_assert(R >= 1 && R <= LPR && (R & (R - 1)) == 0, "rows per group must be a power of two <= lanes per row");
@@ -230,10 +236,11 @@ struct ScalarKernelArgs {
     const int* unit_len;  // per-unit row counts of a ragged slot, or nullptr (then n holds for all)
 };
 
-template <typename T, int D, int G>
-__global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G>::MIN_BLOCKS)
+template <typename T, int D, int G, int GEOM>
+__global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G, GEOM>::MIN_BLOCKS)
     decode_splitk_scalar(const ScalarKernelArgs a) {
-    using S = ScalarShape<T, D, G>;
+    using S = ScalarShape<T, D, G, GEOM>;
+    constexpr int kTile = S::TILE;
     constexpr int RB = S::RB, LPR = S::LPR, EPL = S::EPL, NG = S::NG, TN = S::TN, R = S::R, STAGES = S::STAGES;
     constexpr int SH = Log2<LPR>::value - Log2<R>::value;  // lane-in-group >> SH = row index held after the reduction
 
@@ -285,10 +292,10 @@ __global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G>::MIN_BLOC
                 if (kv && bytes) {
                     const long long off = (u * a.row_stride + row0) * (long long)RB;
                     bulk_g2s(sb, a.kplane + off, bytes, &full_bar[st]);
-                    bulk_g2s(sb + kTileBytes, a.vplane + off, bytes, &full_bar[st]);
+                    bulk_g2s(sb + kTile, a.vplane + off, bytes, &full_bar[st]);
                 }
                 if (qpart && with_q)
-                    bulk_g2s(sb + 2 * kTileBytes, a.q + u * (long long)S::QBYTES, S::QBYTES, &full_bar[st]);
+                    bulk_g2s(sb + 2 * kTile, a.q + u * (long long)S::QBYTES, S::QBYTES, &full_bar[st]);
             };
             // Before the preceding kernel in the stream is known to have finished, only K/V
             // tiles made entirely of rows that no kernel still in flight can be writing are
@@ -350,9 +357,9 @@ __global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G>::MIN_BLOC
             const int st = it % STAGES;
             if (!mbar_wait_bounded(&full_bar[st], (it / STAGES) & 1, abort_flag, a.status)) return;
             const unsigned char* ks = stage_base + st * S::STAGE_BYTES;
-            const unsigned char* vs = ks + kTileBytes;
+            const unsigned char* vs = ks + kTile;
             if (k == 0) {
-                const unsigned char* qs = vs + kTileBytes;
+                const unsigned char* qs = vs + kTile;
 #pragma unroll
                 for (int g = 0; g < G; ++g) {
                     const uint4 raw = *reinterpret_cast<const uint4*>(qs + g * RB + lig * 16);
@@ -496,41 +503,46 @@ cudaError_t launch_combine(const DecodeArgs& a, const DecodePlan& plan, cudaStre
 // --------------------------------------------------------------------------------------
 // Launch plumbing for the scalar kernel.
 // --------------------------------------------------------------------------------------
-template <typename T, int D, int G>
+template <typename T, int D, int G, int GEOM>
 static cudaError_t set_attr_one() {
-    return cudaFuncSetAttribute(decode_splitk_scalar<T, D, G>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                ScalarShape<T, D, G>::SMEM_BYTES);
+    return cudaFuncSetAttribute(decode_splitk_scalar<T, D, G, GEOM>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                ScalarShape<T, D, G, GEOM>::SMEM_BYTES);
 }
 
 template <typename T, int D>
 static cudaError_t set_attr_groups() {
     cudaError_t e;
-    if ((e = set_attr_one<T, D, 1>()) != cudaSuccess) return e;
-    if ((e = set_attr_one<T, D, 2>()) != cudaSuccess) return e;
-    if ((e = set_attr_one<T, D, 4>()) != cudaSuccess) return e;
-    return set_attr_one<T, D, 8>();
+    if ((e = set_attr_one<T, D, 1, 0>()) != cudaSuccess) return e;
+    if ((e = set_attr_one<T, D, 1, 1>()) != cudaSuccess) return e;
+    if ((e = set_attr_one<T, D, 2, 0>()) != cudaSuccess) return e;
+    if ((e = set_attr_one<T, D, 4, 0>()) != cudaSuccess) return e;
+    return set_attr_one<T, D, 8, 0>();
 }
 
-template <typename T, int D, int G>
+template <typename T, int D, int G, int GEOM>
 static cudaError_t launch_scalar_one(const ScalarKernelArgs& ka, int NC, bool programmatic, cudaStream_t stream) {
-    return launch_kernel(decode_splitk_scalar<T, D, G>, dim3(NC), dim3(kScalarThreads),
-                         ScalarShape<T, D, G>::SMEM_BYTES, stream, programmatic, ka);
+    return launch_kernel(decode_splitk_scalar<T, D, G, GEOM>, dim3(NC), dim3(kScalarThreads),
+                         ScalarShape<T, D, G, GEOM>::SMEM_BYTES, stream, programmatic, ka);
 }
 
 template <typename T, int D>
-static cudaError_t launch_scalar_groups(int G, const ScalarKernelArgs& ka, int NC, bool pdl, cudaStream_t stream) {
+static cudaError_t launch_scalar_groups(int G, int geom, const ScalarKernelArgs& ka, int NC, bool pdl,
+                                        cudaStream_t stream) {
     switch (G) {
-        case 1: return launch_scalar_one<T, D, 1>(ka, NC, pdl, stream);
-        case 2: return launch_scalar_one<T, D, 2>(ka, NC, pdl, stream);
-        case 4: return launch_scalar_one<T, D, 4>(ka, NC, pdl, stream);
-        case 8: return launch_scalar_one<T, D, 8>(ka, NC, pdl, stream);
+        case 1:
+            return geom == 1 ? launch_scalar_one<T, D, 1, 1>(ka, NC, pdl, stream)
+                             : launch_scalar_one<T, D, 1, 0>(ka, NC, pdl, stream);
+        case 2: return launch_scalar_one<T, D, 2, 0>(ka, NC, pdl, stream);
+        case 4: return launch_scalar_one<T, D, 4, 0>(ka, NC, pdl, stream);
+        case 8: return launch_scalar_one<T, D, 8, 0>(ka, NC, pdl, stream);
         default: return cudaErrorInvalidValue;
     }
 }
 
 void plan_decode_scalar(int units, int n, int G, int D, int dtype, int sm_count, int max_ctas, DecodePlan* plan) {
     const int rb = D * (dtype == 0 ? 2 : 4);
-    plan->tile_rows = kTileBytes / rb;
+    plan->geom = (G == 1 && 2LL * units * n * rb >= kLongLaunchBytes) ? 1 : 0;
+    plan->tile_rows = (plan->geom == 1 ? kLongTileBytes : kTileBytes) / rb;
     plan->tpu = (n + plan->tile_rows - 1) / plan->tile_rows;
     plan->T = (long long)units * plan->tpu;
     const int per_sm = (G <= 2) ? KVS_BLOCKS_PER_SM : 1;
@@ -558,11 +570,11 @@ cudaError_t launch_decode_scalar(const DecodeArgs& a, const DecodePlan& plan, cu
     ka.unit_len = a.unit_len;
     const bool pdl = a.programmatic;
     if (a.dtype == 0) {
-        if (a.D == 128) return launch_scalar_groups<__nv_bfloat16, 128>(a.G, ka, plan.NC, pdl, stream);
-        if (a.D == 64) return launch_scalar_groups<__nv_bfloat16, 64>(a.G, ka, plan.NC, pdl, stream);
+        if (a.D == 128) return launch_scalar_groups<__nv_bfloat16, 128>(a.G, plan.geom, ka, plan.NC, pdl, stream);
+        if (a.D == 64) return launch_scalar_groups<__nv_bfloat16, 64>(a.G, plan.geom, ka, plan.NC, pdl, stream);
     } else {
-        if (a.D == 128) return launch_scalar_groups<float, 128>(a.G, ka, plan.NC, pdl, stream);
-        if (a.D == 64) return launch_scalar_groups<float, 64>(a.G, ka, plan.NC, pdl, stream);
+        if (a.D == 128) return launch_scalar_groups<float, 128>(a.G, plan.geom, ka, plan.NC, pdl, stream);
+        if (a.D == 64) return launch_scalar_groups<float, 64>(a.G, plan.geom, ka, plan.NC, pdl, stream);
     }
     return cudaErrorInvalidValue;
 }
