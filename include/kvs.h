@@ -87,11 +87,14 @@ typedef struct {
 typedef enum {
     KVS_OPT_MAX_CTAS = 0,   /* upper bound on thread blocks of the split-K kernel; 0 = auto  */
     KVS_OPT_KERNEL = 1,     /* 0 = auto, 1 = scalar-FMA path, 2 = grouped tensor-core path   */
-    KVS_OPT_EARLY_START = 2 /* 1 (default): kernels are launched so that they may start while
+    KVS_OPT_EARLY_START = 2,/* 1 (default): kernels are launched so that they may start while
                                the previous kernel on the stream drains, and prefetch K/V rows
                                that nothing in flight writes; they wait for the previous kernel
                                before reading q, newly appended rows, or writing anything.
                                0: plain stream-ordered launches.  Results are identical.      */
+    KVS_OPT_REPLAY = 3      /* 1: launches also read a device-side growth counter, so that a
+                               recorded decode step can be replayed as a CUDA graph (see
+                               kvs_replay_advance).  0 (default): lengths come from the host only. */
 } kvs_option;
 
 /* ---- life cycle ------------------------------------------------------------ */
@@ -221,6 +224,32 @@ kvs_status kvs_layer_distances(kvs_ctx* ctx, int32_t batch, float* dist, void* s
  * over the samples and *out (device, float32) receives cos(mean a, mean b).  Two kernels.       */
 kvs_status kvs_mean_cosine(kvs_ctx* ctx, const void* a, const void* b, int32_t n_samples, int64_t dim,
                            float* out, void* stream);
+
+/* ---- replaying a recorded decode step (CUDA graphs) ------------------------------------------
+ * Slot lengths are host-side numbers baked into each launch, so a recorded launch would repeat
+ * the same step.  With KVS_OPT_REPLAY = 1 every kvs_append / kvs_decode_attention launch also
+ * adds a device-side counter to the lengths it was recorded with, and kvs_replay_advance
+ * (record it as the last call of the step) adds one to that counter.  Each replay of
+ * [append + attention for every layer, kvs_replay_advance] then appends one row further along and
+ * attends over one row more: it is the next decode step (its inputs are read from the same device
+ * buffers, which the caller refills between replays).  The thread blocks launched stay as
+ * recorded; the split of the rows among them follows the grown length.
+ *   - kvs_replay_advance only records something while `stream` is being captured; called on a
+ *     stream that is not capturing it does nothing, so the same step function can first be run
+ *     eagerly (an ordinary step) and then recorded.
+ *   - While a stream is being captured, calls do their host bookkeeping as usual: the context's
+ *     lengths advance as if the recorded step had run once.
+ *   - After the recorded step has run `times_run` times in all (graph launches; if it was also
+ *     run eagerly before capture with the counter at zero, those runs are ordinary steps and are
+ *     not counted), call kvs_replay_commit(ctx, times_run, stream): the host lengths catch up
+ *     (times_run - 1 more rows) and the counter is cleared on `stream`.  Make no eager call on
+ *     the context between the first replay and the commit.
+ *   - One-token decode steps only; every computing layer must append exactly once per step.
+ *   - A replay that would pass max_seq appends nothing for that layer and sets the device status
+ *     word to KVS_ERR_CAPACITY; kvs_replay_commit returns CAPACITY instead of advancing.
+ * Errors: STATE unless bound and KVS_OPT_REPLAY is 1; INVALID_ARG for times_run < 1.            */
+kvs_status kvs_replay_advance(kvs_ctx* ctx, void* stream);
+kvs_status kvs_replay_commit(kvs_ctx* ctx, int32_t times_run, void* stream);
 
 /* One whole decode step from HOST buffers: for every layer in order, append the
  * layer's new token (own-cache layers only) and run its attention.

@@ -8,7 +8,7 @@ from __future__ import annotations
 
 from . import binding
 from .binding import (  # noqa: F401
-    KVS_BF16, KVS_F32, KVS_OK, KVS_OPT_EARLY_START, KVS_OPT_KERNEL, KVS_OPT_MAX_CTAS, KvsError,
+    KVS_BF16, KVS_F32, KVS_OK, KVS_OPT_EARLY_START, KVS_OPT_KERNEL, KVS_OPT_MAX_CTAS, KVS_OPT_REPLAY, KvsError,
 )
 
 __all__ = ["binding", "SharedKVCache", "KvsError"]
@@ -119,6 +119,12 @@ class SharedKVCache:
         out = torch.empty(1, dtype=torch.float32, device=self.device)
         binding.kvs_mean_cosine(self.ctx, a, b, a.shape[0], a.shape[1], out, self._stream())
         return out
+
+    def replay_advance(self):
+        binding.kvs_replay_advance(self.ctx, self._stream())
+
+    def replay_commit(self, times_run):
+        binding.kvs_replay_commit(self.ctx, times_run, self._stream())
 
     def step_host(self, q_host, k_host, v_host, out_host):
         """One decode step over all layers from host tensors (see ``kvs_step_host``)."""

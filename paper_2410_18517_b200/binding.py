@@ -29,6 +29,7 @@ KVS_F32 = 1
 KVS_OPT_MAX_CTAS = 0
 KVS_OPT_KERNEL = 1
 KVS_OPT_EARLY_START = 2
+KVS_OPT_REPLAY = 3
 
 # every symbol include/kvs.h declares
 EXPORTS = (
@@ -38,6 +39,7 @@ EXPORTS = (
     "kvs_last_device_status", "kvs_set_option", "kvs_last_launch", "kvs_status_string",
     "kvs_read_roof", "kvs_decode_attention_static", "kvs_prefill_attention",
     "kvs_evict", "kvs_unit_len", "kvs_layer_distances", "kvs_mean_cosine",
+    "kvs_replay_advance", "kvs_replay_commit",
 )
 
 
@@ -87,6 +89,8 @@ def load() -> ctypes.CDLL:
         "kvs_prefill_attention": [vp, i32, vp, vp, i32, i32, vp],
         "kvs_evict": [vp, i32, vp, P(i32), i32, i32, vp],
         "kvs_unit_len": [vp, i32, i32, i32, P(i32)],
+        "kvs_replay_advance": [vp, vp],
+        "kvs_replay_commit": [vp, i32, vp],
         "kvs_layer_distances": [vp, i32, vp, vp],
         "kvs_mean_cosine": [vp, vp, vp, i32, ctypes.c_int64, vp, vp],
         "kvs_step_host": [vp, vp, vp, vp, vp, i32, vp, P(ctypes.c_uint64), P(ctypes.c_uint64)],
@@ -198,6 +202,14 @@ def kvs_layer_distances(ctx: int, batch: int, dist, stream: int = 0) -> None:
 
 def kvs_mean_cosine(ctx: int, a, b, n_samples: int, dim: int, out, stream: int = 0) -> None:
     _check(load().kvs_mean_cosine(ctx, _ptr(a), _ptr(b), n_samples, dim, _ptr(out), stream), "kvs_mean_cosine")
+
+
+def kvs_replay_advance(ctx: int, stream: int = 0) -> None:
+    _check(load().kvs_replay_advance(ctx, stream), "kvs_replay_advance")
+
+
+def kvs_replay_commit(ctx: int, times_run: int, stream: int = 0) -> None:
+    _check(load().kvs_replay_commit(ctx, times_run, stream), "kvs_replay_commit")
 
 
 def kvs_decode_attention_static(ctx: int, layer: int, q, out, batch: int, stream: int = 0, device_status=None) -> None:

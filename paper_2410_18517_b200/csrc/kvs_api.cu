@@ -45,7 +45,7 @@ struct kvs_ctx {
 
     // workspace carve-up (byte offsets)
     size_t off_status = 0, off_part_o = 0, off_part_ml = 0, off_stage_q = 0, off_stage_k = 0, off_stage_v = 0,
-           off_stage_out = 0, off_unit_len = 0, off_counts = 0, off_search = 0, ws_bytes = 0;
+           off_stage_out = 0, off_unit_len = 0, off_counts = 0, off_search = 0, off_replay = 0, ws_bytes = 0;
 
     alignas(64) unsigned char tensor_map[128];  // TMA view of the pool (bf16 storage only)
     bool have_tensor_map = false;
@@ -68,6 +68,7 @@ struct kvs_ctx {
     int opt_max_ctas = 0;
     int opt_kernel = 0;
     int opt_pdl = 1;
+    int opt_replay = 0;   // launches carry the device-side growth counter (for CUDA-graph replay)
     kvs::DecodePlan last_plan{};
     kvs_stats_t stats{};
 };
@@ -97,6 +98,10 @@ void resolve_map(kvs_ctx* c) {
     c->app_start_latest.assign(n, 0);
     c->ragged.assign(n, 0);
     c->unit_len_host.assign(n, std::vector<int32_t>());
+}
+
+const int* replay_counter(const kvs_ctx* c) {
+    return c->opt_replay ? reinterpret_cast<const int*>(c->ws + c->off_replay) : nullptr;
 }
 
 int* unit_len_dev(const kvs_ctx* c, int slot) {
@@ -135,6 +140,8 @@ void layout_workspace(kvs_ctx* c) {
     off = align_up(off + L * units * sizeof(int32_t), kAlign);
     c->off_counts = off;        // staging for the kept-row counts of one kvs_evict call
     off = align_up(off + units * sizeof(int32_t), kAlign);
+    c->off_replay = off;        // one int: rows every slot has grown by since a recorded launch
+    off += kAlign;
     c->off_search = off;        // per-block partial sums of the strategy-search reductions
     {
         const size_t need = std::max(kvs::distance_partial_bytes(f.n_layers <= kvs::kMaxLayersSearch ? f.n_layers : 4),
@@ -203,7 +210,8 @@ kvs_status do_append(kvs_ctx* c, int layer, const void* k, const void* v, int ba
     char* vp = kp + c->plane_bytes;
     const bool rag = c->ragged[slot] != 0;
     if (kvs::launch_append(k, v, kp, vp, batch, n_new, c->cfg.n_kv_heads, c->row_bytes, c->row_stride,
-                           c->slot_len[slot], rag ? unit_len_dev(c, slot) : nullptr, c->opt_pdl != 0, st) != cudaSuccess)
+                           c->slot_len[slot], rag ? unit_len_dev(c, slot) : nullptr, replay_counter(c), c->cfg.max_seq,
+                           reinterpret_cast<int*>(c->ws + c->off_status), c->opt_pdl != 0, st) != cudaSuccess)
         return KVS_ERR_CUDA;
     if (rag) {
         const int units = batch * c->cfg.n_kv_heads;
@@ -263,6 +271,7 @@ kvs_status run_attention(kvs_ctx* c, int slot, const void* q, float* out, int ba
     a.programmatic = scratch.programmatic;
     a.safe_rows = scratch.programmatic ? safe_rows_of(c, slot) : 0;
     a.unit_len = c->ragged[slot] ? unit_len_dev(c, slot) : nullptr;
+    a.n_extra = replay_counter(c);
     c->seq += 2;                       // split-K kernel, then combine
     c->last_splitk_seq = c->seq - 1;
     if (use_mma) {
@@ -562,6 +571,42 @@ kvs_status kvs_mean_cosine(kvs_ctx* ctx, const void* a, const void* b, int32_t n
     return KVS_OK;
 }
 
+kvs_status kvs_replay_advance(kvs_ctx* ctx, void* stream) {
+    if (!ctx) return KVS_ERR_INVALID_ARG;
+    if (!ctx->bound || !ctx->opt_replay) return KVS_ERR_STATE;
+    DeviceGuard guard(ctx->cfg.device);
+    if (!guard.ok) return KVS_ERR_CUDA;
+    // Outside stream capture the host lengths already advance with every call, so there is nothing
+    // to count: the same step function can be run eagerly and recorded.
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(static_cast<cudaStream_t>(stream), &cap) != cudaSuccess) return KVS_ERR_CUDA;
+    if (cap != cudaStreamCaptureStatusActive) return KVS_OK;
+    if (kvs::launch_replay_advance(reinterpret_cast<int*>(ctx->ws + ctx->off_replay), ctx->opt_pdl != 0,
+                                   static_cast<cudaStream_t>(stream)) != cudaSuccess)
+        return KVS_ERR_CUDA;
+    ctx->seq += 1;
+    return KVS_OK;
+}
+
+kvs_status kvs_replay_commit(kvs_ctx* ctx, int32_t times_run, void* stream) {
+    if (!ctx || times_run < 1) return KVS_ERR_INVALID_ARG;
+    if (!ctx->bound || !ctx->opt_replay) return KVS_ERR_STATE;
+    const int extra = times_run - 1;     // the recording itself was already counted once
+    for (int s = 0; s < ctx->n_slots; ++s)
+        if (ctx->slot_len[s] > 0 && (long long)ctx->slot_len[s] + extra > ctx->cfg.max_seq) return KVS_ERR_CAPACITY;
+    DeviceGuard guard(ctx->cfg.device);
+    if (!guard.ok) return KVS_ERR_CUDA;
+    if (cudaMemsetAsync(ctx->ws + ctx->off_replay, 0, sizeof(int), static_cast<cudaStream_t>(stream)) != cudaSuccess)
+        return KVS_ERR_CUDA;
+    for (int s = 0; s < ctx->n_slots; ++s) {
+        if (ctx->slot_len[s] == 0) continue;
+        ctx->slot_len[s] += extra;
+        if (ctx->ragged[s])
+            for (int u = 0; u < ctx->cur_batch * ctx->cfg.n_kv_heads; ++u) ctx->unit_len_host[s][u] += extra;
+    }
+    return KVS_OK;
+}
+
 kvs_status kvs_step_host(kvs_ctx* ctx, const void* q_host, const void* k_host, const void* v_host, float* out_host,
                          int32_t batch, void* stream, uint64_t* h2d_bytes, uint64_t* d2h_bytes) {
     if (!ctx || !q_host || !k_host || !v_host || !out_host) return KVS_ERR_INVALID_ARG;
@@ -713,6 +758,10 @@ kvs_status kvs_set_option(kvs_ctx* ctx, int32_t option, int32_t value) {
         case KVS_OPT_EARLY_START:
             if (value != 0 && value != 1) return KVS_ERR_INVALID_ARG;
             ctx->opt_pdl = value;
+            return KVS_OK;
+        case KVS_OPT_REPLAY:
+            if (value != 0 && value != 1) return KVS_ERR_INVALID_ARG;
+            ctx->opt_replay = value;
             return KVS_OK;
         case KVS_OPT_KERNEL:
             if (value < 0 || value > 2) return KVS_ERR_INVALID_ARG;

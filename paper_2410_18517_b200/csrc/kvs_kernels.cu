@@ -17,9 +17,15 @@ namespace kvs {
 __global__ void __launch_bounds__(256) kv_append_kernel(const uint4* __restrict__ k, const uint4* __restrict__ v,
                                                         uint4* __restrict__ kplane, uint4* __restrict__ vplane,
                                                         long long total_vecs, int n_new, int Hkv, int row_vecs,
-                                                        int row_stride, int len0, const int* __restrict__ unit_len) {
+                                                        int row_stride, int len0, const int* __restrict__ unit_len,
+                                                        const int* __restrict__ n_extra, int capacity, int* status) {
     pdl_launch_dependents();
     pdl_wait();
+    if (n_extra) len0 += *n_extra;   // replayed launch: the slot has grown since the launch was recorded
+    if (!unit_len && len0 + n_new > capacity) {   // can only happen in a replay that outran the capacity
+        if (threadIdx.x == 0 && blockIdx.x == 0) atomicExch(status, 4);
+        return;
+    }
     const uint4* __restrict__ src = blockIdx.y == 0 ? k : v;
     uint4* __restrict__ dst = blockIdx.y == 0 ? kplane : vplane;
     for (long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x; idx < total_vecs;
@@ -37,13 +43,15 @@ __global__ void __launch_bounds__(256) kv_append_kernel(const uint4* __restrict_
 }
 
 cudaError_t launch_append(const void* k, const void* v, void* kplane, void* vplane, int B, int n_new, int Hkv,
-                          int row_bytes, int row_stride, int len0, const int* unit_len, bool programmatic, cudaStream_t stream) {
+                          int row_bytes, int row_stride, int len0, const int* unit_len, const int* n_extra, int capacity, int* status,
+                          bool programmatic, cudaStream_t stream) {
     const int row_vecs = row_bytes / 16;
     const long long total = (long long)B * n_new * Hkv * row_vecs;
     const long long blocks = std::min<long long>((total + 255) / 256, 148 * 16);
     dim3 grid((unsigned)blocks, 2);
     return launch_kernel(kv_append_kernel, grid, dim3(256), 0, stream, programmatic, (const uint4*)k, (const uint4*)v,
-                         (uint4*)kplane, (uint4*)vplane, total, n_new, Hkv, row_vecs, row_stride, len0, unit_len);
+                         (uint4*)kplane, (uint4*)vplane, total, n_new, Hkv, row_vecs, row_stride, len0, unit_len, n_extra, capacity,
+                         status);
 }
 
 // --------------------------------------------------------------------------------------
@@ -110,6 +118,16 @@ cudaError_t launch_evict(void* kplane, void* vplane, const int* keep, const int*
 cudaError_t launch_set_len(int* unit_len, const int* counts, int units, bool programmatic, cudaStream_t stream) {
     return launch_kernel(set_len_kernel, dim3((units + 127) / 128), dim3(128), 0, stream, programmatic, unit_len, counts,
                          units);
+}
+
+__global__ void replay_advance_kernel(int* n_extra) {
+    pdl_launch_dependents();
+    pdl_wait();
+    if (threadIdx.x == 0) *n_extra += 1;
+}
+
+cudaError_t launch_replay_advance(int* n_extra, bool programmatic, cudaStream_t stream) {
+    return launch_kernel(replay_advance_kernel, dim3(1), dim3(32), 0, stream, programmatic, n_extra);
 }
 
 cudaError_t launch_add_len(int* unit_len, int delta, int units, bool programmatic, cudaStream_t stream) {
@@ -234,12 +252,22 @@ struct ScalarKernelArgs {
     float scale_log2;
     int safe_rows;  // rows of every unit that no kernel possibly still running writes
     const int* unit_len;  // per-unit row counts of a ragged slot, or nullptr (then n holds for all)
+    const int* n_extra;   // graph replay: rows every slot has grown by since the launch was recorded, or nullptr
+    int units;
 };
 
 template <typename T, int D, int G, int GEOM>
 __global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G, GEOM>::MIN_BLOCKS)
-    decode_splitk_scalar(const ScalarKernelArgs a) {
+    decode_splitk_scalar(const ScalarKernelArgs a_in) {
     using S = ScalarShape<T, D, G, GEOM>;
+    ScalarKernelArgs a = a_in;
+    if (a.n_extra != nullptr) {
+        // A replayed launch: the lengths recorded with it have grown on the device since.
+        pdl_wait();
+        a.n += *a.n_extra;
+        a.tpu = (a.n + S::TN - 1) / S::TN;
+        a.T = (long long)a.units * a.tpu;
+    }
     constexpr int kTile = S::TILE;
     constexpr int RB = S::RB, LPR = S::LPR, EPL = S::EPL, NG = S::NG, TN = S::TN, R = S::R, STAGES = S::STAGES;
     constexpr int SH = Log2<LPR>::value - Log2<R>::value;  // lane-in-group >> SH = row index held after the reduction
@@ -474,9 +502,14 @@ __global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G, GEOM>::MI
 // piece order so that the result does not depend on which block finished first.
 // --------------------------------------------------------------------------------------
 __global__ void decode_combine_kernel(const float* __restrict__ part_o, const float* __restrict__ part_ml,
-                                      float* __restrict__ out, int G, int D, int tpu, long long T, int NC) {
+                                      float* __restrict__ out, int G, int D, int tpu, long long T, int NC,
+                                      const int* __restrict__ n_extra, int n, int tile_rows, int units) {
     pdl_launch_dependents();
     pdl_wait();
+    if (n_extra) {   // replayed launch: recompute the tile line from the grown length
+        tpu = (n + *n_extra + tile_rows - 1) / tile_rows;
+        T = (long long)units * tpu;
+    }
     const long long u = blockIdx.x / G;
     const int g = blockIdx.x % G;
     const int c0 = cta_of_tile(u * tpu, T, NC);
@@ -497,7 +530,8 @@ __global__ void decode_combine_kernel(const float* __restrict__ part_o, const fl
 
 cudaError_t launch_combine(const DecodeArgs& a, const DecodePlan& plan, cudaStream_t stream) {
     return launch_kernel(decode_combine_kernel, dim3(a.units * a.G), dim3(a.D), 0, stream, a.programmatic,
-                         (const float*)a.part_o, (const float*)a.part_ml, a.out, a.G, a.D, plan.tpu, plan.T, plan.NC);
+                         (const float*)a.part_o, (const float*)a.part_ml, a.out, a.G, a.D, plan.tpu, plan.T, plan.NC, a.n_extra,
+                         a.n, plan.tile_rows, a.units);
 }
 
 // --------------------------------------------------------------------------------------
@@ -568,6 +602,9 @@ cudaError_t launch_decode_scalar(const DecodeArgs& a, const DecodePlan& plan, cu
     ka.scale_log2 = a.scale_log2;
     ka.safe_rows = (a.programmatic && !a.unit_len) ? a.safe_rows : 0;
     ka.unit_len = a.unit_len;
+    ka.n_extra = a.n_extra;
+    ka.units = a.units;
+    if (a.n_extra) ka.safe_rows = 0;   // the tile line is only known after the wait
     const bool pdl = a.programmatic;
     if (a.dtype == 0) {
         if (a.D == 128) return launch_scalar_groups<__nv_bfloat16, 128>(a.G, plan.geom, ka, plan.NC, pdl, stream);

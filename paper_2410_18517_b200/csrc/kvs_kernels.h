@@ -37,6 +37,7 @@ struct DecodeArgs {
     int dtype;            // 0 bf16, 1 f32
     float scale_log2;     // softmax scale * log2(e)
     const int* unit_len;  // device, [units]: rows cached per unit when units differ (else nullptr and n holds)
+    const int* n_extra;   // device int: rows grown since the launch was recorded (graph replay), or nullptr
     int safe_rows;        // rows per unit that no kernel possibly still in flight is writing
     bool programmatic;    // launch with programmatic stream serialization (early start, explicit wait)
 };
@@ -80,7 +81,9 @@ cudaError_t launch_mean_cosine(const void* a, const void* b, int S, long long di
                                float* out, int sm_count, cudaStream_t stream);
 
 cudaError_t launch_append(const void* k, const void* v, void* kplane, void* vplane, int B, int n_new, int Hkv,
-                          int row_bytes, int row_stride, int len0, const int* unit_len, bool programmatic, cudaStream_t stream);
+                          int row_bytes, int row_stride, int len0, const int* unit_len, const int* n_extra, int capacity, int* status,
+                          bool programmatic, cudaStream_t stream);
+cudaError_t launch_replay_advance(int* n_extra, bool programmatic, cudaStream_t stream);
 
 // Ragged slots (rows evicted by an outside intra-layer method).
 //   launch_evict:   per unit u, rows keep[u*keep_stride + j], j < counts[u], move to rows 0..counts[u]-1

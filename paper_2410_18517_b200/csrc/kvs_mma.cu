@@ -105,14 +105,24 @@ struct MmaKernelArgs {
     int safe_rows;  // rows of every unit that no kernel possibly still running writes
     const int* unit_len;  // per-unit row counts of a ragged slot, or nullptr (then n holds for all)
     int G;          // q-heads per kv-head, 1..8
+    const int* n_extra;  // graph replay: rows every slot has grown by since the launch was recorded, or nullptr
+    int units;
 };
 
 // G (q-heads per kv-head, 1..8) is a run-time argument: it only selects which rows of the padded
 // 16-row M side are real, so one kernel per head size serves every group size.
 template <int D>
 __global__ void __launch_bounds__(kMmaThreads, KVS_MMA_BLOCKS_PER_SM)
-    decode_splitk_mma(const __grid_constant__ CUtensorMap tmap, const MmaKernelArgs a) {
+    decode_splitk_mma(const __grid_constant__ CUtensorMap tmap, const MmaKernelArgs a_in) {
     using S = MmaShape<D>;
+    MmaKernelArgs a = a_in;
+    if (a.n_extra != nullptr) {
+        // A replayed launch: the lengths recorded with it have grown on the device since.
+        pdl_wait();
+        a.n += *a.n_extra;
+        a.tpu = (a.n + S::TN - 1) / S::TN;
+        a.T = (long long)a.units * a.tpu;
+    }
     constexpr int TN = S::TN, KSTEPS = S::KSTEPS, NB = S::NB, BPW = S::BPW;
     const int G = a.G;
     const int QBYTES = G * S::RB;
@@ -434,6 +444,9 @@ cudaError_t launch_decode_mma(const DecodeArgs& a, const DecodePlan& plan, const
     ka.unit_len = a.unit_len;
     const CUtensorMap& tm = *reinterpret_cast<const CUtensorMap*>(tensor_map);
     ka.G = a.G;
+    ka.n_extra = a.n_extra;
+    ka.units = a.units;
+    if (a.n_extra) ka.safe_rows = 0;   // the tile line is only known after the wait
     if (a.G < 1 || a.G > 8) return cudaErrorInvalidValue;
     if (a.D == 128) return launch_one<128>(tm, ka, plan.NC, a.programmatic, stream);
     if (a.D == 64) return launch_one<64>(tm, ka, plan.NC, a.programmatic, stream);

@@ -5,9 +5,9 @@ tokens/s, KV-read GB/s and pool size.
     python -m paper_2410_18517_b200.sweep [--out FILE] [--steps K] [--only B,N,P]
 
 A *step* is one pass over all layers (append on computing layers + attention on every layer).
-Each point is timed twice: launched call by call from Python, and as a replay of a CUDA graph of
-one step (which takes the host's launch cost out; the graph re-runs the same step, so the cache
-length stays fixed while it is timed).  All computing layers are loaded with the same seeded K/V
+Each point is timed twice: launched call by call from Python, and as replays of a CUDA graph of one
+recorded step (which takes the host's launch cost out; with the library's replay counter every
+replay is the next decode step, one row further along).  All computing layers are loaded with the same seeded K/V
 block: values do not affect bandwidth and parity is checked elsewhere.
 """
 from __future__ import annotations
@@ -19,7 +19,7 @@ import sys
 import torch
 
 import synth_inputs as si
-from paper_2410_18517_b200 import SharedKVCache
+from paper_2410_18517_b200 import KVS_OPT_REPLAY, SharedKVCache
 
 HBM_BYTES_USABLE = 170 * 2**30      # leave head-room below the 180 GB of a B200
 
@@ -30,7 +30,7 @@ def pool_bytes(w: si.Workload, extra_rows: int) -> int:
 
 
 def time_point(w: si.Workload, steps: int, device=0) -> dict:
-    extra = 2 * steps + 16
+    extra = 3 * steps + 24
     rec = {"workload": w.name, "batch": w.B, "context": w.context, "shared_layers": w.n_shared,
            "pool_bytes": pool_bytes(w, extra), "pool_bytes_unshared": pool_bytes(w.scaled(n_shared=0), extra)}
     if rec["pool_bytes"] > HBM_BYTES_USABLE:
@@ -49,12 +49,15 @@ def time_point(w: si.Workload, steps: int, device=0) -> dict:
     ins = [si.step_qkv(w, 0, l, device=dev) for l in range(w.L)]
     outs = [torch.empty(w.B, w.Hq, w.D, dtype=torch.float32, device=dev) for _ in range(w.L)]
 
+    cache.set_option(KVS_OPT_REPLAY, 1)
+
     def one_step():
         for l in range(w.L):
             q, kk, vv = ins[l]
             if sm[l] == l:
                 cache.append(l, kk, vv)
             cache.decode_attention(l, q, outs[l])
+        cache.replay_advance()           # recorded only while capturing
 
     def timed(fn, n):
         torch.cuda.synchronize(dev)
@@ -88,6 +91,9 @@ def time_point(w: si.Workload, steps: int, device=0) -> dict:
     torch.cuda.current_stream(dev).wait_stream(side)
     graph.replay()
     ms_g = timed(graph.replay, steps)
+    cache.replay_commit(1 + steps)
+    torch.cuda.synchronize(dev)
+    rec.update(replayed_to=cache.seq_len(0))
     rec.update(graph_ms_per_step=ms_g, graph_tokens_per_s=w.B / (ms_g * 1e-3),
                graph_kv_read_gbs=read_graph / (ms_g * 1e-3) / 1e9, device_status=cache.device_status())
     cache.close()
