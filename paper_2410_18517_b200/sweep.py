@@ -7,8 +7,8 @@ tokens/s, KV-read GB/s and pool size.
 A *step* is one pass over all layers (append on computing layers + attention on every layer).
 Each point is timed twice: launched call by call from Python, and as replays of a CUDA graph of one
 recorded step (which takes the host's launch cost out; with the library's replay counter every
-replay is the next decode step, one row further along).  All computing layers are loaded with the same seeded K/V
-block: values do not affect bandwidth and parity is checked elsewhere.
+replay is the next decode step, one row further along).  All computing layers are loaded with the
+same seeded K/V block: values do not affect bandwidth and parity is checked elsewhere.
 """
 from __future__ import annotations
 
@@ -49,8 +49,6 @@ def time_point(w: si.Workload, steps: int, device=0) -> dict:
     ins = [si.step_qkv(w, 0, l, device=dev) for l in range(w.L)]
     outs = [torch.empty(w.B, w.Hq, w.D, dtype=torch.float32, device=dev) for _ in range(w.L)]
 
-    cache.set_option(KVS_OPT_REPLAY, 1)
-
     def one_step():
         for l in range(w.L):
             q, kk, vv = ins[l]
@@ -78,7 +76,8 @@ def time_point(w: si.Workload, steps: int, device=0) -> dict:
                kv_bytes_read_per_step=read_per_step, kernel=cache.last_launch()["kernel"],
                ctas=cache.last_launch()["ctas"])
 
-    # graph replay of one step
+    # graph replays of one recorded step; the replay counter makes every replay the next step
+    cache.set_option(KVS_OPT_REPLAY, 1)
     side = torch.cuda.Stream(device=dev)
     side.wait_stream(torch.cuda.current_stream(dev))
     with torch.cuda.stream(side):
