@@ -69,6 +69,10 @@ struct kvs_ctx {
     int opt_kernel = 0;
     int opt_pdl = 1;
     int opt_replay = 0;   // launches carry the device-side growth counter (for CUDA-graph replay)
+    // The split-K kernels read the growth counter before their wait.  That is safe because the
+    // first launch after anything wrote the counter never starts early (full dependency): it and
+    // everything after it then begin with the write complete.
+    bool counter_written = false;
     kvs::DecodePlan last_plan{};
     kvs_stats_t stats{};
 };
@@ -98,6 +102,13 @@ void resolve_map(kvs_ctx* c) {
     c->app_start_latest.assign(n, 0);
     c->ragged.assign(n, 0);
     c->unit_len_host.assign(n, std::vector<int32_t>());
+}
+
+// Whether the next launch may start early; consumes the "counter was just written" mark.
+bool take_early_start(kvs_ctx* c) {
+    const bool early = c->opt_pdl != 0 && !c->counter_written;
+    c->counter_written = false;
+    return early;
 }
 
 const int* replay_counter(const kvs_ctx* c) {
@@ -211,7 +222,7 @@ kvs_status do_append(kvs_ctx* c, int layer, const void* k, const void* v, int ba
     const bool rag = c->ragged[slot] != 0;
     if (kvs::launch_append(k, v, kp, vp, batch, n_new, c->cfg.n_kv_heads, c->row_bytes, c->row_stride,
                            c->slot_len[slot], rag ? unit_len_dev(c, slot) : nullptr, replay_counter(c), c->cfg.max_seq,
-                           reinterpret_cast<int*>(c->ws + c->off_status), c->opt_pdl != 0, st) != cudaSuccess)
+                           reinterpret_cast<int*>(c->ws + c->off_status), take_early_start(c), st) != cudaSuccess)
         return KVS_ERR_CUDA;
     if (rag) {
         const int units = batch * c->cfg.n_kv_heads;
@@ -302,7 +313,7 @@ kvs_status do_attention(kvs_ctx* c, int layer, const void* q, float* out, int ba
     const bool use_mma = choose_plan(c, batch * c->cfg.n_kv_heads, c->slot_len[slot], &plan);
     const AttentionScratch scratch = {reinterpret_cast<float*>(c->ws + c->off_part_o),
                                       reinterpret_cast<float*>(c->ws + c->off_part_ml),
-                                      reinterpret_cast<int*>(c->ws + c->off_status), c->opt_pdl != 0};
+                                      reinterpret_cast<int*>(c->ws + c->off_status), take_early_start(c)};
     return run_attention(c, slot, q, out, batch, plan, use_mma, scratch, st);
 }
 
@@ -476,6 +487,7 @@ kvs_status kvs_prefill_attention(kvs_ctx* ctx, int32_t layer, const void* q, flo
     ctx->seq += 1;
     ctx->last_splitk_seq = ctx->seq;
     ctx->stats.prefill_launches += 1;
+    ctx->counter_written = false;   // a plain launch: full dependency on everything before it
     ctx->stats.kv_bytes_read += 0;  // prefill is compute-bound; its K/V reads are not counted as decode traffic
     return KVS_OK;
 }
@@ -520,6 +532,7 @@ kvs_status kvs_evict(kvs_ctx* ctx, int32_t layer, const int32_t* keep, const int
     ctx->app_seq_latest[slot] = ctx->seq;
     ctx->app_start_latest[slot] = 0;
     ctx->stats.evict_launches += 1;
+    ctx->counter_written = false;   // a plain launch: full dependency on everything before it
     return KVS_OK;
 }
 
@@ -551,6 +564,7 @@ kvs_status kvs_layer_distances(kvs_ctx* ctx, int32_t batch, float* dist, void* s
     ctx->seq += 2;
     ctx->last_splitk_seq = ctx->seq;     // plain launches: everything before them has finished when they run
     ctx->stats.search_launches += 2;
+    ctx->counter_written = false;   // a plain launch: full dependency on everything before it
     return KVS_OK;
 }
 
@@ -568,6 +582,7 @@ kvs_status kvs_mean_cosine(kvs_ctx* ctx, const void* a, const void* b, int32_t n
     ctx->seq += 2;
     ctx->last_splitk_seq = ctx->seq;
     ctx->stats.search_launches += 2;
+    ctx->counter_written = false;   // a plain launch: full dependency on everything before it
     return KVS_OK;
 }
 
@@ -585,6 +600,7 @@ kvs_status kvs_replay_advance(kvs_ctx* ctx, void* stream) {
                                    static_cast<cudaStream_t>(stream)) != cudaSuccess)
         return KVS_ERR_CUDA;
     ctx->seq += 1;
+    ctx->counter_written = true;
     return KVS_OK;
 }
 
@@ -598,6 +614,7 @@ kvs_status kvs_replay_commit(kvs_ctx* ctx, int32_t times_run, void* stream) {
     if (!guard.ok) return KVS_ERR_CUDA;
     if (cudaMemsetAsync(ctx->ws + ctx->off_replay, 0, sizeof(int), static_cast<cudaStream_t>(stream)) != cudaSuccess)
         return KVS_ERR_CUDA;
+    ctx->counter_written = true;
     for (int s = 0; s < ctx->n_slots; ++s) {
         if (ctx->slot_len[s] == 0) continue;
         ctx->slot_len[s] += extra;
@@ -872,6 +889,7 @@ kvs_status kvs_decode_attention_static(kvs_ctx* ctx, int32_t layer, const void* 
     const AttentionScratch scratch = {reinterpret_cast<float*>(base + kStaticStatusBytes),
                                       reinterpret_cast<float*>(base + kStaticStatusBytes + part_o_bytes), status_word,
                                       false};
+    c->counter_written = false;
     return run_attention(c, slot, q, out, batch, plan, use_mma, scratch, st);
 }
 

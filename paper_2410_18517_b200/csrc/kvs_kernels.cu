@@ -262,8 +262,9 @@ __global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G, GEOM>::MI
     using S = ScalarShape<T, D, G, GEOM>;
     ScalarKernelArgs a = a_in;
     if (a.n_extra != nullptr) {
-        // A replayed launch: the lengths recorded with it have grown on the device since.
-        pdl_wait();
+        // A replayed launch: the lengths recorded with it have grown on the device since.  The
+        // counter is stable here without a wait: the host gives the first launch after every write
+        // of the counter a full dependency, so that write is complete before any reader starts.
         a.n += *a.n_extra;
         a.tpu = (a.n + S::TN - 1) / S::TN;
         a.T = (long long)a.units * a.tpu;
@@ -604,7 +605,6 @@ cudaError_t launch_decode_scalar(const DecodeArgs& a, const DecodePlan& plan, cu
     ka.unit_len = a.unit_len;
     ka.n_extra = a.n_extra;
     ka.units = a.units;
-    if (a.n_extra) ka.safe_rows = 0;   // the tile line is only known after the wait
     const bool pdl = a.programmatic;
     if (a.dtype == 0) {
         if (a.D == 128) return launch_scalar_groups<__nv_bfloat16, 128>(a.G, plan.geom, ka, plan.NC, pdl, stream);

@@ -117,8 +117,9 @@ __global__ void __launch_bounds__(kMmaThreads, KVS_MMA_BLOCKS_PER_SM)
     using S = MmaShape<D>;
     MmaKernelArgs a = a_in;
     if (a.n_extra != nullptr) {
-        // A replayed launch: the lengths recorded with it have grown on the device since.
-        pdl_wait();
+        // A replayed launch: the lengths recorded with it have grown on the device since.  The
+        // counter is stable here without a wait: the host gives the first launch after every write
+        // of the counter a full dependency, so that write is complete before any reader starts.
         a.n += *a.n_extra;
         a.tpu = (a.n + S::TN - 1) / S::TN;
         a.T = (long long)a.units * a.tpu;
@@ -446,7 +447,6 @@ cudaError_t launch_decode_mma(const DecodeArgs& a, const DecodePlan& plan, const
     ka.G = a.G;
     ka.n_extra = a.n_extra;
     ka.units = a.units;
-    if (a.n_extra) ka.safe_rows = 0;   // the tile line is only known after the wait
     if (a.G < 1 || a.G > 8) return cudaErrorInvalidValue;
     if (a.D == 128) return launch_one<128>(tm, ka, plan.NC, a.programmatic, stream);
     if (a.D == 64) return launch_one<64>(tm, ka, plan.NC, a.programmatic, stream);

@@ -49,13 +49,14 @@ def time_point(w: si.Workload, steps: int, device=0) -> dict:
     ins = [si.step_qkv(w, 0, l, device=dev) for l in range(w.L)]
     outs = [torch.empty(w.B, w.Hq, w.D, dtype=torch.float32, device=dev) for _ in range(w.L)]
 
-    def one_step():
+    def one_step(replay=False):
         for l in range(w.L):
             q, kk, vv = ins[l]
             if sm[l] == l:
                 cache.append(l, kk, vv)
             cache.decode_attention(l, q, outs[l])
-        cache.replay_advance()           # recorded only while capturing
+        if replay:
+            cache.replay_advance()       # recorded only while capturing
 
     def timed(fn, n):
         torch.cuda.synchronize(dev)
@@ -81,11 +82,11 @@ def time_point(w: si.Workload, steps: int, device=0) -> dict:
     side = torch.cuda.Stream(device=dev)
     side.wait_stream(torch.cuda.current_stream(dev))
     with torch.cuda.stream(side):
-        one_step()
+        one_step(True)
         graph = torch.cuda.CUDAGraph()
         b0 = cache.stats()["kv_bytes_read"]
         with torch.cuda.graph(graph, stream=side):
-            one_step()
+            one_step(True)
         read_graph = cache.stats()["kv_bytes_read"] - b0
     torch.cuda.current_stream(dev).wait_stream(side)
     graph.replay()
