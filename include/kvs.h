@@ -92,9 +92,11 @@ typedef enum {
                                that nothing in flight writes; they wait for the previous kernel
                                before reading q, newly appended rows, or writing anything.
                                0: plain stream-ordered launches.  Results are identical.      */
-    KVS_OPT_REPLAY = 3      /* 1: launches also read a device-side growth counter, so that a
+    KVS_OPT_REPLAY = 3,     /* 1: launches also read a device-side growth counter, so that a
                                recorded decode step can be replayed as a CUDA graph (see
                                kvs_replay_advance).  0 (default): lengths come from the host only. */
+    KVS_OPT_HOST_CHUNKS = 4 /* kvs_step_host: number of pieces (1..8, default 4) the layers are cut
+                               into for overlapping the host copies with the kernels.            */
 } kvs_option;
 
 /* ---- life cycle ------------------------------------------------------------ */

@@ -30,6 +30,7 @@ KVS_OPT_MAX_CTAS = 0
 KVS_OPT_KERNEL = 1
 KVS_OPT_EARLY_START = 2
 KVS_OPT_REPLAY = 3
+KVS_OPT_HOST_CHUNKS = 4
 
 # every symbol include/kvs.h declares
 EXPORTS = (

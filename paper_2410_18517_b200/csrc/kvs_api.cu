@@ -68,6 +68,7 @@ struct kvs_ctx {
     int opt_max_ctas = 0;
     int opt_kernel = 0;
     int opt_pdl = 1;
+    int opt_host_chunks = 4;
     int opt_replay = 0;   // launches carry the device-side growth counter (for CUDA-graph replay)
     // The split-K kernels read the growth counter before their wait.  That is safe because the
     // first launch after anything wrote the counter never starts early (full dependency): it and
@@ -662,13 +663,22 @@ kvs_status kvs_step_host(kvs_ctx* ctx, const void* q_host, const void* k_host, c
     }
     cudaStream_t cs = ctx->copy_stream, os = ctx->out_stream;
     const int L = f.n_layers;
-    const int chunks = L < kvs_ctx::kChunks ? L : kvs_ctx::kChunks;
+    const int chunks = L < ctx->opt_host_chunks ? L : ctx->opt_host_chunks;
     // the copy streams start after whatever the caller already queued on `st`
     if (cudaEventRecord(ctx->ev_start, st) != cudaSuccess || cudaStreamWaitEvent(cs, ctx->ev_start, 0) != cudaSuccess ||
         cudaStreamWaitEvent(os, ctx->ev_start, 0) != cudaSuccess)
         return KVS_ERR_CUDA;
+    // Chunk c covers layers [edge(c), edge(c+1)).  With three or more chunks the first and the last are
+    // a single layer, so that the input copy nothing can hide and the output copy nothing can hide
+    // are as small as they can be; the layers between are cut evenly.
+    auto edge = [&](int c) -> int {
+        if (chunks < 3 || L < chunks + 2) return (int)((long long)c * L / chunks);
+        if (c == 0) return 0;
+        if (c == chunks) return L;
+        return 1 + (int)((long long)(c - 1) * (L - 2) / (chunks - 2));
+    };
     auto copy_in = [&](int c) -> bool {
-        const int l0 = (int)((long long)c * L / chunks), l1 = (int)((long long)(c + 1) * L / chunks);
+        const int l0 = edge(c), l1 = edge(c + 1);
         if (cudaMemcpyAsync(dq + q_layer * l0, (const char*)q_host + q_layer * l0, q_layer * (l1 - l0),
                             cudaMemcpyHostToDevice, cs) != cudaSuccess)
             return false;
@@ -689,7 +699,7 @@ kvs_status kvs_step_host(kvs_ctx* ctx, const void* q_host, const void* k_host, c
     };
     if (!copy_in(0)) return KVS_ERR_CUDA;
     for (int c = 0; c < chunks; ++c) {
-        const int l0 = (int)((long long)c * L / chunks), l1 = (int)((long long)(c + 1) * L / chunks);
+        const int l0 = edge(c), l1 = edge(c + 1);
         if (c + 1 < chunks && !copy_in(c + 1)) return KVS_ERR_CUDA;
         if (cudaStreamWaitEvent(st, ctx->ev_in[c], 0) != cudaSuccess) return KVS_ERR_CUDA;
         for (int l = l0; l < l1; ++l) {
@@ -779,6 +789,10 @@ kvs_status kvs_set_option(kvs_ctx* ctx, int32_t option, int32_t value) {
         case KVS_OPT_REPLAY:
             if (value != 0 && value != 1) return KVS_ERR_INVALID_ARG;
             ctx->opt_replay = value;
+            return KVS_OK;
+        case KVS_OPT_HOST_CHUNKS:
+            if (value < 1 || value > kvs_ctx::kChunks) return KVS_ERR_INVALID_ARG;
+            ctx->opt_host_chunks = value;
             return KVS_OK;
         case KVS_OPT_KERNEL:
             if (value < 0 || value > 2) return KVS_ERR_INVALID_ARG;

@@ -157,6 +157,10 @@ def test_options_and_null_arguments():
         kb.kvs_set_option(c, kb.KVS_OPT_MAX_CTAS, 100000)
     with pytest.raises(kb.KvsError):
         kb.kvs_set_option(c, 99, 0)
+    kb.kvs_set_option(c, kb.KVS_OPT_HOST_CHUNKS, 3)
+    for bad in (0, 9):
+        with pytest.raises(kb.KvsError):
+            kb.kvs_set_option(c, kb.KVS_OPT_HOST_CHUNKS, bad)
     with pytest.raises(kb.KvsError):
         kb.kvs_slot_of_layer(c, 4)
     lib = kb.load()

@@ -261,10 +261,19 @@ def test_repeat_runs_are_bit_identical():
         assert torch.equal(a, cache.decode_attention(0, q))
 
 
-def test_step_host_equals_per_layer_calls():
+@pytest.mark.parametrize("layers,chunks", [(4, None), (4, 1), (11, 1), (11, 2), (11, 3), (11, 4), (11, 8)])
+def test_step_host_equals_per_layer_calls(layers, chunks):
     w = si.WORKLOADS["tiny"]
+    if layers != w.L:
+        w = w.scaled(L=layers, fixed_map=None, n_shared=3, map_seed=5)
+    sm = w.share_map()
+    n_own = int((sm == np.arange(w.L)).sum())
     a, b = make_cache(w, 4), make_cache(w, 4)
+    if chunks is not None:
+        a.set_option(kb.KVS_OPT_HOST_CHUNKS, chunks)
     for l in range(w.L):
+        if sm[l] != l:
+            continue
         k, v = si.context_kv(w, l)
         a.append(l, k.cuda(), v.cuda())
         b.append(l, k.cuda(), v.cuda())
@@ -274,9 +283,10 @@ def test_step_host_equals_per_layer_calls():
         oh = torch.empty(w.L, w.B, w.Hq, w.D, dtype=torch.float32).pin_memory()
         h2d, d2h = a.step_host(qh, kh, vh, oh)
         assert d2h == oh.numel() * 4
-        assert h2d == qh.numel() * 4 + 2 * 3 * kh[0].numel() * 4      # K/V of the 3 own-cache layers only
+        assert h2d == qh.numel() * 4 + 2 * n_own * kh[0].numel() * 4      # K/V of the own-cache layers only
         for l in range(w.L):
-            b.append(l, ks[l].cuda(), vs[l].cuda())
+            if sm[l] == l:
+                b.append(l, ks[l].cuda(), vs[l].cuda())
             assert torch.equal(b.decode_attention(l, qs[l].cuda()).cpu(), oh[l])
     torch.cuda.synchronize()
     assert torch.equal(a.pool, b.pool)
