@@ -2,16 +2,21 @@
 //
 // n_q queries per head (the newest n_q positions of the slot the layer reads, causal mask)
 // against the slot's K/V rows: a dense contraction, so it runs on tcgen05.mma with the
-// accumulators in tensor memory.  One thread block = 128 queries of one (sequence, q-head):
-//   warp 4 (one lane)  TMA producer: Q tile once, then K and V tiles of 128 keys
-//   warp 5 (one lane)  MMA issuer:   S = Q K^T  (128x128x128, bf16 -> fp32 in TMEM)
+// accumulators in tensor memory.  One thread block = 128 queries of one (sequence, q-head),
+// walking over the keys in tiles of 64:
+//   warp 8 (one lane)  TMA producer: Q tile once, then K and V tiles, two stages each
+//   warp 9 (one lane)  MMA issuer:   S = Q K^T  (128x64x128, bf16 -> fp32 in TMEM), into one
+//                                    of two score buffers, so that S of tile j+1 is computed
+//                                    while the softmax of tile j runs;
 //                                    O += P V with P = P_hi + P_lo (two bf16 terms, read from TMEM)
-//   warps 0..3         softmax: thread r owns query row r = TMEM lane r; reads S with
-//                      tcgen05.ld, writes P_hi / P_lo over S with tcgen05.st, and rescales the
-//                      output row in TMEM only when the running maximum grows by more than 2^8
-// Two blocks share an SM (96 KiB of shared memory and 256 TMEM columns each), so one block's
-// softmax overlaps the other's tensor-core work.  K/V/Q tiles land in the 128-byte-swizzled
-// layout the MMA shared-memory descriptors expect (K and Q K-major, V MN-major).
+//   warps 0..7         softmax: two threads per query row (= TMEM lane), warp w and warp w+4,
+//                      32 keys of the tile each.  A thread reads its scores with tcgen05.ld,
+//                      the two exchange their maxima through shared memory, then each writes
+//                      its part of P_hi / P_lo over S with tcgen05.st; the output row in TMEM is
+//                      rescaled only when the running maximum grows by more than 2^8
+// Two blocks share an SM (99 KiB of shared memory and 256 TMEM columns each), so four key
+// tiles are in flight per SM.  K/V/Q tiles land in the 128-byte-swizzled layout the MMA
+// shared-memory descriptors expect (K and Q K-major, V MN-major).
 // bf16 storage, head size 128.
 #include <cuda.h>
 
@@ -24,12 +29,15 @@ namespace kvs {
 
 namespace {
 
-constexpr int kPfThreads = 192;
-constexpr int kPfTile = 128;                 // queries per block and keys per tile
-constexpr int kPfHalfBytes = kPfTile * 128;  // 128 rows x 64 bf16: one swizzled column block
-constexpr int kPfMatBytes = 2 * kPfHalfBytes;  // a 128 x 128 bf16 operand
-constexpr int kPfSmemBytes = 1024 + 3 * kPfMatBytes /*Q, K, V*/ + 256;
-constexpr uint32_t kTmemCols = 256;          // S: columns [0,128), O tile: [128,256)
+constexpr int kPfSoftmaxWarps = 8;
+constexpr int kPfThreads = (kPfSoftmaxWarps + 2) * 32;
+constexpr int kPfTile = 128;                 // queries per block
+constexpr int kPfKeys = 64;                  // keys per tile
+constexpr int kPfQBytes = kPfTile * 256;     // 128 x 128 bf16: two swizzled blocks of 64 columns
+constexpr int kPfKvBytes = kPfKeys * 256;    // 64 x 128 bf16: two swizzled blocks of 64 columns
+constexpr int kPfSmemBytes = 1024 + kPfQBytes + 4 * kPfKvBytes /*K, V: two stages each*/ + 256 +
+                             6 * kPfTile * 4 /*row maxima, row sums*/;
+constexpr uint32_t kTmemCols = 256;          // two score buffers: columns [0,64), [64,128); O tile: [128,256)
 
 __device__ __forceinline__ void tma_load_2d_pf(void* dst, const CUtensorMap* tmap, int x, int y, uint64_t* bar) {
     asm volatile(
@@ -61,9 +69,9 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr, uint32_t lbo
 }
 
 // Instruction descriptor for kind::f16: fp32 accumulate, bf16 A and B, A K-major,
-// B K-major (b_mn = 0) or MN-major (b_mn = 1), M = 128, N = 128.
-__device__ __forceinline__ uint32_t instr_desc_bf16(int b_mn) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)b_mn << 16) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+// B K-major (b_mn = 0) or MN-major (b_mn = 1), M = 128, N = n.
+__device__ __forceinline__ uint32_t instr_desc_bf16(int b_mn, uint32_t n) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)b_mn << 16) | ((n >> 3) << 17) | ((128u >> 4) << 24);
 }
 
 __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc,
@@ -117,26 +125,27 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
     for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
 
-// 32 fp32 columns of this thread's TMEM lane, written back.
-__device__ __forceinline__ void tmem_st32(uint32_t taddr, const float (&v)[32]) {
+// Multiply 8 fp32 columns of this thread's TMEM lane by alpha in place.
+__device__ __forceinline__ void tmem_scale8(uint32_t taddr, float alpha) {
+    uint32_t r[8];
     asm volatile(
-        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
-        "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,"
-        "%31,%32};" ::"r"(taddr),
-        "f"(v[0]), "f"(v[1]), "f"(v[2]), "f"(v[3]), "f"(v[4]), "f"(v[5]), "f"(v[6]), "f"(v[7]), "f"(v[8]), "f"(v[9]),
-        "f"(v[10]), "f"(v[11]), "f"(v[12]), "f"(v[13]), "f"(v[14]), "f"(v[15]), "f"(v[16]), "f"(v[17]), "f"(v[18]),
-        "f"(v[19]), "f"(v[20]), "f"(v[21]), "f"(v[22]), "f"(v[23]), "f"(v[24]), "f"(v[25]), "f"(v[26]), "f"(v[27]),
-        "f"(v[28]), "f"(v[29]), "f"(v[30]), "f"(v[31])
+        "tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];\n\t"
+        "tcgen05.wait::ld.sync.aligned;"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+        : "r"(taddr)
         : "memory");
+#pragma unroll
+    for (int i = 0; i < 8; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * alpha);
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"r"(taddr), "r"(r[0]),
+                 "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
+                 : "memory");
 }
 
-// 16 packed 32-bit columns (32 bf16 values) of this thread's TMEM lane.
-__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&v)[16]) {
-    asm volatile(
-        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};" ::"r"(taddr),
-        "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]), "r"(v[8]), "r"(v[9]),
-        "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15])
-        : "memory");
+// 8 packed 32-bit columns (16 bf16 values) of this thread's TMEM lane.
+__device__ __forceinline__ void tmem_st8(uint32_t taddr, const uint32_t (&v)[8]) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"r"(taddr), "r"(v[0]),
+                 "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7])
+                 : "memory");
 }
 
 __device__ __forceinline__ uint32_t pack2_bf16(float lo, float hi) {
@@ -155,8 +164,6 @@ struct PrefillArgs {
     float scale_log2;
 };
 
-// One softmax pass over a 32-column chunk of S: p = 2^(x*scale - m_ref) (0 where masked),
-// split into bf16 hi and lo words (2 keys per word).  Returns the chunk's sum of p.
 // max(a, b, c) in one instruction
 __device__ __forceinline__ float fmax3(float a, float b, float c) {
     float d;
@@ -164,18 +171,18 @@ __device__ __forceinline__ float fmax3(float a, float b, float c) {
     return d;
 }
 
-// One softmax pass over a 32-column chunk of S: p = 2^(x*scale - m_ref) (0 where masked),
-// split into bf16 hi and lo words (2 keys per word).  Returns the chunk's sum of p.  The scale,
-// the sum and the hi/lo split use the packed two-float instructions.
-template <bool MASK>
+// One softmax pass over 16 scores x[OFF .. OFF+15]: p = 2^(x*scale - m_ref) (0 where masked),
+// split into bf16 hi and lo words (2 keys per word).  Returns the sum of p.  The scale, the
+// sum and the hi/lo split use the packed two-float instructions.
+template <bool MASK, int OFF>
 __device__ __forceinline__ float softmax_chunk(const float (&x)[32], float scale_log2, float m_ref, int key_first,
-                                               int limit, uint32_t (&hi)[16], uint32_t (&lo)[16]) {
+                                               int limit, uint32_t (&hi)[8], uint32_t (&lo)[8]) {
     const float2 sc = make_float2(scale_log2, scale_log2), nm = make_float2(-m_ref, -m_ref);
     const float2 minus1 = make_float2(-1.f, -1.f);
     float2 sum = make_float2(0.f, 0.f);
 #pragma unroll
-    for (int i = 0; i < 32; i += 2) {
-        const float2 t = __ffma2_rn(make_float2(x[i], x[i + 1]), sc, nm);
+    for (int i = 0; i < 16; i += 2) {
+        const float2 t = __ffma2_rn(make_float2(x[OFF + i], x[OFF + i + 1]), sc, nm);
         float2 p = make_float2(fast_exp2(t.x), fast_exp2(t.y));
         if (MASK) {
             p.x = (key_first + i <= limit) ? p.x : 0.f;
@@ -196,19 +203,22 @@ __global__ void __launch_bounds__(kPfThreads, 2)
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     unsigned char* sQ = smem;
-    unsigned char* sK = sQ + kPfMatBytes;
-    unsigned char* sV = sK + kPfMatBytes;
-    uint64_t* bars = reinterpret_cast<uint64_t*>(sV + kPfMatBytes);
+    unsigned char* sK = sQ + kPfQBytes;             // two stages
+    unsigned char* sV = sK + 2 * kPfKvBytes;        // two stages
+    uint64_t* bars = reinterpret_cast<uint64_t*>(sV + 2 * kPfKvBytes);
     uint64_t* q_full = bars;
-    uint64_t* k_full = bars + 1;
-    uint64_t* k_empty = bars + 2;
-    uint64_t* v_full = bars + 3;
-    uint64_t* v_empty = bars + 4;
-    uint64_t* s_full = bars + 5;
-    uint64_t* p_full = bars + 6;        // 128 arrivals
-    uint64_t* o_full = bars + 7;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 8);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 9);
+    uint64_t* o_full = bars + 1;        // one phase per PV group: tile j's output contribution is in O
+    uint64_t* k_full = bars + 2;        // [2] per K stage
+    uint64_t* k_empty = bars + 4;
+    uint64_t* v_full = bars + 6;        // [2] per V stage
+    uint64_t* v_empty = bars + 8;
+    uint64_t* s_full = bars + 10;       // [2] per score buffer
+    uint64_t* p_full = bars + 12;       // [2] per score buffer, one arrival per softmax thread
+    uint64_t* pair_bar = bars + 14;     // [4]: the two warps that share 32 query rows, 64 arrivals
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 18);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 19);
+    float* exch_m = reinterpret_cast<float*>(bars + 32);   // [2 tile parities][2 key halves][128] row maxima
+    float* exch_l = exch_m + 4 * kPfTile;                  // [2 key halves][128] row sums
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int qb = gridDim.x - 1 - blockIdx.x;       // blocks with the most keys first
@@ -216,12 +226,15 @@ __global__ void __launch_bounds__(kPfThreads, 2)
     const int hk = hq / a.G;
     const int Hkv = a.Hq / a.G;
     const int q0 = qb * kPfTile;
-    // last key any query of this block may see, and the tiles that cover keys 0..that
+    // last key any query of this block may see, and the key tiles that cover keys 0..that
     const int last_key = min(a.n - a.T + q0 + kPfTile - 1, a.n - 1);
-    const int nt = last_key / kPfTile + 1;
+    const int nt = last_key / kPfKeys + 1;
 
     if (tid == 0) {
-        for (int i = 0; i < 8; ++i) mbar_init(&bars[i], i == 6 ? 128 : 1);
+        for (int i = 0; i < 12; ++i) mbar_init(&bars[i], 1);
+        mbar_init(&p_full[0], kPfSoftmaxWarps * 32);
+        mbar_init(&p_full[1], kPfSoftmaxWarps * 32);
+        for (int i = 0; i < 4; ++i) mbar_init(&pair_bar[i], 64);
         abort_flag[0] = 0;
         fence_mbar_init();
     }
@@ -235,172 +248,183 @@ __global__ void __launch_bounds__(kPfThreads, 2)
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
-    const uint32_t tmem_s = tmem_base;         // S (fp32, 128 columns); P_hi / P_lo (bf16 pairs) overwrite it
+    const uint32_t tmem_s = tmem_base;         // two score buffers of 64 fp32 columns; P_hi / P_lo overwrite them
     const uint32_t tmem_o = tmem_base + 128;   // running output rows
 
-    if (warp == 4) {
+    if (warp == kPfSoftmaxWarps) {
         // ------------------------------ TMA producer ------------------------------
         if (lane == 0) {
-            mbar_arrive_expect_tx(q_full, kPfMatBytes);
+            mbar_arrive_expect_tx(q_full, kPfQBytes);
             tma_load_4d(sQ, &tmap_q, 0, hq, q0, b, q_full);
-            tma_load_4d(sQ + kPfHalfBytes, &tmap_q, 64, hq, q0, b, q_full);
+            tma_load_4d(sQ + kPfQBytes / 2, &tmap_q, 64, hq, q0, b, q_full);
             const long long unit_row = ((long long)b * Hkv + hk) * a.row_stride;
             for (int j = 0; j < nt; ++j) {
-                const long long row = unit_row + (long long)j * kPfTile;
-                if (j >= 1 && !mbar_wait_bounded(k_empty, (j - 1) & 1, abort_flag, a.status)) break;
-                mbar_arrive_expect_tx(k_full, kPfMatBytes);
+                const int st = j & 1;
+                const uint32_t prev = (uint32_t)((j >> 1) - 1) & 1u;   // phase in which tile j-2 released the stage
+                const long long row = unit_row + (long long)j * kPfKeys;
+                if (j >= 2 && !mbar_wait_bounded(&k_empty[st], prev, abort_flag, a.status)) break;
+                mbar_arrive_expect_tx(&k_full[st], kPfKvBytes);
 #pragma unroll
                 for (int h = 0; h < 2; ++h)
-#pragma unroll
-                    for (int rb = 0; rb < 2; ++rb)
-                        tma_load_2d_pf(sK + h * kPfHalfBytes + rb * 8192, &tmap_kv, h * 64, (int)(a.krow0 + row + rb * 64),
-                                       k_full);
-                if (j >= 1 && !mbar_wait_bounded(v_empty, (j - 1) & 1, abort_flag, a.status)) break;
-                mbar_arrive_expect_tx(v_full, kPfMatBytes);
+                    tma_load_2d_pf(sK + st * kPfKvBytes + h * (kPfKvBytes / 2), &tmap_kv, h * 64, (int)(a.krow0 + row),
+                                   &k_full[st]);
+                if (j >= 2 && !mbar_wait_bounded(&v_empty[st], prev, abort_flag, a.status)) break;
+                mbar_arrive_expect_tx(&v_full[st], kPfKvBytes);
 #pragma unroll
                 for (int h = 0; h < 2; ++h)
-#pragma unroll
-                    for (int rb = 0; rb < 2; ++rb)
-                        tma_load_2d_pf(sV + h * kPfHalfBytes + rb * 8192, &tmap_kv, h * 64, (int)(a.vrow0 + row + rb * 64),
-                                       v_full);
+                    tma_load_2d_pf(sV + st * kPfKvBytes + h * (kPfKvBytes / 2), &tmap_kv, h * 64, (int)(a.vrow0 + row),
+                                   &v_full[st]);
             }
         }
-    } else if (warp == 5) {
+    } else if (warp == kPfSoftmaxWarps + 1) {
         // ------------------------------ MMA issuer ------------------------------
+        // Order on the tensor pipe: S_0, then per tile j: S_{j+1} (into the other score buffer, so
+        // that the softmax of tile j+1 can start the moment the one of tile j ends), PV_j.  The
+        // pipe runs one thread's MMAs in issue order, so S_{j+1} overwrites its buffer only after
+        // PV_{j-1} has read P_{j-1} from it.
         if (lane == 0) {
-            const uint32_t idesc_s = instr_desc_bf16(0);
-            const uint32_t idesc_o = instr_desc_bf16(1);
+            const uint32_t idesc_s = instr_desc_bf16(0, kPfKeys);
+            const uint32_t idesc_o = instr_desc_bf16(1, 128);
             const uint32_t q_addr = smem_u32(sQ), k_addr = smem_u32(sK), v_addr = smem_u32(sV);
-            auto issue_s = [&]() {
+            auto issue_s = [&](int j) {
+                const int st = j & 1;
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {   // 16 head-dim columns per step; 4 steps per 64-column block
-                    const uint32_t off = (ks >> 2) * kPfHalfBytes + (ks & 3) * 32;
-                    umma_bf16(tmem_s, smem_desc_sw128(q_addr + off, 16, 1024), smem_desc_sw128(k_addr + off, 16, 1024),
-                              idesc_s, ks > 0);
+                    const uint32_t qoff = (ks >> 2) * (kPfQBytes / 2) + (ks & 3) * 32;
+                    const uint32_t koff = st * kPfKvBytes + (ks >> 2) * (kPfKvBytes / 2) + (ks & 3) * 32;
+                    umma_bf16(tmem_s + st * kPfKeys, smem_desc_sw128(q_addr + qoff, 16, 1024),
+                              smem_desc_sw128(k_addr + koff, 16, 1024), idesc_s, ks > 0);
                 }
-                umma_commit(s_full);
-                umma_commit(k_empty);     // the K tile may be overwritten once S is done
+                umma_commit(&s_full[st]);
+                umma_commit(&k_empty[st]);     // the K stage may be overwritten once S is done
             };
             bool ok = mbar_wait_bounded(q_full, 0, abort_flag, a.status) &&
-                      mbar_wait_bounded(k_full, 0, abort_flag, a.status);
+                      mbar_wait_bounded(&k_full[0], 0, abort_flag, a.status);
             if (ok) {
                 tc_fence_after();
-                issue_s();
+                issue_s(0);
             }
             for (int j = 0; j < nt && ok; ++j) {
-                ok = mbar_wait_bounded(p_full, j & 1, abort_flag, a.status) &&
-                     mbar_wait_bounded(v_full, j & 1, abort_flag, a.status);
+                const int st = j & 1;
+                const uint32_t ph = (uint32_t)(j >> 1) & 1u;
+                if (j + 1 < nt) {
+                    ok = mbar_wait_bounded(&k_full[st ^ 1], (uint32_t)((j + 1) >> 1) & 1u, abort_flag, a.status);
+                    if (!ok) break;
+                    tc_fence_after();
+                    issue_s(j + 1);
+                }
+                ok = mbar_wait_bounded(&p_full[st], ph, abort_flag, a.status) &&
+                     mbar_wait_bounded(&v_full[st], ph, abort_flag, a.status);
                 if (!ok) break;
                 tc_fence_after();
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {   // 16 keys per step: 8 TMEM columns of bf16 pairs
+                for (int ks = 0; ks < kPfKeys / 16; ++ks) {   // 16 keys per step: 8 TMEM columns of bf16 pairs
                     // V is MN-major: 64 head-dim columns contiguous per key row, the other 64 one
                     // column block (LBO) away; 8-key groups 1024 bytes (SBO) apart
-                    const uint64_t vdesc = smem_desc_sw128(v_addr + ks * 16 * 128, kPfHalfBytes, 1024);
-                    umma_bf16_ts(tmem_o, tmem_s + ks * 8, vdesc, idesc_o, (j > 0) || (ks > 0));        // P_hi
-                    umma_bf16_ts(tmem_o, tmem_s + 64 + ks * 8, vdesc, idesc_o, 1);                   // P_lo
+                    const uint64_t vdesc =
+                        smem_desc_sw128(v_addr + st * kPfKvBytes + ks * 16 * 128, kPfKvBytes / 2, 1024);
+                    umma_bf16_ts(tmem_o, tmem_s + st * kPfKeys + ks * 8, vdesc, idesc_o, (j > 0) || (ks > 0));     // P_hi
+                    umma_bf16_ts(tmem_o, tmem_s + st * kPfKeys + kPfKeys / 2 + ks * 8, vdesc, idesc_o, 1);       // P_lo
                 }
                 umma_commit(o_full);
-                umma_commit(v_empty);
-                if (j + 1 < nt) {
-                    ok = mbar_wait_bounded(k_full, (j + 1) & 1, abort_flag, a.status);
-                    if (!ok) break;
-                    tc_fence_after();
-                    issue_s();
-                }
+                umma_commit(&v_empty[st]);
             }
         }
     } else {
         // ------------------------------ softmax / output rows ------------------------------
-        const int r = tid;                                   // query row in the block = TMEM lane
+        const int w4 = warp & 3, hf = warp >> 2;             // TMEM lane quarter, key half of a tile
+        const int r = w4 * 32 + lane;                        // query row in the block = TMEM lane
         const int qpos = min(q0 + r, a.T - 1);               // padding rows repeat the last query
         const int limit = a.n - a.T + qpos;                  // last key this query may see
         const int block_min_limit = a.n - a.T + q0;          // smallest limit of any row of the block
-        const uint32_t lane_addr = (uint32_t)(warp * 32) << 16;
-        const uint32_t ts = tmem_s + lane_addr, to = tmem_o + lane_addr;
+        const uint32_t lane_addr = (uint32_t)(w4 * 32) << 16;
+        const uint32_t to = tmem_o + lane_addr + hf * 64;        // this thread's 64 columns of the output row
         float m_ref = -1.0e30f, l = 0.f;                     // p is taken relative to m_ref (log2 domain)
         bool ok = true;
         for (int j = 0; j < nt; ++j) {
-            ok = mbar_wait_bounded(s_full, j & 1, abort_flag, a.status);
+            const int st = j & 1;
+            ok = mbar_wait_bounded(&s_full[st], (uint32_t)(j >> 1) & 1u, abort_flag, a.status);
             if (!ok) break;
             tc_fence_after();
-            const int key0 = j * kPfTile;
-            const bool mask = key0 + kPfTile - 1 > block_min_limit;   // block-uniform
-            // pass 1: row maximum of the (masked) scores
+            const uint32_t sb = tmem_s + lane_addr + st * kPfKeys;
+            const uint32_t ts = sb + hf * 32;                     // this thread's 32 scores
+            const uint32_t tph = sb + hf * 16;                    // P_hi words of its keys (key k -> column k/2)
+            const uint32_t tpl = sb + kPfKeys / 2 + hf * 16;      // P_lo words (column 32 + k/2)
+            const int key0 = j * kPfKeys + hf * 32;
+            const bool mask = j * kPfKeys + kPfKeys - 1 > block_min_limit;   // block-uniform
+            float x[32];
+            tmem_ld32(ts, x);
+            // row maximum of the (masked) scores: own half, then the partner warp's through shared
+            // memory.  After the pair barrier both halves of S have been read, so P may overwrite it.
             float mx = -INFINITY;
-#pragma unroll 1
-            for (int c = 0; c < 4; ++c) {
-                float x[32];
-                tmem_ld32(ts + c * 32, x);
-                if (mask) {
+            if (mask) {
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) mx = fmaxf(mx, (key0 + c * 32 + i <= limit) ? x[i] : -INFINITY);
-                } else {
+                for (int i = 0; i < 32; ++i) mx = fmaxf(mx, (key0 + i <= limit) ? x[i] : -INFINITY);
+            } else {
 #pragma unroll
-                    for (int i = 0; i < 32; i += 2) mx = fmax3(mx, x[i], x[i + 1]);
-                }
+                for (int i = 0; i < 32; i += 2) mx = fmax3(mx, x[i], x[i + 1]);
             }
-            mx *= a.scale_log2;
+            float* em = exch_m + st * 2 * kPfTile;
+            em[hf * kPfTile + r] = mx;
+            tc_fence_before();
+            mbar_arrive(&pair_bar[w4]);
+            ok = mbar_wait_bounded(&pair_bar[w4], (uint32_t)j & 1u, abort_flag, a.status);
+            if (!ok) break;
+            tc_fence_after();
+            mx = fmaxf(mx, em[(hf ^ 1) * kPfTile + r]) * a.scale_log2;
             // The reference maximum only moves when the new one is more than 8 (a factor 256) above
-            // it; then the output row and the sum accumulated so far are rescaled.  PV of the
-            // previous tile has finished (S of this tile was issued after it), so O is quiet.
+            // it; then the output row and the sum accumulated so far are rescaled, once every PV
+            // issued so far has landed in O (PV of this tile cannot start before this thread's
+            // arrival below).  Both threads of a row take the same decision from the same numbers.
             const bool grow = mx > m_ref + 8.0f;
             if (__any_sync(0xffffffffu, grow)) {
                 const float m_new = grow ? mx : m_ref;
                 const float alpha = fast_exp2(m_ref - m_new);
                 if (j > 0) {
+                    ok = mbar_wait_bounded(o_full, (uint32_t)(j - 1) & 1u, abort_flag, a.status);
+                    if (!ok) break;
+                    tc_fence_after();
 #pragma unroll 1
-                    for (int c = 0; c < 4; ++c) {
-                        float o[32];
-                        tmem_ld32(to + c * 32, o);
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) o[i] *= alpha;
-                        tmem_st32(to + c * 32, o);
-                    }
+                    for (int c = 0; c < 8; ++c) tmem_scale8(to + c * 8, alpha);
                 }
                 l *= alpha;
                 m_ref = m_new;
             }
-            // pass 2, upper key half first: P_hi / P_lo overwrite S, so a column may only be written
-            // once the scores in it have been read.  P_hi[keys k] -> columns k/2, P_lo -> 64 + k/2.
-            uint32_t hi3[16], hi2[16], hi1[16], hi0[16], lo[16];
             float lsum = 0.f;
-            {
-                float x[32];
-                tmem_ld32(ts + 96, x);
-                lsum += mask ? softmax_chunk<true>(x, a.scale_log2, m_ref, key0 + 96, limit, hi3, lo)
-                             : softmax_chunk<false>(x, a.scale_log2, m_ref, key0 + 96, limit, hi3, lo);
-                tmem_ld32(ts + 64, x);          // all scores of columns 64..127 are now in registers
-                tmem_st16(ts + 64 + 48, lo);
-                lsum += mask ? softmax_chunk<true>(x, a.scale_log2, m_ref, key0 + 64, limit, hi2, lo)
-                             : softmax_chunk<false>(x, a.scale_log2, m_ref, key0 + 64, limit, hi2, lo);
-                tmem_st16(ts + 64 + 32, lo);
-                tmem_ld32(ts + 32, x);
-                lsum += mask ? softmax_chunk<true>(x, a.scale_log2, m_ref, key0 + 32, limit, hi1, lo)
-                             : softmax_chunk<false>(x, a.scale_log2, m_ref, key0 + 32, limit, hi1, lo);
-                tmem_st16(ts + 64 + 16, lo);
-                tmem_ld32(ts, x);               // columns 0..63 are now in registers too
-                tmem_st16(ts + 32, hi2);
-                tmem_st16(ts + 48, hi3);
-                tmem_st16(ts + 16, hi1);
-                lsum += mask ? softmax_chunk<true>(x, a.scale_log2, m_ref, key0, limit, hi0, lo)
-                             : softmax_chunk<false>(x, a.scale_log2, m_ref, key0, limit, hi0, lo);
-                tmem_st16(ts, hi0);
-                tmem_st16(ts + 64, lo);
-            }
+#define KVS_PF_CHUNK(OFF)                                                                                      \
+    {                                                                                                          \
+        uint32_t hi[8], lo[8];                                                                                 \
+        lsum += mask ? softmax_chunk<true, OFF>(x, a.scale_log2, m_ref, key0 + OFF, limit, hi, lo)             \
+                     : softmax_chunk<false, OFF>(x, a.scale_log2, m_ref, key0 + OFF, limit, hi, lo);           \
+        tmem_st8(tph + OFF / 2, hi);                                                                           \
+        tmem_st8(tpl + OFF / 2, lo);                                                                           \
+    }
+            KVS_PF_CHUNK(0)
+            KVS_PF_CHUNK(16)
+#undef KVS_PF_CHUNK
             l += lsum;
             asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
             tc_fence_before();
-            mbar_arrive(p_full);
+            mbar_arrive(&p_full[st]);
         }
-        if (ok) ok = mbar_wait_bounded(o_full, (nt - 1) & 1, abort_flag, a.status);
+        // the row's sum is the two halves' sums (both relative to the same reference maximum)
+        if (ok) {
+            exch_l[hf * kPfTile + r] = l;
+            mbar_arrive(&pair_bar[w4]);
+            ok = mbar_wait_bounded(&pair_bar[w4], (uint32_t)nt & 1u, abort_flag, a.status);
+        }
+        if (ok) {
+            l += exch_l[(hf ^ 1) * kPfTile + r];
+            ok = mbar_wait_bounded(o_full, (uint32_t)(nt - 1) & 1u, abort_flag, a.status);
+        }
         if (ok) {
             tc_fence_after();
             const float inv = 1.0f / l;
             const bool store = q0 + r < a.T;
-            float4* dst = reinterpret_cast<float4*>(a.out + (((long long)b * a.T + min(q0 + r, a.T - 1)) * a.Hq + hq) * 128);
+            float4* dst = reinterpret_cast<float4*>(a.out + (((long long)b * a.T + min(q0 + r, a.T - 1)) * a.Hq + hq) * 128) +
+                          hf * 16;
 #pragma unroll 1
-            for (int c = 0; c < 4; ++c) {
+            for (int c = 0; c < 2; ++c) {
                 float o[32];
                 tmem_ld32(to + c * 32, o);
                 if (store) {
