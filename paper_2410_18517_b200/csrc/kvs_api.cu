@@ -479,9 +479,11 @@ kvs_status kvs_prefill_attention(kvs_ctx* ctx, int32_t layer, const void* q, flo
     DeviceGuard guard(ctx->cfg.device);
     if (!guard.ok) return KVS_ERR_CUDA;
     const long long plane_rows = (long long)ctx->cfg.max_batch * ctx->cfg.n_kv_heads * ctx->row_stride;
-    if (kvs::launch_prefill(q, out, reinterpret_cast<int*>(ctx->ws + ctx->off_status), ctx->tensor_map, batch, n_q,
+    // the prefill kernel's work counter lives in the status block, 64 bytes after the status word
+    if (kvs::launch_prefill(q, out, reinterpret_cast<int*>(ctx->ws + ctx->off_status),
+                            reinterpret_cast<int*>(ctx->ws + ctx->off_status + 64), ctx->tensor_map, batch, n_q,
                             ctx->cfg.n_q_heads, ctx->G, n, ctx->row_stride, plane_rows * (2 * slot),
-                            plane_rows * (2 * slot + 1), ctx->scale * 1.4426950408889634f,
+                            plane_rows * (2 * slot + 1), ctx->scale * 1.4426950408889634f, ctx->sm_count,
                             static_cast<cudaStream_t>(stream)) != cudaSuccess)
         return KVS_ERR_CUDA;
     // a plain launch: it starts only after everything before it on the stream has finished

@@ -66,9 +66,10 @@ cudaError_t launch_decode_mma(const DecodeArgs& a, const DecodePlan& plan, const
 
 // Tensor-core prefill attention (bf16, head size 128): q [B][T][Hq][128], out fp32 of the same shape.
 cudaError_t init_prefill_kernels();
-cudaError_t launch_prefill(const void* q, float* out, int* status, const void* pool_tensor_map, int B, int T, int Hq,
-                           int G, int n, int row_stride, long long krow0, long long vrow0, float scale_log2,
-                           cudaStream_t stream);
+// `sched`: a device int for the kernel's work counter (zeroed on `stream` by the launch).
+cudaError_t launch_prefill(const void* q, float* out, int* status, int* sched, const void* pool_tensor_map, int B, int T,
+                           int Hq, int G, int n, int row_stride, long long krow0, long long vrow0, float scale_log2,
+                           int sm_count, cudaStream_t stream);
 
 // Strategy-search reductions (see kvs_search.cu).
 constexpr int kMaxLayersSearch = 80;     // shared-memory bound of the distance kernel

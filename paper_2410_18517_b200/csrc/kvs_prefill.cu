@@ -154,15 +154,44 @@ __device__ __forceinline__ uint32_t pack2_bf16(float lo, float hi) {
 }
 
 struct PrefillArgs {
-    float* out;      // [B][T][Hq][128]
     int* status;
+    int* sched;      // work counter, zero when the kernel starts
     int n;           // rows cached in the slot (after this pass's append)
     int T;           // queries per head
-    int Hq, G;
+    int Hq, G, B;
     int row_stride;
     long long krow0, vrow0;  // first row of the slot's K / V plane in the pool-wide row numbering
     float scale_log2;
 };
+
+// A work item = 128 queries of one (sequence, q-head).  Items are numbered so that the ones with
+// the most keys come first; neighbours in the numbering share a query block, and the q-heads of
+// one kv-head are adjacent (their K/V tiles meet in L2).
+struct PrefillItem {
+    int q0, hq, b, nt;
+};
+__device__ __forceinline__ PrefillItem decode_item(int w, const PrefillArgs& a) {
+    const int per_qb = a.Hq * a.B;
+    const int nqb = (a.T + kPfTile - 1) / kPfTile;
+    const int qb = nqb - 1 - w / per_qb;
+    const int rem = w % per_qb;
+    PrefillItem it;
+    it.q0 = qb * kPfTile;
+    it.hq = rem % a.Hq;
+    it.b = rem / a.Hq;
+    // last key any query of the block may see, and the key tiles that cover keys 0..that
+    const int last_key = min(a.n - a.T + it.q0 + kPfTile - 1, a.n - 1);
+    it.nt = last_key / kPfKeys + 1;
+    return it;
+}
+
+// TMA store of one [128 rows][32 floats] block (128-byte swizzle) of the output tile.
+__device__ __forceinline__ void tma_store_4d(const CUtensorMap* tmap, const void* src, int c0, int c1, int c2, int c3) {
+    asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.bulk_group [%0, {%1, %2, %3, %4}], [%5];" ::"l"(
+                     reinterpret_cast<uint64_t>(tmap)),
+                 "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(smem_u32(src))
+                 : "memory");
+}
 
 // max(a, b, c) in one instruction
 __device__ __forceinline__ float fmax3(float a, float b, float c) {
@@ -199,42 +228,45 @@ __device__ __forceinline__ float softmax_chunk(const float (&x)[32], float scale
 
 __global__ void __launch_bounds__(kPfThreads, 2)
     prefill_attention_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_kv,
-                         const PrefillArgs a) {
+                         const __grid_constant__ CUtensorMap tmap_out, const PrefillArgs a) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
-    unsigned char* sQ = smem;
+    unsigned char* sQ = smem;                       // Q tile; after an item's last MMA, staging for its output
     unsigned char* sK = sQ + kPfQBytes;             // two stages
     unsigned char* sV = sK + 2 * kPfKvBytes;        // two stages
     uint64_t* bars = reinterpret_cast<uint64_t*>(sV + 2 * kPfKvBytes);
     uint64_t* q_full = bars;
-    uint64_t* o_full = bars + 1;        // one phase per PV group: tile j's output contribution is in O
-    uint64_t* k_full = bars + 2;        // [2] per K stage
-    uint64_t* k_empty = bars + 4;
-    uint64_t* v_full = bars + 6;        // [2] per V stage
-    uint64_t* v_empty = bars + 8;
-    uint64_t* s_full = bars + 10;       // [2] per score buffer
-    uint64_t* p_full = bars + 12;       // [2] per score buffer, one arrival per softmax thread
-    uint64_t* pair_bar = bars + 14;     // [4]: the two warps that share 32 query rows, 64 arrivals
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 18);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 19);
+    uint64_t* q_free = bars + 1;        // the output staged in the Q buffer has been read by the TMA store
+    uint64_t* o_full = bars + 2;        // one phase per PV group: that tile's contribution is in O
+    uint64_t* epi_bar = bars + 3;       // all softmax threads, used around the output staging
+    uint64_t* k_full = bars + 4;        // [2] per K stage
+    uint64_t* k_empty = bars + 6;
+    uint64_t* v_full = bars + 8;        // [2] per V stage
+    uint64_t* v_empty = bars + 10;
+    uint64_t* s_full = bars + 12;       // [2] per score buffer
+    uint64_t* p_full = bars + 14;       // [2] per score buffer, one arrival per softmax thread
+    uint64_t* pair_bar = bars + 16;     // [4]: the two warps that share 32 query rows, 64 arrivals
+    uint64_t* item_full = bars + 20;    // [2] work-item ring: written by the producer lane
+    uint64_t* item_empty = bars + 22;   // [2] released by the MMA lane and every softmax thread
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 24);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(bars + 25);
+    volatile int* ring = reinterpret_cast<volatile int*>(bars + 26);   // [2] item numbers, -1 = no more work
     float* exch_m = reinterpret_cast<float*>(bars + 32);   // [2 tile parities][2 key halves][128] row maxima
     float* exch_l = exch_m + 4 * kPfTile;                  // [2 key halves][128] row sums
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int qb = gridDim.x - 1 - blockIdx.x;       // blocks with the most keys first
-    const int hq = blockIdx.y, b = blockIdx.z;
-    const int hk = hq / a.G;
     const int Hkv = a.Hq / a.G;
-    const int q0 = qb * kPfTile;
-    // last key any query of this block may see, and the key tiles that cover keys 0..that
-    const int last_key = min(a.n - a.T + q0 + kPfTile - 1, a.n - 1);
-    const int nt = last_key / kPfKeys + 1;
+    const int total_items = ((a.T + kPfTile - 1) / kPfTile) * a.Hq * a.B;
+    constexpr int kSoftmaxThreads = kPfSoftmaxWarps * 32;
 
     if (tid == 0) {
-        for (int i = 0; i < 12; ++i) mbar_init(&bars[i], 1);
-        mbar_init(&p_full[0], kPfSoftmaxWarps * 32);
-        mbar_init(&p_full[1], kPfSoftmaxWarps * 32);
+        for (int i = 0; i < 24; ++i) mbar_init(&bars[i], 1);
+        mbar_init(epi_bar, kSoftmaxThreads);
+        mbar_init(&p_full[0], kSoftmaxThreads);
+        mbar_init(&p_full[1], kSoftmaxThreads);
         for (int i = 0; i < 4; ++i) mbar_init(&pair_bar[i], 64);
+        mbar_init(&item_empty[0], kSoftmaxThreads + 1);
+        mbar_init(&item_empty[1], kSoftmaxThreads + 1);
         abort_flag[0] = 0;
         fence_mbar_init();
     }
@@ -251,29 +283,56 @@ __global__ void __launch_bounds__(kPfThreads, 2)
     const uint32_t tmem_s = tmem_base;         // two score buffers of 64 fp32 columns; P_hi / P_lo overwrite them
     const uint32_t tmem_o = tmem_base + 128;   // running output rows
 
+    // Every role walks the same sequence of work items (numbers handed out by the producer lane
+    // through a two-entry ring) and keeps its own count `t` of key tiles done in earlier items:
+    // stage = t & 1, and a stage's barrier is in phase (t >> 1) & 1.
     if (warp == kPfSoftmaxWarps) {
-        // ------------------------------ TMA producer ------------------------------
+        // ------------------------------ scheduler + TMA producer ------------------------------
         if (lane == 0) {
-            mbar_arrive_expect_tx(q_full, kPfQBytes);
-            tma_load_4d(sQ, &tmap_q, 0, hq, q0, b, q_full);
-            tma_load_4d(sQ + kPfQBytes / 2, &tmap_q, 64, hq, q0, b, q_full);
-            const long long unit_row = ((long long)b * Hkv + hk) * a.row_stride;
-            for (int j = 0; j < nt; ++j) {
-                const int st = j & 1;
-                const uint32_t prev = (uint32_t)((j >> 1) - 1) & 1u;   // phase in which tile j-2 released the stage
-                const long long row = unit_row + (long long)j * kPfKeys;
-                if (j >= 2 && !mbar_wait_bounded(&k_empty[st], prev, abort_flag, a.status)) break;
-                mbar_arrive_expect_tx(&k_full[st], kPfKvBytes);
+            int t = 0;
+            bool ok = true;
+            for (int it = 0; ok; ++it) {
+                const int slot = it & 1;
+                if (it >= 2) ok = mbar_wait_bounded(&item_empty[slot], (uint32_t)((it >> 1) - 1) & 1u, abort_flag, a.status);
+                if (!ok) break;
+                int w = atomicAdd(a.sched, 1);
+                if (w >= total_items) w = -1;
+                ring[slot] = w;
+                mbar_arrive(&item_full[slot]);
+                if (w < 0) break;
+                const PrefillItem item = decode_item(w, a);
+                const long long unit_row = ((long long)item.b * Hkv + item.hq / a.G) * a.row_stride;
+                auto load_q = [&]() {
+                    // the Q buffer doubles as the previous item's output staging
+                    if (it >= 1 && !mbar_wait_bounded(q_free, (uint32_t)(it - 1) & 1u, abort_flag, a.status)) return false;
+                    mbar_arrive_expect_tx(q_full, kPfQBytes);
+                    tma_load_4d(sQ, &tmap_q, 0, item.hq, item.q0, item.b, q_full);
+                    tma_load_4d(sQ + kPfQBytes / 2, &tmap_q, 64, item.hq, item.q0, item.b, q_full);
+                    return true;
+                };
+                for (int j = 0; j < item.nt && ok; ++j) {
+                    // the first two K/V tiles do not depend on the previous item's output being
+                    // gone from the Q buffer, so they are fetched before Q
+                    if (j == 2) ok = load_q();
+                    if (!ok) break;
+                    const int tt = t + j, st = tt & 1;
+                    const uint32_t prev = (uint32_t)((tt >> 1) - 1) & 1u;   // phase in which tile tt-2 released the stage
+                    const long long row = unit_row + (long long)j * kPfKeys;
+                    if (tt >= 2 && !mbar_wait_bounded(&k_empty[st], prev, abort_flag, a.status)) { ok = false; break; }
+                    mbar_arrive_expect_tx(&k_full[st], kPfKvBytes);
 #pragma unroll
-                for (int h = 0; h < 2; ++h)
-                    tma_load_2d_pf(sK + st * kPfKvBytes + h * (kPfKvBytes / 2), &tmap_kv, h * 64, (int)(a.krow0 + row),
-                                   &k_full[st]);
-                if (j >= 2 && !mbar_wait_bounded(&v_empty[st], prev, abort_flag, a.status)) break;
-                mbar_arrive_expect_tx(&v_full[st], kPfKvBytes);
+                    for (int h = 0; h < 2; ++h)
+                        tma_load_2d_pf(sK + st * kPfKvBytes + h * (kPfKvBytes / 2), &tmap_kv, h * 64, (int)(a.krow0 + row),
+                                       &k_full[st]);
+                    if (tt >= 2 && !mbar_wait_bounded(&v_empty[st], prev, abort_flag, a.status)) { ok = false; break; }
+                    mbar_arrive_expect_tx(&v_full[st], kPfKvBytes);
 #pragma unroll
-                for (int h = 0; h < 2; ++h)
-                    tma_load_2d_pf(sV + st * kPfKvBytes + h * (kPfKvBytes / 2), &tmap_kv, h * 64, (int)(a.vrow0 + row),
-                                   &v_full[st]);
+                    for (int h = 0; h < 2; ++h)
+                        tma_load_2d_pf(sV + st * kPfKvBytes + h * (kPfKvBytes / 2), &tmap_kv, h * 64, (int)(a.vrow0 + row),
+                                       &v_full[st]);
+                }
+                if (ok && item.nt <= 2) ok = load_q();
+                t += item.nt;
             }
         }
     } else if (warp == kPfSoftmaxWarps + 1) {
@@ -281,13 +340,14 @@ __global__ void __launch_bounds__(kPfThreads, 2)
         // Order on the tensor pipe: S_0, then per tile j: S_{j+1} (into the other score buffer, so
         // that the softmax of tile j+1 can start the moment the one of tile j ends), PV_j.  The
         // pipe runs one thread's MMAs in issue order, so S_{j+1} overwrites its buffer only after
-        // PV_{j-1} has read P_{j-1} from it.
+        // PV_{j-1} has read P_{j-1} from it.  PV_0 of an item starts a fresh output tile; the
+        // softmax threads arrive for it only after they have read the previous item's output.
         if (lane == 0) {
             const uint32_t idesc_s = instr_desc_bf16(0, kPfKeys);
             const uint32_t idesc_o = instr_desc_bf16(1, 128);
             const uint32_t q_addr = smem_u32(sQ), k_addr = smem_u32(sK), v_addr = smem_u32(sV);
-            auto issue_s = [&](int j) {
-                const int st = j & 1;
+            auto issue_s = [&](int tt) {
+                const int st = tt & 1;
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {   // 16 head-dim columns per step; 4 steps per 64-column block
                     const uint32_t qoff = (ks >> 2) * (kPfQBytes / 2) + (ks & 3) * 32;
@@ -298,99 +358,125 @@ __global__ void __launch_bounds__(kPfThreads, 2)
                 umma_commit(&s_full[st]);
                 umma_commit(&k_empty[st]);     // the K stage may be overwritten once S is done
             };
-            bool ok = mbar_wait_bounded(q_full, 0, abort_flag, a.status) &&
-                      mbar_wait_bounded(&k_full[0], 0, abort_flag, a.status);
-            if (ok) {
-                tc_fence_after();
-                issue_s(0);
-            }
-            for (int j = 0; j < nt && ok; ++j) {
-                const int st = j & 1;
-                const uint32_t ph = (uint32_t)(j >> 1) & 1u;
-                if (j + 1 < nt) {
-                    ok = mbar_wait_bounded(&k_full[st ^ 1], (uint32_t)((j + 1) >> 1) & 1u, abort_flag, a.status);
-                    if (!ok) break;
-                    tc_fence_after();
-                    issue_s(j + 1);
-                }
-                ok = mbar_wait_bounded(&p_full[st], ph, abort_flag, a.status) &&
-                     mbar_wait_bounded(&v_full[st], ph, abort_flag, a.status);
+            int t = 0;
+            bool ok = true;
+            for (int it = 0; ok; ++it) {
+                const int slot = it & 1;
+                ok = mbar_wait_bounded(&item_full[slot], (uint32_t)(it >> 1) & 1u, abort_flag, a.status);
+                if (!ok) break;
+                const int w = ring[slot];
+                if (w < 0) break;
+                const int nt = decode_item(w, a).nt;
+                ok = mbar_wait_bounded(q_full, (uint32_t)it & 1u, abort_flag, a.status) &&
+                     mbar_wait_bounded(&k_full[t & 1], (uint32_t)(t >> 1) & 1u, abort_flag, a.status);
                 if (!ok) break;
                 tc_fence_after();
+                issue_s(t);
+                for (int j = 0; j < nt; ++j) {
+                    const int tt = t + j, st = tt & 1;
+                    const uint32_t ph = (uint32_t)(tt >> 1) & 1u;
+                    if (j + 1 < nt) {
+                        ok = mbar_wait_bounded(&k_full[st ^ 1], (uint32_t)((tt + 1) >> 1) & 1u, abort_flag, a.status);
+                        if (!ok) break;
+                        tc_fence_after();
+                        issue_s(tt + 1);
+                    }
+                    ok = mbar_wait_bounded(&p_full[st], ph, abort_flag, a.status) &&
+                         mbar_wait_bounded(&v_full[st], ph, abort_flag, a.status);
+                    if (!ok) break;
+                    tc_fence_after();
 #pragma unroll
-                for (int ks = 0; ks < kPfKeys / 16; ++ks) {   // 16 keys per step: 8 TMEM columns of bf16 pairs
-                    // V is MN-major: 64 head-dim columns contiguous per key row, the other 64 one
-                    // column block (LBO) away; 8-key groups 1024 bytes (SBO) apart
-                    const uint64_t vdesc =
-                        smem_desc_sw128(v_addr + st * kPfKvBytes + ks * 16 * 128, kPfKvBytes / 2, 1024);
-                    umma_bf16_ts(tmem_o, tmem_s + st * kPfKeys + ks * 8, vdesc, idesc_o, (j > 0) || (ks > 0));     // P_hi
-                    umma_bf16_ts(tmem_o, tmem_s + st * kPfKeys + kPfKeys / 2 + ks * 8, vdesc, idesc_o, 1);       // P_lo
+                    for (int ks = 0; ks < kPfKeys / 16; ++ks) {   // 16 keys per step: 8 TMEM columns of bf16 pairs
+                        // V is MN-major: 64 head-dim columns contiguous per key row, the other 64 one
+                        // column block (LBO) away; 8-key groups 1024 bytes (SBO) apart
+                        const uint64_t vdesc =
+                            smem_desc_sw128(v_addr + st * kPfKvBytes + ks * 16 * 128, kPfKvBytes / 2, 1024);
+                        umma_bf16_ts(tmem_o, tmem_s + st * kPfKeys + ks * 8, vdesc, idesc_o, (j > 0) || (ks > 0));   // P_hi
+                        umma_bf16_ts(tmem_o, tmem_s + st * kPfKeys + kPfKeys / 2 + ks * 8, vdesc, idesc_o, 1);     // P_lo
+                    }
+                    umma_commit(o_full);
+                    umma_commit(&v_empty[st]);
                 }
-                umma_commit(o_full);
-                umma_commit(&v_empty[st]);
+                if (!ok) break;
+                mbar_arrive(&item_empty[slot]);
+                t += nt;
             }
         }
     } else {
         // ------------------------------ softmax / output rows ------------------------------
         const int w4 = warp & 3, hf = warp >> 2;             // TMEM lane quarter, key half of a tile
         const int r = w4 * 32 + lane;                        // query row in the block = TMEM lane
-        const int qpos = min(q0 + r, a.T - 1);               // padding rows repeat the last query
-        const int limit = a.n - a.T + qpos;                  // last key this query may see
-        const int block_min_limit = a.n - a.T + q0;          // smallest limit of any row of the block
         const uint32_t lane_addr = (uint32_t)(w4 * 32) << 16;
         const uint32_t to = tmem_o + lane_addr + hf * 64;        // this thread's 64 columns of the output row
-        float m_ref = -1.0e30f, l = 0.f;                     // p is taken relative to m_ref (log2 domain)
+        // output staging: [128 rows][32 floats] blocks, 128-byte swizzle; this thread's row of the
+        // block its key half owns
+        unsigned char* stage_row = sQ + hf * (kPfQBytes / 2) + r * 128;
+        int t = 0;
+        uint32_t pp = 0, ep = 0;                             // phases used so far of pair_bar[w4] and epi_bar
         bool ok = true;
-        for (int j = 0; j < nt; ++j) {
-            const int st = j & 1;
-            ok = mbar_wait_bounded(&s_full[st], (uint32_t)(j >> 1) & 1u, abort_flag, a.status);
+        for (int it = 0; ok; ++it) {
+            const int slot = it & 1;
+            ok = mbar_wait_bounded(&item_full[slot], (uint32_t)(it >> 1) & 1u, abort_flag, a.status);
             if (!ok) break;
-            tc_fence_after();
-            const uint32_t sb = tmem_s + lane_addr + st * kPfKeys;
-            const uint32_t ts = sb + hf * 32;                     // this thread's 32 scores
-            const uint32_t tph = sb + hf * 16;                    // P_hi words of its keys (key k -> column k/2)
-            const uint32_t tpl = sb + kPfKeys / 2 + hf * 16;      // P_lo words (column 32 + k/2)
-            const int key0 = j * kPfKeys + hf * 32;
-            const bool mask = j * kPfKeys + kPfKeys - 1 > block_min_limit;   // block-uniform
-            float x[32];
-            tmem_ld32(ts, x);
-            // row maximum of the (masked) scores: own half, then the partner warp's through shared
-            // memory.  After the pair barrier both halves of S have been read, so P may overwrite it.
-            float mx = -INFINITY;
-            if (mask) {
+            const int w = ring[slot];
+            if (w < 0) break;
+            const PrefillItem item = decode_item(w, a);
+            const int nt = item.nt;
+            const int qpos = min(item.q0 + r, a.T - 1);          // padding rows repeat the last query
+            const int limit = a.n - a.T + qpos;                  // last key this query may see
+            const int block_min_limit = a.n - a.T + item.q0;     // smallest limit of any row of the block
+            float m_ref = -1.0e30f, l = 0.f;                     // p is taken relative to m_ref (log2 domain)
+            for (int j = 0; j < nt; ++j) {
+                const int tt = t + j, st = tt & 1;
+                ok = mbar_wait_bounded(&s_full[st], (uint32_t)(tt >> 1) & 1u, abort_flag, a.status);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t sb = tmem_s + lane_addr + st * kPfKeys;
+                const uint32_t ts = sb + hf * 32;                     // this thread's 32 scores
+                const uint32_t tph = sb + hf * 16;                    // P_hi words of its keys (key k -> column k/2)
+                const uint32_t tpl = sb + kPfKeys / 2 + hf * 16;      // P_lo words (column 32 + k/2)
+                const int key0 = j * kPfKeys + hf * 32;
+                const bool mask = j * kPfKeys + kPfKeys - 1 > block_min_limit;   // block-uniform
+                float x[32];
+                tmem_ld32(ts, x);
+                // row maximum of the (masked) scores: own half, then the partner warp's through shared
+                // memory.  After the pair barrier both halves of S have been read, so P may overwrite it.
+                float mx = -INFINITY;
+                if (mask) {
 #pragma unroll
-                for (int i = 0; i < 32; ++i) mx = fmaxf(mx, (key0 + i <= limit) ? x[i] : -INFINITY);
-            } else {
+                    for (int i = 0; i < 32; ++i) mx = fmaxf(mx, (key0 + i <= limit) ? x[i] : -INFINITY);
+                } else {
 #pragma unroll
-                for (int i = 0; i < 32; i += 2) mx = fmax3(mx, x[i], x[i + 1]);
-            }
-            float* em = exch_m + st * 2 * kPfTile;
-            em[hf * kPfTile + r] = mx;
-            tc_fence_before();
-            mbar_arrive(&pair_bar[w4]);
-            ok = mbar_wait_bounded(&pair_bar[w4], (uint32_t)j & 1u, abort_flag, a.status);
-            if (!ok) break;
-            tc_fence_after();
-            mx = fmaxf(mx, em[(hf ^ 1) * kPfTile + r]) * a.scale_log2;
-            // The reference maximum only moves when the new one is more than 8 (a factor 256) above
-            // it; then the output row and the sum accumulated so far are rescaled, once every PV
-            // issued so far has landed in O (PV of this tile cannot start before this thread's
-            // arrival below).  Both threads of a row take the same decision from the same numbers.
-            const bool grow = mx > m_ref + 8.0f;
-            if (__any_sync(0xffffffffu, grow)) {
-                const float m_new = grow ? mx : m_ref;
-                const float alpha = fast_exp2(m_ref - m_new);
-                if (j > 0) {
-                    ok = mbar_wait_bounded(o_full, (uint32_t)(j - 1) & 1u, abort_flag, a.status);
-                    if (!ok) break;
-                    tc_fence_after();
-#pragma unroll 1
-                    for (int c = 0; c < 8; ++c) tmem_scale8(to + c * 8, alpha);
+                    for (int i = 0; i < 32; i += 2) mx = fmax3(mx, x[i], x[i + 1]);
                 }
-                l *= alpha;
-                m_ref = m_new;
-            }
-            float lsum = 0.f;
+                float* em = exch_m + st * 2 * kPfTile;
+                em[hf * kPfTile + r] = mx;
+                tc_fence_before();
+                mbar_arrive(&pair_bar[w4]);
+                ok = mbar_wait_bounded(&pair_bar[w4], pp & 1u, abort_flag, a.status);
+                ++pp;
+                if (!ok) break;
+                tc_fence_after();
+                mx = fmaxf(mx, em[(hf ^ 1) * kPfTile + r]) * a.scale_log2;
+                // The reference maximum only moves when the new one is more than 8 (a factor 256) above
+                // it; then the output row and the sum accumulated so far are rescaled, once every PV
+                // issued so far has landed in O (PV of this tile cannot start before this thread's
+                // arrival below).  Both threads of a row take the same decision from the same numbers.
+                const bool grow = mx > m_ref + 8.0f;
+                if (__any_sync(0xffffffffu, grow)) {
+                    const float m_new = grow ? mx : m_ref;
+                    const float alpha = fast_exp2(m_ref - m_new);
+                    if (j > 0) {
+                        ok = mbar_wait_bounded(o_full, (uint32_t)(tt - 1) & 1u, abort_flag, a.status);
+                        if (!ok) break;
+                        tc_fence_after();
+#pragma unroll 1
+                        for (int c = 0; c < 8; ++c) tmem_scale8(to + c * 8, alpha);
+                    }
+                    l *= alpha;
+                    m_ref = m_new;
+                }
+                float lsum = 0.f;
 #define KVS_PF_CHUNK(OFF)                                                                                      \
     {                                                                                                          \
         uint32_t hi[8], lo[8];                                                                                 \
@@ -399,41 +485,63 @@ __global__ void __launch_bounds__(kPfThreads, 2)
         tmem_st8(tph + OFF / 2, hi);                                                                           \
         tmem_st8(tpl + OFF / 2, lo);                                                                           \
     }
-            KVS_PF_CHUNK(0)
-            KVS_PF_CHUNK(16)
+                KVS_PF_CHUNK(0)
+                KVS_PF_CHUNK(16)
 #undef KVS_PF_CHUNK
-            l += lsum;
-            asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
-            tc_fence_before();
-            mbar_arrive(&p_full[st]);
-        }
-        // the row's sum is the two halves' sums (both relative to the same reference maximum)
-        if (ok) {
+                l += lsum;
+                asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+                tc_fence_before();
+                mbar_arrive(&p_full[st]);
+            }
+            if (!ok) break;
+            // the row's sum is the two halves' sums (both relative to the same reference maximum)
             exch_l[hf * kPfTile + r] = l;
             mbar_arrive(&pair_bar[w4]);
-            ok = mbar_wait_bounded(&pair_bar[w4], (uint32_t)nt & 1u, abort_flag, a.status);
-        }
-        if (ok) {
+            ok = mbar_wait_bounded(&pair_bar[w4], pp & 1u, abort_flag, a.status);
+            ++pp;
+            if (!ok) break;
             l += exch_l[(hf ^ 1) * kPfTile + r];
-            ok = mbar_wait_bounded(o_full, (uint32_t)(nt - 1) & 1u, abort_flag, a.status);
-        }
-        if (ok) {
+            ok = mbar_wait_bounded(o_full, (uint32_t)(t + nt - 1) & 1u, abort_flag, a.status);
+            if (!ok) break;
             tc_fence_after();
+            // Output: every MMA of the item is done, so the Q buffer is free.  Each thread scales its
+            // 64 columns and stages them there, 32 columns per round, in the swizzled layout of a TMA
+            // store; one thread issues the stores (rows past the last query are clipped by the
+            // tensor map) and waits until they have read the buffer.
             const float inv = 1.0f / l;
-            const bool store = q0 + r < a.T;
-            float4* dst = reinterpret_cast<float4*>(a.out + (((long long)b * a.T + min(q0 + r, a.T - 1)) * a.Hq + hq) * 128) +
-                          hf * 16;
 #pragma unroll 1
             for (int c = 0; c < 2; ++c) {
                 float o[32];
                 tmem_ld32(to + c * 32, o);
-                if (store) {
 #pragma unroll
-                    for (int i = 0; i < 8; ++i)
-                        dst[c * 8 + i] = make_float4(o[4 * i] * inv, o[4 * i + 1] * inv, o[4 * i + 2] * inv, o[4 * i + 3] * inv);
+                for (int i = 0; i < 8; ++i)
+                    *reinterpret_cast<float4*>(stage_row + ((i ^ (r & 7)) << 4)) =
+                        make_float4(o[4 * i] * inv, o[4 * i + 1] * inv, o[4 * i + 2] * inv, o[4 * i + 3] * inv);
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                mbar_arrive(epi_bar);
+                ok = mbar_wait_bounded(epi_bar, ep & 1u, abort_flag, a.status);
+                ++ep;
+                if (!ok) break;
+                if (tid == 0) {
+                    tma_store_4d(&tmap_out, sQ, c * 32, item.hq, item.q0, item.b);
+                    tma_store_4d(&tmap_out, sQ + kPfQBytes / 2, 64 + c * 32, item.hq, item.q0, item.b);
+                    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+                    asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                    if (c == 1) mbar_arrive(q_free);
+                }
+                if (c == 0) {   // the buffer is reused by the second round
+                    mbar_arrive(epi_bar);
+                    ok = mbar_wait_bounded(epi_bar, ep & 1u, abort_flag, a.status);
+                    ++ep;
+                    if (!ok) break;
                 }
             }
+            if (!ok) break;
+            tc_fence_before();
+            mbar_arrive(&item_empty[slot]);
+            t += nt;
         }
+        if (tid == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // the stores have reached memory
     }
     // every thread of every role ends here; tensor memory is released by the warp that took it
     tc_fence_before();
@@ -464,36 +572,50 @@ cudaError_t init_prefill_kernels() {
     return cudaFuncSetAttribute(prefill_attention_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kPfSmemBytes);
 }
 
-// q: [B][T][Hq][128] bf16.  One block per (128 queries, q-head, sequence).
-cudaError_t launch_prefill(const void* q, float* out, int* status, const void* pool_tensor_map, int B, int T, int Hq,
-                           int G, int n, int row_stride, long long krow0, long long vrow0, float scale_log2,
-                           cudaStream_t stream) {
+// q: [B][T][Hq][128] bf16.  Persistent blocks (two per SM) take (128 queries, q-head, sequence)
+// items from a counter, heaviest first.  `sched` is a device int the launch zeroes on `stream`.
+cudaError_t launch_prefill(const void* q, float* out, int* status, int* sched, const void* pool_tensor_map, int B, int T,
+                           int Hq, int G, int n, int row_stride, long long krow0, long long vrow0, float scale_log2,
+                           int sm_count, cudaStream_t stream) {
     EncodeFn encode = nullptr;
     cudaError_t e = get_encode(&encode);
     if (e != cudaSuccess) return e;
-    alignas(64) CUtensorMap tq;
+    alignas(64) CUtensorMap tq, to;
     cuuint64_t dims[4] = {128, (cuuint64_t)Hq, (cuuint64_t)T, (cuuint64_t)B};
-    cuuint64_t strides[3] = {128 * 2, (cuuint64_t)Hq * 128 * 2, (cuuint64_t)T * Hq * 128 * 2};
-    cuuint32_t box[4] = {64, 1, (cuuint32_t)kPfTile, 1};
     cuuint32_t estr[4] = {1, 1, 1, 1};
-    if (encode(&tq, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(q), dims, strides, box, estr,
-               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-        return cudaErrorInvalidValue;
+    {
+        cuuint64_t strides[3] = {128 * 2, (cuuint64_t)Hq * 128 * 2, (cuuint64_t)T * Hq * 128 * 2};
+        cuuint32_t box[4] = {64, 1, (cuuint32_t)kPfTile, 1};
+        if (encode(&tq, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(q), dims, strides, box, estr,
+                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return cudaErrorInvalidValue;
+    }
+    {
+        cuuint64_t strides[3] = {128 * 4, (cuuint64_t)Hq * 128 * 4, (cuuint64_t)T * Hq * 128 * 4};
+        cuuint32_t box[4] = {32, 1, (cuuint32_t)kPfTile, 1};
+        if (encode(&to, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, out, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                   CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) !=
+            CUDA_SUCCESS)
+            return cudaErrorInvalidValue;
+    }
     PrefillArgs a;
-    a.out = out;
     a.status = status;
+    a.sched = sched;
     a.n = n;
     a.T = T;
     a.Hq = Hq;
     a.G = G;
+    a.B = B;
     a.row_stride = row_stride;
     a.krow0 = krow0;
     a.vrow0 = vrow0;
     a.scale_log2 = scale_log2;
-    dim3 grid((T + kPfTile - 1) / kPfTile, Hq, B);
-    prefill_attention_tc<<<grid, kPfThreads, kPfSmemBytes, stream>>>(
-        tq, *reinterpret_cast<const CUtensorMap*>(pool_tensor_map), a);
+    if ((e = cudaMemsetAsync(sched, 0, sizeof(int), stream)) != cudaSuccess) return e;
+    const long long items = (long long)((T + kPfTile - 1) / kPfTile) * Hq * B;
+    const int blocks = (int)std::min<long long>(items, 2LL * sm_count);
+    prefill_attention_tc<<<blocks, kPfThreads, kPfSmemBytes, stream>>>(
+        tq, *reinterpret_cast<const CUtensorMap*>(pool_tensor_map), to, a);
     return cudaGetLastError();
 }
 
