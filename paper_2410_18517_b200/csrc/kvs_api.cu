@@ -42,6 +42,7 @@ struct kvs_ctx {
     char* pool = nullptr;
     char* ws = nullptr;
     int sm_count = 148;
+    long long l2_bytes = 64ll << 20;
 
     // workspace carve-up (byte offsets)
     size_t off_status = 0, off_part_o = 0, off_part_ml = 0, off_stage_q = 0, off_stage_k = 0, off_stage_v = 0,
@@ -421,6 +422,10 @@ kvs_status kvs_bind_memory(kvs_ctx* ctx, void* pool, size_t pool_bytes, void* wo
         ctx->have_tensor_map = true;
     }
     ctx->sm_count = sms;
+    {
+        int l2 = 0;
+        if (cudaDeviceGetAttribute(&l2, cudaDevAttrL2CacheSize, ctx->cfg.device) == cudaSuccess && l2 > 0) ctx->l2_bytes = l2;
+    }
     ctx->pool = static_cast<char*>(pool);
     ctx->ws = static_cast<char*>(workspace);
     ctx->bound = true;
@@ -483,7 +488,7 @@ kvs_status kvs_prefill_attention(kvs_ctx* ctx, int32_t layer, const void* q, flo
     if (kvs::launch_prefill(q, out, reinterpret_cast<int*>(ctx->ws + ctx->off_status),
                             reinterpret_cast<int*>(ctx->ws + ctx->off_status + 64), ctx->tensor_map, batch, n_q,
                             ctx->cfg.n_q_heads, ctx->G, n, ctx->row_stride, plane_rows * (2 * slot),
-                            plane_rows * (2 * slot + 1), ctx->scale * 1.4426950408889634f, ctx->sm_count,
+                            plane_rows * (2 * slot + 1), ctx->scale * 1.4426950408889634f, ctx->sm_count, ctx->l2_bytes,
                             static_cast<cudaStream_t>(stream)) != cudaSuccess)
         return KVS_ERR_CUDA;
     // a plain launch: it starts only after everything before it on the stream has finished

@@ -69,7 +69,7 @@ cudaError_t init_prefill_kernels();
 // `sched`: a device int for the kernel's work counter (zeroed on `stream` by the launch).
 cudaError_t launch_prefill(const void* q, float* out, int* status, int* sched, const void* pool_tensor_map, int B, int T,
                            int Hq, int G, int n, int row_stride, long long krow0, long long vrow0, float scale_log2,
-                           int sm_count, cudaStream_t stream);
+                           int sm_count, long long l2_bytes, cudaStream_t stream);
 
 // Strategy-search reductions (see kvs_search.cu).
 constexpr int kMaxLayersSearch = 80;     // shared-memory bound of the distance kernel

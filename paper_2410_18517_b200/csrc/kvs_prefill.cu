@@ -159,26 +159,33 @@ struct PrefillArgs {
     int n;           // rows cached in the slot (after this pass's append)
     int T;           // queries per head
     int Hq, G, B;
+    int group_heads; // q-heads per scheduling group (a multiple of G)
     int row_stride;
     long long krow0, vrow0;  // first row of the slot's K / V plane in the pool-wide row numbering
     float scale_log2;
 };
 
-// A work item = 128 queries of one (sequence, q-head).  Items are numbered so that the ones with
-// the most keys come first; neighbours in the numbering share a query block, and the q-heads of
-// one kv-head are adjacent (their K/V tiles meet in L2).
+// A work item = 128 queries of one (sequence, q-head).  The q-heads (numbered sequence-major, so
+// the heads of one kv-head are adjacent) are taken in groups of `group_heads`; inside a group the
+// items run from the query blocks with the most keys down, all heads of the group per block.
+// The group is sized on the host so that the K/V rows its heads stream fit in L2 together, while
+// the blocks running at one moment still spread over as many kv-heads as that allows.
 struct PrefillItem {
     int q0, hq, b, nt;
 };
 __device__ __forceinline__ PrefillItem decode_item(int w, const PrefillArgs& a) {
-    const int per_qb = a.Hq * a.B;
     const int nqb = (a.T + kPfTile - 1) / kPfTile;
-    const int qb = nqb - 1 - w / per_qb;
-    const int rem = w % per_qb;
+    const int nheads = a.Hq * a.B;
+    const int ipg = nqb * a.group_heads;                       // items of a full group
+    const int g = min(w / ipg, (nheads - 1) / a.group_heads);
+    const int r = w - g * ipg;
+    const int gh = min(a.group_heads, nheads - g * a.group_heads);   // the last group may be smaller
+    const int qb = nqb - 1 - r / gh;
+    const int head = g * a.group_heads + r % gh;
     PrefillItem it;
     it.q0 = qb * kPfTile;
-    it.hq = rem % a.Hq;
-    it.b = rem / a.Hq;
+    it.hq = head % a.Hq;
+    it.b = head / a.Hq;
     // last key any query of the block may see, and the key tiles that cover keys 0..that
     const int last_key = min(a.n - a.T + it.q0 + kPfTile - 1, a.n - 1);
     it.nt = last_key / kPfKeys + 1;
@@ -576,7 +583,7 @@ cudaError_t init_prefill_kernels() {
 // items from a counter, heaviest first.  `sched` is a device int the launch zeroes on `stream`.
 cudaError_t launch_prefill(const void* q, float* out, int* status, int* sched, const void* pool_tensor_map, int B, int T,
                            int Hq, int G, int n, int row_stride, long long krow0, long long vrow0, float scale_log2,
-                           int sm_count, cudaStream_t stream) {
+                           int sm_count, long long l2_bytes, cudaStream_t stream) {
     EncodeFn encode = nullptr;
     cudaError_t e = get_encode(&encode);
     if (e != cudaSuccess) return e;
@@ -611,6 +618,15 @@ cudaError_t launch_prefill(const void* q, float* out, int* status, int* sched, c
     a.krow0 = krow0;
     a.vrow0 = vrow0;
     a.scale_log2 = scale_log2;
+    {
+        // kv-heads whose K/V rows (n rows of 256 bytes, K and V) fit in three quarters of L2
+        // together; groups of equal size
+        const long long streams = (long long)B * (Hq / G);
+        const long long stream_bytes = 2LL * n * 256;
+        const long long fit = std::max<long long>(1, (l2_bytes / 4 * 3) / stream_bytes);
+        const long long groups = (streams + fit - 1) / fit;
+        a.group_heads = (int)((streams + groups - 1) / groups) * G;
+    }
     if ((e = cudaMemsetAsync(sched, 0, sizeof(int), stream)) != cudaSuccess) return e;
     const long long items = (long long)((T + kPfTile - 1) / kPfTile) * Hq * B;
     const int blocks = (int)std::min<long long>(items, 2LL * sm_count);
