@@ -22,7 +22,8 @@
  *   - work is enqueued on the given CUDA stream (a cudaStream_t passed as
  *     void*, NULL = the legacy default stream) and returns without waiting,
  *     except where a call says otherwise;
- *   - all sequences of a batch have the same length (no ragged batches).
+ *   - all sequences of a batch are appended to together and have the same length, until
+ *     kvs_evict makes the (sequence, head) units of a slot differ.
  *
  * Memory layout of the pool (device, caller-owned, bound with kvs_bind_memory):
  *   plane(slot, kv) with kv = 0 for K and 1 for V, each plane being
@@ -180,7 +181,7 @@ kvs_status kvs_decode_attention(kvs_ctx* ctx, int32_t layer, const void* q, floa
  * chunk of it (n > n_q).
  *   q:   device, [batch][n_q][n_q_heads][head_dim], storage type, 16-byte aligned
  *   out: device, [batch][n_q][n_q_heads][head_dim], float32
- * One tcgen05 tensor-core kernel on `stream`; bf16 storage and head_dim 128 only (other
+ * One 4-byte clear and one tcgen05 tensor-core kernel on `stream`; bf16 storage and head_dim 128 only (other
  * configurations: INVALID_ARG).  Other errors as kvs_decode_attention; n_q > n: INVALID_ARG. */
 kvs_status kvs_prefill_attention(kvs_ctx* ctx, int32_t layer, const void* q, float* out,
                                  int32_t batch, int32_t n_q, void* stream);
@@ -262,7 +263,7 @@ kvs_status kvs_replay_commit(kvs_ctx* ctx, int32_t times_run, void* stream);
  * Copies inputs host->device into the workspace staging area, runs the layers on
  * `stream`, copies the result device->host, and waits until all of it is done.  The
  * copies run on two extra streams owned by the context (created at the first call,
- * together with a few events) in eight chunks of layers, so that they overlap the
+ * together with a few events) in chunks of layers (KVS_OPT_HOST_CHUNKS), so that they overlap the
  * layers of the neighbouring chunks.
  * Pinned host memory makes the copies asynchronous; pageable memory also works.
  * h2d_bytes / d2h_bytes (host, may be NULL) receive the bytes copied.
