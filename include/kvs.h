@@ -96,13 +96,8 @@ typedef enum {
     KVS_OPT_REPLAY = 3,     /* 1: launches also read a device-side growth counter, so that a
                                recorded decode step can be replayed as a CUDA graph (see
                                kvs_replay_advance).  0 (default): lengths come from the host only. */
-    KVS_OPT_HOST_CHUNKS = 4,/* kvs_step_host: number of pieces (1..8, default 4) the layers are cut
+    KVS_OPT_HOST_CHUNKS = 4 /* kvs_step_host: number of pieces (1..8, default 4) the layers are cut
                                into for overlapping the host copies with the kernels.            */
-    KVS_OPT_FUSED_COMBINE = 5 /* 1 (default): the split-K kernel also merges the pieces of every
-                               (sequence, kv-head) unit -- the last thread block to finish a unit
-                               does it, always in block order -- so an attention call is one
-                               kernel.  0: a separate combine kernel follows.  Results are
-                               identical bit for bit.                                           */
 } kvs_option;
 
 /* ---- life cycle ------------------------------------------------------------ */
@@ -169,10 +164,9 @@ kvs_status kvs_append(kvs_ctx* ctx, int32_t layer, const void* k, const void* v,
  * over all n cached rows j, no mask, G = n_q_heads / n_kv_heads.
  *   q:   device, [batch][n_q_heads][head_dim], storage type
  *   out: device, [batch][n_q_heads][head_dim], float32
- * Launches the split-K kernel on `stream` (plus a combine kernel if
- * KVS_OPT_FUSED_COMBINE is 0); partial results and per-unit arrival counters go
- * through the bound workspace, so calls on one context must not overlap on the
- * GPU (use one stream, or order them).
+ * Launches the split-K kernel and the combine kernel on `stream`; partial
+ * results go through the bound workspace, so calls on one context must not
+ * overlap on the GPU (use one stream, or order them).
  * Errors: STATE before kvs_bind_memory or when the slot is empty; INVALID_ARG
  * for a bad layer, NULLs, batch < 1 or batch > the batch the slot was filled for. */
 kvs_status kvs_decode_attention(kvs_ctx* ctx, int32_t layer, const void* q, float* out,
@@ -290,10 +284,9 @@ kvs_status kvs_step_host(kvs_ctx* ctx, const void* q_host, const void* k_host, c
  * still pass the inputs and outputs (q, out, and the context whose pool holds K/V); what they
  * cannot provide is the scratch for split-K partial results.
  *
- * What it does: exactly what kvs_decode_attention does, with the same split-K kernel and the
- * same result bit for bit, except that the partial results and the device status word live in a
- * fixed 2 MiB array inside the library image instead of the bound workspace, and that the pieces
- * are always merged by the separate combine kernel (no arrival counters are needed).  The call
+ * What it does: exactly what kvs_decode_attention does, with the same kernels and the same
+ * result bit for bit, except that the partial results and the device status word live in a
+ * fixed 2 MiB array inside the library image instead of the bound workspace.  The call
  * allocates nothing and frees nothing, on the device or through any library.
  *   - Every GPU that loads the library holds those 2 MiB until the process exits.
  *   - Limit: (batch * n_kv_heads + blocks launched) * group * (head_dim + 2) * 4 bytes, plus
@@ -325,9 +318,7 @@ kvs_status kvs_plane_offset(const kvs_ctx* ctx, int32_t slot, int32_t kv, size_t
 kvs_status kvs_stats(const kvs_ctx* ctx, kvs_stats_t* stats);
 /* Reads the device status word (waits for the default stream's prior work on it):
  * 0 = no device-side problem; KVS_ERR_TIMEOUT = a bounded wait inside a kernel ran
- * out and the kernel returned early (its output is then undefined).  When it is not 0
- * the call also clears the workspace's arrival counters, which such a kernel may have
- * left half way; synchronise the context's streams before calling it in that case.   */
+ * out and the kernel returned early (its output is then undefined).             */
 kvs_status kvs_last_device_status(kvs_ctx* ctx, int32_t* device_status);
 kvs_status kvs_set_option(kvs_ctx* ctx, int32_t option, int32_t value);
 /* How the last kvs_decode_attention call was decomposed: thread blocks launched,

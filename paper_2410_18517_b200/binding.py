@@ -31,7 +31,6 @@ KVS_OPT_KERNEL = 1
 KVS_OPT_EARLY_START = 2
 KVS_OPT_REPLAY = 3
 KVS_OPT_HOST_CHUNKS = 4
-KVS_OPT_FUSED_COMBINE = 5
 
 # every symbol include/kvs.h declares
 EXPORTS = (

@@ -46,7 +46,7 @@ struct kvs_ctx {
 
     // workspace carve-up (byte offsets)
     size_t off_status = 0, off_part_o = 0, off_part_ml = 0, off_stage_q = 0, off_stage_k = 0, off_stage_v = 0,
-           off_stage_out = 0, off_unit_len = 0, off_counts = 0, off_search = 0, off_replay = 0, off_arrive = 0, ws_bytes = 0;
+           off_stage_out = 0, off_unit_len = 0, off_counts = 0, off_search = 0, off_replay = 0, ws_bytes = 0;
 
     alignas(64) unsigned char tensor_map[128];  // TMA view of the pool (bf16 storage only)
     bool have_tensor_map = false;
@@ -70,7 +70,6 @@ struct kvs_ctx {
     int opt_kernel = 0;
     int opt_pdl = 1;
     int opt_host_chunks = 4;
-    int opt_fused_combine = 1;
     int opt_replay = 0;   // launches carry the device-side growth counter (for CUDA-graph replay)
     // The split-K kernels read the growth counter before their wait.  That is safe because the
     // first launch after anything wrote the counter never starts early (full dependency): it and
@@ -156,8 +155,6 @@ void layout_workspace(kvs_ctx* c) {
     off = align_up(off + units * sizeof(int32_t), kAlign);
     c->off_replay = off;        // one int: rows every slot has grown by since a recorded launch
     off += kAlign;
-    c->off_arrive = off;        // per-unit arrival counters of the split-K kernels (zero between launches)
-    off = align_up(off + units * sizeof(int32_t), kAlign);
     c->off_search = off;        // per-block partial sums of the strategy-search reductions
     {
         const size_t need = std::max(kvs::distance_partial_bytes(f.n_layers <= kvs::kMaxLayersSearch ? f.n_layers : 4),
@@ -252,7 +249,6 @@ struct AttentionScratch {
     float* part_o;
     float* part_ml;
     int* status;
-    int* arrive;         // per-unit arrival counters (combine inside the split-K kernel), or nullptr
     bool programmatic;   // early-start launches (only when the call follows this context's own kernels)
 };
 
@@ -267,8 +263,7 @@ bool choose_plan(const kvs_ctx* c, int units, int n, kvs::DecodePlan* plan) {
     return use_mma;
 }
 
-// Split-K kernel (+ combine kernel, unless the split-K kernel combines itself) of one layer, with the
-// given plan and scratch.
+// Split-K kernel + combine kernel of one layer, with the given plan and scratch.
 kvs_status run_attention(kvs_ctx* c, int slot, const void* q, float* out, int batch, const kvs::DecodePlan& plan,
                          bool use_mma, const AttentionScratch& scratch, cudaStream_t st) {
     kvs::DecodeArgs a;
@@ -279,7 +274,6 @@ kvs_status run_attention(kvs_ctx* c, int slot, const void* q, float* out, int ba
     a.part_ml = scratch.part_ml;
     a.out = out;
     a.status = scratch.status;
-    a.arrive = scratch.arrive;
     a.n = c->slot_len[slot];
     a.row_stride = c->row_stride;
     a.units = batch * c->cfg.n_kv_heads;
@@ -291,9 +285,8 @@ kvs_status run_attention(kvs_ctx* c, int slot, const void* q, float* out, int ba
     a.safe_rows = scratch.programmatic ? safe_rows_of(c, slot) : 0;
     a.unit_len = c->ragged[slot] ? unit_len_dev(c, slot) : nullptr;
     a.n_extra = replay_counter(c);
-    const bool fused = a.arrive != nullptr;
-    c->seq += fused ? 1 : 2;           // split-K kernel, then (unless it combines itself) the combine kernel
-    c->last_splitk_seq = fused ? c->seq : c->seq - 1;
+    c->seq += 2;                       // split-K kernel, then combine
+    c->last_splitk_seq = c->seq - 1;
     if (use_mma) {
         const long long plane_rows = (long long)c->cfg.max_batch * c->cfg.n_kv_heads * c->row_stride;
         if (kvs::launch_decode_mma(a, plan, c->tensor_map, plane_rows * (2 * slot), plane_rows * (2 * slot + 1), st) !=
@@ -302,10 +295,10 @@ kvs_status run_attention(kvs_ctx* c, int slot, const void* q, float* out, int ba
     } else {
         if (kvs::launch_decode_scalar(a, plan, st) != cudaSuccess) return KVS_ERR_CUDA;
     }
-    if (!fused && kvs::launch_combine(a, plan, st) != cudaSuccess) return KVS_ERR_CUDA;
+    if (kvs::launch_combine(a, plan, st) != cudaSuccess) return KVS_ERR_CUDA;
     c->last_plan = plan;
     c->stats.attention_launches += 1;
-    c->stats.combine_launches += fused ? 0 : 1;
+    c->stats.combine_launches += 1;
     if (c->ragged[slot]) {
         unsigned long long rows = 0;
         for (int u = 0; u < a.units; ++u) rows += c->unit_len_host[slot][u];
@@ -322,9 +315,7 @@ kvs_status do_attention(kvs_ctx* c, int layer, const void* q, float* out, int ba
     const bool use_mma = choose_plan(c, batch * c->cfg.n_kv_heads, c->slot_len[slot], &plan);
     const AttentionScratch scratch = {reinterpret_cast<float*>(c->ws + c->off_part_o),
                                       reinterpret_cast<float*>(c->ws + c->off_part_ml),
-                                      reinterpret_cast<int*>(c->ws + c->off_status),
-                                      c->opt_fused_combine ? reinterpret_cast<int*>(c->ws + c->off_arrive) : nullptr,
-                                      take_early_start(c)};
+                                      reinterpret_cast<int*>(c->ws + c->off_status), take_early_start(c)};
     return run_attention(c, slot, q, out, batch, plan, use_mma, scratch, st);
 }
 
@@ -788,11 +779,6 @@ kvs_status kvs_last_device_status(kvs_ctx* ctx, int32_t* device_status) {
     if (cudaMemcpy(&v, ctx->ws + ctx->off_status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess)
         return KVS_ERR_CUDA;
     *device_status = v;
-    if (v != 0) {
-        // a kernel that gave up may have left arrival counters of the split-K kernels half way
-        const size_t units = (size_t)ctx->cfg.max_batch * ctx->cfg.n_kv_heads;
-        if (cudaMemset(ctx->ws + ctx->off_arrive, 0, units * sizeof(int32_t)) != cudaSuccess) return KVS_ERR_CUDA;
-    }
     return KVS_OK;
 }
 
@@ -814,10 +800,6 @@ kvs_status kvs_set_option(kvs_ctx* ctx, int32_t option, int32_t value) {
         case KVS_OPT_HOST_CHUNKS:
             if (value < 1 || value > kvs_ctx::kChunks) return KVS_ERR_INVALID_ARG;
             ctx->opt_host_chunks = value;
-            return KVS_OK;
-        case KVS_OPT_FUSED_COMBINE:
-            if (value != 0 && value != 1) return KVS_ERR_INVALID_ARG;
-            ctx->opt_fused_combine = value;
             return KVS_OK;
         case KVS_OPT_KERNEL:
             if (value < 0 || value > 2) return KVS_ERR_INVALID_ARG;
@@ -927,7 +909,6 @@ kvs_status kvs_decode_attention_static(kvs_ctx* ctx, int32_t layer, const void* 
     // plain launches: the kernels start after everything before them on the stream
     const AttentionScratch scratch = {reinterpret_cast<float*>(base + kStaticStatusBytes),
                                       reinterpret_cast<float*>(base + kStaticStatusBytes + part_o_bytes), status_word,
-                                      nullptr /* separate combine kernel: nothing in the array has to start at zero */,
                                       false};
     c->counter_written = false;
     return run_attention(c, slot, q, out, batch, plan, use_mma, scratch, st);

@@ -160,52 +160,3 @@ inline cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block
 }
 
 }  // namespace kvs
-
-namespace kvs {
-
-// Work decomposition shared by the split-K kernels and the combine step.
-// Thread block c owns tiles [c*T/NC, (c+1)*T/NC) of the line of T tiles.
-__host__ __device__ __forceinline__ long long first_tile_of_cta(long long c, long long T, int NC) {
-    return (c * T) / NC;
-}
-// The thread block that owns tile gt (inverse of the above).
-__host__ __device__ __forceinline__ int cta_of_tile(long long gt, long long T, int NC) {
-    return (int)(((gt + 1) * NC + T - 1) / T - 1);
-}
-
-// Combine inside the split-K kernel.  Called by all NTHREADS consumer threads of a block (named
-// barrier 1) after they have written the block's partial result of unit u, which blocks c0..c1
-// share (c1 > c0).  Every block adds one to the unit's arrival counter; the one that finds all
-// the others already there merges the pieces, in block order whoever comes last, exactly as
-// the separate combine kernel does, and puts the counter back to zero for the next launch.
-template <int NTHREADS>
-__device__ __forceinline__ void arrive_and_combine(int tid, long long u, int c0, int c1, int G, int D,
-                                                   const float* part_o, const float* part_ml, float* out, int* arrive,
-                                                   volatile int* flag) {
-    __threadfence();                       // this thread's partial results, before the block's arrival
-    named_bar_sync(1, NTHREADS);
-    if (tid == 0) {
-        const int last = atomicAdd(&arrive[u], 1) == c1 - c0;
-        if (last) arrive[u] = 0;
-        __threadfence();
-        *flag = last;
-    }
-    named_bar_sync(1, NTHREADS);
-    if (*flag == 0) return;
-    for (int idx = tid; idx < G * D; idx += NTHREADS) {
-        const int g = idx / D, d = idx - g * D;
-        float M = -1.0e30f;
-        for (int c = c0; c <= c1; ++c) M = fmaxf(M, __ldcg(&part_ml[((u + c) * G + g) * 2]));
-        float o = 0.f, den = 0.f;
-#pragma unroll 4
-        for (int c = c0; c <= c1; ++c) {
-            const long long pid = u + c;
-            const float w = fast_exp2(__ldcg(&part_ml[(pid * G + g) * 2]) - M);
-            o = fmaf(w, __ldcg(&part_o[(pid * G + g) * D + d]), o);
-            den = fmaf(w, __ldcg(&part_ml[(pid * G + g) * 2 + 1]), den);
-        }
-        out[(u * G + g) * D + d] = o / den;
-    }
-}
-
-}  // namespace kvs

@@ -136,6 +136,18 @@ cudaError_t launch_add_len(int* unit_len, int delta, int units, bool programmati
 }
 
 // --------------------------------------------------------------------------------------
+// Work decomposition shared by the split-K kernel and the combine kernel.
+// Thread block c owns tiles [c*T/NC, (c+1)*T/NC) of the line of T tiles.
+// --------------------------------------------------------------------------------------
+__host__ __device__ __forceinline__ long long first_tile_of_cta(long long c, long long T, int NC) {
+    return (c * T) / NC;
+}
+// The thread block that owns tile gt (inverse of the above).
+__host__ __device__ __forceinline__ int cta_of_tile(long long gt, long long T, int NC) {
+    return (int)(((gt + 1) * NC + T - 1) / T - 1);
+}
+
+// --------------------------------------------------------------------------------------
 // K2a: scalar split-K decode attention.
 //
 // Shapes: T = storage type, D = head size, G = q-heads per kv-head.
@@ -242,8 +254,6 @@ struct ScalarKernelArgs {
     const int* unit_len;  // per-unit row counts of a ragged slot, or nullptr (then n holds for all)
     const int* n_extra;   // graph replay: rows every slot has grown by since the launch was recorded, or nullptr
     int units;
-    float* out;           // final output, written here when `arrive` is set
-    int* arrive;          // per-unit arrival counters (combine inside this kernel), or nullptr
 };
 
 template <typename T, int D, int G, int GEOM>
@@ -450,9 +460,6 @@ __global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G, GEOM>::MI
 
         // ---- end of piece: merge the NG lane groups, one q-head at a time ----
         const long long pid = u + blockIdx.x;
-        // blocks that share this unit; a unit this block has to itself is finished here
-        const int c0 = cta_of_tile(u * a.tpu, a.T, NC), c1 = cta_of_tile((u + 1) * a.tpu - 1, a.T, NC);
-        const bool whole = a.arrive != nullptr && c0 == c1;
 #pragma unroll
         for (int g = 0; g < G; ++g) {
             // lanes with equal top bits hold duplicates of lsum; add across the R distinct ones
@@ -479,10 +486,6 @@ __global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G, GEOM>::MI
                     o = fmaf(w, scratch[j * (D + 2) + d], o);
                     den = fmaf(w, scratch[j * (D + 2) + D + 1], den);
                 }
-                if (whole) {
-                    a.out[(u * G + g) * D + d] = o / den;
-                    continue;
-                }
                 a.part_o[(pid * G + g) * D + d] = o;
                 if (d == 0) {
                     a.part_ml[(pid * G + g) * 2] = M;
@@ -490,8 +493,6 @@ __global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G, GEOM>::MI
                 }
             }
         }
-        if (a.arrive != nullptr && !whole)
-            arrive_and_combine<kConsumerThreads>(tid, u, c0, c1, G, D, a.part_o, a.part_ml, a.out, a.arrive, abort_flag + 2);
         gt += piece_tiles;
     }
 }
@@ -604,8 +605,6 @@ cudaError_t launch_decode_scalar(const DecodeArgs& a, const DecodePlan& plan, cu
     ka.unit_len = a.unit_len;
     ka.n_extra = a.n_extra;
     ka.units = a.units;
-    ka.out = a.out;
-    ka.arrive = a.arrive;
     const bool pdl = a.programmatic;
     if (a.dtype == 0) {
         if (a.D == 128) return launch_scalar_groups<__nv_bfloat16, 128>(a.G, plan.geom, ka, plan.NC, pdl, stream);

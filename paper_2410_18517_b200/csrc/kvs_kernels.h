@@ -29,7 +29,6 @@ struct DecodeArgs {
     float* part_ml;       // [units + NC][G][2]  (max in log2 domain, sum)
     float* out;           // [B][Hq][D]
     int* status;          // device status word
-    int* arrive;          // [units] arrival counters, all zero: the split-K kernel combines; nullptr: combine kernel
     int n;                // rows cached per unit
     int row_stride;       // rows between units of a plane
     int units;            // B * Hkv

@@ -107,8 +107,6 @@ struct MmaKernelArgs {
     int G;          // q-heads per kv-head, 1..8
     const int* n_extra;  // graph replay: rows every slot has grown by since the launch was recorded, or nullptr
     int units;
-    float* out;          // final output, written here when `arrive` is set
-    int* arrive;         // per-unit arrival counters (combine inside this kernel), or nullptr
 };
 
 // G (q-heads per kv-head, 1..8) is a run-time argument: it only selects which rows of the padded
@@ -337,9 +335,6 @@ __global__ void __launch_bounds__(kMmaThreads, KVS_MMA_BLOCKS_PER_SM)
 
         // ---- end of piece: merge the four warps, one q-head at a time ----
         const long long pid = u + blockIdx.x;
-        // blocks that share this unit; a unit this block has to itself is finished here
-        const int c0 = cta_of_tile(u * a.tpu, a.T, NC), c1 = cta_of_tile((u + 1) * a.tpu - 1, a.T, NC);
-        const bool whole = a.arrive != nullptr && c0 == c1;
         float l = lsum;
         l += __shfl_xor_sync(0xffffffffu, l, 1);
         l += __shfl_xor_sync(0xffffffffu, l, 2);
@@ -369,10 +364,6 @@ __global__ void __launch_bounds__(kMmaThreads, KVS_MMA_BLOCKS_PER_SM)
                     acc = fmaf(w, scratch[j * (D + 2) + d], acc);
                     den = fmaf(w, scratch[j * (D + 2) + D + 1], den);
                 }
-                if (whole) {
-                    a.out[(u * G + g) * D + d] = acc / den;
-                    continue;
-                }
                 a.part_o[(pid * G + g) * D + d] = acc;
                 if (d == 0) {
                     a.part_ml[(pid * G + g) * 2] = M;
@@ -380,9 +371,6 @@ __global__ void __launch_bounds__(kMmaThreads, KVS_MMA_BLOCKS_PER_SM)
                 }
             }
         }
-        if (a.arrive != nullptr && !whole)
-            arrive_and_combine<kMmaConsumerThreads>(tid, u, c0, c1, G, D, a.part_o, a.part_ml, a.out, a.arrive,
-                                                    abort_flag + 2);
         gt += piece_tiles;
     }
 }
@@ -459,8 +447,6 @@ cudaError_t launch_decode_mma(const DecodeArgs& a, const DecodePlan& plan, const
     ka.G = a.G;
     ka.n_extra = a.n_extra;
     ka.units = a.units;
-    ka.out = a.out;
-    ka.arrive = a.arrive;
     if (a.G < 1 || a.G > 8) return cudaErrorInvalidValue;
     if (a.D == 128) return launch_one<128>(tm, ka, plan.NC, a.programmatic, stream);
     if (a.D == 64) return launch_one<64>(tm, ka, plan.NC, a.programmatic, stream);
