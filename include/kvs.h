@@ -82,17 +82,12 @@ typedef struct {
     uint64_t prefill_launches;    /* tensor-core prefill kernels launched                    */
     uint64_t evict_launches;      /* kvs_evict calls that launched                           */
     uint64_t search_launches;     /* kernels launched by kvs_layer_distances / kvs_mean_cosine */
-    uint64_t fused_appends;       /* kvs_decode_step calls whose append rode in the attention kernel */
 } kvs_stats_t;
 
 /* Tuning knobs for kvs_set_option.  Defaults are chosen by the library. */
 typedef enum {
     KVS_OPT_MAX_CTAS = 0,   /* upper bound on thread blocks of the split-K kernel; 0 = auto  */
-    KVS_OPT_KERNEL = 1,     /* 0 = auto, 1 = scalar-FMA path, 2 = grouped tensor-core path,
-                               3 = one-kernel cluster path whenever the call allows it (groups
-                               of 1, 2, 4, 8 q-heads; slots nothing was evicted from), else auto.
-                               Auto sends launches that stream at most 24 MiB to the cluster
-                               path.                                                           */
+    KVS_OPT_KERNEL = 1,     /* 0 = auto, 1 = scalar-FMA path, 2 = grouped tensor-core path   */
     KVS_OPT_EARLY_START = 2,/* 1 (default): kernels are launched so that they may start while
                                the previous kernel on the stream drains, and prefetch K/V rows
                                that nothing in flight writes; they wait for the previous kernel
@@ -169,30 +164,13 @@ kvs_status kvs_append(kvs_ctx* ctx, int32_t layer, const void* k, const void* v,
  * over all n cached rows j, no mask, G = n_q_heads / n_kv_heads.
  *   q:   device, [batch][n_q_heads][head_dim], storage type
  *   out: device, [batch][n_q_heads][head_dim], float32
- * Launches the split-K kernel and the combine kernel on `stream` (or, for small
- * launches, the single cluster kernel: see KVS_OPT_KERNEL); partial results go
- * through the bound workspace, so calls on one context must not overlap on the
- * GPU (use one stream, or order them).
+ * Launches the split-K kernel and the combine kernel on `stream`; partial
+ * results go through the bound workspace, so calls on one context must not
+ * overlap on the GPU (use one stream, or order them).
  * Errors: STATE before kvs_bind_memory or when the slot is empty; INVALID_ARG
  * for a bad layer, NULLs, batch < 1 or batch > the batch the slot was filled for. */
 kvs_status kvs_decode_attention(kvs_ctx* ctx, int32_t layer, const void* q, float* out,
                                 int32_t batch, void* stream);
-
-/* One decode step of one layer: kvs_append of one token (n_new = 1) followed by
- * kvs_decode_attention, with the same arguments, layouts, results and errors as those two
- * calls in that order (Section 3.2; on a layer whose cache is replaced k and v are not read and
- * may be NULL, and nothing is appended).
- *   q: device, [batch][n_q_heads][head_dim];  k, v: device, [batch][1][n_kv_heads][head_dim];
- *   out: device, float32 [batch][n_q_heads][head_dim]
- * Where latency rather than bandwidth bounds the call (see KVS_OPT_KERNEL) and k and v are
- * 16-byte aligned, the whole step is ONE kernel: a thread-block cluster per (sequence, kv-head)
- * splits the cached rows, the block that meets the new row takes it from k / v (and stores it
- * in the slot), and the pieces are merged through distributed shared memory.  Otherwise the
- * append kernel, the split-K kernel and the combine kernel are launched as by the two calls.
- * The cached bits and the output do not depend on which way was taken beyond the summation
- * order of the output (inside the tolerance).                                                  */
-kvs_status kvs_decode_step(kvs_ctx* ctx, int32_t layer, const void* q, const void* k, const void* v,
-                           float* out, int32_t batch, void* stream);
 
 /* Prefill attention of one layer (Section 3.2: the strategy is applied to the prefill pass
  * as it is to generation).  The n_q queries per head are the newest n_q positions of the cache
@@ -269,8 +247,7 @@ kvs_status kvs_mean_cosine(kvs_ctx* ctx, const void* a, const void* b, int32_t n
  *     not counted), call kvs_replay_commit(ctx, times_run, stream): the host lengths catch up
  *     (times_run - 1 more rows) and the counter is cleared on `stream`.  Make no eager call on
  *     the context between the first replay and the commit.
- *   - One-token decode steps only; every computing layer must append exactly once per step
- *     (kvs_append, or kvs_decode_step).
+ *   - One-token decode steps only; every computing layer must append exactly once per step.
  *   - A replay that would pass max_seq appends nothing for that layer and sets the device status
  *     word to KVS_ERR_CAPACITY; kvs_replay_commit returns CAPACITY instead of advancing.
  * Errors: STATE unless bound and KVS_OPT_REPLAY is 1; INVALID_ARG for times_run < 1.            */
@@ -344,8 +321,8 @@ kvs_status kvs_stats(const kvs_ctx* ctx, kvs_stats_t* stats);
  * out and the kernel returned early (its output is then undefined).             */
 kvs_status kvs_last_device_status(kvs_ctx* ctx, int32_t* device_status);
 kvs_status kvs_set_option(kvs_ctx* ctx, int32_t option, int32_t value);
-/* How the last kvs_decode_attention / kvs_decode_step call was decomposed: thread blocks
- * launched, rows per tile, and 1, 2 or 3 for the scalar / tensor-core / cluster kernel.  */
+/* How the last kvs_decode_attention call was decomposed: thread blocks launched,
+ * rows per tile, and 1 or 2 for the scalar / tensor-core kernel.                */
 kvs_status kvs_last_launch(const kvs_ctx* ctx, int32_t* ctas, int32_t* tile_rows, int32_t* kernel);
 const char* kvs_status_string(kvs_status s);
 

@@ -8,8 +8,8 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libkvs.so")
-SOURCES = ["kvs_api.cu", "kvs_kernels.cu", "kvs_mma.cu", "kvs_prefill.cu", "kvs_search.cu", "kvs_cluster.cu"]
-HEADERS = ["kvs_device.cuh", "kvs_kernels.h", "kvs_scalar.cuh", os.path.join("..", "..", "include", "kvs.h")]
+SOURCES = ["kvs_api.cu", "kvs_kernels.cu", "kvs_mma.cu", "kvs_prefill.cu", "kvs_search.cu"]
+HEADERS = ["kvs_device.cuh", "kvs_kernels.h", os.path.join("..", "..", "include", "kvs.h")]
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a",

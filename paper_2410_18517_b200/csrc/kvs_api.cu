@@ -71,7 +71,6 @@ struct kvs_ctx {
     int opt_pdl = 1;
     int opt_host_chunks = 4;
     int opt_replay = 0;   // launches carry the device-side growth counter (for CUDA-graph replay)
-    int max_cluster = 1;  // largest thread-block cluster the device places for the one-kernel decode path
     // The split-K kernels read the growth counter before their wait.  That is safe because the
     // first launch after anything wrote the counter never starts early (full dependency): it and
     // everything after it then begin with the write complete.
@@ -167,7 +166,6 @@ void layout_workspace(kvs_ctx* c) {
 
 std::once_flag g_init_flag[64];
 cudaError_t g_init_err[64];
-int g_max_cluster[64];
 
 cudaError_t init_device_once(int device) {
     if (device < 0 || device >= 64) return cudaErrorInvalidDevice;
@@ -175,8 +173,6 @@ cudaError_t init_device_once(int device) {
         g_init_err[device] = kvs::init_kernels();
         if (g_init_err[device] == cudaSuccess) g_init_err[device] = kvs::init_mma_kernels();
         if (g_init_err[device] == cudaSuccess) g_init_err[device] = kvs::init_prefill_kernels();
-        g_max_cluster[device] = 1;
-        if (g_init_err[device] == cudaSuccess) g_init_err[device] = kvs::init_cluster_kernels(&g_max_cluster[device]);
     });
     return g_init_err[device];
 }
@@ -256,35 +252,20 @@ struct AttentionScratch {
     bool programmatic;   // early-start launches (only when the call follows this context's own kernels)
 };
 
-// Launches that stream less than this are bound by latency, not bandwidth: they go to the
-// one-kernel cluster path (measured cross-over on B200).
-constexpr long long kClusterMaxBytes = 24ll << 20;
-
-// Which kernel serves the context's shape and how the call is cut into work.  Small launches of an
-// un-evicted slot take the cluster kernel (append, attention and merge in one launch); otherwise
-// bf16 groups of three or more q-heads per kv-head are a real (if thin) contraction and go to the
-// tensor cores, the rest to the scalar kernel.  Returns 1, 2 or 3 (= plan->kernel).
-int choose_plan(const kvs_ctx* c, int slot, int units, int n, kvs::DecodePlan* plan) {
-    const bool small = 2ll * units * n * c->row_bytes <= kClusterMaxBytes;
-    if (!c->ragged[slot] && (c->opt_kernel == 3 || (c->opt_kernel == 0 && small)) &&
-        kvs::plan_decode_cluster(units, n, c->G, c->cfg.head_dim, c->cfg.dtype, c->sm_count, c->max_cluster, plan))
-        return 3;
-    const bool pow2_group = c->G == 1 || c->G == 2 || c->G == 4 || c->G == 8;
-    const bool use_mma = c->have_tensor_map && (c->opt_kernel == 2 || !pow2_group || (c->opt_kernel != 1 && c->G >= 3));
+// Which kernel serves the context's shape and how the call is cut into work.  bf16 groups of three
+// or more q-heads per kv-head are a real (if thin) contraction and go to the tensor cores.
+bool choose_plan(const kvs_ctx* c, int units, int n, kvs::DecodePlan* plan) {
+    const bool use_mma = c->have_tensor_map && (c->opt_kernel == 2 || (c->opt_kernel == 0 && c->G >= 3));
     if (use_mma)
         kvs::plan_decode_mma(units, n, c->cfg.head_dim, c->sm_count, c->opt_max_ctas, plan);
     else
         kvs::plan_decode_scalar(units, n, c->G, c->cfg.head_dim, c->cfg.dtype, c->sm_count, c->opt_max_ctas, plan);
-    return plan->kernel;
+    return use_mma;
 }
 
-// The kernels of one layer's attention with the given plan and scratch: split-K kernel + combine
-// kernel, or the cluster kernel alone.  With k_new / v_new (cluster plan only) the launch also
-// appends that one row per unit: the slot's length must already count it, `old_len` is the
-// length before.
+// Split-K kernel + combine kernel of one layer, with the given plan and scratch.
 kvs_status run_attention(kvs_ctx* c, int slot, const void* q, float* out, int batch, const kvs::DecodePlan& plan,
-                         const AttentionScratch& scratch, cudaStream_t st, const void* k_new = nullptr,
-                         const void* v_new = nullptr) {
+                         bool use_mma, const AttentionScratch& scratch, cudaStream_t st) {
     kvs::DecodeArgs a;
     a.q = q;
     a.kplane = c->pool + (size_t)(2 * slot) * c->plane_bytes;
@@ -304,27 +285,20 @@ kvs_status run_attention(kvs_ctx* c, int slot, const void* q, float* out, int ba
     a.safe_rows = scratch.programmatic ? safe_rows_of(c, slot) : 0;
     a.unit_len = c->ragged[slot] ? unit_len_dev(c, slot) : nullptr;
     a.n_extra = replay_counter(c);
-    if (plan.kernel == 3) {
-        if (k_new) a.safe_rows = std::min(a.safe_rows, a.n - 1);
-        c->seq += 1;
-        c->last_splitk_seq = c->seq;
-        if (kvs::launch_decode_cluster(a, plan, k_new, v_new, c->cfg.max_seq, st) != cudaSuccess) return KVS_ERR_CUDA;
+    c->seq += 2;                       // split-K kernel, then combine
+    c->last_splitk_seq = c->seq - 1;
+    if (use_mma) {
+        const long long plane_rows = (long long)c->cfg.max_batch * c->cfg.n_kv_heads * c->row_stride;
+        if (kvs::launch_decode_mma(a, plan, c->tensor_map, plane_rows * (2 * slot), plane_rows * (2 * slot + 1), st) !=
+            cudaSuccess)
+            return KVS_ERR_CUDA;
     } else {
-        c->seq += 2;                       // split-K kernel, then combine
-        c->last_splitk_seq = c->seq - 1;
-        if (plan.kernel == 2) {
-            const long long plane_rows = (long long)c->cfg.max_batch * c->cfg.n_kv_heads * c->row_stride;
-            if (kvs::launch_decode_mma(a, plan, c->tensor_map, plane_rows * (2 * slot), plane_rows * (2 * slot + 1), st) !=
-                cudaSuccess)
-                return KVS_ERR_CUDA;
-        } else {
-            if (kvs::launch_decode_scalar(a, plan, st) != cudaSuccess) return KVS_ERR_CUDA;
-        }
-        if (kvs::launch_combine(a, plan, st) != cudaSuccess) return KVS_ERR_CUDA;
-        c->stats.combine_launches += 1;
+        if (kvs::launch_decode_scalar(a, plan, st) != cudaSuccess) return KVS_ERR_CUDA;
     }
+    if (kvs::launch_combine(a, plan, st) != cudaSuccess) return KVS_ERR_CUDA;
     c->last_plan = plan;
     c->stats.attention_launches += 1;
+    c->stats.combine_launches += 1;
     if (c->ragged[slot]) {
         unsigned long long rows = 0;
         for (int u = 0; u < a.units; ++u) rows += c->unit_len_host[slot][u];
@@ -335,39 +309,14 @@ kvs_status run_attention(kvs_ctx* c, int slot, const void* q, float* out, int ba
     return KVS_OK;
 }
 
-AttentionScratch workspace_scratch(kvs_ctx* c) {
-    return {reinterpret_cast<float*>(c->ws + c->off_part_o), reinterpret_cast<float*>(c->ws + c->off_part_ml),
-            reinterpret_cast<int*>(c->ws + c->off_status), take_early_start(c)};
-}
-
 kvs_status do_attention(kvs_ctx* c, int layer, const void* q, float* out, int batch, cudaStream_t st) {
     const int slot = c->slot_of_layer[layer];
     kvs::DecodePlan plan;
-    choose_plan(c, slot, batch * c->cfg.n_kv_heads, c->slot_len[slot], &plan);
-    return run_attention(c, slot, q, out, batch, plan, workspace_scratch(c), st);
-}
-
-// Append of one row per unit and attention in one cluster-kernel launch (the caller has checked
-// the arguments and that the plan is a cluster plan for the length after the append).
-kvs_status do_fused_step(kvs_ctx* c, int layer, const void* q, const void* k, const void* v, float* out, int batch,
-                         const kvs::DecodePlan& plan, cudaStream_t st) {
-    const int slot = c->slot_of_layer[layer];
-    const AttentionScratch scratch = workspace_scratch(c);
-    const int old_len = c->slot_len[slot];
-    c->slot_len[slot] = old_len + 1;
-    c->cur_batch = batch;
-    // safe_rows_of must still see the appends before this one while run_attention computes it
-    const kvs_status s = run_attention(c, slot, q, out, batch, plan, scratch, st, k, v);
-    if (s != KVS_OK) {
-        c->slot_len[slot] = old_len;
-        return s;
-    }
-    c->app_seq_prev[slot] = c->app_seq_latest[slot];
-    c->app_seq_latest[slot] = c->seq;          // the launch that appended is the attention launch itself
-    c->app_start_latest[slot] = old_len;
-    c->stats.fused_appends += 1;
-    c->stats.kv_bytes_appended += 2ull * batch * c->cfg.n_kv_heads * c->row_bytes;
-    return KVS_OK;
+    const bool use_mma = choose_plan(c, batch * c->cfg.n_kv_heads, c->slot_len[slot], &plan);
+    const AttentionScratch scratch = {reinterpret_cast<float*>(c->ws + c->off_part_o),
+                                      reinterpret_cast<float*>(c->ws + c->off_part_ml),
+                                      reinterpret_cast<int*>(c->ws + c->off_status), take_early_start(c)};
+    return run_attention(c, slot, q, out, batch, plan, use_mma, scratch, st);
 }
 
 }  // namespace
@@ -473,7 +422,6 @@ kvs_status kvs_bind_memory(kvs_ctx* ctx, void* pool, size_t pool_bytes, void* wo
         ctx->have_tensor_map = true;
     }
     ctx->sm_count = sms;
-    ctx->max_cluster = g_max_cluster[ctx->cfg.device];
     {
         int l2 = 0;
         if (cudaDeviceGetAttribute(&l2, cudaDevAttrL2CacheSize, ctx->cfg.device) == cudaSuccess && l2 > 0) ctx->l2_bytes = l2;
@@ -519,33 +467,6 @@ kvs_status kvs_decode_attention(kvs_ctx* ctx, int32_t layer, const void* q, floa
     DeviceGuard guard(ctx->cfg.device);
     if (!guard.ok) return KVS_ERR_CUDA;
     return do_attention(ctx, layer, q, out, batch, static_cast<cudaStream_t>(stream));
-}
-
-kvs_status kvs_decode_step(kvs_ctx* ctx, int32_t layer, const void* q, const void* k, const void* v, float* out,
-                           int32_t batch, void* stream) {
-    bool sharing = false;
-    kvs_status s = check_append(ctx, layer, k, v, batch, 1, &sharing);
-    if (s != KVS_OK) return s;
-    if (!q || !out) return KVS_ERR_INVALID_ARG;
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (sharing) {
-        s = check_attention(ctx, layer, q, out, batch);
-        if (s != KVS_OK) return s;
-        DeviceGuard guard(ctx->cfg.device);
-        if (!guard.ok) return KVS_ERR_CUDA;
-        ctx->stats.append_skipped += 1;
-        return do_attention(ctx, layer, q, out, batch, st);
-    }
-    DeviceGuard guard(ctx->cfg.device);
-    if (!guard.ok) return KVS_ERR_CUDA;
-    const int slot = ctx->slot_of_layer[layer];
-    kvs::DecodePlan plan;
-    const bool aligned = ((uintptr_t)k % 16) == 0 && ((uintptr_t)v % 16) == 0;
-    if (aligned && choose_plan(ctx, slot, batch * ctx->cfg.n_kv_heads, ctx->slot_len[slot] + 1, &plan) == 3)
-        return do_fused_step(ctx, layer, q, k, v, out, batch, plan, st);
-    s = do_append(ctx, layer, k, v, batch, 1, st);
-    if (s != KVS_OK) return s;
-    return do_attention(ctx, layer, q, out, batch, st);
 }
 
 kvs_status kvs_prefill_attention(kvs_ctx* ctx, int32_t layer, const void* q, float* out, int32_t batch, int32_t n_q,
@@ -881,10 +802,8 @@ kvs_status kvs_set_option(kvs_ctx* ctx, int32_t option, int32_t value) {
             ctx->opt_host_chunks = value;
             return KVS_OK;
         case KVS_OPT_KERNEL:
-            if (value < 0 || value > 3) return KVS_ERR_INVALID_ARG;
+            if (value < 0 || value > 2) return KVS_ERR_INVALID_ARG;
             if (value == 2 && ctx->cfg.dtype != KVS_BF16) return KVS_ERR_INVALID_ARG;  // tensor-core path is bf16 only
-            if (value == 3 && ctx->G != 1 && ctx->G != 2 && ctx->G != 4 && ctx->G != 8)
-                return KVS_ERR_INVALID_ARG;                                          // cluster path: groups of 1, 2, 4, 8
             if (value == 1 && ctx->G != 1 && ctx->G != 2 && ctx->G != 4 && ctx->G != 8)
                 return KVS_ERR_INVALID_ARG;                                          // scalar path: groups of 1, 2, 4, 8
             ctx->opt_kernel = value;
@@ -972,9 +891,8 @@ kvs_status kvs_decode_attention_static(kvs_ctx* ctx, int32_t layer, const void* 
     const int units = batch * c->cfg.n_kv_heads;
     const int D = c->cfg.head_dim;
     kvs::DecodePlan plan;
-    choose_plan(c, slot, units, c->slot_len[slot], &plan);
-    // one partial (o[D], m, l) per (piece, q-head); pieces are indexed unit + block (the cluster
-    // kernel needs none of this scratch, the size check still uses the general formula)
+    const bool use_mma = choose_plan(c, units, c->slot_len[slot], &plan);
+    // one partial (o[D], m, l) per (piece, q-head); pieces are indexed unit + block
     const size_t pieces = (size_t)units + plan.NC;
     const size_t part_o_bytes = align_up(pieces * c->G * D * sizeof(float), kAlign);
     const size_t part_ml_bytes = align_up(pieces * c->G * 2 * sizeof(float), kAlign);
@@ -993,7 +911,7 @@ kvs_status kvs_decode_attention_static(kvs_ctx* ctx, int32_t layer, const void* 
                                       reinterpret_cast<float*>(base + kStaticStatusBytes + part_o_bytes), status_word,
                                       false};
     c->counter_written = false;
-    return run_attention(c, slot, q, out, batch, plan, scratch, st);
+    return run_attention(c, slot, q, out, batch, plan, use_mma, scratch, st);
 }
 
 }  // extern "C"

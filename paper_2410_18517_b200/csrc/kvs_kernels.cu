@@ -5,7 +5,6 @@
 //   read_roof_kernel      the same ring with no arithmetic (bandwidth ceiling)
 #include "kvs_device.cuh"
 #include "kvs_kernels.h"
-#include "kvs_scalar.cuh"
 
 #include <algorithm>
 
@@ -206,6 +205,39 @@ struct ScalarShape {
     static_assert(TN % NG == 0, "tile rows must divide evenly among lane groups");
 };
 
+template <int N>
+struct Log2 {
+    static constexpr int value = 1 + Log2<N / 2>::value;
+};
+template <>
+struct Log2<1> {
+    static constexpr int value = 0;
+};
+
+// Sum NV per-lane partial sums over a group of lanes by recursive halving: after the
+// call, the lane whose index within the group has top bits i holds the full sum of
+// value i.  OFF is the current xor distance (starts at lanes-per-group / 2).
+template <int NV, int OFF>
+__device__ __forceinline__ float reduce_transpose(float (&v)[NV], int lig) {
+    if constexpr (NV == 1) {
+        float x = v[0];
+#pragma unroll
+        for (int o = OFF; o >= 1; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+        return x;
+    } else {
+        constexpr int H = NV / 2;
+        const bool upper = (lig & OFF) != 0;
+        float w[H];
+#pragma unroll
+        for (int k = 0; k < H; ++k) {
+            const float send = upper ? v[k] : v[k + H];
+            const float keep = upper ? v[k + H] : v[k];
+            w[k] = keep + __shfl_xor_sync(0xffffffffu, send, OFF);
+        }
+        return reduce_transpose<H, OFF / 2>(w, lig);
+    }
+}
+
 struct ScalarKernelArgs {
     const char* q;
     const char* kplane;
@@ -238,7 +270,8 @@ __global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G, GEOM>::MI
         a.T = (long long)a.units * a.tpu;
     }
     constexpr int kTile = S::TILE;
-    constexpr int RB = S::RB, LPR = S::LPR, NG = S::NG, TN = S::TN, STAGES = S::STAGES;
+    constexpr int RB = S::RB, LPR = S::LPR, EPL = S::EPL, NG = S::NG, TN = S::TN, R = S::R, STAGES = S::STAGES;
+    constexpr int SH = Log2<LPR>::value - Log2<R>::value;  // lane-in-group >> SH = row index held after the reduction
 
     extern __shared__ __align__(128) unsigned char smem[];
     unsigned char* stage_base = smem;
@@ -327,9 +360,9 @@ __global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G, GEOM>::MI
     // ---------------------------------- consumers ----------------------------------
     pdl_wait();               // partial results of the previous call may still be read until here
     pdl_launch_dependents();
-    using Math = ScalarMath<T, D, G, NG, TN>;
     const int lig = lane & (LPR - 1);                 // lane within its row group
     const int grp = warp * S::GPW + lane / LPR;       // row group within the block
+    const int my_i = lig >> SH;                       // row (of the R) whose score this lane ends up holding
 
     int it = 0;
     long long gt = t0;
@@ -339,30 +372,127 @@ __global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G, GEOM>::MI
         const int piece_tiles = (int)min((long long)(a.tpu - ti0), t1 - gt);
         const int n_u = a.unit_len ? a.unit_len[u] : a.n;
 
-        typename Math::State st_;
-        Math::reset(st_);
+        float qf[G][EPL];
+        float m[G], lsum[G], acc[G][EPL];
+#pragma unroll
+        for (int g = 0; g < G; ++g) {
+            m[g] = -1.0e30f;
+            lsum[g] = 0.f;
+#pragma unroll
+            for (int e = 0; e < EPL; ++e) acc[g][e] = 0.f;
+        }
 
         for (int k = 0; k < piece_tiles; ++k, ++it) {
             const int st = it % STAGES;
             if (!mbar_wait_bounded(&full_bar[st], (it / STAGES) & 1, abort_flag, a.status)) return;
             const unsigned char* ks = stage_base + st * S::STAGE_BYTES;
             const unsigned char* vs = ks + kTile;
-            if (k == 0) Math::load_q(st_, vs + kTile, lig, a.scale_log2);
+            if (k == 0) {
+                const unsigned char* qs = vs + kTile;
+#pragma unroll
+                for (int g = 0; g < G; ++g) {
+                    const uint4 raw = *reinterpret_cast<const uint4*>(qs + g * RB + lig * 16);
+                    Unpack<T>::run(raw, qf[g]);
+#pragma unroll
+                    for (int e = 0; e < EPL; ++e) qf[g][e] *= a.scale_log2;
+                }
+            }
             const int valid = min(TN, n_u - (ti0 + k) * TN);   // <= 0 for tiles past a ragged unit's end
-            if (valid > 0) Math::tile(st_, ks, vs, valid, lig, grp);
+            if (valid <= 0) {
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&empty_bar[st]);
+                continue;
+            }
+
+            // scores: partial dot products of this lane's 16-byte chunk
+            float s[G][R];
+#pragma unroll
+            for (int i = 0; i < R; ++i) {
+                const int row = grp + NG * i;
+                const uint4 raw = *reinterpret_cast<const uint4*>(ks + row * RB + lig * 16);
+                float kf[EPL];
+                Unpack<T>::run(raw, kf);
+#pragma unroll
+                for (int g = 0; g < G; ++g) {
+                    float d = 0.f;
+#pragma unroll
+                    for (int e = 0; e < EPL; ++e) d = fmaf(qf[g][e], kf[e], d);
+                    s[g][i] = d;
+                }
+            }
+            // online softmax per q-head, local to the lane group
+            float p[G][R];
+            const bool mine_valid = (grp + NG * my_i) < valid;
+#pragma unroll
+            for (int g = 0; g < G; ++g) {
+                float sv = reduce_transpose<R, LPR / 2>(s[g], lig);
+                sv = mine_valid ? sv : -INFINITY;
+                float tmax = sv;
+#pragma unroll
+                for (int o = LPR / 2; o >= LPR / R; o >>= 1) tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, o));
+                const float m_new = fmaxf(m[g], tmax);
+                const float alpha = fast_exp2(m[g] - m_new);
+                const float pv = fast_exp2(sv - m_new);
+                m[g] = m_new;
+                lsum[g] = lsum[g] * alpha + pv;
+#pragma unroll
+                for (int e = 0; e < EPL; ++e) acc[g][e] *= alpha;
+#pragma unroll
+                for (int i = 0; i < R; ++i) p[g][i] = __shfl_sync(0xffffffffu, pv, i << SH, LPR);
+            }
+            // weighted sum of value rows
+#pragma unroll
+            for (int i = 0; i < R; ++i) {
+                const int row = grp + NG * i;
+                if (row < valid) {
+                    const uint4 raw = *reinterpret_cast<const uint4*>(vs + row * RB + lig * 16);
+                    float vf[EPL];
+                    Unpack<T>::run(raw, vf);
+#pragma unroll
+                    for (int g = 0; g < G; ++g)
+#pragma unroll
+                        for (int e = 0; e < EPL; ++e) acc[g][e] = fmaf(p[g][i], vf[e], acc[g][e]);
+                }
+            }
             __syncwarp();
             if (lane == 0) mbar_arrive(&empty_bar[st]);
         }
 
         // ---- end of piece: merge the NG lane groups, one q-head at a time ----
         const long long pid = u + blockIdx.x;
-        Math::template merge<kConsumerThreads>(st_, scratch, tid, lig, grp, [&](int g, int d, float o, float M, float den) {
-            a.part_o[(pid * G + g) * D + d] = o;
-            if (d == 0) {
-                a.part_ml[(pid * G + g) * 2] = M;
-                a.part_ml[(pid * G + g) * 2 + 1] = den;
+#pragma unroll
+        for (int g = 0; g < G; ++g) {
+            // lanes with equal top bits hold duplicates of lsum; add across the R distinct ones
+            float l = lsum[g];
+#pragma unroll
+            for (int o = LPR / 2; o >= LPR / R; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
+            named_bar_sync(1, kConsumerThreads);  // scratch free again
+            float* row = scratch + grp * (D + 2);
+#pragma unroll
+            for (int e = 0; e < EPL; ++e) row[lig * EPL + e] = acc[g][e];
+            if (lig == 0) {
+                row[D] = m[g];
+                row[D + 1] = l;
             }
-        });
+            named_bar_sync(1, kConsumerThreads);
+            for (int d = tid; d < D; d += kConsumerThreads) {
+                float M = -1.0e30f;
+#pragma unroll
+                for (int j = 0; j < NG; ++j) M = fmaxf(M, scratch[j * (D + 2) + D]);
+                float o = 0.f, den = 0.f;
+#pragma unroll
+                for (int j = 0; j < NG; ++j) {
+                    const float w = fast_exp2(scratch[j * (D + 2) + D] - M);
+                    o = fmaf(w, scratch[j * (D + 2) + d], o);
+                    den = fmaf(w, scratch[j * (D + 2) + D + 1], den);
+                }
+                a.part_o[(pid * G + g) * D + d] = o;
+                if (d == 0) {
+                    a.part_ml[(pid * G + g) * 2] = M;
+                    a.part_ml[(pid * G + g) * 2 + 1] = den;
+                }
+            }
+        }
         gt += piece_tiles;
     }
 }

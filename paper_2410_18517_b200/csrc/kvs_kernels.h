@@ -17,9 +17,8 @@ struct DecodePlan {
     int tpu;         // tiles per unit = ceil(n / tile_rows)
     long long T;     // total tiles = units * tpu
     int NC;          // thread blocks launched
-    int kernel;      // 1 = scalar, 2 = tensor-core, 3 = cluster (one kernel per step)
-    int geom;        // scalar kernel: 0 = default ring geometry, 1 = the one for multi-gigabyte launches;
-                     // cluster kernel: thread blocks per unit
+    int kernel;      // 1 = scalar, 2 = tensor-core
+    int geom;        // scalar kernel: 0 = default ring geometry, 1 = the one for multi-gigabyte launches
 };
 
 struct DecodeArgs {
@@ -81,17 +80,6 @@ cudaError_t launch_layer_distances(const void* pool, long long plane_bytes, cons
                                    int sm_count, cudaStream_t stream);
 cudaError_t launch_mean_cosine(const void* a, const void* b, int S, long long dim, int dtype, double* partial,
                                float* out, int sm_count, cudaStream_t stream);
-
-// One-kernel decode step for latency-bound launches (see kvs_cluster.cu): a thread-block cluster
-// per (sequence, kv-head) unit; the pieces are merged through distributed shared memory, and the
-// append of the step's new row can ride along (k_new / v_new: [B][1][Hkv][D], or nullptr).
-constexpr int kMaxClusterSize = 16;
-cudaError_t init_cluster_kernels(int* max_cluster_size);
-// Fills `plan` (kernel = 3, geom = blocks per unit); false if the shape has no cluster kernel.
-bool plan_decode_cluster(int units, int n, int G, int D, int dtype, int sm_count, int max_cluster_size,
-                         DecodePlan* plan);
-cudaError_t launch_decode_cluster(const DecodeArgs& a, const DecodePlan& plan, const void* k_new, const void* v_new,
-                                  int capacity, cudaStream_t stream);
 
 cudaError_t launch_append(const void* k, const void* v, void* kplane, void* vplane, int B, int n_new, int Hkv,
                           int row_bytes, int row_stride, int len0, const int* unit_len, const int* n_extra, int capacity, int* status,

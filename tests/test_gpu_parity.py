@@ -41,8 +41,7 @@ def test_tiny_config_every_output_and_every_cached_bit():
     assert cache.num_slots() == 3
     st = cache.stats()
     assert st["append_launches"] == 3 + 9 * 3 and st["append_skipped"] == 1 + 9
-    assert st["attention_launches"] == 9 * 4
-    assert st["combine_launches"] == 0 and cache.last_launch()["kernel"] == 3   # small launches: the cluster kernel
+    assert st["attention_launches"] == 9 * 4 and st["combine_launches"] == 9 * 4
     assert [cache.seq_len(l) for l in range(4)] == [137] * 4
     assert worst[0] < 1e-4       # fp32 storage: far inside the bf16 tolerance
 
@@ -58,17 +57,12 @@ SHAPES = [
 
 @pytest.mark.parametrize("dtype,D,Hq,Hkv", SHAPES)
 @pytest.mark.parametrize("context", [0, 63, 64, 65, 200, 1031])
-@pytest.mark.parametrize("path", ["auto", "persistent"])
-def test_shapes_and_ragged_tails(dtype, D, Hq, Hkv, context, path):
-    """Context lengths around the 32/64/128-row tile edges, 3 decode steps, chain strategy; on the
-    kernel the library picks for launches this small (the cluster kernel) and on the persistent
-    split-K kernel it picks for large ones (tensor-core for bf16 groups of 3 or more, else scalar)."""
+def test_shapes_and_ragged_tails(dtype, D, Hq, Hkv, context):
+    """Context lengths around the 32/64/128-row tile edges, 3 decode steps, chain strategy."""
     w = si.Workload(f"s_{dtype}_{D}_{Hq}_{Hkv}_{context}", L=4, Hq=Hq, Hkv=Hkv, D=D, B=3, context=context,
                     dtype=dtype, n_shared=0, map_seed=0, steps=3, fixed_map=(0, 0, 1, 2))
-    big = 2 if (dtype == "bf16" and Hq // Hkv >= 3) else 1
-    cache, orc, _ = run_small(w, steps=3, options=[] if path == "auto" else [(KVS_OPT_KERNEL, big)])
+    cache, orc, _ = run_small(w, steps=3)
     assert cache.num_slots() == 1
-    assert cache.last_launch()["kernel"] == (3 if path == "auto" else big)
 
 
 @pytest.mark.parametrize("kernel", [1, 2])
@@ -96,17 +90,13 @@ def test_group_sizes_that_are_not_powers_of_two(G, D):
 
 
 def test_auto_kernel_choice():
-    """Launches that stream more than 24 MiB: groups of four or more bf16 q-heads go to the tensor
-    cores, fp32 storage never does.  Smaller launches go to the cluster kernel."""
+    """Groups of four or more bf16 q-heads go to the tensor cores; fp32 storage never does."""
     for Hq, Hkv, dtype, want in [(4, 4, "bf16", 1), (4, 2, "bf16", 1), (8, 2, "bf16", 2), (8, 1, "bf16", 2),
                                  (8, 2, "f32", 1)]:
-        w = si.Workload(f"auto_{Hq}_{Hkv}_{dtype}", L=1, Hq=Hq, Hkv=Hkv, D=128, B=1, context=60000, dtype=dtype,
+        w = si.Workload(f"auto_{Hq}_{Hkv}_{dtype}", L=1, Hq=Hq, Hkv=Hkv, D=128, B=1, context=100, dtype=dtype,
                         n_shared=0, map_seed=0, steps=1)
         cache, _, _ = run_small(w, steps=1)
         assert cache.last_launch()["kernel"] == want
-        small = si.Workload(f"auto_small_{Hq}_{Hkv}_{dtype}", L=1, Hq=Hq, Hkv=Hkv, D=128, B=1, context=100, dtype=dtype,
-                            n_shared=0, map_seed=0, steps=1)
-        assert run_small(small, steps=1)[0].last_launch()["kernel"] == 3
     with pytest.raises(KvsError):
         cache.set_option(KVS_OPT_KERNEL, 2)          # the last cache is fp32
 
@@ -124,7 +114,7 @@ def test_any_split_of_the_tile_line_gives_the_same_answer(max_ctas):
     """The tile line of all units is cut at arbitrary places; results must not depend on it."""
     w = si.Workload(f"split_{max_ctas}", L=2, Hq=4, Hkv=4, D=128, B=2, context=1500, dtype="bf16",
                     n_shared=1, map_seed=0, steps=2, fixed_map=(0, 0))
-    cache, _, _ = run_small(w, steps=2, options=[(KVS_OPT_MAX_CTAS, max_ctas), (KVS_OPT_KERNEL, 1)])
+    cache, _, _ = run_small(w, steps=2, options=[(KVS_OPT_MAX_CTAS, max_ctas)])
     if max_ctas:
         assert cache.last_launch()["ctas"] == max_ctas
 

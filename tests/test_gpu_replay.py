@@ -22,8 +22,7 @@ def _built():
 
 @pytest.mark.parametrize("Hq,Hkv,dtype,context,evict", [(4, 4, "bf16", 300, False), (8, 2, "bf16", 127, False),
                                                          (4, 2, "f32", 60, False), (8, 2, "bf16", 200, True)])
-@pytest.mark.parametrize("use_step", [False, True])
-def test_graph_replay_is_the_next_step_every_time(Hq, Hkv, dtype, context, evict, use_step):
+def test_graph_replay_is_the_next_step_every_time(Hq, Hkv, dtype, context, evict):
     sm = [0, 1, 2, 1]
     L, D, B, replays = 4, 128, 2, 6
     w = si.Workload(f"replay_{Hq}_{Hkv}_{dtype}", L=L, Hq=Hq, Hkv=Hkv, D=D, B=B, context=context, dtype=dtype,
@@ -60,10 +59,6 @@ def test_graph_replay_is_the_next_step_every_time(Hq, Hkv, dtype, context, evict
 
     def one_step():
         for l in range(L):
-            if use_step:                         # kvs_decode_step: one kernel per layer where the slot is not ragged
-                own = sm[l] == l
-                cache.decode_step(l, qb[l], kbuf[l] if own else None, vbuf[l] if own else None, ob[l])
-                continue
             if sm[l] == l:
                 cache.append(l, kbuf[l], vbuf[l])
             else:
