@@ -501,10 +501,16 @@ __global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G, GEOM>::MI
 // K3: combine.  One block per (unit, q-head), D threads; out = sum_c w_c o_c / sum_c w_c l_c
 // with w_c = 2^(m_c - M), M = max_c m_c over the pieces c of the unit, always summed in
 // piece order so that the result does not depend on which block finished first.
+// The (m, l) pairs of all pieces are fetched first, one piece per lane (independent loads, one
+// round trip to L2), the weights go through shared memory, and the loop over the pieces'
+// output vectors keeps eight loads in flight: with the pieces read one after the other this
+// kernel was the slowest of a small decode step.
 // --------------------------------------------------------------------------------------
 __global__ void decode_combine_kernel(const float* __restrict__ part_o, const float* __restrict__ part_ml,
                                       float* __restrict__ out, int G, int D, int tpu, long long T, int NC,
                                       const int* __restrict__ n_extra, int n, int tile_rows, int units) {
+    __shared__ float wsm[kMaxCtas], lsm[kMaxCtas];
+    __shared__ float msm[4];
     pdl_launch_dependents();
     pdl_wait();
     if (n_extra) {   // replayed launch: recompute the tile line from the grown length
@@ -514,17 +520,32 @@ __global__ void decode_combine_kernel(const float* __restrict__ part_o, const fl
     const long long u = blockIdx.x / G;
     const int g = blockIdx.x % G;
     const int c0 = cta_of_tile(u * tpu, T, NC);
-    const int c1 = cta_of_tile((u + 1) * tpu - 1, T, NC);
-    const int d = threadIdx.x;
-    float M = -1.0e30f;
-    for (int c = c0; c <= c1; ++c) M = fmaxf(M, part_ml[((u + c) * G + g) * 2]);
+    const int np = cta_of_tile((u + 1) * tpu - 1, T, NC) - c0 + 1;       // pieces of this unit
+    const int d = threadIdx.x, lane = d & 31, warp = d >> 5;
+    const float2* ml = reinterpret_cast<const float2*>(part_ml) + (u + c0) * G + g;   // piece c: ml[c * G]
+    // every warp takes a share of the pieces: maxima and sums to shared memory
+    float mx = -1.0e30f;
+    for (int c = d; c < np; c += blockDim.x) {
+        const float2 v = ml[(long long)c * G];
+        wsm[c] = v.x;
+        lsm[c] = v.y;
+        mx = fmaxf(mx, v.x);
+    }
+#pragma unroll
+    for (int o = 16; o >= 1; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    if (lane == 0) msm[warp] = mx;
+    __syncthreads();
+    float M = msm[0];
+    for (int w = 1; w < (int)(blockDim.x >> 5); ++w) M = fmaxf(M, msm[w]);
+    for (int c = d; c < np; c += blockDim.x) wsm[c] = fast_exp2(wsm[c] - M);
+    __syncthreads();
     float o = 0.f, den = 0.f;
-#pragma unroll 4
-    for (int c = c0; c <= c1; ++c) {
-        const long long pid = u + c;
-        const float w = fast_exp2(part_ml[(pid * G + g) * 2] - M);
-        o = fmaf(w, part_o[(pid * G + g) * D + d], o);
-        den = fmaf(w, part_ml[(pid * G + g) * 2 + 1], den);
+    const float* po = part_o + ((u + c0) * G + g) * D + d;               // piece c: po[c * G * D]
+#pragma unroll 8
+    for (int c = 0; c < np; ++c) {
+        const float w = wsm[c];
+        o = fmaf(w, po[(long long)c * G * D], o);
+        den = fmaf(w, lsm[c], den);
     }
     out[(u * G + g) * D + d] = o / den;
 }

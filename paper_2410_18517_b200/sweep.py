@@ -2,9 +2,10 @@
 context and shared-layer fraction.  One JSON line per point: time per decode step, attention-path
 tokens/s, KV-read GB/s and pool size.
 
-    python -m paper_2410_18517_b200.sweep [--out FILE] [--steps K] [--only B,N,P]
+    python -m paper_2410_18517_b200.sweep [--out FILE] [--steps K] [--only B,N,P] [--shared P] [--kernel K]
 
 A *step* is one pass over all layers (append on computing layers + attention on every layer).
+--kernel forces KVS_OPT_KERNEL (1 scalar, 2 tensor-core) instead of the library's own choice.
 Each point is timed twice: launched call by call from Python, and as replays of a CUDA graph of one
 recorded step (which takes the host's launch cost out; with the library's replay counter every
 replay is the next decode step, one row further along).  All computing layers are loaded with the
@@ -19,7 +20,7 @@ import sys
 import torch
 
 import synth_inputs as si
-from paper_2410_18517_b200 import KVS_OPT_REPLAY, SharedKVCache
+from paper_2410_18517_b200 import KVS_OPT_KERNEL, KVS_OPT_REPLAY, SharedKVCache
 
 HBM_BYTES_USABLE = 170 * 2**30      # leave head-room below the 180 GB of a B200
 
@@ -29,7 +30,7 @@ def pool_bytes(w: si.Workload, extra_rows: int) -> int:
     return (w.L - w.n_shared) * 2 * w.B * w.Hkv * rs * w.D * w.elem_bytes
 
 
-def time_point(w: si.Workload, steps: int, device=0) -> dict:
+def time_point(w: si.Workload, steps: int, device=0, kernel=0) -> dict:
     extra = 3 * steps + 24
     rec = {"workload": w.name, "batch": w.B, "context": w.context, "shared_layers": w.n_shared,
            "pool_bytes": pool_bytes(w, extra), "pool_bytes_unshared": pool_bytes(w.scaled(n_shared=0), extra)}
@@ -41,6 +42,8 @@ def time_point(w: si.Workload, steps: int, device=0) -> dict:
     rec["share_map"] = [int(x) for x in sm]
     dev = torch.device("cuda", device)
     cache = SharedKVCache(w.L, w.Hq, w.Hkv, w.D, w.B, w.context + extra, w.dtype, share_map=sm, device=device)
+    if kernel:
+        cache.set_option(KVS_OPT_KERNEL, kernel)
     k, v = si.context_kv(w, 0, device=dev)
     for l in range(w.L):
         if sm[l] == l:
@@ -107,14 +110,18 @@ def main():
     ap.add_argument("--out", default=None)
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--only", default=None, help="B,N,P of a single point")
+    ap.add_argument("--shared", type=int, default=None, help="only the points with this many shared layers")
+    ap.add_argument("--kernel", type=int, default=0, help="force KVS_OPT_KERNEL (0 = the library's choice)")
     args = ap.parse_args()
     pts = si.sweep_points()
+    if args.shared is not None:
+        pts = [p for p in pts if p.n_shared == args.shared]
     if args.only:
         B, N, P = (int(x) for x in args.only.split(","))
         pts = [p for p in pts if (p.B, p.context, p.n_shared) == (B, N, P)]
     f = open(args.out, "w") if args.out else None
     for w in pts:
-        rec = time_point(w, args.steps)
+        rec = time_point(w, args.steps, kernel=args.kernel)
         line = json.dumps(rec)
         print(line, flush=True)
         if f:
