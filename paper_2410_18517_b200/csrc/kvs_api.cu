@@ -276,6 +276,7 @@ kvs_status run_attention(kvs_ctx* c, int slot, const void* q, float* out, int ba
     a.status = scratch.status;
     a.n = c->slot_len[slot];
     a.row_stride = c->row_stride;
+    a.capacity = c->cfg.max_seq;
     a.units = batch * c->cfg.n_kv_heads;
     a.G = c->G;
     a.D = c->cfg.head_dim;

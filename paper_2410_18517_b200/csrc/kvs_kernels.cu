@@ -37,6 +37,10 @@ __global__ void __launch_bounds__(256) kv_append_kernel(const uint4* __restrict_
         const int t = (int)(r % n_new);
         const long long b = r / n_new;
         const int first = unit_len ? unit_len[b * Hkv + h] : len0;   // ragged slots append per unit
+        if (first + t >= capacity) {   // only a replay that outran the capacity gets here
+            if (c == 0) atomicExch(status, 4);
+            continue;
+        }
         const long long drow = (b * Hkv + h) * (long long)row_stride + first + t;
         dst[drow * row_vecs + c] = src[idx];
     }
@@ -254,6 +258,7 @@ struct ScalarKernelArgs {
     const int* unit_len;  // per-unit row counts of a ragged slot, or nullptr (then n holds for all)
     const int* n_extra;   // graph replay: rows every slot has grown by since the launch was recorded, or nullptr
     int units;
+    int cap;              // rows a unit can hold: lengths that grew on the device are cut off there
 };
 
 template <typename T, int D, int G, int GEOM>
@@ -265,7 +270,7 @@ __global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G, GEOM>::MI
         // A replayed launch: the lengths recorded with it have grown on the device since.  The
         // counter is stable here without a wait: the host gives the first launch after every write
         // of the counter a full dependency, so that write is complete before any reader starts.
-        a.n += *a.n_extra;
+        a.n = min(a.n + *a.n_extra, a.cap);   // a replay that outran the capacity appended nothing more
         a.tpu = (a.n + S::TN - 1) / S::TN;
         a.T = (long long)a.units * a.tpu;
     }
@@ -308,7 +313,7 @@ __global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G, GEOM>::MI
                 const long long u = gt / a.tpu;
                 const int ti = (int)(gt - u * a.tpu);
                 const int row0 = ti * TN;
-                const int n_u = a.unit_len ? a.unit_len[u] : a.n;
+                const int n_u = a.unit_len ? min(a.unit_len[u], a.cap) : a.n;
                 const int rows = max(0, min(TN, n_u - row0));     // a ragged unit may end before this tile
                 const uint32_t bytes = (uint32_t)rows * RB;
                 const bool with_q = (gt == t0) || (ti == 0);
@@ -370,7 +375,7 @@ __global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G, GEOM>::MI
         const long long u = gt / a.tpu;
         const int ti0 = (int)(gt - u * a.tpu);
         const int piece_tiles = (int)min((long long)(a.tpu - ti0), t1 - gt);
-        const int n_u = a.unit_len ? a.unit_len[u] : a.n;
+        const int n_u = a.unit_len ? min(a.unit_len[u], a.cap) : a.n;
 
         float qf[G][EPL];
         float m[G], lsum[G], acc[G][EPL];
@@ -508,13 +513,13 @@ __global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G, GEOM>::MI
 // --------------------------------------------------------------------------------------
 __global__ void decode_combine_kernel(const float* __restrict__ part_o, const float* __restrict__ part_ml,
                                       float* __restrict__ out, int G, int D, int tpu, long long T, int NC,
-                                      const int* __restrict__ n_extra, int n, int tile_rows, int units) {
+                                      const int* __restrict__ n_extra, int n, int tile_rows, int units, int cap) {
     __shared__ float wsm[kMaxCtas], lsm[kMaxCtas];
     __shared__ float msm[4];
     pdl_launch_dependents();
     pdl_wait();
     if (n_extra) {   // replayed launch: recompute the tile line from the grown length
-        tpu = (n + *n_extra + tile_rows - 1) / tile_rows;
+        tpu = (min(n + *n_extra, cap) + tile_rows - 1) / tile_rows;
         T = (long long)units * tpu;
     }
     const long long u = blockIdx.x / G;
@@ -553,7 +558,7 @@ __global__ void decode_combine_kernel(const float* __restrict__ part_o, const fl
 cudaError_t launch_combine(const DecodeArgs& a, const DecodePlan& plan, cudaStream_t stream) {
     return launch_kernel(decode_combine_kernel, dim3(a.units * a.G), dim3(a.D), 0, stream, a.programmatic,
                          (const float*)a.part_o, (const float*)a.part_ml, a.out, a.G, a.D, plan.tpu, plan.T, plan.NC, a.n_extra,
-                         a.n, plan.tile_rows, a.units);
+                         a.n, plan.tile_rows, a.units, a.capacity);
 }
 
 // --------------------------------------------------------------------------------------
@@ -626,6 +631,7 @@ cudaError_t launch_decode_scalar(const DecodeArgs& a, const DecodePlan& plan, cu
     ka.unit_len = a.unit_len;
     ka.n_extra = a.n_extra;
     ka.units = a.units;
+    ka.cap = a.capacity;
     const bool pdl = a.programmatic;
     if (a.dtype == 0) {
         if (a.D == 128) return launch_scalar_groups<__nv_bfloat16, 128>(a.G, plan.geom, ka, plan.NC, pdl, stream);

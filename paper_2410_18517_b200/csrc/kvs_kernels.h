@@ -31,6 +31,7 @@ struct DecodeArgs {
     int* status;          // device status word
     int n;                // rows cached per unit
     int row_stride;       // rows between units of a plane
+    int capacity;         // rows a unit can hold (max_seq): lengths that grew on the device are cut off there
     int units;            // B * Hkv
     int G;                // q-heads per kv-head
     int D;

@@ -107,6 +107,7 @@ struct MmaKernelArgs {
     int G;          // q-heads per kv-head, 1..8
     const int* n_extra;  // graph replay: rows every slot has grown by since the launch was recorded, or nullptr
     int units;
+    int cap;             // rows a unit can hold: lengths that grew on the device are cut off there
 };
 
 // G (q-heads per kv-head, 1..8) is a run-time argument: it only selects which rows of the padded
@@ -120,7 +121,7 @@ __global__ void __launch_bounds__(kMmaThreads, KVS_MMA_BLOCKS_PER_SM)
         // A replayed launch: the lengths recorded with it have grown on the device since.  The
         // counter is stable here without a wait: the host gives the first launch after every write
         // of the counter a full dependency, so that write is complete before any reader starts.
-        a.n += *a.n_extra;
+        a.n = min(a.n + *a.n_extra, a.cap);   // a replay that outran the capacity appended nothing more
         a.tpu = (a.n + S::TN - 1) / S::TN;
         a.T = (long long)a.units * a.tpu;
     }
@@ -161,7 +162,7 @@ __global__ void __launch_bounds__(kMmaThreads, KVS_MMA_BLOCKS_PER_SM)
                 const long long u = gt / a.tpu;
                 const int ti = (int)(gt - u * a.tpu);
                 const bool with_q = (gt == t0) || (ti == 0);
-                const int n_u = a.unit_len ? a.unit_len[u] : a.n;
+                const int n_u = a.unit_len ? min(a.unit_len[u], a.cap) : a.n;
                 const bool have = ti * TN < n_u;                  // a ragged unit may end before this tile
                 unsigned char* sb = smem + st * S::STAGE_BYTES;
                 if (arm) {
@@ -225,7 +226,7 @@ __global__ void __launch_bounds__(kMmaThreads, KVS_MMA_BLOCKS_PER_SM)
         const long long u = gt / a.tpu;
         const int ti0 = (int)(gt - u * a.tpu);
         const int piece_tiles = (int)min((long long)(a.tpu - ti0), t1 - gt);
-        const int n_u = a.unit_len ? a.unit_len[u] : a.n;
+        const int n_u = a.unit_len ? min(a.unit_len[u], a.cap) : a.n;
 
         uint32_t qa[KSTEPS][2];
         float o[NB][2];
@@ -447,6 +448,7 @@ cudaError_t launch_decode_mma(const DecodeArgs& a, const DecodePlan& plan, const
     ka.G = a.G;
     ka.n_extra = a.n_extra;
     ka.units = a.units;
+    ka.cap = a.capacity;
     if (a.G < 1 || a.G > 8) return cudaErrorInvalidValue;
     if (a.D == 128) return launch_one<128>(tm, ka, plan.NC, a.programmatic, stream);
     if (a.D == 64) return launch_one<64>(tm, ka, plan.NC, a.programmatic, stream);

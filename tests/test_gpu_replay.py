@@ -120,3 +120,57 @@ def test_replay_calls_need_the_option():
     with pytest.raises(KvsError) as e:           # 16 rows cached, capacity 16: no room for 3 more
         cache.replay_commit(4)
     assert e.value.status == kb.KVS_ERR_CAPACITY
+
+
+@pytest.mark.parametrize("Hq,Hkv,evict", [(4, 4, False), (8, 2, False), (4, 2, True)])
+def test_replays_past_the_capacity_stop_appending_and_report(Hq, Hkv, evict):
+    """Capacity 128 rows (one whole row stride), 126 cached, the recorded step makes 127: the replays
+    after the first would need rows 128, 129, ...  The kernels' own checks append nothing there, attend
+    over the rows that exist, set the status word, and the commit refuses; no row outside a unit is
+    touched (the neighbouring units and the rest of the pool keep their bits)."""
+    L, D, B, cap = 2, 128, 2, 128
+    sm = [0, 0]
+    w = si.Workload(f"replay_over_{Hq}_{Hkv}", L=L, Hq=Hq, Hkv=Hkv, D=D, B=B, context=cap - 2, dtype="bf16", n_shared=1,
+                    map_seed=0, steps=8, fixed_map=tuple(sm))
+    cache = SharedKVCache(L, Hq, Hkv, D, B, cap, "bf16", share_map=sm)
+    cache.set_option(KVS_OPT_REPLAY, 1)
+    k, v = si.context_kv(w, 0)
+    cache.append(0, k.cuda(), v.cuda())
+    if evict:                                     # a ragged slot: the longest unit keeps every row
+        n_keep = np.full((B, Hkv), cap - 2, dtype=np.int32)
+        n_keep[0, 0] = 40
+        keep = np.tile(np.arange(cap - 2, dtype=np.int32), (B, Hkv, 1))
+        cache.evict(0, torch.from_numpy(keep).cuda(), n_keep)
+    q, kk, vv = (t.cuda() for t in si.step_qkv(w, 0, 0))
+    out = torch.empty(B, Hq, D, dtype=torch.float32, device="cuda")
+
+    def one_step():
+        cache.append(0, kk, vv)
+        cache.decode_attention(0, q, out)
+        cache.decode_attention(1, q, out)
+        cache.replay_advance()
+
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            one_step()
+    before = cache.pool.clone()
+    for _ in range(5):                            # rows 126, 127 fit; 128.. do not
+        graph.replay()
+    torch.cuda.synchronize()
+    assert cache.device_status() == kb.KVS_ERR_CAPACITY
+    with pytest.raises(KvsError) as e:
+        cache.replay_commit(5)
+    assert e.value.status == kb.KVS_ERR_CAPACITY
+    assert torch.isfinite(out).all()
+    # only the rows the replays could legally append may differ from the pool before the replays:
+    # rows 126 and 127 of a full unit, rows 40..44 of the unit that was cut to 40 rows
+    changed = (cache.pool != before).view(1, 2, B, Hkv, cap, D * 2).any(dim=-1)
+    expect = torch.zeros_like(changed)
+    expect[..., cap - 2 :] = True
+    if evict:
+        expect[:, :, 0, 0, :] = False
+        expect[:, :, 0, 0, 40:45] = True
+    assert torch.equal(changed, expect)
