@@ -181,7 +181,7 @@ kvs_status kvs_decode_attention(kvs_ctx* ctx, int32_t layer, const void* q, floa
  * chunk of it (n > n_q).
  *   q:   device, [batch][n_q][n_q_heads][head_dim], storage type, 16-byte aligned
  *   out: device, [batch][n_q][n_q_heads][head_dim], float32
- * One 4-byte clear and one tcgen05 tensor-core kernel on `stream`; bf16 storage and head_dim 128 only (other
+ * One 4-byte clear and one tcgen05 tensor-core kernel on `stream`; bf16 storage only (other
  * configurations: INVALID_ARG).  Other errors as kvs_decode_attention; n_q > n: INVALID_ARG. */
 kvs_status kvs_prefill_attention(kvs_ctx* ctx, int32_t layer, const void* q, float* out,
                                  int32_t batch, int32_t n_q, void* stream);

@@ -476,7 +476,7 @@ kvs_status kvs_prefill_attention(kvs_ctx* ctx, int32_t layer, const void* q, flo
     if (!ctx->bound) return KVS_ERR_STATE;
     if (layer < 0 || layer >= ctx->cfg.n_layers || !q || !out) return KVS_ERR_INVALID_ARG;
     if (batch < 1 || batch > ctx->cfg.max_batch || n_q < 1) return KVS_ERR_INVALID_ARG;
-    if (ctx->cfg.dtype != KVS_BF16 || ctx->cfg.head_dim != 128 || !ctx->have_tensor_map) return KVS_ERR_INVALID_ARG;
+    if (ctx->cfg.dtype != KVS_BF16 || !ctx->have_tensor_map) return KVS_ERR_INVALID_ARG;
     if (((uintptr_t)q % 16) != 0 || ((uintptr_t)out % 16) != 0) return KVS_ERR_INVALID_ARG;
     const int slot = ctx->slot_of_layer[layer];
     const int n = ctx->slot_len[slot];
@@ -488,7 +488,7 @@ kvs_status kvs_prefill_attention(kvs_ctx* ctx, int32_t layer, const void* q, flo
     // the prefill kernel's work counter lives in the status block, 64 bytes after the status word
     if (kvs::launch_prefill(q, out, reinterpret_cast<int*>(ctx->ws + ctx->off_status),
                             reinterpret_cast<int*>(ctx->ws + ctx->off_status + 64), ctx->tensor_map, batch, n_q,
-                            ctx->cfg.n_q_heads, ctx->G, n, ctx->row_stride, plane_rows * (2 * slot),
+                            ctx->cfg.n_q_heads, ctx->G, ctx->cfg.head_dim, n, ctx->row_stride, plane_rows * (2 * slot),
                             plane_rows * (2 * slot + 1), ctx->scale * 1.4426950408889634f, ctx->sm_count, ctx->l2_bytes,
                             static_cast<cudaStream_t>(stream)) != cudaSuccess)
         return KVS_ERR_CUDA;

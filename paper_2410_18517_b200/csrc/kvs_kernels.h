@@ -65,12 +65,12 @@ cudaError_t make_pool_tensor_map(void* storage, void* pool, long long total_rows
 cudaError_t launch_decode_mma(const DecodeArgs& a, const DecodePlan& plan, const void* tensor_map, long long krow0,
                               long long vrow0, cudaStream_t stream);
 
-// Tensor-core prefill attention (bf16, head size 128): q [B][T][Hq][128], out fp32 of the same shape.
+// Tensor-core prefill attention (bf16, head size D = 64 or 128): q [B][T][Hq][D], out fp32 of the same shape.
 cudaError_t init_prefill_kernels();
 // `sched`: a device int for the kernel's work counter (zeroed on `stream` by the launch).
 cudaError_t launch_prefill(const void* q, float* out, int* status, int* sched, const void* pool_tensor_map, int B, int T,
-                           int Hq, int G, int n, int row_stride, long long krow0, long long vrow0, float scale_log2,
-                           int sm_count, long long l2_bytes, cudaStream_t stream);
+                           int Hq, int G, int D, int n, int row_stride, long long krow0, long long vrow0,
+                           float scale_log2, int sm_count, long long l2_bytes, cudaStream_t stream);
 
 // Strategy-search reductions (see kvs_search.cu).
 constexpr int kMaxLayersSearch = 80;     // shared-memory bound of the distance kernel

@@ -17,7 +17,7 @@
 // Two blocks share an SM (99 KiB of shared memory and 256 TMEM columns each), so four key
 // tiles are in flight per SM.  K/V/Q tiles land in the 128-byte-swizzled layout the MMA
 // shared-memory descriptors expect (K and Q K-major, V MN-major).
-// bf16 storage, head size 128.
+// bf16 storage, head size 64 or 128.
 #include <cuda.h>
 
 #include <algorithm>
@@ -33,11 +33,21 @@ constexpr int kPfSoftmaxWarps = 8;
 constexpr int kPfThreads = (kPfSoftmaxWarps + 2) * 32;
 constexpr int kPfTile = 128;                 // queries per block
 constexpr int kPfKeys = 64;                  // keys per tile
-constexpr int kPfQBytes = kPfTile * 256;     // 128 x 128 bf16: two swizzled blocks of 64 columns
-constexpr int kPfKvBytes = kPfKeys * 256;    // 64 x 128 bf16: two swizzled blocks of 64 columns
-constexpr int kPfSmemBytes = 1024 + kPfQBytes + 4 * kPfKvBytes /*K, V: two stages each*/ + 256 +
-                             6 * kPfTile * 4 /*row maxima, row sums*/;
-constexpr uint32_t kTmemCols = 256;          // two score buffers: columns [0,64), [64,128); O tile: [128,256)
+constexpr int kPfQBlock = kPfTile * 128;     // one swizzled block of Q: 128 rows x 64 bf16 columns
+constexpr int kPfKvBlock = kPfKeys * 128;    // one swizzled block of K or V: 64 rows x 64 bf16 columns
+// Head size D = 64 or 128: rows are D/64 swizzled blocks wide.
+template <int D>
+struct PfShape {
+    static constexpr int HALVES = D / 64;
+    static constexpr int Q_BYTES = HALVES * kPfQBlock;
+    static constexpr int KV_BYTES = HALVES * kPfKvBlock;
+    static constexpr int Q_BUF = 2 * kPfQBlock;   // the Q tile; later two [128 rows][32 floats] blocks of staged output
+    static constexpr int SMEM_BYTES = 1024 + Q_BUF + 4 * KV_BYTES /*K, V: two stages each*/ + 256 +
+                                      6 * kPfTile * 4 /*row maxima, row sums*/;
+    static constexpr int OC = D / 2;              // output columns per softmax thread
+    static constexpr int ROUNDS = OC / 32;        // staging rounds of 32 columns per thread
+};
+constexpr uint32_t kTmemCols = 256;          // two score buffers: columns [0,64), [64,128); O tile: [128,128+D)
 
 __device__ __forceinline__ void tma_load_2d_pf(void* dst, const CUtensorMap* tmap, int x, int y, uint64_t* bar) {
     asm volatile(
@@ -233,15 +243,18 @@ __device__ __forceinline__ float softmax_chunk(const float (&x)[32], float scale
     return sum.x + sum.y;
 }
 
+template <int D>
 __global__ void __launch_bounds__(kPfThreads, 2)
     prefill_attention_tc(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_kv,
                          const __grid_constant__ CUtensorMap tmap_out, const PrefillArgs a) {
     extern __shared__ unsigned char smem_raw[];
     unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
     unsigned char* sQ = smem;                       // Q tile; after an item's last MMA, staging for its output
-    unsigned char* sK = sQ + kPfQBytes;             // two stages
-    unsigned char* sV = sK + 2 * kPfKvBytes;        // two stages
-    uint64_t* bars = reinterpret_cast<uint64_t*>(sV + 2 * kPfKvBytes);
+    using S = PfShape<D>;
+    constexpr int kKvBytes = S::KV_BYTES;
+    unsigned char* sK = sQ + S::Q_BUF;              // two stages
+    unsigned char* sV = sK + 2 * kKvBytes;          // two stages
+    uint64_t* bars = reinterpret_cast<uint64_t*>(sV + 2 * kKvBytes);
     uint64_t* q_full = bars;
     uint64_t* q_free = bars + 1;        // the output staged in the Q buffer has been read by the TMA store
     uint64_t* o_full = bars + 2;        // one phase per PV group: that tile's contribution is in O
@@ -312,9 +325,10 @@ __global__ void __launch_bounds__(kPfThreads, 2)
                 auto load_q = [&]() {
                     // the Q buffer doubles as the previous item's output staging
                     if (it >= 1 && !mbar_wait_bounded(q_free, (uint32_t)(it - 1) & 1u, abort_flag, a.status)) return false;
-                    mbar_arrive_expect_tx(q_full, kPfQBytes);
-                    tma_load_4d(sQ, &tmap_q, 0, item.hq, item.q0, item.b, q_full);
-                    tma_load_4d(sQ + kPfQBytes / 2, &tmap_q, 64, item.hq, item.q0, item.b, q_full);
+                    mbar_arrive_expect_tx(q_full, S::Q_BYTES);
+#pragma unroll
+                    for (int h = 0; h < S::HALVES; ++h)
+                        tma_load_4d(sQ + h * kPfQBlock, &tmap_q, h * 64, item.hq, item.q0, item.b, q_full);
                     return true;
                 };
                 for (int j = 0; j < item.nt && ok; ++j) {
@@ -326,16 +340,16 @@ __global__ void __launch_bounds__(kPfThreads, 2)
                     const uint32_t prev = (uint32_t)((tt >> 1) - 1) & 1u;   // phase in which tile tt-2 released the stage
                     const long long row = unit_row + (long long)j * kPfKeys;
                     if (tt >= 2 && !mbar_wait_bounded(&k_empty[st], prev, abort_flag, a.status)) { ok = false; break; }
-                    mbar_arrive_expect_tx(&k_full[st], kPfKvBytes);
+                    mbar_arrive_expect_tx(&k_full[st], kKvBytes);
 #pragma unroll
-                    for (int h = 0; h < 2; ++h)
-                        tma_load_2d_pf(sK + st * kPfKvBytes + h * (kPfKvBytes / 2), &tmap_kv, h * 64, (int)(a.krow0 + row),
+                    for (int h = 0; h < S::HALVES; ++h)
+                        tma_load_2d_pf(sK + st * kKvBytes + h * kPfKvBlock, &tmap_kv, h * 64, (int)(a.krow0 + row),
                                        &k_full[st]);
                     if (tt >= 2 && !mbar_wait_bounded(&v_empty[st], prev, abort_flag, a.status)) { ok = false; break; }
-                    mbar_arrive_expect_tx(&v_full[st], kPfKvBytes);
+                    mbar_arrive_expect_tx(&v_full[st], kKvBytes);
 #pragma unroll
-                    for (int h = 0; h < 2; ++h)
-                        tma_load_2d_pf(sV + st * kPfKvBytes + h * (kPfKvBytes / 2), &tmap_kv, h * 64, (int)(a.vrow0 + row),
+                    for (int h = 0; h < S::HALVES; ++h)
+                        tma_load_2d_pf(sV + st * kKvBytes + h * kPfKvBlock, &tmap_kv, h * 64, (int)(a.vrow0 + row),
                                        &v_full[st]);
                 }
                 if (ok && item.nt <= 2) ok = load_q();
@@ -351,14 +365,14 @@ __global__ void __launch_bounds__(kPfThreads, 2)
         // softmax threads arrive for it only after they have read the previous item's output.
         if (lane == 0) {
             const uint32_t idesc_s = instr_desc_bf16(0, kPfKeys);
-            const uint32_t idesc_o = instr_desc_bf16(1, 128);
+            const uint32_t idesc_o = instr_desc_bf16(1, D);
             const uint32_t q_addr = smem_u32(sQ), k_addr = smem_u32(sK), v_addr = smem_u32(sV);
             auto issue_s = [&](int tt) {
                 const int st = tt & 1;
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {   // 16 head-dim columns per step; 4 steps per 64-column block
-                    const uint32_t qoff = (ks >> 2) * (kPfQBytes / 2) + (ks & 3) * 32;
-                    const uint32_t koff = st * kPfKvBytes + (ks >> 2) * (kPfKvBytes / 2) + (ks & 3) * 32;
+                for (int ks = 0; ks < D / 16; ++ks) {   // 16 head-dim columns per step; 4 steps per 64-column block
+                    const uint32_t qoff = (ks >> 2) * kPfQBlock + (ks & 3) * 32;
+                    const uint32_t koff = st * kKvBytes + (ks >> 2) * kPfKvBlock + (ks & 3) * 32;
                     umma_bf16(tmem_s + st * kPfKeys, smem_desc_sw128(q_addr + qoff, 16, 1024),
                               smem_desc_sw128(k_addr + koff, 16, 1024), idesc_s, ks > 0);
                 }
@@ -394,10 +408,9 @@ __global__ void __launch_bounds__(kPfThreads, 2)
                     tc_fence_after();
 #pragma unroll
                     for (int ks = 0; ks < kPfKeys / 16; ++ks) {   // 16 keys per step: 8 TMEM columns of bf16 pairs
-                        // V is MN-major: 64 head-dim columns contiguous per key row, the other 64 one
-                        // column block (LBO) away; 8-key groups 1024 bytes (SBO) apart
-                        const uint64_t vdesc =
-                            smem_desc_sw128(v_addr + st * kPfKvBytes + ks * 16 * 128, kPfKvBytes / 2, 1024);
+                        // V is MN-major: 64 head-dim columns contiguous per key row, the other 64 (D = 128)
+                        // one column block (LBO) away; 8-key groups 1024 bytes (SBO) apart
+                        const uint64_t vdesc = smem_desc_sw128(v_addr + st * kKvBytes + ks * 16 * 128, kPfKvBlock, 1024);
                         umma_bf16_ts(tmem_o, tmem_s + st * kPfKeys + ks * 8, vdesc, idesc_o, (j > 0) || (ks > 0));   // P_hi
                         umma_bf16_ts(tmem_o, tmem_s + st * kPfKeys + kPfKeys / 2 + ks * 8, vdesc, idesc_o, 1);     // P_lo
                     }
@@ -414,10 +427,10 @@ __global__ void __launch_bounds__(kPfThreads, 2)
         const int w4 = warp & 3, hf = warp >> 2;             // TMEM lane quarter, key half of a tile
         const int r = w4 * 32 + lane;                        // query row in the block = TMEM lane
         const uint32_t lane_addr = (uint32_t)(w4 * 32) << 16;
-        const uint32_t to = tmem_o + lane_addr + hf * 64;        // this thread's 64 columns of the output row
+        const uint32_t to = tmem_o + lane_addr + hf * S::OC;     // this thread's D/2 columns of the output row
         // output staging: [128 rows][32 floats] blocks, 128-byte swizzle; this thread's row of the
         // block its key half owns
-        unsigned char* stage_row = sQ + hf * (kPfQBytes / 2) + r * 128;
+        unsigned char* stage_row = sQ + hf * kPfQBlock + r * 128;
         int t = 0;
         uint32_t pp = 0, ep = 0;                             // phases used so far of pair_bar[w4] and epi_bar
         bool ok = true;
@@ -478,7 +491,7 @@ __global__ void __launch_bounds__(kPfThreads, 2)
                         if (!ok) break;
                         tc_fence_after();
 #pragma unroll 1
-                        for (int c = 0; c < 8; ++c) tmem_scale8(to + c * 8, alpha);
+                        for (int c = 0; c < S::OC / 8; ++c) tmem_scale8(to + c * 8, alpha);
                     }
                     l *= alpha;
                     m_ref = m_new;
@@ -512,12 +525,12 @@ __global__ void __launch_bounds__(kPfThreads, 2)
             if (!ok) break;
             tc_fence_after();
             // Output: every MMA of the item is done, so the Q buffer is free.  Each thread scales its
-            // 64 columns and stages them there, 32 columns per round, in the swizzled layout of a TMA
+            // D/2 columns and stages them there, 32 columns per round, in the swizzled layout of a TMA
             // store; one thread issues the stores (rows past the last query are clipped by the
             // tensor map) and waits until they have read the buffer.
             const float inv = 1.0f / l;
 #pragma unroll 1
-            for (int c = 0; c < 2; ++c) {
+            for (int c = 0; c < S::ROUNDS; ++c) {
                 float o[32];
                 tmem_ld32(to + c * 32, o);
 #pragma unroll
@@ -531,12 +544,12 @@ __global__ void __launch_bounds__(kPfThreads, 2)
                 if (!ok) break;
                 if (tid == 0) {
                     tma_store_4d(&tmap_out, sQ, c * 32, item.hq, item.q0, item.b);
-                    tma_store_4d(&tmap_out, sQ + kPfQBytes / 2, 64 + c * 32, item.hq, item.q0, item.b);
+                    tma_store_4d(&tmap_out, sQ + kPfQBlock, S::OC + c * 32, item.hq, item.q0, item.b);
                     asm volatile("cp.async.bulk.commit_group;" ::: "memory");
                     asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-                    if (c == 1) mbar_arrive(q_free);
+                    if (c == S::ROUNDS - 1) mbar_arrive(q_free);
                 }
-                if (c == 0) {   // the buffer is reused by the second round
+                if (c < S::ROUNDS - 1) {   // the buffer is reused by the next round
                     mbar_arrive(epi_bar);
                     ok = mbar_wait_bounded(epi_bar, ep & 1u, abort_flag, a.status);
                     ++ep;
@@ -576,22 +589,28 @@ cudaError_t get_encode(EncodeFn* out) {
 }  // namespace
 
 cudaError_t init_prefill_kernels() {
-    return cudaFuncSetAttribute(prefill_attention_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kPfSmemBytes);
+    cudaError_t e = cudaFuncSetAttribute(prefill_attention_tc<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         PfShape<128>::SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    return cudaFuncSetAttribute(prefill_attention_tc<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                PfShape<64>::SMEM_BYTES);
 }
 
-// q: [B][T][Hq][128] bf16.  Persistent blocks (two per SM) take (128 queries, q-head, sequence)
-// items from a counter, heaviest first.  `sched` is a device int the launch zeroes on `stream`.
+// q: [B][T][Hq][D] bf16, D = 64 or 128.  Persistent blocks (two per SM) take (128 queries, q-head,
+// sequence) items from a counter, heaviest first.  `sched` is a device int the launch zeroes on `stream`.
 cudaError_t launch_prefill(const void* q, float* out, int* status, int* sched, const void* pool_tensor_map, int B, int T,
-                           int Hq, int G, int n, int row_stride, long long krow0, long long vrow0, float scale_log2,
-                           int sm_count, long long l2_bytes, cudaStream_t stream) {
+                           int Hq, int G, int D, int n, int row_stride, long long krow0, long long vrow0,
+                           float scale_log2, int sm_count, long long l2_bytes, cudaStream_t stream) {
+    if (D != 64 && D != 128) return cudaErrorInvalidValue;
     EncodeFn encode = nullptr;
     cudaError_t e = get_encode(&encode);
     if (e != cudaSuccess) return e;
     alignas(64) CUtensorMap tq, to;
-    cuuint64_t dims[4] = {128, (cuuint64_t)Hq, (cuuint64_t)T, (cuuint64_t)B};
+    const cuuint64_t d = (cuuint64_t)D;
+    cuuint64_t dims[4] = {d, (cuuint64_t)Hq, (cuuint64_t)T, (cuuint64_t)B};
     cuuint32_t estr[4] = {1, 1, 1, 1};
     {
-        cuuint64_t strides[3] = {128 * 2, (cuuint64_t)Hq * 128 * 2, (cuuint64_t)T * Hq * 128 * 2};
+        cuuint64_t strides[3] = {d * 2, (cuuint64_t)Hq * d * 2, (cuuint64_t)T * Hq * d * 2};
         cuuint32_t box[4] = {64, 1, (cuuint32_t)kPfTile, 1};
         if (encode(&tq, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(q), dims, strides, box, estr,
                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -599,7 +618,7 @@ cudaError_t launch_prefill(const void* q, float* out, int* status, int* sched, c
             return cudaErrorInvalidValue;
     }
     {
-        cuuint64_t strides[3] = {128 * 4, (cuuint64_t)Hq * 128 * 4, (cuuint64_t)T * Hq * 128 * 4};
+        cuuint64_t strides[3] = {d * 4, (cuuint64_t)Hq * d * 4, (cuuint64_t)T * Hq * d * 4};
         cuuint32_t box[4] = {32, 1, (cuuint32_t)kPfTile, 1};
         if (encode(&to, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, out, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                    CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) !=
@@ -619,10 +638,10 @@ cudaError_t launch_prefill(const void* q, float* out, int* status, int* sched, c
     a.vrow0 = vrow0;
     a.scale_log2 = scale_log2;
     {
-        // kv-heads whose K/V rows (n rows of 256 bytes, K and V) fit in three quarters of L2
+        // kv-heads whose K/V rows (n rows of 2 D bytes, K and V) fit in three quarters of L2
         // together; groups of equal size
         const long long streams = (long long)B * (Hq / G);
-        const long long stream_bytes = 2LL * n * 256;
+        const long long stream_bytes = 2LL * n * D * 2;
         const long long fit = std::max<long long>(1, (l2_bytes / 4 * 3) / stream_bytes);
         const long long groups = (streams + fit - 1) / fit;
         a.group_heads = (int)((streams + groups - 1) / groups) * G;
@@ -630,8 +649,11 @@ cudaError_t launch_prefill(const void* q, float* out, int* status, int* sched, c
     if ((e = cudaMemsetAsync(sched, 0, sizeof(int), stream)) != cudaSuccess) return e;
     const long long items = (long long)((T + kPfTile - 1) / kPfTile) * Hq * B;
     const int blocks = (int)std::min<long long>(items, 2LL * sm_count);
-    prefill_attention_tc<<<blocks, kPfThreads, kPfSmemBytes, stream>>>(
-        tq, *reinterpret_cast<const CUtensorMap*>(pool_tensor_map), to, a);
+    const CUtensorMap& tkv = *reinterpret_cast<const CUtensorMap*>(pool_tensor_map);
+    if (D == 128)
+        prefill_attention_tc<128><<<blocks, kPfThreads, PfShape<128>::SMEM_BYTES, stream>>>(tq, tkv, to, a);
+    else
+        prefill_attention_tc<64><<<blocks, kPfThreads, PfShape<64>::SMEM_BYTES, stream>>>(tq, tkv, to, a);
     return cudaGetLastError();
 }
 

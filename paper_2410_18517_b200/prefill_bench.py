@@ -1,6 +1,6 @@
 """Throughput of the tensor-core prefill kernel (one layer's causal attention over a prompt).
 
-    python -m paper_2410_18517_b200.prefill_bench [--batch B --heads Hq --kv-heads Hkv --tokens T --iters N]
+    python -m paper_2410_18517_b200.prefill_bench [--batch B --heads Hq --kv-heads Hkv --tokens T --head-dim D --iters N]
 
 Prints one JSON line: milliseconds per call, causal algorithmic TFLOP/s (4 B Hq D T(T+1)/2 flops: the
 flops of the unmasked triangle of QK^T and PV), the tensor-core flops actually issued (the kernel runs
@@ -28,10 +28,11 @@ def main():
     ap.add_argument("--heads", type=int, default=32)
     ap.add_argument("--kv-heads", type=int, default=32)
     ap.add_argument("--tokens", type=int, default=4096)
+    ap.add_argument("--head-dim", type=int, default=128, choices=[64, 128])
     ap.add_argument("--iters", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     a = ap.parse_args()
-    B, Hq, Hkv, T, D = a.batch, a.heads, a.kv_heads, a.tokens, 128
+    B, Hq, Hkv, T, D = a.batch, a.heads, a.kv_heads, a.tokens, a.head_dim
     w = si.Workload("prefill_bench", L=2, Hq=Hq, Hkv=Hkv, D=D, B=B, context=T, dtype="bf16", n_shared=1, map_seed=0,
                     steps=1, fixed_map=(0, 0))
     cache = SharedKVCache(w.L, Hq, Hkv, D, B, T, "bf16", share_map=w.share_map())
@@ -52,7 +53,7 @@ def main():
     ms = e0.elapsed_time(e1) / a.iters
     algo = 4.0 * B * Hq * D * T * (T + 1) / 2
     tiles = sum(min(qb + 1, (T + 127) // 128) for qb in range((T + 127) // 128))     # 128x128 tiles visited per head
-    issued = B * Hq * tiles * 3 * 2.0 * 128 * 128 * 128                               # S + PV(hi) + PV(lo)
+    issued = B * Hq * tiles * 3 * 2.0 * 128 * 128 * D                                 # S + PV(hi) + PV(lo)
     try:
         peak = float(json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))["bf16_tflops"])
         kind = "of measured"

@@ -20,9 +20,9 @@ def _built():
     kbuild.build()
 
 
-def _prefill_both(Hq, Hkv, B, chunks, share_map, seed=0):
+def _prefill_both(Hq, Hkv, B, chunks, share_map, seed=0, D=128):
     """Feed the prompt in `chunks` (list of chunk lengths) to both sides, layer by layer."""
-    L, D = len(share_map), 128
+    L = len(share_map)
     total = sum(chunks)
     cache = SharedKVCache(L, Hq, Hkv, D, B, total, "bf16", share_map=share_map)
     orc = oracle.Oracle(L, Hq, Hkv, D, B, share_map)
@@ -52,6 +52,12 @@ def test_one_tile():
 @pytest.mark.parametrize("chunks", [[1], [127], [129], [300], [512], [200, 333], [128, 1, 77]])
 def test_prompt_lengths_chunks_and_sharing(Hq, Hkv, chunks):
     _prefill_both(Hq, Hkv, 2, chunks, [0, 0, 2, 0])
+
+
+@pytest.mark.parametrize("Hq,Hkv", [(2, 2), (8, 2)])
+@pytest.mark.parametrize("chunks", [[1], [64], [129], [300], [200, 333]])
+def test_head_size_64(Hq, Hkv, chunks):
+    _prefill_both(Hq, Hkv, 2, chunks, [0, 0, 2, 0], D=64)
 
 
 def test_prefill_then_decode_continues_from_the_same_cache():
@@ -86,9 +92,9 @@ def test_prefill_argument_checks():
     with pytest.raises(KvsError) as e:          # more queries than cached rows
         c.prefill_attention(0, q)
     assert e.value.status == kb.KVS_ERR_INVALID_ARG
-    f = SharedKVCache(1, 2, 2, 64, 1, 64, "bf16")
-    kk = torch.zeros(1, 4, 2, 64, dtype=torch.bfloat16, device="cuda")
+    f = SharedKVCache(1, 2, 2, 64, 1, 64, "f32")
+    kk = torch.zeros(1, 4, 2, 64, dtype=torch.float32, device="cuda")
     f.append(0, kk, kk)
-    with pytest.raises(KvsError) as e:          # head size 64 is not built for prefill
+    with pytest.raises(KvsError) as e:          # fp32 storage is not built for prefill
         kb.kvs_prefill_attention(f.ctx, 0, kk, torch.zeros(1, 4, 2, 64, device="cuda"), 1, 4, 0)
     assert e.value.status == kb.KVS_ERR_INVALID_ARG
