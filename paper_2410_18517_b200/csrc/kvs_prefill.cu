@@ -257,7 +257,10 @@ __global__ void __launch_bounds__(kPfThreads, 2)
     uint64_t* bars = reinterpret_cast<uint64_t*>(sV + 2 * kKvBytes);
     uint64_t* q_full = bars;
     uint64_t* q_free = bars + 1;        // the output staged in the Q buffer has been read by the TMA store
-    uint64_t* o_full = bars + 2;        // one phase per PV group: that tile's contribution is in O
+    // o_full[tile & 1]: one phase per PV group of a tile of that parity (the tile's contribution is in O).
+    // Two barriers, because the PV groups of two consecutive tiles can be outstanding at once and a
+    // parity wait cannot tell a phase from the one two before it.
+    uint64_t* o_full = bars + 28;
     uint64_t* epi_bar = bars + 3;       // all softmax threads, used around the output staging
     uint64_t* k_full = bars + 4;        // [2] per K stage
     uint64_t* k_empty = bars + 6;
@@ -281,6 +284,8 @@ __global__ void __launch_bounds__(kPfThreads, 2)
 
     if (tid == 0) {
         for (int i = 0; i < 24; ++i) mbar_init(&bars[i], 1);
+        mbar_init(&o_full[0], 1);
+        mbar_init(&o_full[1], 1);
         mbar_init(epi_bar, kSoftmaxThreads);
         mbar_init(&p_full[0], kSoftmaxThreads);
         mbar_init(&p_full[1], kSoftmaxThreads);
@@ -414,7 +419,7 @@ __global__ void __launch_bounds__(kPfThreads, 2)
                         umma_bf16_ts(tmem_o, tmem_s + st * kPfKeys + ks * 8, vdesc, idesc_o, (j > 0) || (ks > 0));   // P_hi
                         umma_bf16_ts(tmem_o, tmem_s + st * kPfKeys + kPfKeys / 2 + ks * 8, vdesc, idesc_o, 1);     // P_lo
                     }
-                    umma_commit(o_full);
+                    umma_commit(&o_full[st]);
                     umma_commit(&v_empty[st]);
                 }
                 if (!ok) break;
@@ -487,7 +492,7 @@ __global__ void __launch_bounds__(kPfThreads, 2)
                     const float m_new = grow ? mx : m_ref;
                     const float alpha = fast_exp2(m_ref - m_new);
                     if (j > 0) {
-                        ok = mbar_wait_bounded(o_full, (uint32_t)(tt - 1) & 1u, abort_flag, a.status);
+                        ok = mbar_wait_bounded(&o_full[(tt - 1) & 1], (uint32_t)((tt - 1) >> 1) & 1u, abort_flag, a.status);
                         if (!ok) break;
                         tc_fence_after();
 #pragma unroll 1
@@ -521,7 +526,8 @@ __global__ void __launch_bounds__(kPfThreads, 2)
             ++pp;
             if (!ok) break;
             l += exch_l[(hf ^ 1) * kPfTile + r];
-            ok = mbar_wait_bounded(o_full, (uint32_t)(t + nt - 1) & 1u, abort_flag, a.status);
+            // the last tile's PV group is behind every other MMA of the item on the pipe
+            ok = mbar_wait_bounded(&o_full[(t + nt - 1) & 1], (uint32_t)((t + nt - 1) >> 1) & 1u, abort_flag, a.status);
             if (!ok) break;
             tc_fence_after();
             // Output: every MMA of the item is done, so the Q buffer is free.  Each thread scales its
