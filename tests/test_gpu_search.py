@@ -37,7 +37,8 @@ def _load_both(L, Hq, Hkv, D, B, n, dtype, share_map, max_batch=None):
 
 @pytest.mark.parametrize("L,Hq,Hkv,D,B,n,dtype", [
     (6, 4, 2, 64, 5, 37, "bf16"), (6, 4, 2, 128, 3, 64, "f32"), (5, 2, 1, 128, 7, 129, "bf16"),
-    (32, 8, 8, 128, 6, 64, "bf16"), (40, 4, 2, 64, 4, 33, "bf16"), (80, 2, 1, 64, 2, 16, "bf16")])
+    (32, 8, 8, 128, 6, 64, "bf16"), (40, 4, 2, 64, 4, 33, "bf16"), (80, 2, 1, 64, 2, 16, "bf16"),
+    (8, 4, 4, 128, 3, 600, "bf16"), (5, 2, 2, 128, 2, 1100, "f32")])     # the last two: several chunks per thread block
 def test_layer_distances(L, Hq, Hkv, D, B, n, dtype):
     sm = list(range(L))
     sm[L - 1] = 1                                   # one sharing layer: it has layer 1's cache
@@ -77,7 +78,8 @@ def test_layer_distances_state_errors():
     assert float(d[0, 1]) == 0.0                                   # both layers hold the same rows
 
 
-@pytest.mark.parametrize("S,dim,dtype", [(30, 4096, "bf16"), (3, 10, "f32"), (7, 64 * 5120, "bf16")])
+@pytest.mark.parametrize("S,dim,dtype", [(30, 4096, "bf16"), (3, 10, "f32"), (7, 64 * 5120, "bf16"),
+                                          (3, 3 * 1024 * 1024, "bf16"), (2, 1024 * 1024 + 6, "f32")])   # several passes per block
 def test_mean_cosine(S, dim, dtype):
     cache = SharedKVCache(1, 1, 1, 64, 1, 8, dtype)
     td = torch.bfloat16 if dtype == "bf16" else torch.float32
