@@ -88,6 +88,48 @@ def test_evict_then_decode_with_sharing(dtype, D, Hq, Hkv, context, lo_frac):
     assert cache.unit_len(0, 1, 0) == context + 5 == cache.seq_len(0)
 
 
+@pytest.mark.parametrize("Hq,Hkv,kernel", [(8, 8, 1), (32, 8, 2), (16, 4, 1)])
+def test_ragged_slots_at_sizes_where_a_block_spans_several_units(Hq, Hkv, kernel):
+    """64 or 32 units of up to 3000 rows cut to random lengths between 5 % and 100 %: every thread
+    block's share of the tile line crosses units, many of its tiles lie past a unit's end, and units
+    are shared by several blocks.  Inputs are made on the GPU; sampled (sequence, q-head) pairs are
+    checked against the oracle run as a one-head problem on the kept rows sliced from those inputs,
+    on the computing layer and on the layer that shares its slot, before and after two appends."""
+    D, B, n = 128, 8, 3000
+    sm = [0, 0]
+    cache = SharedKVCache(2, Hq, Hkv, D, B, n + 4, "bf16", share_map=sm)
+    cache.set_option(kb.KVS_OPT_KERNEL, kernel)
+    k = si.normal((9, "rag_big_k", Hq, Hkv), (B, n, Hkv, D), torch.bfloat16, device="cuda")
+    v = si.normal((9, "rag_big_v", Hq, Hkv), (B, n, Hkv, D), torch.bfloat16, device="cuda")
+    cache.append(0, k, v)
+    rng = np.random.default_rng(Hq * 100 + Hkv)
+    keep, n_keep = _random_keep(rng, B, Hkv, np.full((B, Hkv), n), 0.05)
+    cache.evict(0, torch.from_numpy(keep).cuda(), n_keep)
+    G = Hq // Hkv
+    pairs = sorted({(0, 0), (B - 1, Hq - 1)} | {(int(rng.integers(B)), int(rng.integers(Hq))) for _ in range(10)})
+    new_k, new_v = [], []
+    for step in range(3):
+        q = si.normal((9, "rag_big_q", Hq, step), (B, Hq, D), torch.bfloat16, device="cuda")
+        outs = [cache.decode_attention(l, q) for l in range(2)]
+        assert torch.equal(outs[0].view(torch.int32), outs[1].view(torch.int32))     # the sharing layer reads the same slot
+        assert cache.last_launch()["kernel"] == kernel
+        for b, hq in pairs:
+            hk = hq // G
+            rows = torch.from_numpy(keep[b, hk, : n_keep[b, hk]].astype(np.int64)).cuda()
+            kk = torch.cat([k[b, rows, hk]] + [t[b, :, hk] for t in new_k]).double().cpu().numpy()[None, :, None, :]
+            vv = torch.cat([v[b, rows, hk]] + [t[b, :, hk] for t in new_v]).double().cpu().numpy()[None, :, None, :]
+            one = oracle.Oracle(1, 1, 1, D, 1, [0])
+            ref = one.layer_forward(0, q[b : b + 1, hq : hq + 1].double().cpu().numpy(), kk, vv)
+            assert_close(outs[0][b : b + 1, hq : hq + 1].cpu().numpy(), ref, f"step {step} sequence {b} head {hq}")
+            assert cache.unit_len(0, b, hk) == n_keep[b, hk] + step
+        k1 = si.normal((9, "rag_big_k1", Hq, step), (B, 1, Hkv, D), torch.bfloat16, device="cuda")
+        v1 = si.normal((9, "rag_big_v1", Hq, step), (B, 1, Hkv, D), torch.bfloat16, device="cuda")
+        cache.append(0, k1, v1)
+        new_k.append(k1)
+        new_v.append(v1)
+    assert cache.device_status() == 0
+
+
 def test_evict_argument_checks_and_bad_lists():
     sm = [0, 0]
     cache = SharedKVCache(2, 2, 2, 128, 1, 64, "bf16", share_map=sm)
