@@ -174,3 +174,72 @@ def test_replays_past_the_capacity_stop_appending_and_report(Hq, Hkv, evict):
         expect[:, :, 0, 0, :] = False
         expect[:, :, 0, 0, 40:45] = True
     assert torch.equal(changed, expect)
+
+
+@pytest.mark.parametrize("Hq,Hkv", [(8, 8), (32, 8)])
+def test_graph_replay_at_a_size_that_fills_the_gpu(Hq, Hkv):
+    """32 or 64 units of about 2000 rows: every SM has a thread block, blocks span units, and the tile
+    line is recomputed on the device from the replay counter (the context ends three rows before a
+    tile boundary, so the replays cross it).  Sampled (sequence, q-head) pairs of the computing layer
+    and of the layer sharing its slot are checked against the oracle after every replay."""
+    L, D, B, context, replays = 2, 128, 4 if Hkv == 8 and Hq == 32 else 8, 2045, 5
+    sm = [0, 0]
+    cache = SharedKVCache(L, Hq, Hkv, D, B, context + replays + 2, "bf16", share_map=sm)
+    cache.set_option(KVS_OPT_REPLAY, 1)
+    k = si.normal((13, "rp_big_k", Hq), (B, context, Hkv, D), torch.bfloat16, device="cuda")
+    v = si.normal((13, "rp_big_v", Hq), (B, context, Hkv, D), torch.bfloat16, device="cuda")
+    cache.append(0, k, v)
+    qb = torch.empty(B, Hq, D, dtype=torch.bfloat16, device="cuda")
+    kbuf = torch.empty(B, 1, Hkv, D, dtype=torch.bfloat16, device="cuda")
+    vbuf = torch.empty_like(kbuf)
+    ob = [torch.empty(B, Hq, D, dtype=torch.float32, device="cuda") for _ in range(L)]
+    rng = np.random.default_rng(Hq)
+    G = Hq // Hkv
+    pairs = sorted({(0, 0), (B - 1, Hq - 1)} | {(int(rng.integers(B)), int(rng.integers(Hq))) for _ in range(6)})
+    ks, vs = [k], [v]
+
+    def fill(t):
+        qb.copy_(si.normal((13, "rp_big_q", Hq, t), (B, Hq, D), torch.bfloat16, device="cuda"))
+        kbuf.copy_(si.normal((13, "rp_big_k1", Hq, t), (B, 1, Hkv, D), torch.bfloat16, device="cuda"))
+        vbuf.copy_(si.normal((13, "rp_big_v1", Hq, t), (B, 1, Hkv, D), torch.bfloat16, device="cuda"))
+        ks.append(kbuf.clone())
+        vs.append(vbuf.clone())
+
+    def one_step():
+        cache.append(0, kbuf, vbuf)
+        cache.decode_attention(0, qb, ob[0])
+        cache.decode_attention(1, qb, ob[1])
+        cache.replay_advance()
+
+    def check(what):
+        torch.cuda.synchronize()
+        assert torch.equal(ob[0].view(torch.int32), ob[1].view(torch.int32))
+        kall, vall = torch.cat(ks, dim=1), torch.cat(vs, dim=1)
+        for b, hq in pairs:
+            hk = hq // G
+            one = oracle.Oracle(1, 1, 1, D, 1, [0])
+            ref = one.layer_forward(0, qb[b : b + 1, hq : hq + 1].double().cpu().numpy(),
+                                    kall[b : b + 1, :, hk : hk + 1].double().cpu().numpy(),
+                                    vall[b : b + 1, :, hk : hk + 1].double().cpu().numpy())
+            assert_close(ob[0][b : b + 1, hq : hq + 1].cpu().numpy(), ref, f"{what} sequence {b} head {hq}")
+
+    fill(0)
+    one_step()                                   # eager
+    check("eager step")
+    fill(1)
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            one_step()
+    for r in range(replays):
+        if r > 0:
+            fill(1 + r)
+        graph.replay()
+        check(f"replay {r}")
+    cache.replay_commit(replays)
+    torch.cuda.synchronize()
+    assert cache.device_status() == 0 and cache.seq_len(1) == context + 1 + replays
+    kall = torch.cat(ks, dim=1)
+    assert torch.equal(cache.plane(0, 0)[:B, :, : context + 1 + replays], kall.permute(0, 2, 1, 3))
