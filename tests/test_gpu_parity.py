@@ -292,6 +292,36 @@ def test_step_host_equals_per_layer_calls(layers, chunks):
     assert torch.equal(a.pool, b.pool)
 
 
+@pytest.mark.parametrize("chunks", [1, 4])
+def test_step_host_at_a_size_with_long_kernels(chunks):
+    """Eight layers of the 7B shape at 2000 rows: every attention kernel runs for tens of
+    microseconds, so a copy that did not wait for its kernel (or a kernel for its copy) would show.
+    The whole-step call from host buffers must give the bits of the per-layer calls, outputs and
+    cached rows, over three steps."""
+    L, Hq, D, B, n = 8, 32, 128, 8, 2000
+    w = si.Workload("host_big", L=L, Hq=Hq, Hkv=Hq, D=D, B=B, context=n, dtype="bf16", n_shared=2, map_seed=3, steps=3)
+    sm = w.share_map()
+    a, b = make_cache(w, 4), make_cache(w, 4)
+    a.set_option(kb.KVS_OPT_HOST_CHUNKS, chunks)
+    for l in range(L):
+        if sm[l] != l:
+            continue
+        k, v = si.context_kv(w, l, device="cuda")
+        a.append(l, k, v)
+        b.append(l, k, v)
+    for t in range(3):
+        qs, ks, vs = zip(*[si.step_qkv(w, t, l) for l in range(L)])
+        qh, kh, vh = torch.stack(qs).pin_memory(), torch.stack(ks).pin_memory(), torch.stack(vs).pin_memory()
+        oh = torch.full((L, B, Hq, D), float("nan"), dtype=torch.float32).pin_memory()
+        a.step_host(qh, kh, vh, oh)
+        for l in range(L):
+            if sm[l] == l:
+                b.append(l, ks[l].cuda(), vs[l].cuda())
+            assert torch.equal(b.decode_attention(l, qs[l].cuda()).cpu(), oh[l]), (t, l)
+    torch.cuda.synchronize()
+    assert torch.equal(a.pool, b.pool) and a.device_status() == 0
+
+
 def test_read_roof_checksum():
     x = torch.randint(0, 2**31 - 1, (3 * 32768 // 4 * 7,), dtype=torch.int32, device="cuda")
     chk = torch.zeros(1, dtype=torch.int64, device="cuda")
