@@ -60,36 +60,39 @@ def test_head_size_64(Hq, Hkv, chunks):
     _prefill_both(Hq, Hkv, 2, chunks, [0, 0, 2, 0], D=64)
 
 
-@pytest.mark.parametrize("D,Hq,Hkv,B,T", [(128, 32, 8, 2, 2100), (128, 16, 16, 3, 1500), (64, 32, 8, 2, 2100),
-                                          (128, 32, 32, 2, 4096)])   # the last one: the shape prefill_bench times
-def test_many_items_per_block_sampled_heads(D, Hq, Hkv, B, T):
+@pytest.mark.parametrize("D,Hq,Hkv,B,chunks", [(128, 32, 8, 2, [2100]), (128, 16, 16, 3, [1500]), (64, 32, 8, 2, [2100]),
+                                               (128, 32, 8, 2, [1000, 1100]),
+                                               (128, 32, 32, 2, [4096])])   # the last one: the shape prefill_bench times
+def test_many_items_per_block_sampled_heads(D, Hq, Hkv, B, chunks):
     """Sizes at which every persistent block works through several (query block, head) items one after the
     other (item ring, barrier phases and the output staging carried across items, K/V groups that do
-    not all fit the scheduling group).  The inputs are generated on the GPU; the oracle gets the
-    rows of sampled (sequence, q-head) pairs sliced from those same tensors, each run as a one-head
-    problem, and every query row of a sampled pair is compared."""
+    not all fit the scheduling group), with the prompt in one piece or in two.  The inputs are generated
+    on the GPU; the oracle gets the rows of sampled (sequence, q-head) pairs sliced from those same
+    tensors, each run as a one-head problem, and every query row of a sampled pair is compared."""
     sm = [0, 0]
-    cache = SharedKVCache(2, Hq, Hkv, D, B, T, "bf16", share_map=sm)
-    k = si.normal((5, "pf_big_k", D, Hq, T), (B, T, Hkv, D), torch.bfloat16, device="cuda")
-    v = si.normal((5, "pf_big_v", D, Hq, T), (B, T, Hkv, D), torch.bfloat16, device="cuda")
-    q = si.normal((5, "pf_big_q", D, Hq, T), (B, T, Hq, D), torch.bfloat16, device="cuda")
-    cache.append(0, k, v)
-    outs = [cache.prefill_attention(l % 2, q) for l in range(6)]  # own slot and the sharing layer in turn
-    torch.cuda.synchronize()
-    assert cache.device_status() == 0
-    for o in outs[1:]:                                             # same slot, same queries: the same bits,
-        assert torch.equal(o.view(torch.int32), outs[0].view(torch.int32))   # whichever block ran which item
-    assert torch.isfinite(outs[0]).all()
+    total = sum(chunks)
+    cache = SharedKVCache(2, Hq, Hkv, D, B, total, "bf16", share_map=sm)
     G = Hq // Hkv
     rng = np.random.default_rng(11)
-    pairs = {(0, 0), (B - 1, Hq - 1)} | {(int(rng.integers(B)), int(rng.integers(Hq))) for _ in range(10)}
-    for b, hq in sorted(pairs):
-        hk = hq // G
-        one = oracle.Oracle(1, 1, 1, D, 1, [0])
-        ref = one.layer_prefill(0, q[b : b + 1, :, hq : hq + 1].double().cpu().numpy(),
-                                k[b : b + 1, :, hk : hk + 1].double().cpu().numpy(),
-                                v[b : b + 1, :, hk : hk + 1].double().cpu().numpy())
-        assert_close(outs[0][b : b + 1, :, hq : hq + 1].cpu().numpy(), ref, f"sequence {b} head {hq}")
+    pairs = sorted({(0, 0), (B - 1, Hq - 1)} | {(int(rng.integers(B)), int(rng.integers(Hq))) for _ in range(10)})
+    ones = {p: oracle.Oracle(1, 1, 1, D, 1, [0]) for p in pairs}
+    for c, T in enumerate(chunks):
+        k = si.normal((5, "pf_big_k", D, Hq, total, c), (B, T, Hkv, D), torch.bfloat16, device="cuda")
+        v = si.normal((5, "pf_big_v", D, Hq, total, c), (B, T, Hkv, D), torch.bfloat16, device="cuda")
+        q = si.normal((5, "pf_big_q", D, Hq, total, c), (B, T, Hq, D), torch.bfloat16, device="cuda")
+        cache.append(0, k, v)
+        outs = [cache.prefill_attention(l % 2, q) for l in range(6)]  # own slot and the sharing layer in turn
+        torch.cuda.synchronize()
+        assert cache.device_status() == 0
+        for o in outs[1:]:                                             # same slot, same queries: the same bits,
+            assert torch.equal(o.view(torch.int32), outs[0].view(torch.int32))   # whichever block ran which item
+        assert torch.isfinite(outs[0]).all()
+        for b, hq in pairs:
+            hk = hq // G
+            ref = ones[(b, hq)].layer_prefill(0, q[b : b + 1, :, hq : hq + 1].double().cpu().numpy(),
+                                              k[b : b + 1, :, hk : hk + 1].double().cpu().numpy(),
+                                              v[b : b + 1, :, hk : hk + 1].double().cpu().numpy())
+            assert_close(outs[0][b : b + 1, :, hq : hq + 1].cpu().numpy(), ref, f"chunk {c} sequence {b} head {hq}")
 
 
 def test_prefill_then_decode_continues_from_the_same_cache():
