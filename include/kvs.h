@@ -82,6 +82,7 @@ typedef struct {
     uint64_t prefill_launches;    /* tensor-core prefill kernels launched                    */
     uint64_t evict_launches;      /* kvs_evict calls that launched                           */
     uint64_t search_launches;     /* kernels launched by kvs_layer_distances / kvs_mean_cosine */
+    uint64_t fused_appends;       /* kvs_decode_step calls whose append rode in the split-K kernel */
 } kvs_stats_t;
 
 /* Tuning knobs for kvs_set_option.  Defaults are chosen by the library. */
@@ -172,6 +173,21 @@ kvs_status kvs_append(kvs_ctx* ctx, int32_t layer, const void* k, const void* v,
 kvs_status kvs_decode_attention(kvs_ctx* ctx, int32_t layer, const void* q, float* out,
                                 int32_t batch, void* stream);
 
+/* One decode step of one layer: kvs_append of one token (n_new = 1) followed by
+ * kvs_decode_attention, with the same arguments, layouts, results and errors as those two
+ * calls in that order (Section 3.2; on a layer whose cache is replaced k and v are not read and
+ * may be NULL, and nothing is appended).
+ *   q: device, [batch][n_q_heads][head_dim];  k, v: device, [batch][1][n_kv_heads][head_dim];
+ *   out: device, float32 [batch][n_q_heads][head_dim]
+ * On a computing layer whose slot nothing was evicted from (and with k, v 16-byte aligned) no
+ * append kernel is launched: the split-K kernel stores the new row itself -- the thread block
+ * whose share of the rows ends a (sequence, kv-head) unit writes that unit's row to the slot just
+ * before it fetches the tile that holds it -- so the step is two launches instead of three.  k and
+ * v must stay valid until the call's work on `stream` has run.  Cached bits and output are those
+ * of the two separate calls, bit for bit.  Otherwise the two calls are made as they are.        */
+kvs_status kvs_decode_step(kvs_ctx* ctx, int32_t layer, const void* q, const void* k, const void* v,
+                           float* out, int32_t batch, void* stream);
+
 /* Prefill attention of one layer (Section 3.2: the strategy is applied to the prefill pass
  * as it is to generation).  The n_q queries per head are the newest n_q positions of the cache
  * the layer uses (its own slot, or its source layer's), i.e. call it after kvs_append has
@@ -247,7 +263,8 @@ kvs_status kvs_mean_cosine(kvs_ctx* ctx, const void* a, const void* b, int32_t n
  *     not counted), call kvs_replay_commit(ctx, times_run, stream): the host lengths catch up
  *     (times_run - 1 more rows) and the counter is cleared on `stream`.  Make no eager call on
  *     the context between the first replay and the commit.
- *   - One-token decode steps only; every computing layer must append exactly once per step.
+ *   - One-token decode steps only; every computing layer must append exactly once per step
+ *     (kvs_append or kvs_decode_step).
  *   - A replay that would pass max_seq appends nothing for that layer and sets the device status
  *     word to KVS_ERR_CAPACITY; kvs_replay_commit returns CAPACITY instead of advancing.
  * Errors: STATE unless bound and KVS_OPT_REPLAY is 1; INVALID_ARG for times_run < 1.            */

@@ -77,6 +77,19 @@ class SharedKVCache:
         binding.kvs_decode_attention(self.ctx, layer, q, out, q.shape[0], self._stream())
         return out
 
+    def decode_step(self, layer, q, k=None, v=None, out=None):
+        """Append one token's k, v (``[batch][1][n_kv_heads][head_dim]``; None on a sharing layer) and attend
+        with q: ``append`` then ``decode_attention`` in one call, the append riding in the attention kernel."""
+        torch = self._torch
+        assert q.is_contiguous() and q.dtype == self.dtype and q.shape[1:] == (self.shape[1], self.shape[3])
+        if k is not None:
+            assert k.is_contiguous() and v.is_contiguous() and k.dtype == self.dtype and v.dtype == self.dtype
+            assert k.shape == v.shape == (q.shape[0], 1, self.shape[2], self.shape[3])
+        if out is None:
+            out = torch.empty(q.shape, dtype=torch.float32, device=self.device)
+        binding.kvs_decode_step(self.ctx, layer, q, k, v, out, q.shape[0], self._stream())
+        return out
+
     def prefill_attention(self, layer, q, out=None):
         """q: ``[batch][n_q][n_q_heads][head_dim]`` (the newest n_q positions, causal); returns float32 of that shape."""
         torch = self._torch

@@ -40,7 +40,7 @@ EXPORTS = (
     "kvs_last_device_status", "kvs_set_option", "kvs_last_launch", "kvs_status_string",
     "kvs_read_roof", "kvs_decode_attention_static", "kvs_prefill_attention",
     "kvs_evict", "kvs_unit_len", "kvs_layer_distances", "kvs_mean_cosine",
-    "kvs_replay_advance", "kvs_replay_commit",
+    "kvs_replay_advance", "kvs_replay_commit", "kvs_decode_step",
 )
 
 
@@ -58,7 +58,7 @@ class kvs_stats_t(ctypes.Structure):
         ("attention_launches", ctypes.c_uint64), ("combine_launches", ctypes.c_uint64),
         ("kv_bytes_read", ctypes.c_uint64), ("kv_bytes_appended", ctypes.c_uint64),
         ("prefill_launches", ctypes.c_uint64), ("evict_launches", ctypes.c_uint64),
-        ("search_launches", ctypes.c_uint64),
+        ("search_launches", ctypes.c_uint64), ("fused_appends", ctypes.c_uint64),
     ]
 
 
@@ -86,6 +86,7 @@ def load() -> ctypes.CDLL:
         "kvs_reset": [vp],
         "kvs_append": [vp, i32, vp, vp, i32, i32, vp],
         "kvs_decode_attention": [vp, i32, vp, vp, i32, vp],
+        "kvs_decode_step": [vp, i32, vp, vp, vp, vp, i32, vp],
         "kvs_decode_attention_static": [vp, i32, vp, vp, i32, vp, vp],
         "kvs_prefill_attention": [vp, i32, vp, vp, i32, i32, vp],
         "kvs_evict": [vp, i32, vp, P(i32), i32, i32, vp],
@@ -179,6 +180,10 @@ def kvs_append(ctx: int, layer: int, k, v, batch: int, n_new: int, stream: int =
 
 def kvs_decode_attention(ctx: int, layer: int, q, out, batch: int, stream: int = 0) -> None:
     _check(load().kvs_decode_attention(ctx, layer, _ptr(q), _ptr(out), batch, stream), "kvs_decode_attention")
+
+
+def kvs_decode_step(ctx: int, layer: int, q, k, v, out, batch: int, stream: int = 0) -> None:
+    _check(load().kvs_decode_step(ctx, layer, _ptr(q), _ptr(k), _ptr(v), _ptr(out), batch, stream), "kvs_decode_step")
 
 
 def kvs_prefill_attention(ctx: int, layer: int, q, out, batch: int, n_q: int, stream: int = 0) -> None:

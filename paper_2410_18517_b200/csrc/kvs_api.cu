@@ -264,8 +264,11 @@ bool choose_plan(const kvs_ctx* c, int units, int n, kvs::DecodePlan* plan) {
 }
 
 // Split-K kernel + combine kernel of one layer, with the given plan and scratch.
+// With k_new / v_new the split-K kernel also appends that one row per unit (the slot's length must
+// already count it).
 kvs_status run_attention(kvs_ctx* c, int slot, const void* q, float* out, int batch, const kvs::DecodePlan& plan,
-                         bool use_mma, const AttentionScratch& scratch, cudaStream_t st) {
+                         bool use_mma, const AttentionScratch& scratch, cudaStream_t st, const void* k_new = nullptr,
+                         const void* v_new = nullptr) {
     kvs::DecodeArgs a;
     a.q = q;
     a.kplane = c->pool + (size_t)(2 * slot) * c->plane_bytes;
@@ -286,6 +289,9 @@ kvs_status run_attention(kvs_ctx* c, int slot, const void* q, float* out, int ba
     a.safe_rows = scratch.programmatic ? safe_rows_of(c, slot) : 0;
     a.unit_len = c->ragged[slot] ? unit_len_dev(c, slot) : nullptr;
     a.n_extra = replay_counter(c);
+    a.k_new = k_new;
+    a.v_new = v_new;
+    if (k_new) a.safe_rows = std::min(a.safe_rows, a.n - 1);   // the new row is fetched after the kernel has stored it
     c->seq += 2;                       // split-K kernel, then combine
     c->last_splitk_seq = c->seq - 1;
     if (use_mma) {
@@ -307,6 +313,33 @@ kvs_status run_attention(kvs_ctx* c, int slot, const void* q, float* out, int ba
     } else {
         c->stats.kv_bytes_read += 2ull * a.units * a.n * c->row_bytes;
     }
+    return KVS_OK;
+}
+
+// One decode step of a computing layer with the append riding in the split-K kernel (the caller
+// has checked the arguments; the slot is not ragged).
+kvs_status do_fused_step(kvs_ctx* c, int layer, const void* q, const void* k, const void* v, float* out, int batch,
+                         cudaStream_t st) {
+    const int slot = c->slot_of_layer[layer];
+    const int old_len = c->slot_len[slot];
+    kvs::DecodePlan plan;
+    const bool use_mma = choose_plan(c, batch * c->cfg.n_kv_heads, old_len + 1, &plan);
+    const AttentionScratch scratch = {reinterpret_cast<float*>(c->ws + c->off_part_o),
+                                      reinterpret_cast<float*>(c->ws + c->off_part_ml),
+                                      reinterpret_cast<int*>(c->ws + c->off_status), take_early_start(c)};
+    // run_attention works out which rows are stable from the appends before this one
+    c->slot_len[slot] = old_len + 1;
+    const kvs_status s = run_attention(c, slot, q, out, batch, plan, use_mma, scratch, st, k, v);
+    if (s != KVS_OK) {
+        c->slot_len[slot] = old_len;
+        return s;
+    }
+    c->app_seq_prev[slot] = c->app_seq_latest[slot];
+    c->app_seq_latest[slot] = c->last_splitk_seq;   // the kernel that appended is the split-K kernel itself
+    c->app_start_latest[slot] = old_len;
+    c->cur_batch = batch;
+    c->stats.fused_appends += 1;
+    c->stats.kv_bytes_appended += 2ull * batch * c->cfg.n_kv_heads * c->row_bytes;
     return KVS_OK;
 }
 
@@ -468,6 +501,31 @@ kvs_status kvs_decode_attention(kvs_ctx* ctx, int32_t layer, const void* q, floa
     DeviceGuard guard(ctx->cfg.device);
     if (!guard.ok) return KVS_ERR_CUDA;
     return do_attention(ctx, layer, q, out, batch, static_cast<cudaStream_t>(stream));
+}
+
+kvs_status kvs_decode_step(kvs_ctx* ctx, int32_t layer, const void* q, const void* k, const void* v, float* out,
+                           int32_t batch, void* stream) {
+    bool sharing = false;
+    kvs_status s = check_append(ctx, layer, k, v, batch, 1, &sharing);
+    if (s != KVS_OK) return s;
+    if (!q || !out) return KVS_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (sharing) {
+        s = check_attention(ctx, layer, q, out, batch);
+        if (s != KVS_OK) return s;
+        DeviceGuard guard(ctx->cfg.device);
+        if (!guard.ok) return KVS_ERR_CUDA;
+        ctx->stats.append_skipped += 1;
+        return do_attention(ctx, layer, q, out, batch, st);
+    }
+    DeviceGuard guard(ctx->cfg.device);
+    if (!guard.ok) return KVS_ERR_CUDA;
+    const int slot = ctx->slot_of_layer[layer];
+    const bool aligned = ((uintptr_t)k % 16) == 0 && ((uintptr_t)v % 16) == 0;
+    if (aligned && !ctx->ragged[slot]) return do_fused_step(ctx, layer, q, k, v, out, batch, st);
+    s = do_append(ctx, layer, k, v, batch, 1, st);
+    if (s != KVS_OK) return s;
+    return do_attention(ctx, layer, q, out, batch, st);
 }
 
 kvs_status kvs_prefill_attention(kvs_ctx* ctx, int32_t layer, const void* q, float* out, int32_t batch, int32_t n_q,

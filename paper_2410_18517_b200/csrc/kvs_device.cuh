@@ -160,3 +160,36 @@ inline cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block
 }
 
 }  // namespace kvs
+
+namespace kvs {
+
+// The append of a decode step done by the attention kernel itself.  Called by all lanes of the
+// producer warp of a split-K kernel, after the wait for the previous kernel: for every unit whose
+// last tile lies in this block's share [t0, t1) of the tile line, the unit's new row (row n-1, not
+// in the pool yet) is stored from the caller's buffers k_new / v_new ([units][RB] bytes) to the K
+// and V planes.  Only this block ever fetches that tile, and it does so after this call: the
+// proxy fence orders the warp's plain stores before the bulk (asynchronous-proxy) copies that
+// lane 0 issues next.
+template <int RB>
+__device__ __forceinline__ void store_new_rows(int lane, long long t0, long long t1, int tpu, int n, int row_stride,
+                                               const char* k_new, const char* v_new, char* kplane, char* vplane) {
+    constexpr int LPR = RB / 16;
+    if (t1 > t0) {
+        const long long u0 = t0 / tpu, u1 = (t1 - 1) / tpu;
+        for (long long u = u0; u <= u1; ++u) {
+            const long long last = u * tpu + tpu - 1;
+            if (last < t0 || last >= t1) continue;
+            const long long dst = (u * row_stride + (n - 1)) * (long long)RB;
+            for (int i = lane; i < 2 * LPR; i += 32) {
+                const bool isv = i >= LPR;
+                const int c = isv ? i - LPR : i;
+                const uint4 val = *reinterpret_cast<const uint4*>((isv ? v_new : k_new) + u * RB + c * 16);
+                *reinterpret_cast<uint4*>((isv ? vplane : kplane) + dst + c * 16) = val;
+            }
+        }
+    }
+    asm volatile("fence.proxy.async.global;" ::: "memory");
+    __syncwarp();
+}
+
+}  // namespace kvs

@@ -259,6 +259,8 @@ struct ScalarKernelArgs {
     const int* n_extra;   // graph replay: rows every slot has grown by since the launch was recorded, or nullptr
     int units;
     int cap;              // rows a unit can hold: lengths that grew on the device are cut off there
+    const char* k_new;    // the step's new rows, appended by this kernel (n counts them), or nullptr
+    const char* v_new;
 };
 
 template <typename T, int D, int G, int GEOM>
@@ -266,10 +268,12 @@ __global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G, GEOM>::MI
     decode_splitk_scalar(const ScalarKernelArgs a_in) {
     using S = ScalarShape<T, D, G, GEOM>;
     ScalarKernelArgs a = a_in;
+    bool over = false;    // a replayed launch with an append that would pass the capacity
     if (a.n_extra != nullptr) {
         // A replayed launch: the lengths recorded with it have grown on the device since.  The
         // counter is stable here without a wait: the host gives the first launch after every write
         // of the counter a full dependency, so that write is complete before any reader starts.
+        over = a.n + *a.n_extra > a.cap;
         a.n = min(a.n + *a.n_extra, a.cap);   // a replay that outran the capacity appended nothing more
         a.tpu = (a.n + S::TN - 1) / S::TN;
         a.T = (long long)a.units * a.tpu;
@@ -305,7 +309,9 @@ __global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G, GEOM>::MI
 
     if (warp == kConsumerWarps) {
         // ------------------------------ producer ------------------------------
-        if (lane == 0) {
+        // Lane 0 issues the copies; the whole warp stores the step's new rows when the launch
+        // carries an append.
+        {
             // Issue the copies of tile `gt` into stage `st`.  kv / qpart select which of the
             // stage's copies are issued now; the barrier is armed with the stage's full byte
             // count by whichever call comes first (arm = true).
@@ -335,14 +341,24 @@ __global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G, GEOM>::MI
             // tiles made entirely of rows that no kernel still in flight can be writing are
             // fetched (rows below safe_rows); q and everything else come after the wait.
             int npre = 0;
-            for (; npre < STAGES && t0 + npre < t1; ++npre) {
-                const long long gt = t0 + npre;
-                const int ti = (int)(gt % a.tpu);
-                if ((long long)(ti + 1) * TN > a.safe_rows) break;
-                issue(gt, npre, true, true, false);
+            if (lane == 0) {
+                for (; npre < STAGES && t0 + npre < t1; ++npre) {
+                    const long long gt = t0 + npre;
+                    const int ti = (int)(gt % a.tpu);
+                    if ((long long)(ti + 1) * TN > a.safe_rows) break;
+                    issue(gt, npre, true, true, false);
+                }
             }
             pdl_wait();
             pdl_launch_dependents();
+            if (a.k_new != nullptr) {
+                if (!over)
+                    store_new_rows<RB>(lane, t0, t1, a.tpu, a.n, a.row_stride, a.k_new, a.v_new, const_cast<char*>(a.kplane),
+                                       const_cast<char*>(a.vplane));
+                else if (lane == 0 && blockIdx.x == 0)
+                    atomicExch(a.status, 4);
+            }
+            if (lane != 0) return;
             for (int j = 0; j < npre; ++j) issue(t0 + j, j, false, false, true);
             int it = npre;
             bool ok = true;
@@ -632,6 +648,8 @@ cudaError_t launch_decode_scalar(const DecodeArgs& a, const DecodePlan& plan, cu
     ka.n_extra = a.n_extra;
     ka.units = a.units;
     ka.cap = a.capacity;
+    ka.k_new = (const char*)a.k_new;
+    ka.v_new = (const char*)a.v_new;
     const bool pdl = a.programmatic;
     if (a.dtype == 0) {
         if (a.D == 128) return launch_scalar_groups<__nv_bfloat16, 128>(a.G, plan.geom, ka, plan.NC, pdl, stream);

@@ -41,6 +41,8 @@ struct DecodeArgs {
     const int* n_extra;   // device int: rows grown since the launch was recorded (graph replay), or nullptr
     int safe_rows;        // rows per unit that no kernel possibly still in flight is writing
     bool programmatic;    // launch with programmatic stream serialization (early start, explicit wait)
+    const void* k_new;    // [B][1][Hkv][D] rows the launch also appends (n already counts them), or nullptr
+    const void* v_new;
 };
 
 // Largest number of thread blocks any plan may use (sizes the partial buffers).

@@ -108,6 +108,10 @@ struct MmaKernelArgs {
     const int* n_extra;  // graph replay: rows every slot has grown by since the launch was recorded, or nullptr
     int units;
     int cap;             // rows a unit can hold: lengths that grew on the device are cut off there
+    const char* k_new;   // the step's new rows, appended by this kernel (n counts them), or nullptr
+    const char* v_new;
+    char* kplane;        // planes of the slot (for the append; the tiles are fetched through the tensor map)
+    char* vplane;
 };
 
 // G (q-heads per kv-head, 1..8) is a run-time argument: it only selects which rows of the padded
@@ -117,10 +121,12 @@ __global__ void __launch_bounds__(kMmaThreads, KVS_MMA_BLOCKS_PER_SM)
     decode_splitk_mma(const __grid_constant__ CUtensorMap tmap, const MmaKernelArgs a_in) {
     using S = MmaShape<D>;
     MmaKernelArgs a = a_in;
+    bool over = false;    // a replayed launch with an append that would pass the capacity
     if (a.n_extra != nullptr) {
         // A replayed launch: the lengths recorded with it have grown on the device since.  The
         // counter is stable here without a wait: the host gives the first launch after every write
         // of the counter a full dependency, so that write is complete before any reader starts.
+        over = a.n + *a.n_extra > a.cap;
         a.n = min(a.n + *a.n_extra, a.cap);   // a replay that outran the capacity appended nothing more
         a.tpu = (a.n + S::TN - 1) / S::TN;
         a.T = (long long)a.units * a.tpu;
@@ -155,7 +161,9 @@ __global__ void __launch_bounds__(kMmaThreads, KVS_MMA_BLOCKS_PER_SM)
 
     if (warp == kMmaWarps) {
         // ------------------------------ producer ------------------------------
-        if (lane == 0) {
+        // Lane 0 issues the copies; the whole warp stores the step's new rows when the launch
+        // carries an append.
+        {
             // Issue the copies of tile `gt` into stage `st` (see the scalar kernel: the barrier
             // is armed once with the stage's full byte count, K/V and q may be issued apart).
             auto issue = [&](long long gt, int st, bool arm, bool kv, bool qpart) {
@@ -188,14 +196,23 @@ __global__ void __launch_bounds__(kMmaThreads, KVS_MMA_BLOCKS_PER_SM)
             // Until the preceding kernel in the stream is known to have finished, fetch only
             // K/V tiles made entirely of rows that no kernel still in flight can be writing.
             int npre = 0;
-            for (; npre < kMmaStages && t0 + npre < t1; ++npre) {
-                const long long gt = t0 + npre;
-                const int ti = (int)(gt % a.tpu);
-                if ((long long)(ti + 1) * TN > a.safe_rows) break;
-                issue(gt, npre, true, true, false);
+            if (lane == 0) {
+                for (; npre < kMmaStages && t0 + npre < t1; ++npre) {
+                    const long long gt = t0 + npre;
+                    const int ti = (int)(gt % a.tpu);
+                    if ((long long)(ti + 1) * TN > a.safe_rows) break;
+                    issue(gt, npre, true, true, false);
+                }
             }
             pdl_wait();
             pdl_launch_dependents();
+            if (a.k_new != nullptr) {
+                if (!over)
+                    store_new_rows<S::RB>(lane, t0, t1, a.tpu, a.n, a.row_stride, a.k_new, a.v_new, a.kplane, a.vplane);
+                else if (lane == 0 && blockIdx.x == 0)
+                    atomicExch(a.status, 4);
+            }
+            if (lane != 0) return;
             for (int j = 0; j < npre; ++j) issue(t0 + j, j, false, false, true);
             int it = npre;
             bool ok = true;
@@ -449,6 +466,10 @@ cudaError_t launch_decode_mma(const DecodeArgs& a, const DecodePlan& plan, const
     ka.n_extra = a.n_extra;
     ka.units = a.units;
     ka.cap = a.capacity;
+    ka.k_new = (const char*)a.k_new;
+    ka.v_new = (const char*)a.v_new;
+    ka.kplane = (char*)const_cast<void*>(a.kplane);
+    ka.vplane = (char*)const_cast<void*>(a.vplane);
     if (a.G < 1 || a.G > 8) return cudaErrorInvalidValue;
     if (a.D == 128) return launch_one<128>(tm, ka, plan.NC, a.programmatic, stream);
     if (a.D == 64) return launch_one<64>(tm, ka, plan.NC, a.programmatic, stream);

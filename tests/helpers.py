@@ -30,9 +30,10 @@ def make_cache(w: si.Workload, extra_rows: int, share_map=None, device=0, scale=
                          softmax_scale=scale, device=device)
 
 
-def run_small(w: si.Workload, steps: int, share_map=None, options=(), check_cache=True, scale=None):
+def run_small(w: si.Workload, steps: int, share_map=None, options=(), check_cache=True, scale=None, use_step=False):
     """Whole-workload comparison: context load, then `steps` decode steps, every output and
-    (optionally) every cached bit compared.  Inputs are generated on the CPU and copied."""
+    (optionally) every cached bit compared.  Inputs are generated on the CPU and copied.  With
+    `use_step` a decode step goes through kvs_decode_step instead of kvs_append + kvs_decode_attention."""
     sm = np.asarray(w.share_map() if share_map is None else share_map)
     cache = make_cache(w, steps, sm, scale=0.0 if scale is None else scale)
     for opt, val in options:
@@ -50,8 +51,12 @@ def run_small(w: si.Workload, steps: int, share_map=None, options=(), check_cach
         for l in range(w.L):
             q, k, v = si.step_qkv(w, t, l)
             ref = orc.layer_forward(l, q.double().numpy(), k.double().numpy(), v.double().numpy())
-            cache.append(l, k.to(dev), v.to(dev))
-            out = cache.decode_attention(l, q.to(dev))
+            if use_step:
+                own = sm[l] == l
+                out = cache.decode_step(l, q.to(dev), k.to(dev) if own else None, v.to(dev) if own else None)
+            else:
+                cache.append(l, k.to(dev), v.to(dev))
+                out = cache.decode_attention(l, q.to(dev))
             e = assert_close(out.cpu().numpy(), ref, f"{w.name} step {t} layer {l}")
             worst = (max(worst[0], e[0]), max(worst[1], e[1]))
             assert cache.seq_len(l) == orc.length(l)

@@ -22,7 +22,8 @@ def _built():
 
 @pytest.mark.parametrize("Hq,Hkv,dtype,context,evict", [(4, 4, "bf16", 300, False), (8, 2, "bf16", 127, False),
                                                          (4, 2, "f32", 60, False), (8, 2, "bf16", 200, True)])
-def test_graph_replay_is_the_next_step_every_time(Hq, Hkv, dtype, context, evict):
+@pytest.mark.parametrize("use_step", [False, True])
+def test_graph_replay_is_the_next_step_every_time(Hq, Hkv, dtype, context, evict, use_step):
     sm = [0, 1, 2, 1]
     L, D, B, replays = 4, 128, 2, 6
     w = si.Workload(f"replay_{Hq}_{Hkv}_{dtype}", L=L, Hq=Hq, Hkv=Hkv, D=D, B=B, context=context, dtype=dtype,
@@ -59,6 +60,10 @@ def test_graph_replay_is_the_next_step_every_time(Hq, Hkv, dtype, context, evict
 
     def one_step():
         for l in range(L):
+            if use_step:                         # kvs_decode_step: the append rides in the attention kernel
+                own = sm[l] == l
+                cache.decode_step(l, qb[l], kbuf[l] if own else None, vbuf[l] if own else None, ob[l])
+                continue
             if sm[l] == l:
                 cache.append(l, kbuf[l], vbuf[l])
             else:
@@ -122,8 +127,9 @@ def test_replay_calls_need_the_option():
     assert e.value.status == kb.KVS_ERR_CAPACITY
 
 
-@pytest.mark.parametrize("Hq,Hkv,evict", [(4, 4, False), (8, 2, False), (4, 2, True)])
-def test_replays_past_the_capacity_stop_appending_and_report(Hq, Hkv, evict):
+@pytest.mark.parametrize("Hq,Hkv,evict,use_step", [(4, 4, False, False), (8, 2, False, False), (4, 2, True, False),
+                                                    (4, 4, False, True), (8, 2, False, True)])
+def test_replays_past_the_capacity_stop_appending_and_report(Hq, Hkv, evict, use_step):
     """Capacity 128 rows (one whole row stride), 126 cached, the recorded step makes 127: the replays
     after the first would need rows 128, 129, ...  The kernels' own checks append nothing there, attend
     over the rows that exist, set the status word, and the commit refuses; no row outside a unit is
@@ -145,8 +151,11 @@ def test_replays_past_the_capacity_stop_appending_and_report(Hq, Hkv, evict):
     out = torch.empty(B, Hq, D, dtype=torch.float32, device="cuda")
 
     def one_step():
-        cache.append(0, kk, vv)
-        cache.decode_attention(0, q, out)
+        if use_step:
+            cache.decode_step(0, q, kk, vv, out)
+        else:
+            cache.append(0, kk, vv)
+            cache.decode_attention(0, q, out)
         cache.decode_attention(1, q, out)
         cache.replay_advance()
 
