@@ -4,7 +4,8 @@ tokens/s, KV-read GB/s and pool size.
 
     python -m paper_2410_18517_b200.sweep [--out FILE] [--steps K] [--only B,N,P] [--shared P] [--kernel K]
 
-A *step* is one pass over all layers (append on computing layers + attention on every layer).
+A *step* is one pass over all layers (kvs_decode_step per layer: append on computing layers, riding in
+the attention kernel, + attention on every layer).
 --kernel forces KVS_OPT_KERNEL (1 scalar, 2 tensor-core) instead of the library's own choice.
 Each point is timed twice: launched call by call from Python, and as replays of a CUDA graph of one
 recorded step (which takes the host's launch cost out; with the library's replay counter every
@@ -55,9 +56,8 @@ def time_point(w: si.Workload, steps: int, device=0, kernel=0) -> dict:
     def one_step(replay=False):
         for l in range(w.L):
             q, kk, vv = ins[l]
-            if sm[l] == l:
-                cache.append(l, kk, vv)
-            cache.decode_attention(l, q, outs[l])
+            own = sm[l] == l
+            cache.decode_step(l, q, kk if own else None, vv if own else None, outs[l])
         if replay:
             cache.replay_advance()       # recorded only while capturing
 
