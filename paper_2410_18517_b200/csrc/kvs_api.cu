@@ -769,14 +769,20 @@ kvs_status kvs_step_host(kvs_ctx* ctx, const void* q_host, const void* k_host, c
         if (c + 1 < chunks && !copy_in(c + 1)) return KVS_ERR_CUDA;
         if (cudaStreamWaitEvent(st, ctx->ev_in[c], 0) != cudaSuccess) return KVS_ERR_CUDA;
         for (int l = l0; l < l1; ++l) {
-            if (ctx->share_map[l] == l) {
-                kvs_status s = do_append(ctx, l, dk + kv_layer * l, dv + kv_layer * l, batch, 1, st);
-                if (s != KVS_OK) return s;
+            float* o = reinterpret_cast<float*>(dout + out_layer * l);
+            kvs_status s;
+            if (ctx->share_map[l] == l && !ctx->ragged[ctx->slot_of_layer[l]]) {
+                // the append rides in the split-K kernel (the staging rows are 16-byte aligned)
+                s = do_fused_step(ctx, l, dq + q_layer * l, dk + kv_layer * l, dv + kv_layer * l, o, batch, st);
             } else {
-                ctx->stats.append_skipped += 1;
+                if (ctx->share_map[l] == l) {
+                    s = do_append(ctx, l, dk + kv_layer * l, dv + kv_layer * l, batch, 1, st);
+                    if (s != KVS_OK) return s;
+                } else {
+                    ctx->stats.append_skipped += 1;
+                }
+                s = do_attention(ctx, l, dq + q_layer * l, o, batch, st);
             }
-            kvs_status s =
-                do_attention(ctx, l, dq + q_layer * l, reinterpret_cast<float*>(dout + out_layer * l), batch, st);
             if (s != KVS_OK) return s;
         }
         if (cudaEventRecord(ctx->ev_done[c], st) != cudaSuccess || cudaStreamWaitEvent(os, ctx->ev_done[c], 0) != cudaSuccess)
