@@ -544,6 +544,12 @@ __global__ void decode_combine_kernel(const float* __restrict__ part_o, const fl
     const int np = cta_of_tile((u + 1) * tpu - 1, T, NC) - c0 + 1;       // pieces of this unit
     const int d = threadIdx.x, lane = d & 31, warp = d >> 5;
     const float2* ml = reinterpret_cast<const float2*>(part_ml) + (u + c0) * G + g;   // piece c: ml[c * G]
+    // the first output vectors are requested together with the (max, sum) pairs: one round trip to
+    // L2 for a unit of up to four pieces
+    const float* po = part_o + ((u + c0) * G + g) * D + d;               // piece c: po[c * G * D]
+    float pre[4];
+#pragma unroll
+    for (int c = 0; c < 4; ++c) pre[c] = (np <= 4 && c < np) ? po[(long long)c * G * D] : 0.f;   // (longer units: see below)
     // every warp takes a share of the pieces: maxima and sums to shared memory
     float mx = -1.0e30f;
     for (int c = d; c < np; c += blockDim.x) {
@@ -561,9 +567,15 @@ __global__ void decode_combine_kernel(const float* __restrict__ part_o, const fl
     for (int c = d; c < np; c += blockDim.x) wsm[c] = fast_exp2(wsm[c] - M);
     __syncthreads();
     float o = 0.f, den = 0.f;
-    const float* po = part_o + ((u + c0) * G + g) * D + d;               // piece c: po[c * G * D]
+    const int first = np <= 4 ? np : 0;     // units of more pieces fetch all their vectors here, eight at a time
+#pragma unroll
+    for (int c = 0; c < 4; ++c)
+        if (c < first) {
+            o = fmaf(wsm[c], pre[c], o);
+            den = fmaf(wsm[c], lsm[c], den);
+        }
 #pragma unroll 8
-    for (int c = 0; c < np; ++c) {
+    for (int c = first; c < np; ++c) {
         const float w = wsm[c];
         o = fmaf(w, po[(long long)c * G * D], o);
         den = fmaf(w, lsm[c], den);
