@@ -594,8 +594,13 @@ cudaError_t launch_combine(const DecodeArgs& a, const DecodePlan& plan, cudaStre
 // --------------------------------------------------------------------------------------
 template <typename T, int D, int G, int GEOM>
 static cudaError_t set_attr_one() {
-    return cudaFuncSetAttribute(decode_splitk_scalar<T, D, G, GEOM>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                ScalarShape<T, D, G, GEOM>::SMEM_BYTES);
+    cudaError_t e = cudaFuncSetAttribute(decode_splitk_scalar<T, D, G, GEOM>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         ScalarShape<T, D, G, GEOM>::SMEM_BYTES);
+    if (e != cudaSuccess) return e;
+    // the whole L1 / shared-memory array as shared memory, so that the combine kernel's blocks, launched
+    // early behind this kernel, find room to become resident beside its blocks (see the tensor-core kernel)
+    return cudaFuncSetAttribute(decode_splitk_scalar<T, D, G, GEOM>, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                cudaSharedmemCarveoutMaxShared);
 }
 
 template <typename T, int D>
