@@ -37,10 +37,10 @@ FALLBACK_HBM_GBS = 6650.0
 # of the captured launch; traffic grows in proportion to it, so the bench scales by that
 # ratio.  A record is used only while the kernel sources still hash to `sha256`.
 NCU_TRAFFIC = {
-    1: {"files": ("kvs_kernels.cu", "kvs_device.cuh"), "dram_bytes": 541.69e6, "kv_bytes": 537.13e6,
-        "sha256": "2547e4f6c7cf616fa9e082f12ae3e4d97495d04f33f07bdb86f8a0bbb5df0412"},
-    2: {"files": ("kvs_mma.cu", "kvs_device.cuh"), "dram_bytes": 542.59e6, "kv_bytes": 536.90e6,
-        "sha256": "5d23a1febe68fdde036eb7a7d18dca8ef91c5706c77b8a321fc97ece1b0e0c85"},
+    1: {"files": ("kvs_kernels.cu", "kvs_device.cuh"), "dram_bytes": 542.19e6, "kv_bytes": 537.13e6,
+        "sha256": "ec710c7de996f7cf03d419544067aefc8700e7e5bf1bdd4a97c6edd2d511ad9c"},
+    2: {"files": ("kvs_mma.cu", "kvs_device.cuh"), "dram_bytes": 542.45e6, "kv_bytes": 536.90e6,
+        "sha256": "9590a370614b0bacffbb8db497037d88cf099e5d178c3c7e6a5ee011a6a40fe7"},
 }
 
 
