@@ -22,6 +22,8 @@
  *   - work is enqueued on the given CUDA stream (a cudaStream_t passed as
  *     void*, NULL = the legacy default stream) and returns without waiting,
  *     except where a call says otherwise;
+ *   - device pointers to q, k and v must be 16-byte aligned (INVALID_ARG otherwise): they are read
+ *     with 16-byte vector loads and bulk copies;
  *   - all sequences of a batch are appended to together and have the same length, until
  *     kvs_evict makes the (sequence, head) units of a slot differ.
  *
@@ -179,7 +181,7 @@ kvs_status kvs_decode_attention(kvs_ctx* ctx, int32_t layer, const void* q, floa
  * may be NULL, and nothing is appended).
  *   q: device, [batch][n_q_heads][head_dim];  k, v: device, [batch][1][n_kv_heads][head_dim];
  *   out: device, float32 [batch][n_q_heads][head_dim]
- * On a computing layer whose slot nothing was evicted from (and with k, v 16-byte aligned) no
+ * On a computing layer whose slot nothing was evicted from no
  * append kernel is launched: the split-K kernel stores the new row itself -- the thread block
  * whose share of the rows ends a (sequence, kv-head) unit writes that unit's row to the slot just
  * before it fetches the tile that holds it -- so the step is two launches instead of three.  k and

@@ -200,6 +200,7 @@ kvs_status check_append(kvs_ctx* c, int layer, const void* k, const void* v, int
     *sharing = c->share_map[layer] != layer;
     if (*sharing) return KVS_OK;
     if (!k || !v) return KVS_ERR_INVALID_ARG;
+    if (((uintptr_t)k % 16) != 0 || ((uintptr_t)v % 16) != 0) return KVS_ERR_INVALID_ARG;   // 16-byte vector loads
     if (c->cur_batch != 0 && batch != c->cur_batch) return KVS_ERR_INVALID_ARG;
     const int slot = c->slot_of_layer[layer];
     if ((long long)c->slot_len[slot] + n_new > c->cfg.max_seq) return KVS_ERR_CAPACITY;
@@ -210,6 +211,7 @@ kvs_status check_attention(kvs_ctx* c, int layer, const void* q, const void* out
     if (!c) return KVS_ERR_INVALID_ARG;
     if (!c->bound) return KVS_ERR_STATE;
     if (layer < 0 || layer >= c->cfg.n_layers || !q || !out) return KVS_ERR_INVALID_ARG;
+    if (((uintptr_t)q % 16) != 0 || ((uintptr_t)out % 4) != 0) return KVS_ERR_INVALID_ARG;   // q is fetched by bulk copies
     if (batch < 1 || batch > c->cfg.max_batch) return KVS_ERR_INVALID_ARG;
     const int slot = c->slot_of_layer[layer];
     if (c->slot_len[slot] == 0) return KVS_ERR_STATE;
@@ -521,8 +523,8 @@ kvs_status kvs_decode_step(kvs_ctx* ctx, int32_t layer, const void* q, const voi
     DeviceGuard guard(ctx->cfg.device);
     if (!guard.ok) return KVS_ERR_CUDA;
     const int slot = ctx->slot_of_layer[layer];
-    const bool aligned = ((uintptr_t)k % 16) == 0 && ((uintptr_t)v % 16) == 0;
-    if (aligned && !ctx->ragged[slot]) return do_fused_step(ctx, layer, q, k, v, out, batch, st);
+    if (((uintptr_t)q % 16) != 0 || ((uintptr_t)out % 4) != 0) return KVS_ERR_INVALID_ARG;
+    if (!ctx->ragged[slot]) return do_fused_step(ctx, layer, q, k, v, out, batch, st);
     s = do_append(ctx, layer, k, v, batch, 1, st);
     if (s != KVS_OK) return s;
     return do_attention(ctx, layer, q, out, batch, st);

@@ -242,6 +242,17 @@ def test_error_paths_launch_nothing():
     assert e.value.status == kb.KVS_ERR_STATE
     with pytest.raises(KvsError):
         kb.kvs_append(cache.ctx, 1, None, None, 2, 1)
+    # pointers that are not 16-byte aligned are refused (the kernels read 16-byte vectors)
+    flat = torch.zeros(k1.numel() + 8, dtype=k1.dtype, device="cuda")
+    k_off = flat[1 : 1 + k1.numel()].view(k1.shape)
+    qflat = torch.zeros(q.numel() + 8, dtype=q.dtype, device="cuda")
+    q_off = qflat[1 : 1 + q.numel()].view(q.shape)
+    for call in (lambda: cache.append(1, k_off, k_off), lambda: cache.decode_attention(0, q_off),
+                 lambda: cache.decode_step(1, q_off, v1.cuda(), v1.cuda()),
+                 lambda: cache.decode_step(1, q, k_off, k_off)):
+        with pytest.raises(KvsError) as e:
+            call()
+        assert e.value.status == kb.KVS_ERR_INVALID_ARG
     torch.cuda.synchronize()
     assert torch.equal(before, cache.pool) and cache.seq_len(0) == 128
     cache.reset()
