@@ -9,6 +9,14 @@ resident in HBM before timing starts.
     python bench.py --gpus 1 --steps 100 --warmup 10          # this library
     python bench.py --impl reference --steps 3 --warmup 1      # the fp64 CPU oracle
 
+The headline workload is the largest configuration that fits one GPU (`13b_mha`: 40 layers,
+batch 16, context 8192 = 128K tokens per layer launch, 100 GiB of K/V read per step).  The same
+JSON line carries a `configs` array with further configurations measured the same way (among them
+the long-context grouped-query one and a sweep point with batch x context = 256K tokens) and a
+`prefill` record for the tensor-core prefill kernel.  A timed region is exactly `--steps` decode
+steps; regions are repeated (the cache cut back to the same length in between) until at least a
+second has been timed, and the median region is reported.
+
 Prints ONE JSON line (rank 0).
 """
 from __future__ import annotations
@@ -185,7 +193,8 @@ def run_reference(args, w):
 
 def workload_config(w, n_gpus):
     return {"workload": w.name, "layers": w.L, "q_heads": w.Hq, "kv_heads": w.Hkv, "head_dim": w.D,
-            "batch_per_gpu": w.B, "global_batch": w.B * n_gpus, "context": w.context, "storage": w.dtype,
+            "batch_per_gpu": w.B, "global_batch": w.B * n_gpus, "context": w.context,
+            "batch_x_context_tokens": w.B * w.context, "storage": w.dtype,
             "shared_layers": w.n_shared, "share_map": [int(x) for x in w.share_map()],
             "parallelism": f"batch-sharded x{n_gpus}, no collective on the data path",
             "l2": "inputs larger than L2: every layer launch streams its whole slot "
@@ -193,52 +202,21 @@ def workload_config(w, n_gpus):
                   f"{w.L - w.n_shared} distinct slots are cycled"}
 
 
-def main():
-    ap = argparse.ArgumentParser()
-    ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=100)
-    ap.add_argument("--warmup", type=int, default=10)
-    ap.add_argument("--impl", default="kvs", choices=["kvs", "reference"])
-    ap.add_argument("--workload", default="7b_mha")
-    ap.add_argument("--e2e-steps", type=int, default=20)
-    ap.add_argument("--no-cpu-baseline", action="store_true")
-    args = ap.parse_args()
-    if args.warmup < 3 and args.impl == "kvs":
-        args.warmup = 3
+MIN_TIMED_S = 1.0       # regions of K steps are repeated until this much has been timed
+MAX_REGIONS = 200
 
-    import synth_inputs as si
 
-    w = si.WORKLOADS[args.workload]
-    if args.impl == "reference":
-        run_reference(args, w)
-        return
-
+def measure(w, K, W, E, rank, local_rank, world, dist, with_isolated=True, with_e2e=True):
+    """Decode steps of workload `w` on this rank's GPU.  Returns the measurements of rank 0's line
+    (every rank runs the same steps; times are the maximum over ranks)."""
     import torch
 
+    import synth_inputs as si
     from paper_2410_18517_b200 import SharedKVCache, dist_util
-    from paper_2410_18517_b200 import build as kbuild
 
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-
-        if rank == 0:
-            kbuild.build()
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
-    else:
-        kbuild.build()
-    torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
-    if dist is not None:
-        dist.barrier()
-
-    K, W, E = args.steps, args.warmup, args.e2e_steps
-    total_steps = W + K + K + (3 + E)          # value pass, per-launch-timed pass, e2e pass
     sm = w.share_map()
-    cache = SharedKVCache(w.L, w.Hq, w.Hkv, w.D, w.B, w.context + total_steps, w.dtype, share_map=sm,
+    cache = SharedKVCache(w.L, w.Hq, w.Hkv, w.D, w.B, w.context + W + max(K, 3 + E) + 1, w.dtype, share_map=sm,
                           device=local_rank)
     # Every rank decodes its own batch of sequences (batch sharding): own seed, no exchange.
     seed = 1000 + rank
@@ -278,116 +256,266 @@ def main():
             dist.barrier()
         torch.cuda.synchronize(dev)
 
+    def region():
+        """Exactly K steps from the same cache length, bracketed by a barrier + synchronize."""
+        cache.truncate(n_start)
+        sync_all()
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ev0.record()
+        for t in range(K):
+            one_step(W + t)
+        ev1.record()
+        sync_all()
+        return dist_util.max_over_ranks(ev0.elapsed_time(ev1), dev)
+
     sampler = ClockSampler(local_rank)
     for t in range(W):
         one_step(t)
     sync_all()
+    n_start = cache.seq_len(0)
     if rank == 0:
         sampler.start()
         time.sleep(0.1)
     st0 = cache.stats()
-    n_start = cache.seq_len(0)
-    sync_all()
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    ev0.record()
-    for t in range(K):
-        one_step(W + t)
-    ev1.record()
-    sync_all()
-    ms = ev0.elapsed_time(ev1)
+    region_ms = [region()]
     st1 = cache.stats()
-    ms = dist_util.max_over_ranks(ms, dev)
+    # every rank derives the same count from the same (maximum-over-ranks) first region
+    n_regions = max(1, min(MAX_REGIONS, int(-(-MIN_TIMED_S * 1e3 // region_ms[0]))))
+    for _ in range(n_regions - 1):
+        region_ms.append(region())
+    clocks = sampler.stop() if rank == 0 else None
+    ms = statistics.median(region_ms)
     launches = sum(st1[k] - st0[k] for k in ("append_launches", "attention_launches", "combine_launches"))
     kv_read = st1["kv_bytes_read"] - st0["kv_bytes_read"]
     kv_app = st1["kv_bytes_appended"] - st0["kv_bytes_appended"]
+    n_att = st1["attention_launches"] - st0["attention_launches"]
 
-    # End to end through the host-buffer entry point: pinned host inputs copied in, outputs copied out.
-    # Runs directly after the timed steps so that the context has grown as little as possible.
-    host = []
-    for t in range(4):
-        ql = torch.stack([qs[t][l][0] for l in range(w.L)]).cpu().pin_memory()
-        kl = torch.stack([qs[t][l][1] for l in range(w.L)]).cpu().pin_memory()
-        vl = torch.stack([qs[t][l][2] for l in range(w.L)]).cpu().pin_memory()
-        host.append((ql, kl, vl))
-    out_host = torch.empty(w.L, w.B, w.Hq, w.D, dtype=torch.float32).pin_memory()
-    for t in range(3):
-        h2d, d2h = cache.step_host(*host[t % 4], out_host)
-    sync_all()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    n_e2e = cache.seq_len(0)
-    e0.record()
-    for t in range(E):
-        h2d, d2h = cache.step_host(*host[t % 4], out_host)
-    e1.record()
-    sync_all()
-    e2e_ms = e0.elapsed_time(e1)
-    e2e_ms = dist_util.max_over_ranks(e2e_ms, dev)
+    e2e = None
+    if with_e2e:
+        # End to end through the host-buffer entry point: pinned host inputs copied in, outputs copied
+        # out, every step.  Same cache length as the timed regions.
+        host = []
+        for t in range(4):
+            ql = torch.stack([qs[t][l][0] for l in range(w.L)]).cpu().pin_memory()
+            kl = torch.stack([qs[t][l][1] for l in range(w.L)]).cpu().pin_memory()
+            vl = torch.stack([qs[t][l][2] for l in range(w.L)]).cpu().pin_memory()
+            host.append((ql, kl, vl))
+        out_host = torch.empty(w.L, w.B, w.Hq, w.D, dtype=torch.float32).pin_memory()
+        cache.truncate(n_start)
+        for t in range(3):
+            h2d, d2h = cache.step_host(*host[t % 4], out_host)
+        e2e_regions = []
+        for _ in range(max(1, min(n_regions, 25))):
+            cache.truncate(n_start)
+            sync_all()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for t in range(E):
+                h2d, d2h = cache.step_host(*host[t % 4], out_host)
+            e1.record()
+            sync_all()
+            e2e_regions.append(dist_util.max_over_ranks(e0.elapsed_time(e1), dev))
+        e2e_ms = statistics.median(e2e_regions)
+        e2e = {"value": dist_util.whole_job_rate(w.B, world, e2e_ms / E), "unit": UNIT, "h2d_bytes_per_step": h2d,
+               "d2h_bytes_per_step": d2h, "steps": E, "regions": len(e2e_regions), "ms_per_step": e2e_ms / E,
+               "context_mid_run": n_start + E // 2,
+               "how": "kvs_step_host: pinned host q/k/v in, fp32 outputs back to pinned host memory, every step"}
 
-    # Same K steps again with a CUDA event pair around every attention call: gives the
-    # duration of the dominant kernel's launches (split-K kernel + its small combine).
-    events = []
-    rb0 = cache.stats()["kv_bytes_read"]
-    for t in range(K):
-        one_step(W + K + t, events)
-    sync_all()
-    att_ms = [a.elapsed_time(b) for a, b in events]
-    att_bytes = cache.stats()["kv_bytes_read"] - rb0
-    att_launch_ms = sum(att_ms) / len(att_ms)
-    bytes_per_launch = att_bytes / len(att_ms)
+    isolated = None
+    if with_isolated:
+        # The same K steps with a CUDA event pair around every attention call: the duration of the
+        # dominant kernel's launches (split-K kernel + its small combine) with the overlap forbidden.
+        cache.truncate(n_start)
+        events = []
+        rb0 = cache.stats()["kv_bytes_read"]
+        for t in range(K):
+            one_step(W + t, events)
+        sync_all()
+        att_ms = [a.elapsed_time(b) for a, b in events]
+        att_bytes = cache.stats()["kv_bytes_read"] - rb0
+        isolated = (sum(att_ms) / len(att_ms), att_bytes / len(att_ms), len(att_ms))
 
-    clocks = sampler.stop() if rank == 0 else None
     status = cache.device_status()
+    rec = None
+    if rank == 0:
+        peak, peak_kind = _peak_hbm()
+        # Dominant kernel = the split-K attention kernel, one launch per layer.  Its average launch
+        # duration over the timed region is the region's CUDA-event time divided by its launches: the
+        # kernels of a step overlap (early-start launches), so this includes the hidden remainders of
+        # the combine kernels and is a lower bound on the kernel's own rate.
+        pipelined_ms = ms / n_att
+        pipelined_bytes = kv_read / n_att
+        achieved = pipelined_bytes / (pipelined_ms * 1e-3) / 1e9
+        traffic = None
+        kernel_id = cache.last_launch()["kernel"]
+        nrec = NCU_TRAFFIC.get(kernel_id)
+        if nrec and nrec["sha256"] == _kernel_hash(nrec["files"]):
+            traffic = nrec["dram_bytes"] * pipelined_bytes / nrec["kv_bytes"]
+        step_ms = ms / K
+        pool_unshared = cache.pool_bytes // cache.num_slots() * w.L
+        roofline = {"bound": "hbm", "kernel": ("decode_splitk_scalar", "decode_splitk_mma")[kernel_id - 1]
+                    + " (timed region / launches; the append rides in it, the combine kernel overlaps it)",
+                    "achieved": achieved, "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
+                    "frac": achieved / peak, "frac_of_8tbs_nominal": achieved / NOMINAL_HBM_GBS,
+                    "traffic": traffic, "bytes_per_launch": pipelined_bytes, "ms_per_launch": pipelined_ms,
+                    "launches_timed": n_att, "ctas": cache.last_launch()["ctas"]}
+        if isolated is not None:
+            iso = isolated[1] / (isolated[0] * 1e-3) / 1e9
+            roofline["isolated"] = {"achieved": iso, "frac": iso / peak, "ms_per_call": isolated[0],
+                                    "bytes_per_launch": isolated[1], "launches_timed": isolated[2],
+                                    "how": "event pair around every attention call (split-K + combine), no overlap"}
+        rec = {
+            "value": dist_util.whole_job_rate(w.B, world, step_ms), "unit": UNIT, "ms_per_step": step_ms,
+            "config": workload_config(w, world),
+            "timed": {"regions": len(region_ms), "steps_per_region": K, "seconds": sum(region_ms) * 1e-3,
+                      "region_ms_min": min(region_ms), "region_ms_median": ms, "region_ms_max": max(region_ms),
+                      "how": "each region is exactly `steps` decode steps from the same cache length (kvs_truncate "
+                             "in between), barrier + synchronize on both sides, CUDA events, max over ranks; the "
+                             "median region is reported"},
+            "kv_read_gbs_whole_step": kv_read / (ms * 1e-3) / 1e9,
+            "kv_read_frac_of_8tbs_nominal": kv_read / (ms * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
+            "kv_bytes_read_per_step": kv_read // K, "kv_bytes_appended_per_step": kv_app // K,
+            "pool_bytes": cache.pool_bytes, "pool_bytes_unshared": pool_unshared,
+            "kv_memory_saved_frac": 1.0 - cache.pool_bytes / pool_unshared,
+            "context_mid_run": n_start + K // 2,
+            "roofline": roofline, "e2e": e2e, "gpu_launches": launches, "clocks": clocks, "device_status": status,
+            "ms_per_step_x_sm_mhz": step_ms * clocks["sm_mhz"] if clocks and clocks.get("sm_mhz") else None,
+        }
+    cache.close()
+    del cache, qs, outs
+    import gc
+
+    gc.collect()
+    torch.cuda.empty_cache()
+    return rec
+
+
+def prefill_record(local_rank):
+    """The tensor-core prefill kernel on two prompt shapes: ms per call and TFLOP/s against the
+    measured dense bf16 peak (algorithmic = causal flops 4 B Hq D T(T+1)/2; issued = what the tensor
+    cores are given: S plus two PV terms over whole tiles)."""
+    import torch
+
+    import synth_inputs as si
+    from paper_2410_18517_b200 import SharedKVCache
+
+    try:
+        peak = float(json.load(open(os.path.join(ROOT, "MEASURED_PEAKS.json")))["bf16_tflops"])
+        kind = "of measured"
+    except Exception:
+        peak, kind = 1590.0, "of fallback"
+    out = []
+    for (B, Hq, Hkv, T) in ((2, 32, 32, 4096), (1, 32, 8, 16384)):
+        D = 128
+        w = si.Workload("prefill_bench", L=2, Hq=Hq, Hkv=Hkv, D=D, B=B, context=T, dtype="bf16", n_shared=1,
+                        map_seed=0, steps=1, fixed_map=(0, 0))
+        cache = SharedKVCache(w.L, Hq, Hkv, D, B, T, "bf16", share_map=w.share_map(), device=local_rank)
+        dev = cache.device
+        k, v = si.context_kv(w, 0, device=dev)
+        cache.append(0, k, v)
+        q = si.normal((0, "prefill_bench_q"), (B, T, Hq, D), torch.bfloat16, device=dev)
+        o = torch.empty(B, T, Hq, D, dtype=torch.float32, device=dev)
+        for i in range(3):
+            cache.prefill_attention(i % 2, q, o)
+        torch.cuda.synchronize(dev)
+        iters = 20
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(iters):
+            cache.prefill_attention(i % 2, q, o)     # layer 1 shares layer 0's slot
+        e1.record()
+        torch.cuda.synchronize(dev)
+        ms = e0.elapsed_time(e1) / iters
+        algo = 4.0 * B * Hq * D * T * (T + 1) / 2
+        tiles = sum(min(qb + 1, (T + 127) // 128) for qb in range((T + 127) // 128))
+        issued = B * Hq * tiles * 3 * 2.0 * 128 * 128 * D
+        out.append({"kernel": "prefill_attention_tc", "batch": B, "q_heads": Hq, "kv_heads": Hkv, "tokens": T,
+                    "head_dim": D, "ms_per_call": ms, "algorithmic_tflops": algo / ms / 1e9,
+                    "issued_tflops": issued / ms / 1e9,
+                    "roofline": {"bound": "tensor", "achieved": algo / ms / 1e9, "peak": peak, "peak_kind": kind,
+                                 "unit": "TFLOP/s", "frac": algo / ms / 1e9 / peak,
+                                 "frac_issued": issued / ms / 1e9 / peak},
+                    "device_status": cache.device_status()})
+        cache.close()
+        del cache, k, v, q, o
+        torch.cuda.empty_cache()
+    return out
+
+
+DEFAULT_WORKLOAD = "13b_mha"
+DEFAULT_CONFIGS = "gqa_long,sweep_b32_n8192_p10,7b_mha"
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=64)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="kvs", choices=["kvs", "reference"])
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
+    ap.add_argument("--configs", default=None,
+                    help="comma-separated further configurations for the `configs` array ('' = none; default: "
+                         f"{DEFAULT_CONFIGS} when the headline workload is the default one, at 1 GPU)")
+    ap.add_argument("--e2e-steps", type=int, default=20)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-prefill", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3 and args.impl == "kvs":
+        args.warmup = 3
+
+    import synth_inputs as si
+
+    w = si.workload_by_name(args.workload)
+    if args.impl == "reference":
+        run_reference(args, w)
+        return
+
+    import torch
+
+    from paper_2410_18517_b200 import build as kbuild
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+
+        if rank == 0:
+            kbuild.build()
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    else:
+        kbuild.build()
+    torch.cuda.set_device(local_rank)
+    if dist is not None:
+        dist.barrier()
+
+    K, W, E = args.steps, args.warmup, args.e2e_steps
+    head = measure(w, K, W, E, rank, local_rank, world, dist)
+    extras, prefill = [], None
+    if world == 1:
+        names = args.configs if args.configs is not None else (DEFAULT_CONFIGS if args.workload == DEFAULT_WORKLOAD else "")
+        for name in [x for x in names.split(",") if x]:
+            r = measure(si.workload_by_name(name), K, W, E, rank, local_rank, world, dist, with_isolated=False,
+                        with_e2e=False)
+            r.pop("e2e", None)
+            extras.append(r)
+        if not args.no_prefill:
+            prefill = prefill_record(local_rank)
 
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
         return
 
-    peak, peak_kind = _peak_hbm()
-    # Dominant kernel = the split-K attention kernel, one launch per layer.  Its average launch
-    # duration over the timed region is the region's CUDA-event time divided by its launches: the
-    # kernels of a step overlap (early-start launches), so this includes the hidden remainders of
-    # the append and combine kernels and is a lower bound on the kernel's own rate.  The same K
-    # steps timed with an event pair around every attention call (which forbids the overlap) are
-    # reported beside it as "isolated".
-    n_att = st1["attention_launches"] - st0["attention_launches"]
-    pipelined_ms = ms / n_att
-    pipelined_bytes = kv_read / n_att
-    achieved = pipelined_bytes / (pipelined_ms * 1e-3) / 1e9
-    isolated = bytes_per_launch / (att_launch_ms * 1e-3) / 1e9
-    traffic = None
-    kernel_id = cache.last_launch()["kernel"]
-    rec = NCU_TRAFFIC.get(kernel_id)
-    if rec and rec["sha256"] == _kernel_hash(rec["files"]):
-        traffic = rec["dram_bytes"] * pipelined_bytes / rec["kv_bytes"]
-    step_ms = ms / K
-    n_mid = n_start + K // 2
-    pool_unshared = cache.pool_bytes // cache.num_slots() * w.L
-    line = {
-        "metric": METRIC, "value": dist_util.whole_job_rate(w.B, world, step_ms), "unit": UNIT, "n_gpus": world, "steps": K,
-        "warmup": W, "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "f32", "data": "synthetic", "config": workload_config(w, world),
-        "kv_read_gbs_whole_step": kv_read / (ms * 1e-3) / 1e9,
-        "kv_read_frac_of_8tbs_nominal": kv_read / (ms * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
-        "kv_bytes_read_per_step": kv_read // K, "kv_bytes_appended_per_step": kv_app // K,
-        "pool_bytes": cache.pool_bytes, "pool_bytes_unshared": pool_unshared,
-        "kv_memory_saved_frac": 1.0 - cache.pool_bytes / pool_unshared,
-        "context_mid_run": n_mid,
-        "roofline": {"bound": "hbm", "kernel": ("decode_splitk_scalar", "decode_splitk_mma")[kernel_id - 1]
-                     + " (timed region / launches; the append rides in it, the combine kernel overlaps it)",
-                     "achieved": achieved, "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
-                     "frac": achieved / peak, "frac_of_8tbs_nominal": achieved / NOMINAL_HBM_GBS,
-                     "traffic": traffic, "bytes_per_launch": pipelined_bytes, "ms_per_launch": pipelined_ms,
-                     "launches_timed": n_att,
-                     "isolated": {"achieved": isolated, "frac": isolated / peak, "ms_per_call": att_launch_ms,
-                                  "bytes_per_launch": bytes_per_launch, "launches_timed": len(att_ms),
-                                  "how": "event pair around every attention call (split-K + combine), no overlap"}},
-        "e2e": {"value": dist_util.whole_job_rate(w.B, world, e2e_ms / E), "unit": UNIT, "h2d_bytes_per_step": h2d,
-                "d2h_bytes_per_step": d2h, "steps": E, "ms_per_step": e2e_ms / E, "context_mid_run": n_e2e + E // 2},
-        "gpu_launches": launches,
-        "clocks": clocks,
-        "device_status": status,
-    }
+    line = {"metric": METRIC, "value": head.pop("value"), "unit": head.pop("unit"), "n_gpus": world, "steps": K,
+            "warmup": W, "ms_per_step": head.pop("ms_per_step"), "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic"}
+    line.update(head)
+    if extras:
+        line["configs"] = extras
+    if prefill is not None:
+        line["prefill"] = prefill
     if world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(w)
     print(json.dumps(line))

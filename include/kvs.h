@@ -22,6 +22,12 @@
  *   - work is enqueued on the given CUDA stream (a cudaStream_t passed as
  *     void*, NULL = the legacy default stream) and returns without waiting,
  *     except where a call says otherwise;
+ *   - the calls of one context form ONE ordered chain on the GPU: issue them all on one stream, or,
+ *     when the stream changes from one call to the next, make the new stream wait (event) for
+ *     everything the previous call enqueued.  The library's kernels start early behind one another
+ *     (see KVS_OPT_EARLY_START) and decide on the host which cached rows are already stable; that
+ *     bookkeeping, and the shared workspace, assume this chain.  kvs_decode_attention_static is the
+ *     one call that may run beside the chain (see there);
  *   - device pointers to q, k and v must be 16-byte aligned (INVALID_ARG otherwise): they are read
  *     with 16-byte vector loads and bulk copies;
  *   - all sequences of a batch are appended to together and have the same length, until
@@ -143,6 +149,15 @@ kvs_status kvs_bind_memory(kvs_ctx* ctx, void* pool, size_t pool_bytes,
 /* Forget every cached token (all slot lengths become 0).  Host-side only. */
 kvs_status kvs_reset(kvs_ctx* ctx);
 
+/* Forget the newest tokens: every slot that holds more than n_tokens rows is cut back to n_tokens
+ * (the paper has no counterpart; generation only ever grows a cache, this is the roll-back a caller
+ * needs to drop tokens it decides not to keep, or to run the same decode steps again).  Host-side
+ * only, no launch: the rows stay in the pool and are overwritten by later appends.  Kernels already
+ * queued keep the lengths they were launched with.  Not between the replays of a recorded step and
+ * their kvs_replay_commit.  Errors: INVALID_ARG for n_tokens < 0; STATE if a slot that would be cut
+ * has had rows evicted (its units differ in length).                                              */
+kvs_status kvs_truncate(kvs_ctx* ctx, int32_t n_tokens);
+
 /* ---- the hot path ------------------------------------------------------------ */
 
 /* Store the new tokens' keys and values of one layer (Section 3.2; a layer whose
@@ -169,7 +184,7 @@ kvs_status kvs_append(kvs_ctx* ctx, int32_t layer, const void* k, const void* v,
  *   out: device, [batch][n_q_heads][head_dim], float32
  * Launches the split-K kernel and the combine kernel on `stream`; partial
  * results go through the bound workspace, so calls on one context must not
- * overlap on the GPU (use one stream, or order them).
+ * overlap on the GPU (one stream, or full event ordering: see the conventions above).
  * Errors: STATE before kvs_bind_memory or when the slot is empty; INVALID_ARG
  * for a bad layer, NULLs, batch < 1 or batch > the batch the slot was filled for. */
 kvs_status kvs_decode_attention(kvs_ctx* ctx, int32_t layer, const void* q, float* out,
@@ -231,7 +246,8 @@ kvs_status kvs_unit_len(const kvs_ctx* ctx, int32_t layer, int32_t b, int32_t h,
 /* Euclidean distances between the KV caches of every pair of layers.  The caches currently in
  * the pool play the calibration run: the first `batch` cached sequences are the samples.  Per
  * layer, keys and values are averaged over the samples, each flattened, and laid end to end
- * (reading of the paper's "average the keys and values separately"); dist[i][j] is the 2-norm of
+ * (reading of the averaging step of Section 3.1 / Algorithm 1: mean-K flattened, then mean-V
+ * flattened, one vector per layer); dist[i][j] is the 2-norm of
  * the difference of layers i and j's vectors (a sharing layer has its source's cache: distance 0).
  *   dist: device, float32 [n_layers][n_layers], symmetric, zero diagonal.
  * Two kernels on `stream`; reads every cached element once.  Sorting the pairs (descending, as
@@ -297,11 +313,10 @@ kvs_status kvs_step_host(kvs_ctx* ctx, const void* q_host, const void* k_host, c
  * this library described below.)
  *
  * Who needs it: code that runs after a serving engine has handed all of the GPU's free memory
- * to its own pools and forbids further cudaMalloc (which would also stall the device); code in a
- * plug-in or callback that is given tensors but no allocator; and code between two points where
- * the workspace bound with kvs_bind_memory is already busy with another call.  Such callers
- * still pass the inputs and outputs (q, out, and the context whose pool holds K/V); what they
- * cannot provide is the scratch for split-K partial results.
+ * to its own pools and forbids further cudaMalloc (which would also stall the device); and code
+ * in a plug-in or callback that is given tensors but no allocator.  Such callers still pass the
+ * inputs and outputs (q, out, and the context whose pool holds K/V); what they cannot provide is
+ * the scratch for split-K partial results.
  *
  * What it does: exactly what kvs_decode_attention does, with the same kernels and the same
  * result bit for bit, except that the partial results and the device status word live in a
@@ -311,15 +326,22 @@ kvs_status kvs_step_host(kvs_ctx* ctx, const void* q_host, const void* k_host, c
  *   - Limit: (batch * n_kv_heads + blocks launched) * group * (head_dim + 2) * 4 bytes, plus
  *     512 bytes, must fit in 2 MiB (the 7B shape at batch 8 needs 0.3 MiB, the 32q/8kv shape at
  *     batch 64 needs 1.7 MiB).  Larger calls return KVS_ERR_SCRATCH_LIMIT and launch nothing.
- *   - The first call on each device looks up the device address of the array (one runtime
- *     query, no allocation).  Make that first call before starting any stream capture.
+ *   - The device address of the array is looked up once per GPU as part of kvs_bind_memory's
+ *     per-device set-up (that look-up is also when the driver places the array on the GPU, so it
+ *     happens where allocating is still allowed); the call itself makes no runtime query.
  *   - All calls, from all contexts and streams, share the one array, and it keeps the previous
  *     call's contents.  The call itself clears the only part that must start at zero (the
  *     status word).  Two calls that overlap on the GPU race on the partial results: order
  *     them on one stream or with events.
- *   device_status: device pointer to an int32 that receives 0, or KVS_ERR_TIMEOUT if a bounded
- *     wait inside the kernel ran out; may be NULL (the word inside the array is used and is not
- *     readable by the caller).  It is written on `stream`; read it after synchronising.
+ *   - The call is a plain stream-ordered launch and stays out of the context's launch
+ *     bookkeeping, so it may be issued on another stream than the context's other calls, provided
+ *     that stream waits (event) for the kernels that append the rows the call is to see; the other
+ *     calls need not wait for it.  It reads the slot lengths as they stand on the host at the call.
+ *   device_status: device pointer to an int32 (4-byte aligned, else INVALID_ARG) that receives 0,
+ *     KVS_ERR_TIMEOUT if a bounded wait inside the kernel ran out, or (only under KVS_OPT_REPLAY)
+ *     KVS_ERR_CAPACITY if a replayed launch passed max_seq; may be NULL (the word inside the array
+ *     is used and is not readable by the caller).  It is written on `stream`; read it after
+ *     synchronising.
  * Other arguments, layouts and errors: as kvs_decode_attention.                              */
 kvs_status kvs_decode_attention_static(kvs_ctx* ctx, int32_t layer, const void* q, float* out,
                                        int32_t batch, void* stream, int32_t* device_status);
@@ -339,6 +361,18 @@ kvs_status kvs_stats(const kvs_ctx* ctx, kvs_stats_t* stats);
  * 0 = no device-side problem; KVS_ERR_TIMEOUT = a bounded wait inside a kernel ran
  * out and the kernel returned early (its output is then undefined).             */
 kvs_status kvs_last_device_status(kvs_ctx* ctx, int32_t* device_status);
+/* Set the device status word back to 0 on `stream` (it is otherwise cleared only by kvs_bind_memory). */
+kvs_status kvs_clear_device_status(kvs_ctx* ctx, void* stream);
+/* Failure-detection self-test (the paper has no counterpart; every wait inside the pipelined kernels
+ * is bounded, and this call shows the give-up path working on the device at hand without disturbing
+ * anything).  Launches a one-warp kernel in which one thread waits, for at most limit_us
+ * microseconds (1 .. 1 000 000), on a barrier that nothing ever arrives at, through the same bounded
+ * wait the attention kernels use.  The wait runs out, the kernel sets the device status word to
+ * KVS_ERR_TIMEOUT and returns normally; no copy is in flight, nothing traps, the context stays usable.
+ * The call waits for the kernel; *waited_ns (host, may be NULL) receives how long the wait lasted on
+ * the GPU.  Afterwards kvs_last_device_status reports KVS_ERR_TIMEOUT until kvs_clear_device_status.
+ * Errors: STATE before kvs_bind_memory; INVALID_ARG for a limit out of range.                      */
+kvs_status kvs_selftest_wait_timeout(kvs_ctx* ctx, uint32_t limit_us, uint64_t* waited_ns, void* stream);
 kvs_status kvs_set_option(kvs_ctx* ctx, int32_t option, int32_t value);
 /* How the last kvs_decode_attention call was decomposed: thread blocks launched,
  * rows per tile, and 1 or 2 for the scalar / tensor-core kernel.                */

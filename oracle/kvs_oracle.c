@@ -363,10 +363,11 @@ int oracle_get_cache(const oracle_state *st, int l, double *K_out, double *V_out
 }
 
 /* ---- the data-parallel part of strategy searching (Section 3.1) --------------
- * "KV cache similarity": the cache of every layer is averaged over the calibration
+ * Similarity of KV caches: the cache of every layer is averaged over the calibration
  * samples (here: over the B sequences held), keys and values are each flattened,
  * and the Euclidean distance between the representations of any two layers is
- * taken.  Reading of the ambiguous "average the keys and values separately": the
+ * taken.  The averaging step of Section 3.1 / Algorithm 1 can be read in more than
+ * one way (keys and values are to be averaged apart from each other); reading: the
  * representation of a layer is the sample-mean of its keys, flattened, followed by
  * the sample-mean of its values, flattened; the distance is the 2-norm of the
  * difference of two such vectors.  All layers must hold equally long, un-evicted

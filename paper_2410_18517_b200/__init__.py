@@ -163,6 +163,17 @@ class SharedKVCache:
     def reset(self):
         binding.kvs_reset(self.ctx)
 
+    def truncate(self, n_tokens):
+        """Cut every slot back to at most ``n_tokens`` rows (host bookkeeping only)."""
+        binding.kvs_truncate(self.ctx, n_tokens)
+
+    def clear_device_status(self):
+        binding.kvs_clear_device_status(self.ctx, self._stream())
+
+    def selftest_wait_timeout(self, limit_us=1000):
+        """Make one bounded device-side wait run out; returns the nanoseconds it lasted."""
+        return binding.kvs_selftest_wait_timeout(self.ctx, limit_us, self._stream())
+
     def stats(self):
         return binding.kvs_stats(self.ctx)
 

@@ -41,6 +41,7 @@ EXPORTS = (
     "kvs_read_roof", "kvs_decode_attention_static", "kvs_prefill_attention",
     "kvs_evict", "kvs_unit_len", "kvs_layer_distances", "kvs_mean_cosine",
     "kvs_replay_advance", "kvs_replay_commit", "kvs_decode_step",
+    "kvs_clear_device_status", "kvs_selftest_wait_timeout", "kvs_truncate",
 )
 
 
@@ -84,6 +85,7 @@ def load() -> ctypes.CDLL:
         "kvs_required_bytes": [vp, P(sz), P(sz)],
         "kvs_bind_memory": [vp, vp, sz, vp, sz],
         "kvs_reset": [vp],
+        "kvs_truncate": [vp, i32],
         "kvs_append": [vp, i32, vp, vp, i32, i32, vp],
         "kvs_decode_attention": [vp, i32, vp, vp, i32, vp],
         "kvs_decode_step": [vp, i32, vp, vp, vp, vp, i32, vp],
@@ -103,6 +105,8 @@ def load() -> ctypes.CDLL:
         "kvs_plane_offset": [vp, i32, i32, P(sz)],
         "kvs_stats": [vp, P(kvs_stats_t)],
         "kvs_last_device_status": [vp, P(i32)],
+        "kvs_clear_device_status": [vp, vp],
+        "kvs_selftest_wait_timeout": [vp, ctypes.c_uint32, P(ctypes.c_uint64), vp],
         "kvs_set_option": [vp, i32, i32],
         "kvs_last_launch": [vp, P(i32), P(i32), P(i32)],
         "kvs_read_roof": [vp, sz, vp, i32, vp],
@@ -172,6 +176,10 @@ def kvs_bind_memory(ctx: int, pool, pool_bytes: int, workspace, workspace_bytes:
 
 def kvs_reset(ctx: int) -> None:
     _check(load().kvs_reset(ctx), "kvs_reset")
+
+
+def kvs_truncate(ctx: int, n_tokens: int) -> None:
+    _check(load().kvs_truncate(ctx, n_tokens), "kvs_truncate")
 
 
 def kvs_append(ctx: int, layer: int, k, v, batch: int, n_new: int, stream: int = 0) -> None:
@@ -271,6 +279,17 @@ def kvs_last_device_status(ctx: int) -> int:
     v = ctypes.c_int32()
     _check(load().kvs_last_device_status(ctx, ctypes.byref(v)), "kvs_last_device_status")
     return v.value
+
+
+def kvs_clear_device_status(ctx: int, stream: int = 0) -> None:
+    _check(load().kvs_clear_device_status(ctx, stream), "kvs_clear_device_status")
+
+
+def kvs_selftest_wait_timeout(ctx: int, limit_us: int, stream: int = 0) -> int:
+    """Returns the nanoseconds the wait lasted on the GPU before it gave up."""
+    w = ctypes.c_uint64()
+    _check(load().kvs_selftest_wait_timeout(ctx, limit_us, ctypes.byref(w), stream), "kvs_selftest_wait_timeout")
+    return w.value
 
 
 def kvs_set_option(ctx: int, option: int, value: int) -> None:

@@ -19,6 +19,40 @@ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 }  // namespace
 
+// ---------------------------------------------------------------------------------------
+// Scratch of kvs_decode_attention_static: attention without any caller- or library-allocated
+// scratch memory.
+//
+// The split-K partial results and the device status word of that one entry point live in a
+// fixed array that is part of the loaded library image.  Every GPU that loads the library
+// carries these kStaticScratchBytes until the process exits, and every call, from every
+// context, uses the same bytes.
+// ---------------------------------------------------------------------------------------
+constexpr size_t kStaticScratchBytes = 2u << 20;  // 2 MiB
+constexpr size_t kStaticStatusBytes = 256;        // first 256 bytes: device status word
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+namespace {
+
+// In host code `g_static_scratch` is only a handle for the symbol, not an address the GPU can
+// use, so the device address is looked up once per device, with that device current, as part of
+// the per-device set-up that kvs_bind_memory runs (see init_device_once).  The look-up is also
+// what makes the driver load this file's module and reserve the array on that GPU, so it happens
+// where allocating is still allowed and no stream is being captured; the entry point itself then
+// only reads the cached address.
+cudaError_t g_static_err[64];
+unsigned char* g_static_ptr[64];
+
+cudaError_t resolve_static_scratch(int device) {
+    void* p = nullptr;
+    const cudaError_t e = cudaGetSymbolAddress(&p, g_static_scratch);
+    g_static_err[device] = e;
+    g_static_ptr[device] = e == cudaSuccess ? static_cast<unsigned char*>(p) : nullptr;
+    return e;
+}
+
+}  // namespace
+
 struct kvs_ctx {
     kvs_config cfg;
     int G = 1;
@@ -173,6 +207,7 @@ cudaError_t init_device_once(int device) {
         g_init_err[device] = kvs::init_kernels();
         if (g_init_err[device] == cudaSuccess) g_init_err[device] = kvs::init_mma_kernels();
         if (g_init_err[device] == cudaSuccess) g_init_err[device] = kvs::init_prefill_kernels();
+        if (g_init_err[device] == cudaSuccess) g_init_err[device] = resolve_static_scratch(device);
     });
     return g_init_err[device];
 }
@@ -252,6 +287,7 @@ struct AttentionScratch {
     float* part_ml;
     int* status;
     bool programmatic;   // early-start launches (only when the call follows this context's own kernels)
+    bool tracked;        // the call is part of the context's one ordered chain of launches (see kvs_ctx::seq)
 };
 
 // Which kernel serves the context's shape and how the call is cut into work.  bf16 groups of three
@@ -294,8 +330,10 @@ kvs_status run_attention(kvs_ctx* c, int slot, const void* q, float* out, int ba
     a.k_new = k_new;
     a.v_new = v_new;
     if (k_new) a.safe_rows = std::min(a.safe_rows, a.n - 1);   // the new row is fetched after the kernel has stored it
-    c->seq += 2;                       // split-K kernel, then combine
-    c->last_splitk_seq = c->seq - 1;
+    if (scratch.tracked) {
+        c->seq += 2;                       // split-K kernel, then combine
+        c->last_splitk_seq = c->seq - 1;
+    }
     if (use_mma) {
         const long long plane_rows = (long long)c->cfg.max_batch * c->cfg.n_kv_heads * c->row_stride;
         if (kvs::launch_decode_mma(a, plan, c->tensor_map, plane_rows * (2 * slot), plane_rows * (2 * slot + 1), st) !=
@@ -328,7 +366,7 @@ kvs_status do_fused_step(kvs_ctx* c, int layer, const void* q, const void* k, co
     const bool use_mma = choose_plan(c, batch * c->cfg.n_kv_heads, old_len + 1, &plan);
     const AttentionScratch scratch = {reinterpret_cast<float*>(c->ws + c->off_part_o),
                                       reinterpret_cast<float*>(c->ws + c->off_part_ml),
-                                      reinterpret_cast<int*>(c->ws + c->off_status), take_early_start(c)};
+                                      reinterpret_cast<int*>(c->ws + c->off_status), take_early_start(c), true};
     // run_attention works out which rows are stable from the appends before this one
     c->slot_len[slot] = old_len + 1;
     const kvs_status s = run_attention(c, slot, q, out, batch, plan, use_mma, scratch, st, k, v);
@@ -351,7 +389,7 @@ kvs_status do_attention(kvs_ctx* c, int layer, const void* q, float* out, int ba
     const bool use_mma = choose_plan(c, batch * c->cfg.n_kv_heads, c->slot_len[slot], &plan);
     const AttentionScratch scratch = {reinterpret_cast<float*>(c->ws + c->off_part_o),
                                       reinterpret_cast<float*>(c->ws + c->off_part_ml),
-                                      reinterpret_cast<int*>(c->ws + c->off_status), take_early_start(c)};
+                                      reinterpret_cast<int*>(c->ws + c->off_status), take_early_start(c), true};
     return run_attention(c, slot, q, out, batch, plan, use_mma, scratch, st);
 }
 
@@ -480,6 +518,23 @@ kvs_status kvs_reset(kvs_ctx* ctx) {
     for (auto& x : ctx->ragged) x = 0;
     for (auto& x : ctx->slot_len) x = 0;
     ctx->cur_batch = 0;
+    return KVS_OK;
+}
+
+kvs_status kvs_truncate(kvs_ctx* ctx, int32_t n_tokens) {
+    if (!ctx || n_tokens < 0) return KVS_ERR_INVALID_ARG;
+    // a slot rows were evicted from has per-unit lengths on the device as well: refused, not half-updated
+    for (int s = 0; s < ctx->n_slots; ++s)
+        if (ctx->slot_len[s] > n_tokens && ctx->ragged[s]) return KVS_ERR_STATE;
+    for (int s = 0; s < ctx->n_slots; ++s) {
+        if (ctx->slot_len[s] <= n_tokens) continue;
+        ctx->slot_len[s] = n_tokens;
+        // Rows from n_tokens on will be written again.  Kernels of earlier calls may still be reading
+        // them, but every writer stores only after its wait for its predecessor; and what a later
+        // launch may fetch before its own wait must lie below the old and the new writes alike.
+        ctx->app_start_latest[s] = std::min(ctx->app_start_latest[s], n_tokens);
+    }
+    if (n_tokens == 0) ctx->cur_batch = 0;
     return KVS_OK;
 }
 
@@ -849,6 +904,38 @@ kvs_status kvs_last_device_status(kvs_ctx* ctx, int32_t* device_status) {
     return KVS_OK;
 }
 
+kvs_status kvs_clear_device_status(kvs_ctx* ctx, void* stream) {
+    if (!ctx) return KVS_ERR_INVALID_ARG;
+    if (!ctx->bound) return KVS_ERR_STATE;
+    DeviceGuard guard(ctx->cfg.device);
+    if (!guard.ok) return KVS_ERR_CUDA;
+    if (cudaMemsetAsync(ctx->ws + ctx->off_status, 0, sizeof(int), static_cast<cudaStream_t>(stream)) != cudaSuccess)
+        return KVS_ERR_CUDA;
+    return KVS_OK;
+}
+
+kvs_status kvs_selftest_wait_timeout(kvs_ctx* ctx, uint32_t limit_us, uint64_t* waited_ns, void* stream) {
+    if (!ctx || limit_us < 1 || limit_us > 1000000u) return KVS_ERR_INVALID_ARG;
+    if (!ctx->bound) return KVS_ERR_STATE;
+    DeviceGuard guard(ctx->cfg.device);
+    if (!guard.ok) return KVS_ERR_CUDA;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // the measured wait goes to a spare word of the status block (128 bytes after the status word)
+    unsigned long long* waited_dev = reinterpret_cast<unsigned long long*>(ctx->ws + ctx->off_status + 128);
+    if (kvs::launch_wait_timeout_selftest(reinterpret_cast<int*>(ctx->ws + ctx->off_status), 1000ull * limit_us, waited_dev,
+                                          st) != cudaSuccess)
+        return KVS_ERR_CUDA;
+    ctx->seq += 1;
+    ctx->last_splitk_seq = ctx->seq;   // a plain launch: everything before it has finished when it runs
+    ctx->counter_written = false;
+    unsigned long long w = 0;
+    if (cudaMemcpyAsync(&w, waited_dev, sizeof(w), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+        cudaStreamSynchronize(st) != cudaSuccess)
+        return KVS_ERR_CUDA;
+    if (waited_ns) *waited_ns = w;
+    return KVS_OK;
+}
+
 kvs_status kvs_set_option(kvs_ctx* ctx, int32_t option, int32_t value) {
     if (!ctx) return KVS_ERR_INVALID_ARG;
     switch (option) {
@@ -916,43 +1003,11 @@ kvs_status kvs_read_roof(const void* src, size_t bytes, uint64_t* checksum, int3
     return KVS_OK;
 }
 
-// ---------------------------------------------------------------------------------------
-// Attention without any caller- or library-allocated scratch.
-//
-// The split-K partial results and the device status word of this one entry point live in a
-// fixed array that is part of the loaded library image.  Every GPU that loads the library
-// carries these kStaticScratchBytes until the process exits, and every call, from every
-// context, uses the same bytes.
-// ---------------------------------------------------------------------------------------
-constexpr size_t kStaticScratchBytes = 2u << 20;  // 2 MiB
-constexpr size_t kStaticStatusBytes = 256;        // first 256 bytes: device status word
-static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
-
-namespace {
-
-std::once_flag g_static_flag[64];
-cudaError_t g_static_err[64];
-unsigned char* g_static_ptr[64];
-
-// In host code `g_static_scratch` is only a handle for the symbol, not an address the GPU can
-// use, so the device address is looked up once per device (with that device current).
-cudaError_t static_scratch_for_device(int device, unsigned char** ptr) {
-    if (device < 0 || device >= 64) return cudaErrorInvalidDevice;
-    std::call_once(g_static_flag[device], [device]() {
-        void* p = nullptr;
-        g_static_err[device] = cudaGetSymbolAddress(&p, g_static_scratch);
-        g_static_ptr[device] = static_cast<unsigned char*>(p);
-    });
-    *ptr = g_static_ptr[device];
-    return g_static_err[device];
-}
-
-}  // namespace
-
 kvs_status kvs_decode_attention_static(kvs_ctx* ctx, int32_t layer, const void* q, float* out, int32_t batch,
                                        void* stream, int32_t* device_status) {
     kvs_status s = check_attention(ctx, layer, q, out, batch);
     if (s != KVS_OK) return s;
+    if (((uintptr_t)device_status % 4) != 0) return KVS_ERR_INVALID_ARG;   // the kernels update it atomically
     kvs_ctx* c = ctx;
     const int slot = c->slot_of_layer[layer];
     const int units = batch * c->cfg.n_kv_heads;
@@ -967,17 +1022,21 @@ kvs_status kvs_decode_attention_static(kvs_ctx* ctx, int32_t layer, const void* 
 
     DeviceGuard guard(c->cfg.device);
     if (!guard.ok) return KVS_ERR_CUDA;
-    unsigned char* base = nullptr;
-    if (static_scratch_for_device(c->cfg.device, &base) != cudaSuccess || base == nullptr) return KVS_ERR_CUDA;
+    // the address was looked up when the context's memory was bound (per-device set-up): no
+    // runtime query here
+    unsigned char* base = g_static_ptr[c->cfg.device];
+    if (g_static_err[c->cfg.device] != cudaSuccess || base == nullptr) return KVS_ERR_CUDA;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     int* status_word = device_status ? device_status : reinterpret_cast<int*>(base);
     // the array keeps whatever the previous call left; only the status word must start at zero
     if (cudaMemsetAsync(status_word, 0, sizeof(int), st) != cudaSuccess) return KVS_ERR_CUDA;
-    // plain launches: the kernels start after everything before them on the stream
+    // Plain launches: the kernels start after everything before them on `stream`.  The call may be
+    // on another stream than the context's other calls, so it stays out of the bookkeeping that
+    // decides what those calls may fetch early (untracked), and it leaves the "growth counter was
+    // just written" mark for the next call of the chain.
     const AttentionScratch scratch = {reinterpret_cast<float*>(base + kStaticStatusBytes),
                                       reinterpret_cast<float*>(base + kStaticStatusBytes + part_o_bytes), status_word,
-                                      false};
-    c->counter_written = false;
+                                      false, false};
     return run_attention(c, slot, q, out, batch, plan, use_mma, scratch, st);
 }
 

@@ -57,11 +57,11 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 }
 
 // Wait for the phase with the given parity to complete.  Bounded: gives up when
-// kWaitLimitNs have passed or when another thread of the CTA has already given
-// up (*abort_flag != 0).  Returns false on giving up; the caller must then stop
-// consuming data, and the status word is set to kDevTimeout.
+// limit_ns (by default kWaitLimitNs) have passed or when another thread of the CTA
+// has already given up (*abort_flag != 0).  Returns false on giving up; the caller
+// must then stop consuming data, and the status word is set to kDevTimeout.
 __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, volatile int* abort_flag,
-                                                  int* status) {
+                                                  int* status, unsigned long long limit_ns = kWaitLimitNs) {
     if (mbar_try_wait(bar, parity)) return true;
     const unsigned long long t0 = globaltimer_ns();
     uint32_t spins = 0;
@@ -69,7 +69,7 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity
         if (mbar_try_wait(bar, parity)) return true;
         if ((++spins & 0xffu) == 0) {
             if (*abort_flag != 0) return false;
-            if (globaltimer_ns() - t0 > kWaitLimitNs) {
+            if (globaltimer_ns() - t0 > limit_ns) {
                 *abort_flag = 1;
                 atomicExch(status, kDevTimeout);
                 return false;

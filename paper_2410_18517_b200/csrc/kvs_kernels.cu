@@ -204,7 +204,9 @@ struct ScalarShape {
     static constexpr int QBYTES = G * RB;
     static constexpr int STAGE_BYTES = 2 * TILE + QBYTES;
     static constexpr int SCRATCH_FLOATS = NG * (D + 2);
-    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + SCRATCH_FLOATS * 4 + 2 * STAGES * 8 + 16;
+    // groups of more than four q-heads keep the piece's queries in shared memory instead of registers
+    static constexpr int QKEEP_BYTES = G > 4 ? QBYTES : 0;
+    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + SCRATCH_FLOATS * 4 + 2 * STAGES * 8 + 16 + QKEEP_BYTES;
     static_assert(R >= 1 && R <= LPR && (R & (R - 1)) == 0, "rows per group must be a power of two <= lanes per row");
     static_assert(TN % NG == 0, "tile rows must divide evenly among lane groups");
 };
@@ -281,6 +283,8 @@ __global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G, GEOM>::MI
     constexpr int kTile = S::TILE;
     constexpr int RB = S::RB, LPR = S::LPR, EPL = S::EPL, NG = S::NG, TN = S::TN, R = S::R, STAGES = S::STAGES;
     constexpr int SH = Log2<LPR>::value - Log2<R>::value;  // lane-in-group >> SH = row index held after the reduction
+    // q-heads taken together over a staged tile (bf16 lanes hold eight elements per head, fp32 lanes four)
+    constexpr int GP = G > 4 ? (sizeof(T) == 2 ? 2 : 4) : G;
 
     extern __shared__ __align__(128) unsigned char smem[];
     unsigned char* stage_base = smem;
@@ -288,6 +292,7 @@ __global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G, GEOM>::MI
     uint64_t* full_bar = reinterpret_cast<uint64_t*>(scratch + S::SCRATCH_FLOATS);
     uint64_t* empty_bar = full_bar + STAGES;
     volatile int* abort_flag = reinterpret_cast<volatile int*>(empty_bar + STAGES);
+    uint4* q_keep = reinterpret_cast<uint4*>(reinterpret_cast<unsigned char*>(empty_bar + STAGES) + 16);   // G > 4 only
 
     const int tid = threadIdx.x;
     const int warp = tid >> 5;
@@ -393,7 +398,7 @@ __global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G, GEOM>::MI
         const int piece_tiles = (int)min((long long)(a.tpu - ti0), t1 - gt);
         const int n_u = a.unit_len ? min(a.unit_len[u], a.cap) : a.n;
 
-        float qf[G][EPL];
+        float qf[G > 4 ? 1 : G][EPL];   // larger groups read their queries from q_keep, four heads at a time
         float m[G], lsum[G], acc[G][EPL];
 #pragma unroll
         for (int g = 0; g < G; ++g) {
@@ -410,12 +415,19 @@ __global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G, GEOM>::MI
             const unsigned char* vs = ks + kTile;
             if (k == 0) {
                 const unsigned char* qs = vs + kTile;
+                if constexpr (G > 4) {
+                    // every warp is past the previous piece's last tile (the merge barriers), so the
+                    // buffer is free; the stage that carries q is released after this tile
+                    for (int c = tid; c < G * LPR; c += kConsumerThreads) q_keep[c] = reinterpret_cast<const uint4*>(qs)[c];
+                    named_bar_sync(2, kConsumerThreads);
+                } else {
 #pragma unroll
-                for (int g = 0; g < G; ++g) {
-                    const uint4 raw = *reinterpret_cast<const uint4*>(qs + g * RB + lig * 16);
-                    Unpack<T>::run(raw, qf[g]);
+                    for (int g = 0; g < (G > 4 ? 1 : G); ++g) {
+                        const uint4 raw = *reinterpret_cast<const uint4*>(qs + g * RB + lig * 16);
+                        Unpack<T>::run(raw, qf[g]);
 #pragma unroll
-                    for (int e = 0; e < EPL; ++e) qf[g][e] *= a.scale_log2;
+                        for (int e = 0; e < EPL; ++e) qf[g][e] *= a.scale_log2;
+                    }
                 }
             }
             const int valid = min(TN, n_u - (ti0 + k) * TN);   // <= 0 for tiles past a ragged unit's end
@@ -425,54 +437,73 @@ __global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G, GEOM>::MI
                 continue;
             }
 
-            // scores: partial dot products of this lane's 16-byte chunk
-            float s[G][R];
+            // The q-heads of the group are taken GP at a time over the staged tile (all of them when
+            // the group has at most four): with eight heads at once the scores and weights of a tile
+            // (2 * 8 * R values) and the queries would not fit in registers beside the running state.
 #pragma unroll
-            for (int i = 0; i < R; ++i) {
-                const int row = grp + NG * i;
-                const uint4 raw = *reinterpret_cast<const uint4*>(ks + row * RB + lig * 16);
-                float kf[EPL];
-                Unpack<T>::run(raw, kf);
+            for (int g0 = 0; g0 < G; g0 += GP) {
+                // this pass's queries: registers, or (large groups) this lane's chunk from q_keep
+                float qp[GP][EPL];
 #pragma unroll
-                for (int g = 0; g < G; ++g) {
-                    float d = 0.f;
+                for (int g = 0; g < GP; ++g) {
+                    if constexpr (G > 4) {
+                        Unpack<T>::run(q_keep[(g0 + g) * LPR + lig], qp[g]);
 #pragma unroll
-                    for (int e = 0; e < EPL; ++e) d = fmaf(qf[g][e], kf[e], d);
-                    s[g][i] = d;
+                        for (int e = 0; e < EPL; ++e) qp[g][e] *= a.scale_log2;
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < EPL; ++e) qp[g][e] = qf[g0 + g][e];
+                    }
                 }
-            }
-            // online softmax per q-head, local to the lane group
-            float p[G][R];
-            const bool mine_valid = (grp + NG * my_i) < valid;
+                // scores: partial dot products of this lane's 16-byte chunk
+                float s[GP][R];
 #pragma unroll
-            for (int g = 0; g < G; ++g) {
-                float sv = reduce_transpose<R, LPR / 2>(s[g], lig);
-                sv = mine_valid ? sv : -INFINITY;
-                float tmax = sv;
+                for (int i = 0; i < R; ++i) {
+                    const int row = grp + NG * i;
+                    const uint4 raw = *reinterpret_cast<const uint4*>(ks + row * RB + lig * 16);
+                    float kf[EPL];
+                    Unpack<T>::run(raw, kf);
 #pragma unroll
-                for (int o = LPR / 2; o >= LPR / R; o >>= 1) tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, o));
-                const float m_new = fmaxf(m[g], tmax);
-                const float alpha = fast_exp2(m[g] - m_new);
-                const float pv = fast_exp2(sv - m_new);
-                m[g] = m_new;
-                lsum[g] = lsum[g] * alpha + pv;
+                    for (int g = 0; g < GP; ++g) {
+                        float d = 0.f;
 #pragma unroll
-                for (int e = 0; e < EPL; ++e) acc[g][e] *= alpha;
+                        for (int e = 0; e < EPL; ++e) d = fmaf(qp[g][e], kf[e], d);
+                        s[g][i] = d;
+                    }
+                }
+                // online softmax per q-head, local to the lane group
+                float p[GP][R];
+                const bool mine_valid = (grp + NG * my_i) < valid;
 #pragma unroll
-                for (int i = 0; i < R; ++i) p[g][i] = __shfl_sync(0xffffffffu, pv, i << SH, LPR);
-            }
-            // weighted sum of value rows
+                for (int g = 0; g < GP; ++g) {
+                    float sv = reduce_transpose<R, LPR / 2>(s[g], lig);
+                    sv = mine_valid ? sv : -INFINITY;
+                    float tmax = sv;
 #pragma unroll
-            for (int i = 0; i < R; ++i) {
-                const int row = grp + NG * i;
-                if (row < valid) {
-                    const uint4 raw = *reinterpret_cast<const uint4*>(vs + row * RB + lig * 16);
-                    float vf[EPL];
-                    Unpack<T>::run(raw, vf);
+                    for (int o = LPR / 2; o >= LPR / R; o >>= 1) tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, o));
+                    const float m_new = fmaxf(m[g0 + g], tmax);
+                    const float alpha = fast_exp2(m[g0 + g] - m_new);
+                    const float pv = fast_exp2(sv - m_new);
+                    m[g0 + g] = m_new;
+                    lsum[g0 + g] = lsum[g0 + g] * alpha + pv;
 #pragma unroll
-                    for (int g = 0; g < G; ++g)
+                    for (int e = 0; e < EPL; ++e) acc[g0 + g][e] *= alpha;
 #pragma unroll
-                        for (int e = 0; e < EPL; ++e) acc[g][e] = fmaf(p[g][i], vf[e], acc[g][e]);
+                    for (int i = 0; i < R; ++i) p[g][i] = __shfl_sync(0xffffffffu, pv, i << SH, LPR);
+                }
+                // weighted sum of value rows
+#pragma unroll
+                for (int i = 0; i < R; ++i) {
+                    const int row = grp + NG * i;
+                    if (row < valid) {
+                        const uint4 raw = *reinterpret_cast<const uint4*>(vs + row * RB + lig * 16);
+                        float vf[EPL];
+                        Unpack<T>::run(raw, vf);
+#pragma unroll
+                        for (int g = 0; g < GP; ++g)
+#pragma unroll
+                            for (int e = 0; e < EPL; ++e) acc[g0 + g][e] = fmaf(p[g][i], vf[e], acc[g0 + g][e]);
+                    }
                 }
             }
             __syncwarp();
@@ -748,6 +779,37 @@ cudaError_t launch_read_roof(const void* src, size_t bytes, unsigned long long* 
     cudaError_t e = cudaMemsetAsync(checksum, 0, 8, stream);
     if (e != cudaSuccess) return e;
     read_roof_kernel<<<NC, kScalarThreads, kRoofSmem, stream>>>((const char*)src, n_tiles, checksum);
+    return cudaGetLastError();
+}
+
+// --------------------------------------------------------------------------------------
+// Self-test of the give-up path of the bounded waits: one thread waits on a barrier that
+// nothing ever arrives at, with a short limit, through the same mbar_wait_bounded the
+// pipelined kernels use.  No copy is in flight; the wait runs out, the status word becomes
+// kDevTimeout and the kernel returns normally.
+// --------------------------------------------------------------------------------------
+__global__ void wait_timeout_selftest_kernel(int* status, unsigned long long limit_ns, unsigned long long* waited_ns) {
+    __shared__ uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        abort_flag = 0;
+        fence_mbar_init();
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const unsigned long long t0 = globaltimer_ns();
+        const bool ok = mbar_wait_bounded(&bar, 0, &abort_flag, status, limit_ns);
+        if (waited_ns) *waited_ns = ok ? 0ull : globaltimer_ns() - t0;
+    }
+    __syncthreads();
+    // the other threads see the give-up through the flag, as the consumer warps of the real kernels do
+    if (threadIdx.x == 1 && abort_flag == 0) atomicExch(status, 1);
+}
+
+cudaError_t launch_wait_timeout_selftest(int* status, unsigned long long limit_ns, unsigned long long* waited_ns,
+                                         cudaStream_t stream) {
+    wait_timeout_selftest_kernel<<<1, 32, 0, stream>>>(status, limit_ns, waited_ns);
     return cudaGetLastError();
 }
 

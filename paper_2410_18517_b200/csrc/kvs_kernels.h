@@ -100,6 +100,10 @@ cudaError_t launch_set_len(int* unit_len, const int* counts, int units, bool pro
 cudaError_t launch_add_len(int* unit_len, int delta, int units, bool programmatic, cudaStream_t stream);
 cudaError_t launch_decode_scalar(const DecodeArgs& a, const DecodePlan& plan, cudaStream_t stream);
 cudaError_t launch_combine(const DecodeArgs& a, const DecodePlan& plan, cudaStream_t stream);
+// One thread waits, with the given limit, on a barrier nothing arrives at; *status receives the
+// time-out code and *waited_ns (device, may be null) how long the wait lasted.
+cudaError_t launch_wait_timeout_selftest(int* status, unsigned long long limit_ns, unsigned long long* waited_ns,
+                                         cudaStream_t stream);
 cudaError_t launch_read_roof(const void* src, size_t bytes, unsigned long long* checksum, int sm_count,
                              cudaStream_t stream);
 

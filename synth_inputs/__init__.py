@@ -95,6 +95,16 @@ def sweep_points():
     return pts
 
 
+def workload_by_name(name: str) -> Workload:
+    """A named configuration, or a sweep point by its name (``sweep_b32_n8192_p10``)."""
+    if name in WORKLOADS:
+        return WORKLOADS[name]
+    for w in sweep_points():
+        if w.name == name:
+            return w
+    raise KeyError(f"unknown workload {name!r}")
+
+
 def random_share_map(L: int, n_shared: int, seed: int) -> np.ndarray:
     """A random strategy with ``n_shared`` replaced layers.
 

@@ -51,7 +51,9 @@ SHAPES = [
     # dtype, D, Hq, Hkv
     ("bf16", 128, 4, 4), ("bf16", 128, 8, 2), ("bf16", 128, 4, 2), ("bf16", 128, 8, 1),
     ("bf16", 64, 4, 4), ("bf16", 64, 8, 2),
-    ("f32", 64, 2, 2), ("f32", 128, 2, 2), ("f32", 128, 4, 1),
+    ("f32", 64, 2, 2), ("f32", 128, 2, 2), ("f32", 128, 4, 1), ("f32", 128, 4, 2),
+    # groups of eight q-heads with fp32 storage exist on the scalar kernel only (two passes of four heads)
+    ("f32", 128, 8, 1), ("f32", 64, 8, 1), ("f32", 64, 16, 2),
 ]
 
 
