@@ -105,8 +105,13 @@ typedef enum {
     KVS_OPT_REPLAY = 3,     /* 1: launches also read a device-side growth counter, so that a
                                recorded decode step can be replayed as a CUDA graph (see
                                kvs_replay_advance).  0 (default): lengths come from the host only. */
-    KVS_OPT_HOST_CHUNKS = 4 /* kvs_step_host: number of pieces (1..8, default 4) the layers are cut
+    KVS_OPT_HOST_CHUNKS = 4,/* kvs_step_host: number of pieces (1..8, default 4) the layers are cut
                                into for overlapping the host copies with the kernels.            */
+    KVS_OPT_FINISH_IN_KERNEL = 5 /* 1 (default): when a call has at least as many (sequence, kv-head) units as
+                               thread blocks, no unit is cut into more than two pieces and the split-K
+                               kernel merges them itself (the block that holds a unit's first piece reads
+                               the second, which the next block finished early in the same launch): one
+                               launch per call instead of two.  0: always the separate combine kernel. */
 } kvs_option;
 
 /* ---- life cycle ------------------------------------------------------------ */

@@ -31,6 +31,7 @@ KVS_OPT_KERNEL = 1
 KVS_OPT_EARLY_START = 2
 KVS_OPT_REPLAY = 3
 KVS_OPT_HOST_CHUNKS = 4
+KVS_OPT_FINISH_IN_KERNEL = 5
 
 # every symbol include/kvs.h declares
 EXPORTS = (

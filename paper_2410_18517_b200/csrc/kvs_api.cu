@@ -80,9 +80,10 @@ struct kvs_ctx {
 
     // workspace carve-up (byte offsets)
     size_t off_status = 0, off_part_o = 0, off_part_ml = 0, off_stage_q = 0, off_stage_k = 0, off_stage_v = 0,
-           off_stage_out = 0, off_unit_len = 0, off_counts = 0, off_search = 0, off_replay = 0, ws_bytes = 0;
+           off_stage_out = 0, off_unit_len = 0, off_counts = 0, off_search = 0, off_replay = 0, off_flags = 0, ws_bytes = 0;
 
-    alignas(64) unsigned char tensor_map[128];  // TMA view of the pool (bf16 storage only)
+    alignas(64) unsigned char tensor_map[128];  // TMA view of the pool (bf16 storage only), 64-row boxes
+    alignas(64) unsigned char tensor_map_tail[128];   // the same view with 16-row boxes (partly filled tiles)
     bool have_tensor_map = false;
 
     // Launch bookkeeping for early-start (programmatic) launches.  Every kernel of this context
@@ -104,6 +105,7 @@ struct kvs_ctx {
     int opt_kernel = 0;
     int opt_pdl = 1;
     int opt_host_chunks = 4;
+    int opt_finish = 1;   // units of at most two pieces are finished by the split-K kernel itself (no combine launch)
     int opt_replay = 0;   // launches carry the device-side growth counter (for CUDA-graph replay)
     // The split-K kernels read the growth counter before their wait.  That is safe because the
     // first launch after anything wrote the counter never starts early (full dependency): it and
@@ -189,6 +191,8 @@ void layout_workspace(kvs_ctx* c) {
     off = align_up(off + units * sizeof(int32_t), kAlign);
     c->off_replay = off;        // one int: rows every slot has grown by since a recorded launch
     off += kAlign;
+    c->off_flags = off;         // one int per unit: "second piece written" (zero between launches)
+    off = align_up(off + units * sizeof(int32_t), kAlign);
     c->off_search = off;        // per-block partial sums of the strategy-search reductions
     {
         const size_t need = std::max(kvs::distance_partial_bytes(f.n_layers <= kvs::kMaxLayersSearch ? f.n_layers : 4),
@@ -285,6 +289,7 @@ kvs_status do_append(kvs_ctx* c, int layer, const void* k, const void* v, int ba
 struct AttentionScratch {
     float* part_o;
     float* part_ml;
+    int* flags;          // [units] ints, zero between launches
     int* status;
     bool programmatic;   // early-start launches (only when the call follows this context's own kernels)
     bool tracked;        // the call is part of the context's one ordered chain of launches (see kvs_ctx::seq)
@@ -330,22 +335,26 @@ kvs_status run_attention(kvs_ctx* c, int slot, const void* q, float* out, int ba
     a.k_new = k_new;
     a.v_new = v_new;
     if (k_new) a.safe_rows = std::min(a.safe_rows, a.n - 1);   // the new row is fetched after the kernel has stored it
+    a.finish_in_kernel = c->opt_finish != 0 && kvs::can_finish_in_kernel(plan, a.units);
+    a.flags = scratch.flags;
     if (scratch.tracked) {
-        c->seq += 2;                       // split-K kernel, then combine
-        c->last_splitk_seq = c->seq - 1;
+        c->seq += a.finish_in_kernel ? 1 : 2;     // split-K kernel, then (unless it finishes the units itself) combine
+        c->last_splitk_seq = a.finish_in_kernel ? c->seq : c->seq - 1;
     }
     if (use_mma) {
         const long long plane_rows = (long long)c->cfg.max_batch * c->cfg.n_kv_heads * c->row_stride;
-        if (kvs::launch_decode_mma(a, plan, c->tensor_map, plane_rows * (2 * slot), plane_rows * (2 * slot + 1), st) !=
-            cudaSuccess)
+        if (kvs::launch_decode_mma(a, plan, c->tensor_map, c->tensor_map_tail, plane_rows * (2 * slot),
+                                   plane_rows * (2 * slot + 1), st) != cudaSuccess)
             return KVS_ERR_CUDA;
     } else {
         if (kvs::launch_decode_scalar(a, plan, st) != cudaSuccess) return KVS_ERR_CUDA;
     }
-    if (kvs::launch_combine(a, plan, st) != cudaSuccess) return KVS_ERR_CUDA;
+    if (!a.finish_in_kernel) {
+        if (kvs::launch_combine(a, plan, st) != cudaSuccess) return KVS_ERR_CUDA;
+        c->stats.combine_launches += 1;
+    }
     c->last_plan = plan;
     c->stats.attention_launches += 1;
-    c->stats.combine_launches += 1;
     if (c->ragged[slot]) {
         unsigned long long rows = 0;
         for (int u = 0; u < a.units; ++u) rows += c->unit_len_host[slot][u];
@@ -366,6 +375,7 @@ kvs_status do_fused_step(kvs_ctx* c, int layer, const void* q, const void* k, co
     const bool use_mma = choose_plan(c, batch * c->cfg.n_kv_heads, old_len + 1, &plan);
     const AttentionScratch scratch = {reinterpret_cast<float*>(c->ws + c->off_part_o),
                                       reinterpret_cast<float*>(c->ws + c->off_part_ml),
+                                      reinterpret_cast<int*>(c->ws + c->off_flags),
                                       reinterpret_cast<int*>(c->ws + c->off_status), take_early_start(c), true};
     // run_attention works out which rows are stable from the appends before this one
     c->slot_len[slot] = old_len + 1;
@@ -389,6 +399,7 @@ kvs_status do_attention(kvs_ctx* c, int layer, const void* q, float* out, int ba
     const bool use_mma = choose_plan(c, batch * c->cfg.n_kv_heads, c->slot_len[slot], &plan);
     const AttentionScratch scratch = {reinterpret_cast<float*>(c->ws + c->off_part_o),
                                       reinterpret_cast<float*>(c->ws + c->off_part_ml),
+                                      reinterpret_cast<int*>(c->ws + c->off_flags),
                                       reinterpret_cast<int*>(c->ws + c->off_status), take_early_start(c), true};
     return run_attention(c, slot, q, out, batch, plan, use_mma, scratch, st);
 }
@@ -491,7 +502,8 @@ kvs_status kvs_bind_memory(kvs_ctx* ctx, void* pool, size_t pool_bytes, void* wo
     if (ctx->cfg.dtype == KVS_BF16) {
         const long long total_rows = (long long)(need_pool / ctx->row_bytes);
         if (total_rows >= (1ll << 31)) return KVS_ERR_INVALID_ARG;
-        if (kvs::make_pool_tensor_map(ctx->tensor_map, pool, total_rows, ctx->cfg.head_dim) != cudaSuccess)
+        if (kvs::make_pool_tensor_map(ctx->tensor_map, pool, total_rows, ctx->cfg.head_dim, false) != cudaSuccess ||
+            kvs::make_pool_tensor_map(ctx->tensor_map_tail, pool, total_rows, ctx->cfg.head_dim, true) != cudaSuccess)
             return KVS_ERR_CUDA;
         ctx->have_tensor_map = true;
     }
@@ -955,6 +967,10 @@ kvs_status kvs_set_option(kvs_ctx* ctx, int32_t option, int32_t value) {
             if (value < 1 || value > kvs_ctx::kChunks) return KVS_ERR_INVALID_ARG;
             ctx->opt_host_chunks = value;
             return KVS_OK;
+        case KVS_OPT_FINISH_IN_KERNEL:
+            if (value != 0 && value != 1) return KVS_ERR_INVALID_ARG;
+            ctx->opt_finish = value;
+            return KVS_OK;
         case KVS_OPT_KERNEL:
             if (value < 0 || value > 2) return KVS_ERR_INVALID_ARG;
             if (value == 2 && ctx->cfg.dtype != KVS_BF16) return KVS_ERR_INVALID_ARG;  // tensor-core path is bf16 only
@@ -1018,7 +1034,8 @@ kvs_status kvs_decode_attention_static(kvs_ctx* ctx, int32_t layer, const void* 
     const size_t pieces = (size_t)units + plan.NC;
     const size_t part_o_bytes = align_up(pieces * c->G * D * sizeof(float), kAlign);
     const size_t part_ml_bytes = align_up(pieces * c->G * 2 * sizeof(float), kAlign);
-    if (kStaticStatusBytes + part_o_bytes + part_ml_bytes > kStaticScratchBytes) return KVS_ERR_SCRATCH_LIMIT;
+    const size_t flag_bytes = align_up((size_t)units * sizeof(int32_t), kAlign);   // zero at load, and again after every launch
+    if (kStaticStatusBytes + part_o_bytes + part_ml_bytes + flag_bytes > kStaticScratchBytes) return KVS_ERR_SCRATCH_LIMIT;
 
     DeviceGuard guard(c->cfg.device);
     if (!guard.ok) return KVS_ERR_CUDA;
@@ -1034,9 +1051,10 @@ kvs_status kvs_decode_attention_static(kvs_ctx* ctx, int32_t layer, const void* 
     // on another stream than the context's other calls, so it stays out of the bookkeeping that
     // decides what those calls may fetch early (untracked), and it leaves the "growth counter was
     // just written" mark for the next call of the chain.
-    const AttentionScratch scratch = {reinterpret_cast<float*>(base + kStaticStatusBytes),
-                                      reinterpret_cast<float*>(base + kStaticStatusBytes + part_o_bytes), status_word,
-                                      false, false};
+    // the flags come first so that they sit at the same place whatever the call's size
+    const AttentionScratch scratch = {reinterpret_cast<float*>(base + kStaticStatusBytes + flag_bytes),
+                                      reinterpret_cast<float*>(base + kStaticStatusBytes + flag_bytes + part_o_bytes),
+                                      reinterpret_cast<int*>(base + kStaticStatusBytes), status_word, false, false};
     return run_attention(c, slot, q, out, batch, plan, use_mma, scratch, st);
 }
 

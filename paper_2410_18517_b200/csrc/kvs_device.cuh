@@ -78,6 +78,38 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity
     }
 }
 
+// A flag in global memory through which one thread block tells another, inside one launch, that
+// data it wrote is ready: the writer stores with release semantics after a barrier with the threads
+// that wrote the data, the reader polls with acquire semantics and then passes a barrier with the
+// threads that will read it.
+__device__ __forceinline__ void st_release_gpu(int* p, int v) {
+    asm volatile("st.release.gpu.global.b32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ int ld_acquire_gpu(const int* p) {
+    int v;
+    asm volatile("ld.acquire.gpu.global.b32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+// Bounded like mbar_wait_bounded: false (status word set, *abort_flag raised) when the flag has not
+// taken the value within the limit.
+__device__ __forceinline__ bool flag_wait_bounded(const int* flag, int want, volatile int* abort_flag, int* status,
+                                                  unsigned long long limit_ns = kWaitLimitNs) {
+    if (ld_acquire_gpu(flag) == want) return true;
+    const unsigned long long t0 = globaltimer_ns();
+    uint32_t spins = 0;
+    while (true) {
+        if (ld_acquire_gpu(flag) == want) return true;
+        if ((++spins & 0x3fu) == 0) {
+            if (*abort_flag != 0) return false;
+            if (globaltimer_ns() - t0 > limit_ns) {
+                *abort_flag = 1;
+                atomicExch(status, kDevTimeout);
+                return false;
+            }
+        }
+    }
+}
+
 // 1-D bulk copy global -> shared memory of this CTA; completion is reported as
 // `bytes` transaction bytes on `bar`.  Both addresses must be 16-byte aligned
 // and `bytes` a non-zero multiple of 16.  (The destination state space is

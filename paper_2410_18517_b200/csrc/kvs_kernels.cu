@@ -170,7 +170,7 @@ __host__ __device__ __forceinline__ int cta_of_tile(long long gt, long long T, i
 #endif
 constexpr int kConsumerWarps = KVS_CONSUMER_WARPS;
 constexpr int kConsumerThreads = kConsumerWarps * 32;
-constexpr int kScalarThreads = kConsumerThreads + 32;
+constexpr int kScalarThreads = kConsumerThreads + 64;   // + the producer warp and the hand-over warp
 // Tile size, ring depth and blocks per SM of the scalar kernel for groups of 1 or 2 q-heads
 // (compile-time; the defaults are the measured best on B200).
 #ifndef KVS_TILE_BYTES
@@ -206,7 +206,9 @@ struct ScalarShape {
     static constexpr int SCRATCH_FLOATS = NG * (D + 2);
     // groups of more than four q-heads keep the piece's queries in shared memory instead of registers
     static constexpr int QKEEP_BYTES = G > 4 ? QBYTES : 0;
-    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + SCRATCH_FLOATS * 4 + 2 * STAGES * 8 + 16 + QKEEP_BYTES;
+    static constexpr int HANDOVER_FLOATS = G * (D + 2);   // another block's piece of a cut unit: [q-head][D + 2]
+    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + SCRATCH_FLOATS * 4 + (2 * STAGES + 2) * 8 + 16 + QKEEP_BYTES +
+                                      HANDOVER_FLOATS * 4;
     static_assert(R >= 1 && R <= LPR && (R & (R - 1)) == 0, "rows per group must be a power of two <= lanes per row");
     static_assert(TN % NG == 0, "tile rows must divide evenly among lane groups");
 };
@@ -263,6 +265,9 @@ struct ScalarKernelArgs {
     int cap;              // rows a unit can hold: lengths that grew on the device are cut off there
     const char* k_new;    // the step's new rows, appended by this kernel (n counts them), or nullptr
     const char* v_new;
+    // Finishing inside this kernel (no combine launch): set when no unit has more than two pieces.
+    float* out;           // [units][G][D] final results, or nullptr: every piece goes to part_o / part_ml
+    int* flags;           // [units], all zero between launches: 1 = the unit's second piece is in part_o / part_ml
 };
 
 template <typename T, int D, int G, int GEOM>
@@ -291,8 +296,11 @@ __global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G, GEOM>::MI
     float* scratch = reinterpret_cast<float*>(smem + STAGES * S::STAGE_BYTES);
     uint64_t* full_bar = reinterpret_cast<uint64_t*>(scratch + S::SCRATCH_FLOATS);
     uint64_t* empty_bar = full_bar + STAGES;
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(empty_bar + STAGES);
-    uint4* q_keep = reinterpret_cast<uint4*>(reinterpret_cast<unsigned char*>(empty_bar + STAGES) + 16);   // G > 4 only
+    uint64_t* tail_bar = empty_bar + STAGES;         // every consumer thread has written this block's second-piece partial
+    uint64_t* head_bar = tail_bar + 1;               // the next block's second-piece partial is in handover[]
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(head_bar + 1);
+    uint4* q_keep = reinterpret_cast<uint4*>(reinterpret_cast<unsigned char*>(head_bar + 1) + 16);   // G > 4 only
+    float* handover = reinterpret_cast<float*>(reinterpret_cast<unsigned char*>(q_keep) + S::QKEEP_BYTES);
 
     const int tid = threadIdx.x;
     const int warp = tid >> 5;
@@ -306,6 +314,8 @@ __global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G, GEOM>::MI
             mbar_init(&full_bar[s], 1);
             mbar_init(&empty_bar[s], kConsumerWarps);
         }
+        mbar_init(tail_bar, kConsumerThreads);
+        mbar_init(head_bar, 1);
         abort_flag[0] = 0;
         abort_flag[1] = 0;  // second word: bounds the producer's drain after a give-up
         fence_mbar_init();
@@ -356,6 +366,9 @@ __global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G, GEOM>::MI
             }
             pdl_wait();
             pdl_launch_dependents();
+            // first the queries of the tiles already fetched (the consumers wait for nothing else), then the new rows
+            if (lane == 0)
+                for (int j = 0; j < npre; ++j) issue(t0 + j, j, false, false, true);
             if (a.k_new != nullptr) {
                 if (!over)
                     store_new_rows<RB>(lane, t0, t1, a.tpu, a.n, a.row_stride, a.k_new, a.v_new, const_cast<char*>(a.kplane),
@@ -364,7 +377,6 @@ __global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G, GEOM>::MI
                     atomicExch(a.status, 4);
             }
             if (lane != 0) return;
-            for (int j = 0; j < npre; ++j) issue(t0 + j, j, false, false, true);
             int it = npre;
             bool ok = true;
             for (long long gt = t0 + npre; gt < t1 && ok; ++gt, ++it) {
@@ -378,6 +390,39 @@ __global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G, GEOM>::MI
                 // is in flight into this block's shared memory when it exits.
                 for (int j = max(0, it - STAGES); j < it; ++j)
                     mbar_wait_bounded(&full_bar[j % STAGES], (j / STAGES) & 1, abort_flag + 1, a.status);
+            }
+        }
+        return;
+    }
+
+    if (warp == kConsumerWarps + 1) {
+        // ------------------ hand-over of units that are cut between two blocks ------------------
+        // Only when the kernel finishes the units itself (a.out set).  The global round trips of the
+        // hand-over are made here, beside the stream: this warp raises the flag of the unit whose
+        // second piece this block computed first, and fetches the second piece of the unit whose
+        // first piece this block computes last, so that the consumers find it in shared memory.
+        if (a.out == nullptr || t0 >= t1) return;
+        const bool has_tail = (t0 % a.tpu) != 0, has_head = (t1 % a.tpu) != 0;
+        if (!has_tail && !has_head) return;
+        pdl_wait();   // the flags are back to zero only once the previous launch has completed
+        if (has_tail) {
+            if (!mbar_wait_bounded(tail_bar, 0, abort_flag, a.status)) return;
+            if (lane == 0) st_release_gpu(a.flags + t0 / a.tpu, 1);
+        }
+        if (has_head) {
+            const long long u = (t1 - 1) / a.tpu;
+            int ok = 1;
+            if (lane == 0) ok = flag_wait_bounded(a.flags + u, 1, abort_flag, a.status) ? 1 : 0;
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+            if (!ok) return;
+            // written by another SM during this launch: read past L1
+            const long long pt = u + blockIdx.x + 1;
+            for (int i = lane; i < G * D; i += 32) handover[(i / D) * (D + 2) + (i % D)] = __ldcg(a.part_o + pt * G * D + i);
+            for (int i = lane; i < G * 2; i += 32) handover[(i >> 1) * (D + 2) + D + (i & 1)] = __ldcg(a.part_ml + pt * G * 2 + i);
+            __syncwarp();
+            if (lane == 0) {
+                a.flags[u] = 0;          // this block is the flag's only reader
+                mbar_arrive(head_bar);
             }
         }
         return;
@@ -511,7 +556,18 @@ __global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G, GEOM>::MI
         }
 
         // ---- end of piece: merge the NG lane groups, one q-head at a time ----
+        // With a.out set (no unit has more than two pieces) the kernel finishes the units itself: a unit
+        // that lies inside this block's share is normalised and written out; of a unit cut in two the
+        // second piece, which is the FIRST piece of the next block and so done early in the launch, goes
+        // to part_o / part_ml and the hand-over warp raises the unit's flag; the block that holds the
+        // first piece comes to it LAST, by when its hand-over warp has fetched the second piece into
+        // shared memory; it merges the two in piece order and writes the result.
         const long long pid = u + blockIdx.x;
+        const bool finish = a.out != nullptr;
+        const bool whole = finish && ti0 == 0 && piece_tiles == a.tpu;
+        const bool head = finish && ti0 == 0 && piece_tiles < a.tpu;
+        const bool tail = finish && ti0 > 0;
+        if (head && !mbar_wait_bounded(head_bar, 0, abort_flag, a.status)) return;
 #pragma unroll
         for (int g = 0; g < G; ++g) {
             // lanes with equal top bits hold duplicates of lsum; add across the R distinct ones
@@ -538,86 +594,131 @@ __global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G, GEOM>::MI
                     o = fmaf(w, scratch[j * (D + 2) + d], o);
                     den = fmaf(w, scratch[j * (D + 2) + D + 1], den);
                 }
-                a.part_o[(pid * G + g) * D + d] = o;
-                if (d == 0) {
-                    a.part_ml[(pid * G + g) * 2] = M;
-                    a.part_ml[(pid * G + g) * 2 + 1] = den;
+                if (whole) {
+                    a.out[(u * G + g) * D + d] = o / den;
+                } else if (head) {
+                    const float* hv = handover + g * (D + 2);      // the unit's second piece
+                    const float Mx = fmaxf(M, hv[D]);
+                    const float w0 = fast_exp2(M - Mx), w1 = fast_exp2(hv[D] - Mx);
+                    a.out[(u * G + g) * D + d] = fmaf(w1, hv[d], w0 * o) / fmaf(w1, hv[D + 1], w0 * den);
+                } else {
+                    a.part_o[(pid * G + g) * D + d] = o;
+                    if (d == 0) {
+                        a.part_ml[(pid * G + g) * 2] = M;
+                        a.part_ml[(pid * G + g) * 2 + 1] = den;
+                    }
                 }
             }
         }
+        if (tail) mbar_arrive(tail_bar);   // this thread's part of the piece is written
         gt += piece_tiles;
     }
 }
 
 // --------------------------------------------------------------------------------------
-// K3: combine.  One block per (unit, q-head), D threads; out = sum_c w_c o_c / sum_c w_c l_c
-// with w_c = 2^(m_c - M), M = max_c m_c over the pieces c of the unit, always summed in
-// piece order so that the result does not depend on which block finished first.
-// The (m, l) pairs of all pieces are fetched first, one piece per lane (independent loads, one
-// round trip to L2), the weights go through shared memory, and the loop over the pieces'
-// output vectors keeps eight loads in flight: with the pieces read one after the other this
-// kernel was the slowest of a small decode step.
+// K3: combine.  One WARP per (unit, q-head): out = sum_c w_c o_c / sum_c w_c l_c with
+// w_c = 2^(m_c - M), M = max_c m_c over the pieces c of the unit.  The output vectors are always
+// added in piece order and the denominators in a fixed lane order, so the result does not
+// depend on which block finished first.
+// Lane j fetches the (max, sum) pair of piece j (independent loads, one round trip to L2) while
+// the output vectors of the first pieces are already requested; weights travel by shuffle;
+// each lane owns D/32 consecutive output columns.  No shared memory and at most 48 registers:
+// the whole grid (eight items per block) becomes resident beside the split-K kernel it follows
+// (whose block leaves 14-34 K registers of the SM free), so that the split-K kernel of the NEXT
+// call, which may only start once every block of this grid has started, can move onto each SM
+// the moment the running split-K block leaves it.
 // --------------------------------------------------------------------------------------
-__global__ void decode_combine_kernel(const float* __restrict__ part_o, const float* __restrict__ part_ml,
-                                      float* __restrict__ out, int G, int D, int tpu, long long T, int NC,
-                                      const int* __restrict__ n_extra, int n, int tile_rows, int units, int cap) {
-    __shared__ float wsm[kMaxCtas], lsm[kMaxCtas];
-    __shared__ float msm[4];
+// Two builds: units of at most two pieces (every block's share is at least a unit long) take eight
+// items per block with two vectors requested early; longer units take four items per block and
+// four early vectors (64 registers), so that a unit of up to four pieces still needs one round trip.
+template <int D, int PRE, int kCombineWarps>
+__global__ void __launch_bounds__(kCombineWarps * 32, PRE == 2 ? 5 : 8)
+    decode_combine_kernel(const float* __restrict__ part_o, const float* __restrict__ part_ml, float* __restrict__ out,
+                          int G, int tpu, long long T, int NC, const int* __restrict__ n_extra, int n, int tile_rows,
+                          int units, int cap) {
+    constexpr int VEC = D / 32;
+    struct __align__(VEC * 4) Vec {
+        float v[VEC];
+    };
     pdl_launch_dependents();
     pdl_wait();
     if (n_extra) {   // replayed launch: recompute the tile line from the grown length
         tpu = (min(n + *n_extra, cap) + tile_rows - 1) / tile_rows;
         T = (long long)units * tpu;
     }
-    const long long u = blockIdx.x / G;
-    const int g = blockIdx.x % G;
+    const long long item = (long long)blockIdx.x * kCombineWarps + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (item >= (long long)units * G) return;
+    const long long u = item / G;
+    const int g = (int)(item - u * G);
     const int c0 = cta_of_tile(u * tpu, T, NC);
     const int np = cta_of_tile((u + 1) * tpu - 1, T, NC) - c0 + 1;       // pieces of this unit
-    const int d = threadIdx.x, lane = d & 31, warp = d >> 5;
     const float2* ml = reinterpret_cast<const float2*>(part_ml) + (u + c0) * G + g;   // piece c: ml[c * G]
-    // the first output vectors are requested together with the (max, sum) pairs: one round trip to
-    // L2 for a unit of up to four pieces
-    const float* po = part_o + ((u + c0) * G + g) * D + d;               // piece c: po[c * G * D]
-    float pre[4];
+    const Vec* po = reinterpret_cast<const Vec*>(part_o + ((u + c0) * G + g) * D) + lane;   // piece c: po[c * G * 32]
+    const int pstride = G * 32;     // offsets within one unit's pieces fit 32 bits
+    // first chunk of (max, sum) pairs and, in the same round trip, the first PRE output vectors
+    const float2 v0 = lane < np ? ml[lane * G] : make_float2(-1.0e30f, 0.f);
+    Vec pre[PRE];
 #pragma unroll
-    for (int c = 0; c < 4; ++c) pre[c] = (np <= 4 && c < np) ? po[(long long)c * G * D] : 0.f;   // (longer units: see below)
-    // every warp takes a share of the pieces: maxima and sums to shared memory
-    float mx = -1.0e30f;
-    for (int c = d; c < np; c += blockDim.x) {
-        const float2 v = ml[(long long)c * G];
-        wsm[c] = v.x;
-        lsm[c] = v.y;
-        mx = fmaxf(mx, v.x);
-    }
+    for (int c = 0; c < PRE; ++c)
+        if (c < np) pre[c] = po[c * pstride];
+    float M = v0.x;
+    for (int cb = 32; cb < np; cb += 32)
+        if (cb + lane < np) M = fmaxf(M, ml[(cb + lane) * G].x);
 #pragma unroll
-    for (int o = 16; o >= 1; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-    if (lane == 0) msm[warp] = mx;
-    __syncthreads();
-    float M = msm[0];
-    for (int w = 1; w < (int)(blockDim.x >> 5); ++w) M = fmaxf(M, msm[w]);
-    for (int c = d; c < np; c += blockDim.x) wsm[c] = fast_exp2(wsm[c] - M);
-    __syncthreads();
-    float o = 0.f, den = 0.f;
-    const int first = np <= 4 ? np : 0;     // units of more pieces fetch all their vectors here, eight at a time
+    for (int o = 16; o >= 1; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+    float acc[VEC];
 #pragma unroll
-    for (int c = 0; c < 4; ++c)
-        if (c < first) {
-            o = fmaf(wsm[c], pre[c], o);
-            den = fmaf(wsm[c], lsm[c], den);
+    for (int e = 0; e < VEC; ++e) acc[e] = 0.f;
+    float den = 0.f;     // this lane's share of the denominator (pieces lane, lane + 32, ...)
+    for (int cb = 0; cb < np; cb += 32) {
+        const float2 v = cb == 0 ? v0 : (cb + lane < np ? ml[(cb + lane) * G] : make_float2(-1.0e30f, 0.f));
+        const float w = cb + lane < np ? fast_exp2(v.x - M) : 0.f;
+        den = fmaf(w, v.y, den);
+        const int cnt = min(32, np - cb);
+        int j = 0;
+        if (cb == 0) {
+#pragma unroll
+            for (int c = 0; c < PRE; ++c)
+                if (c < cnt) {
+                    const float wj = __shfl_sync(0xffffffffu, w, c);
+#pragma unroll
+                    for (int e = 0; e < VEC; ++e) acc[e] = fmaf(wj, pre[c].v[e], acc[e]);
+                }
+            j = min(PRE, cnt);
         }
-#pragma unroll 8
-    for (int c = first; c < np; ++c) {
-        const float w = wsm[c];
-        o = fmaf(w, po[(long long)c * G * D], o);
-        den = fmaf(w, lsm[c], den);
+#pragma unroll 2
+        for (; j < cnt; ++j) {
+            const float wj = __shfl_sync(0xffffffffu, w, j);
+            const Vec x = po[(cb + j) * pstride];
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) acc[e] = fmaf(wj, x.v[e], acc[e]);
+        }
     }
-    out[(u * G + g) * D + d] = o / den;
+#pragma unroll
+    for (int o = 16; o >= 1; o >>= 1) den += __shfl_xor_sync(0xffffffffu, den, o);
+    Vec r;
+#pragma unroll
+    for (int e = 0; e < VEC; ++e) r.v[e] = acc[e] / den;
+    reinterpret_cast<Vec*>(out + (u * G + g) * D)[lane] = r;
+}
+
+template <int D, int PRE, int WARPS>
+static cudaError_t launch_combine_one(const DecodeArgs& a, const DecodePlan& plan, cudaStream_t stream) {
+    const long long items = (long long)a.units * a.G;
+    const dim3 grid((unsigned)((items + WARPS - 1) / WARPS)), block(WARPS * 32);
+    return launch_kernel(decode_combine_kernel<D, PRE, WARPS>, grid, block, 0, stream, a.programmatic, (const float*)a.part_o,
+                         (const float*)a.part_ml, a.out, a.G, plan.tpu, plan.T, plan.NC, a.n_extra, a.n, plan.tile_rows,
+                         a.units, a.capacity);
 }
 
 cudaError_t launch_combine(const DecodeArgs& a, const DecodePlan& plan, cudaStream_t stream) {
-    return launch_kernel(decode_combine_kernel, dim3(a.units * a.G), dim3(a.D), 0, stream, a.programmatic,
-                         (const float*)a.part_o, (const float*)a.part_ml, a.out, a.G, a.D, plan.tpu, plan.T, plan.NC, a.n_extra,
-                         a.n, plan.tile_rows, a.units, a.capacity);
+    // a unit has at most two pieces when no block's share is shorter than a unit, i.e. when there are
+    // at least as many units as blocks (whatever the length, also one that grows under graph replay)
+    const bool short_units = a.units >= plan.NC;
+    if (a.D == 128)
+        return short_units ? launch_combine_one<128, 2, 8>(a, plan, stream) : launch_combine_one<128, 4, 4>(a, plan, stream);
+    return short_units ? launch_combine_one<64, 2, 8>(a, plan, stream) : launch_combine_one<64, 4, 4>(a, plan, stream);
 }
 
 // --------------------------------------------------------------------------------------
@@ -698,6 +799,8 @@ cudaError_t launch_decode_scalar(const DecodeArgs& a, const DecodePlan& plan, cu
     ka.cap = a.capacity;
     ka.k_new = (const char*)a.k_new;
     ka.v_new = (const char*)a.v_new;
+    ka.out = a.finish_in_kernel ? a.out : nullptr;
+    ka.flags = a.flags;
     const bool pdl = a.programmatic;
     if (a.dtype == 0) {
         if (a.D == 128) return launch_scalar_groups<__nv_bfloat16, 128>(a.G, plan.geom, ka, plan.NC, pdl, stream);
@@ -717,7 +820,9 @@ constexpr int kRoofTileBytes = 16384;
 constexpr int kRoofStageBytes = 2 * kRoofTileBytes;
 constexpr int kRoofSmem = kRoofStages * kRoofStageBytes + 2 * kRoofStages * 8 + 16;
 
-__global__ void __launch_bounds__(kScalarThreads, 2)
+constexpr int kRoofThreads = kConsumerThreads + 32;   // consumer warps + the producer warp
+
+__global__ void __launch_bounds__(kRoofThreads, 2)
     read_roof_kernel(const char* __restrict__ src, long long n_tiles, unsigned long long* checksum) {
     extern __shared__ __align__(128) unsigned char smem[];
     uint64_t* full_bar = reinterpret_cast<uint64_t*>(smem + kRoofStages * kRoofStageBytes);
@@ -778,7 +883,7 @@ cudaError_t launch_read_roof(const void* src, size_t bytes, unsigned long long* 
     const int NC = (int)std::min<long long>(n_tiles, 2LL * sm_count);
     cudaError_t e = cudaMemsetAsync(checksum, 0, 8, stream);
     if (e != cudaSuccess) return e;
-    read_roof_kernel<<<NC, kScalarThreads, kRoofSmem, stream>>>((const char*)src, n_tiles, checksum);
+    read_roof_kernel<<<NC, kRoofThreads, kRoofSmem, stream>>>((const char*)src, n_tiles, checksum);
     return cudaGetLastError();
 }
 

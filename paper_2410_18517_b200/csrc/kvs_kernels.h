@@ -43,7 +43,14 @@ struct DecodeArgs {
     bool programmatic;    // launch with programmatic stream serialization (early start, explicit wait)
     const void* k_new;    // [B][1][Hkv][D] rows the launch also appends (n already counts them), or nullptr
     const void* v_new;
+    // No unit has more than two pieces (at least as many units as blocks): the split-K kernel merges
+    // the two itself and writes `out`; no combine launch.  flags: [units] ints, zero between launches.
+    bool finish_in_kernel;
+    int* flags;
 };
+
+// Whether a launch of this plan over `units` units can finish inside the split-K kernel.
+inline bool can_finish_in_kernel(const DecodePlan& plan, int units) { return units >= plan.NC; }
 
 // Largest number of thread blocks any plan may use (sizes the partial buffers).
 constexpr int kMaxCtas = 1024;
@@ -60,12 +67,13 @@ cudaError_t init_kernels();
 cudaError_t init_mma_kernels();
 
 // Encode the TMA tensor map of a bf16 pool seen as [total_rows][D]; `storage` is 128 bytes,
-// 64-byte aligned, host memory.
-cudaError_t make_pool_tensor_map(void* storage, void* pool, long long total_rows, int D);
+// 64-byte aligned, host memory.  tail = false: 64-row boxes (whole tiles); true: 16-row boxes (the
+// partly filled last tile of a unit).
+cudaError_t make_pool_tensor_map(void* storage, void* pool, long long total_rows, int D, bool tail);
 
 // krow0 / vrow0: first row of the K / V plane in the pool-wide row numbering.
-cudaError_t launch_decode_mma(const DecodeArgs& a, const DecodePlan& plan, const void* tensor_map, long long krow0,
-                              long long vrow0, cudaStream_t stream);
+cudaError_t launch_decode_mma(const DecodeArgs& a, const DecodePlan& plan, const void* tensor_map,
+                              const void* tensor_map_tail, long long krow0, long long vrow0, cudaStream_t stream);
 
 // Tensor-core prefill attention (bf16, head size D = 64 or 128): q [B][T][Hq][D], out fp32 of the same shape.
 cudaError_t init_prefill_kernels();

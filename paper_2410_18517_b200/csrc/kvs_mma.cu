@@ -33,11 +33,13 @@ namespace {
 #endif
 constexpr int kMmaWarps = KVS_MMA_WARPS;
 constexpr int kMmaConsumerThreads = kMmaWarps * 32;
-constexpr int kMmaThreads = kMmaConsumerThreads + 32;
+constexpr int kMmaThreads = kMmaConsumerThreads + 64;   // + the producer warp and the hand-over warp
 constexpr int kMmaTileBytes = KVS_MMA_TILE_BYTES;
 constexpr int kMmaQBytes = 2048;  // room for 8 heads x 128 x bf16
 constexpr int kMmaStages = KVS_MMA_STAGES;
 constexpr int kBoxRows = 64;      // the pool's tensor map moves boxes of 64 columns x 64 rows (8 KiB)
+constexpr int kTailRows = 16;     // a second map moves 16-row boxes: the last, partly filled tile of a unit
+                                  // is fetched in as many of these as hold rows (16 = the tokens of one MMA block)
 
 template <int D>
 struct MmaShape {
@@ -49,7 +51,9 @@ struct MmaShape {
     static constexpr int NB = D / 8;
     static constexpr int STAGE_BYTES = 2 * kMmaTileBytes + kMmaQBytes;
     static constexpr int SCRATCH_FLOATS = kMmaWarps * 8 * (D + 2);   // [warp][q-head of the group][D + 2]
-    static constexpr int SMEM_BYTES = 1024 + kMmaStages * STAGE_BYTES + SCRATCH_FLOATS * 4 + 2 * kMmaStages * 8 + 16;
+    static constexpr int HANDOVER_FLOATS = 8 * (D + 2);              // another block's piece of a cut unit: [q-head][D + 2]
+    static constexpr int SMEM_BYTES = 1024 + kMmaStages * STAGE_BYTES + (SCRATCH_FLOATS + HANDOVER_FLOATS) * 4 +
+                                      (2 * kMmaStages + 2) * 8 + 16;
 };
 
 __device__ __forceinline__ void tma_load_2d(void* dst_smem, const CUtensorMap* tmap, int x, int y, uint64_t* bar) {
@@ -112,13 +116,17 @@ struct MmaKernelArgs {
     const char* v_new;
     char* kplane;        // planes of the slot (for the append; the tiles are fetched through the tensor map)
     char* vplane;
+    // Finishing inside this kernel (no combine launch): set when no unit has more than two pieces.
+    float* out;          // [units][G][D] final results, or nullptr: every piece goes to part_o / part_ml
+    int* flags;          // [units], all zero between launches: 1 = the unit's second piece is in part_o / part_ml
 };
 
 // G (q-heads per kv-head, 1..8) is a run-time argument: it only selects which rows of the padded
 // 16-row M side are real, so one kernel per head size serves every group size.
 template <int D>
 __global__ void __launch_bounds__(kMmaThreads, KVS_MMA_BLOCKS_PER_SM)
-    decode_splitk_mma(const __grid_constant__ CUtensorMap tmap, const MmaKernelArgs a_in) {
+    decode_splitk_mma(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ CUtensorMap tmap_tail,
+                      const MmaKernelArgs a_in) {
     using S = MmaShape<D>;
     MmaKernelArgs a = a_in;
     bool over = false;    // a replayed launch with an append that would pass the capacity
@@ -141,7 +149,10 @@ __global__ void __launch_bounds__(kMmaThreads, KVS_MMA_BLOCKS_PER_SM)
     float* scratch = reinterpret_cast<float*>(smem + kMmaStages * S::STAGE_BYTES);
     uint64_t* full_bar = reinterpret_cast<uint64_t*>(scratch + S::SCRATCH_FLOATS);
     uint64_t* empty_bar = full_bar + kMmaStages;
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(empty_bar + kMmaStages);
+    uint64_t* tail_bar = empty_bar + kMmaStages;     // every consumer thread has written this block's second-piece partial
+    uint64_t* head_bar = tail_bar + 1;               // the next block's second-piece partial is in handover[]
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(head_bar + 1);
+    float* handover = const_cast<float*>(reinterpret_cast<volatile float*>(abort_flag + 4));
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int NC = gridDim.x;
@@ -153,6 +164,8 @@ __global__ void __launch_bounds__(kMmaThreads, KVS_MMA_BLOCKS_PER_SM)
             mbar_init(&full_bar[s], 1);
             mbar_init(&empty_bar[s], kMmaWarps);
         }
+        mbar_init(tail_bar, kMmaConsumerThreads);
+        mbar_init(head_bar, 1);
         abort_flag[0] = 0;
         abort_flag[1] = 0;
         fence_mbar_init();
@@ -171,24 +184,38 @@ __global__ void __launch_bounds__(kMmaThreads, KVS_MMA_BLOCKS_PER_SM)
                 const int ti = (int)(gt - u * a.tpu);
                 const bool with_q = (gt == t0) || (ti == 0);
                 const int n_u = a.unit_len ? min(a.unit_len[u], a.cap) : a.n;
-                const bool have = ti * TN < n_u;                  // a ragged unit may end before this tile
+                const int rows = min(TN, n_u - ti * TN);          // <= 0: a ragged unit ended before this tile
+                // a full tile comes in 64-row boxes; a partly filled one in 16-row boxes, only those that hold rows
+                const int tail_boxes = rows < TN ? (rows + kTailRows - 1) / kTailRows : 0;
+                const uint32_t kv_bytes = rows <= 0 ? 0u : (rows == TN ? 2u * kMmaTileBytes : 2u * tail_boxes * kTailRows * S::RB);
                 unsigned char* sb = smem + st * S::STAGE_BYTES;
                 if (arm) {
-                    const uint32_t total = (have ? 2 * kMmaTileBytes : 0) + (with_q ? QBYTES : 0);
+                    const uint32_t total = kv_bytes + (with_q ? QBYTES : 0);
                     if (total) mbar_arrive_expect_tx(&full_bar[st], total);
                     else mbar_arrive(&full_bar[st]);
                 }
-                if (kv && have) {
+                if (kv && rows > 0) {
                     const long long row = u * a.row_stride + (long long)ti * TN;
+                    if (rows == TN) {
 #pragma unroll
-                    for (int h = 0; h < S::HALVES; ++h)
+                        for (int h = 0; h < S::HALVES; ++h)
 #pragma unroll
-                        for (int rb = 0; rb < TN / kBoxRows; ++rb) {
-                            const int off = h * (TN * 128) + rb * (kBoxRows * 128);
-                            tma_load_2d(sb + off, &tmap, h * 64, (int)(a.krow0 + row) + rb * kBoxRows, &full_bar[st]);
-                            tma_load_2d(sb + kMmaTileBytes + off, &tmap, h * 64, (int)(a.vrow0 + row) + rb * kBoxRows,
-                                        &full_bar[st]);
-                        }
+                            for (int rb = 0; rb < TN / kBoxRows; ++rb) {
+                                const int off = h * (TN * 128) + rb * (kBoxRows * 128);
+                                tma_load_2d(sb + off, &tmap, h * 64, (int)(a.krow0 + row) + rb * kBoxRows, &full_bar[st]);
+                                tma_load_2d(sb + kMmaTileBytes + off, &tmap, h * 64, (int)(a.vrow0 + row) + rb * kBoxRows,
+                                            &full_bar[st]);
+                            }
+                    } else {
+#pragma unroll
+                        for (int h = 0; h < S::HALVES; ++h)
+                            for (int rb = 0; rb < tail_boxes; ++rb) {
+                                const int off = h * (TN * 128) + rb * (kTailRows * 128);
+                                tma_load_2d(sb + off, &tmap_tail, h * 64, (int)(a.krow0 + row) + rb * kTailRows, &full_bar[st]);
+                                tma_load_2d(sb + kMmaTileBytes + off, &tmap_tail, h * 64,
+                                            (int)(a.vrow0 + row) + rb * kTailRows, &full_bar[st]);
+                            }
+                    }
                 }
                 if (qpart && with_q)
                     bulk_g2s(sb + 2 * kMmaTileBytes, a.q + u * (long long)QBYTES, QBYTES, &full_bar[st]);
@@ -206,6 +233,9 @@ __global__ void __launch_bounds__(kMmaThreads, KVS_MMA_BLOCKS_PER_SM)
             }
             pdl_wait();
             pdl_launch_dependents();
+            // first the queries of the tiles already fetched (the consumers wait for nothing else), then the new rows
+            if (lane == 0)
+                for (int j = 0; j < npre; ++j) issue(t0 + j, j, false, false, true);
             if (a.k_new != nullptr) {
                 if (!over)
                     store_new_rows<S::RB>(lane, t0, t1, a.tpu, a.n, a.row_stride, a.k_new, a.v_new, a.kplane, a.vplane);
@@ -213,7 +243,6 @@ __global__ void __launch_bounds__(kMmaThreads, KVS_MMA_BLOCKS_PER_SM)
                     atomicExch(a.status, 4);
             }
             if (lane != 0) return;
-            for (int j = 0; j < npre; ++j) issue(t0 + j, j, false, false, true);
             int it = npre;
             bool ok = true;
             for (long long gt = t0 + npre; gt < t1; ++gt, ++it) {
@@ -226,6 +255,39 @@ __global__ void __launch_bounds__(kMmaThreads, KVS_MMA_BLOCKS_PER_SM)
             if (!ok) {
                 for (int j = max(0, it - kMmaStages); j < it; ++j)
                     mbar_wait_bounded(&full_bar[j % kMmaStages], (j / kMmaStages) & 1, abort_flag + 1, a.status);
+            }
+        }
+        return;
+    }
+
+    if (warp == kMmaWarps + 1) {
+        // ------------------ hand-over of units that are cut between two blocks ------------------
+        // Only when the kernel finishes the units itself (a.out set).  The global round trips of the
+        // hand-over are made here, beside the stream: this warp raises the flag of the unit whose
+        // second piece this block computed first, and fetches the second piece of the unit whose
+        // first piece this block computes last, so that the consumers find it in shared memory.
+        if (a.out == nullptr || t0 >= t1) return;
+        const bool has_tail = (t0 % a.tpu) != 0, has_head = (t1 % a.tpu) != 0;
+        if (!has_tail && !has_head) return;
+        pdl_wait();   // the flags are back to zero only once the previous launch has completed
+        if (has_tail) {
+            if (!mbar_wait_bounded(tail_bar, 0, abort_flag, a.status)) return;
+            if (lane == 0) st_release_gpu(a.flags + t0 / a.tpu, 1);
+        }
+        if (has_head) {
+            const long long u = (t1 - 1) / a.tpu;
+            int ok = 1;
+            if (lane == 0) ok = flag_wait_bounded(a.flags + u, 1, abort_flag, a.status) ? 1 : 0;
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+            if (!ok) return;
+            // written by another SM during this launch: read past L1
+            const long long pt = u + blockIdx.x + 1;
+            for (int i = lane; i < G * D; i += 32) handover[(i / D) * (D + 2) + (i % D)] = __ldcg(a.part_o + pt * G * D + i);
+            for (int i = lane; i < G * 2; i += 32) handover[(i >> 1) * (D + 2) + D + (i & 1)] = __ldcg(a.part_ml + pt * G * 2 + i);
+            __syncwarp();
+            if (lane == 0) {
+                a.flags[u] = 0;          // this block is the flag's only reader
+                mbar_arrive(head_bar);
             }
         }
         return;
@@ -276,20 +338,36 @@ __global__ void __launch_bounds__(kMmaThreads, KVS_MMA_BLOCKS_PER_SM)
 #pragma unroll
             for (int blk = 0; blk < BPW; ++blk) {
                 const int tok0 = (warp * BPW + blk) * 16;
+                if (tok0 >= valid) continue;   // no row of this block exists (and a partly filled tile was not fetched that far)
                 // ---- S = Q K^T for 16 tokens: two 8-token column blocks ----
+                // All K fragments are fetched first and the products of even and odd 16-column steps go to
+                // separate accumulators, so that neither the shared-memory latency nor the latency of one
+                // MMA feeding the next sits KSTEPS times on the path of a tile (one warp per scheduler: nothing
+                // else hides it).
                 float s[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
                 {
                     const int t = tok0 + ((lane >> 4) << 3) + (lane & 7);
                     const uint32_t rowaddr = ks_u32 + t * 128;
                     const int sw = t & 7;
+                    uint32_t b[KSTEPS][4];
 #pragma unroll
                     for (int st_k = 0; st_k < KSTEPS; ++st_k) {
                         const int half = st_k >> 2;
                         const int chunk = ((st_k & 3) << 1) + ((lane >> 3) & 1);
-                        uint32_t b[4];
-                        ldmatrix_x4(b, rowaddr + half * (TN * 128) + ((chunk ^ sw) << 4));
-                        mma_bf16_upper(s[0][0], s[0][1], qa[st_k][0], qa[st_k][1], b[0], b[1]);
-                        mma_bf16_upper(s[1][0], s[1][1], qa[st_k][0], qa[st_k][1], b[2], b[3]);
+                        ldmatrix_x4(b[st_k], rowaddr + half * (TN * 128) + ((chunk ^ sw) << 4));
+                    }
+                    float s2[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
+#pragma unroll
+                    for (int st_k = 0; st_k < KSTEPS; st_k += 2) {
+                        mma_bf16_upper(s[0][0], s[0][1], qa[st_k][0], qa[st_k][1], b[st_k][0], b[st_k][1]);
+                        mma_bf16_upper(s[1][0], s[1][1], qa[st_k][0], qa[st_k][1], b[st_k][2], b[st_k][3]);
+                        mma_bf16_upper(s2[0][0], s2[0][1], qa[st_k + 1][0], qa[st_k + 1][1], b[st_k + 1][0], b[st_k + 1][1]);
+                        mma_bf16_upper(s2[1][0], s2[1][1], qa[st_k + 1][0], qa[st_k + 1][1], b[st_k + 1][2], b[st_k + 1][3]);
+                    }
+#pragma unroll
+                    for (int nb = 0; nb < 2; ++nb) {
+                        s[nb][0] += s2[nb][0];
+                        s[nb][1] += s2[nb][1];
                     }
                 }
                 // ---- online softmax for row `row`, tokens tok0 + nb*8 + quad*2 + j ----
@@ -329,21 +407,32 @@ __global__ void __launch_bounds__(kMmaThreads, KVS_MMA_BLOCKS_PER_SM)
                 const uint32_t plo_lo = pack_bf16(p[0][0] - h00, p[0][1] - h01);
                 const uint32_t plo_hi = pack_bf16(p[1][0] - h10, p[1][1] - h11);
                 // ---- O += P V: 16 tokens x D, two 8-wide column blocks per ldmatrix ----
+                // Four column blocks at a time: their P_hi products are issued before their P_lo products, so
+                // that an MMA never waits for the one just before it (same accumulator).
                 {
                     const int t = tok0 + (((lane >> 3) & 1) << 3) + (lane & 7);
                     const uint32_t rowaddr = vs_u32 + t * 128;
                     const int sw = t & 7;
 #pragma unroll
-                    for (int nbp = 0; nbp < NB / 2; ++nbp) {
-                        const int chunkg = nbp * 2 + (lane >> 4);
-                        const int half = chunkg >> 3;
-                        const int chunk = chunkg & 7;
-                        uint32_t b[4];
-                        ldmatrix_x4_trans(b, rowaddr + half * (TN * 128) + ((chunk ^ sw) << 4));
-                        mma_bf16_upper(o[2 * nbp][0], o[2 * nbp][1], phi_lo, phi_hi, b[0], b[1]);
-                        mma_bf16_upper(o[2 * nbp][0], o[2 * nbp][1], plo_lo, plo_hi, b[0], b[1]);
-                        mma_bf16_upper(o[2 * nbp + 1][0], o[2 * nbp + 1][1], phi_lo, phi_hi, b[2], b[3]);
-                        mma_bf16_upper(o[2 * nbp + 1][0], o[2 * nbp + 1][1], plo_lo, plo_hi, b[2], b[3]);
+                    for (int nbp = 0; nbp < NB / 2; nbp += 2) {
+                        uint32_t b[2][4];
+#pragma unroll
+                        for (int x = 0; x < 2; ++x) {
+                            const int chunkg = (nbp + x) * 2 + (lane >> 4);
+                            const int half = chunkg >> 3;
+                            const int chunk = chunkg & 7;
+                            ldmatrix_x4_trans(b[x], rowaddr + half * (TN * 128) + ((chunk ^ sw) << 4));
+                        }
+#pragma unroll
+                        for (int x = 0; x < 2; ++x) {
+                            mma_bf16_upper(o[2 * (nbp + x)][0], o[2 * (nbp + x)][1], phi_lo, phi_hi, b[x][0], b[x][1]);
+                            mma_bf16_upper(o[2 * (nbp + x) + 1][0], o[2 * (nbp + x) + 1][1], phi_lo, phi_hi, b[x][2], b[x][3]);
+                        }
+#pragma unroll
+                        for (int x = 0; x < 2; ++x) {
+                            mma_bf16_upper(o[2 * (nbp + x)][0], o[2 * (nbp + x)][1], plo_lo, plo_hi, b[x][0], b[x][1]);
+                            mma_bf16_upper(o[2 * (nbp + x) + 1][0], o[2 * (nbp + x) + 1][1], plo_lo, plo_hi, b[x][2], b[x][3]);
+                        }
                     }
                 }
             }
@@ -353,8 +442,18 @@ __global__ void __launch_bounds__(kMmaThreads, KVS_MMA_BLOCKS_PER_SM)
 
         // ---- end of piece: merge the consumer warps, all q-heads of the group in one round ----
         // scratch[warp][q-head][D + 2]: one barrier before (the previous piece's readers are done),
-        // one after the writes
+        // one after the writes.
+        // With a.out set (no unit has more than two pieces) the kernel finishes the units itself: a unit
+        // that lies inside this block's share is normalised and written out; of a unit cut in two the
+        // second piece, which is the FIRST piece of the next block and so done early in the launch, goes
+        // to part_o / part_ml and the hand-over warp raises the unit's flag; the block that holds the
+        // first piece comes to it LAST, by when its hand-over warp has fetched the second piece into
+        // shared memory; it merges the two in piece order and writes the result.
         const long long pid = u + blockIdx.x;
+        const bool finish = a.out != nullptr;
+        const bool whole = finish && ti0 == 0 && piece_tiles == a.tpu;
+        const bool head = finish && ti0 == 0 && piece_tiles < a.tpu;
+        const bool tail = finish && ti0 > 0;
         float l = lsum;
         l += __shfl_xor_sync(0xffffffffu, l, 1);
         l += __shfl_xor_sync(0xffffffffu, l, 2);
@@ -371,6 +470,7 @@ __global__ void __launch_bounds__(kMmaThreads, KVS_MMA_BLOCKS_PER_SM)
                 dst[D + 1] = l;
             }
         }
+        if (head && !mbar_wait_bounded(head_bar, 0, abort_flag, a.status)) return;
         named_bar_sync(1, kMmaConsumerThreads);
         for (int idx = tid; idx < G * D; idx += kMmaConsumerThreads) {
             const int g = idx / D, d = idx - g * D;
@@ -386,12 +486,22 @@ __global__ void __launch_bounds__(kMmaThreads, KVS_MMA_BLOCKS_PER_SM)
                 acc = fmaf(w, src[j * WS + d], acc);
                 den = fmaf(w, src[j * WS + D + 1], den);
             }
-            a.part_o[(pid * G + g) * D + d] = acc;
-            if (d == 0) {
-                a.part_ml[(pid * G + g) * 2] = M;
-                a.part_ml[(pid * G + g) * 2 + 1] = den;
+            if (whole) {
+                a.out[(u * G + g) * D + d] = acc / den;
+            } else if (head) {
+                const float* hv = handover + g * (D + 2);      // the unit's second piece
+                const float Mx = fmaxf(M, hv[D]);
+                const float w0 = fast_exp2(M - Mx), w1 = fast_exp2(hv[D] - Mx);
+                a.out[(u * G + g) * D + d] = fmaf(w1, hv[d], w0 * acc) / fmaf(w1, hv[D + 1], w0 * den);
+            } else {
+                a.part_o[(pid * G + g) * D + d] = acc;
+                if (d == 0) {
+                    a.part_ml[(pid * G + g) * 2] = M;
+                    a.part_ml[(pid * G + g) * 2 + 1] = den;
+                }
             }
         }
+        if (tail) mbar_arrive(tail_bar);   // this thread's part of the piece is written
         gt += piece_tiles;
     }
 }
@@ -410,8 +520,10 @@ cudaError_t set_attr() {
 }
 
 template <int D>
-cudaError_t launch_one(const CUtensorMap& tm, const MmaKernelArgs& ka, int NC, bool pdl, cudaStream_t stream) {
-    return launch_kernel(decode_splitk_mma<D>, dim3(NC), dim3(kMmaThreads), MmaShape<D>::SMEM_BYTES, stream, pdl, tm, ka);
+cudaError_t launch_one(const CUtensorMap& tm, const CUtensorMap& tm_tail, const MmaKernelArgs& ka, int NC, bool pdl,
+                       cudaStream_t stream) {
+    return launch_kernel(decode_splitk_mma<D>, dim3(NC), dim3(kMmaThreads), MmaShape<D>::SMEM_BYTES, stream, pdl, tm, tm_tail,
+                         ka);
 }
 
 }  // namespace
@@ -421,9 +533,10 @@ cudaError_t init_mma_kernels() {
     return e != cudaSuccess ? e : set_attr<64>();
 }
 
-// Tensor map over the whole pool seen as [total_rows][D] bf16, box = 64 columns x 64 rows,
-// 128-byte swizzle.  `storage` must be 64-byte aligned and hold sizeof(CUtensorMap) = 128 bytes.
-cudaError_t make_pool_tensor_map(void* storage, void* pool, long long total_rows, int D) {
+// Tensor map over the whole pool seen as [total_rows][D] bf16, box = 64 columns x 64 rows (or, with
+// `tail`, x 16 rows), 128-byte swizzle.  `storage` must be 64-byte aligned and hold
+// sizeof(CUtensorMap) = 128 bytes.
+cudaError_t make_pool_tensor_map(void* storage, void* pool, long long total_rows, int D, bool tail) {
     typedef CUresult (*EncodeFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -434,7 +547,7 @@ cudaError_t make_pool_tensor_map(void* storage, void* pool, long long total_rows
     if (qres != cudaDriverEntryPointSuccess || fn == nullptr) return cudaErrorNotSupported;
     cuuint64_t dims[2] = {(cuuint64_t)D, (cuuint64_t)total_rows};
     cuuint64_t strides[1] = {(cuuint64_t)D * 2};
-    cuuint32_t box[2] = {64u, (cuuint32_t)kBoxRows};
+    cuuint32_t box[2] = {64u, (cuuint32_t)(tail ? kTailRows : kBoxRows)};
     cuuint32_t estr[2] = {1u, 1u};
     CUresult r = reinterpret_cast<EncodeFn>(fn)(reinterpret_cast<CUtensorMap*>(storage), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16,
                                                 2, pool, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
@@ -455,8 +568,8 @@ void plan_decode_mma(int units, int n, int D, int sm_count, int max_ctas, Decode
     plan->geom = 0;
 }
 
-cudaError_t launch_decode_mma(const DecodeArgs& a, const DecodePlan& plan, const void* tensor_map, long long krow0,
-                              long long vrow0, cudaStream_t stream) {
+cudaError_t launch_decode_mma(const DecodeArgs& a, const DecodePlan& plan, const void* tensor_map,
+                              const void* tensor_map_tail, long long krow0, long long vrow0, cudaStream_t stream) {
     MmaKernelArgs ka;
     ka.q = (const char*)a.q;
     ka.part_o = a.part_o;
@@ -472,6 +585,7 @@ cudaError_t launch_decode_mma(const DecodeArgs& a, const DecodePlan& plan, const
     ka.safe_rows = (a.programmatic && !a.unit_len) ? a.safe_rows : 0;
     ka.unit_len = a.unit_len;
     const CUtensorMap& tm = *reinterpret_cast<const CUtensorMap*>(tensor_map);
+    const CUtensorMap& tm_tail = *reinterpret_cast<const CUtensorMap*>(tensor_map_tail);
     ka.G = a.G;
     ka.n_extra = a.n_extra;
     ka.units = a.units;
@@ -480,9 +594,11 @@ cudaError_t launch_decode_mma(const DecodeArgs& a, const DecodePlan& plan, const
     ka.v_new = (const char*)a.v_new;
     ka.kplane = (char*)const_cast<void*>(a.kplane);
     ka.vplane = (char*)const_cast<void*>(a.vplane);
+    ka.out = a.finish_in_kernel ? a.out : nullptr;
+    ka.flags = a.flags;
     if (a.G < 1 || a.G > 8) return cudaErrorInvalidValue;
-    if (a.D == 128) return launch_one<128>(tm, ka, plan.NC, a.programmatic, stream);
-    if (a.D == 64) return launch_one<64>(tm, ka, plan.NC, a.programmatic, stream);
+    if (a.D == 128) return launch_one<128>(tm, tm_tail, ka, plan.NC, a.programmatic, stream);
+    if (a.D == 64) return launch_one<64>(tm, tm_tail, ka, plan.NC, a.programmatic, stream);
     return cudaErrorInvalidValue;
 }
 
