@@ -63,7 +63,10 @@ typedef enum {
     KVS_ERR_OOM = 5,           /* a bound buffer is smaller than kvs_required_bytes said      */
     KVS_ERR_CUDA = 6,          /* a CUDA runtime or driver call failed                        */
     KVS_ERR_TIMEOUT = 7,       /* a bounded device-side wait ran out (see kvs_last_device_status) */
-    KVS_ERR_SCRATCH_LIMIT = 8  /* kvs_decode_attention_static: the call needs more than the built-in scratch */
+    KVS_ERR_SCRATCH_LIMIT = 8, /* kvs_decode_attention_static: the call needs more than the built-in scratch */
+    KVS_ERR_BOUNDS = 9         /* device status word only, bounds-checking build (-DKVS_DEBUG_BOUNDS) only: a
+                                  kernel computed an offset outside the buffer it belongs to; the access was
+                                  redirected or dropped and the launch ran on                               */
 } kvs_status;
 
 typedef enum { KVS_BF16 = 0, KVS_F32 = 1 } kvs_dtype;
@@ -378,6 +381,12 @@ kvs_status kvs_clear_device_status(kvs_ctx* ctx, void* stream);
  * the GPU.  Afterwards kvs_last_device_status reports KVS_ERR_TIMEOUT until kvs_clear_device_status.
  * Errors: STATE before kvs_bind_memory; INVALID_ARG for a limit out of range.                      */
 kvs_status kvs_selftest_wait_timeout(kvs_ctx* ctx, uint32_t limit_us, uint64_t* waited_ns, void* stream);
+/* Self-test of the bounds-checking build (the library compiled with -DKVS_DEBUG_BOUNDS, in which every
+ * global offset the kernels compute is checked against the buffer it must fall in; the paper has no
+ * counterpart).  Launches one kernel that hands the check an offset outside its buffer WITHOUT touching
+ * memory; afterwards kvs_last_device_status reports KVS_ERR_BOUNDS, which shows that a real violation
+ * would be recorded.  In a normal build the checks are compiled out: STATE, nothing is launched.   */
+kvs_status kvs_selftest_bounds(kvs_ctx* ctx, void* stream);
 kvs_status kvs_set_option(kvs_ctx* ctx, int32_t option, int32_t value);
 /* How the last kvs_decode_attention call was decomposed: thread blocks launched,
  * rows per tile, and 1 or 2 for the scalar / tensor-core kernel.                */

@@ -36,13 +36,17 @@ class SharedKVCache:
             if share_map is not None:
                 binding.kvs_set_share_map(self.ctx, share_map)
             self.pool_bytes, self.workspace_bytes = binding.kvs_required_bytes(self.ctx)
-            self.pool = torch.empty(self.pool_bytes, dtype=torch.uint8, device=self.device)
-            self.workspace = torch.empty(self.workspace_bytes, dtype=torch.uint8, device=self.device)
+            self.pool = self._allocate(self.pool_bytes)
+            self.workspace = self._allocate(self.workspace_bytes)
             binding.kvs_bind_memory(self.ctx, self.pool, self.pool_bytes, self.workspace, self.workspace_bytes)
         except Exception:
             binding.kvs_destroy(self.ctx)
             self.ctx = None
             raise
+
+    def _allocate(self, nbytes):
+        """Device memory for the pool or the workspace (256-byte aligned uint8 tensor of ``nbytes``)."""
+        return self._torch.empty(nbytes, dtype=self._torch.uint8, device=self.device)
 
     def close(self):
         if getattr(self, "ctx", None):

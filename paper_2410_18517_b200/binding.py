@@ -11,7 +11,8 @@ import ctypes
 import os
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libkvs.so")
+# KVS_LIBRARY names another build of the same library (the bounds-checking one, for instance)
+LIB_PATH = os.environ.get("KVS_LIBRARY") or os.path.join(_HERE, "libkvs.so")
 
 KVS_OK = 0
 KVS_ERR_INVALID_ARG = 1
@@ -22,6 +23,7 @@ KVS_ERR_OOM = 5
 KVS_ERR_CUDA = 6
 KVS_ERR_TIMEOUT = 7
 KVS_ERR_SCRATCH_LIMIT = 8
+KVS_ERR_BOUNDS = 9
 
 KVS_BF16 = 0
 KVS_F32 = 1
@@ -43,6 +45,7 @@ EXPORTS = (
     "kvs_evict", "kvs_unit_len", "kvs_layer_distances", "kvs_mean_cosine",
     "kvs_replay_advance", "kvs_replay_commit", "kvs_decode_step",
     "kvs_clear_device_status", "kvs_selftest_wait_timeout", "kvs_truncate",
+    "kvs_selftest_bounds",
 )
 
 
@@ -108,6 +111,7 @@ def load() -> ctypes.CDLL:
         "kvs_last_device_status": [vp, P(i32)],
         "kvs_clear_device_status": [vp, vp],
         "kvs_selftest_wait_timeout": [vp, ctypes.c_uint32, P(ctypes.c_uint64), vp],
+        "kvs_selftest_bounds": [vp, vp],
         "kvs_set_option": [vp, i32, i32],
         "kvs_last_launch": [vp, P(i32), P(i32), P(i32)],
         "kvs_read_roof": [vp, sz, vp, i32, vp],
@@ -291,6 +295,10 @@ def kvs_selftest_wait_timeout(ctx: int, limit_us: int, stream: int = 0) -> int:
     w = ctypes.c_uint64()
     _check(load().kvs_selftest_wait_timeout(ctx, limit_us, ctypes.byref(w), stream), "kvs_selftest_wait_timeout")
     return w.value
+
+
+def kvs_selftest_bounds(ctx: int, stream: int = 0) -> None:
+    _check(load().kvs_selftest_bounds(ctx, stream), "kvs_selftest_bounds")
 
 
 def kvs_set_option(ctx: int, option: int, value: int) -> None:

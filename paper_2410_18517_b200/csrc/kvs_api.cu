@@ -265,7 +265,8 @@ kvs_status do_append(kvs_ctx* c, int layer, const void* k, const void* v, int ba
     const bool rag = c->ragged[slot] != 0;
     if (kvs::launch_append(k, v, kp, vp, batch, n_new, c->cfg.n_kv_heads, c->row_bytes, c->row_stride,
                            c->slot_len[slot], rag ? unit_len_dev(c, slot) : nullptr, replay_counter(c), c->cfg.max_seq,
-                           reinterpret_cast<int*>(c->ws + c->off_status), take_early_start(c), st) != cudaSuccess)
+                           reinterpret_cast<int*>(c->ws + c->off_status), (long long)c->plane_bytes, take_early_start(c),
+                           st) != cudaSuccess)
         return KVS_ERR_CUDA;
     if (rag) {
         const int units = batch * c->cfg.n_kv_heads;
@@ -335,6 +336,7 @@ kvs_status run_attention(kvs_ctx* c, int slot, const void* q, float* out, int ba
     a.k_new = k_new;
     a.v_new = v_new;
     if (k_new) a.safe_rows = std::min(a.safe_rows, a.n - 1);   // the new row is fetched after the kernel has stored it
+    a.plane_bytes = (long long)c->plane_bytes;
     a.finish_in_kernel = c->opt_finish != 0 && kvs::can_finish_in_kernel(plan, a.units);
     a.flags = scratch.flags;
     if (scratch.tracked) {
@@ -616,7 +618,7 @@ kvs_status kvs_prefill_attention(kvs_ctx* ctx, int32_t layer, const void* q, flo
     if (kvs::launch_prefill(q, out, reinterpret_cast<int*>(ctx->ws + ctx->off_status),
                             reinterpret_cast<int*>(ctx->ws + ctx->off_status + 64), ctx->tensor_map, batch, n_q,
                             ctx->cfg.n_q_heads, ctx->G, ctx->cfg.head_dim, n, ctx->row_stride, plane_rows * (2 * slot),
-                            plane_rows * (2 * slot + 1), ctx->scale * 1.4426950408889634f, ctx->sm_count, ctx->l2_bytes,
+                            plane_rows * (2 * slot + 1), plane_rows, ctx->scale * 1.4426950408889634f, ctx->sm_count, ctx->l2_bytes,
                             static_cast<cudaStream_t>(stream)) != cudaSuccess)
         return KVS_ERR_CUDA;
     // a plain launch: it starts only after everything before it on the stream has finished
@@ -948,6 +950,20 @@ kvs_status kvs_selftest_wait_timeout(kvs_ctx* ctx, uint32_t limit_us, uint64_t* 
     return KVS_OK;
 }
 
+kvs_status kvs_selftest_bounds(kvs_ctx* ctx, void* stream) {
+    if (!ctx) return KVS_ERR_INVALID_ARG;
+    if (!ctx->bound || !kvs::is_bounds_checking_build()) return KVS_ERR_STATE;
+    DeviceGuard guard(ctx->cfg.device);
+    if (!guard.ok) return KVS_ERR_CUDA;
+    if (kvs::launch_bounds_selftest(reinterpret_cast<int*>(ctx->ws + ctx->off_status), static_cast<cudaStream_t>(stream)) !=
+        cudaSuccess)
+        return KVS_ERR_CUDA;
+    ctx->seq += 1;
+    ctx->last_splitk_seq = ctx->seq;   // a plain launch: everything before it has finished when it runs
+    ctx->counter_written = false;
+    return KVS_OK;
+}
+
 kvs_status kvs_set_option(kvs_ctx* ctx, int32_t option, int32_t value) {
     if (!ctx) return KVS_ERR_INVALID_ARG;
     switch (option) {
@@ -1002,6 +1018,7 @@ const char* kvs_status_string(kvs_status s) {
         case KVS_ERR_CUDA: return "CUDA call failed";
         case KVS_ERR_TIMEOUT: return "device-side wait timed out";
         case KVS_ERR_SCRATCH_LIMIT: return "call needs more scratch than the built-in scratch array holds";
+        case KVS_ERR_BOUNDS: return "a bounds-checking build found an offset outside its buffer";
     }
     return "unknown status";
 }

@@ -10,6 +10,23 @@ namespace kvs {
 // Device status word values (mirrors kvs_status in the public header).
 constexpr int kDevOk = 0;
 constexpr int kDevTimeout = 7;
+constexpr int kDevBounds = 9;
+
+// Bounds-checking build (-DKVS_DEBUG_BOUNDS): every global offset the kernels compute for a pool
+// plane, the query / new-row buffers or the partial results is checked against the buffer it
+// must fall in.  The first violation is recorded in the status word (kDevBounds; nothing traps)
+// and the access is redirected to offset 0 of the same buffer (reads) or dropped (writes), so
+// that the launch still runs to its end.  In a normal build the checks compile to nothing.
+#ifdef KVS_DEBUG_BOUNDS
+__device__ __forceinline__ bool bounds_ok(long long off, long long len, long long limit, int* status) {
+    if (off >= 0 && len >= 0 && off + len <= limit) return true;
+    atomicCAS(status, kDevOk, kDevBounds);
+    return false;
+}
+#define KVS_BOUNDS_OK(off, len, limit, status) ::kvs::bounds_ok((long long)(off), (long long)(len), (long long)(limit), (status))
+#else
+#define KVS_BOUNDS_OK(off, len, limit, status) true
+#endif
 
 // A wait gives up after this many nanoseconds of wall time on the GPU.
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
@@ -204,7 +221,8 @@ namespace kvs {
 // lane 0 issues next.
 template <int RB>
 __device__ __forceinline__ void store_new_rows(int lane, long long t0, long long t1, int tpu, int n, int row_stride,
-                                               const char* k_new, const char* v_new, char* kplane, char* vplane) {
+                                               const char* k_new, const char* v_new, char* kplane, char* vplane,
+                                               long long plane_bytes, int units, int* status) {
     constexpr int LPR = RB / 16;
     if (t1 > t0) {
         const long long u0 = t0 / tpu, u1 = (t1 - 1) / tpu;
@@ -212,6 +230,7 @@ __device__ __forceinline__ void store_new_rows(int lane, long long t0, long long
             const long long last = u * tpu + tpu - 1;
             if (last < t0 || last >= t1) continue;
             const long long dst = (u * row_stride + (n - 1)) * (long long)RB;
+            if (!KVS_BOUNDS_OK(dst, RB, plane_bytes, status) || !KVS_BOUNDS_OK(u, 1, units, status)) continue;
             for (int i = lane; i < 2 * LPR; i += 32) {
                 const bool isv = i >= LPR;
                 const int c = isv ? i - LPR : i;

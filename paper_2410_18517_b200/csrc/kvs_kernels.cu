@@ -18,7 +18,8 @@ __global__ void __launch_bounds__(256) kv_append_kernel(const uint4* __restrict_
                                                         uint4* __restrict__ kplane, uint4* __restrict__ vplane,
                                                         long long total_vecs, int n_new, int Hkv, int row_vecs,
                                                         int row_stride, int len0, const int* __restrict__ unit_len,
-                                                        const int* __restrict__ n_extra, int capacity, int* status) {
+                                                        const int* __restrict__ n_extra, int capacity, int* status,
+                                                        long long plane_vecs) {
     pdl_launch_dependents();
     pdl_wait();
     if (n_extra) len0 += *n_extra;   // replayed launch: the slot has grown since the launch was recorded
@@ -42,20 +43,21 @@ __global__ void __launch_bounds__(256) kv_append_kernel(const uint4* __restrict_
             continue;
         }
         const long long drow = (b * Hkv + h) * (long long)row_stride + first + t;
+        if (!KVS_BOUNDS_OK(drow * row_vecs + c, 1, plane_vecs, status)) continue;
         dst[drow * row_vecs + c] = src[idx];
     }
 }
 
 cudaError_t launch_append(const void* k, const void* v, void* kplane, void* vplane, int B, int n_new, int Hkv,
                           int row_bytes, int row_stride, int len0, const int* unit_len, const int* n_extra, int capacity, int* status,
-                          bool programmatic, cudaStream_t stream) {
+                          long long plane_bytes, bool programmatic, cudaStream_t stream) {
     const int row_vecs = row_bytes / 16;
     const long long total = (long long)B * n_new * Hkv * row_vecs;
     const long long blocks = std::min<long long>((total + 255) / 256, 148 * 16);
     dim3 grid((unsigned)blocks, 2);
     return launch_kernel(kv_append_kernel, grid, dim3(256), 0, stream, programmatic, (const uint4*)k, (const uint4*)v,
                          (uint4*)kplane, (uint4*)vplane, total, n_new, Hkv, row_vecs, row_stride, len0, unit_len, n_extra, capacity,
-                         status);
+                         status, plane_bytes / 16);
 }
 
 // --------------------------------------------------------------------------------------
@@ -89,10 +91,13 @@ __global__ void __launch_bounds__(256) kv_evict_kernel(uint4* __restrict__ kplan
                 if (v == 0) atomicExch(status, 1);
                 src = c0 + j;
             }
+            if (!KVS_BOUNDS_OK(src, 1, row_stride, status)) src = 0;
             buf[idx] = base[(long long)src * row_vecs + v];
         }
         __syncthreads();
-        for (int idx = threadIdx.x; idx < rows * row_vecs; idx += blockDim.x) base[(long long)c0 * row_vecs + idx] = buf[idx];
+        for (int idx = threadIdx.x; idx < rows * row_vecs; idx += blockDim.x)
+            if (KVS_BOUNDS_OK((long long)c0 * row_vecs + idx, 1, (long long)row_stride * row_vecs, status))
+                base[(long long)c0 * row_vecs + idx] = buf[idx];
         __syncthreads();
     }
 }
@@ -268,6 +273,7 @@ struct ScalarKernelArgs {
     // Finishing inside this kernel (no combine launch): set when no unit has more than two pieces.
     float* out;           // [units][G][D] final results, or nullptr: every piece goes to part_o / part_ml
     int* flags;           // [units], all zero between launches: 1 = the unit's second piece is in part_o / part_ml
+    long long plane_bytes;  // size of one plane (what a bounds-checking build checks tile offsets against)
 };
 
 template <typename T, int D, int G, int GEOM>
@@ -345,12 +351,14 @@ __global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G, GEOM>::MI
                     else mbar_arrive(&full_bar[st]);
                 }
                 if (kv && bytes) {
-                    const long long off = (u * a.row_stride + row0) * (long long)RB;
+                    long long off = (u * a.row_stride + row0) * (long long)RB;
+                    if (!KVS_BOUNDS_OK(off, bytes, a.plane_bytes, a.status) || !KVS_BOUNDS_OK(u, 1, a.units, a.status)) off = 0;
                     bulk_g2s(sb, a.kplane + off, bytes, &full_bar[st]);
                     bulk_g2s(sb + kTile, a.vplane + off, bytes, &full_bar[st]);
                 }
                 if (qpart && with_q)
-                    bulk_g2s(sb + 2 * kTile, a.q + u * (long long)S::QBYTES, S::QBYTES, &full_bar[st]);
+                    bulk_g2s(sb + 2 * kTile, a.q + (KVS_BOUNDS_OK(u, 1, a.units, a.status) ? u : 0) * (long long)S::QBYTES,
+                             S::QBYTES, &full_bar[st]);
             };
             // Before the preceding kernel in the stream is known to have finished, only K/V
             // tiles made entirely of rows that no kernel still in flight can be writing are
@@ -372,7 +380,7 @@ __global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G, GEOM>::MI
             if (a.k_new != nullptr) {
                 if (!over)
                     store_new_rows<RB>(lane, t0, t1, a.tpu, a.n, a.row_stride, a.k_new, a.v_new, const_cast<char*>(a.kplane),
-                                       const_cast<char*>(a.vplane));
+                                       const_cast<char*>(a.vplane), a.plane_bytes, a.units, a.status);
                 else if (lane == 0 && blockIdx.x == 0)
                     atomicExch(a.status, 4);
             }
@@ -601,7 +609,7 @@ __global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G, GEOM>::MI
                     const float Mx = fmaxf(M, hv[D]);
                     const float w0 = fast_exp2(M - Mx), w1 = fast_exp2(hv[D] - Mx);
                     a.out[(u * G + g) * D + d] = fmaf(w1, hv[d], w0 * o) / fmaf(w1, hv[D + 1], w0 * den);
-                } else {
+                } else if (KVS_BOUNDS_OK(pid, 1, a.units + (long long)gridDim.x, a.status)) {
                     a.part_o[(pid * G + g) * D + d] = o;
                     if (d == 0) {
                         a.part_ml[(pid * G + g) * 2] = M;
@@ -635,7 +643,7 @@ template <int D, int PRE, int kCombineWarps>
 __global__ void __launch_bounds__(kCombineWarps * 32, PRE == 2 ? 5 : 8)
     decode_combine_kernel(const float* __restrict__ part_o, const float* __restrict__ part_ml, float* __restrict__ out,
                           int G, int tpu, long long T, int NC, const int* __restrict__ n_extra, int n, int tile_rows,
-                          int units, int cap) {
+                          int units, int cap, int* status) {
     constexpr int VEC = D / 32;
     struct __align__(VEC * 4) Vec {
         float v[VEC];
@@ -652,7 +660,10 @@ __global__ void __launch_bounds__(kCombineWarps * 32, PRE == 2 ? 5 : 8)
     const long long u = item / G;
     const int g = (int)(item - u * G);
     const int c0 = cta_of_tile(u * tpu, T, NC);
-    const int np = cta_of_tile((u + 1) * tpu - 1, T, NC) - c0 + 1;       // pieces of this unit
+    int np = cta_of_tile((u + 1) * tpu - 1, T, NC) - c0 + 1;             // pieces of this unit
+#ifdef KVS_DEBUG_BOUNDS
+    if (!KVS_BOUNDS_OK(u + c0, np, (long long)units + NC, status)) np = 1;
+#endif
     const float2* ml = reinterpret_cast<const float2*>(part_ml) + (u + c0) * G + g;   // piece c: ml[c * G]
     const Vec* po = reinterpret_cast<const Vec*>(part_o + ((u + c0) * G + g) * D) + lane;   // piece c: po[c * G * 32]
     const int pstride = G * 32;     // offsets within one unit's pieces fit 32 bits
@@ -709,7 +720,7 @@ static cudaError_t launch_combine_one(const DecodeArgs& a, const DecodePlan& pla
     const dim3 grid((unsigned)((items + WARPS - 1) / WARPS)), block(WARPS * 32);
     return launch_kernel(decode_combine_kernel<D, PRE, WARPS>, grid, block, 0, stream, a.programmatic, (const float*)a.part_o,
                          (const float*)a.part_ml, a.out, a.G, plan.tpu, plan.T, plan.NC, a.n_extra, a.n, plan.tile_rows,
-                         a.units, a.capacity);
+                         a.units, a.capacity, a.status);
 }
 
 cudaError_t launch_combine(const DecodeArgs& a, const DecodePlan& plan, cudaStream_t stream) {
@@ -801,6 +812,7 @@ cudaError_t launch_decode_scalar(const DecodeArgs& a, const DecodePlan& plan, cu
     ka.v_new = (const char*)a.v_new;
     ka.out = a.finish_in_kernel ? a.out : nullptr;
     ka.flags = a.flags;
+    ka.plane_bytes = a.plane_bytes;
     const bool pdl = a.programmatic;
     if (a.dtype == 0) {
         if (a.D == 128) return launch_scalar_groups<__nv_bfloat16, 128>(a.G, plan.geom, ka, plan.NC, pdl, stream);
@@ -915,6 +927,27 @@ __global__ void wait_timeout_selftest_kernel(int* status, unsigned long long lim
 cudaError_t launch_wait_timeout_selftest(int* status, unsigned long long limit_ns, unsigned long long* waited_ns,
                                          cudaStream_t stream) {
     wait_timeout_selftest_kernel<<<1, 32, 0, stream>>>(status, limit_ns, waited_ns);
+    return cudaGetLastError();
+}
+
+// Self-test of the bounds-checking build: hands the check an offset that lies outside its buffer
+// (no memory is touched) and lets it record the violation.  `is_checking_build` tells the host which
+// build this is.
+__global__ void bounds_selftest_kernel(int* status) {
+    // 5 + 8 > 10; in a normal build the check is compiled out and nothing is recorded
+    if (threadIdx.x == 0 && KVS_BOUNDS_OK(5, 8, 10, status)) return;
+}
+
+bool is_bounds_checking_build() {
+#ifdef KVS_DEBUG_BOUNDS
+    return true;
+#else
+    return false;
+#endif
+}
+
+cudaError_t launch_bounds_selftest(int* status, cudaStream_t stream) {
+    bounds_selftest_kernel<<<1, 32, 0, stream>>>(status);
     return cudaGetLastError();
 }
 

@@ -47,6 +47,7 @@ struct DecodeArgs {
     // the two itself and writes `out`; no combine launch.  flags: [units] ints, zero between launches.
     bool finish_in_kernel;
     int* flags;
+    long long plane_bytes;   // size of one plane: what a bounds-checking build checks tile offsets against
 };
 
 // Whether a launch of this plan over `units` units can finish inside the split-K kernel.
@@ -80,7 +81,7 @@ cudaError_t init_prefill_kernels();
 // `sched`: a device int for the kernel's work counter (zeroed on `stream` by the launch).
 cudaError_t launch_prefill(const void* q, float* out, int* status, int* sched, const void* pool_tensor_map, int B, int T,
                            int Hq, int G, int D, int n, int row_stride, long long krow0, long long vrow0,
-                           float scale_log2, int sm_count, long long l2_bytes, cudaStream_t stream);
+                           long long plane_rows, float scale_log2, int sm_count, long long l2_bytes, cudaStream_t stream);
 
 // Strategy-search reductions (see kvs_search.cu).
 constexpr int kMaxLayersSearch = 80;     // shared-memory bound of the distance kernel
@@ -94,7 +95,7 @@ cudaError_t launch_mean_cosine(const void* a, const void* b, int S, long long di
 
 cudaError_t launch_append(const void* k, const void* v, void* kplane, void* vplane, int B, int n_new, int Hkv,
                           int row_bytes, int row_stride, int len0, const int* unit_len, const int* n_extra, int capacity, int* status,
-                          bool programmatic, cudaStream_t stream);
+                          long long plane_bytes, bool programmatic, cudaStream_t stream);
 cudaError_t launch_replay_advance(int* n_extra, bool programmatic, cudaStream_t stream);
 
 // Ragged slots (rows evicted by an outside intra-layer method).
@@ -112,6 +113,10 @@ cudaError_t launch_combine(const DecodeArgs& a, const DecodePlan& plan, cudaStre
 // time-out code and *waited_ns (device, may be null) how long the wait lasted.
 cudaError_t launch_wait_timeout_selftest(int* status, unsigned long long limit_ns, unsigned long long* waited_ns,
                                          cudaStream_t stream);
+// Whether this library was compiled with -DKVS_DEBUG_BOUNDS, and a launch that makes its offset check
+// record one violation (KVS_ERR_BOUNDS in *status) without touching memory.
+bool is_bounds_checking_build();
+cudaError_t launch_bounds_selftest(int* status, cudaStream_t stream);
 cudaError_t launch_read_roof(const void* src, size_t bytes, unsigned long long* checksum, int sm_count,
                              cudaStream_t stream);
 

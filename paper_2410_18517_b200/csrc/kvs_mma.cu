@@ -119,6 +119,7 @@ struct MmaKernelArgs {
     // Finishing inside this kernel (no combine launch): set when no unit has more than two pieces.
     float* out;          // [units][G][D] final results, or nullptr: every piece goes to part_o / part_ml
     int* flags;          // [units], all zero between launches: 1 = the unit's second piece is in part_o / part_ml
+    long long plane_rows;   // rows of one plane (what a bounds-checking build checks tile rows against)
 };
 
 // G (q-heads per kv-head, 1..8) is a run-time argument: it only selects which rows of the padded
@@ -195,7 +196,11 @@ __global__ void __launch_bounds__(kMmaThreads, KVS_MMA_BLOCKS_PER_SM)
                     else mbar_arrive(&full_bar[st]);
                 }
                 if (kv && rows > 0) {
-                    const long long row = u * a.row_stride + (long long)ti * TN;
+                    long long row = u * a.row_stride + (long long)ti * TN;
+                    // (a whole box is fetched even where the unit has fewer rows: it stays inside the unit's row_stride)
+                    if (!KVS_BOUNDS_OK(row, rows == TN ? TN : tail_boxes * kTailRows, a.plane_rows, a.status) ||
+                        !KVS_BOUNDS_OK(u, 1, a.units, a.status))
+                        row = 0;
                     if (rows == TN) {
 #pragma unroll
                         for (int h = 0; h < S::HALVES; ++h)
@@ -218,7 +223,8 @@ __global__ void __launch_bounds__(kMmaThreads, KVS_MMA_BLOCKS_PER_SM)
                     }
                 }
                 if (qpart && with_q)
-                    bulk_g2s(sb + 2 * kMmaTileBytes, a.q + u * (long long)QBYTES, QBYTES, &full_bar[st]);
+                    bulk_g2s(sb + 2 * kMmaTileBytes, a.q + (KVS_BOUNDS_OK(u, 1, a.units, a.status) ? u : 0) * (long long)QBYTES,
+                             QBYTES, &full_bar[st]);
             };
             // Until the preceding kernel in the stream is known to have finished, fetch only
             // K/V tiles made entirely of rows that no kernel still in flight can be writing.
@@ -238,7 +244,8 @@ __global__ void __launch_bounds__(kMmaThreads, KVS_MMA_BLOCKS_PER_SM)
                 for (int j = 0; j < npre; ++j) issue(t0 + j, j, false, false, true);
             if (a.k_new != nullptr) {
                 if (!over)
-                    store_new_rows<S::RB>(lane, t0, t1, a.tpu, a.n, a.row_stride, a.k_new, a.v_new, a.kplane, a.vplane);
+                    store_new_rows<S::RB>(lane, t0, t1, a.tpu, a.n, a.row_stride, a.k_new, a.v_new, a.kplane, a.vplane,
+                                          a.plane_rows * S::RB, a.units, a.status);
                 else if (lane == 0 && blockIdx.x == 0)
                     atomicExch(a.status, 4);
             }
@@ -493,7 +500,7 @@ __global__ void __launch_bounds__(kMmaThreads, KVS_MMA_BLOCKS_PER_SM)
                 const float Mx = fmaxf(M, hv[D]);
                 const float w0 = fast_exp2(M - Mx), w1 = fast_exp2(hv[D] - Mx);
                 a.out[(u * G + g) * D + d] = fmaf(w1, hv[d], w0 * acc) / fmaf(w1, hv[D + 1], w0 * den);
-            } else {
+            } else if (KVS_BOUNDS_OK(pid, 1, a.units + (long long)gridDim.x, a.status)) {
                 a.part_o[(pid * G + g) * D + d] = acc;
                 if (d == 0) {
                     a.part_ml[(pid * G + g) * 2] = M;
@@ -596,6 +603,7 @@ cudaError_t launch_decode_mma(const DecodeArgs& a, const DecodePlan& plan, const
     ka.vplane = (char*)const_cast<void*>(a.vplane);
     ka.out = a.finish_in_kernel ? a.out : nullptr;
     ka.flags = a.flags;
+    ka.plane_rows = a.plane_bytes / (a.D * 2);
     if (a.G < 1 || a.G > 8) return cudaErrorInvalidValue;
     if (a.D == 128) return launch_one<128>(tm, tm_tail, ka, plan.NC, a.programmatic, stream);
     if (a.D == 64) return launch_one<64>(tm, tm_tail, ka, plan.NC, a.programmatic, stream);

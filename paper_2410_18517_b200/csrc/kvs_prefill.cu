@@ -172,6 +172,7 @@ struct PrefillArgs {
     int group_heads; // q-heads per scheduling group (a multiple of G)
     int row_stride;
     long long krow0, vrow0;  // first row of the slot's K / V plane in the pool-wide row numbering
+    long long plane_rows;    // rows of one plane (what a bounds-checking build checks tile rows against)
     float scale_log2;
 };
 
@@ -343,7 +344,8 @@ __global__ void __launch_bounds__(kPfThreads, 2)
                     if (!ok) break;
                     const int tt = t + j, st = tt & 1;
                     const uint32_t prev = (uint32_t)((tt >> 1) - 1) & 1u;   // phase in which tile tt-2 released the stage
-                    const long long row = unit_row + (long long)j * kPfKeys;
+                    long long row = unit_row + (long long)j * kPfKeys;
+                    if (!KVS_BOUNDS_OK(row, kPfKeys, a.plane_rows, a.status)) row = 0;
                     if (tt >= 2 && !mbar_wait_bounded(&k_empty[st], prev, abort_flag, a.status)) { ok = false; break; }
                     mbar_arrive_expect_tx(&k_full[st], kKvBytes);
 #pragma unroll
@@ -606,7 +608,7 @@ cudaError_t init_prefill_kernels() {
 // sequence) items from a counter, heaviest first.  `sched` is a device int the launch zeroes on `stream`.
 cudaError_t launch_prefill(const void* q, float* out, int* status, int* sched, const void* pool_tensor_map, int B, int T,
                            int Hq, int G, int D, int n, int row_stride, long long krow0, long long vrow0,
-                           float scale_log2, int sm_count, long long l2_bytes, cudaStream_t stream) {
+                           long long plane_rows, float scale_log2, int sm_count, long long l2_bytes, cudaStream_t stream) {
     if (D != 64 && D != 128) return cudaErrorInvalidValue;
     EncodeFn encode = nullptr;
     cudaError_t e = get_encode(&encode);
@@ -642,6 +644,7 @@ cudaError_t launch_prefill(const void* q, float* out, int* status, int* sched, c
     a.row_stride = row_stride;
     a.krow0 = krow0;
     a.vrow0 = vrow0;
+    a.plane_rows = plane_rows;
     a.scale_log2 = scale_log2;
     {
         // kv-heads whose K/V rows (n rows of 2 D bytes, K and V) fit in three quarters of L2

@@ -24,10 +24,52 @@ def assert_close(got: np.ndarray, ref: np.ndarray, what=""):
     return err, rel
 
 
-def make_cache(w: si.Workload, extra_rows: int, share_map=None, device=0, scale=0.0) -> SharedKVCache:
+GUARD_BYTES = 1 << 16
+CANARY = 0xA5
+
+
+class GuardedCache(SharedKVCache):
+    """A cache whose pool and workspace sit between guard zones filled with a pattern, and whose
+    rows that no token may ever occupy (rows max_seq .. row_stride-1 of every (sequence, head) unit,
+    and whole units beyond the batch in use) are filled with the same pattern after binding.
+    `check_canaries` verifies that no kernel wrote to any of them."""
+
+    def _allocate(self, nbytes):
+        big = self._torch.full((nbytes + 2 * GUARD_BYTES,), CANARY, dtype=self._torch.uint8, device=self.device)
+        self.__dict__.setdefault("_guarded", []).append(big)
+        return big[GUARD_BYTES:GUARD_BYTES + nbytes]
+
+    def paint(self, max_seq, batch_in_use):
+        self._max_seq, self._batch_in_use = max_seq, batch_in_use
+        for s in range(self.num_slots()):
+            for kv in (0, 1):
+                p = self.plane(s, kv).view(self._torch.uint8)
+                p[:, :, max_seq:] = CANARY
+                p[batch_in_use:] = CANARY
+
+    def check_canaries(self):
+        torch_ = self._torch
+        for big in self._guarded[:1]:      # the pool (the workspace is scratch the kernels may write anywhere in)
+            assert bool((big[:GUARD_BYTES] == CANARY).all()) and bool((big[-GUARD_BYTES:] == CANARY).all()), "guard zone hit"
+        for big in self._guarded[1:]:
+            assert bool((big[:GUARD_BYTES] == CANARY).all()) and bool((big[-GUARD_BYTES:] == CANARY).all()), "workspace guard hit"
+        for s in range(self.num_slots()):
+            for kv in (0, 1):
+                p = self.plane(s, kv).view(torch_.uint8)
+                assert bool((p[:, :, self._max_seq:] == CANARY).all()), f"padding rows of plane ({s},{kv}) written"
+                assert bool((p[self._batch_in_use:] == CANARY).all()), f"unused units of plane ({s},{kv}) written"
+
+
+CACHE_CLASS = SharedKVCache       # the bounds-checking driver swaps in GuardedCache
+
+
+def make_cache(w: si.Workload, extra_rows: int, share_map=None, device=0, scale=0.0, max_batch=None) -> SharedKVCache:
     sm = w.share_map() if share_map is None else share_map
-    return SharedKVCache(w.L, w.Hq, w.Hkv, w.D, w.B, w.context + extra_rows, w.dtype, share_map=sm,
-                         softmax_scale=scale, device=device)
+    cache = CACHE_CLASS(w.L, w.Hq, w.Hkv, w.D, max_batch or w.B, w.context + extra_rows, w.dtype, share_map=sm,
+                        softmax_scale=scale, device=device)
+    if isinstance(cache, GuardedCache):
+        cache.paint(w.context + extra_rows, w.B)
+    return cache
 
 
 def run_small(w: si.Workload, steps: int, share_map=None, options=(), check_cache=True, scale=None, use_step=False):

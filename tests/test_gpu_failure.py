@@ -71,3 +71,10 @@ def test_self_test_argument_checks():
         kb.kvs_clear_device_status(ctx)
     assert e.value.status == kb.KVS_ERR_STATE
     kb.kvs_destroy(ctx)
+
+
+def test_bounds_self_test_is_refused_by_the_normal_build():
+    w, cache, _, _ = _small_cache()
+    with pytest.raises(KvsError) as e:
+        kb.kvs_selftest_bounds(cache.ctx)
+    assert e.value.status == kb.KVS_ERR_STATE and cache.device_status() == 0

@@ -408,3 +408,18 @@ def test_units_finished_inside_the_split_k_kernel(Hq, Hkv, B, dtype, kernel, con
     err = (a - c).abs().max().item()
     assert err <= 1e-5, err          # same pieces, merged in the same order by different code: rounding only
     assert cache.device_status() == 0
+
+
+# ------------------------------------------------------------------ sweep points at full size
+@pytest.mark.parametrize("name", ["sweep_b32_n1024_p10", "sweep_b64_n1024_p4", "sweep_b32_n8192_p8"])
+def test_sweep_points_sampled_units(name):
+    """32 q-heads over 8 kv-heads at batch 32 and 64 (more units than thread blocks: the tensor-core kernel
+    finishes the units itself), in the launch configuration the sweep and the benchmark time."""
+    w = si.workload_by_name(name)
+    run = SampledRun(w, steps=2, n_samples=w.n_shared + 24, seed=3)
+    run.load_context()
+    for t in range(2):
+        run.step(t, check=True)
+    run.check_cached_rows()
+    assert run.cache.last_launch()["kernel"] == 2 and run.cache.stats()["combine_launches"] == 0
+    assert run.cache.device_status() == 0
