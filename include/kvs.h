@@ -258,8 +258,10 @@ kvs_status kvs_unit_len(const kvs_ctx* ctx, int32_t layer, int32_t b, int32_t h,
  * flattened, one vector per layer); dist[i][j] is the 2-norm of
  * the difference of layers i and j's vectors (a sharing layer has its source's cache: distance 0).
  *   dist: device, float32 [n_layers][n_layers], symmetric, zero diagonal.
- * Two kernels on `stream`; reads every cached element once.  Sorting the pairs (descending, as
- * the search does) is left to the caller.
+ * Reads every cached element once: per slab of positions (sized so that the slab's sample means,
+ * which pass through the workspace, stay in L2) one kernel averages the samples and one adds the
+ * squared differences of every pair of cache slots; a last kernel sums, takes roots and expands
+ * slots to layers.  Sorting the pairs (descending, as the search does) is left to the caller.
  * Errors: STATE unless every slot holds the same non-zero number of rows and none is ragged;
  * INVALID_ARG for batch > cached batch or more than 80 layers.                                */
 kvs_status kvs_layer_distances(kvs_ctx* ctx, int32_t batch, float* dist, void* stream);

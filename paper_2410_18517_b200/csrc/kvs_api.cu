@@ -80,7 +80,8 @@ struct kvs_ctx {
 
     // workspace carve-up (byte offsets)
     size_t off_status = 0, off_part_o = 0, off_part_ml = 0, off_stage_q = 0, off_stage_k = 0, off_stage_v = 0,
-           off_stage_out = 0, off_unit_len = 0, off_counts = 0, off_search = 0, off_replay = 0, off_flags = 0, ws_bytes = 0;
+           off_stage_out = 0, off_unit_len = 0, off_counts = 0, off_search = 0, off_replay = 0, off_flags = 0, ws_bytes = 0,
+           search_bytes = 0;
 
     alignas(64) unsigned char tensor_map[128];  // TMA view of the pool (bf16 storage only), 64-row boxes
     alignas(64) unsigned char tensor_map_tail[128];   // the same view with 16-row boxes (partly filled tiles)
@@ -195,8 +196,11 @@ void layout_workspace(kvs_ctx* c) {
     off = align_up(off + units * sizeof(int32_t), kAlign);
     c->off_search = off;        // per-block partial sums of the strategy-search reductions
     {
-        const size_t need = std::max(kvs::distance_partial_bytes(f.n_layers <= kvs::kMaxLayersSearch ? f.n_layers : 4),
+        // at most one slot per layer, at most max_seq rows: enough for every strategy and length
+        const size_t need = std::max(kvs::distance_scratch_bytes(f.n_layers <= kvs::kMaxLayersSearch ? f.n_layers : 4,
+                                                                 2LL * f.n_kv_heads * f.max_seq * f.head_dim),
                                      (size_t)kvs::kSearchMaxBlocks * 3 * sizeof(double));
+        c->search_bytes = need;
         off = align_up(off + need, kAlign);
     }
     c->ws_bytes = off;
@@ -694,14 +698,15 @@ kvs_status kvs_layer_distances(kvs_ctx* ctx, int32_t batch, float* dist, void* s
         if (ctx->slot_len[s] != n || ctx->ragged[s]) return KVS_ERR_STATE;   // equally long, un-evicted caches only
     DeviceGuard guard(ctx->cfg.device);
     if (!guard.ok) return KVS_ERR_CUDA;
+    int launches = 0;
     if (kvs::launch_layer_distances(ctx->pool, (long long)ctx->plane_bytes, ctx->slot_of_layer.data(), ctx->cfg.n_layers,
-                                    batch, ctx->cfg.n_kv_heads, n, ctx->row_stride, ctx->cfg.head_dim, ctx->cfg.dtype,
-                                    reinterpret_cast<float*>(ctx->ws + ctx->off_search), dist, ctx->sm_count,
-                                    static_cast<cudaStream_t>(stream)) != cudaSuccess)
+                                    ctx->n_slots, batch, ctx->cfg.n_kv_heads, n, ctx->row_stride, ctx->cfg.head_dim,
+                                    ctx->cfg.dtype, reinterpret_cast<float*>(ctx->ws + ctx->off_search), ctx->search_bytes,
+                                    dist, ctx->sm_count, &launches, static_cast<cudaStream_t>(stream)) != cudaSuccess)
         return KVS_ERR_CUDA;
-    ctx->seq += 2;
+    ctx->seq += launches;
     ctx->last_splitk_seq = ctx->seq;     // plain launches: everything before them has finished when they run
-    ctx->stats.search_launches += 2;
+    ctx->stats.search_launches += launches;
     ctx->counter_written = false;   // a plain launch: full dependency on everything before it
     return KVS_OK;
 }

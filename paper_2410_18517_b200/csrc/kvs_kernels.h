@@ -84,12 +84,17 @@ cudaError_t launch_prefill(const void* q, float* out, int* status, int* sched, c
                            long long plane_rows, float scale_log2, int sm_count, long long l2_bytes, cudaStream_t stream);
 
 // Strategy-search reductions (see kvs_search.cu).
-constexpr int kMaxLayersSearch = 80;     // shared-memory bound of the distance kernel
-constexpr int kSearchMaxBlocks = 512;    // sizes the per-block partial buffers
-size_t distance_partial_bytes(int L);
-cudaError_t launch_layer_distances(const void* pool, long long plane_bytes, const int* slot_of_layer, int L, int B,
-                                   int Hkv, int n, int row_stride, int D, int dtype, float* partial, float* dist,
-                                   int sm_count, cudaStream_t stream);
+constexpr int kMaxLayersSearch = 80;     // bound of the layer -> slot table handed to the finishing kernel
+constexpr int kSearchMaxBlocks = 640;    // sizes the per-block partial buffers
+// The sample means of a slab of positions go through scratch memory between the two passes; a slab is
+// sized so that they stay in L2 (a fraction of its 126 MB).
+constexpr long long kMeanSlabBytes = 48ll << 20;
+// Scratch the distance reduction needs for `n_slots` cache slots of `positions` = 2 * Hkv * n * D elements.
+size_t distance_scratch_bytes(int n_slots, long long positions);
+// *launches receives the number of kernels launched (two per slab and two to finish).
+cudaError_t launch_layer_distances(const void* pool, long long plane_bytes, const int* slot_of_layer, int L, int n_slots,
+                                   int B, int Hkv, int n, int row_stride, int D, int dtype, float* scratch,
+                                   size_t scratch_bytes, float* dist, int sm_count, int* launches, cudaStream_t stream);
 cudaError_t launch_mean_cosine(const void* a, const void* b, int S, long long dim, int dtype, double* partial,
                                float* out, int sm_count, cudaStream_t stream);
 

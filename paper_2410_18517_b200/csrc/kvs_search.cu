@@ -1,10 +1,13 @@
 // The data-parallel reductions of KVSharer's strategy search (Section 3.1, Algorithm 1), run
 // on caches already resident in the pool:
-//   layer_distance_kernel   sample-mean K/V representation of every layer, then the squared
-//                           Euclidean distance of every pair of layers (one pass over the pool)
-//   distance_finish_kernel  fixed-order sum of the per-block partial matrices, square root
+//   layer_mean_kernel       sample-mean K/V representation of every cache slot over a slab of
+//                           positions, streamed in long contiguous runs (one pass over the pool)
+//   mean_distance_kernel    squared Euclidean distances of every pair of slots over that slab,
+//                           from the means (which stay in L2 between the two kernels)
+//   distance_sum_kernel     fixed-order sum of the per-block partial matrices
+//   distance_finish_kernel  square roots, slot pairs expanded to layer pairs
 //   mean_cosine_kernel      cosine similarity of the sample-means of two [S][dim] tensors
-// Both are bandwidth-bound: every cached element is read exactly once.
+// All are bandwidth-bound: every cached element is read exactly once.
 #include "kvs_device.cuh"
 #include "kvs_kernels.h"
 
@@ -14,15 +17,17 @@ namespace kvs {
 
 namespace {
 
+constexpr int kMeanThreads = 256;
+constexpr int kMeanChunk = kMeanThreads * 8;   // positions per work item of the mean kernel: 8 per thread (16-byte loads of bf16)
 constexpr int kDistThreads = 256;
-constexpr int kDistChunk = 512;          // positions per chunk: two per thread
-constexpr int kDistStride = kDistChunk + 1;   // padded row of the mean tile (bank = layer + position)
+constexpr int kDistChunk = 512;                // positions per chunk of the distance kernel: two per thread
+constexpr int kDistStride = kDistChunk + 1;    // padded row of the mean tile (bank = slot + position)
 
-// 1, 2, 4 or 8 thread groups share the positions of a chunk when there are few layer-pair blocks.
+// As many thread groups as the block has threads for (at most 16) share the positions of a chunk, so that
+// every thread has a 4x4 block of slot pairs to work on.
 __host__ __device__ inline int dist_groups(int items) {
-    int g = 1;
-    while (g < 8 && 2 * g * items <= kDistThreads) g *= 2;
-    return g;
+    const int g = kDistThreads / items;
+    return g < 1 ? 1 : (g > 16 ? 16 : g);
 }
 
 template <typename T>
@@ -55,112 +60,180 @@ __device__ __forceinline__ void add8<float>(const float* p, float (&s)[8]) {
     s[4] += b.x; s[5] += b.y; s[6] += b.z; s[7] += b.w;
 }
 
-struct DistArgs {
+// The same for data that is read exactly once (streaming load: it is the first to leave the caches).
+template <typename T>
+__device__ __forceinline__ void add8_once(const T* p, float (&s)[8]);
+template <>
+__device__ __forceinline__ void add8_once<__nv_bfloat16>(const __nv_bfloat16* p, float (&s)[8]) {
+    const uint4 r = __ldcs(reinterpret_cast<const uint4*>(p));
+    float f[8];
+    Unpack<__nv_bfloat16>::run(r, f);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) s[i] += f[i];
+}
+template <>
+__device__ __forceinline__ void add8_once<float>(const float* p, float (&s)[8]) {
+    const float4 a = __ldcs(reinterpret_cast<const float4*>(p)), b = __ldcs(reinterpret_cast<const float4*>(p + 4));
+    s[0] += a.x; s[1] += a.y; s[2] += a.z; s[3] += a.w;
+    s[4] += b.x; s[5] += b.y; s[6] += b.z; s[7] += b.w;
+}
+
+// ---- pass 1: sample means --------------------------------------------------------------------
+// Positions p of a layer's representation run over (K or V, kv-head, row, column): P = 2 * Hkv * n * D.
+// A work item is (slot, chunk of kMeanChunk positions of the slab [p0, p1)): every thread owns 8
+// consecutive positions and adds the B samples' values, which lie one (sequence) stride apart, so a
+// block reads B runs of 4 KiB (bf16) and neighbouring blocks continue the same runs.  The means go
+// to `mean` as [slot][p - p0] fp32: small enough (the slab is sized for it) to stay in L2 until the
+// distance kernel has read them.
+struct MeanArgs {
     const char* pool;
-    float* partial;            // [blocks][Lp*Lp]
+    float* mean;               // [n_slots][slab]
     long long plane_bytes;
-    int slot_of_layer[kMaxLayersSearch];
-    int L, Lp;                 // layers, rounded up to a multiple of 4
-    int B, Hkv, n, row_stride, D;
-    long long P;               // positions: 2 * Hkv * n * D
+    int n_slots, B, Hkv, n, row_stride, D;
+    long long p0, p1, slab;    // slab = positions per slot row of `mean` (>= p1 - p0)
 };
 
-// Shared memory: mean tile M[Lp][kDistStride] fp32, then accumulators acc[groups][Lp*Lp].
 template <typename T>
-__global__ void __launch_bounds__(kDistThreads) layer_distance_kernel(const DistArgs a) {
-    extern __shared__ float sm[];
-    float* M = sm;
-    float* acc = sm + a.Lp * kDistStride;
-    const int tid = threadIdx.x;
-    const int tiles = a.Lp / 4;
-    const int items = tiles * tiles;                               // 4x4 blocks of layer pairs
-    const int groups = dist_groups(items);                         // thread groups splitting the positions
-    for (int i = tid; i < groups * a.Lp * a.Lp; i += kDistThreads) acc[i] = 0.f;
-    for (int i = tid; i < (a.Lp - a.L) * kDistStride; i += kDistThreads) M[a.L * kDistStride + i] = 0.f;  // padding layers
-    __syncthreads();
-
+__global__ void __launch_bounds__(kMeanThreads) layer_mean_kernel(const MeanArgs a) {
     const long long unit_elems = (long long)a.n * a.D;            // cached elements of one (sequence, head)
     const long long kv_elems = (long long)a.Hkv * unit_elems;
-    const long long chunks = (a.P + kDistChunk - 1) / kDistChunk;
+    const long long bstride = (long long)a.Hkv * a.row_stride * a.D;
+    const long long chunks = (a.p1 - a.p0 + kMeanChunk - 1) / kMeanChunk;
     const float inv_b = 1.0f / a.B;
+    for (long long item = blockIdx.x; item < chunks * a.n_slots; item += gridDim.x) {
+        const int slot = (int)(item / chunks);
+        const long long p = a.p0 + (item - slot * chunks) * kMeanChunk + 8 * threadIdx.x;
+        if (p >= a.p1) continue;
+        // a unit holds a multiple of 8 elements, so the 8 positions never straddle two units
+        const int kv = (int)(p / kv_elems);
+        const long long rem = p - kv * kv_elems;
+        const int h = (int)(rem / unit_elems);
+        const long long e = rem - h * unit_elems;
+        const T* base = reinterpret_cast<const T*>(a.pool + (long long)(2 * slot + kv) * a.plane_bytes) +
+                        (long long)h * a.row_stride * a.D + e;
+        float s8[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+#pragma unroll 10
+        for (int b = 0; b < a.B; ++b) add8_once<T>(base + b * bstride, s8);
+        float4* dst = reinterpret_cast<float4*>(a.mean + (long long)slot * a.slab + (p - a.p0));
+        dst[0] = make_float4(s8[0] * inv_b, s8[1] * inv_b, s8[2] * inv_b, s8[3] * inv_b);
+        dst[1] = make_float4(s8[4] * inv_b, s8[5] * inv_b, s8[6] * inv_b, s8[7] * inv_b);
+    }
+}
+
+// ---- pass 2: squared differences of every slot pair over the slab ---------------------------
+// Per 512-position chunk a block copies every slot's means into a shared-memory tile ([slots][513],
+// padded so that slot-pair reads are conflict-free), then 4x4 register blocks of slot pairs (upper
+// triangle only: the matrix is symmetric) accumulate squared differences of the means (differences,
+// not a Gram matrix, so near-identical layers do not cancel).  A block adds its chunks' sums to its
+// own partial matrix, slab after slab, always in the same order.
+struct DistArgs {
+    const float* mean;         // [n_slots][slab]
+    float* partial;            // [blocks][Sp*Sp]
+    int S, Sp;                 // slots, rounded up to a multiple of 4
+    long long count, slab;     // positions of this slab, row length of `mean`
+    int first;                 // 1: the partial matrices start from zero with this launch
+};
+
+__global__ void __launch_bounds__(kDistThreads) mean_distance_kernel(const DistArgs a) {
+    extern __shared__ float sm[];
+    float* M = sm;
+    float* acc = sm + a.Sp * kDistStride;
+    const int tid = threadIdx.x;
+    const int tiles = a.Sp / 4;
+    const int items = tiles * (tiles + 1) / 2;                     // 4x4 blocks of slot pairs with ti <= tj
+    const int groups = dist_groups(items);                         // thread groups splitting the positions
+    for (int i = tid; i < groups * a.Sp * a.Sp; i += kDistThreads) acc[i] = 0.f;
+    for (int i = tid; i < (a.Sp - a.S) * kDistStride; i += kDistThreads) M[a.S * kDistStride + i] = 0.f;  // padding slots
+    __syncthreads();
+    const long long chunks = (a.count + kDistChunk - 1) / kDistChunk;
     for (long long c = blockIdx.x; c < chunks; c += gridDim.x) {
-        // ---- means of this chunk's positions, all layers ----
-        // 64 groups of 8 consecutive positions (16-byte loads); the 4 quarters of the block take
-        // every fourth layer.  A unit holds a multiple of 8 elements, so a group never straddles two.
-        // Position 8*pg + i of the chunk is stored at column 64*i + pg: the order of positions inside
-        // a chunk is irrelevant to the sums and this one keeps the stores conflict-free.
-        {
-            const int pg = tid & 63, lq = tid >> 6;
-            const long long p = c * kDistChunk + 8 * pg;
-            if (p < a.P) {
-                const int kv = (int)(p / kv_elems);
-                const long long rem = p - kv * kv_elems;
-                const int h = (int)(rem / unit_elems);
-                const long long e = rem - h * unit_elems;
-                const long long bstride = (long long)a.Hkv * a.row_stride * a.D;
-                for (int l = lq; l < a.L; l += 4) {
-                    const T* base = reinterpret_cast<const T*>(a.pool + (long long)(2 * a.slot_of_layer[l] + kv) * a.plane_bytes) +
-                                    (long long)h * a.row_stride * a.D + e;
-                    float s8[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-#pragma unroll 8
-                    for (int b = 0; b < a.B; ++b) add8<T>(base + b * bstride, s8);
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) M[l * kDistStride + 64 * i + pg] = s8[i] * inv_b;
-                }
-            } else {
-                for (int l = lq; l < a.L; l += 4)
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) M[l * kDistStride + 64 * i + pg] = 0.f;
-            }
+        const long long p = c * kDistChunk;
+        const int have = (int)min((long long)kDistChunk, a.count - p);
+        // a warp reads 32 consecutive positions of one slot and stores them to 32 different banks; sixteen loads
+        // are in flight per thread (the means come from L2)
+#pragma unroll 16
+        for (int i = tid; i < a.S * kDistChunk; i += kDistThreads) {
+            const int sl = i / kDistChunk, q = i - sl * kDistChunk;
+            M[sl * kDistStride + q] = q < have ? __ldcg(a.mean + (long long)sl * a.slab + p + q) : 0.f;
         }
         __syncthreads();
-        // ---- squared differences of every layer pair over the chunk ----
         for (int w = tid; w < groups * items; w += kDistThreads) {
-            const int g = w / items, it = w - g * items;
-            const int ti = (it / tiles) * 4, tj = (it % tiles) * 4;
+            const int g = w / items;
+            int it = w - g * items, ti = 0;
+            while (it >= tiles - ti) {       // row ti of the upper triangle holds tiles - ti blocks
+                it -= tiles - ti;
+                ++ti;
+            }
+            const int tj = ti + it;
             float d[4][4];
 #pragma unroll
             for (int x = 0; x < 4; ++x)
 #pragma unroll
                 for (int y = 0; y < 4; ++y) d[x][y] = 0.f;
-            const int per = kDistChunk / groups;
-            for (int q = g * per; q < (g + 1) * per; ++q) {
-                float mi[4], mj[4];
+            const int per = (kDistChunk + groups - 1) / groups;
+            const int q1 = min(kDistChunk, (g + 1) * per);
+            for (int q = g * per; q < q1; ++q) {
+                float mi[4];
+                float2 mj[2];
 #pragma unroll
-                for (int x = 0; x < 4; ++x) {
-                    mi[x] = M[(ti + x) * kDistStride + q];
-                    mj[x] = M[(tj + x) * kDistStride + q];
-                }
+                for (int x = 0; x < 4; ++x) mi[x] = M[(4 * ti + x) * kDistStride + q];
+                mj[0] = make_float2(M[(4 * tj) * kDistStride + q], M[(4 * tj + 1) * kDistStride + q]);
+                mj[1] = make_float2(M[(4 * tj + 2) * kDistStride + q], M[(4 * tj + 3) * kDistStride + q]);
+                // two slot pairs per instruction (packed fp32): t = mi - mj, d += t * t
+                const float2 minus1 = make_float2(-1.f, -1.f);
 #pragma unroll
                 for (int x = 0; x < 4; ++x)
 #pragma unroll
-                    for (int y = 0; y < 4; ++y) {
-                        const float t = mi[x] - mj[y];
-                        d[x][y] = fmaf(t, t, d[x][y]);
+                    for (int y = 0; y < 2; ++y) {
+                        const float2 t = __ffma2_rn(mj[y], minus1, make_float2(mi[x], mi[x]));
+                        const float2 r = __ffma2_rn(t, t, make_float2(d[x][2 * y], d[x][2 * y + 1]));
+                        d[x][2 * y] = r.x;
+                        d[x][2 * y + 1] = r.y;
                     }
             }
-            float* dst = acc + g * a.Lp * a.Lp;
+            float* dst = acc + g * a.Sp * a.Sp;
 #pragma unroll
             for (int x = 0; x < 4; ++x)
 #pragma unroll
-                for (int y = 0; y < 4; ++y) dst[(ti + x) * a.Lp + tj + y] += d[x][y];   // (g, item) has one owner
+                for (int y = 0; y < 4; ++y) dst[(4 * ti + x) * a.Sp + 4 * tj + y] += d[x][y];   // (g, block) has one owner
         }
         __syncthreads();
     }
-    for (int i = tid; i < a.Lp * a.Lp; i += kDistThreads) {
+    for (int i = tid; i < a.Sp * a.Sp; i += kDistThreads) {
         float s = 0.f;
-        for (int g = 0; g < groups; ++g) s += acc[g * a.Lp * a.Lp + i];
-        a.partial[(long long)blockIdx.x * a.Lp * a.Lp + i] = s;
+        for (int g = 0; g < groups; ++g) s += acc[g * a.Sp * a.Sp + i];
+        float* dst = a.partial + (long long)blockIdx.x * a.Sp * a.Sp + i;
+        *dst = a.first ? s : *dst + s;
     }
 }
 
-__global__ void distance_finish_kernel(const float* __restrict__ partial, float* __restrict__ dist, int L, int Lp,
-                                       int blocks) {
+// slot_dist2[r][c] (r < c) = sum over blocks of the (r, c) entries of their partial matrices: one warp
+// per entry, lane l adds blocks l, l + 32, ... and the lanes are added in a fixed order.
+__global__ void __launch_bounds__(256) distance_sum_kernel(const float* __restrict__ partial, double* __restrict__ slot_dist2,
+                                                           int S, int Sp, int blocks) {
+    const int entry = blockIdx.x * 8 + (threadIdx.x >> 5), lane = threadIdx.x & 31;
+    if (entry >= S * S) return;
+    const int r = entry / S, c = entry - r * S;
+    double s = 0.0;
+    if (r < c)
+        for (int b = lane; b < blocks; b += 32) s += partial[(long long)b * Sp * Sp + r * Sp + c];
+#pragma unroll
+    for (int o = 16; o >= 1; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    if (lane == 0) slot_dist2[entry] = s;
+}
+
+struct FinishArgs {
+    int slot_of_layer[kMaxLayersSearch];
+};
+
+// dist[i][j] = sqrt of the entry of the two layers' slots (zero for two layers on one slot).
+__global__ void distance_finish_kernel(const double* __restrict__ slot_dist2, float* __restrict__ dist, int L, int S,
+                                       const FinishArgs f) {
     const int i = blockIdx.x, j = threadIdx.x;
     if (j >= L) return;
-    double s = 0.0;
-    for (int c = 0; c < blocks; ++c) s += partial[(long long)c * Lp * Lp + i * Lp + j];
-    dist[i * L + j] = (i == j) ? 0.f : (float)sqrt(s);
+    const int si = f.slot_of_layer[i], sj = f.slot_of_layer[j];
+    const int r = min(si, sj), c = max(si, sj);
+    dist[i * L + j] = r == c ? 0.f : (float)sqrt(slot_dist2[r * S + c]);
 }
 
 // ---- mean cosine --------------------------------------------------------------------------
@@ -231,43 +304,69 @@ __global__ void cosine_finish_kernel(const double* __restrict__ partial, int blo
 
 }  // namespace
 
-size_t distance_partial_bytes(int L) {
-    const int Lp = (L + 3) / 4 * 4;
-    return (size_t)kSearchMaxBlocks * Lp * Lp * sizeof(float);
+size_t distance_scratch_bytes(int n_slots, long long positions) {
+    // per-block partial matrices, then the slab of means: as many positions per slot as fit the budget
+    const int Sp = (n_slots + 3) / 4 * 4;
+    const size_t partial = ((size_t)kSearchMaxBlocks * Sp * Sp * sizeof(float) + 255) / 256 * 256;
+    long long slab = std::min<long long>(kMeanSlabBytes / ((long long)n_slots * 4), positions);
+    slab = std::max<long long>((slab + kMeanChunk - 1) / kMeanChunk * kMeanChunk, kMeanChunk);
+    return partial + (size_t)n_slots * slab * sizeof(float);
 }
 
-cudaError_t launch_layer_distances(const void* pool, long long plane_bytes, const int* slot_of_layer, int L, int B,
-                                   int Hkv, int n, int row_stride, int D, int dtype, float* partial, float* dist,
-                                   int sm_count, cudaStream_t stream) {
+cudaError_t launch_layer_distances(const void* pool, long long plane_bytes, const int* slot_of_layer, int L, int n_slots,
+                                   int B, int Hkv, int n, int row_stride, int D, int dtype, float* scratch,
+                                   size_t scratch_bytes, float* dist, int sm_count, int* launches, cudaStream_t stream) {
     if (L > kMaxLayersSearch) return cudaErrorInvalidValue;
-    DistArgs a;
-    a.pool = (const char*)pool;
-    a.partial = partial;
-    a.plane_bytes = plane_bytes;
-    for (int l = 0; l < L; ++l) a.slot_of_layer[l] = slot_of_layer[l];
-    a.L = L;
-    a.Lp = (L + 3) / 4 * 4;
-    a.B = B; a.Hkv = Hkv; a.n = n; a.row_stride = row_stride; a.D = D;
-    a.P = 2LL * Hkv * n * D;
-    const int tiles = a.Lp / 4, items = tiles * tiles;
+    const int S = n_slots, Sp = (S + 3) / 4 * 4;
+    const long long P = 2LL * Hkv * n * D;
+    const size_t partial_bytes = ((size_t)kSearchMaxBlocks * Sp * Sp * sizeof(float) + 255) / 256 * 256;
+    if (scratch_bytes < partial_bytes + (size_t)S * kMeanChunk * sizeof(float)) return cudaErrorInvalidValue;
+    // positions per slab: what the scratch holds, in whole mean-kernel chunks
+    long long slab = (long long)((scratch_bytes - partial_bytes) / sizeof(float) / S);
+    slab = std::min(slab / kMeanChunk * kMeanChunk, (P + kMeanChunk - 1) / kMeanChunk * kMeanChunk);
+    float* partial = scratch;
+    float* mean = reinterpret_cast<float*>(reinterpret_cast<char*>(scratch) + partial_bytes);
+
+    const int tiles = Sp / 4, items = tiles * (tiles + 1) / 2;
     const int groups = dist_groups(items);
-    const size_t smem = ((size_t)a.Lp * kDistStride + (size_t)groups * a.Lp * a.Lp) * sizeof(float);
-    const long long chunks = (a.P + kDistChunk - 1) / kDistChunk;
-    const int blocks = (int)std::min<long long>(chunks, std::min(2 * sm_count, kSearchMaxBlocks));
+    const size_t smem = ((size_t)Sp * kDistStride + (size_t)groups * Sp * Sp) * sizeof(float);
     cudaError_t e;
-    if (dtype == 0) {
-        if ((e = cudaFuncSetAttribute(layer_distance_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                      (int)smem)) != cudaSuccess)
-            return e;
-        layer_distance_kernel<__nv_bfloat16><<<blocks, kDistThreads, smem, stream>>>(a);
-    } else {
-        if ((e = cudaFuncSetAttribute(layer_distance_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                      (int)smem)) != cudaSuccess)
-            return e;
-        layer_distance_kernel<float><<<blocks, kDistThreads, smem, stream>>>(a);
+    if ((e = cudaFuncSetAttribute(mean_distance_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess)
+        return e;
+    const int dist_blocks = (int)std::min<long long>((std::min(slab, P) + kDistChunk - 1) / kDistChunk,
+                                                     std::min(2 * sm_count, kSearchMaxBlocks));
+    *launches = 0;
+    for (long long p0 = 0; p0 < P; p0 += slab) {
+        MeanArgs m;
+        m.pool = (const char*)pool;
+        m.mean = mean;
+        m.plane_bytes = plane_bytes;
+        m.n_slots = S; m.B = B; m.Hkv = Hkv; m.n = n; m.row_stride = row_stride; m.D = D;
+        m.p0 = p0; m.p1 = std::min(P, p0 + slab); m.slab = slab;
+        const long long mean_items = (m.p1 - m.p0 + kMeanChunk - 1) / kMeanChunk * S;
+        const int mean_blocks = (int)std::min<long long>(mean_items, 16LL * sm_count);
+        if (dtype == 0) layer_mean_kernel<__nv_bfloat16><<<mean_blocks, kMeanThreads, 0, stream>>>(m);
+        else layer_mean_kernel<float><<<mean_blocks, kMeanThreads, 0, stream>>>(m);
+        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+        DistArgs a;
+        a.mean = mean;
+        a.partial = partial;
+        a.S = S; a.Sp = Sp;
+        a.count = m.p1 - m.p0; a.slab = slab;
+        a.first = p0 == 0 ? 1 : 0;
+        // the same number of blocks for every slab: block b's partial matrix is its own, slab after slab
+        mean_distance_kernel<<<dist_blocks, kDistThreads, smem, stream>>>(a);
+        if ((e = cudaGetLastError()) != cudaSuccess) return e;
+        *launches += 2;
     }
+    // the slab of means is no longer needed: its first bytes hold the slot-pair sums for a moment
+    double* slot_dist2 = reinterpret_cast<double*>(mean);
+    distance_sum_kernel<<<(S * S + 7) / 8, 256, 0, stream>>>(partial, slot_dist2, S, Sp, dist_blocks);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
-    distance_finish_kernel<<<L, a.Lp, 0, stream>>>(partial, dist, L, a.Lp, blocks);
+    FinishArgs f;
+    for (int l = 0; l < L; ++l) f.slot_of_layer[l] = slot_of_layer[l];
+    distance_finish_kernel<<<L, (L + 31) / 32 * 32, 0, stream>>>(slot_dist2, dist, L, S, f);
+    *launches += 2;
     return cudaGetLastError();
 }
 

@@ -56,7 +56,7 @@ def test_layer_distances(L, Hq, Hkv, D, B, n, dtype):
     clear = np.abs(np.diff(sorted_ref)) > 4 * REL * sorted_ref[:-1]       # gap k | k+1 is unambiguous
     isolated = np.append(clear, True) & np.append(True, clear)             # both neighbours clearly apart
     assert np.array_equal(order_ref[isolated], order_got[isolated])
-    assert cache.device_status() == 0 and cache.stats()["search_launches"] == 2
+    assert cache.device_status() == 0 and cache.stats()["search_launches"] >= 3
 
 
 def test_layer_distances_state_errors():
