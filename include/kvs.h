@@ -222,8 +222,9 @@ kvs_status kvs_decode_step(kvs_ctx* ctx, int32_t layer, const void* q, const voi
  * chunk of it (n > n_q).
  *   q:   device, [batch][n_q][n_q_heads][head_dim], storage type, 16-byte aligned
  *   out: device, [batch][n_q][n_q_heads][head_dim], float32
- * One 4-byte clear and one tcgen05 tensor-core kernel on `stream`; bf16 storage only (other
- * configurations: INVALID_ARG).  Other errors as kvs_decode_attention; n_q > n: INVALID_ARG. */
+ * bf16 storage: one 4-byte clear and one tcgen05 tensor-core kernel on `stream`.  fp32 storage (the
+ * small configuration): one plain fp32 kernel, a warp per query.  A slot rows were evicted from:
+ * STATE.  Other errors as kvs_decode_attention; n_q > n: INVALID_ARG.                             */
 kvs_status kvs_prefill_attention(kvs_ctx* ctx, int32_t layer, const void* q, float* out,
                                  int32_t batch, int32_t n_q, void* stream);
 

@@ -10,7 +10,7 @@ CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libkvs.so")
 # the same sources with -DKVS_DEBUG_BOUNDS: every computed global offset is checked on the device
 LIB_BOUNDS = os.path.join(HERE, "libkvs_bounds.so")
-SOURCES = ["kvs_api.cu", "kvs_kernels.cu", "kvs_mma.cu", "kvs_prefill.cu", "kvs_search.cu"]
+SOURCES = ["kvs_api.cu", "kvs_kernels.cu", "kvs_mma.cu", "kvs_prefill.cu", "kvs_prefill_f32.cu", "kvs_search.cu"]
 HEADERS = ["kvs_device.cuh", "kvs_kernels.h", os.path.join("..", "..", "include", "kvs.h")]
 
 NVCC_FLAGS = [

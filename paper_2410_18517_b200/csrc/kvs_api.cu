@@ -609,7 +609,7 @@ kvs_status kvs_prefill_attention(kvs_ctx* ctx, int32_t layer, const void* q, flo
     if (!ctx->bound) return KVS_ERR_STATE;
     if (layer < 0 || layer >= ctx->cfg.n_layers || !q || !out) return KVS_ERR_INVALID_ARG;
     if (batch < 1 || batch > ctx->cfg.max_batch || n_q < 1) return KVS_ERR_INVALID_ARG;
-    if (ctx->cfg.dtype != KVS_BF16 || !ctx->have_tensor_map) return KVS_ERR_INVALID_ARG;
+    if (ctx->cfg.dtype == KVS_BF16 && !ctx->have_tensor_map) return KVS_ERR_STATE;
     if (((uintptr_t)q % 16) != 0 || ((uintptr_t)out % 16) != 0) return KVS_ERR_INVALID_ARG;
     const int slot = ctx->slot_of_layer[layer];
     const int n = ctx->slot_len[slot];
@@ -617,6 +617,19 @@ kvs_status kvs_prefill_attention(kvs_ctx* ctx, int32_t layer, const void* q, flo
     if (batch > ctx->cur_batch || n_q > n) return KVS_ERR_INVALID_ARG;
     DeviceGuard guard(ctx->cfg.device);
     if (!guard.ok) return KVS_ERR_CUDA;
+    if (ctx->cfg.dtype == KVS_F32) {
+        // fp32 storage: the plain fp32 kernel (a plain launch, like the tensor-core one)
+        const char* kp = ctx->pool + (size_t)(2 * slot) * ctx->plane_bytes;
+        if (kvs::launch_prefill_f32(q, out, kp, kp + ctx->plane_bytes, batch, n_q, ctx->cfg.n_q_heads, ctx->G,
+                                    ctx->cfg.head_dim, n, ctx->row_stride, ctx->scale * 1.4426950408889634f,
+                                    static_cast<cudaStream_t>(stream)) != cudaSuccess)
+            return KVS_ERR_CUDA;
+        ctx->seq += 1;
+        ctx->last_splitk_seq = ctx->seq;
+        ctx->stats.prefill_launches += 1;
+        ctx->counter_written = false;
+        return KVS_OK;
+    }
     const long long plane_rows = (long long)ctx->cfg.max_batch * ctx->cfg.n_kv_heads * ctx->row_stride;
     // the prefill kernel's work counter lives in the status block, 64 bytes after the status word
     if (kvs::launch_prefill(q, out, reinterpret_cast<int*>(ctx->ws + ctx->off_status),

@@ -83,6 +83,10 @@ cudaError_t launch_prefill(const void* q, float* out, int* status, int* sched, c
                            int Hq, int G, int D, int n, int row_stride, long long krow0, long long vrow0,
                            long long plane_rows, float scale_log2, int sm_count, long long l2_bytes, cudaStream_t stream);
 
+// The same causal prefill attention for fp32 storage (plain fp32 kernel; see kvs_prefill_f32.cu).
+cudaError_t launch_prefill_f32(const void* q, float* out, const void* kplane, const void* vplane, int B, int T, int Hq,
+                               int G, int D, int n, int row_stride, float scale_log2, cudaStream_t stream);
+
 // Strategy-search reductions (see kvs_search.cu).
 constexpr int kMaxLayersSearch = 80;     // bound of the layer -> slot table handed to the finishing kernel
 constexpr int kSearchMaxBlocks = 640;    // sizes the per-block partial buffers

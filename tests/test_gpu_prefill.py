@@ -20,19 +20,20 @@ def _built():
     kbuild.build()
 
 
-def _prefill_both(Hq, Hkv, B, chunks, share_map, seed=0, D=128):
+def _prefill_both(Hq, Hkv, B, chunks, share_map, seed=0, D=128, dtype="bf16"):
     """Feed the prompt in `chunks` (list of chunk lengths) to both sides, layer by layer."""
     L = len(share_map)
     total = sum(chunks)
-    cache = SharedKVCache(L, Hq, Hkv, D, B, total, "bf16", share_map=share_map)
+    tdt = torch.bfloat16 if dtype == "bf16" else torch.float32
+    cache = SharedKVCache(L, Hq, Hkv, D, B, total, dtype, share_map=share_map)
     orc = oracle.Oracle(L, Hq, Hkv, D, B, share_map)
     worst = (0.0, 0.0)
     for c, T in enumerate(chunks):
         for l in range(L):
-            w = si.Workload(f"pf_{seed}_{c}", L=L, Hq=Hq, Hkv=Hkv, D=D, B=B, context=T, dtype="bf16", n_shared=0,
+            w = si.Workload(f"pf_{seed}_{c}", L=L, Hq=Hq, Hkv=Hkv, D=D, B=B, context=T, dtype=dtype, n_shared=0,
                             map_seed=0, steps=1)
             k, v = si.context_kv(w, l, base_seed=seed)
-            q = si.normal((seed, "pf_q", c, l), (B, T, Hq, D), torch.bfloat16)
+            q = si.normal((seed, "pf_q", c, l), (B, T, Hq, D), tdt)
             ref = orc.layer_prefill(l, q.double().numpy(), k.double().numpy(), v.double().numpy())
             if share_map[l] == l:
                 cache.append(l, k.cuda(), v.cuda())
@@ -58,6 +59,15 @@ def test_prompt_lengths_chunks_and_sharing(Hq, Hkv, chunks):
 @pytest.mark.parametrize("chunks", [[1], [64], [129], [300], [200, 333]])
 def test_head_size_64(Hq, Hkv, chunks):
     _prefill_both(Hq, Hkv, 2, chunks, [0, 0, 2, 0], D=64)
+
+
+@pytest.mark.parametrize("D,Hq,Hkv", [(64, 4, 4), (128, 4, 2), (128, 8, 1), (64, 2, 1)])
+@pytest.mark.parametrize("chunks", [[1], [33], [128], [200, 77], [128, 1, 8]])
+def test_fp32_storage(D, Hq, Hkv, chunks):
+    """fp32 Q/K/V (the small configuration: 4 heads, head size 64, 128 context rows) go through the plain
+    fp32 prefill kernel; same oracle, same strategy handling, and far inside the bf16 tolerance."""
+    _, _, worst = _prefill_both(Hq, Hkv, 2, chunks, [0, 1, 2, 1], D=D, dtype="f32")
+    assert worst[0] < 1e-4
 
 
 @pytest.mark.parametrize("D,Hq,Hkv,B,chunks", [(128, 32, 8, 2, [2100]), (128, 16, 16, 3, [1500]), (64, 32, 8, 2, [2100]),
@@ -130,6 +140,7 @@ def test_prefill_argument_checks():
     f = SharedKVCache(1, 2, 2, 64, 1, 64, "f32")
     kk = torch.zeros(1, 4, 2, 64, dtype=torch.float32, device="cuda")
     f.append(0, kk, kk)
-    with pytest.raises(KvsError) as e:          # fp32 storage is not built for prefill
-        kb.kvs_prefill_attention(f.ctx, 0, kk, torch.zeros(1, 4, 2, 64, device="cuda"), 1, 4, 0)
+    with pytest.raises(KvsError) as e:          # fp32 storage has its own kernel; the checks are the same
+        kb.kvs_prefill_attention(f.ctx, 0, torch.zeros(1, 8, 2, 64, device="cuda"), torch.zeros(1, 8, 2, 64, device="cuda"),
+                                 1, 8, 0)
     assert e.value.status == kb.KVS_ERR_INVALID_ARG
