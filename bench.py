@@ -202,7 +202,7 @@ def workload_config(w, n_gpus):
                   f"{w.L - w.n_shared} distinct slots are cycled"}
 
 
-MIN_TIMED_S = 1.0       # regions of K steps are repeated until this much has been timed
+MIN_TIMED_S = 1.0       # regions of K steps are repeated until this much has been timed (--min-seconds)
 MAX_REGIONS = 200
 
 
@@ -280,7 +280,7 @@ def measure(w, K, W, E, rank, local_rank, world, dist, with_isolated=True, with_
     region_ms = [region()]
     st1 = cache.stats()
     # every rank derives the same count from the same (maximum-over-ranks) first region
-    n_regions = max(1, min(MAX_REGIONS, int(-(-MIN_TIMED_S * 1e3 // region_ms[0]))))
+    n_regions = max(1, min(MAX_REGIONS, int(-(-MIN_TIMED_S * 1e3 // max(region_ms[0], 1e-3)))))
     for _ in range(n_regions - 1):
         region_ms.append(region())
     clocks = sampler.stop() if rank == 0 else None
@@ -459,7 +459,11 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=20)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-prefill", action="store_true")
+    ap.add_argument("--min-seconds", type=float, default=MIN_TIMED_S,
+                    help="regions of --steps steps are repeated until this much has been timed (0: one region, for "
+                         "profiler captures)")
     args = ap.parse_args()
+    globals()["MIN_TIMED_S"] = args.min_seconds
     if args.warmup < 3 and args.impl == "kvs":
         args.warmup = 3
 

@@ -95,10 +95,12 @@ constexpr int kSearchMaxBlocks = 640;    // sizes the per-block partial buffers
 constexpr long long kMeanSlabBytes = 48ll << 20;
 // Scratch the distance reduction needs for `n_slots` cache slots of `positions` = 2 * Hkv * n * D elements.
 size_t distance_scratch_bytes(int n_slots, long long positions);
-// *launches receives the number of kernels launched (two per slab and two to finish).
+// *launches receives the number of kernels launched (two per slab and two to finish).  The distance pass of
+// a slab runs on `side` beside the mean pass of the next slab on `stream`; ev_mean / ev_dist: two events each.
 cudaError_t launch_layer_distances(const void* pool, long long plane_bytes, const int* slot_of_layer, int L, int n_slots,
                                    int B, int Hkv, int n, int row_stride, int D, int dtype, float* scratch,
-                                   size_t scratch_bytes, float* dist, int sm_count, int* launches, cudaStream_t stream);
+                                   size_t scratch_bytes, float* dist, int sm_count, int* launches, cudaStream_t stream,
+                                   cudaStream_t side, cudaEvent_t* ev_mean, cudaEvent_t* ev_dist);
 cudaError_t launch_mean_cosine(const void* a, const void* b, int S, long long dim, int dtype, double* partial,
                                float* out, int sm_count, cudaStream_t stream);
 

@@ -304,28 +304,37 @@ __global__ void cosine_finish_kernel(const double* __restrict__ partial, int blo
 
 }  // namespace
 
-size_t distance_scratch_bytes(int n_slots, long long positions) {
-    // per-block partial matrices, then the slab of means: as many positions per slot as fit the budget
+// Scratch layout: per-block partial matrices, then TWO slabs of means (the distance pass of one slab runs
+// beside the mean pass of the next).
+static size_t distance_partial_bytes(int n_slots) {
     const int Sp = (n_slots + 3) / 4 * 4;
-    const size_t partial = ((size_t)kSearchMaxBlocks * Sp * Sp * sizeof(float) + 255) / 256 * 256;
-    long long slab = std::min<long long>(kMeanSlabBytes / ((long long)n_slots * 4), positions);
+    return ((size_t)kSearchMaxBlocks * Sp * Sp * sizeof(float) + 255) / 256 * 256;
+}
+
+size_t distance_scratch_bytes(int n_slots, long long positions) {
+    // as many positions per slot as fit half the budget, in whole mean-kernel chunks
+    long long slab = std::min<long long>(kMeanSlabBytes / 2 / ((long long)n_slots * 4), positions);
     slab = std::max<long long>((slab + kMeanChunk - 1) / kMeanChunk * kMeanChunk, kMeanChunk);
-    return partial + (size_t)n_slots * slab * sizeof(float);
+    return distance_partial_bytes(n_slots) + 2 * (size_t)n_slots * slab * sizeof(float);
 }
 
 cudaError_t launch_layer_distances(const void* pool, long long plane_bytes, const int* slot_of_layer, int L, int n_slots,
                                    int B, int Hkv, int n, int row_stride, int D, int dtype, float* scratch,
-                                   size_t scratch_bytes, float* dist, int sm_count, int* launches, cudaStream_t stream) {
+                                   size_t scratch_bytes, float* dist, int sm_count, int* launches, cudaStream_t stream,
+                                   cudaStream_t side, cudaEvent_t* ev_mean, cudaEvent_t* ev_dist) {
     if (L > kMaxLayersSearch) return cudaErrorInvalidValue;
     const int S = n_slots, Sp = (S + 3) / 4 * 4;
     const long long P = 2LL * Hkv * n * D;
-    const size_t partial_bytes = ((size_t)kSearchMaxBlocks * Sp * Sp * sizeof(float) + 255) / 256 * 256;
-    if (scratch_bytes < partial_bytes + (size_t)S * kMeanChunk * sizeof(float)) return cudaErrorInvalidValue;
-    // positions per slab: what the scratch holds, in whole mean-kernel chunks
-    long long slab = (long long)((scratch_bytes - partial_bytes) / sizeof(float) / S);
-    slab = std::min(slab / kMeanChunk * kMeanChunk, (P + kMeanChunk - 1) / kMeanChunk * kMeanChunk);
+    const size_t partial_bytes = distance_partial_bytes(S);
+    if (scratch_bytes < partial_bytes + 2 * (size_t)S * kMeanChunk * sizeof(float)) return cudaErrorInvalidValue;
+    // positions per slab: what half of the scratch holds, in whole mean-kernel chunks; slabs of equal size
+    long long slab = (long long)((scratch_bytes - partial_bytes) / 2 / sizeof(float) / S) / kMeanChunk * kMeanChunk;
+    const long long n_slabs = (P + slab - 1) / slab;
+    slab = ((P + n_slabs - 1) / n_slabs + kMeanChunk - 1) / kMeanChunk * kMeanChunk;
     float* partial = scratch;
-    float* mean = reinterpret_cast<float*>(reinterpret_cast<char*>(scratch) + partial_bytes);
+    float* mean[2];
+    mean[0] = reinterpret_cast<float*>(reinterpret_cast<char*>(scratch) + partial_bytes);
+    mean[1] = mean[0] + (size_t)S * slab;
 
     const int tiles = Sp / 4, items = tiles * (tiles + 1) / 2;
     const int groups = dist_groups(items);
@@ -335,11 +344,17 @@ cudaError_t launch_layer_distances(const void* pool, long long plane_bytes, cons
         return e;
     const int dist_blocks = (int)std::min<long long>((std::min(slab, P) + kDistChunk - 1) / kDistChunk,
                                                      std::min(2 * sm_count, kSearchMaxBlocks));
+    // The mean pass (memory-bound) runs on `stream`, the distance pass (arithmetic on data in L2) on `side`:
+    // slab k's distances are added while slab k + 1 is averaged.  Buffer k % 2 is written again only after
+    // its distance pass has finished.
     *launches = 0;
-    for (long long p0 = 0; p0 < P; p0 += slab) {
+    int k = 0;
+    for (long long p0 = 0; p0 < P; p0 += slab, ++k) {
+        const int buf = k & 1;
+        if (k >= 2 && (e = cudaStreamWaitEvent(stream, ev_dist[buf], 0)) != cudaSuccess) return e;
         MeanArgs m;
         m.pool = (const char*)pool;
-        m.mean = mean;
+        m.mean = mean[buf];
         m.plane_bytes = plane_bytes;
         m.n_slots = S; m.B = B; m.Hkv = Hkv; m.n = n; m.row_stride = row_stride; m.D = D;
         m.p0 = p0; m.p1 = std::min(P, p0 + slab); m.slab = slab;
@@ -348,19 +363,25 @@ cudaError_t launch_layer_distances(const void* pool, long long plane_bytes, cons
         if (dtype == 0) layer_mean_kernel<__nv_bfloat16><<<mean_blocks, kMeanThreads, 0, stream>>>(m);
         else layer_mean_kernel<float><<<mean_blocks, kMeanThreads, 0, stream>>>(m);
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
+        if ((e = cudaEventRecord(ev_mean[buf], stream)) != cudaSuccess) return e;
+        if ((e = cudaStreamWaitEvent(side, ev_mean[buf], 0)) != cudaSuccess) return e;
         DistArgs a;
-        a.mean = mean;
+        a.mean = mean[buf];
         a.partial = partial;
         a.S = S; a.Sp = Sp;
         a.count = m.p1 - m.p0; a.slab = slab;
         a.first = p0 == 0 ? 1 : 0;
         // the same number of blocks for every slab: block b's partial matrix is its own, slab after slab
-        mean_distance_kernel<<<dist_blocks, kDistThreads, smem, stream>>>(a);
+        // (the distance passes follow one another on `side`, so the additions keep their order)
+        mean_distance_kernel<<<dist_blocks, kDistThreads, smem, side>>>(a);
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
+        if ((e = cudaEventRecord(ev_dist[buf], side)) != cudaSuccess) return e;
         *launches += 2;
     }
-    // the slab of means is no longer needed: its first bytes hold the slot-pair sums for a moment
-    double* slot_dist2 = reinterpret_cast<double*>(mean);
+    // `stream` goes on once the last distance pass (and with it every earlier one) is done
+    if ((e = cudaStreamWaitEvent(stream, ev_dist[(k - 1) & 1], 0)) != cudaSuccess) return e;
+    // the slabs of means are no longer needed: the first bytes hold the slot-pair sums for a moment
+    double* slot_dist2 = reinterpret_cast<double*>(mean[0]);
     distance_sum_kernel<<<(S * S + 7) / 8, 256, 0, stream>>>(partial, slot_dist2, S, Sp, dist_blocks);
     if ((e = cudaGetLastError()) != cudaSuccess) return e;
     FinishArgs f;
