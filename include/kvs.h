@@ -110,6 +110,8 @@ typedef enum {
                                kvs_replay_advance).  0 (default): lengths come from the host only. */
     KVS_OPT_HOST_CHUNKS = 4,/* kvs_step_host: number of pieces (1..8, default 4) the layers are cut
                                into for overlapping the host copies with the kernels.            */
+    KVS_OPT_WAIT_LIMIT_US = 6,   /* limit of every wait inside the split-K kernels in microseconds (100 ..
+                               10 000 000, default 2 000 000); on expiry the kernel gives up, see KVS_ERR_TIMEOUT */
     KVS_OPT_FINISH_IN_KERNEL = 5 /* 1 (default): when a call has at least as many (sequence, kv-head) units as
                                thread blocks, no unit is cut into more than two pieces and the split-K
                                kernel merges them itself (the block that holds a unit's first piece reads
@@ -336,15 +338,17 @@ kvs_status kvs_step_host(kvs_ctx* ctx, const void* q_host, const void* k_host, c
  * fixed 2 MiB array inside the library image instead of the bound workspace.  The call
  * allocates nothing and frees nothing, on the device or through any library.
  *   - Every GPU that loads the library holds those 2 MiB until the process exits.
- *   - Limit: (batch * n_kv_heads + blocks launched) * group * (head_dim + 2) * 4 bytes, plus
- *     512 bytes, must fit in 2 MiB (the 7B shape at batch 8 needs 0.3 MiB, the 32q/8kv shape at
- *     batch 64 needs 1.7 MiB).  Larger calls return KVS_ERR_SCRATCH_LIMIT and launch nothing.
+ *   - Limit: (batch * n_kv_heads + blocks launched) * group * (head_dim + 2) * 4 bytes of partial
+ *     results, 4 bytes per (sequence, kv-head) of hand-over flags and 768 bytes of rounding must
+ *     fit in 2 MiB (the 7B shape at batch 8 needs 0.3 MiB, the 32q/8kv shape at batch 64 needs
+ *     1.7 MiB).  Larger calls return KVS_ERR_SCRATCH_LIMIT and launch nothing.
  *   - The device address of the array is looked up once per GPU as part of kvs_bind_memory's
  *     per-device set-up (that look-up is also when the driver places the array on the GPU, so it
  *     happens where allocating is still allowed); the call itself makes no runtime query.
  *   - All calls, from all contexts and streams, share the one array, and it keeps the previous
- *     call's contents.  The call itself clears the only part that must start at zero (the
- *     status word).  Two calls that overlap on the GPU race on the partial results: order
+ *     call's contents.  The call itself clears the status word; the hand-over flags are zero
+ *     when the library is loaded and every launch leaves them zero again; nothing else must
+ *     start at zero.  Two calls that overlap on the GPU race on the partial results: order
  *     them on one stream or with events.
  *   - The call is a plain stream-ordered launch and stays out of the context's launch
  *     bookkeeping, so it may be issued on another stream than the context's other calls, provided
@@ -374,8 +378,19 @@ kvs_status kvs_stats(const kvs_ctx* ctx, kvs_stats_t* stats);
  * 0 = no device-side problem; KVS_ERR_TIMEOUT = a bounded wait inside a kernel ran
  * out and the kernel returned early (its output is then undefined).             */
 kvs_status kvs_last_device_status(kvs_ctx* ctx, int32_t* device_status);
-/* Set the device status word back to 0 on `stream` (it is otherwise cleared only by kvs_bind_memory). */
+/* Set the device status word back to 0 on `stream` (it is otherwise cleared only by kvs_bind_memory),
+ * together with the per-unit hand-over flags a launch that gave up may have left raised: the way
+ * back to a usable context after KVS_ERR_TIMEOUT (the output of the launch that gave up is lost). */
 kvs_status kvs_clear_device_status(kvs_ctx* ctx, void* stream);
+/* Failure-detection self-test of the attention kernels themselves (the paper has no counterpart).
+ * Runs kvs_decode_attention with the same arguments, except that the producer of the thread block that
+ * owns the middle tile of the call arms that tile's barrier and then withholds its K/V copies: the wait
+ * for the tile runs out after KVS_OPT_WAIT_LIMIT_US (set it to a few milliseconds first), the block's
+ * warps hand the give-up to one another, the producer waits for the copies it did issue, other blocks
+ * that depend on this one give up in turn, and the launch ends normally with the device status word at
+ * KVS_ERR_TIMEOUT and `out` undefined.  Nothing traps or faults, every wait on the way is bounded, and
+ * kvs_clear_device_status brings the context back.  Same errors as kvs_decode_attention.               */
+kvs_status kvs_selftest_stalled_copy(kvs_ctx* ctx, int32_t layer, const void* q, float* out, int32_t batch, void* stream);
 /* Failure-detection self-test (the paper has no counterpart; every wait inside the pipelined kernels
  * is bounded, and this call shows the give-up path working on the device at hand without disturbing
  * anything).  Launches a one-warp kernel in which one thread waits, for at most limit_us

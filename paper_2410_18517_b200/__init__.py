@@ -8,7 +8,7 @@ from __future__ import annotations
 
 from . import binding
 from .binding import (  # noqa: F401
-    KVS_BF16, KVS_F32, KVS_OK, KVS_OPT_EARLY_START, KVS_OPT_FINISH_IN_KERNEL, KVS_OPT_HOST_CHUNKS, KVS_OPT_KERNEL, KVS_OPT_MAX_CTAS, KVS_OPT_REPLAY, KvsError,
+    KVS_BF16, KVS_F32, KVS_OK, KVS_OPT_EARLY_START, KVS_OPT_FINISH_IN_KERNEL, KVS_OPT_HOST_CHUNKS, KVS_OPT_KERNEL, KVS_OPT_MAX_CTAS, KVS_OPT_REPLAY, KVS_OPT_WAIT_LIMIT_US, KvsError,
 )
 
 __all__ = ["binding", "SharedKVCache", "KvsError"]

@@ -34,6 +34,7 @@ KVS_OPT_EARLY_START = 2
 KVS_OPT_REPLAY = 3
 KVS_OPT_HOST_CHUNKS = 4
 KVS_OPT_FINISH_IN_KERNEL = 5
+KVS_OPT_WAIT_LIMIT_US = 6
 
 # every symbol include/kvs.h declares
 EXPORTS = (
@@ -45,7 +46,7 @@ EXPORTS = (
     "kvs_evict", "kvs_unit_len", "kvs_layer_distances", "kvs_mean_cosine",
     "kvs_replay_advance", "kvs_replay_commit", "kvs_decode_step",
     "kvs_clear_device_status", "kvs_selftest_wait_timeout", "kvs_truncate",
-    "kvs_selftest_bounds",
+    "kvs_selftest_bounds", "kvs_selftest_stalled_copy",
 )
 
 
@@ -112,6 +113,7 @@ def load() -> ctypes.CDLL:
         "kvs_clear_device_status": [vp, vp],
         "kvs_selftest_wait_timeout": [vp, ctypes.c_uint32, P(ctypes.c_uint64), vp],
         "kvs_selftest_bounds": [vp, vp],
+        "kvs_selftest_stalled_copy": [vp, i32, vp, vp, i32, vp],
         "kvs_set_option": [vp, i32, i32],
         "kvs_last_launch": [vp, P(i32), P(i32), P(i32)],
         "kvs_read_roof": [vp, sz, vp, i32, vp],
@@ -299,6 +301,10 @@ def kvs_selftest_wait_timeout(ctx: int, limit_us: int, stream: int = 0) -> int:
 
 def kvs_selftest_bounds(ctx: int, stream: int = 0) -> None:
     _check(load().kvs_selftest_bounds(ctx, stream), "kvs_selftest_bounds")
+
+
+def kvs_selftest_stalled_copy(ctx: int, layer: int, q, out, batch: int, stream: int = 0) -> None:
+    _check(load().kvs_selftest_stalled_copy(ctx, layer, _ptr(q), _ptr(out), batch, stream), "kvs_selftest_stalled_copy")
 
 
 def kvs_set_option(ctx: int, option: int, value: int) -> None:

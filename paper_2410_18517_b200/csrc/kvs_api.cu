@@ -110,6 +110,8 @@ struct kvs_ctx {
     int opt_kernel = 0;
     int opt_pdl = 1;
     int opt_host_chunks = 4;
+    int opt_wait_us = 2000000;   // limit of the waits inside the split-K kernels, microseconds
+    long long stall_tile = -1;   // kvs_selftest_stalled_copy: tile whose copies the next attention launch withholds
     int opt_finish = 1;   // units of at most two pieces are finished by the split-K kernel itself (no combine launch)
     int opt_replay = 0;   // launches carry the device-side growth counter (for CUDA-graph replay)
     // The split-K kernels read the growth counter before their wait.  That is safe because the
@@ -345,6 +347,9 @@ kvs_status run_attention(kvs_ctx* c, int slot, const void* q, float* out, int ba
     a.v_new = v_new;
     if (k_new) a.safe_rows = std::min(a.safe_rows, a.n - 1);   // the new row is fetched after the kernel has stored it
     a.plane_bytes = (long long)c->plane_bytes;
+    a.wait_ns = 1000ull * (unsigned long long)c->opt_wait_us;
+    a.stall_tile = c->stall_tile >= 0 ? std::min<long long>(c->stall_tile, plan.T - 1) : -1;
+    c->stall_tile = -1;
     a.finish_in_kernel = c->opt_finish != 0 && kvs::can_finish_in_kernel(plan, a.units);
     a.flags = scratch.flags;
     if (scratch.tracked) {
@@ -974,9 +979,30 @@ kvs_status kvs_clear_device_status(kvs_ctx* ctx, void* stream) {
     if (!ctx->bound) return KVS_ERR_STATE;
     DeviceGuard guard(ctx->cfg.device);
     if (!guard.ok) return KVS_ERR_CUDA;
-    if (cudaMemsetAsync(ctx->ws + ctx->off_status, 0, sizeof(int), static_cast<cudaStream_t>(stream)) != cudaSuccess)
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    // a launch that gave up may have left hand-over flags raised: they go back to zero with the status word
+    if (cudaMemsetAsync(ctx->ws + ctx->off_status, 0, sizeof(int), st) != cudaSuccess ||
+        cudaMemsetAsync(ctx->ws + ctx->off_flags, 0, sizeof(int32_t) * ctx->cfg.max_batch * ctx->cfg.n_kv_heads, st) !=
+            cudaSuccess)
         return KVS_ERR_CUDA;
+    ctx->counter_written = true;   // the next launch takes a full dependency: it starts with the clears done
     return KVS_OK;
+}
+
+kvs_status kvs_selftest_stalled_copy(kvs_ctx* ctx, int32_t layer, const void* q, float* out, int32_t batch, void* stream) {
+    kvs_status s = check_attention(ctx, layer, q, out, batch);
+    if (s != KVS_OK) return s;
+    DeviceGuard guard(ctx->cfg.device);
+    if (!guard.ok) return KVS_ERR_CUDA;
+    const int slot = ctx->slot_of_layer[layer];
+    kvs::DecodePlan plan;
+    choose_plan(ctx, batch * ctx->cfg.n_kv_heads, ctx->slot_len[slot], &plan);
+    ctx->stall_tile = plan.T / 2;          // a tile in the middle of the line
+    ctx->counter_written = true;           // a plain launch, and so is whatever follows it
+    s = do_attention(ctx, layer, q, out, batch, static_cast<cudaStream_t>(stream));
+    ctx->stall_tile = -1;
+    ctx->counter_written = true;
+    return s;
 }
 
 kvs_status kvs_selftest_wait_timeout(kvs_ctx* ctx, uint32_t limit_us, uint64_t* waited_ns, void* stream) {
@@ -1033,6 +1059,10 @@ kvs_status kvs_set_option(kvs_ctx* ctx, int32_t option, int32_t value) {
         case KVS_OPT_HOST_CHUNKS:
             if (value < 1 || value > kvs_ctx::kChunks) return KVS_ERR_INVALID_ARG;
             ctx->opt_host_chunks = value;
+            return KVS_OK;
+        case KVS_OPT_WAIT_LIMIT_US:
+            if (value < 100 || value > 10000000) return KVS_ERR_INVALID_ARG;
+            ctx->opt_wait_us = value;
             return KVS_OK;
         case KVS_OPT_FINISH_IN_KERNEL:
             if (value != 0 && value != 1) return KVS_ERR_INVALID_ARG;

@@ -274,6 +274,8 @@ struct ScalarKernelArgs {
     float* out;           // [units][G][D] final results, or nullptr: every piece goes to part_o / part_ml
     int* flags;           // [units], all zero between launches: 1 = the unit's second piece is in part_o / part_ml
     long long plane_bytes;  // size of one plane (what a bounds-checking build checks tile offsets against)
+    unsigned long long wait_ns;   // limit of every wait inside the kernel
+    long long stall_tile;         // self-test only: the K/V copies of this tile are withheld (-1: none)
 };
 
 template <typename T, int D, int G, int GEOM>
@@ -350,7 +352,7 @@ __global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G, GEOM>::MI
                     if (total) mbar_arrive_expect_tx(&full_bar[st], total);
                     else mbar_arrive(&full_bar[st]);
                 }
-                if (kv && bytes) {
+                if (kv && bytes && gt != a.stall_tile) {
                     long long off = (u * a.row_stride + row0) * (long long)RB;
                     if (!KVS_BOUNDS_OK(off, bytes, a.plane_bytes, a.status) || !KVS_BOUNDS_OK(u, 1, a.units, a.status)) off = 0;
                     bulk_g2s(sb, a.kplane + off, bytes, &full_bar[st]);
@@ -389,7 +391,7 @@ __global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G, GEOM>::MI
             bool ok = true;
             for (long long gt = t0 + npre; gt < t1 && ok; ++gt, ++it) {
                 const int st = it % STAGES;
-                if (it >= STAGES) ok = mbar_wait_bounded(&empty_bar[st], ((it / STAGES) - 1) & 1, abort_flag, a.status);
+                if (it >= STAGES) ok = mbar_wait_bounded(&empty_bar[st], ((it / STAGES) - 1) & 1, abort_flag, a.status, a.wait_ns);
                 if (!ok) break;
                 issue(gt, st, true, true, true);
             }
@@ -397,7 +399,7 @@ __global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G, GEOM>::MI
                 // Gave up: still wait (bounded) for copies already issued, so that none
                 // is in flight into this block's shared memory when it exits.
                 for (int j = max(0, it - STAGES); j < it; ++j)
-                    mbar_wait_bounded(&full_bar[j % STAGES], (j / STAGES) & 1, abort_flag + 1, a.status);
+                    mbar_wait_bounded(&full_bar[j % STAGES], (j / STAGES) & 1, abort_flag + 1, a.status, a.wait_ns);
             }
         }
         return;
@@ -414,13 +416,13 @@ __global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G, GEOM>::MI
         if (!has_tail && !has_head) return;
         pdl_wait();   // the flags are back to zero only once the previous launch has completed
         if (has_tail) {
-            if (!mbar_wait_bounded(tail_bar, 0, abort_flag, a.status)) return;
+            if (!mbar_wait_bounded(tail_bar, 0, abort_flag, a.status, a.wait_ns)) return;
             if (lane == 0) st_release_gpu(a.flags + t0 / a.tpu, 1);
         }
         if (has_head) {
             const long long u = (t1 - 1) / a.tpu;
             int ok = 1;
-            if (lane == 0) ok = flag_wait_bounded(a.flags + u, 1, abort_flag, a.status) ? 1 : 0;
+            if (lane == 0) ok = flag_wait_bounded(a.flags + u, 1, abort_flag, a.status, a.wait_ns) ? 1 : 0;
             ok = __shfl_sync(0xffffffffu, ok, 0);
             if (!ok) return;
             // written by another SM during this launch: read past L1
@@ -463,7 +465,7 @@ __global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G, GEOM>::MI
 
         for (int k = 0; k < piece_tiles; ++k, ++it) {
             const int st = it % STAGES;
-            if (!mbar_wait_bounded(&full_bar[st], (it / STAGES) & 1, abort_flag, a.status)) return;
+            if (!mbar_wait_bounded(&full_bar[st], (it / STAGES) & 1, abort_flag, a.status, a.wait_ns)) return;
             const unsigned char* ks = stage_base + st * S::STAGE_BYTES;
             const unsigned char* vs = ks + kTile;
             if (k == 0) {
@@ -575,7 +577,7 @@ __global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G, GEOM>::MI
         const bool whole = finish && ti0 == 0 && piece_tiles == a.tpu;
         const bool head = finish && ti0 == 0 && piece_tiles < a.tpu;
         const bool tail = finish && ti0 > 0;
-        if (head && !mbar_wait_bounded(head_bar, 0, abort_flag, a.status)) return;
+        if (head && !mbar_wait_bounded(head_bar, 0, abort_flag, a.status, a.wait_ns)) return;
 #pragma unroll
         for (int g = 0; g < G; ++g) {
             // lanes with equal top bits hold duplicates of lsum; add across the R distinct ones
@@ -636,11 +638,10 @@ __global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G, GEOM>::MI
 // call, which may only start once every block of this grid has started, can move onto each SM
 // the moment the running split-K block leaves it.
 // --------------------------------------------------------------------------------------
-// Two builds: units of at most two pieces (every block's share is at least a unit long) take eight
-// items per block with two vectors requested early; longer units take four items per block and
-// four early vectors (64 registers), so that a unit of up to four pieces still needs one round trip.
+// This build serves calls whose units have at most two pieces (every block's share is at least a
+// unit long): eight items per block, two vectors requested early.  Longer units: decode_combine_long_kernel.
 template <int D, int PRE, int kCombineWarps>
-__global__ void __launch_bounds__(kCombineWarps * 32, PRE == 2 ? 5 : 8)
+__global__ void __launch_bounds__(kCombineWarps * 32, 5)
     decode_combine_kernel(const float* __restrict__ part_o, const float* __restrict__ part_ml, float* __restrict__ out,
                           int G, int tpu, long long T, int NC, const int* __restrict__ n_extra, int n, int tile_rows,
                           int units, int cap, int* status) {
@@ -714,11 +715,121 @@ __global__ void __launch_bounds__(kCombineWarps * 32, PRE == 2 ? 5 : 8)
     reinterpret_cast<Vec*>(out + (u * G + g) * D)[lane] = r;
 }
 
-template <int D, int PRE, int WARPS>
-static cudaError_t launch_combine_one(const DecodeArgs& a, const DecodePlan& plan, cudaStream_t stream) {
+// Units of three or more pieces (fewer units than blocks): one BLOCK of four warps per (unit, q-head).
+// Warp w takes pieces w, w + 4, ...: with up to four pieces per warp in flight a unit of 16 pieces needs
+// one round trip for the (max, sum) pairs and one for the vectors (the first of which is requested
+// together with the pairs).  The warps' sums are added in warp order by warp 0: a fixed order.
+constexpr int kLongWarps = 4;
+
+template <int D>
+__global__ void __launch_bounds__(kLongWarps * 32, 8)
+    decode_combine_long_kernel(const float* __restrict__ part_o, const float* __restrict__ part_ml, float* __restrict__ out,
+                               int G, int tpu, long long T, int NC, const int* __restrict__ n_extra, int n, int tile_rows,
+                               int units, int cap, int* status) {
+    constexpr int VEC = D / 32;
+    struct __align__(VEC * 4) Vec {
+        float v[VEC];
+    };
+    __shared__ float s_max[kLongWarps], s_den[kLongWarps];
+    __shared__ float s_acc[kLongWarps][D];
+    pdl_launch_dependents();
+    pdl_wait();
+    if (n_extra) {   // replayed launch: recompute the tile line from the grown length
+        tpu = (min(n + *n_extra, cap) + tile_rows - 1) / tile_rows;
+        T = (long long)units * tpu;
+    }
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const long long u = blockIdx.x / G;
+    const int g = blockIdx.x - (int)u * G;
+    const int c0 = cta_of_tile(u * tpu, T, NC);
+    int np = cta_of_tile((u + 1) * tpu - 1, T, NC) - c0 + 1;             // pieces of this unit
+#ifdef KVS_DEBUG_BOUNDS
+    if (!KVS_BOUNDS_OK(u + c0, np, (long long)units + NC, status)) np = 1;
+#endif
+    const float2* ml = reinterpret_cast<const float2*>(part_ml) + (u + c0) * G + g;   // piece c: ml[c * G]
+    const Vec* po = reinterpret_cast<const Vec*>(part_o + ((u + c0) * G + g) * D) + lane;   // piece c: po[c * G * 32]
+    const int pstride = G * 32;
+    const int mine = np > warp ? (np - warp + kLongWarps - 1) / kLongWarps : 0;       // pieces warp, warp + 4, ... of this warp
+    // this warp's first 32 pairs and, in the same round trip, its first four vectors
+    constexpr int PRE = 4;
+    const float2 v0 = lane < mine ? ml[(warp + kLongWarps * lane) * G] : make_float2(-1.0e30f, 0.f);
+    Vec pre[PRE];
+#pragma unroll
+    for (int j = 0; j < PRE; ++j)
+        if (j < mine) pre[j] = po[(warp + kLongWarps * j) * pstride];
+    float M = v0.x;
+    for (int jb = 32; jb < mine; jb += 32)
+        if (jb + lane < mine) M = fmaxf(M, ml[(warp + kLongWarps * (jb + lane)) * G].x);
+#pragma unroll
+    for (int o = 16; o >= 1; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+    if (lane == 0) s_max[warp] = M;
+    __syncthreads();
+    M = fmaxf(fmaxf(s_max[0], s_max[1]), fmaxf(s_max[2], s_max[3]));
+    float acc[VEC];
+#pragma unroll
+    for (int e = 0; e < VEC; ++e) acc[e] = 0.f;
+    float den = 0.f;
+    for (int jb = 0; jb < mine; jb += 32) {
+        const float2 v = jb == 0 ? v0 : (jb + lane < mine ? ml[(warp + kLongWarps * (jb + lane)) * G] : make_float2(-1.0e30f, 0.f));
+        const float w = jb + lane < mine ? fast_exp2(v.x - M) : 0.f;
+        den = fmaf(w, v.y, den);
+        const int cnt = min(32, mine - jb);
+        int j = 0;
+        if (jb == 0) {
+#pragma unroll
+            for (int t = 0; t < PRE; ++t)
+                if (t < cnt) {
+                    const float wj = __shfl_sync(0xffffffffu, w, t);
+#pragma unroll
+                    for (int e = 0; e < VEC; ++e) acc[e] = fmaf(wj, pre[t].v[e], acc[e]);
+                }
+            j = min(PRE, cnt);
+        }
+#pragma unroll 4
+        for (; j < cnt; ++j) {
+            const float wj = __shfl_sync(0xffffffffu, w, j);
+            const Vec x = po[(warp + kLongWarps * (jb + j)) * pstride];
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) acc[e] = fmaf(wj, x.v[e], acc[e]);
+        }
+    }
+#pragma unroll
+    for (int o = 16; o >= 1; o >>= 1) den += __shfl_xor_sync(0xffffffffu, den, o);
+    if (lane == 0) s_den[warp] = den;
+#pragma unroll
+    for (int e = 0; e < VEC; ++e) s_acc[warp][lane * VEC + e] = acc[e];
+    __syncthreads();
+    if (warp == 0) {
+        float d = 0.f;
+        Vec r;
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) r.v[e] = 0.f;
+#pragma unroll
+        for (int wq = 0; wq < kLongWarps; ++wq) {
+            d += s_den[wq];
+#pragma unroll
+            for (int e = 0; e < VEC; ++e) r.v[e] += s_acc[wq][lane * VEC + e];
+        }
+#pragma unroll
+        for (int e = 0; e < VEC; ++e) r.v[e] /= d;
+        reinterpret_cast<Vec*>(out + (u * G + g) * D)[lane] = r;
+    }
+}
+
+template <int D>
+static cudaError_t launch_combine_short(const DecodeArgs& a, const DecodePlan& plan, cudaStream_t stream) {
+    constexpr int WARPS = 8;
     const long long items = (long long)a.units * a.G;
     const dim3 grid((unsigned)((items + WARPS - 1) / WARPS)), block(WARPS * 32);
-    return launch_kernel(decode_combine_kernel<D, PRE, WARPS>, grid, block, 0, stream, a.programmatic, (const float*)a.part_o,
+    return launch_kernel(decode_combine_kernel<D, 2, WARPS>, grid, block, 0, stream, a.programmatic, (const float*)a.part_o,
+                         (const float*)a.part_ml, a.out, a.G, plan.tpu, plan.T, plan.NC, a.n_extra, a.n, plan.tile_rows,
+                         a.units, a.capacity, a.status);
+}
+
+template <int D>
+static cudaError_t launch_combine_long(const DecodeArgs& a, const DecodePlan& plan, cudaStream_t stream) {
+    const dim3 grid((unsigned)(a.units * a.G)), block(kLongWarps * 32);
+    return launch_kernel(decode_combine_long_kernel<D>, grid, block, 0, stream, a.programmatic, (const float*)a.part_o,
                          (const float*)a.part_ml, a.out, a.G, plan.tpu, plan.T, plan.NC, a.n_extra, a.n, plan.tile_rows,
                          a.units, a.capacity, a.status);
 }
@@ -727,9 +838,8 @@ cudaError_t launch_combine(const DecodeArgs& a, const DecodePlan& plan, cudaStre
     // a unit has at most two pieces when no block's share is shorter than a unit, i.e. when there are
     // at least as many units as blocks (whatever the length, also one that grows under graph replay)
     const bool short_units = a.units >= plan.NC;
-    if (a.D == 128)
-        return short_units ? launch_combine_one<128, 2, 8>(a, plan, stream) : launch_combine_one<128, 4, 4>(a, plan, stream);
-    return short_units ? launch_combine_one<64, 2, 8>(a, plan, stream) : launch_combine_one<64, 4, 4>(a, plan, stream);
+    if (a.D == 128) return short_units ? launch_combine_short<128>(a, plan, stream) : launch_combine_long<128>(a, plan, stream);
+    return short_units ? launch_combine_short<64>(a, plan, stream) : launch_combine_long<64>(a, plan, stream);
 }
 
 // --------------------------------------------------------------------------------------
@@ -813,6 +923,8 @@ cudaError_t launch_decode_scalar(const DecodeArgs& a, const DecodePlan& plan, cu
     ka.out = a.finish_in_kernel ? a.out : nullptr;
     ka.flags = a.flags;
     ka.plane_bytes = a.plane_bytes;
+    ka.wait_ns = a.wait_ns;
+    ka.stall_tile = a.stall_tile;
     const bool pdl = a.programmatic;
     if (a.dtype == 0) {
         if (a.D == 128) return launch_scalar_groups<__nv_bfloat16, 128>(a.G, plan.geom, ka, plan.NC, pdl, stream);

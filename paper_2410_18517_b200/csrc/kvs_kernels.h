@@ -48,6 +48,8 @@ struct DecodeArgs {
     bool finish_in_kernel;
     int* flags;
     long long plane_bytes;   // size of one plane: what a bounds-checking build checks tile offsets against
+    unsigned long long wait_ns;   // limit of every wait inside the split-K kernels
+    long long stall_tile;    // self-test only: the K/V copies of this tile of the line are withheld (-1: none)
 };
 
 // Whether a launch of this plan over `units` units can finish inside the split-K kernel.

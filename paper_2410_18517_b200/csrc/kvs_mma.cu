@@ -120,6 +120,8 @@ struct MmaKernelArgs {
     float* out;          // [units][G][D] final results, or nullptr: every piece goes to part_o / part_ml
     int* flags;          // [units], all zero between launches: 1 = the unit's second piece is in part_o / part_ml
     long long plane_rows;   // rows of one plane (what a bounds-checking build checks tile rows against)
+    unsigned long long wait_ns;   // limit of every wait inside the kernel
+    long long stall_tile;         // self-test only: the K/V copies of this tile are withheld (-1: none)
 };
 
 // G (q-heads per kv-head, 1..8) is a run-time argument: it only selects which rows of the padded
@@ -195,7 +197,7 @@ __global__ void __launch_bounds__(kMmaThreads, KVS_MMA_BLOCKS_PER_SM)
                     if (total) mbar_arrive_expect_tx(&full_bar[st], total);
                     else mbar_arrive(&full_bar[st]);
                 }
-                if (kv && rows > 0) {
+                if (kv && rows > 0 && gt != a.stall_tile) {
                     long long row = u * a.row_stride + (long long)ti * TN;
                     // (a whole box is fetched even where the unit has fewer rows: it stays inside the unit's row_stride)
                     if (!KVS_BOUNDS_OK(row, rows == TN ? TN : tail_boxes * kTailRows, a.plane_rows, a.status) ||
@@ -255,13 +257,13 @@ __global__ void __launch_bounds__(kMmaThreads, KVS_MMA_BLOCKS_PER_SM)
             for (long long gt = t0 + npre; gt < t1; ++gt, ++it) {
                 const int st = it % kMmaStages;
                 if (it >= kMmaStages)
-                    ok = mbar_wait_bounded(&empty_bar[st], ((it / kMmaStages) - 1) & 1, abort_flag, a.status);
+                    ok = mbar_wait_bounded(&empty_bar[st], ((it / kMmaStages) - 1) & 1, abort_flag, a.status, a.wait_ns);
                 if (!ok) break;
                 issue(gt, st, true, true, true);
             }
             if (!ok) {
                 for (int j = max(0, it - kMmaStages); j < it; ++j)
-                    mbar_wait_bounded(&full_bar[j % kMmaStages], (j / kMmaStages) & 1, abort_flag + 1, a.status);
+                    mbar_wait_bounded(&full_bar[j % kMmaStages], (j / kMmaStages) & 1, abort_flag + 1, a.status, a.wait_ns);
             }
         }
         return;
@@ -278,13 +280,13 @@ __global__ void __launch_bounds__(kMmaThreads, KVS_MMA_BLOCKS_PER_SM)
         if (!has_tail && !has_head) return;
         pdl_wait();   // the flags are back to zero only once the previous launch has completed
         if (has_tail) {
-            if (!mbar_wait_bounded(tail_bar, 0, abort_flag, a.status)) return;
+            if (!mbar_wait_bounded(tail_bar, 0, abort_flag, a.status, a.wait_ns)) return;
             if (lane == 0) st_release_gpu(a.flags + t0 / a.tpu, 1);
         }
         if (has_head) {
             const long long u = (t1 - 1) / a.tpu;
             int ok = 1;
-            if (lane == 0) ok = flag_wait_bounded(a.flags + u, 1, abort_flag, a.status) ? 1 : 0;
+            if (lane == 0) ok = flag_wait_bounded(a.flags + u, 1, abort_flag, a.status, a.wait_ns) ? 1 : 0;
             ok = __shfl_sync(0xffffffffu, ok, 0);
             if (!ok) return;
             // written by another SM during this launch: read past L1
@@ -322,7 +324,7 @@ __global__ void __launch_bounds__(kMmaThreads, KVS_MMA_BLOCKS_PER_SM)
 
         for (int k = 0; k < piece_tiles; ++k, ++it) {
             const int st = it % kMmaStages;
-            if (!mbar_wait_bounded(&full_bar[st], (it / kMmaStages) & 1, abort_flag, a.status)) return;
+            if (!mbar_wait_bounded(&full_bar[st], (it / kMmaStages) & 1, abort_flag, a.status, a.wait_ns)) return;
             const unsigned char* ks = smem + st * S::STAGE_BYTES;
             const uint32_t ks_u32 = smem_u32(ks);
             const uint32_t vs_u32 = ks_u32 + kMmaTileBytes;
@@ -477,7 +479,7 @@ __global__ void __launch_bounds__(kMmaThreads, KVS_MMA_BLOCKS_PER_SM)
                 dst[D + 1] = l;
             }
         }
-        if (head && !mbar_wait_bounded(head_bar, 0, abort_flag, a.status)) return;
+        if (head && !mbar_wait_bounded(head_bar, 0, abort_flag, a.status, a.wait_ns)) return;
         named_bar_sync(1, kMmaConsumerThreads);
         for (int idx = tid; idx < G * D; idx += kMmaConsumerThreads) {
             const int g = idx / D, d = idx - g * D;
@@ -604,6 +606,8 @@ cudaError_t launch_decode_mma(const DecodeArgs& a, const DecodePlan& plan, const
     ka.out = a.finish_in_kernel ? a.out : nullptr;
     ka.flags = a.flags;
     ka.plane_rows = a.plane_bytes / (a.D * 2);
+    ka.wait_ns = a.wait_ns;
+    ka.stall_tile = a.stall_tile;
     if (a.G < 1 || a.G > 8) return cudaErrorInvalidValue;
     if (a.D == 128) return launch_one<128>(tm, tm_tail, ka, plan.NC, a.programmatic, stream);
     if (a.D == 64) return launch_one<64>(tm, tm_tail, ka, plan.NC, a.programmatic, stream);

@@ -78,3 +78,46 @@ def test_bounds_self_test_is_refused_by_the_normal_build():
     with pytest.raises(KvsError) as e:
         kb.kvs_selftest_bounds(cache.ctx)
     assert e.value.status == kb.KVS_ERR_STATE and cache.device_status() == 0
+
+
+@pytest.mark.parametrize("Hq,Hkv,B,dtype,context", [(8, 8, 4, "bf16", 3000),      # scalar kernel, units < blocks: combine follows
+                                                    (8, 8, 40, "bf16", 700),      # scalar kernel finishes the units itself
+                                                    (16, 4, 2, "bf16", 9000),     # tensor-core kernel, combine follows
+                                                    (16, 4, 64, "bf16", 500),     # tensor-core kernel finishes the units itself
+                                                    (4, 4, 3, "f32", 2000)])
+def test_a_withheld_copy_makes_the_attention_kernel_give_up_and_the_context_recovers(Hq, Hkv, B, dtype, context):
+    """The give-up path of the real split-K kernels: one block's producer arms a tile's barrier and withholds
+    the copies.  The consumers' wait runs out (2 ms), they hand the give-up to the producer, which waits for
+    the copies it did issue; blocks that depend on the stalled one give up as well; the launch ends, the
+    status word says TIMEOUT, and after kvs_clear_device_status the next call matches the oracle."""
+    from paper_2410_18517_b200 import KVS_OPT_WAIT_LIMIT_US
+
+    w = si.Workload(f"stall_{Hq}_{Hkv}_{B}_{dtype}", L=2, Hq=Hq, Hkv=Hkv, D=128, B=B, context=context, dtype=dtype,
+                    n_shared=1, map_seed=0, steps=1, fixed_map=(0, 0))
+    cache = SharedKVCache(w.L, w.Hq, w.Hkv, w.D, w.B, w.context + 4, w.dtype, share_map=w.share_map())
+    k, v = si.context_kv(w, 0)
+    cache.append(0, k.cuda(), v.cuda())
+    q = si.step_qkv(w, 0, 1)[0]
+    good = cache.decode_attention(1, q.cuda()).clone()
+    cache.set_option(KVS_OPT_WAIT_LIMIT_US, 2000)
+    out = torch.zeros_like(good)
+    t0 = torch.cuda.Event(enable_timing=True)
+    t1 = torch.cuda.Event(enable_timing=True)
+    t0.record()
+    kb.kvs_selftest_stalled_copy(cache.ctx, 1, q.cuda(), out, w.B, torch.cuda.current_stream().cuda_stream)
+    t1.record()
+    torch.cuda.synchronize()
+    assert cache.device_status() == kb.KVS_ERR_TIMEOUT
+    assert 1.5 <= t0.elapsed_time(t1) <= 50.0          # it gave up after about the limit, not after seconds
+    cache.clear_device_status()
+    assert cache.device_status() == 0
+    cache.set_option(KVS_OPT_WAIT_LIMIT_US, 2000000)
+    again = cache.decode_attention(1, q.cuda())
+    assert torch.equal(again, good)                      # the context works as before
+    K, V = k.double().numpy(), v.double().numpy()
+    rng = np.random.default_rng(0)
+    for _ in range(6):
+        b, hq = int(rng.integers(w.B)), int(rng.integers(w.Hq))
+        ref = oracle.attend_unit(q[b, hq].double().numpy(), K[b, :, hq // w.G], V[b, :, hq // w.G])
+        assert_close(again[b, hq].cpu().numpy(), ref, f"after the stalled launch, unit {(b, hq)}")
+    assert cache.device_status() == 0
