@@ -424,6 +424,7 @@ __global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G, GEOM>::MI
             int ok = 1;
             if (lane == 0) ok = flag_wait_bounded(a.flags + u, 1, abort_flag, a.status, a.wait_ns) ? 1 : 0;
             ok = __shfl_sync(0xffffffffu, ok, 0);
+            __syncwarp();    // lane 0's acquire comes before every lane's loads of the piece
             if (!ok) return;
             // written by another SM during this launch: read past L1
             const long long pt = u + blockIdx.x + 1;
