@@ -401,6 +401,18 @@ kvs_status kvs_selftest_stalled_copy(kvs_ctx* ctx, int32_t layer, const void* q,
  * the GPU.  Afterwards kvs_last_device_status reports KVS_ERR_TIMEOUT until kvs_clear_device_status.
  * Errors: STATE before kvs_bind_memory; INVALID_ARG for a limit out of range.                      */
 kvs_status kvs_selftest_wait_timeout(kvs_ctx* ctx, uint32_t limit_us, uint64_t* waited_ns, void* stream);
+/* Per-block timeline of the attention kernels (the paper has no counterpart; the library compiled with
+ * -DKVS_TRACE only, STATE otherwise).  Between kvs_trace_begin and kvs_trace_end every attention call of the
+ * context (kvs_decode_attention, kvs_decode_step, ...) writes 160 rows of 32 uint64 words to `buffer` (device,
+ * 8-byte aligned, caller-owned), call after call, until `bytes` are used up: row b < 148 holds the GPU's
+ * nanosecond timer as thread block b of the split-K kernel saw it at entry [0], when its producer's / its
+ * consumers' wait for the previous kernel returned [1] / [2], when the first tile had arrived [3], when the
+ * tiles of its k-th piece were done [4 + 2k] and the piece was merged and written [5 + 2k] (k < 8), when the
+ * consumers ended [20], the number of pieces [21], and when the producer began to wait [22]; rows 150 and
+ * 151 hold entry [0], end of wait [1] and end [2] of the first and the last block of the combine kernel
+ * (zero when the call launched none).  kvs_trace_end stops the recording and reports the calls recorded.   */
+kvs_status kvs_trace_begin(kvs_ctx* ctx, void* buffer, size_t bytes);
+kvs_status kvs_trace_end(kvs_ctx* ctx, int32_t* launches_recorded);
 /* Self-test of the bounds-checking build (the library compiled with -DKVS_DEBUG_BOUNDS, in which every
  * global offset the kernels compute is checked against the buffer it must fall in; the paper has no
  * counterpart).  Launches one kernel that hands the check an offset outside its buffer WITHOUT touching

@@ -46,7 +46,7 @@ EXPORTS = (
     "kvs_evict", "kvs_unit_len", "kvs_layer_distances", "kvs_mean_cosine",
     "kvs_replay_advance", "kvs_replay_commit", "kvs_decode_step",
     "kvs_clear_device_status", "kvs_selftest_wait_timeout", "kvs_truncate",
-    "kvs_selftest_bounds", "kvs_selftest_stalled_copy",
+    "kvs_selftest_bounds", "kvs_selftest_stalled_copy", "kvs_trace_begin", "kvs_trace_end",
 )
 
 
@@ -113,6 +113,8 @@ def load() -> ctypes.CDLL:
         "kvs_clear_device_status": [vp, vp],
         "kvs_selftest_wait_timeout": [vp, ctypes.c_uint32, P(ctypes.c_uint64), vp],
         "kvs_selftest_bounds": [vp, vp],
+        "kvs_trace_begin": [vp, vp, sz],
+        "kvs_trace_end": [vp, P(i32)],
         "kvs_selftest_stalled_copy": [vp, i32, vp, vp, i32, vp],
         "kvs_set_option": [vp, i32, i32],
         "kvs_last_launch": [vp, P(i32), P(i32), P(i32)],
@@ -297,6 +299,17 @@ def kvs_selftest_wait_timeout(ctx: int, limit_us: int, stream: int = 0) -> int:
     w = ctypes.c_uint64()
     _check(load().kvs_selftest_wait_timeout(ctx, limit_us, ctypes.byref(w), stream), "kvs_selftest_wait_timeout")
     return w.value
+
+
+def kvs_trace_begin(ctx: int, buffer, nbytes: int) -> None:
+    _check(load().kvs_trace_begin(ctx, _ptr(buffer), nbytes), "kvs_trace_begin")
+
+
+def kvs_trace_end(ctx: int) -> int:
+    """Stops the recording; returns the number of attention calls recorded."""
+    n = ctypes.c_int32()
+    _check(load().kvs_trace_end(ctx, ctypes.byref(n)), "kvs_trace_end")
+    return n.value
 
 
 def kvs_selftest_bounds(ctx: int, stream: int = 0) -> None:

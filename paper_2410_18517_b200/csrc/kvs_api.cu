@@ -110,6 +110,9 @@ struct kvs_ctx {
     int opt_kernel = 0;
     int opt_pdl = 1;
     int opt_host_chunks = 4;
+    // tracing build: where the next attention launch stamps its timeline (kvs_trace_begin / kvs_trace_end)
+    unsigned long long* trace_buf = nullptr;
+    int trace_capacity = 0, trace_launch = 0;
     int opt_wait_us = 2000000;   // limit of the waits inside the split-K kernels, microseconds
     long long stall_tile = -1;   // kvs_selftest_stalled_copy: tile whose copies the next attention launch withholds
     int opt_finish = 1;   // units of at most two pieces are finished by the split-K kernel itself (no combine launch)
@@ -348,6 +351,9 @@ kvs_status run_attention(kvs_ctx* c, int slot, const void* q, float* out, int ba
     if (k_new) a.safe_rows = std::min(a.safe_rows, a.n - 1);   // the new row is fetched after the kernel has stored it
     a.plane_bytes = (long long)c->plane_bytes;
     a.wait_ns = 1000ull * (unsigned long long)c->opt_wait_us;
+    a.trace = nullptr;
+    if (c->trace_buf && c->trace_launch < c->trace_capacity)
+        a.trace = c->trace_buf + (size_t)(c->trace_launch++) * kvs::kTraceLaunchWords;
     a.stall_tile = c->stall_tile >= 0 ? std::min<long long>(c->stall_tile, plan.T - 1) : -1;
     c->stall_tile = -1;
     a.finish_in_kernel = c->opt_finish != 0 && kvs::can_finish_in_kernel(plan, a.units);
@@ -1024,6 +1030,25 @@ kvs_status kvs_selftest_wait_timeout(kvs_ctx* ctx, uint32_t limit_us, uint64_t* 
         cudaStreamSynchronize(st) != cudaSuccess)
         return KVS_ERR_CUDA;
     if (waited_ns) *waited_ns = w;
+    return KVS_OK;
+}
+
+kvs_status kvs_trace_begin(kvs_ctx* ctx, void* buffer, size_t bytes) {
+    if (!ctx || !buffer || ((uintptr_t)buffer % 8) != 0) return KVS_ERR_INVALID_ARG;
+    if (!ctx->bound || !kvs::is_tracing_build()) return KVS_ERR_STATE;
+    const size_t per_launch = (size_t)kvs::kTraceLaunchWords * sizeof(unsigned long long);
+    if (bytes < per_launch) return KVS_ERR_INVALID_ARG;
+    ctx->trace_buf = static_cast<unsigned long long*>(buffer);
+    ctx->trace_capacity = (int)std::min<size_t>(bytes / per_launch, 1 << 20);
+    ctx->trace_launch = 0;
+    return KVS_OK;
+}
+
+kvs_status kvs_trace_end(kvs_ctx* ctx, int32_t* launches_recorded) {
+    if (!ctx) return KVS_ERR_INVALID_ARG;
+    if (launches_recorded) *launches_recorded = ctx->trace_launch;
+    ctx->trace_buf = nullptr;
+    ctx->trace_capacity = ctx->trace_launch = 0;
     return KVS_OK;
 }
 

@@ -12,6 +12,30 @@ constexpr int kDevOk = 0;
 constexpr int kDevTimeout = 7;
 constexpr int kDevBounds = 9;
 
+// Tracing build (-DKVS_TRACE): the split-K and combine kernels stamp %globaltimer into a caller-provided
+// buffer at fixed points (one row of kTraceSlots words per thread block and launch), from which the
+// per-block timeline of a launch can be read.  In a normal build the stamps compile to nothing.
+constexpr int kTraceSlots = 32;     // words per (launch, block)
+constexpr int kTraceBlocks = 160;   // rows per launch: blocks 0..147 of the split-K kernel, rows 150 / 151 the
+                                    // first / last block of the combine kernel
+enum TraceSlot {
+    kTrEntry = 0,          // kernel entry (thread 0)
+    kTrProducerGo = 1,     // producer: its wait for the previous kernel has returned
+    kTrConsumerGo = 2,     // consumers: their wait has returned
+    kTrFirstTile = 3,      // the first tile (with q) has arrived
+    kTrPiece = 4,          // 4 + 2k: piece k's tiles are done, 5 + 2k: piece k is merged and written (k < 8)
+    kTrEnd = 20,           // consumers are done
+    kTrPieces = 21,        // number of pieces of the block
+    kTrProducerPre = 22,   // producer: early tiles issued, about to wait
+};
+#ifdef KVS_TRACE
+#define KVS_TRACE_STAMP(row, slot) do { if ((row) != nullptr) (row)[slot] = ::kvs::globaltimer_ns(); } while (0)
+#define KVS_TRACE_VALUE(row, slot, v) do { if ((row) != nullptr) (row)[slot] = (unsigned long long)(v); } while (0)
+#else
+#define KVS_TRACE_STAMP(row, slot) do { (void)(row); } while (0)
+#define KVS_TRACE_VALUE(row, slot, v) do { (void)(row); (void)(v); } while (0)
+#endif
+
 // Bounds-checking build (-DKVS_DEBUG_BOUNDS): every global offset the kernels compute for a pool
 // plane, the query / new-row buffers or the partial results is checked against the buffer it
 // must fall in.  The first violation is recorded in the status word (kDevBounds; nothing traps)

@@ -276,6 +276,7 @@ struct ScalarKernelArgs {
     long long plane_bytes;  // size of one plane (what a bounds-checking build checks tile offsets against)
     unsigned long long wait_ns;   // limit of every wait inside the kernel
     long long stall_tile;         // self-test only: the K/V copies of this tile are withheld (-1: none)
+    unsigned long long* trace;    // tracing build: this launch's rows of time stamps, or nullptr
 };
 
 template <typename T, int D, int G, int GEOM>
@@ -283,6 +284,8 @@ __global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G, GEOM>::MI
     decode_splitk_scalar(const ScalarKernelArgs a_in) {
     using S = ScalarShape<T, D, G, GEOM>;
     ScalarKernelArgs a = a_in;
+    unsigned long long* tr = a.trace ? a.trace + (size_t)blockIdx.x * kTraceSlots : nullptr;
+    if (threadIdx.x == 0) KVS_TRACE_STAMP(tr, kTrEntry);
     bool over = false;    // a replayed launch with an append that would pass the capacity
     if (a.n_extra != nullptr) {
         // A replayed launch: the lengths recorded with it have grown on the device since.  The
@@ -374,7 +377,9 @@ __global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G, GEOM>::MI
                     issue(gt, npre, true, true, false);
                 }
             }
+            if (lane == 0) KVS_TRACE_STAMP(tr, kTrProducerPre);
             pdl_wait();
+            if (lane == 0) KVS_TRACE_STAMP(tr, kTrProducerGo);
             pdl_launch_dependents();
             // first the queries of the tiles already fetched (the consumers wait for nothing else), then the new rows
             if (lane == 0)
@@ -441,7 +446,9 @@ __global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G, GEOM>::MI
 
     // ---------------------------------- consumers ----------------------------------
     pdl_wait();               // partial results of the previous call may still be read until here
+    if (tid == 0) KVS_TRACE_STAMP(tr, kTrConsumerGo);
     pdl_launch_dependents();
+    int trace_piece = 0;
     const int lig = lane & (LPR - 1);                 // lane within its row group
     const int grp = warp * S::GPW + lane / LPR;       // row group within the block
     const int my_i = lig >> SH;                       // row (of the R) whose score this lane ends up holding
@@ -467,6 +474,7 @@ __global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G, GEOM>::MI
         for (int k = 0; k < piece_tiles; ++k, ++it) {
             const int st = it % STAGES;
             if (!mbar_wait_bounded(&full_bar[st], (it / STAGES) & 1, abort_flag, a.status, a.wait_ns)) return;
+            if (tid == 0 && it == 0) KVS_TRACE_STAMP(tr, kTrFirstTile);
             const unsigned char* ks = stage_base + st * S::STAGE_BYTES;
             const unsigned char* vs = ks + kTile;
             if (k == 0) {
@@ -574,6 +582,7 @@ __global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G, GEOM>::MI
         // first piece comes to it LAST, by when its hand-over warp has fetched the second piece into
         // shared memory; it merges the two in piece order and writes the result.
         const long long pid = u + blockIdx.x;
+        if (tid == 0 && trace_piece < 8) KVS_TRACE_STAMP(tr, kTrPiece + 2 * trace_piece);
         const bool finish = a.out != nullptr;
         const bool whole = finish && ti0 == 0 && piece_tiles == a.tpu;
         const bool head = finish && ti0 == 0 && piece_tiles < a.tpu;
@@ -622,7 +631,13 @@ __global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G, GEOM>::MI
             }
         }
         if (tail) mbar_arrive(tail_bar);   // this thread's part of the piece is written
+        if (tid == 0 && trace_piece < 8) KVS_TRACE_STAMP(tr, kTrPiece + 2 * trace_piece + 1);
+        ++trace_piece;
         gt += piece_tiles;
+    }
+    if (tid == 0) {
+        KVS_TRACE_STAMP(tr, kTrEnd);
+        KVS_TRACE_VALUE(tr, kTrPieces, trace_piece);
     }
 }
 
@@ -645,13 +660,17 @@ template <int D, int PRE, int kCombineWarps>
 __global__ void __launch_bounds__(kCombineWarps * 32, 5)
     decode_combine_kernel(const float* __restrict__ part_o, const float* __restrict__ part_ml, float* __restrict__ out,
                           int G, int tpu, long long T, int NC, const int* __restrict__ n_extra, int n, int tile_rows,
-                          int units, int cap, int* status) {
+                          int units, int cap, int* status, unsigned long long* trace) {
     constexpr int VEC = D / 32;
     struct __align__(VEC * 4) Vec {
         float v[VEC];
     };
+    unsigned long long* tr = (trace && threadIdx.x == 0 && (blockIdx.x == 0 || blockIdx.x == gridDim.x - 1))
+                                 ? trace + (size_t)(150 + (blockIdx.x != 0)) * kTraceSlots : nullptr;
+    KVS_TRACE_STAMP(tr, 0);
     pdl_launch_dependents();
     pdl_wait();
+    KVS_TRACE_STAMP(tr, 1);
     if (n_extra) {   // replayed launch: recompute the tile line from the grown length
         tpu = (min(n + *n_extra, cap) + tile_rows - 1) / tile_rows;
         T = (long long)units * tpu;
@@ -714,6 +733,7 @@ __global__ void __launch_bounds__(kCombineWarps * 32, 5)
 #pragma unroll
     for (int e = 0; e < VEC; ++e) r.v[e] = acc[e] / den;
     reinterpret_cast<Vec*>(out + (u * G + g) * D)[lane] = r;
+    KVS_TRACE_STAMP(tr, 2);
 }
 
 // Units of three or more pieces (fewer units than blocks): one BLOCK of four warps per (unit, q-head).
@@ -726,15 +746,19 @@ template <int D>
 __global__ void __launch_bounds__(kLongWarps * 32, 8)
     decode_combine_long_kernel(const float* __restrict__ part_o, const float* __restrict__ part_ml, float* __restrict__ out,
                                int G, int tpu, long long T, int NC, const int* __restrict__ n_extra, int n, int tile_rows,
-                               int units, int cap, int* status) {
+                               int units, int cap, int* status, unsigned long long* trace) {
     constexpr int VEC = D / 32;
     struct __align__(VEC * 4) Vec {
         float v[VEC];
     };
     __shared__ float s_max[kLongWarps], s_den[kLongWarps];
     __shared__ float s_acc[kLongWarps][D];
+    unsigned long long* tr = (trace && threadIdx.x == 0 && (blockIdx.x == 0 || blockIdx.x == gridDim.x - 1))
+                                 ? trace + (size_t)(150 + (blockIdx.x != 0)) * kTraceSlots : nullptr;
+    KVS_TRACE_STAMP(tr, 0);
     pdl_launch_dependents();
     pdl_wait();
+    KVS_TRACE_STAMP(tr, 1);
     if (n_extra) {   // replayed launch: recompute the tile line from the grown length
         tpu = (min(n + *n_extra, cap) + tile_rows - 1) / tile_rows;
         T = (long long)units * tpu;
@@ -814,6 +838,7 @@ __global__ void __launch_bounds__(kLongWarps * 32, 8)
 #pragma unroll
         for (int e = 0; e < VEC; ++e) r.v[e] /= d;
         reinterpret_cast<Vec*>(out + (u * G + g) * D)[lane] = r;
+        KVS_TRACE_STAMP(tr, 2);
     }
 }
 
@@ -824,7 +849,7 @@ static cudaError_t launch_combine_short(const DecodeArgs& a, const DecodePlan& p
     const dim3 grid((unsigned)((items + WARPS - 1) / WARPS)), block(WARPS * 32);
     return launch_kernel(decode_combine_kernel<D, 2, WARPS>, grid, block, 0, stream, a.programmatic, (const float*)a.part_o,
                          (const float*)a.part_ml, a.out, a.G, plan.tpu, plan.T, plan.NC, a.n_extra, a.n, plan.tile_rows,
-                         a.units, a.capacity, a.status);
+                         a.units, a.capacity, a.status, a.trace);
 }
 
 template <int D>
@@ -832,7 +857,7 @@ static cudaError_t launch_combine_long(const DecodeArgs& a, const DecodePlan& pl
     const dim3 grid((unsigned)(a.units * a.G)), block(kLongWarps * 32);
     return launch_kernel(decode_combine_long_kernel<D>, grid, block, 0, stream, a.programmatic, (const float*)a.part_o,
                          (const float*)a.part_ml, a.out, a.G, plan.tpu, plan.T, plan.NC, a.n_extra, a.n, plan.tile_rows,
-                         a.units, a.capacity, a.status);
+                         a.units, a.capacity, a.status, a.trace);
 }
 
 cudaError_t launch_combine(const DecodeArgs& a, const DecodePlan& plan, cudaStream_t stream) {
@@ -926,6 +951,7 @@ cudaError_t launch_decode_scalar(const DecodeArgs& a, const DecodePlan& plan, cu
     ka.plane_bytes = a.plane_bytes;
     ka.wait_ns = a.wait_ns;
     ka.stall_tile = a.stall_tile;
+    ka.trace = a.trace;
     const bool pdl = a.programmatic;
     if (a.dtype == 0) {
         if (a.D == 128) return launch_scalar_groups<__nv_bfloat16, 128>(a.G, plan.geom, ka, plan.NC, pdl, stream);
@@ -1049,6 +1075,14 @@ cudaError_t launch_wait_timeout_selftest(int* status, unsigned long long limit_n
 __global__ void bounds_selftest_kernel(int* status) {
     // 5 + 8 > 10; in a normal build the check is compiled out and nothing is recorded
     if (threadIdx.x == 0 && KVS_BOUNDS_OK(5, 8, 10, status)) return;
+}
+
+bool is_tracing_build() {
+#ifdef KVS_TRACE
+    return true;
+#else
+    return false;
+#endif
 }
 
 bool is_bounds_checking_build() {

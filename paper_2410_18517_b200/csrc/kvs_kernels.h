@@ -50,6 +50,7 @@ struct DecodeArgs {
     long long plane_bytes;   // size of one plane: what a bounds-checking build checks tile offsets against
     unsigned long long wait_ns;   // limit of every wait inside the split-K kernels
     long long stall_tile;    // self-test only: the K/V copies of this tile of the line are withheld (-1: none)
+    unsigned long long* trace;    // tracing build only: this launch's [kTraceBlocks][kTraceSlots] words, or nullptr
 };
 
 // Whether a launch of this plan over `units` units can finish inside the split-K kernel.
@@ -126,6 +127,11 @@ cudaError_t launch_combine(const DecodeArgs& a, const DecodePlan& plan, cudaStre
 // time-out code and *waited_ns (device, may be null) how long the wait lasted.
 cudaError_t launch_wait_timeout_selftest(int* status, unsigned long long limit_ns, unsigned long long* waited_ns,
                                          cudaStream_t stream);
+// Whether this library was compiled with -DKVS_TRACE (kernels stamp their timeline into DecodeArgs::trace).
+bool is_tracing_build();
+// Words one attention call (split-K kernel + combine kernel) occupies in a trace buffer: 160 rows of 32 words
+// (rows 0..147: the split-K kernel's blocks; rows 150 / 151: the first / last block of the combine kernel).
+constexpr int kTraceLaunchWords = 160 * 32;
 // Whether this library was compiled with -DKVS_DEBUG_BOUNDS, and a launch that makes its offset check
 // record one violation (KVS_ERR_BOUNDS in *status) without touching memory.
 bool is_bounds_checking_build();

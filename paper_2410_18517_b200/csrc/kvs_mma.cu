@@ -122,6 +122,7 @@ struct MmaKernelArgs {
     long long plane_rows;   // rows of one plane (what a bounds-checking build checks tile rows against)
     unsigned long long wait_ns;   // limit of every wait inside the kernel
     long long stall_tile;         // self-test only: the K/V copies of this tile are withheld (-1: none)
+    unsigned long long* trace;    // tracing build: this launch's rows of time stamps, or nullptr
 };
 
 // G (q-heads per kv-head, 1..8) is a run-time argument: it only selects which rows of the padded
@@ -132,6 +133,8 @@ __global__ void __launch_bounds__(kMmaThreads, KVS_MMA_BLOCKS_PER_SM)
                       const MmaKernelArgs a_in) {
     using S = MmaShape<D>;
     MmaKernelArgs a = a_in;
+    unsigned long long* tr = a.trace ? a.trace + (size_t)blockIdx.x * kTraceSlots : nullptr;
+    if (threadIdx.x == 0) KVS_TRACE_STAMP(tr, kTrEntry);
     bool over = false;    // a replayed launch with an append that would pass the capacity
     if (a.n_extra != nullptr) {
         // A replayed launch: the lengths recorded with it have grown on the device since.  The
@@ -239,7 +242,9 @@ __global__ void __launch_bounds__(kMmaThreads, KVS_MMA_BLOCKS_PER_SM)
                     issue(gt, npre, true, true, false);
                 }
             }
+            if (lane == 0) KVS_TRACE_STAMP(tr, kTrProducerPre);
             pdl_wait();
+            if (lane == 0) KVS_TRACE_STAMP(tr, kTrProducerGo);
             pdl_launch_dependents();
             // first the queries of the tiles already fetched (the consumers wait for nothing else), then the new rows
             if (lane == 0)
@@ -305,7 +310,9 @@ __global__ void __launch_bounds__(kMmaThreads, KVS_MMA_BLOCKS_PER_SM)
 
     // ---------------------------------- consumers ----------------------------------
     pdl_wait();               // partial results of the previous call may still be read until here
+    if (tid == 0) KVS_TRACE_STAMP(tr, kTrConsumerGo);
     pdl_launch_dependents();
+    int trace_piece = 0;
     const int row = lane >> 2;   // q-head row of the accumulator fragment (rows 8..15 are padding)
     const int quad = lane & 3;
 
@@ -326,6 +333,7 @@ __global__ void __launch_bounds__(kMmaThreads, KVS_MMA_BLOCKS_PER_SM)
         for (int k = 0; k < piece_tiles; ++k, ++it) {
             const int st = it % kMmaStages;
             if (!mbar_wait_bounded(&full_bar[st], (it / kMmaStages) & 1, abort_flag, a.status, a.wait_ns)) return;
+            if (tid == 0 && it == 0) KVS_TRACE_STAMP(tr, kTrFirstTile);
             const unsigned char* ks = smem + st * S::STAGE_BYTES;
             const uint32_t ks_u32 = smem_u32(ks);
             const uint32_t vs_u32 = ks_u32 + kMmaTileBytes;
@@ -460,6 +468,7 @@ __global__ void __launch_bounds__(kMmaThreads, KVS_MMA_BLOCKS_PER_SM)
         // first piece comes to it LAST, by when its hand-over warp has fetched the second piece into
         // shared memory; it merges the two in piece order and writes the result.
         const long long pid = u + blockIdx.x;
+        if (tid == 0 && trace_piece < 8) KVS_TRACE_STAMP(tr, kTrPiece + 2 * trace_piece);
         const bool finish = a.out != nullptr;
         const bool whole = finish && ti0 == 0 && piece_tiles == a.tpu;
         const bool head = finish && ti0 == 0 && piece_tiles < a.tpu;
@@ -512,7 +521,13 @@ __global__ void __launch_bounds__(kMmaThreads, KVS_MMA_BLOCKS_PER_SM)
             }
         }
         if (tail) mbar_arrive(tail_bar);   // this thread's part of the piece is written
+        if (tid == 0 && trace_piece < 8) KVS_TRACE_STAMP(tr, kTrPiece + 2 * trace_piece + 1);
+        ++trace_piece;
         gt += piece_tiles;
+    }
+    if (tid == 0) {
+        KVS_TRACE_STAMP(tr, kTrEnd);
+        KVS_TRACE_VALUE(tr, kTrPieces, trace_piece);
     }
 }
 
@@ -609,6 +624,7 @@ cudaError_t launch_decode_mma(const DecodeArgs& a, const DecodePlan& plan, const
     ka.plane_rows = a.plane_bytes / (a.D * 2);
     ka.wait_ns = a.wait_ns;
     ka.stall_tile = a.stall_tile;
+    ka.trace = a.trace;
     if (a.G < 1 || a.G > 8) return cudaErrorInvalidValue;
     if (a.D == 128) return launch_one<128>(tm, tm_tail, ka, plan.NC, a.programmatic, stream);
     if (a.D == 64) return launch_one<64>(tm, tm_tail, ka, plan.NC, a.programmatic, stream);

@@ -185,13 +185,15 @@ def test_replays_past_the_capacity_stop_appending_and_report(Hq, Hkv, evict, use
     assert torch.equal(changed, expect)
 
 
-@pytest.mark.parametrize("Hq,Hkv", [(8, 8), (32, 8)])
-def test_graph_replay_at_a_size_that_fills_the_gpu(Hq, Hkv):
+@pytest.mark.parametrize("Hq,Hkv,B", [(8, 8, 8), (32, 8, 4), (8, 8, 24), (32, 8, 24)])
+def test_graph_replay_at_a_size_that_fills_the_gpu(Hq, Hkv, B):
     """32 or 64 units of about 2000 rows: every SM has a thread block, blocks span units, and the tile
     line is recomputed on the device from the replay counter (the context ends three rows before a
-    tile boundary, so the replays cross it).  Sampled (sequence, q-head) pairs of the computing layer
+    tile boundary, so the replays cross it).  With batch 24 there are 192 units, more than thread blocks:
+    the split-K kernel finishes the units itself (no combine launch; the hand-over flags must be back
+    to zero after every replay).  Sampled (sequence, q-head) pairs of the computing layer
     and of the layer sharing its slot are checked against the oracle after every replay."""
-    L, D, B, context, replays = 2, 128, 4 if Hkv == 8 and Hq == 32 else 8, 2045, 5
+    L, D, context, replays = 2, 128, 2045, 5
     sm = [0, 0]
     cache = SharedKVCache(L, Hq, Hkv, D, B, context + replays + 2, "bf16", share_map=sm)
     cache.set_option(KVS_OPT_REPLAY, 1)
@@ -250,5 +252,6 @@ def test_graph_replay_at_a_size_that_fills_the_gpu(Hq, Hkv):
     cache.replay_commit(replays)
     torch.cuda.synchronize()
     assert cache.device_status() == 0 and cache.seq_len(1) == context + 1 + replays
+    assert (cache.stats()["combine_launches"] == 0) == (B * Hkv >= 148)
     kall = torch.cat(ks, dim=1)
     assert torch.equal(cache.plane(0, 0)[:B, :, : context + 1 + replays], kall.permute(0, 2, 1, 3))
