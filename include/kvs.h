@@ -408,7 +408,8 @@ kvs_status kvs_selftest_wait_timeout(kvs_ctx* ctx, uint32_t limit_us, uint64_t* 
  * nanosecond timer as thread block b of the split-K kernel saw it at entry [0], when its producer's / its
  * consumers' wait for the previous kernel returned [1] / [2], when the first tile had arrived [3], when the
  * tiles of its k-th piece were done [4 + 2k] and the piece was merged and written [5 + 2k] (k < 8), when the
- * consumers ended [20], the number of pieces [21], and when the producer began to wait [22]; rows 150 and
+ * consumers ended [20], the number of pieces [21], when the producer began to wait [22], and the SM the
+ * block ran on [23]; rows 150 and
  * 151 hold entry [0], end of wait [1] and end [2] of the first and the last block of the combine kernel
  * (zero when the call launched none).  kvs_trace_end stops the recording and reports the calls recorded.   */
 kvs_status kvs_trace_begin(kvs_ctx* ctx, void* buffer, size_t bytes);

@@ -27,6 +27,7 @@ enum TraceSlot {
     kTrEnd = 20,           // consumers are done
     kTrPieces = 21,        // number of pieces of the block
     kTrProducerPre = 22,   // producer: early tiles issued, about to wait
+    kTrSm = 23,            // the SM the block ran on
 };
 #ifdef KVS_TRACE
 #define KVS_TRACE_STAMP(row, slot) do { if ((row) != nullptr) (row)[slot] = ::kvs::globaltimer_ns(); } while (0)
@@ -57,6 +58,12 @@ constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
     return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+
+__device__ __forceinline__ unsigned int sm_id() {
+    unsigned int v;
+    asm volatile("mov.u32 %0, %%smid;" : "=r"(v));
+    return v;
 }
 
 __device__ __forceinline__ unsigned long long globaltimer_ns() {

@@ -285,7 +285,10 @@ __global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G, GEOM>::MI
     using S = ScalarShape<T, D, G, GEOM>;
     ScalarKernelArgs a = a_in;
     unsigned long long* tr = a.trace ? a.trace + (size_t)blockIdx.x * kTraceSlots : nullptr;
-    if (threadIdx.x == 0) KVS_TRACE_STAMP(tr, kTrEntry);
+    if (threadIdx.x == 0) {
+        KVS_TRACE_STAMP(tr, kTrEntry);
+        KVS_TRACE_VALUE(tr, kTrSm, sm_id());
+    }
     bool over = false;    // a replayed launch with an append that would pass the capacity
     if (a.n_extra != nullptr) {
         // A replayed launch: the lengths recorded with it have grown on the device since.  The

@@ -93,11 +93,27 @@ def main():
             rec["period"] = float((base - prev_base) / 1e3)
         prev_base = base
         per.append(rec)
+    # Is a block late because of the SM it ran on?  Per launch: each block's stream time (first tile to end)
+    # relative to the launch's median; then, per SM, the mean over the launches (what is systematic) and the
+    # spread of the rest (what is not).
+    rel, sms = [], []
+    for li in range(w.L, n_launches):
+        blk = t[li, :ctas]
+        d = blk[:, 20] - blk[:, 3]
+        rel.append(d / np.median(d) - 1.0)
+        sms.append(blk[:, 23].astype(int))
+    rel, sms = np.concatenate(rel), np.concatenate(sms)
+    per_sm = {int(sm_): rel[sms == sm_] for sm_ in np.unique(sms)}
+    sm_mean = np.array([v.mean() for v in per_sm.values()])
+    resid = np.concatenate([v - v.mean() for v in per_sm.values()])
+    out_sm = {"sms_seen": len(per_sm), "systematic_std_pct": round(100 * float(sm_mean.std()), 2),
+              "systematic_min_max_pct": [round(100 * float(sm_mean.min()), 2), round(100 * float(sm_mean.max()), 2)],
+              "residual_std_pct": round(100 * float(resid.std()), 2)}
     out = {"workload": {"batch": a.batch, "context": a.context, "q_heads": a.heads, "kv_heads": a.kv_heads, "layers": a.layers,
                         "kernel": cache.last_launch()["kernel"], "blocks": ctas,
                         "kv_mb_per_launch": w.kv_read_bytes_per_layer(w.context) / 1e6,
                         "combine_launches": cache.stats()["combine_launches"]},
-           "launches_reported": len(per)}
+           "launches_reported": len(per), "stream_time_by_sm": out_sm}
     for key in ("entry", "producer_wait_returns", "consumer_wait_returns", "first_tile", "end", "combine_first_block",
                 "combine_last_block"):
         vals = [r[key] for r in per if key in r]
