@@ -267,8 +267,8 @@ kvs_status kvs_unit_len(const kvs_ctx* ctx, int32_t layer, int32_t b, int32_t h,
  * the first call, so that it runs beside the averaging of the next slab; `stream` waits for it);
  * two last kernels sum, take roots and expand slots to layers.  Not during stream capture.
  * Sorting the pairs (descending, as the search does) is left to the caller.
- * Errors: STATE unless every slot holds the same non-zero number of rows and none is ragged;
- * INVALID_ARG for batch > cached batch or more than 80 layers.                                */
+ * Errors: STATE unless every slot holds the same non-zero number of rows and none is ragged, and while
+ * `stream` is being captured; INVALID_ARG for batch > cached batch or more than 80 layers.                                */
 kvs_status kvs_layer_distances(kvs_ctx* ctx, int32_t batch, float* dist, void* stream);
 
 /* Cosine similarity of two models' averaged output representations: a and b are device tensors
@@ -339,9 +339,10 @@ kvs_status kvs_step_host(kvs_ctx* ctx, const void* q_host, const void* k_host, c
  * allocates nothing and frees nothing, on the device or through any library.
  *   - Every GPU that loads the library holds those 2 MiB until the process exits.
  *   - Limit: (batch * n_kv_heads + blocks launched) * group * (head_dim + 2) * 4 bytes of partial
- *     results, 4 bytes per (sequence, kv-head) of hand-over flags and 768 bytes of rounding must
- *     fit in 2 MiB (the 7B shape at batch 8 needs 0.3 MiB, the 32q/8kv shape at batch 64 needs
- *     1.7 MiB).  Larger calls return KVS_ERR_SCRATCH_LIMIT and launch nothing.
+ *     results, rounded up twice to 256 bytes, must fit in 2 MiB less 33 KiB (a status word and
+ *     8192 per-unit hand-over flags at a fixed place); batch * n_kv_heads <= 8192.  The 7B shape at
+ *     batch 8 needs 0.3 MiB, the 32q/8kv shape at batch 64 1.7 MiB.  Larger calls return
+ *     KVS_ERR_SCRATCH_LIMIT and launch nothing.
  *   - The device address of the array is looked up once per GPU as part of kvs_bind_memory's
  *     per-device set-up (that look-up is also when the driver places the array on the GPU, so it
  *     happens where allocating is still allowed); the call itself makes no runtime query.

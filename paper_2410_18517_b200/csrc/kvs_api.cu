@@ -30,6 +30,10 @@ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 // ---------------------------------------------------------------------------------------
 constexpr size_t kStaticScratchBytes = 2u << 20;  // 2 MiB
 constexpr size_t kStaticStatusBytes = 256;        // first 256 bytes: device status word
+// then the per-unit hand-over flags, at a fixed place and of a fixed size, so that no call's partial results
+// (which follow) ever lie where another call, of another size, keeps its flags: they are zero when the library
+// is loaded and every launch leaves them zero
+constexpr size_t kStaticFlagBytes = 32768;        // 8192 (sequence, kv-head) units
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
 
 namespace {
@@ -737,6 +741,12 @@ kvs_status kvs_layer_distances(kvs_ctx* ctx, int32_t batch, float* dist, void* s
         if (ctx->slot_len[s] != n || ctx->ragged[s]) return KVS_ERR_STATE;   // equally long, un-evicted caches only
     DeviceGuard guard(ctx->cfg.device);
     if (!guard.ok) return KVS_ERR_CUDA;
+    {
+        // the pair sums run on a second stream with events in between: not something a capture can record
+        cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+        if (cudaStreamIsCapturing(static_cast<cudaStream_t>(stream), &cap) != cudaSuccess) return KVS_ERR_CUDA;
+        if (cap != cudaStreamCaptureStatusNone) return KVS_ERR_STATE;
+    }
     if (!ctx->search_ready) {
         int lo = 0, hi = 0;     // the side stream gets the highest priority: its short kernels slip in beside the long ones
         if (cudaDeviceGetStreamPriorityRange(&lo, &hi) != cudaSuccess ||
@@ -1157,8 +1167,10 @@ kvs_status kvs_decode_attention_static(kvs_ctx* ctx, int32_t layer, const void* 
     const size_t pieces = (size_t)units + plan.NC;
     const size_t part_o_bytes = align_up(pieces * c->G * D * sizeof(float), kAlign);
     const size_t part_ml_bytes = align_up(pieces * c->G * 2 * sizeof(float), kAlign);
-    const size_t flag_bytes = align_up((size_t)units * sizeof(int32_t), kAlign);   // zero at load, and again after every launch
-    if (kStaticStatusBytes + part_o_bytes + part_ml_bytes + flag_bytes > kStaticScratchBytes) return KVS_ERR_SCRATCH_LIMIT;
+    const size_t flag_bytes = kStaticFlagBytes;
+    if ((size_t)units * sizeof(int32_t) > kStaticFlagBytes ||
+        kStaticStatusBytes + part_o_bytes + part_ml_bytes + flag_bytes > kStaticScratchBytes)
+        return KVS_ERR_SCRATCH_LIMIT;
 
     DeviceGuard guard(c->cfg.device);
     if (!guard.ok) return KVS_ERR_CUDA;
@@ -1174,7 +1186,7 @@ kvs_status kvs_decode_attention_static(kvs_ctx* ctx, int32_t layer, const void* 
     // on another stream than the context's other calls, so it stays out of the bookkeeping that
     // decides what those calls may fetch early (untracked), and it leaves the "growth counter was
     // just written" mark for the next call of the chain.
-    // the flags come first so that they sit at the same place whatever the call's size
+    // layout: status word, flags (fixed size), partial outputs, partial (max, sum) pairs
     const AttentionScratch scratch = {reinterpret_cast<float*>(base + kStaticStatusBytes + flag_bytes),
                                       reinterpret_cast<float*>(base + kStaticStatusBytes + flag_bytes + part_o_bytes),
                                       reinterpret_cast<int*>(base + kStaticStatusBytes), status_word, false, false};

@@ -76,6 +76,18 @@ def test_layer_distances_state_errors():
     assert e.value.status == kb.KVS_ERR_INVALID_ARG                # more samples than cached
     kb.kvs_layer_distances(cache.ctx, 2, d, 0)
     assert float(d[0, 1]) == 0.0                                   # both layers hold the same rows
+    # the reduction forks onto a second stream: a stream that is being captured is refused, the capture survives
+    side, graph = torch.cuda.Stream(), torch.cuda.CUDAGraph()
+    marker = torch.zeros(4, device="cuda")
+    torch.cuda.synchronize()
+    with torch.cuda.graph(graph, stream=side):
+        with pytest.raises(KvsError) as e:
+            kb.kvs_layer_distances(cache.ctx, 2, d, side.cuda_stream)
+        marker += 1.0
+    assert e.value.status == kb.KVS_ERR_STATE
+    graph.replay()
+    torch.cuda.synchronize()
+    assert float(marker[0]) == 1.0
 
 
 @pytest.mark.parametrize("S,dim,dtype", [(30, 4096, "bf16"), (3, 10, "f32"), (7, 64 * 5120, "bf16"),

@@ -86,6 +86,30 @@ def test_static_scratch_matches_workspace_scratch_twice_in_a_row(Hq, Hkv, dtype)
     assert torch.cuda.mem_get_info()[0] >= free_before
 
 
+def test_static_calls_of_different_sizes_share_the_array():
+    """A call with few units, whose partial results fill the front of the array, then one with hundreds of
+    units that hands pieces over through per-unit flags, then the small one again: the flags of the large
+    call lie where no call keeps partial results, so nothing the small call left can be read as a flag."""
+    small = si.Workload("noalloc_small", L=1, Hq=8, Hkv=2, D=128, B=4, context=3000, dtype="bf16",
+                        n_shared=0, map_seed=0, steps=1, fixed_map=(0,))
+    large = si.Workload("noalloc_large", L=1, Hq=32, Hkv=8, D=128, B=32, context=700, dtype="bf16",
+                        n_shared=0, map_seed=0, steps=1, fixed_map=(0,))
+    made = [(w,) + _loaded_cache(w) for w in (small, large)]
+    stream = torch.cuda.current_stream().cuda_stream
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    for rep, (w, cache, rows) in enumerate([made[0], made[1], made[0], made[1]]):
+        q = si.step_qkv(w, rep, 0, device="cuda")[0]
+        ref = cache.decode_attention(0, q)
+        out = torch.full_like(ref, float("nan"))
+        kb.kvs_decode_attention_static(cache.ctx, 0, q, out, w.B, stream, status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        assert torch.equal(out, ref), rep
+        K, V = rows[0]
+        _check_units_against_oracle(w, 0, q, K, V, out, f"call {rep} ({w.name})")
+    assert made[1][1].stats()["combine_launches"] == 0      # the large calls were finished inside the split-K kernel
+
+
 def test_static_call_on_a_second_stream_beside_the_contexts_chain():
     """A decode step on stream A (the append rides in the attention kernel), the static call on
     stream B after an event, then the next decode step on A without waiting for B: the static call
