@@ -45,10 +45,10 @@ FALLBACK_HBM_GBS = 6650.0
 # of the captured launch; traffic grows in proportion to it, so the bench scales by that
 # ratio.  A record is used only while the kernel sources still hash to `sha256`.
 NCU_TRAFFIC = {
-    1: {"files": ("kvs_kernels.cu", "kvs_device.cuh"), "dram_bytes": 541.89e6, "kv_bytes": 537.13e6,
-        "sha256": "064b16bcfffe71336efc2768c7c5243c98e637a1bee229c40fb5eb29333f9242"},
-    2: {"files": ("kvs_mma.cu", "kvs_device.cuh"), "dram_bytes": 541.42e6, "kv_bytes": 536.90e6,
-        "sha256": "b304676938f01afe26c18d0bc87545a2072e2db255fdf26c5d720ae81689acb6"},
+    1: {"files": ("kvs_kernels.cu", "kvs_device.cuh"), "dram_bytes": 542.11e6, "kv_bytes": 537.13e6,
+        "sha256": "9c83af405cda6a601a3f59a8d9772f96a80ef6bf2d2c466c6dc54c92cd008722"},
+    2: {"files": ("kvs_mma.cu", "kvs_device.cuh"), "dram_bytes": 541.27e6, "kv_bytes": 536.90e6,
+        "sha256": "0d4e43aad08ae1382abe41ccecb78d1794592a6cc69f308cd7c2b19a271f590c"},
 }
 
 
