@@ -410,6 +410,43 @@ def test_units_finished_inside_the_split_k_kernel(Hq, Hkv, B, dtype, kernel, con
     assert cache.device_status() == 0
 
 
+@pytest.mark.parametrize("Hq,Hkv,B,context,dtype", [(32, 8, 32, 1024, "bf16"), (32, 32, 8, 4096, "bf16"), (8, 1, 160, 129, "bf16"),
+                                                   (4, 4, 40, 700, "f32"), (32, 8, 8, 8192, "bf16")])
+def test_launches_back_to_back_give_the_same_bits(Hq, Hkv, B, context, dtype):
+    """Hundreds of launches queued without a pause, each starting early beside the one before: the hand-over
+    flags and partial results of one launch must be gone before the next uses them.  Same inputs, so the same
+    bits every time; then decode steps (the append rides in the kernel) twice from the same cache length."""
+    reps = 100
+    w = si.Workload(f"b2b_{Hq}_{Hkv}_{B}_{context}", L=4, Hq=Hq, Hkv=Hkv, D=128, B=B, context=context, dtype=dtype,
+                    n_shared=1, map_seed=0, steps=1, fixed_map=(0, 1, 2, 0))
+    cache = make_cache(w, reps + 8)
+    for l in range(3):
+        k, v = si.context_kv(w, l, device="cuda")
+        cache.append(l, k, v)
+    ins = [si.step_qkv(w, 0, l, device="cuda") for l in range(4)]
+    outs = [[torch.empty(B, Hq, 128, device="cuda") for _ in range(4)] for _ in range(reps)]
+    torch.cuda.synchronize()
+    for r in range(reps):
+        for l in range(4):
+            cache.decode_attention(l, ins[l][0], out=outs[r][l])
+    torch.cuda.synchronize()
+    assert all(torch.equal(outs[r][l], outs[0][l]) for r in range(1, reps) for l in range(4))
+    assert not torch.equal(outs[0][0], outs[0][3]) and cache.device_status() == 0     # layer 3 reads slot 0 with its own q
+    runs = []
+    for _ in range(2):
+        cache.truncate(context)
+        res = []
+        for r in range(32):
+            for l in range(4):
+                q, k, v = ins[l]
+                own = l < 3
+                res.append(cache.decode_step(l, q, k if own else None, v if own else None))
+        torch.cuda.synchronize()
+        runs.append(res)
+    assert all(torch.equal(a, b) for a, b in zip(*runs))
+    assert cache.device_status() == 0
+
+
 # ------------------------------------------------------------------ sweep points at full size
 @pytest.mark.parametrize("name", ["sweep_b32_n1024_p10", "sweep_b64_n1024_p4", "sweep_b32_n8192_p8"])
 def test_sweep_points_sampled_units(name):
