@@ -212,7 +212,7 @@ void layout_workspace(kvs_ctx* c) {
         // at most one slot per layer, at most max_seq rows: enough for every strategy and length
         const size_t need = std::max(kvs::distance_scratch_bytes(f.n_layers <= kvs::kMaxLayersSearch ? f.n_layers : 4,
                                                                  2LL * f.n_kv_heads * f.max_seq * f.head_dim),
-                                     (size_t)kvs::kSearchMaxBlocks * 3 * sizeof(double));
+                                     (size_t)kvs::kCosineMaxBlocks * 3 * sizeof(double));
         c->search_bytes = need;
         off = align_up(off + need, kAlign);
     }

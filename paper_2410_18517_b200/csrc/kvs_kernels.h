@@ -93,6 +93,7 @@ cudaError_t launch_prefill_f32(const void* q, float* out, const void* kplane, co
 // Strategy-search reductions (see kvs_search.cu).
 constexpr int kMaxLayersSearch = 80;     // bound of the layer -> slot table handed to the finishing kernel
 constexpr int kSearchMaxBlocks = 640;    // sizes the per-block partial buffers
+constexpr int kCosineMaxBlocks = 4096;   // the same for the cosine reduction (three doubles per block)
 // The sample means of a slab of positions go through scratch memory between the two passes; a slab is
 // sized so that they stay in L2 (a fraction of its 126 MB).
 constexpr long long kMeanSlabBytes = 48ll << 20;
