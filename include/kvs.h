@@ -263,9 +263,10 @@ kvs_status kvs_unit_len(const kvs_ctx* ctx, int32_t layer, int32_t b, int32_t h,
  *   dist: device, float32 [n_layers][n_layers], symmetric, zero diagonal.
  * Reads every cached element once: per slab of positions (sized so that the slab's sample means,
  * which pass through the workspace, stay in L2) one kernel averages the samples and one adds the
- * squared differences of every pair of cache slots (on a second stream the context owns, created at
- * the first call, so that it runs beside the averaging of the next slab; `stream` waits for it);
- * two last kernels sum, take roots and expand slots to layers.  Not during stream capture.
+ * squared differences of every pair of cache slots; the averaging of the next slab is launched
+ * behind it so that it starts beside it (a programmatic dependent launch on `stream`: no other
+ * stream is used); two last kernels sum, take roots and expand slots to layers.  Not during
+ * stream capture.
  * Sorting the pairs (descending, as the search does) is left to the caller.
  * Errors: STATE unless every slot holds the same non-zero number of rows and none is ragged, and while
  * `stream` is being captured; INVALID_ARG for batch > cached batch or more than 80 layers.                                */

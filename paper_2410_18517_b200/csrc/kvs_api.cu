@@ -106,9 +106,6 @@ struct kvs_ctx {
     cudaStream_t copy_stream = nullptr, out_stream = nullptr;
     cudaEvent_t ev_in[kChunks] = {}, ev_done[kChunks] = {}, ev_start = nullptr;
     // kvs_layer_distances: a second stream on which the pair sums of one slab run beside the averaging of the next
-    bool search_ready = false;
-    cudaStream_t search_stream = nullptr;
-    cudaEvent_t ev_mean[2] = {}, ev_dist[2] = {}, ev_search_start = nullptr;
 
     int opt_max_ctas = 0;
     int opt_kernel = 0;
@@ -468,17 +465,6 @@ kvs_status kvs_create(const kvs_config* cfg, kvs_ctx** out) {
 
 kvs_status kvs_destroy(kvs_ctx* ctx) {
     if (!ctx) return KVS_ERR_INVALID_ARG;
-    if (ctx->search_ready) {
-        DeviceGuard guard(ctx->cfg.device);
-        if (guard.ok) {
-            for (int i = 0; i < 2; ++i) {
-                cudaEventDestroy(ctx->ev_mean[i]);
-                cudaEventDestroy(ctx->ev_dist[i]);
-            }
-            cudaEventDestroy(ctx->ev_search_start);
-            cudaStreamDestroy(ctx->search_stream);
-        }
-    }
     if (ctx->copy_ready) {
         DeviceGuard guard(ctx->cfg.device);
         if (guard.ok) {
@@ -742,37 +728,21 @@ kvs_status kvs_layer_distances(kvs_ctx* ctx, int32_t batch, float* dist, void* s
     DeviceGuard guard(ctx->cfg.device);
     if (!guard.ok) return KVS_ERR_CUDA;
     {
-        // the pair sums run on a second stream with events in between: not something a capture can record
+        // not recorded into graphs: the launch pattern (programmatic dependents between plain launches) is
+        // only exercised on a live stream
         cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
         if (cudaStreamIsCapturing(static_cast<cudaStream_t>(stream), &cap) != cudaSuccess) return KVS_ERR_CUDA;
         if (cap != cudaStreamCaptureStatusNone) return KVS_ERR_STATE;
     }
-    if (!ctx->search_ready) {
-        int lo = 0, hi = 0;     // the side stream gets the highest priority: its short kernels slip in beside the long ones
-        if (cudaDeviceGetStreamPriorityRange(&lo, &hi) != cudaSuccess ||
-            cudaStreamCreateWithPriority(&ctx->search_stream, cudaStreamNonBlocking, hi) != cudaSuccess)
-            return KVS_ERR_CUDA;
-        for (int i = 0; i < 2; ++i)
-            if (cudaEventCreateWithFlags(&ctx->ev_mean[i], cudaEventDisableTiming) != cudaSuccess ||
-                cudaEventCreateWithFlags(&ctx->ev_dist[i], cudaEventDisableTiming) != cudaSuccess)
-                return KVS_ERR_CUDA;
-        if (cudaEventCreateWithFlags(&ctx->ev_search_start, cudaEventDisableTiming) != cudaSuccess) return KVS_ERR_CUDA;
-        ctx->search_ready = true;
-    }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    // the side stream starts after whatever the caller already queued on `stream`
-    if (cudaEventRecord(ctx->ev_search_start, st) != cudaSuccess ||
-        cudaStreamWaitEvent(ctx->search_stream, ctx->ev_search_start, 0) != cudaSuccess)
-        return KVS_ERR_CUDA;
     int launches = 0;
     if (kvs::launch_layer_distances(ctx->pool, (long long)ctx->plane_bytes, ctx->slot_of_layer.data(), ctx->cfg.n_layers,
                                     ctx->n_slots, batch, ctx->cfg.n_kv_heads, n, ctx->row_stride, ctx->cfg.head_dim,
                                     ctx->cfg.dtype, reinterpret_cast<float*>(ctx->ws + ctx->off_search), ctx->search_bytes,
-                                    dist, ctx->sm_count, &launches, st, ctx->search_stream, ctx->ev_mean, ctx->ev_dist) !=
-        cudaSuccess)
+                                    dist, ctx->sm_count, &launches, st) != cudaSuccess)
         return KVS_ERR_CUDA;
     ctx->seq += launches;
-    ctx->last_splitk_seq = ctx->seq;     // plain launches: everything before them has finished when they run
+    ctx->last_splitk_seq = ctx->seq;     // the first and the last launches are plain: everything before them has finished
     ctx->stats.search_launches += launches;
     ctx->counter_written = false;   // a plain launch: full dependency on everything before it
     return KVS_OK;

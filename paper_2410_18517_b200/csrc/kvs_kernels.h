@@ -99,12 +99,12 @@ constexpr int kCosineMaxBlocks = 4096;   // the same for the cosine reduction (t
 constexpr long long kMeanSlabBytes = 48ll << 20;
 // Scratch the distance reduction needs for `n_slots` cache slots of `positions` = 2 * Hkv * n * D elements.
 size_t distance_scratch_bytes(int n_slots, long long positions);
-// *launches receives the number of kernels launched (two per slab and two to finish).  The distance pass of
-// a slab runs on `side` beside the mean pass of the next slab on `stream`; ev_mean / ev_dist: two events each.
+// *launches receives the number of kernels launched (two per slab and two to finish), all on `stream`: the
+// distance pass of a slab runs beside the mean pass of the next, which is launched behind it as a programmatic
+// dependent.
 cudaError_t launch_layer_distances(const void* pool, long long plane_bytes, const int* slot_of_layer, int L, int n_slots,
                                    int B, int Hkv, int n, int row_stride, int D, int dtype, float* scratch,
-                                   size_t scratch_bytes, float* dist, int sm_count, int* launches, cudaStream_t stream,
-                                   cudaStream_t side, cudaEvent_t* ev_mean, cudaEvent_t* ev_dist);
+                                   size_t scratch_bytes, float* dist, int sm_count, int* launches, cudaStream_t stream);
 cudaError_t launch_mean_cosine(const void* a, const void* b, int S, long long dim, int dtype, double* partial,
                                float* out, int sm_count, cudaStream_t stream);
 

@@ -20,7 +20,7 @@ namespace {
 constexpr int kMeanThreads = 256;
 constexpr int kMeanChunk = kMeanThreads * 8;   // positions per work item of the mean kernel: 8 per thread (16-byte loads of bf16)
 constexpr int kDistThreads = 256;
-constexpr int kDistChunk = 512;                // positions per chunk of the distance kernel: two per thread
+constexpr int kDistChunk = 256;                // positions per chunk of the distance kernel: one per thread
 constexpr int kDistStride = kDistChunk + 1;    // padded row of the mean tile (bank = slot + position)
 
 // As many thread groups as the block has threads for (at most 16) share the positions of a chunk, so that
@@ -118,20 +118,37 @@ struct DistArgs {
 };
 
 __global__ void __launch_bounds__(kDistThreads) mean_distance_kernel(const DistArgs a) {
-    extern __shared__ float sm[];
-    float* M = sm;
-    float* acc = sm + a.Sp * kDistStride;
+    // The mean pass of the next slab is launched behind this kernel as a programmatic dependent: it may move
+    // onto the SMs as soon as every block of this kernel has got here (it reads nothing this kernel writes).
+    pdl_launch_dependents();
+    extern __shared__ float M[];
     const int tid = threadIdx.x;
     const int tiles = a.Sp / 4;
     const int items = tiles * (tiles + 1) / 2;                     // 4x4 blocks of slot pairs with ti <= tj
     const int groups = dist_groups(items);                         // thread groups splitting the positions
-    for (int i = tid; i < groups * a.Sp * a.Sp; i += kDistThreads) acc[i] = 0.f;
+    // A thread keeps one 4x4 block of slot pairs and one share of every chunk's positions for the whole launch
+    // (groups * items <= threads), so its sixteen sums stay in registers from the first chunk to the last.
+    const bool active = tid < groups * items;
+    const int g = active ? tid / items : 0;
+    int it = active ? tid - g * items : 0, ti = 0;
+    while (it >= tiles - ti) {               // row ti of the upper triangle holds tiles - ti blocks
+        it -= tiles - ti;
+        ++ti;
+    }
+    const int tj = ti + it;
+    const int per = (kDistChunk + groups - 1) / groups;
+    const int q0 = g * per, q1 = min(kDistChunk, q0 + per);
+    float d[4][4];
+#pragma unroll
+    for (int x = 0; x < 4; ++x)
+#pragma unroll
+        for (int y = 0; y < 4; ++y) d[x][y] = 0.f;
     for (int i = tid; i < (a.Sp - a.S) * kDistStride; i += kDistThreads) M[a.S * kDistStride + i] = 0.f;  // padding slots
-    __syncthreads();
     const long long chunks = (a.count + kDistChunk - 1) / kDistChunk;
     for (long long c = blockIdx.x; c < chunks; c += gridDim.x) {
         const long long p = c * kDistChunk;
         const int have = (int)min((long long)kDistChunk, a.count - p);
+        __syncthreads();                     // the tile is free again (and, the first time, the padding is in place)
         // a warp reads 32 consecutive positions of one slot and stores them to 32 different banks; sixteen loads
         // are in flight per thread (the means come from L2)
 #pragma unroll 16
@@ -140,28 +157,17 @@ __global__ void __launch_bounds__(kDistThreads) mean_distance_kernel(const DistA
             M[sl * kDistStride + q] = q < have ? __ldcg(a.mean + (long long)sl * a.slab + p + q) : 0.f;
         }
         __syncthreads();
-        for (int w = tid; w < groups * items; w += kDistThreads) {
-            const int g = w / items;
-            int it = w - g * items, ti = 0;
-            while (it >= tiles - ti) {       // row ti of the upper triangle holds tiles - ti blocks
-                it -= tiles - ti;
-                ++ti;
-            }
-            const int tj = ti + it;
-            float d[4][4];
-#pragma unroll
-            for (int x = 0; x < 4; ++x)
-#pragma unroll
-                for (int y = 0; y < 4; ++y) d[x][y] = 0.f;
-            const int per = (kDistChunk + groups - 1) / groups;
-            const int q1 = min(kDistChunk, (g + 1) * per);
-            for (int q = g * per; q < q1; ++q) {
+        if (active) {
+            const float* mi_row = M + (4 * ti) * kDistStride;
+            const float* mj_row = M + (4 * tj) * kDistStride;
+#pragma unroll 2
+            for (int q = q0; q < q1; ++q) {
                 float mi[4];
                 float2 mj[2];
 #pragma unroll
-                for (int x = 0; x < 4; ++x) mi[x] = M[(4 * ti + x) * kDistStride + q];
-                mj[0] = make_float2(M[(4 * tj) * kDistStride + q], M[(4 * tj + 1) * kDistStride + q]);
-                mj[1] = make_float2(M[(4 * tj + 2) * kDistStride + q], M[(4 * tj + 3) * kDistStride + q]);
+                for (int x = 0; x < 4; ++x) mi[x] = mi_row[x * kDistStride + q];
+                mj[0] = make_float2(mj_row[q], mj_row[kDistStride + q]);
+                mj[1] = make_float2(mj_row[2 * kDistStride + q], mj_row[3 * kDistStride + q]);
                 // two slot pairs per instruction (packed fp32): t = mi - mj, d += t * t
                 const float2 minus1 = make_float2(-1.f, -1.f);
 #pragma unroll
@@ -174,17 +180,24 @@ __global__ void __launch_bounds__(kDistThreads) mean_distance_kernel(const DistA
                         d[x][2 * y + 1] = r.y;
                     }
             }
-            float* dst = acc + g * a.Sp * a.Sp;
-#pragma unroll
-            for (int x = 0; x < 4; ++x)
-#pragma unroll
-                for (int y = 0; y < 4; ++y) dst[(4 * ti + x) * a.Sp + 4 * tj + y] += d[x][y];   // (g, block) has one owner
         }
-        __syncthreads();
     }
+    // The groups' sums meet in shared memory (in the tile's place: the launch sizes it for both), are added
+    // in group order and go to the block's own partial matrix.
+    __syncthreads();
+    for (int i = tid; i < groups * a.Sp * a.Sp; i += kDistThreads) M[i] = 0.f;
+    __syncthreads();
+    if (active) {
+        float* dst = M + g * a.Sp * a.Sp;
+#pragma unroll
+        for (int x = 0; x < 4; ++x)
+#pragma unroll
+            for (int y = 0; y < 4; ++y) dst[(4 * ti + x) * a.Sp + 4 * tj + y] = d[x][y];   // (g, block) has one owner
+    }
+    __syncthreads();
     for (int i = tid; i < a.Sp * a.Sp; i += kDistThreads) {
         float s = 0.f;
-        for (int g = 0; g < groups; ++g) s += acc[g * a.Sp * a.Sp + i];
+        for (int gg = 0; gg < groups; ++gg) s += M[gg * a.Sp * a.Sp + i];
         float* dst = a.partial + (long long)blockIdx.x * a.Sp * a.Sp + i;
         *dst = a.first ? s : *dst + s;
     }
@@ -322,8 +335,7 @@ size_t distance_scratch_bytes(int n_slots, long long positions) {
 
 cudaError_t launch_layer_distances(const void* pool, long long plane_bytes, const int* slot_of_layer, int L, int n_slots,
                                    int B, int Hkv, int n, int row_stride, int D, int dtype, float* scratch,
-                                   size_t scratch_bytes, float* dist, int sm_count, int* launches, cudaStream_t stream,
-                                   cudaStream_t side, cudaEvent_t* ev_mean, cudaEvent_t* ev_dist) {
+                                   size_t scratch_bytes, float* dist, int sm_count, int* launches, cudaStream_t stream) {
     if (L > kMaxLayersSearch) return cudaErrorInvalidValue;
     const int S = n_slots, Sp = (S + 3) / 4 * 4;
     const long long P = 2LL * Hkv * n * D;
@@ -340,20 +352,24 @@ cudaError_t launch_layer_distances(const void* pool, long long plane_bytes, cons
 
     const int tiles = Sp / 4, items = tiles * (tiles + 1) / 2;
     const int groups = dist_groups(items);
-    const size_t smem = ((size_t)Sp * kDistStride + (size_t)groups * Sp * Sp) * sizeof(float);
+    const size_t smem = std::max((size_t)Sp * kDistStride, (size_t)groups * Sp * Sp) * sizeof(float);
     cudaError_t e;
     if ((e = cudaFuncSetAttribute(mean_distance_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess)
         return e;
+    // Two distance blocks per SM when there are few slabs (the last distance pass runs alone and should be
+    // short); one when there are many: each pass then has a whole mean pass to hide behind, and the fewer
+    // registers it holds the more mean blocks stay resident beside it (measured on 3, 4 and 21 slabs).
+    const int per_sm = n_slabs >= 8 ? 1 : 2;
     const int dist_blocks = (int)std::min<long long>((std::min(slab, P) + kDistChunk - 1) / kDistChunk,
-                                                     std::min(2 * sm_count, kSearchMaxBlocks));
-    // The mean pass (memory-bound) runs on `stream`, the distance pass (arithmetic on data in L2) on `side`:
-    // slab k's distances are added while slab k + 1 is averaged.  Buffer k % 2 is written again only after
-    // its distance pass has finished.
+                                                     std::min(per_sm * sm_count, kSearchMaxBlocks));
+    // One stream.  The distance pass of slab k is a plain launch (it waits for the mean pass of slab k and for
+    // the distance pass before it); the mean pass of slab k + 1 follows it as a programmatic dependent that
+    // never waits: it starts as soon as the distance blocks are resident and streams beside them.  It writes
+    // the buffer that the distance pass of slab k - 1 read, which has completed by then.
     *launches = 0;
     int k = 0;
     for (long long p0 = 0; p0 < P; p0 += slab, ++k) {
         const int buf = k & 1;
-        if (k >= 2 && (e = cudaStreamWaitEvent(stream, ev_dist[buf], 0)) != cudaSuccess) return e;
         MeanArgs m;
         m.pool = (const char*)pool;
         m.mean = mean[buf];
@@ -361,12 +377,10 @@ cudaError_t launch_layer_distances(const void* pool, long long plane_bytes, cons
         m.n_slots = S; m.B = B; m.Hkv = Hkv; m.n = n; m.row_stride = row_stride; m.D = D;
         m.p0 = p0; m.p1 = std::min(P, p0 + slab); m.slab = slab;
         const long long mean_items = (m.p1 - m.p0 + kMeanChunk - 1) / kMeanChunk * S;
-        const int mean_blocks = (int)std::min<long long>(mean_items, 16LL * sm_count);
-        if (dtype == 0) layer_mean_kernel<__nv_bfloat16><<<mean_blocks, kMeanThreads, 0, stream>>>(m);
-        else layer_mean_kernel<float><<<mean_blocks, kMeanThreads, 0, stream>>>(m);
-        if ((e = cudaGetLastError()) != cudaSuccess) return e;
-        if ((e = cudaEventRecord(ev_mean[buf], stream)) != cudaSuccess) return e;
-        if ((e = cudaStreamWaitEvent(side, ev_mean[buf], 0)) != cudaSuccess) return e;
+        const int blocks = (int)std::min<long long>(mean_items, 16LL * sm_count);
+        e = dtype == 0 ? launch_kernel(layer_mean_kernel<__nv_bfloat16>, dim3(blocks), dim3(kMeanThreads), 0, stream, k > 0, m)
+                       : launch_kernel(layer_mean_kernel<float>, dim3(blocks), dim3(kMeanThreads), 0, stream, k > 0, m);
+        if (e != cudaSuccess) return e;
         DistArgs a;
         a.mean = mean[buf];
         a.partial = partial;
@@ -374,14 +388,10 @@ cudaError_t launch_layer_distances(const void* pool, long long plane_bytes, cons
         a.count = m.p1 - m.p0; a.slab = slab;
         a.first = p0 == 0 ? 1 : 0;
         // the same number of blocks for every slab: block b's partial matrix is its own, slab after slab
-        // (the distance passes follow one another on `side`, so the additions keep their order)
-        mean_distance_kernel<<<dist_blocks, kDistThreads, smem, side>>>(a);
+        mean_distance_kernel<<<dist_blocks, kDistThreads, smem, stream>>>(a);
         if ((e = cudaGetLastError()) != cudaSuccess) return e;
-        if ((e = cudaEventRecord(ev_dist[buf], side)) != cudaSuccess) return e;
         *launches += 2;
     }
-    // `stream` goes on once the last distance pass (and with it every earlier one) is done
-    if ((e = cudaStreamWaitEvent(stream, ev_dist[(k - 1) & 1], 0)) != cudaSuccess) return e;
     // the slabs of means are no longer needed: the first bytes hold the slot-pair sums for a moment
     double* slot_dist2 = reinterpret_cast<double*>(mean[0]);
     distance_sum_kernel<<<(S * S + 7) / 8, 256, 0, stream>>>(partial, slot_dist2, S, Sp, dist_blocks);

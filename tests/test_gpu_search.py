@@ -76,7 +76,7 @@ def test_layer_distances_state_errors():
     assert e.value.status == kb.KVS_ERR_INVALID_ARG                # more samples than cached
     kb.kvs_layer_distances(cache.ctx, 2, d, 0)
     assert float(d[0, 1]) == 0.0                                   # both layers hold the same rows
-    # the reduction forks onto a second stream: a stream that is being captured is refused, the capture survives
+    # a stream that is being captured is refused (the call is not meant for graphs); the capture survives
     side, graph = torch.cuda.Stream(), torch.cuda.CUDAGraph()
     marker = torch.zeros(4, device="cuda")
     torch.cuda.synchronize()
