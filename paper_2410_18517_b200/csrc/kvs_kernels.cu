@@ -29,8 +29,8 @@ __global__ void __launch_bounds__(256) kv_append_kernel(const uint4* __restrict_
     }
     const uint4* __restrict__ src = blockIdx.y == 0 ? k : v;
     uint4* __restrict__ dst = blockIdx.y == 0 ? kplane : vplane;
-    for (long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x; idx < total_vecs;
-         idx += (long long)gridDim.x * blockDim.x) {
+    // where vector idx of the source goes in the plane (-1: nowhere)
+    auto target = [&](long long idx) -> long long {
         const int c = (int)(idx % row_vecs);
         long long r = idx / row_vecs;
         const int h = (int)(r % Hkv);
@@ -40,11 +40,27 @@ __global__ void __launch_bounds__(256) kv_append_kernel(const uint4* __restrict_
         const int first = unit_len ? unit_len[b * Hkv + h] : len0;   // ragged slots append per unit
         if (first + t >= capacity) {   // only a replay that outran the capacity gets here
             if (c == 0) atomicExch(status, 4);
-            continue;
+            return -1;
         }
         const long long drow = (b * Hkv + h) * (long long)row_stride + first + t;
-        if (!KVS_BOUNDS_OK(drow * row_vecs + c, 1, plane_vecs, status)) continue;
-        dst[drow * row_vecs + c] = src[idx];
+        if (!KVS_BOUNDS_OK(drow * row_vecs + c, 1, plane_vecs, status)) return -1;
+        return drow * row_vecs + c;
+    };
+    // four vectors per thread and turn, all four loads issued before the first store (a prompt's worth of
+    // rows is a plain copy at memory speed; one token's worth fits in the first turn of a few blocks)
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    long long idx = blockIdx.x * (long long)blockDim.x + threadIdx.x;
+    for (; idx < total_vecs; idx += 4 * stride) {
+        uint4 x[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+            if (idx + i * stride < total_vecs) x[i] = __ldcs(src + idx + i * stride);      // read once
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            if (idx + i * stride >= total_vecs) break;
+            const long long d = target(idx + i * stride);
+            if (d >= 0) dst[d] = x[i];
+        }
     }
 }
 
