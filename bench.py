@@ -390,6 +390,26 @@ def measure(w, K, W, E, rank, local_rank, world, dist, with_isolated=True, with_
     return rec
 
 
+def search_record(local_rank):
+    """The strategy search's reductions (layer-pair KV distances on the paper's calibration shape for a 7B and a
+    13B model, the mean-representation cosine on 1 GB) and decode over an evicted slot: time and GB/s of
+    algorithmic bytes against the measured copy bandwidth."""
+    import torch
+
+    from paper_2410_18517_b200 import next_rows_bench as nr
+
+    peak, kind = _peak_hbm()
+    out = []
+    with torch.cuda.device(local_rank):
+        for rec in (nr.distances(32, 32, 30, 64), nr.distances(40, 40, 30, 64), nr.cosine(30, 2048 * 4096),
+                    nr.ragged_decode(32, 8, 4, 32768, 0.8)):
+            gbs = rec.get("gbs", rec.get("kv_gbs_of_existing_rows"))
+            rec["roofline"] = {"bound": "hbm", "achieved": gbs, "peak": peak, "peak_kind": f"of {kind}", "unit": "GB/s",
+                               "frac": gbs / peak}
+            out.append(rec)
+    return out
+
+
 def prefill_record(local_rank):
     """The tensor-core prefill kernel on two prompt shapes: ms per call and TFLOP/s against the
     measured dense bf16 peak (algorithmic = causal flops 4 B Hq D T(T+1)/2; issued = what the tensor
@@ -459,6 +479,7 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=20)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-prefill", action="store_true")
+    ap.add_argument("--no-search", action="store_true", help="skip the record of the search reductions and the evicted-slot decode")
     ap.add_argument("--min-seconds", type=float, default=MIN_TIMED_S,
                     help="regions of --steps steps are repeated until this much has been timed (0: one region, for "
                          "profiler captures)")
@@ -496,7 +517,7 @@ def main():
 
     K, W, E = args.steps, args.warmup, args.e2e_steps
     head = measure(w, K, W, E, rank, local_rank, world, dist)
-    extras, prefill = [], None
+    extras, prefill, search = [], None, None
     if world == 1:
         names = args.configs if args.configs is not None else (DEFAULT_CONFIGS if args.workload == DEFAULT_WORKLOAD else "")
         for name in [x for x in names.split(",") if x]:
@@ -506,6 +527,8 @@ def main():
             extras.append(r)
         if not args.no_prefill:
             prefill = prefill_record(local_rank)
+        if not args.no_search and args.workload == DEFAULT_WORKLOAD and args.configs is None:   # the full default run only
+            search = search_record(local_rank)
 
     if rank != 0:
         if dist is not None:
@@ -520,6 +543,8 @@ def main():
         line["configs"] = extras
     if prefill is not None:
         line["prefill"] = prefill
+    if search is not None:
+        line["search_and_evicted"] = search
     if world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(w)
     print(json.dumps(line))
