@@ -191,7 +191,13 @@ __host__ __device__ __forceinline__ int cta_of_tile(long long gt, long long T, i
 #endif
 constexpr int kConsumerWarps = KVS_CONSUMER_WARPS;
 constexpr int kConsumerThreads = kConsumerWarps * 32;
-constexpr int kScalarThreads = kConsumerThreads + 64;   // + the producer warp and the hand-over warp
+// The second geometry (below) has twice the consumer warps: with 16 KiB tiles a tile is in the consumers'
+// hands for a shorter time, so more of the ring is in flight (13B shape: 15.55 -> 14.86 ms per step on one
+// box, 16.56 -> 15.83 on a slower one; the default geometry gains nothing from it).
+#ifndef KVS_LONG_CONSUMER_WARPS
+#define KVS_LONG_CONSUMER_WARPS 16
+#endif
+constexpr int kLongConsumerWarps = KVS_LONG_CONSUMER_WARPS;
 // Tile size, ring depth and blocks per SM of the scalar kernel for groups of 1 or 2 q-heads
 // (compile-time; the defaults are the measured best on B200).
 #ifndef KVS_TILE_BYTES
@@ -208,7 +214,10 @@ constexpr int kTileBytes = KVS_TILE_BYTES;  // per K tile and per V tile (defaul
 // 5 stages of 16 KiB tiles sustain ~3 % more on multi-gigabyte launches, the default is better below.
 constexpr int kLongTileBytes = 16384;
 constexpr int kLongStages = 5;
-constexpr long long kLongLaunchBytes = 1500000000LL;
+#ifndef KVS_LONG_LAUNCH_BYTES
+#define KVS_LONG_LAUNCH_BYTES 1500000000LL
+#endif
+constexpr long long kLongLaunchBytes = KVS_LONG_LAUNCH_BYTES;
 
 template <typename T, int D, int G, int GEOM = 0>
 struct ScalarShape {
@@ -216,8 +225,12 @@ struct ScalarShape {
     static constexpr int RB = D * (int)sizeof(T);
     static constexpr int LPR = RB / 16;
     static constexpr int EPL = 16 / (int)sizeof(T);
+    // consumer warps (128-byte rows keep eight in both geometries: with sixteen that kernel would spill)
+    static constexpr int WARPS = (GEOM == 1 && RB >= 256) ? kLongConsumerWarps : kConsumerWarps;
+    static constexpr int CTHREADS = WARPS * 32;           // consumer threads
+    static constexpr int THREADS = CTHREADS + 64;         // + the producer warp and the hand-over warp
     static constexpr int GPW = 32 / LPR;                  // lane groups per warp
-    static constexpr int NG = kConsumerWarps * GPW;       // lane groups per block
+    static constexpr int NG = WARPS * GPW;                // lane groups per block
     static constexpr int TN = TILE / RB;                  // rows per tile
     static constexpr int R = TN / NG;                     // rows per group per tile
     static constexpr int STAGES = GEOM == 1 ? kLongStages : ((G <= 2) ? KVS_STAGES : (6 * 16384) / kTileBytes);
@@ -296,7 +309,7 @@ struct ScalarKernelArgs {
 };
 
 template <typename T, int D, int G, int GEOM>
-__global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G, GEOM>::MIN_BLOCKS)
+__global__ void __launch_bounds__(ScalarShape<T, D, G, GEOM>::THREADS, ScalarShape<T, D, G, GEOM>::MIN_BLOCKS)
     decode_splitk_scalar(const ScalarKernelArgs a_in) {
     using S = ScalarShape<T, D, G, GEOM>;
     ScalarKernelArgs a = a_in;
@@ -342,9 +355,9 @@ __global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G, GEOM>::MI
     if (tid == 0) {
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(&full_bar[s], 1);
-            mbar_init(&empty_bar[s], kConsumerWarps);
+            mbar_init(&empty_bar[s], S::WARPS);
         }
-        mbar_init(tail_bar, kConsumerThreads);
+        mbar_init(tail_bar, S::CTHREADS);
         mbar_init(head_bar, 1);
         abort_flag[0] = 0;
         abort_flag[1] = 0;  // second word: bounds the producer's drain after a give-up
@@ -352,7 +365,7 @@ __global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G, GEOM>::MI
     }
     __syncthreads();
 
-    if (warp == kConsumerWarps) {
+    if (warp == S::WARPS) {
         // ------------------------------ producer ------------------------------
         // Lane 0 issues the copies; the whole warp stores the step's new rows when the launch
         // carries an append.
@@ -429,7 +442,7 @@ __global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G, GEOM>::MI
         return;
     }
 
-    if (warp == kConsumerWarps + 1) {
+    if (warp == S::WARPS + 1) {
         // ------------------ hand-over of units that are cut between two blocks ------------------
         // Only when the kernel finishes the units itself (a.out set).  The global round trips of the
         // hand-over are made here, beside the stream: this warp raises the flag of the unit whose
@@ -501,8 +514,8 @@ __global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G, GEOM>::MI
                 if constexpr (G > 4) {
                     // every warp is past the previous piece's last tile (the merge barriers), so the
                     // buffer is free; the stage that carries q is released after this tile
-                    for (int c = tid; c < G * LPR; c += kConsumerThreads) q_keep[c] = reinterpret_cast<const uint4*>(qs)[c];
-                    named_bar_sync(2, kConsumerThreads);
+                    for (int c = tid; c < G * LPR; c += S::CTHREADS) q_keep[c] = reinterpret_cast<const uint4*>(qs)[c];
+                    named_bar_sync(2, S::CTHREADS);
                 } else {
 #pragma unroll
                     for (int g = 0; g < (G > 4 ? 1 : G); ++g) {
@@ -613,7 +626,7 @@ __global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G, GEOM>::MI
             float l = lsum[g];
 #pragma unroll
             for (int o = LPR / 2; o >= LPR / R; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
-            named_bar_sync(1, kConsumerThreads);  // scratch free again
+            named_bar_sync(1, S::CTHREADS);  // scratch free again
             float* row = scratch + grp * (D + 2);
 #pragma unroll
             for (int e = 0; e < EPL; ++e) row[lig * EPL + e] = acc[g][e];
@@ -621,8 +634,8 @@ __global__ void __launch_bounds__(kScalarThreads, ScalarShape<T, D, G, GEOM>::MI
                 row[D] = m[g];
                 row[D + 1] = l;
             }
-            named_bar_sync(1, kConsumerThreads);
-            for (int d = tid; d < D; d += kConsumerThreads) {
+            named_bar_sync(1, S::CTHREADS);
+            for (int d = tid; d < D; d += S::CTHREADS) {
                 float M = -1.0e30f;
 #pragma unroll
                 for (int j = 0; j < NG; ++j) M = fmaxf(M, scratch[j * (D + 2) + D]);
@@ -913,7 +926,7 @@ static cudaError_t set_attr_groups() {
 
 template <typename T, int D, int G, int GEOM>
 static cudaError_t launch_scalar_one(const ScalarKernelArgs& ka, int NC, bool programmatic, cudaStream_t stream) {
-    return launch_kernel(decode_splitk_scalar<T, D, G, GEOM>, dim3(NC), dim3(kScalarThreads),
+    return launch_kernel(decode_splitk_scalar<T, D, G, GEOM>, dim3(NC), dim3(ScalarShape<T, D, G, GEOM>::THREADS),
                          ScalarShape<T, D, G, GEOM>::SMEM_BYTES, stream, programmatic, ka);
 }
 
