@@ -191,13 +191,6 @@ __host__ __device__ __forceinline__ int cta_of_tile(long long gt, long long T, i
 #endif
 constexpr int kConsumerWarps = KVS_CONSUMER_WARPS;
 constexpr int kConsumerThreads = kConsumerWarps * 32;
-// The second geometry (below) has twice the consumer warps: with 16 KiB tiles a tile is in the consumers'
-// hands for a shorter time, so more of the ring is in flight (13B shape: 15.55 -> 14.86 ms per step on one
-// box, 16.56 -> 15.83 on a slower one; the default geometry gains nothing from it).
-#ifndef KVS_LONG_CONSUMER_WARPS
-#define KVS_LONG_CONSUMER_WARPS 16
-#endif
-constexpr int kLongConsumerWarps = KVS_LONG_CONSUMER_WARPS;
 // Tile size, ring depth and blocks per SM of the scalar kernel for groups of 1 or 2 q-heads
 // (compile-time; the defaults are the measured best on B200).
 #ifndef KVS_TILE_BYTES
@@ -209,31 +202,26 @@ constexpr int kLongConsumerWarps = KVS_LONG_CONSUMER_WARPS;
 #ifndef KVS_BLOCKS_PER_SM
 #define KVS_BLOCKS_PER_SM 1
 #endif
-constexpr int kTileBytes = KVS_TILE_BYTES;  // per K tile and per V tile (default geometry)
-// Second geometry, used for one q-head per kv-head when a launch streams more than kLongLaunchBytes:
-// 5 stages of 16 KiB tiles sustain ~3 % more on multi-gigabyte launches, the default is better below.
-constexpr int kLongTileBytes = 16384;
-constexpr int kLongStages = 5;
-#ifndef KVS_LONG_LAUNCH_BYTES
-#define KVS_LONG_LAUNCH_BYTES 1500000000LL
-#endif
-constexpr long long kLongLaunchBytes = KVS_LONG_LAUNCH_BYTES;
-
-template <typename T, int D, int G, int GEOM = 0>
+constexpr int kTileBytes = KVS_TILE_BYTES;  // per K tile and per V tile
+// One geometry serves every launch size.  (A second one for multi-gigabyte launches, 5 stages of 16 KiB tiles,
+// was 3 % ahead when it was introduced and 5-9 % behind the default by the time the kernel finished its units
+// itself: 13B shape, same box, builds alternating, 16.56 against 15.09 ms per step at 1.5-1.7 GHz, 15.55 against
+// 14.86 at 1.84 GHz.  Sixteen consumer warps instead of eight repair that geometry (15.83 / 14.86) but add
+// nothing to this one: 15.10 against 15.09 ms on the 13B shape, 2.566 against 2.548 on the 7B shape.)
+template <typename T, int D, int G>
 struct ScalarShape {
-    static constexpr int TILE = GEOM == 1 ? kLongTileBytes : kTileBytes;
+    static constexpr int TILE = kTileBytes;
     static constexpr int RB = D * (int)sizeof(T);
     static constexpr int LPR = RB / 16;
     static constexpr int EPL = 16 / (int)sizeof(T);
-    // consumer warps (128-byte rows keep eight in both geometries: with sixteen that kernel would spill)
-    static constexpr int WARPS = (GEOM == 1 && RB >= 256) ? kLongConsumerWarps : kConsumerWarps;
+    static constexpr int WARPS = kConsumerWarps;          // consumer warps
     static constexpr int CTHREADS = WARPS * 32;           // consumer threads
     static constexpr int THREADS = CTHREADS + 64;         // + the producer warp and the hand-over warp
     static constexpr int GPW = 32 / LPR;                  // lane groups per warp
     static constexpr int NG = WARPS * GPW;                // lane groups per block
     static constexpr int TN = TILE / RB;                  // rows per tile
     static constexpr int R = TN / NG;                     // rows per group per tile
-    static constexpr int STAGES = GEOM == 1 ? kLongStages : ((G <= 2) ? KVS_STAGES : (6 * 16384) / kTileBytes);
+    static constexpr int STAGES = (G <= 2) ? KVS_STAGES : (6 * 16384) / kTileBytes;
     static constexpr int MIN_BLOCKS = (G <= 2) ? KVS_BLOCKS_PER_SM : 1;
     static constexpr int QBYTES = G * RB;
     static constexpr int STAGE_BYTES = 2 * TILE + QBYTES;
@@ -308,10 +296,10 @@ struct ScalarKernelArgs {
     unsigned long long* trace;    // tracing build: this launch's rows of time stamps, or nullptr
 };
 
-template <typename T, int D, int G, int GEOM>
-__global__ void __launch_bounds__(ScalarShape<T, D, G, GEOM>::THREADS, ScalarShape<T, D, G, GEOM>::MIN_BLOCKS)
+template <typename T, int D, int G>
+__global__ void __launch_bounds__(ScalarShape<T, D, G>::THREADS, ScalarShape<T, D, G>::MIN_BLOCKS)
     decode_splitk_scalar(const ScalarKernelArgs a_in) {
-    using S = ScalarShape<T, D, G, GEOM>;
+    using S = ScalarShape<T, D, G>;
     ScalarKernelArgs a = a_in;
     unsigned long long* tr = a.trace ? a.trace + (size_t)blockIdx.x * kTraceSlots : nullptr;
     if (threadIdx.x == 0) {
@@ -903,51 +891,46 @@ cudaError_t launch_combine(const DecodeArgs& a, const DecodePlan& plan, cudaStre
 // --------------------------------------------------------------------------------------
 // Launch plumbing for the scalar kernel.
 // --------------------------------------------------------------------------------------
-template <typename T, int D, int G, int GEOM>
+template <typename T, int D, int G>
 static cudaError_t set_attr_one() {
-    cudaError_t e = cudaFuncSetAttribute(decode_splitk_scalar<T, D, G, GEOM>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         ScalarShape<T, D, G, GEOM>::SMEM_BYTES);
+    cudaError_t e = cudaFuncSetAttribute(decode_splitk_scalar<T, D, G>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         ScalarShape<T, D, G>::SMEM_BYTES);
     if (e != cudaSuccess) return e;
     // the whole L1 / shared-memory array as shared memory, so that the combine kernel's blocks, launched
     // early behind this kernel, find room to become resident beside its blocks (see the tensor-core kernel)
-    return cudaFuncSetAttribute(decode_splitk_scalar<T, D, G, GEOM>, cudaFuncAttributePreferredSharedMemoryCarveout,
+    return cudaFuncSetAttribute(decode_splitk_scalar<T, D, G>, cudaFuncAttributePreferredSharedMemoryCarveout,
                                 cudaSharedmemCarveoutMaxShared);
 }
 
 template <typename T, int D>
 static cudaError_t set_attr_groups() {
     cudaError_t e;
-    if ((e = set_attr_one<T, D, 1, 0>()) != cudaSuccess) return e;
-    if ((e = set_attr_one<T, D, 1, 1>()) != cudaSuccess) return e;
-    if ((e = set_attr_one<T, D, 2, 0>()) != cudaSuccess) return e;
-    if ((e = set_attr_one<T, D, 4, 0>()) != cudaSuccess) return e;
-    return set_attr_one<T, D, 8, 0>();
+    if ((e = set_attr_one<T, D, 1>()) != cudaSuccess) return e;
+    if ((e = set_attr_one<T, D, 2>()) != cudaSuccess) return e;
+    if ((e = set_attr_one<T, D, 4>()) != cudaSuccess) return e;
+    return set_attr_one<T, D, 8>();
 }
 
-template <typename T, int D, int G, int GEOM>
+template <typename T, int D, int G>
 static cudaError_t launch_scalar_one(const ScalarKernelArgs& ka, int NC, bool programmatic, cudaStream_t stream) {
-    return launch_kernel(decode_splitk_scalar<T, D, G, GEOM>, dim3(NC), dim3(ScalarShape<T, D, G, GEOM>::THREADS),
-                         ScalarShape<T, D, G, GEOM>::SMEM_BYTES, stream, programmatic, ka);
+    return launch_kernel(decode_splitk_scalar<T, D, G>, dim3(NC), dim3(ScalarShape<T, D, G>::THREADS),
+                         ScalarShape<T, D, G>::SMEM_BYTES, stream, programmatic, ka);
 }
 
 template <typename T, int D>
-static cudaError_t launch_scalar_groups(int G, int geom, const ScalarKernelArgs& ka, int NC, bool pdl,
-                                        cudaStream_t stream) {
+static cudaError_t launch_scalar_groups(int G, const ScalarKernelArgs& ka, int NC, bool pdl, cudaStream_t stream) {
     switch (G) {
-        case 1:
-            return geom == 1 ? launch_scalar_one<T, D, 1, 1>(ka, NC, pdl, stream)
-                             : launch_scalar_one<T, D, 1, 0>(ka, NC, pdl, stream);
-        case 2: return launch_scalar_one<T, D, 2, 0>(ka, NC, pdl, stream);
-        case 4: return launch_scalar_one<T, D, 4, 0>(ka, NC, pdl, stream);
-        case 8: return launch_scalar_one<T, D, 8, 0>(ka, NC, pdl, stream);
+        case 1: return launch_scalar_one<T, D, 1>(ka, NC, pdl, stream);
+        case 2: return launch_scalar_one<T, D, 2>(ka, NC, pdl, stream);
+        case 4: return launch_scalar_one<T, D, 4>(ka, NC, pdl, stream);
+        case 8: return launch_scalar_one<T, D, 8>(ka, NC, pdl, stream);
         default: return cudaErrorInvalidValue;
     }
 }
 
 void plan_decode_scalar(int units, int n, int G, int D, int dtype, int sm_count, int max_ctas, DecodePlan* plan) {
     const int rb = D * (dtype == 0 ? 2 : 4);
-    plan->geom = (G == 1 && 2LL * units * n * rb >= kLongLaunchBytes) ? 1 : 0;
-    plan->tile_rows = (plan->geom == 1 ? kLongTileBytes : kTileBytes) / rb;
+    plan->tile_rows = kTileBytes / rb;
     plan->tpu = (n + plan->tile_rows - 1) / plan->tile_rows;
     plan->T = (long long)units * plan->tpu;
     const int per_sm = (G <= 2) ? KVS_BLOCKS_PER_SM : 1;
@@ -986,11 +969,11 @@ cudaError_t launch_decode_scalar(const DecodeArgs& a, const DecodePlan& plan, cu
     ka.trace = a.trace;
     const bool pdl = a.programmatic;
     if (a.dtype == 0) {
-        if (a.D == 128) return launch_scalar_groups<__nv_bfloat16, 128>(a.G, plan.geom, ka, plan.NC, pdl, stream);
-        if (a.D == 64) return launch_scalar_groups<__nv_bfloat16, 64>(a.G, plan.geom, ka, plan.NC, pdl, stream);
+        if (a.D == 128) return launch_scalar_groups<__nv_bfloat16, 128>(a.G, ka, plan.NC, pdl, stream);
+        if (a.D == 64) return launch_scalar_groups<__nv_bfloat16, 64>(a.G, ka, plan.NC, pdl, stream);
     } else {
-        if (a.D == 128) return launch_scalar_groups<float, 128>(a.G, plan.geom, ka, plan.NC, pdl, stream);
-        if (a.D == 64) return launch_scalar_groups<float, 64>(a.G, plan.geom, ka, plan.NC, pdl, stream);
+        if (a.D == 128) return launch_scalar_groups<float, 128>(a.G, ka, plan.NC, pdl, stream);
+        if (a.D == 64) return launch_scalar_groups<float, 64>(a.G, ka, plan.NC, pdl, stream);
     }
     return cudaErrorInvalidValue;
 }

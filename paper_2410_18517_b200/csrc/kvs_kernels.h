@@ -18,7 +18,6 @@ struct DecodePlan {
     long long T;     // total tiles = units * tpu
     int NC;          // thread blocks launched
     int kernel;      // 1 = scalar, 2 = tensor-core
-    int geom;        // scalar kernel: 0 = default ring geometry, 1 = the one for multi-gigabyte launches
 };
 
 struct DecodeArgs {

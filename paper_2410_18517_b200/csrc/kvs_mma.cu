@@ -593,7 +593,6 @@ void plan_decode_mma(int units, int n, int D, int sm_count, int max_ctas, Decode
     cap = std::min(cap, kMaxCtas);
     plan->NC = (int)std::min<long long>(plan->T, cap);
     plan->kernel = 2;
-    plan->geom = 0;
 }
 
 cudaError_t launch_decode_mma(const DecodeArgs& a, const DecodePlan& plan, const void* tensor_map,

@@ -71,6 +71,10 @@ WORKLOADS = {
                           n_shared=1, map_seed=0, steps=20, fixed_map=(0, 1, 2, 1)),
     "gqa_long_l4": Workload("gqa_long_l4", L=4, Hq=32, Hkv=8, D=128, B=4, context=32768, dtype="bf16",
                             n_shared=1, map_seed=0, steps=20, fixed_map=(0, 1, 2, 1)),
+    # the 13B shape cut to 3 layers and 4736 rows (3 GiB pool): the smallest launches (1.55 GB) that still take
+    # the scalar kernel's long-launch geometry, for profiler captures of that kernel
+    "13b_mha_l3": Workload("13b_mha_l3", L=3, Hq=40, Hkv=40, D=128, B=16, context=4736, dtype="bf16",
+                           n_shared=1, map_seed=0, steps=20, fixed_map=(0, 1, 0)),
     "13b_mha": Workload("13b_mha", L=40, Hq=40, Hkv=40, D=128, B=16, context=8192, dtype="bf16",
                         n_shared=12, map_seed=3, steps=64),
     "gqa_long": Workload("gqa_long", L=32, Hq=32, Hkv=8, D=128, B=4, context=32768, dtype="bf16",
