@@ -37,23 +37,43 @@ constexpr int kMmaThreads = kMmaConsumerThreads + 64;   // + the producer warp a
 constexpr int kMmaTileBytes = KVS_MMA_TILE_BYTES;
 constexpr int kMmaQBytes = 2048;  // room for 8 heads x 128 x bf16
 constexpr int kMmaStages = KVS_MMA_STAGES;
+// Second ring geometry, for launches that give every block at least kMmaBigMinTiles of its (larger) tiles: 3
+// stages of 32 KiB tiles.  Half as many barrier round trips, piece bookkeeping and tile set-ups per byte: with
+// one warp per scheduler all of that is exposed, and the kernel follows the SM clock that the power cap
+// leaves (same box at 1.5-1.7 GHz, builds alternating: 32q/8kv, B=4, n=32768 2.77 -> 2.63 ms per step; B=32,
+// n=8192 5.46 -> 5.15; B=32, n=1024 0.846 -> 0.835).  Small launches keep the 16 KiB tiles: they need the finer
+// split over the blocks.
+#ifndef KVS_MMA_BIG_TILE_BYTES
+#define KVS_MMA_BIG_TILE_BYTES 32768
+#endif
+#ifndef KVS_MMA_BIG_STAGES
+#define KVS_MMA_BIG_STAGES 3
+#endif
+#ifndef KVS_MMA_BIG_MIN_TILES
+#define KVS_MMA_BIG_MIN_TILES 12
+#endif
+constexpr int kMmaBigTileBytes = KVS_MMA_BIG_TILE_BYTES;
+constexpr int kMmaBigStages = KVS_MMA_BIG_STAGES;
+constexpr int kMmaBigMinTiles = KVS_MMA_BIG_MIN_TILES;
 constexpr int kBoxRows = 64;      // the pool's tensor map moves boxes of 64 columns x 64 rows (8 KiB)
 constexpr int kTailRows = 16;     // a second map moves 16-row boxes: the last, partly filled tile of a unit
                                   // is fetched in as many of these as hold rows (16 = the tokens of one MMA block)
 
-template <int D>
+template <int D, int BIG>
 struct MmaShape {
+    static constexpr int TILE = BIG ? kMmaBigTileBytes : kMmaTileBytes;   // bytes per K tile and per V tile
+    static constexpr int STAGES = BIG ? kMmaBigStages : kMmaStages;
     static constexpr int RB = D * 2;
     static constexpr int HALVES = D / 64;                  // 128-byte column blocks per row
-    static constexpr int TN = kMmaTileBytes / RB;          // rows per tile: 64 (D=128) or 128 (D=64)
+    static constexpr int TN = TILE / RB;                   // rows per tile: 64 or 128 (D=128), 128 or 256 (D=64)
     static constexpr int BPW = TN / (kMmaWarps * 16);      // 16-token blocks per warp per tile
     static constexpr int KSTEPS = D / 16;
     static constexpr int NB = D / 8;
-    static constexpr int STAGE_BYTES = 2 * kMmaTileBytes + kMmaQBytes;
+    static constexpr int STAGE_BYTES = 2 * TILE + kMmaQBytes;
     static constexpr int SCRATCH_FLOATS = kMmaWarps * 8 * (D + 2);   // [warp][q-head of the group][D + 2]
     static constexpr int HANDOVER_FLOATS = 8 * (D + 2);              // another block's piece of a cut unit: [q-head][D + 2]
-    static constexpr int SMEM_BYTES = 1024 + kMmaStages * STAGE_BYTES + (SCRATCH_FLOATS + HANDOVER_FLOATS) * 4 +
-                                      (2 * kMmaStages + 2) * 8 + 16;
+    static constexpr int SMEM_BYTES = 1024 + STAGES * STAGE_BYTES + (SCRATCH_FLOATS + HANDOVER_FLOATS) * 4 +
+                                      (2 * STAGES + 2) * 8 + 16;
 };
 
 __device__ __forceinline__ void tma_load_2d(void* dst_smem, const CUtensorMap* tmap, int x, int y, uint64_t* bar) {
@@ -127,11 +147,12 @@ struct MmaKernelArgs {
 
 // G (q-heads per kv-head, 1..8) is a run-time argument: it only selects which rows of the padded
 // 16-row M side are real, so one kernel per head size serves every group size.
-template <int D>
+template <int D, int BIG>
 __global__ void __launch_bounds__(kMmaThreads, KVS_MMA_BLOCKS_PER_SM)
     decode_splitk_mma(const __grid_constant__ CUtensorMap tmap, const __grid_constant__ CUtensorMap tmap_tail,
                       const MmaKernelArgs a_in) {
-    using S = MmaShape<D>;
+    using S = MmaShape<D, BIG>;
+    constexpr int kTile = S::TILE, kStages = S::STAGES;
     MmaKernelArgs a = a_in;
     unsigned long long* tr = a.trace ? a.trace + (size_t)blockIdx.x * kTraceSlots : nullptr;
     if (threadIdx.x == 0) {
@@ -155,10 +176,10 @@ __global__ void __launch_bounds__(kMmaThreads, KVS_MMA_BLOCKS_PER_SM)
     extern __shared__ unsigned char smem_raw[];
     // 128-byte swizzled tiles need 1024-byte aligned bases
     unsigned char* smem = smem_raw + ((1024u - (smem_u32(smem_raw) & 1023u)) & 1023u);
-    float* scratch = reinterpret_cast<float*>(smem + kMmaStages * S::STAGE_BYTES);
+    float* scratch = reinterpret_cast<float*>(smem + kStages * S::STAGE_BYTES);
     uint64_t* full_bar = reinterpret_cast<uint64_t*>(scratch + S::SCRATCH_FLOATS);
-    uint64_t* empty_bar = full_bar + kMmaStages;
-    uint64_t* tail_bar = empty_bar + kMmaStages;     // every consumer thread has written this block's second-piece partial
+    uint64_t* empty_bar = full_bar + kStages;
+    uint64_t* tail_bar = empty_bar + kStages;     // every consumer thread has written this block's second-piece partial
     uint64_t* head_bar = tail_bar + 1;               // the next block's second-piece partial is in handover[]
     volatile int* abort_flag = reinterpret_cast<volatile int*>(head_bar + 1);
     float* handover = const_cast<float*>(reinterpret_cast<volatile float*>(abort_flag + 4));
@@ -169,7 +190,7 @@ __global__ void __launch_bounds__(kMmaThreads, KVS_MMA_BLOCKS_PER_SM)
     const long long t1 = ((long long)(blockIdx.x + 1) * a.T) / NC;
 
     if (tid == 0) {
-        for (int s = 0; s < kMmaStages; ++s) {
+        for (int s = 0; s < kStages; ++s) {
             mbar_init(&full_bar[s], 1);
             mbar_init(&empty_bar[s], kMmaWarps);
         }
@@ -196,7 +217,7 @@ __global__ void __launch_bounds__(kMmaThreads, KVS_MMA_BLOCKS_PER_SM)
                 const int rows = min(TN, n_u - ti * TN);          // <= 0: a ragged unit ended before this tile
                 // a full tile comes in 64-row boxes; a partly filled one in 16-row boxes, only those that hold rows
                 const int tail_boxes = rows < TN ? (rows + kTailRows - 1) / kTailRows : 0;
-                const uint32_t kv_bytes = rows <= 0 ? 0u : (rows == TN ? 2u * kMmaTileBytes : 2u * tail_boxes * kTailRows * S::RB);
+                const uint32_t kv_bytes = rows <= 0 ? 0u : (rows == TN ? 2u * kTile : 2u * tail_boxes * kTailRows * S::RB);
                 unsigned char* sb = smem + st * S::STAGE_BYTES;
                 if (arm) {
                     const uint32_t total = kv_bytes + (with_q ? QBYTES : 0);
@@ -216,7 +237,7 @@ __global__ void __launch_bounds__(kMmaThreads, KVS_MMA_BLOCKS_PER_SM)
                             for (int rb = 0; rb < TN / kBoxRows; ++rb) {
                                 const int off = h * (TN * 128) + rb * (kBoxRows * 128);
                                 tma_load_2d(sb + off, &tmap, h * 64, (int)(a.krow0 + row) + rb * kBoxRows, &full_bar[st]);
-                                tma_load_2d(sb + kMmaTileBytes + off, &tmap, h * 64, (int)(a.vrow0 + row) + rb * kBoxRows,
+                                tma_load_2d(sb + kTile + off, &tmap, h * 64, (int)(a.vrow0 + row) + rb * kBoxRows,
                                             &full_bar[st]);
                             }
                     } else {
@@ -225,20 +246,20 @@ __global__ void __launch_bounds__(kMmaThreads, KVS_MMA_BLOCKS_PER_SM)
                             for (int rb = 0; rb < tail_boxes; ++rb) {
                                 const int off = h * (TN * 128) + rb * (kTailRows * 128);
                                 tma_load_2d(sb + off, &tmap_tail, h * 64, (int)(a.krow0 + row) + rb * kTailRows, &full_bar[st]);
-                                tma_load_2d(sb + kMmaTileBytes + off, &tmap_tail, h * 64,
+                                tma_load_2d(sb + kTile + off, &tmap_tail, h * 64,
                                             (int)(a.vrow0 + row) + rb * kTailRows, &full_bar[st]);
                             }
                     }
                 }
                 if (qpart && with_q)
-                    bulk_g2s(sb + 2 * kMmaTileBytes, a.q + (KVS_BOUNDS_OK(u, 1, a.units, a.status) ? u : 0) * (long long)QBYTES,
+                    bulk_g2s(sb + 2 * kTile, a.q + (KVS_BOUNDS_OK(u, 1, a.units, a.status) ? u : 0) * (long long)QBYTES,
                              QBYTES, &full_bar[st]);
             };
             // Until the preceding kernel in the stream is known to have finished, fetch only
             // K/V tiles made entirely of rows that no kernel still in flight can be writing.
             int npre = 0;
             if (lane == 0) {
-                for (; npre < kMmaStages && t0 + npre < t1; ++npre) {
+                for (; npre < kStages && t0 + npre < t1; ++npre) {
                     const long long gt = t0 + npre;
                     const int ti = (int)(gt % a.tpu);
                     if ((long long)(ti + 1) * TN > a.safe_rows) break;
@@ -263,15 +284,15 @@ __global__ void __launch_bounds__(kMmaThreads, KVS_MMA_BLOCKS_PER_SM)
             int it = npre;
             bool ok = true;
             for (long long gt = t0 + npre; gt < t1; ++gt, ++it) {
-                const int st = it % kMmaStages;
-                if (it >= kMmaStages)
-                    ok = mbar_wait_bounded(&empty_bar[st], ((it / kMmaStages) - 1) & 1, abort_flag, a.status, a.wait_ns);
+                const int st = it % kStages;
+                if (it >= kStages)
+                    ok = mbar_wait_bounded(&empty_bar[st], ((it / kStages) - 1) & 1, abort_flag, a.status, a.wait_ns);
                 if (!ok) break;
                 issue(gt, st, true, true, true);
             }
             if (!ok) {
-                for (int j = max(0, it - kMmaStages); j < it; ++j)
-                    mbar_wait_bounded(&full_bar[j % kMmaStages], (j / kMmaStages) & 1, abort_flag + 1, a.status, a.wait_ns);
+                for (int j = max(0, it - kStages); j < it; ++j)
+                    mbar_wait_bounded(&full_bar[j % kStages], (j / kStages) & 1, abort_flag + 1, a.status, a.wait_ns);
             }
         }
         return;
@@ -334,15 +355,15 @@ __global__ void __launch_bounds__(kMmaThreads, KVS_MMA_BLOCKS_PER_SM)
         for (int nb = 0; nb < NB; ++nb) o[nb][0] = o[nb][1] = 0.f;
 
         for (int k = 0; k < piece_tiles; ++k, ++it) {
-            const int st = it % kMmaStages;
-            if (!mbar_wait_bounded(&full_bar[st], (it / kMmaStages) & 1, abort_flag, a.status, a.wait_ns)) return;
+            const int st = it % kStages;
+            if (!mbar_wait_bounded(&full_bar[st], (it / kStages) & 1, abort_flag, a.status, a.wait_ns)) return;
             if (tid == 0 && it == 0) KVS_TRACE_STAMP(tr, kTrFirstTile);
             const unsigned char* ks = smem + st * S::STAGE_BYTES;
             const uint32_t ks_u32 = smem_u32(ks);
-            const uint32_t vs_u32 = ks_u32 + kMmaTileBytes;
+            const uint32_t vs_u32 = ks_u32 + kTile;
             if (k == 0) {
                 // A fragments of Q: row g < G real, the rest zero
-                const uint32_t* qs = reinterpret_cast<const uint32_t*>(ks + 2 * kMmaTileBytes);
+                const uint32_t* qs = reinterpret_cast<const uint32_t*>(ks + 2 * kTile);
 #pragma unroll
                 for (int s = 0; s < KSTEPS; ++s) {
                     qa[s][0] = row < G ? qs[row * (D / 2) + s * 8 + quad] : 0u;
@@ -534,31 +555,34 @@ __global__ void __launch_bounds__(kMmaThreads, KVS_MMA_BLOCKS_PER_SM)
     }
 }
 
-template <int D>
+template <int D, int BIG>
 cudaError_t set_attr() {
-    cudaError_t e = cudaFuncSetAttribute(decode_splitk_mma<D>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         MmaShape<D>::SMEM_BYTES);
+    cudaError_t e = cudaFuncSetAttribute(decode_splitk_mma<D, BIG>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         MmaShape<D, BIG>::SMEM_BYTES);
     if (e != cudaSuccess) return e;
     // All of the SM's L1 / shared-memory array as shared memory: the kernel gains nothing from L1
     // (its loads are bulk copies), and the blocks of the small kernels launched early behind it
     // (combine) only become resident beside it if the carve-out has room for them.  Measured: with
     // the default carve-out a footprint of 157 KiB instead of 142 KiB cost 2.8 us per layer.
-    return cudaFuncSetAttribute(decode_splitk_mma<D>, cudaFuncAttributePreferredSharedMemoryCarveout,
+    return cudaFuncSetAttribute(decode_splitk_mma<D, BIG>, cudaFuncAttributePreferredSharedMemoryCarveout,
                                 cudaSharedmemCarveoutMaxShared);
 }
 
-template <int D>
+template <int D, int BIG>
 cudaError_t launch_one(const CUtensorMap& tm, const CUtensorMap& tm_tail, const MmaKernelArgs& ka, int NC, bool pdl,
                        cudaStream_t stream) {
-    return launch_kernel(decode_splitk_mma<D>, dim3(NC), dim3(kMmaThreads), MmaShape<D>::SMEM_BYTES, stream, pdl, tm, tm_tail,
-                         ka);
+    return launch_kernel(decode_splitk_mma<D, BIG>, dim3(NC), dim3(kMmaThreads), MmaShape<D, BIG>::SMEM_BYTES, stream, pdl, tm,
+                         tm_tail, ka);
 }
 
 }  // namespace
 
 cudaError_t init_mma_kernels() {
-    cudaError_t e = set_attr<128>();
-    return e != cudaSuccess ? e : set_attr<64>();
+    cudaError_t e;
+    if ((e = set_attr<128, 0>()) != cudaSuccess || (e = set_attr<128, 1>()) != cudaSuccess ||
+        (e = set_attr<64, 0>()) != cudaSuccess)
+        return e;
+    return set_attr<64, 1>();
 }
 
 // Tensor map over the whole pool seen as [total_rows][D] bf16, box = 64 columns x 64 rows (or, with
@@ -585,12 +609,15 @@ cudaError_t make_pool_tensor_map(void* storage, void* pool, long long total_rows
 }
 
 void plan_decode_mma(int units, int n, int D, int sm_count, int max_ctas, DecodePlan* plan) {
-    plan->tile_rows = kMmaTileBytes / (D * 2);
-    plan->tpu = (n + plan->tile_rows - 1) / plan->tile_rows;
-    plan->T = (long long)units * plan->tpu;
     int cap = sm_count * KVS_MMA_BLOCKS_PER_SM;
     if (max_ctas > 0) cap = std::min(cap, max_ctas);
     cap = std::min(cap, kMaxCtas);
+    // the larger tiles when every block still gets kMmaBigMinTiles of them
+    const int big_rows = kMmaBigTileBytes / (D * 2);
+    const long long big_T = (long long)units * ((n + big_rows - 1) / big_rows);
+    plan->tile_rows = big_T >= (long long)kMmaBigMinTiles * cap ? big_rows : kMmaTileBytes / (D * 2);
+    plan->tpu = (n + plan->tile_rows - 1) / plan->tile_rows;
+    plan->T = (long long)units * plan->tpu;
     plan->NC = (int)std::min<long long>(plan->T, cap);
     plan->kernel = 2;
 }
@@ -628,8 +655,13 @@ cudaError_t launch_decode_mma(const DecodeArgs& a, const DecodePlan& plan, const
     ka.stall_tile = a.stall_tile;
     ka.trace = a.trace;
     if (a.G < 1 || a.G > 8) return cudaErrorInvalidValue;
-    if (a.D == 128) return launch_one<128>(tm, tm_tail, ka, plan.NC, a.programmatic, stream);
-    if (a.D == 64) return launch_one<64>(tm, tm_tail, ka, plan.NC, a.programmatic, stream);
+    const bool big = plan.tile_rows * a.D * 2 == kMmaBigTileBytes && kMmaBigTileBytes != kMmaTileBytes;
+    if (a.D == 128)
+        return big ? launch_one<128, 1>(tm, tm_tail, ka, plan.NC, a.programmatic, stream)
+                   : launch_one<128, 0>(tm, tm_tail, ka, plan.NC, a.programmatic, stream);
+    if (a.D == 64)
+        return big ? launch_one<64, 1>(tm, tm_tail, ka, plan.NC, a.programmatic, stream)
+                   : launch_one<64, 0>(tm, tm_tail, ka, plan.NC, a.programmatic, stream);
     return cudaErrorInvalidValue;
 }
 
