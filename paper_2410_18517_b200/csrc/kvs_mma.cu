@@ -377,17 +377,27 @@ __global__ void __launch_bounds__(kMmaThreads, KVS_MMA_BLOCKS_PER_SM)
                 continue;
             }
 
+            if (warp * BPW * 16 >= valid) {   // none of this warp's rows exists in this (partly filled) tile
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&empty_bar[st]);
+                continue;
+            }
+            // A warp's BPW blocks of 16 tokens go through the tile in three phases - all score products, one
+            // online-softmax update over all of them, all output products - so that the blocks' chains of
+            // loads and MMAs overlap and the running state is rescaled once per tile (one warp per scheduler:
+            // nothing else hides those latencies).
+            // ---- S = Q K^T, per block two 8-token column blocks ----
+            // All K fragments of a block are fetched first and the products of even and odd 16-column steps go
+            // to separate accumulators, so that neither the shared-memory latency nor the latency of one MMA
+            // feeding the next sits KSTEPS times on the path of a tile.
+            float s[BPW][2][2];
+            float tmax = -INFINITY;
 #pragma unroll
             for (int blk = 0; blk < BPW; ++blk) {
                 const int tok0 = (warp * BPW + blk) * 16;
-                if (tok0 >= valid) continue;   // no row of this block exists (and a partly filled tile was not fetched that far)
-                // ---- S = Q K^T for 16 tokens: two 8-token column blocks ----
-                // All K fragments are fetched first and the products of even and odd 16-column steps go to
-                // separate accumulators, so that neither the shared-memory latency nor the latency of one
-                // MMA feeding the next sits KSTEPS times on the path of a tile (one warp per scheduler: nothing
-                // else hides it).
-                float s[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
-                {
+#pragma unroll
+                for (int nb = 0; nb < 2; ++nb) s[blk][nb][0] = s[blk][nb][1] = 0.f;
+                if (tok0 < valid) {   // else no row of this block exists (and a partly filled tile was not fetched that far)
                     const int t = tok0 + ((lane >> 4) << 3) + (lane & 7);
                     const uint32_t rowaddr = ks_u32 + t * 128;
                     const int sw = t & 7;
@@ -401,80 +411,85 @@ __global__ void __launch_bounds__(kMmaThreads, KVS_MMA_BLOCKS_PER_SM)
                     float s2[2][2] = {{0.f, 0.f}, {0.f, 0.f}};
 #pragma unroll
                     for (int st_k = 0; st_k < KSTEPS; st_k += 2) {
-                        mma_bf16_upper(s[0][0], s[0][1], qa[st_k][0], qa[st_k][1], b[st_k][0], b[st_k][1]);
-                        mma_bf16_upper(s[1][0], s[1][1], qa[st_k][0], qa[st_k][1], b[st_k][2], b[st_k][3]);
+                        mma_bf16_upper(s[blk][0][0], s[blk][0][1], qa[st_k][0], qa[st_k][1], b[st_k][0], b[st_k][1]);
+                        mma_bf16_upper(s[blk][1][0], s[blk][1][1], qa[st_k][0], qa[st_k][1], b[st_k][2], b[st_k][3]);
                         mma_bf16_upper(s2[0][0], s2[0][1], qa[st_k + 1][0], qa[st_k + 1][1], b[st_k + 1][0], b[st_k + 1][1]);
                         mma_bf16_upper(s2[1][0], s2[1][1], qa[st_k + 1][0], qa[st_k + 1][1], b[st_k + 1][2], b[st_k + 1][3]);
                     }
 #pragma unroll
                     for (int nb = 0; nb < 2; ++nb) {
-                        s[nb][0] += s2[nb][0];
-                        s[nb][1] += s2[nb][1];
+                        s[blk][nb][0] += s2[nb][0];
+                        s[blk][nb][1] += s2[nb][1];
                     }
                 }
-                // ---- online softmax for row `row`, tokens tok0 + nb*8 + quad*2 + j ----
-                float tmax = -INFINITY;
+                // scores in the log2 domain; tokens that do not exist count as minus infinity
 #pragma unroll
                 for (int nb = 0; nb < 2; ++nb)
 #pragma unroll
                     for (int j = 0; j < 2; ++j) {
                         const int tok = tok0 + nb * 8 + quad * 2 + j;
-                        s[nb][j] = tok < valid ? s[nb][j] * a.scale_log2 : -INFINITY;
-                        tmax = fmaxf(tmax, s[nb][j]);
+                        s[blk][nb][j] = tok < valid ? s[blk][nb][j] * a.scale_log2 : -INFINITY;
+                        tmax = fmaxf(tmax, s[blk][nb][j]);
                     }
-                tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 1));
-                tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 2));
-                const float m_new = fmaxf(m, tmax);
-                const float alpha = fast_exp2(m - m_new);
-                m = m_new;
-                float p[2][2];
-                float psum = 0.f;
+            }
+            // ---- one online-softmax update for row `row` over the warp's tokens of this tile ----
+            tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 1));
+            tmax = fmaxf(tmax, __shfl_xor_sync(0xffffffffu, tmax, 2));
+            const float m_new = fmaxf(m, tmax);
+            const float alpha = fast_exp2(m - m_new);
+            m = m_new;
+            float p[BPW][2][2];
+            float psum = 0.f;
+#pragma unroll
+            for (int blk = 0; blk < BPW; ++blk)
 #pragma unroll
                 for (int nb = 0; nb < 2; ++nb)
 #pragma unroll
                     for (int j = 0; j < 2; ++j) {
-                        p[nb][j] = fast_exp2(s[nb][j] - m_new);
-                        psum += p[nb][j];
+                        p[blk][nb][j] = fast_exp2(s[blk][nb][j] - m_new);
+                        psum += p[blk][nb][j];
                     }
-                lsum = lsum * alpha + psum;
+            lsum = lsum * alpha + psum;
 #pragma unroll
-                for (int nb = 0; nb < NB; ++nb) {
-                    o[nb][0] *= alpha;
-                    o[nb][1] *= alpha;
-                }
+            for (int nb = 0; nb < NB; ++nb) {
+                o[nb][0] *= alpha;
+                o[nb][1] *= alpha;
+            }
+            // ---- O += P V, per block 16 tokens x D, two 8-wide column blocks per ldmatrix ----
+#pragma unroll
+            for (int blk = 0; blk < BPW; ++blk) {
+                const int tok0 = (warp * BPW + blk) * 16;
+                if (tok0 >= valid) continue;
                 // P = P_hi + P_lo as A fragments (k = tokens): klo = tokens 0..7, khi = tokens 8..15
-                const float h00 = bf16_round(p[0][0]), h01 = bf16_round(p[0][1]);
-                const float h10 = bf16_round(p[1][0]), h11 = bf16_round(p[1][1]);
+                const float h00 = bf16_round(p[blk][0][0]), h01 = bf16_round(p[blk][0][1]);
+                const float h10 = bf16_round(p[blk][1][0]), h11 = bf16_round(p[blk][1][1]);
                 const uint32_t phi_lo = pack_bf16(h00, h01), phi_hi = pack_bf16(h10, h11);
-                const uint32_t plo_lo = pack_bf16(p[0][0] - h00, p[0][1] - h01);
-                const uint32_t plo_hi = pack_bf16(p[1][0] - h10, p[1][1] - h11);
-                // ---- O += P V: 16 tokens x D, two 8-wide column blocks per ldmatrix ----
+                const uint32_t plo_lo = pack_bf16(p[blk][0][0] - h00, p[blk][0][1] - h01);
+                const uint32_t plo_hi = pack_bf16(p[blk][1][0] - h10, p[blk][1][1] - h11);
                 // Four column blocks at a time: their P_hi products are issued before their P_lo products, so
                 // that an MMA never waits for the one just before it (same accumulator).
-                {
-                    const int t = tok0 + (((lane >> 3) & 1) << 3) + (lane & 7);
-                    const uint32_t rowaddr = vs_u32 + t * 128;
-                    const int sw = t & 7;
+                const int t = tok0 + (((lane >> 3) & 1) << 3) + (lane & 7);
+                const uint32_t rowaddr = vs_u32 + t * 128;
+                const int sw = t & 7;
 #pragma unroll
-                    for (int nbp = 0; nbp < NB / 2; nbp += 2) {
-                        uint32_t b[2][4];
+                for (int nbp = 0; nbp < NB / 2; nbp += 2) {
+                    uint32_t b[2][4];
 #pragma unroll
-                        for (int x = 0; x < 2; ++x) {
-                            const int chunkg = (nbp + x) * 2 + (lane >> 4);
-                            const int half = chunkg >> 3;
-                            const int chunk = chunkg & 7;
-                            ldmatrix_x4_trans(b[x], rowaddr + half * (TN * 128) + ((chunk ^ sw) << 4));
-                        }
+                    for (int x = 0; x < 2; ++x) {
+                        const int chunkg = (nbp + x) * 2 + (lane >> 4);
+                        const int half = chunkg >> 3;
+                        const int chunk = chunkg & 7;
+                        ldmatrix_x4_trans(b[x], rowaddr + half * (TN * 128) + ((chunk ^ sw) << 4));
+                    }
 #pragma unroll
-                        for (int x = 0; x < 2; ++x) {
-                            mma_bf16_upper(o[2 * (nbp + x)][0], o[2 * (nbp + x)][1], phi_lo, phi_hi, b[x][0], b[x][1]);
-                            mma_bf16_upper(o[2 * (nbp + x) + 1][0], o[2 * (nbp + x) + 1][1], phi_lo, phi_hi, b[x][2], b[x][3]);
-                        }
+                    for (int x = 0; x < 2; ++x) {
+                        mma_bf16_upper(o[2 * (nbp + x)][0], o[2 * (nbp + x)][1], phi_lo, phi_hi, b[x][0], b[x][1]);
+                        mma_bf16_upper(o[2 * (nbp + x) + 1][0], o[2 * (nbp + x) + 1][1], phi_lo, phi_hi, b[x][2], b[x][3]);
+                    }
 #pragma unroll
-                        for (int x = 0; x < 2; ++x) {
-                            mma_bf16_upper(o[2 * (nbp + x)][0], o[2 * (nbp + x)][1], plo_lo, plo_hi, b[x][0], b[x][1]);
-                            mma_bf16_upper(o[2 * (nbp + x) + 1][0], o[2 * (nbp + x) + 1][1], plo_lo, plo_hi, b[x][2], b[x][3]);
-                        }
+                    for (int x = 0; x < 2; ++x) {
+                        mma_bf16_upper(o[2 * (nbp + x)][0], o[2 * (nbp + x)][1], plo_lo, plo_hi, b[x][0], b[x][1]);
+                        mma_bf16_upper(o[2 * (nbp + x) + 1][0], o[2 * (nbp + x) + 1][1], plo_lo, plo_hi, b[x][2], b[x][3]);
                     }
                 }
             }
