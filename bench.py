@@ -47,8 +47,8 @@ FALLBACK_HBM_GBS = 6650.0
 NCU_TRAFFIC = {
     1: {"files": ("kvs_kernels.cu", "kvs_device.cuh"), "dram_bytes": 1557.51e6, "kv_bytes": 1552.55e6,
         "sha256": "a6b6b4437657743776030cf2ad57be5b9385213ccd1d31712ac119e110e59e81"},
-    2: {"files": ("kvs_mma.cu", "kvs_device.cuh"), "dram_bytes": 542.66e6, "kv_bytes": 536.90e6,
-        "sha256": "55ae88a733ca7fe65393ef47bd2dedb01c1986a11e015b2ab01d080f95577971"},
+    2: {"files": ("kvs_mma.cu", "kvs_device.cuh"), "dram_bytes": 541.22e6, "kv_bytes": 536.90e6,
+        "sha256": "e8e9a2c490fd7d0a26c8ceb3a470e7f81085cdd57c3752f23dd2b1a41da37fca"},
 }
 
 
